@@ -1,0 +1,170 @@
+"""TEST INFRASTRUCTURE (CPU oracle) -- the source programs as sets of function
+graphs (Figure 2 style) and the operator tables the interpreter needs.
+
+Programs:
+  * the factorial example of Section 2.4:  result = fact(3)+5;
+    fact(n) = if (n==1) then n else n*fact(n-1);
+  * fib(n) = if n<2 then n else fib(n-1)+fib(n-2).  The paper names `fib` in
+    Table 1 without printing its definition; this is the textbook reading
+    (fib 0 = 0, fib 1 = 1);
+  * integer tree folds (sum of leaf tokens, leaf count, height) used to pin
+    the tree-walking machinery;
+  * the recursive tree networks: TreeRNN  h(v) = E[tok v] at a leaf,
+    tanh(W [h(l); h(r)] + b) otherwise; the binary TreeLSTM; both optionally
+    returning the pair (state, summed per-node loss).  The paper's Section 6.2
+    names the TreeRNN sentiment model without giving its equations; the cell
+    forms are the ones fixed by the workload list.
+
+Only tests, the smoke check and the CPU-baseline leg of the benchmark may
+import anything under `oracle/`.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from .graphs import FunctionGraph
+
+
+# --------------------------------------------------------------------------
+# integer programs
+# --------------------------------------------------------------------------
+INT_OPS = {
+    "+": lambda a, b: a + b,
+    "-": lambda a, b: a - b,
+    "*": lambda a, b: a * b,
+    "<": lambda a, b: a < b,
+    "==": lambda a, b: a == b,
+    "id": lambda a: a,
+    "max": lambda a, b: a if a > b else b,
+}
+
+
+def fact_program(arg=3, addend=5):
+    """Figure 2: the two graphs `result` and `fact`."""
+    r = FunctionGraph("result", 0)
+    r.output(r.op("+", r.const(addend), r.call("fact", r.const(arg))))
+    f = FunctionGraph("fact", 1)
+    n = f.param(0)
+    t, e = f.switch(f.op("==", f.const(1), n), n)
+    rec = f.call("fact", f.op("-", e, f.const(1)))
+    f.output(f.merge(f.op("id", t), f.op("*", e, rec)))
+    return [r, f]
+
+
+def fib_program():
+    r = FunctionGraph("result", 1)
+    r.output(r.call("fib", r.param(0)))
+    f = FunctionGraph("fib", 1)
+    n = f.param(0)
+    t, e = f.switch(f.op("<", n, f.const(2)), n)
+    a = f.call("fib", f.op("-", e, f.const(1)))
+    b = f.call("fib", f.op("-", e, f.const(2)))
+    f.output(f.merge(f.op("id", t), f.op("+", a, b)))
+    return [r, f]
+
+
+def tree_fold_program(leaf_op: str, combine: str, plus_one: bool = False):
+    """fold(v) = leaf_op(v) at a leaf, combine(fold(left v), fold(right v)) [+1]."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("fold", r.param(0)))
+    f = FunctionGraph("fold", 1)
+    v = f.param(0)
+    t, e = f.switch(f.op("is_leaf", v), v)
+    a = f.call("fold", f.op("left", e))
+    b = f.call("fold", f.op("right", e))
+    c = f.op(combine, a, b)
+    if plus_one:
+        c = f.op("+", c, f.const(1))
+    f.output(f.merge(f.op(leaf_op, t), c))
+    return [r, f]
+
+
+def tree_ops(tb):
+    """Accessors over one flat tree batch (indices are global node numbers)."""
+    ops = dict(INT_OPS)
+    ops.update({
+        "is_leaf": lambda v: bool(tb.left[v] < 0),
+        "left": lambda v: int(tb.left[v]),
+        "right": lambda v: int(tb.right[v]),
+        "tok": lambda v: int(tb.tok[v]),
+        "one": lambda v: 1,
+        "zero": lambda v: 0,
+    })
+    return ops
+
+
+# --------------------------------------------------------------------------
+# recursive tree networks
+# --------------------------------------------------------------------------
+def tree_net_program(cell: str, with_loss: bool):
+    """h(v) = leaf(tok v) if is_leaf(v) else cell(h(left v), h(right v)).
+
+    With `with_loss`, a call returns the pair (state, loss summed over the
+    subtree) and `result` returns that pair for the root.
+    cell is 'rnn' or 'lstm' (the operator names are cell_rnn/leaf_rnn etc.).
+    """
+    r = FunctionGraph("result", 1)
+    r.output(r.call("h", r.param(0)))
+    f = FunctionGraph("h", 1)
+    v = f.param(0)
+    t, e = f.switch(f.op("is_leaf", v), v)
+    if not with_loss:
+        leaf = f.op("leaf_" + cell, f.op("tok", t))
+        a = f.call("h", f.op("left", e))
+        b = f.call("h", f.op("right", e))
+        f.output(f.merge(leaf, f.op("cell_" + cell, a, b)))
+        return [r, f]
+    leaf = f.op("leaf_" + cell, f.op("tok", t))
+    leaf_pair = f.op("pack", leaf, f.op("node_loss", leaf, t))
+    a = f.call("h", f.op("left", e))
+    b = f.call("h", f.op("right", e))
+    x = f.op("cell_" + cell, f.op("fst", a), f.op("fst", b))
+    below = f.op("+", f.op("snd", a), f.op("snd", b))
+    pair = f.op("pack", x, f.op("+", f.op("node_loss", x, e), below))
+    f.output(f.merge(leaf_pair, pair))
+    return [r, f]
+
+
+def sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+def node_loss_value(h, W_s, b_s, label):
+    """-log softmax(W_s h + b_s)[label], written out directly."""
+    z = W_s @ h + b_s
+    p = np.exp(z) / np.exp(z).sum()
+    return float(-np.log(p[label]))
+
+
+def tree_net_ops(tb, params, cell: str):
+    """Operator table for the tree networks; fp64 throughout.  An LSTM state
+    is the pair (h, c); the loss head reads h."""
+    P = {k: np.asarray(v, dtype=np.float64) for k, v in params.items()}
+    ops = tree_ops(tb)
+    ops["pack"] = lambda a, b: (a, b)
+    ops["fst"] = lambda p: p[0]
+    ops["snd"] = lambda p: p[1]
+    if cell == "rnn":
+        ops["leaf_rnn"] = lambda tok: P["E"][tok]
+        ops["cell_rnn"] = lambda hl, hr: np.tanh(P["W"] @ np.concatenate([hl, hr]) + P["b"])
+        ops["node_loss"] = lambda h, v: node_loss_value(h, P["W_s"], P["b_s"], int(tb.label[v]))
+    else:
+        H = P["W"].shape[0] // 5
+
+        def leaf_lstm(tok):
+            g = P["W_x"] @ P["E"][tok] + P["b_x"]
+            i, o, u = g[:H], g[H:2 * H], g[2 * H:]
+            c = sigmoid(i) * np.tanh(u)
+            return (sigmoid(o) * np.tanh(c), c)
+
+        def cell_lstm(l, r):
+            (hl, cl), (hr, cr) = l, r
+            g = P["W"] @ np.concatenate([hl, hr]) + P["b"]
+            i, fl, fr, o, u = (g[k * H:(k + 1) * H] for k in range(5))
+            c = sigmoid(i) * np.tanh(u) + sigmoid(fl) * cl + sigmoid(fr) * cr
+            return (sigmoid(o) * np.tanh(c), c)
+
+        ops["leaf_lstm"] = leaf_lstm
+        ops["cell_lstm"] = cell_lstm
+        ops["node_loss"] = lambda s, v: node_loss_value(s[0], P["W_s"], P["b_s"], int(tb.label[v]))
+    return ops

@@ -1,0 +1,279 @@
+"""Pins for the integer side of the CPU oracle: the Section 3 transformation,
+the Call/Return semantics and the tagged interpreter, against what the paper
+and arithmetic fix (Figure 3, the factorial example, closed forms for fib)."""
+import collections
+import math
+import os
+
+import numpy as np
+import pytest
+
+import workloads
+from oracle import direct, programs, tagged, transform
+from oracle.graphs import FunctionGraph, Graph
+
+
+# --------------------------------------------------------------------------
+# Figure 3
+# --------------------------------------------------------------------------
+def _read_fig3(path):
+    nodes, edges = {}, []
+    for line in open(path):
+        p = line.split()
+        if not p or p[0].startswith("#"):
+            continue
+        if p[0] == "node":
+            nodes[p[1]] = (p[2], p[3])
+        elif p[0] == "edge":
+            edges.append((p[1], int(p[2]), p[3], int(p[4]), False))
+        elif p[0] == "control":
+            edges.append((p[1], 0, p[2], -1, True))
+    return nodes, edges
+
+
+def _sig_fixture(kind, detail):
+    return f"{kind}:{detail}"
+
+
+def _sig_node(n):
+    if n.kind == "op":
+        return f"op:{n.name}"
+    if n.kind in ("Call", "Return", "const"):
+        return f"{n.kind}:{n.value}"
+    if n.kind == "merge":
+        return "merge:entry" if n.name == "entry" else "merge:if"
+    return f"{n.kind}:-"
+
+
+def test_transform_reproduces_figure_3(golden_dir):
+    fn, fe = _read_fig3(os.path.join(golden_dir, "fact_fig3_graph.txt"))
+    g = transform.transform(programs.fact_program())
+    assert collections.Counter(_sig_fixture(*v) for v in fn.values()) == \
+        collections.Counter(_sig_node(n) for n in g.nodes)
+    want = collections.Counter((_sig_fixture(*fn[s]), sp, _sig_fixture(*fn[d]), dp, c) for s, sp, d, dp, c in fe)
+    got = collections.Counter((_sig_node(g.nodes[e.src]), e.src_port if not e.control else 0,
+                               _sig_node(g.nodes[e.dst]), e.dst_port, e.control) for e in g.edges)
+    assert want == got
+    # counts the text states: two Calls, two Returns, one control edge per pair
+    assert g.count("Call") == 2 and g.count("Return") == 2 and g.count("merge") == 2 and g.count("switch") == 1
+    assert g.count("fcall") == 0 and g.count("in") == 0 and g.count("out") == 1
+
+
+def test_transform_general_counts():
+    """n call sites of an m-parameter function give n*m Call nodes, n Return
+    nodes, m entry Merges with n inputs each, n*m control edges (Section 3)."""
+    r = FunctionGraph("result", 2)
+    a = r.call("g", r.param(0), r.param(1))
+    b = r.call("g", r.param(1), r.param(0))
+    r.output(r.op("+", a, b))
+    f = FunctionGraph("g", 2)
+    x, y = f.param(0), f.param(1)
+    t, e = f.switch(f.op("<", x, f.const(1)), x)
+    rec = f.call("g", f.op("-", e, f.const(1)), y)
+    f.output(f.merge(f.op("id", t), f.op("+", rec, f.const(1))))
+    g = transform.transform([r, f])
+    assert g.count("Call") == 3 * 2 and g.count("Return") == 3
+    entry = [n for n in g.nodes if n.kind == "merge" and n.name == "entry"]
+    assert len(entry) == 2 and all(n.n_in == 3 for n in entry)
+    ctrl = [e for e in g.edges if e.control and g.nodes[e.src].kind == "Call"]
+    assert len(ctrl) == 6
+    assert all(g.nodes[e.dst].kind == "Return" and g.nodes[e.dst].value == g.nodes[e.src].value for e in ctrl)
+    labels = sorted(n.value for n in g.nodes if n.kind == "Return")
+    assert labels == [0, 1, 2]
+
+
+# --------------------------------------------------------------------------
+# Call_i / Return_i semantic equations
+# --------------------------------------------------------------------------
+def _single(kind, label):
+    """in -> Call_label -> out, or in -> Return_label -> out, as a bare graph."""
+    g = Graph()
+    i = g.add("in", value=0)
+    n = g.add(kind, value=label, n_in=1)
+    o = g.add("out", n_in=1)
+    g.connect(i, n, 0)
+    g.connect(n, o, 0)
+    return g
+
+
+def test_call_prefixes_label():
+    r = tagged.run(_single("Call", 7), {0: 42}, {})
+    assert r.outputs == {(7,): 42}          # Call_i <t,d> = <i:t,d>
+
+
+def test_call_then_return_is_identity_and_mismatch_is_silent():
+    def chain(call_label, ret_label):
+        g = Graph()
+        i = g.add("in", value=0)
+        c = g.add("Call", value=call_label, n_in=1)
+        c2 = g.add("Call", value=3, n_in=1)
+        r2 = g.add("Return", value=3, n_in=1)
+        r = g.add("Return", value=ret_label, n_in=1)
+        o = g.add("out", n_in=1)
+        g.connect(i, c, 0)
+        g.connect(c, c2, 0)
+        g.connect(c2, r2, 0)
+        g.connect(c2, r2, -1, control=True)
+        g.connect(r2, r, 0)
+        g.connect(c, r, -1, control=True)
+        g.connect(r, o, 0)
+        return g
+    assert tagged.run(chain(5, 5), {0: -9}, {}).outputs == {(): -9}
+    assert tagged.run(chain(5, 4), {0: -9}, {}).outputs == {}     # head 5 != 4: no output
+
+
+def test_switch_merge_and_hiaton_propagation():
+    f = FunctionGraph("result", 2)
+    t, e = f.switch(f.param(0), f.param(1))
+    f.output(f.merge(f.op("+", t, f.const(10)), f.op("*", e, f.const(3))))
+    g = transform.transform([f])
+    for dead in (True, False):
+        assert tagged.run(g, {0: True, 1: 4}, programs.INT_OPS, dead_tokens=dead).value == 14
+        assert tagged.run(g, {0: False, 1: 4}, programs.INT_OPS, dead_tokens=dead).value == 12
+    assert tagged.run(g, {0: True, 1: 4}, programs.INT_OPS, dead_tokens=True).leftover == 0
+
+
+# --------------------------------------------------------------------------
+# the factorial example
+# --------------------------------------------------------------------------
+def test_fact_example_trace(golden_dir):
+    inv, result = {}, None
+    for line in open(os.path.join(golden_dir, "fact_trace.txt")):
+        p = line.split()
+        if p and p[0] == "invocation":
+            inv[tuple(int(x) for x in p[1].split(","))] = (int(p[2]), int(p[3]))
+        elif p and p[0] == "result":
+            result = int(p[1])
+    g = transform.transform(programs.fact_program())
+    for dead in (True, False):
+        r = tagged.run(g, {}, programs.INT_OPS, dead_tokens=dead)
+        assert r.value == result == 11
+        assert {t: (a[0], r.returns[t]) for t, a in r.calls.items()} == inv
+    assert tagged.run(g, {}, programs.INT_OPS, dead_tokens=True).leftover == 0
+
+
+@pytest.mark.parametrize("n", [1, 2, 5, 10, 15])
+def test_fact_against_math_factorial(n):
+    g = transform.transform(programs.fact_program(arg=n, addend=0))
+    r = tagged.run(g, {}, programs.INT_OPS)
+    assert r.value == math.factorial(n) == direct.fact(n)
+    assert len(r.calls) == n and r.max_depth == n
+
+
+# --------------------------------------------------------------------------
+# fib: closed forms
+# --------------------------------------------------------------------------
+def _fib_iter(n):
+    a, b = 0, 1
+    for _ in range(n):
+        a, b = b, a + b
+    return a
+
+
+def test_fib_values_recurrence_and_binet():
+    phi = (1 + 5 ** 0.5) / 2
+    for n in range(0, 26):
+        assert direct.fib(n) == _fib_iter(n) == round(phi ** n / 5 ** 0.5)
+    assert direct.fib(18) == 2584
+
+
+@pytest.fixture(scope="module")
+def fib_graph():
+    return transform.transform(programs.fib_program())
+
+
+def test_fib_graph_structure(fib_graph):
+    g = fib_graph
+    assert g.count("Call") == 3 and g.count("Return") == 3 and g.count("switch") == 1
+    entry = [n for n in g.nodes if n.kind == "merge" and n.name == "entry"]
+    assert len(entry) == 1 and entry[0].n_in == 3
+    plus = [n for n in g.nodes if n.kind == "op" and n.name == "+"][0]
+    srcs = sorted(g.nodes[e.src].value for e in g.in_edges(plus.id))
+    assert srcs == [1, 2] and all(g.nodes[e.src].kind == "Return" for e in g.in_edges(plus.id))
+
+
+@pytest.mark.parametrize("n", list(range(0, 13)) + [18])
+def test_fib_tagged_equals_direct_and_counts(fib_graph, n):
+    r = tagged.run(fib_graph, {0: n}, programs.INT_OPS)
+    assert r.value == _fib_iter(n)
+    assert r.leftover == 0
+    # invocations: calls(n) = 2 F(n+1) - 1, tag depth max(1, n)
+    assert len(r.calls) == 2 * _fib_iter(n + 1) - 1
+    assert r.max_depth == max(1, n)
+    # every invocation returns fib(argument); the trace equals direct recursion with call paths
+    _, inv = direct.fib_invocations(n)
+    assert {t: (a, v) for t, a, v in inv} == {t: (a[0], r.returns[t]) for t, a in r.calls.items()}
+    for t, a in r.calls.items():
+        assert r.returns[t] == _fib_iter(a[0])
+    # tags: distinct by construction (dict keys), prefix closed, rooted at call site 0
+    for t in r.calls:
+        assert t[-1] == 0 and all(x in (1, 2) for x in t[:-1])
+        assert len(t) == 1 or t[1:] in r.calls
+    r2 = tagged.run(fib_graph, {0: n}, programs.INT_OPS, dead_tokens=False)
+    assert r2.value == r.value and r2.calls == r.calls and r2.returns == r.returns
+
+
+def test_fib_wave_widths_by_recurrence(fib_graph):
+    """Invocations at tag depth d for n=18 follow w_n(d) = w_{n-1}(d-1) + w_{n-2}(d-1)."""
+    def w(n, d):
+        if d == 1:
+            return 1
+        if n < 2:
+            return 0
+        return w(n - 1, d - 1) + w(n - 2, d - 1)
+    r = tagged.run(fib_graph, {0: 18}, programs.INT_OPS, dead_tokens=False)
+    got = collections.Counter(len(t) for t in r.calls)
+    assert [got[d] for d in range(1, 19)] == [w(18, d) for d in range(1, 19)]
+    assert max(got.values()) == 2048 and got[13] == 2048
+    assert sum(2 * _fib_iter(n + 1) - 1 for n in range(19)) == 21871
+
+
+def test_fib_batch_totals():
+    x = workloads.config(1)["x"]
+    assert x.shape == (1024,) and x.min() >= 0 and x.max() <= 18
+    total = sum(2 * _fib_iter(int(n) + 1) - 1 for n in x)
+    assert abs(total - 1024 * 21871 / 19) < 0.1 * total      # the seed's N is near its expectation
+
+
+# --------------------------------------------------------------------------
+# integer tree folds pin the tree-walking machinery
+# --------------------------------------------------------------------------
+@pytest.fixture(scope="module")
+def small_trees():
+    return workloads.config(2, B=12)["trees"]
+
+
+def test_tree_sum_count_height(small_trees):
+    tb = small_trees
+    ops = programs.tree_ops(tb)
+    gsum = transform.transform(programs.tree_fold_program("tok", "+"))
+    gcnt = transform.transform(programs.tree_fold_program("one", "+"))
+    ghgt = transform.transform(programs.tree_fold_program("zero", "max", plus_one=True))
+    sizes = tb.tree_sizes()
+    for t in range(tb.B):
+        root = int(tb.tree_root[t])
+        sl = slice(root, root + int(sizes[t]))
+        leaf_tok = tb.tok[sl][tb.left[sl] < 0]
+        r = tagged.run(gsum, {0: root}, ops)
+        assert r.value == int(leaf_tok.sum()) == direct.tree_fold(tb, root, lambda v: int(tb.tok[v]), lambda a, b: a + b)
+        L = (sizes[t] + 1) // 2
+        assert tagged.run(gcnt, {0: root}, ops).value == L
+        assert len(r.calls) == 2 * L - 1                     # N = 2L - 1 invocations
+        h = tagged.run(ghgt, {0: root}, ops).value
+        assert h == direct.tree_fold(tb, root, lambda v: 0, lambda a, b: max(a, b) + 1)
+        assert r.max_depth == h + 1
+        # tag <-> tree node bijection: the tag is the reversed root-to-node path
+        inv = direct.deep(direct.tree_invocations, tb, root)
+        assert {tg: v for tg, v in inv} == {tg: a[0] for tg, a in r.calls.items()}
+
+
+def test_chain_and_perfect_shapes():
+    l, r = workloads.chain_tree_shape(40)
+    tb = workloads.tree_batch_from_shapes([(l, r), workloads.perfect_tree_shape(5)], seed=1, vocab=10)
+    height = lambda root: direct.deep(direct.tree_fold, tb, root, lambda v: 0, lambda a, b: max(a, b) + 1)  # noqa: E731
+    assert height(int(tb.tree_root[0])) == 40 and height(int(tb.tree_root[1])) == 5
+    assert tb.tree_sizes().tolist() == [81, 63]
+    assert np.all(tb.right[tb.left >= 0] >= 0)
+    # every right child of the chain is a leaf
+    chain_int = [v for v in range(81) if tb.left[v] >= 0]
+    assert all(tb.left[tb.right[v]] < 0 for v in chain_int)
