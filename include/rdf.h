@@ -1,0 +1,252 @@
+/* rdf.h -- recursive dataflow on one GPU: C boundary of the library.
+ *
+ * The library executes recursive function definitions as ONE static dataflow
+ * graph extended with two tag operations (paper, Section 3):
+ *
+ *     Call_i   <t, d>   = <i:t, d>      tag-push on a recursive invocation
+ *     Return_i <i:t, d> = <t, d>        tag-pop on return
+ *
+ * Tokens <tag, datum> of many concurrent invocations flow through the fixed
+ * graph; an operator fires when all its inputs hold tokens with exactly the
+ * same tag (Section 2.2), and all operators that are ready at the same time
+ * fire as one batch on the device.
+ *
+ * Conventions for every function below
+ *   - returns an int status: RDF_OK (0) or a negative RDF_ERR_* code; nothing
+ *     throws, aborts or traps.  Conditions found on the device (capacity, tag
+ *     overflow, an expired bounded wait) are written to a status word, all
+ *     thread blocks leave, and the code is reported by rdf_last_status().
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA
+ *     global memory of the current device, at least 16-byte aligned, owned by
+ *     the caller and valid until the stream has passed the call.
+ *   - rdf_eval / rdf_grad are stream-ordered: they enqueue work on `stream`
+ *     (a cudaStream_t passed as void*) and return without synchronising.
+ *     They allocate no device memory; all scratch comes from `workspace`.
+ */
+#ifndef RDF_H
+#define RDF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ------------------------------------------------------------------ status */
+enum {
+    RDF_OK = 0,
+    RDF_ERR_BAD_PROGRAM = -1,        /* unknown callee, arity mismatch, no `result`, malformed expression */
+    RDF_ERR_BAD_ARG = -2,            /* NULL or inconsistent argument */
+    RDF_ERR_WORKSPACE_TOO_SMALL = -3,
+    RDF_ERR_TAG_OVERFLOW = -4,       /* call depth x label bits exceeds the packed path field */
+    RDF_ERR_STORE_FULL = -5,         /* token store has no free slot */
+    RDF_ERR_FRAMES_FULL = -6,        /* more invocations than rdf_batch.max_invocations */
+    RDF_ERR_QUEUE_FULL = -7,         /* more tokens in one wave than the queues hold */
+    RDF_ERR_WAVE_LIMIT = -8,         /* guard against recursion that never reaches a base case */
+    RDF_ERR_TIMEOUT = -9,            /* a bounded device-side wait expired */
+    RDF_ERR_CUDA = -10,              /* a CUDA runtime call failed */
+    RDF_ERR_UNSUPPORTED = -11        /* valid program outside what the device executor lowers */
+};
+
+/* ----------------------------------------------------------------- program
+ * A program is a set of function definitions, one of which is `result`
+ * (Section 3, "Assume we are given a set S of dataflow graphs ...").  Each
+ * definition is an expression DAG over its formal parameters.  A CALL node is
+ * a node "labeled with the name of f" (Section 2.4, Figure 2); IF is the
+ * Switch/Merge conditional of Figure 2.
+ */
+typedef enum {
+    RDF_OP_PARAM = 0,    /* imm = parameter index                                   */
+    RDF_OP_CONST,        /* imm = value                                             */
+    RDF_OP_ADD, RDF_OP_SUB, RDF_OP_MUL, RDF_OP_MAX,   /* a, b                       */
+    RDF_OP_LT, RDF_OP_EQ,                             /* a, b -> 0/1                */
+    RDF_OP_IF,           /* a = condition, b = then, c = else                       */
+    RDF_OP_CALL,         /* imm = callee function index, a = argument expression    */
+    /* accessors on the batch's flat tree arrays; operand = node index           */
+    RDF_OP_IS_LEAF, RDF_OP_LEFT, RDF_OP_RIGHT, RDF_OP_TOK,
+    /* vector-valued operators of the tree networks                               */
+    RDF_OP_EMBED,        /* a = token id          -> E[tok]                         */
+    RDF_OP_CELL_RNN,     /* a, b = child states   -> tanh(W [a; b] + b)             */
+    RDF_OP_LEAF_LSTM,    /* a = token id          -> (h, c) of a TreeLSTM leaf      */
+    RDF_OP_CELL_LSTM,    /* a, b = child states   -> (h, c) of a binary TreeLSTM    */
+    RDF_OP_NODE_LOSS,    /* a = state, b = node index; passes the state through and
+                            marks the invocation as a term of the summed per-node
+                            softmax cross-entropy loss that rdf_grad differentiates */
+    RDF_OP__COUNT
+} rdf_opcode;
+
+typedef struct {
+    int32_t op;          /* rdf_opcode */
+    int32_t a, b, c;     /* operand expression indices within the same function, -1 if unused */
+    int64_t imm;
+} rdf_expr;
+
+typedef struct {
+    const char*     name;        /* host, NUL-terminated, copied by rdf_graph_build */
+    int32_t         n_params;    /* m >= 0 formal parameters */
+    int32_t         n_exprs;
+    const rdf_expr* exprs;       /* host, [n_exprs]; a DAG (no cycles) */
+    int32_t         root;        /* index of the expression that is the function's output */
+} rdf_function;
+
+typedef enum { RDF_TAGS_PATH = 0, RDF_TAGS_FRAME = 1 } rdf_tag_mode;
+
+typedef struct {
+    int32_t             n_functions;
+    const rdf_function* functions;   /* host, [n_functions] */
+    int32_t             result;      /* index of the definition of `result` */
+    /* Tag representation on the device.
+     * RDF_TAGS_PATH : the label list itself, packed in 64 bits
+     *                 [63:44] instance | [43:38] depth | [37:0] labels, `label_bits` each, innermost lowest.
+     *                 Matching uses an open-addressing hash table keyed by the packed tag.
+     * RDF_TAGS_FRAME: an interned frame id; a frame record holds the parent frame and the label
+     *                 (the paper's own representation, Section 5.1).  Needed for deep recursion
+     *                 and for vector-valued programs. */
+    int32_t             tag_mode;
+} rdf_program;
+
+typedef struct rdf_graph rdf_graph;      /* opaque, owned by the library */
+
+/* Section 3 transformation + lowering for the device.  All inputs are host
+ * memory and are not retained.  On success *out_graph must be released with
+ * rdf_graph_free.  Errors: BAD_PROGRAM, BAD_ARG, UNSUPPORTED. */
+int  rdf_graph_build(const rdf_program* prog, rdf_graph** out_graph);
+void rdf_graph_free(rdf_graph* g);
+
+/* The literal static graph after the transformation of Section 3, for
+ * inspection: Call_i / Return_i nodes, entry Merge nodes, Switch/Merge of the
+ * conditionals, control edges Call_i -> Return_i (and entry Merge -> constant,
+ * Figure 3).  Arrays are host memory owned by the graph. */
+typedef enum {
+    RDF_NODE_IN = 0, RDF_NODE_OUT, RDF_NODE_CONST, RDF_NODE_OP, RDF_NODE_SWITCH,
+    RDF_NODE_MERGE, RDF_NODE_ENTRY_MERGE, RDF_NODE_CALL, RDF_NODE_RETURN
+} rdf_node_kind;
+
+typedef struct {
+    int32_t kind;        /* rdf_node_kind */
+    int32_t op;          /* rdf_opcode for RDF_NODE_OP, else -1 */
+    int32_t label;       /* i of Call_i / Return_i (numbered per callee from 0), else -1 */
+    int32_t func;        /* function the node belongs to (Call/Return: the caller) */
+    int32_t param;       /* parameter index for IN / ENTRY_MERGE / CALL */
+    int32_t n_in;        /* number of data inputs */
+    int64_t value;       /* constant value */
+} rdf_node;
+
+typedef struct {
+    int32_t src, src_port;   /* Switch: output 0 = true side, 1 = false side */
+    int32_t dst, dst_port;   /* dst_port = -1 for a control edge */
+    int32_t control;
+} rdf_edge;
+
+typedef struct {
+    int32_t         n_nodes, n_edges;
+    const rdf_node* nodes;
+    const rdf_edge* edges;
+    int32_t         n_labels;    /* call sites in the whole program (device label ids are global: 0..n_labels-1) */
+    int32_t         label_bits;  /* bits per label in the packed path tag */
+    int32_t         n_match;     /* operators with more than one tagged input (token-store users) */
+    int32_t         n_code;      /* instructions in the lowered device program */
+} rdf_graph_desc;
+
+int rdf_graph_describe(const rdf_graph* g, rdf_graph_desc* out);
+
+/* ------------------------------------------------------------------- batch */
+typedef struct {
+    int64_t        B;            /* independent instances; each starts with the empty tag */
+    const int64_t* x;            /* device [B]: argument of `result` for integer programs, NULL for tree programs */
+    const int32_t* tree_root;    /* device [B]: root node of each tree (tree programs; the argument of `result`) */
+    int64_t        N;            /* tree nodes in the flat arrays below (0 for integer programs) */
+    const int32_t* left;         /* device [N], -1 at a leaf */
+    const int32_t* right;        /* device [N], -1 at a leaf */
+    const int32_t* tok;          /* device [N], token id at leaves */
+    const int32_t* label;        /* device [N], class of every node (rdf_grad / NODE_LOSS), may be NULL for rdf_eval */
+    int64_t        max_invocations; /* capacity: upper bound on Call firings over the batch (tree programs: N) */
+    int64_t        max_wave_tokens; /* capacity of one wave's token queue; 0 = max_invocations + B */
+} rdf_batch;
+
+/* Parameters of the tree networks: fp32, row-major, device.  `compute` picks
+ * the arithmetic of the cell contraction: RDF_F32 = fp32 FMA; RDF_BF16 = bf16
+ * operands (states and weights rounded to bf16) with fp32 accumulation. */
+typedef enum { RDF_F32 = 0, RDF_BF16 = 1 } rdf_compute;
+
+typedef struct {
+    int32_t      compute;        /* rdf_compute */
+    int32_t      H, D, V, n_classes;
+    const float* E;              /* [V, D]                                          */
+    const float* W;              /* TreeRNN [H, 2H]; TreeLSTM [5H, 2H] (i, f_l, f_r, o, u) */
+    const float* b;              /* [H] or [5H]                                     */
+    const float* W_x;            /* TreeLSTM leaf projection [3H, D] (i, o, u) or NULL */
+    const float* b_x;            /* [3H] or NULL                                    */
+    const float* W_s;            /* loss head [n_classes, H] or NULL                */
+    const float* b_s;            /* [n_classes] or NULL                             */
+} rdf_params;
+
+/* One record per Call firing and one per Return firing, in no particular
+ * order (optional; for parity checks of tags). */
+typedef struct {
+    uint64_t tag;        /* PATH: packed tag of the invocation; FRAME: its frame id */
+    int64_t  value;      /* kind 0: the argument; kind 1: the returned integer (vector programs: frame id of the state) */
+    uint32_t kind;       /* 0 = Call fired (tag after the push), 1 = Return fired (tag before the pop) */
+    uint32_t label;      /* i of Call_i / Return_i (global label id) */
+    uint32_t parent;     /* FRAME: frame id of the caller's context; PATH: 0 */
+    uint32_t instance;   /* FRAME: unused (0); PATH: bits [63:44] of the tag */
+} rdf_trace_rec;
+
+typedef struct {
+    int64_t*       y;            /* device [B]: integer results, or NULL */
+    float*         h_root;       /* device [B, H]: root states, or NULL */
+    float*         loss;         /* device [1]: summed loss (rdf_grad), or NULL */
+    rdf_trace_rec* trace;        /* device [trace_capacity] or NULL */
+    int64_t        trace_capacity;
+    uint64_t*      trace_count;  /* device [1]: records written (may exceed capacity: the excess was dropped) */
+} rdf_outputs;
+
+typedef struct {                 /* all device, fp32, shapes of the parameters; overwritten, not accumulated */
+    float *dE, *dW, *db, *dW_x, *db_x, *dW_s, *db_s;
+} rdf_param_grads;
+
+typedef struct {
+    int32_t  status;             /* RDF_OK or the first RDF_ERR_* the device recorded */
+    uint32_t waves;              /* scheduler waves run (forward) */
+    uint32_t waves_backward;
+    uint32_t max_wave_tokens;    /* widest wave */
+    uint64_t invocations;        /* Call firings */
+    uint64_t tokens;             /* tokens taken from the wave queues */
+    uint64_t store_inserts;      /* operands parked in the token store */
+    uint64_t store_matches;      /* firings completed by a match */
+    uint64_t store_probes;       /* hash slots inspected (PATH mode) */
+    uint32_t max_probe;          /* longest probe sequence */
+    uint32_t max_depth;          /* deepest tag (PATH mode) */
+    uint64_t cells;              /* batched cell firings */
+    uint64_t leaves;             /* batched leaf firings */
+} rdf_stats;
+
+/* Bytes of device scratch rdf_eval (want_grad = 0) or rdf_grad (1) needs for
+ * this graph and batch shape (only the sizes in `in` and `params` are read). */
+int rdf_workspace_bytes(const rdf_graph* g, const rdf_batch* in, const rdf_params* params,
+                        int want_grad, size_t* bytes);
+
+/* Forward evaluation of `result` on every instance of the batch (Section 5.1:
+ * run the static graph until no token is left).  Outputs: y or h_root. */
+int rdf_eval(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
+             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Forward + reverse mode (Section 4): forward values are retained per
+ * invocation; the gradient pass re-enters every invocation under the tag its
+ * forward Call_i created and accumulates parameter gradients over all
+ * invocations.  Loss = sum over all invocations marked by NODE_LOSS of the
+ * softmax cross-entropy of W_s h + b_s against label[node]. */
+int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
+             rdf_param_grads* grads, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises the stream of the last rdf_eval/rdf_grad on this graph and
+ * copies the device status word and counters out (host struct). */
+int rdf_last_status(rdf_graph* g, rdf_stats* s);
+
+const char* rdf_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RDF_H */

@@ -1,0 +1,347 @@
+// Device-side data structures and primitives of the executor: tokens, packed
+// tags, frames, the token store (hash and dense forms), wave queues, the grid
+// barrier.  Everything lives in the caller's workspace.
+//
+// Memory rule of the persistent kernels: data that one SM writes and another
+// reads in a later phase is read through L2 (__ldcg / __ldcv), never through
+// the non-coherent L1.
+#pragma once
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rdf_internal.h"
+
+namespace cg = cooperative_groups;
+
+// A token <tag, datum> on its way to the segment that starts at `pc`.
+struct __align__(16) Token {
+    uint64_t tag;
+    int64_t  datum;
+    uint32_t pc;
+    uint32_t aux;
+    uint64_t pad;
+};
+static_assert(sizeof(Token) == 32, "two 128-bit words");
+
+// Frame record (frame-form tags): the paper's frame with its label field and
+// the reference to the previous scope (Section 5.1).
+struct __align__(16) Frame {
+    uint32_t parent;
+    uint32_t label;
+    int64_t  arg;
+};
+
+// Hash-store slot: a parked operand keyed by the packed tag.
+struct __align__(16) Slot {
+    uint64_t key;
+    int64_t  val;
+};
+static const uint64_t SLOT_EMPTY = ~0ull;     // depth field 63: never a tag
+
+struct __align__(16) CellItem {               // one ready cell: state of `out` from states of l, r
+    uint32_t out, l, r, pad;
+};
+struct __align__(8) LeafItem {
+    uint32_t slot;
+    int32_t  tok;
+};
+
+// Counters and control words, one 4 KB block at the start of the workspace.
+struct Control {
+    int32_t  status;
+    uint32_t bar;                 // grid barrier arrivals (monotone)
+    uint32_t qcount[3];           // tokens in the queue of wave w at [w % 3]
+    uint32_t cell_count[2];       // ready cells of wave w at [w % 2]
+    uint32_t leaf_count[2];
+    uint32_t frame_count;
+    uint32_t waves, waves_backward, max_wave_tokens, max_probe, max_depth;
+    uint32_t all_cells;           // backward: cells seen so far (length of the all-cells list)
+    uint32_t all_leaves;          // backward: leaves seen so far
+    uint32_t bq_count[3];         // backward wave queues
+    uint32_t bar2;                // barrier counter of the backward kernel
+    unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
+    unsigned long long trace_count;
+    float    loss;
+};
+
+struct DevCtx {
+    // lowered program (copied into the workspace at every call)
+    const VmInstr*   code;
+    const MatchNode* match;
+    const LabelInfo* labels;
+    const int64_t*   consts;
+    int n_code, n_match, n_labels, n_consts;
+    int label_bits, tag_mode, result_entry_pc, n_ports_total, K;   // K = call sites per body (children per frame)
+    // batch
+    long long B, N;
+    const int64_t* x;
+    const int32_t *tree_root, *left, *right, *tok, *label;
+    // wave queues
+    Token*   q[2];
+    uint32_t qcap;
+    // frames (frame-form tags)
+    Frame*    frames;
+    uint32_t* children;           // [frame_cap * K]: frame created by call site k of this frame's body
+    uint32_t  frame_cap;
+    // token store, dense form: one cell per (frame, port) and an arrival counter per (frame, match node)
+    int64_t*  port_val;
+    uint32_t* arrived;
+    // token store, hash form: one open-addressing table per match node
+    Slot*     table;
+    uint64_t  table_cap;          // slots per match node, power of two
+    // batched operators
+    CellItem* cell_items;
+    LeafItem* leaf_items;
+    uint32_t  work_cap;
+    uint32_t* op_l;               // per frame: operand frames of the operator that made its state
+    uint32_t* op_r;               //            (leaf: op_l = LEAF_MARK, op_r = token id)
+    float*    arena;              // [frame_cap, H] fp32 states
+    // parameters
+    int H, D, V, n_classes, compute;
+    const float *E, *W, *b, *W_x, *b_x, *W_s, *b_s;
+    // outputs
+    int64_t* y;                   // integer results / for vector programs the frame holding the root state
+    rdf_trace_rec* trace;
+    long long trace_cap;
+    // gradient pass
+    float*    dhp;                // [frame_cap, H]: gradient arriving from the parent, then dz (cell) / dh (leaf)
+    float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
+    uint32_t* bq[2];              // backward wave queues (frame ids)
+    uint32_t* all_cells;          // every cell frame, in backward wave order
+    uint32_t* all_leaves;         // every leaf frame
+    float*    loss_partial;       // per-block partial sums of the loss
+    float    *dE, *dW, *db, *dW_x, *db_x, *dW_s, *db_s;
+    float*    loss_out;
+    // control
+    Control*  ctl;
+    uint32_t  wave_limit;
+    long long spin_limit;         // clock64 ticks a barrier wait may last
+};
+
+static const uint32_t LEAF_MARK = 0xFFFFFFFFu;
+
+// ---------------------------------------------------------------- utilities
+__device__ __forceinline__ void set_status(const DevCtx& c, int code) { atomicCAS(&c.ctl->status, 0, code); }
+
+__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) {
+    return *reinterpret_cast<const volatile uint32_t*>(p);
+}
+__device__ __forceinline__ int32_t ld_volatile_i32(const int32_t* p) {
+    return *reinterpret_cast<const volatile int32_t*>(p);
+}
+
+// One atomic per converged group of threads instead of one per thread.
+__device__ __forceinline__ uint32_t aggregated_inc(uint32_t* counter) {
+    cg::coalesced_group g = cg::coalesced_threads();
+    uint32_t base = 0;
+    if (g.thread_rank() == 0) base = atomicAdd(counter, g.size());
+    return g.shfl(base, 0) + g.thread_rank();
+}
+
+// Grid-wide barrier with a bounded wait.  All blocks of the (cooperatively
+// launched, hence co-resident) grid call it the same number of times.  The
+// counter only grows; generation k is complete when it reaches k * gridDim.x.
+// Returns false when the wait expired or any block reported an error; the
+// caller then leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter, uint32_t& generation) {
+    __shared__ int ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ++generation;
+        const uint32_t target = generation * gridDim.x;
+        __threadfence();
+        atomicAdd(counter, 1u);
+        const long long t0 = clock64();
+        int good = 1;
+        while (ld_volatile_u32(counter) < target) {
+            if (clock64() - t0 > c.spin_limit) {
+                set_status(c, RDF_ERR_TIMEOUT);
+                good = 0;
+                break;
+            }
+            __nanosleep(32);
+        }
+        __threadfence();
+        if (ld_volatile_i32(&c.ctl->status) != 0) good = 0;
+        ok = good;
+    }
+    __syncthreads();
+    return ok != 0;
+}
+
+// ------------------------------------------------------------------- queues
+__device__ __forceinline__ void store_token(Token* dst_tok, uint64_t tag, int64_t datum, uint32_t pc) {
+    uint4* dst = reinterpret_cast<uint4*>(dst_tok);
+    dst[0] = make_uint4((uint32_t)tag, (uint32_t)(tag >> 32), (uint32_t)datum, (uint32_t)((uint64_t)datum >> 32));
+    dst[1] = make_uint4(pc, 0u, 0u, 0u);
+}
+
+__device__ __forceinline__ void push_token(const DevCtx& c, uint32_t wave, uint64_t tag, int64_t datum, uint32_t pc) {
+    const uint32_t idx = aggregated_inc(&c.ctl->qcount[(wave + 1) % 3]);
+    if (idx >= c.qcap) {
+        set_status(c, RDF_ERR_QUEUE_FULL);
+        return;
+    }
+    store_token(&c.q[(wave + 1) & 1][idx], tag, datum, pc);
+}
+
+// two coalesced 128-bit loads per token, through L2
+__device__ __forceinline__ Token load_token(const Token* p) {
+    const uint4* src = reinterpret_cast<const uint4*>(p);
+    const uint4 a = __ldcg(src), b = __ldcg(src + 1);
+    Token t;
+    t.tag = (uint64_t)a.x | ((uint64_t)a.y << 32);
+    t.datum = (int64_t)((uint64_t)a.z | ((uint64_t)a.w << 32));
+    t.pc = b.x;
+    t.aux = 0;
+    t.pad = 0;
+    return t;
+}
+
+// --------------------------------------------------------------------- tags
+// Packed path form: [63:44] instance | [43:38] depth | [37:0] labels, innermost lowest.
+__device__ __forceinline__ uint64_t path_root(long long instance) { return (uint64_t)instance << RDF_INST_SHIFT; }
+
+__device__ __forceinline__ void trace_rec(const DevCtx& c, uint64_t tag, int64_t value, uint32_t kind, uint32_t label,
+                                          uint32_t parent) {
+    if (!c.trace) return;
+    const unsigned long long i = atomicAdd(&c.ctl->trace_count, 1ull);
+    if ((long long)i < c.trace_cap) {
+        rdf_trace_rec r;
+        r.tag = tag; r.value = value; r.kind = kind; r.label = label;
+        r.parent = c.tag_mode == RDF_TAGS_PATH ? 0u : parent;
+        r.instance = c.tag_mode == RDF_TAGS_PATH ? (uint32_t)(tag >> RDF_INST_SHIFT) : 0u;
+        c.trace[i] = r;
+    }
+}
+
+// Call_i: <t, d> -> <i:t, d>.  Returns false (status set) when the tag cannot be formed.
+__device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label,
+                                         int64_t arg, uint64_t& out) {
+    if (c.tag_mode == RDF_TAGS_PATH) {
+        const uint32_t depth = (uint32_t)(tag >> RDF_DEPTH_SHIFT) & 63u;
+        if ((depth + 1) * (uint32_t)c.label_bits > (uint32_t)RDF_PATH_BITS) {
+            set_status(c, RDF_ERR_TAG_OVERFLOW);
+            return false;
+        }
+        const uint64_t path = tag & ((1ull << RDF_PATH_BITS) - 1);
+        out = (tag & ~((1ull << RDF_INST_SHIFT) - 1)) | ((uint64_t)(depth + 1) << RDF_DEPTH_SHIFT) |
+              ((path << c.label_bits) | label);
+        trace_rec(c, out, arg, 0, label, 0);
+        return true;
+    }
+    const uint32_t id = aggregated_inc(&c.ctl->frame_count);
+    if (id >= c.frame_cap) {
+        set_status(c, RDF_ERR_FRAMES_FULL);
+        return false;
+    }
+    Frame f;
+    f.parent = (uint32_t)tag; f.label = label; f.arg = arg;
+    c.frames[id] = f;
+    c.children[(size_t)tag * c.K + labels[label].child_index] = id;
+    out = id;
+    trace_rec(c, out, arg, 0, label, (uint32_t)tag);
+    return true;
+}
+
+// Return_i: <i:t, d> -> <t, d>; yields the label i that the frame/tag carries.
+__device__ __forceinline__ void tag_pop(const DevCtx& c, uint64_t tag, uint32_t& label, uint64_t& parent) {
+    if (c.tag_mode == RDF_TAGS_PATH) {
+        const uint32_t depth = (uint32_t)(tag >> RDF_DEPTH_SHIFT) & 63u;
+        const uint64_t path = tag & ((1ull << RDF_PATH_BITS) - 1);
+        label = (uint32_t)(path & ((1ull << c.label_bits) - 1));
+        parent = (tag & ~((1ull << RDF_INST_SHIFT) - 1)) | ((uint64_t)(depth - 1) << RDF_DEPTH_SHIFT) |
+                 (path >> c.label_bits);
+    } else {
+        const uint4 f = __ldcg(reinterpret_cast<const uint4*>(&c.frames[tag]));   // {parent, label, arg}
+        label = f.y;
+        parent = f.x;
+    }
+}
+
+// -------------------------------------------------------------- token store
+__device__ __forceinline__ void cas128(Slot* addr, uint64_t cmp_lo, uint64_t cmp_hi, uint64_t new_lo,
+                                       uint64_t new_hi, uint64_t& old_lo, uint64_t& old_hi) {
+    asm volatile(
+        "{\n"
+        " .reg .b128 c, n, o;\n"
+        " mov.b128 c, {%2, %3};\n"
+        " mov.b128 n, {%4, %5};\n"
+        " atom.global.cas.b128 o, [%6], c, n;\n"
+        " mov.b128 {%0, %1}, o;\n"
+        "}\n"
+        : "=l"(old_lo), "=l"(old_hi)
+        : "l"(cmp_lo), "l"(cmp_hi), "l"(new_lo), "l"(new_hi), "l"(addr)
+        : "memory");
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t k) {
+    k ^= k >> 33; k *= 0xff51afd7ed558ccdull;
+    k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ull;
+    k ^= k >> 33;
+    return k;
+}
+
+struct StoreCounters {
+    uint32_t inserts = 0, matches = 0, probes = 0, max_probe = 0;
+};
+
+// Hash form, two-input operators: the first operand to arrive is parked under
+// its tag, the second finds it and takes it (insert-or-consume).  A key is
+// looked up exactly twice in the whole run, so a consumed entry is simply left
+// in place; capacity is sized for all insertions of the run.
+// Returns 1 and the partner's value when the match completed, 0 when parked,
+// -1 when the table is full.
+__device__ __forceinline__ int hash_insert_or_consume(const DevCtx& c, int node, uint64_t key, int64_t val,
+                                                      int64_t& partner, StoreCounters& sc) {
+    Slot* tab = c.table + (size_t)node * c.table_cap;
+    const uint64_t mask = c.table_cap - 1;
+    uint64_t h = mix64(key) & mask;
+    for (uint64_t probe = 0; probe < c.table_cap; ++probe) {
+        ++sc.probes;
+        const uint4 raw = __ldcv(reinterpret_cast<const uint4*>(&tab[h]));
+        uint64_t k = (uint64_t)raw.x | ((uint64_t)raw.y << 32);
+        if (k == SLOT_EMPTY) {
+            uint64_t old_lo, old_hi;
+            cas128(&tab[h], SLOT_EMPTY, ~0ull, key, (uint64_t)val, old_lo, old_hi);
+            if (old_lo == SLOT_EMPTY) {
+                ++sc.inserts;
+                if ((uint32_t)probe > sc.max_probe) sc.max_probe = (uint32_t)probe;
+                return 0;
+            }
+            if (old_lo == key) {             // the partner took this slot meanwhile
+                partner = (int64_t)old_hi;   // (the CAS returned key and value as one unit)
+                ++sc.matches;
+                return 1;
+            }
+        } else if (k == key) {
+            // read key and value as one 128-bit unit: a failing CAS returns the slot's contents
+            uint64_t old_lo, old_hi;
+            cas128(&tab[h], SLOT_EMPTY, ~0ull, SLOT_EMPTY, ~0ull, old_lo, old_hi);
+            partner = (int64_t)old_hi;
+            ++sc.matches;
+            return 1;
+        }
+        h = (h + 1) & mask;
+    }
+    return -1;
+}
+
+// Dense form (frame tags): the operand goes to its (frame, port) cell; the
+// arrival that completes the set reads the others.  Returns 1 when complete.
+__device__ __forceinline__ int dense_deliver(const DevCtx& c, const MatchNode& M, int node, uint64_t frame, int port,
+                                             int64_t val, int64_t* regs, StoreCounters& sc) {
+    int64_t* cells = c.port_val + (size_t)frame * c.n_ports_total + M.port_base;
+    cells[port] = val;
+    __threadfence();
+    const uint32_t before = atomicAdd(&c.arrived[(size_t)frame * c.n_match + node], 1u);
+    if (before + 1 < (uint32_t)M.n_ports) {
+        ++sc.inserts;
+        return 0;
+    }
+    __threadfence();
+    for (int p = 0; p < M.n_ports; ++p) regs[p] = __ldcv(reinterpret_cast<const long long*>(&cells[p]));
+    ++sc.matches;
+    return 1;
+}

@@ -1,0 +1,564 @@
+// Device executor, forward: a persistent, cooperatively launched kernel runs
+// all waves of the tagged dataflow graph without returning to the host.  Each
+// wave
+//   S) takes the wave's tokens, runs their segments (tag push / pop, Switch,
+//      token-store insert or match), emits the next wave's tokens and the lists
+//      of ready batched operators;
+//   C) fires every ready leaf / cell operator of the wave as one batch.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+#include "rdf_exec.h"
+
+// ===========================================================================
+// S phase: the segment interpreter
+// ===========================================================================
+struct SharedProgram {
+    VmInstr   code[RDF_MAX_CODE];
+    MatchNode match[RDF_MAX_MATCH];
+    LabelInfo labels[RDF_MAX_LABELS];
+    int64_t   consts[RDF_MAX_CONSTS];
+};
+
+struct ThreadStats {
+    uint32_t invocations = 0, tokens = 0, cells = 0, leaves = 0, max_depth = 0;
+    StoreCounters sc;
+};
+
+__device__ __forceinline__ void load_program(const DevCtx& c, SharedProgram& sp) {
+    for (int i = threadIdx.x; i < c.n_code; i += blockDim.x) sp.code[i] = c.code[i];
+    for (int i = threadIdx.x; i < c.n_match; i += blockDim.x) sp.match[i] = c.match[i];
+    for (int i = threadIdx.x; i < c.n_labels; i += blockDim.x) sp.labels[i] = c.labels[i];
+    for (int i = threadIdx.x; i < c.n_consts; i += blockDim.x) sp.consts[i] = c.consts[i];
+    __syncthreads();
+}
+
+// A completed match of a batched (cell) operator: queue the cell and the token
+// that carries its state onwards in the next wave.
+__device__ __forceinline__ void fire_cell(const DevCtx& c, const MatchNode& M, uint32_t wave, uint64_t tag,
+                                          const int64_t* regs, ThreadStats& st) {
+    const uint32_t i = aggregated_inc(&c.ctl->cell_count[wave & 1]);
+    if (i >= c.work_cap) {
+        set_status(c, RDF_ERR_QUEUE_FULL);
+        return;
+    }
+    CellItem it;
+    it.out = (uint32_t)tag; it.l = (uint32_t)regs[0]; it.r = (uint32_t)regs[1]; it.pad = 0;
+    c.cell_items[i] = it;
+    c.op_l[tag] = it.l;
+    c.op_r[tag] = it.r;
+    ++st.cells;
+    push_token(c, wave, tag, (int64_t)tag, (uint32_t)M.cont_pc);
+}
+
+// Runs one token through its segment and on through every continuation it
+// completes (a returning value that finds its partner in the store carries on
+// in the caller's context in the same thread).
+__device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wave, Token t, ThreadStats& st) {
+    int64_t r[RDF_MAX_REGS];
+    uint64_t tag = t.tag;
+    int pc = (int)t.pc;
+    r[0] = t.datum;
+    ++st.tokens;
+    // One instruction per iteration; the bound only guards against a corrupted program.
+    for (uint32_t step = 0; step < (1u << 22); ++step) {
+        const VmInstr in = sp.code[pc++];
+        switch (in.op) {
+            case VM_MOVI: r[in.dst] = in.imm; break;
+            case VM_MOVC: r[in.dst] = sp.consts[in.imm]; break;
+            case VM_MOV: r[in.dst] = r[in.a]; break;
+            case VM_ADD: r[in.dst] = r[in.a] + r[in.b]; break;
+            case VM_SUB: r[in.dst] = r[in.a] - r[in.b]; break;
+            case VM_MUL: r[in.dst] = r[in.a] * r[in.b]; break;
+            case VM_MAX: r[in.dst] = r[in.a] > r[in.b] ? r[in.a] : r[in.b]; break;
+            case VM_LT: r[in.dst] = r[in.a] < r[in.b]; break;
+            case VM_EQ: r[in.dst] = r[in.a] == r[in.b]; break;
+            case VM_ISLEAF: r[in.dst] = __ldg(&c.left[r[in.a]]) < 0; break;
+            case VM_LEFT: r[in.dst] = __ldg(&c.left[r[in.a]]); break;
+            case VM_RIGHT: r[in.dst] = __ldg(&c.right[r[in.a]]); break;
+            case VM_TOK: r[in.dst] = __ldg(&c.tok[r[in.a]]); break;
+            case VM_BRZ: if (r[in.a] == 0) pc = in.imm; break;     // Switch: the false side
+            case VM_JMP: pc = in.imm; break;
+            case VM_CALL: {                                         // Call_i
+                uint64_t nt;
+                if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt)) return;
+                ++st.invocations;
+                if (c.tag_mode == RDF_TAGS_PATH) {
+                    const uint32_t d = (uint32_t)(nt >> RDF_DEPTH_SHIFT) & 63u;
+                    if (d > st.max_depth) st.max_depth = d;
+                }
+                push_token(c, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
+                break;
+            }
+            case VM_RET:
+            case VM_PORT: {
+                const int64_t val = r[in.a];
+                int node = -1, port = 0;
+                if (in.op == VM_PORT) {
+                    node = in.imm;
+                    port = in.b;
+                } else {
+                    // Return_i: pop until the value reaches an operator of some caller
+                    for (;;) {
+                        uint32_t label;
+                        uint64_t parent;
+                        tag_pop(c, tag, label, parent);
+                        trace_rec(c, tag, val, 1, label, (uint32_t)parent);
+                        tag = parent;
+                        const LabelInfo& L = sp.labels[label];
+                        if (L.k_kind == K_RET) continue;           // the call was the caller's own output
+                        if (L.k_kind == K_SEG) {
+                            r[0] = val;
+                            pc = L.k_pc;
+                        } else {
+                            node = L.k_node;
+                            port = L.k_port;
+                        }
+                        break;
+                    }
+                    if (node < 0) break;                            // continue in the caller's segment
+                }
+                const MatchNode& M = sp.match[node];
+                int done;
+                if (c.tag_mode == RDF_TAGS_PATH) {
+                    int64_t partner = 0;
+                    done = hash_insert_or_consume(c, node, tag, val, partner, st.sc);
+                    if (done < 0) {
+                        set_status(c, RDF_ERR_STORE_FULL);
+                        return;
+                    }
+                    if (done) {
+                        r[port] = val;
+                        r[1 - port] = partner;
+                    }
+                } else {
+                    done = dense_deliver(c, M, node, tag, port, val, r, st.sc);
+                }
+                if (!done) {
+                    if (in.op == VM_RET) return;                    // parked: this token's journey ends here
+                    break;                                          // VM_PORT inside a segment: carry on
+                }
+                if (M.kind == MATCH_INT) {
+                    pc = M.cont_pc;                                 // r[0..n) hold the operands
+                    break;
+                }
+                fire_cell(c, M, wave, tag, r, st);
+                return;
+            }
+            case VM_OUT: {
+                const long long inst = c.tag_mode == RDF_TAGS_PATH ? (long long)(tag >> RDF_INST_SHIFT) : (long long)tag;
+                if (inst >= 0 && inst < c.B) c.y[inst] = r[in.a];
+                return;
+            }
+            case VM_EMBED:
+            case VM_LEAF_LSTM: {
+                const uint32_t i = aggregated_inc(&c.ctl->leaf_count[wave & 1]);
+                if (i >= c.work_cap) {
+                    set_status(c, RDF_ERR_QUEUE_FULL);
+                    return;
+                }
+                LeafItem it;
+                it.slot = (uint32_t)tag;
+                it.tok = (int32_t)r[in.a];
+                c.leaf_items[i] = it;
+                c.op_l[tag] = LEAF_MARK;
+                c.op_r[tag] = (uint32_t)it.tok;
+                ++st.leaves;
+                push_token(c, wave, tag, (int64_t)tag, (uint32_t)in.imm);
+                break;
+            }
+            default:   // VM_HALT
+                return;
+        }
+    }
+    set_status(c, RDF_ERR_WAVE_LIMIT);
+}
+
+// ===========================================================================
+// C phase, fp32: leaf gather and the TreeRNN cell as a tiled FFMA contraction
+// ===========================================================================
+// out[i][j] = tanh( sum_k W[j][k] * x_i[k] + b[j] ),  x_i = [state(l_i) ; state(r_i)]
+__device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) {
+    const int H = c.H, K2 = 2 * c.H;
+    const int tiles_m = (n_items + TM - 1) / TM, tiles_n = (H + TN - 1) / TN;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int lrow = threadIdx.x / 4, lk = (threadIdx.x % 4) * 4;
+    for (int tile = blockIdx.x; tile < tiles_m * tiles_n; tile += gridDim.x) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int row0 = tm * TM, col0 = tn * TN;
+        // this thread's source rows for the operand loads
+        const int arow = row0 + lrow;
+        const float *xl = nullptr, *xr = nullptr;
+        if (arow < (int)n_items) {
+            const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[arow]));   // {out, l, r, -}
+            xl = c.arena + (size_t)it.y * H;
+            xr = c.arena + (size_t)it.z * H;
+        }
+        const int bcol = col0 + lrow;
+        const float* wrow = bcol < H ? c.W + (size_t)bcol * K2 : nullptr;
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int k0 = 0; k0 < K2; k0 += TK) {
+            const int k = k0 + lk;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            if (xl && k < K2) a = k < H ? ldcg4(xl + k) : ldcg4(xr + (k - H));
+            if (wrow && k < K2) b = __ldg(reinterpret_cast<const float4*>(wrow + k));
+            __syncthreads();
+            sm.As[lk + 0][lrow] = a.x; sm.As[lk + 1][lrow] = a.y; sm.As[lk + 2][lrow] = a.z; sm.As[lk + 3][lrow] = a.w;
+            sm.Bs[lk + 0][lrow] = b.x; sm.Bs[lk + 1][lrow] = b.y; sm.Bs[lk + 2][lrow] = b.z; sm.Bs[lk + 3][lrow] = b.w;
+            __syncthreads();
+            gemm_tile_step(sm, tx, ty, acc);
+        }
+        const int col = col0 + tx * 4;
+        if (col < H) {
+            const float4 bias = __ldg(reinterpret_cast<const float4*>(c.b + col));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = row0 + ty * 4 + i;
+                if (row < (int)n_items) {
+                    const uint32_t out = __ldcg(&c.cell_items[row].out);
+                    float4 v;
+                    v.x = tanhf(acc[i][0] + bias.x); v.y = tanhf(acc[i][1] + bias.y);
+                    v.z = tanhf(acc[i][2] + bias.z); v.w = tanhf(acc[i][3] + bias.w);
+                    *reinterpret_cast<float4*>(c.arena + (size_t)out * H + col) = v;
+                }
+            }
+        }
+    }
+}
+
+__device__ void rnn_leaf_rows(const DevCtx& c, uint32_t n_items) {
+    // one warp per leaf: state(slot) = E[tok]
+    const int H = c.H;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
+    const int n_warps = gridDim.x * blockDim.x / 32;
+    for (uint32_t i = warp; i < n_items; i += n_warps) {
+        const uint2 it = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[i]));          // {slot, tok}
+        const float4* src = reinterpret_cast<const float4*>(c.E + (size_t)it.y * c.D);
+        float4* dst = reinterpret_cast<float4*>(c.arena + (size_t)it.x * H);
+        for (int k = lane; k < H / 4; k += 32) dst[k] = __ldg(src + k);
+    }
+}
+
+// ===========================================================================
+// the persistent forward kernel
+// ===========================================================================
+__global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= c.B) return;
+    // one token <[], x_b> per instance enters `result`
+    uint64_t tag;
+    const int64_t datum = c.x ? c.x[b] : (int64_t)c.tree_root[b];
+    if (c.tag_mode == RDF_TAGS_PATH) {
+        tag = path_root(b);
+    } else {
+        tag = (uint64_t)b;            // frames 0..B-1 are the contexts of `result`
+        Frame f;
+        f.parent = LEAF_MARK; f.label = 0; f.arg = datum;
+        c.frames[b] = f;
+    }
+    store_token(&c.q[0][b], tag, datum, (uint32_t)c.result_entry_pc);
+    if (b == 0) {
+        c.ctl->qcount[0] = (uint32_t)c.B;
+        c.ctl->frame_count = c.tag_mode == RDF_TAGS_FRAME ? (uint32_t)c.B : 0u;
+    }
+}
+
+__global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ SharedProgram sp;
+    __shared__ GemmSmem gsm;
+    load_program(c, sp);
+    ThreadStats st;
+    uint32_t generation = 0, wave = 0, widest = 0;
+    for (;; ++wave) {
+        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
+        if (n == 0) break;
+        if (wave >= c.wave_limit) {
+            set_status(c, RDF_ERR_WAVE_LIMIT);
+            break;
+        }
+        widest = max(widest, n);
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            c.ctl->qcount[(wave + 2) % 3] = 0;       // the counter the next wave appends to
+            c.ctl->cell_count[(wave + 1) & 1] = 0;
+            c.ctl->leaf_count[(wave + 1) & 1] = 0;
+        }
+        // ---- S: every token of this wave, one per thread
+        const Token* q = c.q[wave & 1];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+            run_token(c, sp, wave, load_token(&q[i]), st);
+        if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        // ---- C: the wave's ready batched operators
+        const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
+        const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
+        if (n_leaf | n_cell) {
+            if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
+            if (n_cell) rnn_cell_tiles(c, gsm, min(n_cell, c.work_cap));
+            if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        }
+    }
+    // ---- statistics
+    atomicAdd(&c.ctl->invocations, (unsigned long long)st.invocations);
+    atomicAdd(&c.ctl->tokens, (unsigned long long)st.tokens);
+    atomicAdd(&c.ctl->cells, (unsigned long long)st.cells);
+    atomicAdd(&c.ctl->leaves, (unsigned long long)st.leaves);
+    atomicAdd(&c.ctl->store_inserts, (unsigned long long)st.sc.inserts);
+    atomicAdd(&c.ctl->store_matches, (unsigned long long)st.sc.matches);
+    atomicAdd(&c.ctl->store_probes, (unsigned long long)st.sc.probes);
+    atomicMax(&c.ctl->max_probe, st.sc.max_probe);
+    atomicMax(&c.ctl->max_depth, st.max_depth);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        c.ctl->waves = wave;
+        c.ctl->max_wave_tokens = widest;
+    }
+}
+
+// root states: h_root[b] = state(frame y[b])
+__global__ void rdf_gather_roots_kernel(const DevCtx c, float* h_root) {
+    const int b = blockIdx.x;
+    const long long slot = c.y[b];
+    if (slot < 0 || slot >= (long long)c.frame_cap) return;
+    for (int k = threadIdx.x; k < c.H; k += blockDim.x) h_root[(size_t)b * c.H + k] = c.arena[(size_t)slot * c.H + k];
+}
+
+// ===========================================================================
+// host side: workspace plan, launches
+// ===========================================================================
+namespace {
+
+struct Plan {
+    size_t off = 0;
+    template <class T>
+    size_t take(size_t count) {
+        off = (off + 255) & ~(size_t)255;
+        size_t at = off;
+        off += count * sizeof(T);
+        return at;
+    }
+};
+
+uint64_t pow2_at_least(uint64_t v) {
+    uint64_t p = 1024;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* params, int want_grad, Layout& L) {
+    if (!g || !in || in->B <= 0 || in->max_invocations <= 0) return RDF_ERR_BAD_ARG;
+    if (g->has_vector_ops && (!params || params->H <= 0 || params->H % 4 != 0)) return RDF_ERR_BAD_ARG;
+    if (in->B + in->max_invocations >= 0xFFFFFFF0ll) return RDF_ERR_BAD_ARG;
+    if (g->tag_mode == RDF_TAGS_PATH && in->B > (1ll << 20)) return RDF_ERR_BAD_ARG;
+    if (want_grad && !g->has_vector_ops) return RDF_ERR_UNSUPPORTED;
+    const int H = g->has_vector_ops ? params->H : 0;
+    Plan P;
+    L.qcap = (uint32_t)std::min<long long>(in->max_wave_tokens > 0 ? in->max_wave_tokens : in->max_invocations + in->B,
+                                           0x7FFFFFFFll);
+    L.qcap = std::max<uint32_t>(L.qcap, (uint32_t)in->B);
+    L.frame_cap = g->tag_mode == RDF_TAGS_FRAME ? (uint32_t)(in->B + in->max_invocations) : 0;
+    L.work_cap = g->has_vector_ops ? L.qcap : 0;
+    L.ctl = P.take<char>(4096);
+    L.code = P.take<VmInstr>(g->code.size());
+    L.match = P.take<MatchNode>(std::max<size_t>(1, g->match.size()));
+    L.labels = P.take<LabelInfo>(std::max<size_t>(1, g->labels.size()));
+    L.consts = P.take<int64_t>(std::max<size_t>(1, g->consts.size()));
+    L.q0 = P.take<Token>(L.qcap);
+    L.q1 = P.take<Token>(L.qcap);
+    L.frames = P.take<Frame>(L.frame_cap);
+    L.children = P.take<uint32_t>((size_t)L.frame_cap * g->max_calls_per_body);
+    L.port_val = P.take<int64_t>((size_t)L.frame_cap * g->n_ports_total);
+    L.arrived_bytes = (size_t)L.frame_cap * std::max<size_t>(1, g->match.size()) * sizeof(uint32_t);
+    L.arrived = P.take<char>(L.arrived_bytes);
+    L.table_cap = g->tag_mode == RDF_TAGS_PATH && !g->match.empty() ? pow2_at_least((uint64_t)in->max_invocations) : 0;
+    L.table_bytes = (size_t)L.table_cap * g->match.size() * sizeof(Slot);
+    L.table = P.take<char>(L.table_bytes);
+    L.cell_items = P.take<CellItem>(L.work_cap);
+    L.leaf_items = P.take<LeafItem>(L.work_cap);
+    const size_t vf = g->has_vector_ops ? L.frame_cap : 0;
+    L.op_l = P.take<uint32_t>(vf);
+    L.op_r = P.take<uint32_t>(vf);
+    L.arena = P.take<float>(vf * H);
+    L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
+    const size_t gf = want_grad ? L.frame_cap : 0;
+    L.dhp = P.take<float>(gf * H);
+    L.dlog = P.take<float>(gf * 8);
+    L.bq0 = P.take<uint32_t>(gf);
+    L.bq1 = P.take<uint32_t>(gf);
+    L.all_cells = P.take<uint32_t>(gf);
+    L.all_leaves = P.take<uint32_t>(gf);
+    L.loss_partial = P.take<float>(want_grad ? 4096 : 0);
+    L.total = (P.off + 255) & ~(size_t)255;
+    return RDF_OK;
+}
+
+ExecState* rdf_state_of(rdf_graph* g) {
+    if (!g->dev) g->dev = new ExecState();
+    return static_cast<ExecState*>(g->dev);
+}
+
+int rdf_prepare_device(rdf_graph* g, ExecState* S) {
+    (void)g;
+    int dev = 0;
+    CUDA_OK(cudaGetDevice(&dev));
+    if (S->device == dev && S->grid > 0) return RDF_OK;
+    int sms = 0, per_sm = 0, coop = 0;
+    CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUDA_OK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    CUDA_OK(cudaDeviceGetAttribute(&S->clock_khz, cudaDevAttrClockRate, dev));
+    if (!coop) return RDF_ERR_CUDA;
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, 0));
+    if (per_sm < 1) return RDF_ERR_CUDA;
+    S->grid = sms;                 // one persistent block per SM
+    S->device = dev;
+    return RDF_OK;
+}
+
+void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, char* ws,
+                  const Layout& L, ExecState* S, DevCtx& c) {
+    memset(&c, 0, sizeof(c));
+    c.code = reinterpret_cast<const VmInstr*>(ws + L.code);
+    c.match = reinterpret_cast<const MatchNode*>(ws + L.match);
+    c.labels = reinterpret_cast<const LabelInfo*>(ws + L.labels);
+    c.consts = reinterpret_cast<const int64_t*>(ws + L.consts);
+    c.n_code = (int)g->code.size(); c.n_match = (int)g->match.size();
+    c.n_labels = (int)g->labels.size(); c.n_consts = (int)g->consts.size();
+    c.label_bits = g->label_bits; c.tag_mode = g->tag_mode; c.result_entry_pc = g->result_entry_pc;
+    c.n_ports_total = g->n_ports_total; c.K = g->max_calls_per_body;
+    c.B = in->B; c.N = in->N; c.x = in->x;
+    c.tree_root = in->tree_root; c.left = in->left; c.right = in->right; c.tok = in->tok; c.label = in->label;
+    c.q[0] = reinterpret_cast<Token*>(ws + L.q0); c.q[1] = reinterpret_cast<Token*>(ws + L.q1);
+    c.qcap = L.qcap;
+    c.frames = reinterpret_cast<Frame*>(ws + L.frames);
+    c.children = reinterpret_cast<uint32_t*>(ws + L.children);
+    c.frame_cap = L.frame_cap;
+    c.port_val = reinterpret_cast<int64_t*>(ws + L.port_val);
+    c.arrived = reinterpret_cast<uint32_t*>(ws + L.arrived);
+    c.table = reinterpret_cast<Slot*>(ws + L.table);
+    c.table_cap = L.table_cap;
+    c.cell_items = reinterpret_cast<CellItem*>(ws + L.cell_items);
+    c.leaf_items = reinterpret_cast<LeafItem*>(ws + L.leaf_items);
+    c.work_cap = L.work_cap;
+    c.op_l = reinterpret_cast<uint32_t*>(ws + L.op_l);
+    c.op_r = reinterpret_cast<uint32_t*>(ws + L.op_r);
+    c.arena = reinterpret_cast<float*>(ws + L.arena);
+    if (g->has_vector_ops) {
+        c.H = params->H; c.D = params->D; c.V = params->V; c.n_classes = params->n_classes; c.compute = params->compute;
+        c.E = params->E; c.W = params->W; c.b = params->b; c.W_x = params->W_x; c.b_x = params->b_x;
+        c.W_s = params->W_s; c.b_s = params->b_s;
+        c.y = reinterpret_cast<int64_t*>(ws + L.ybuf);
+    } else {
+        c.y = out->y;
+    }
+    c.trace = out->trace; c.trace_cap = out->trace ? out->trace_capacity : 0;
+    c.dhp = reinterpret_cast<float*>(ws + L.dhp);
+    c.dlog = reinterpret_cast<float*>(ws + L.dlog);
+    c.bq[0] = reinterpret_cast<uint32_t*>(ws + L.bq0); c.bq[1] = reinterpret_cast<uint32_t*>(ws + L.bq1);
+    c.all_cells = reinterpret_cast<uint32_t*>(ws + L.all_cells);
+    c.all_leaves = reinterpret_cast<uint32_t*>(ws + L.all_leaves);
+    c.loss_partial = reinterpret_cast<float*>(ws + L.loss_partial);
+    c.loss_out = out->loss;
+    c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
+    c.wave_limit = 1u << 24;
+    c.spin_limit = (long long)S->clock_khz * 2000ll;       // about two seconds of SM clock
+}
+
+int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, void* ws) {
+    if (!g || !in || !out || !ws) return RDF_ERR_BAD_ARG;
+    if ((uintptr_t)ws & 255) return RDF_ERR_BAD_ARG;
+    if (g->uses_tree) {
+        if (!in->tree_root || !in->left || !in->right || !in->tok || in->N <= 0) return RDF_ERR_BAD_ARG;
+    } else if (!in->x) {
+        return RDF_ERR_BAD_ARG;
+    }
+    if (g->has_vector_ops) {
+        if (!params || !params->E || !params->W || !params->b || !out->h_root) return RDF_ERR_BAD_ARG;
+        if (params->D != params->H) return RDF_ERR_UNSUPPORTED;
+        if (g->has_lstm) return RDF_ERR_UNSUPPORTED;
+        if (params->compute != RDF_F32 && params->compute != RDF_BF16) return RDF_ERR_BAD_ARG;
+    } else if (!out->y) {
+        return RDF_ERR_BAD_ARG;
+    }
+    if (out->trace && (!out->trace_count || out->trace_capacity <= 0)) return RDF_ERR_BAD_ARG;
+    return RDF_OK;
+}
+
+// zero what must start at zero, upload the program, seed, run all waves
+int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
+                       DevCtx& c, cudaStream_t stream) {
+    CUDA_OK(cudaMemsetAsync(ws + L.ctl, 0, 4096, stream));
+    if (L.arrived_bytes && g->tag_mode == RDF_TAGS_FRAME) CUDA_OK(cudaMemsetAsync(ws + L.arrived, 0, L.arrived_bytes, stream));
+    if (L.table_bytes) CUDA_OK(cudaMemsetAsync(ws + L.table, 0xFF, L.table_bytes, stream));
+    CUDA_OK(cudaMemcpyAsync(ws + L.code, g->code.data(), g->code.size() * sizeof(VmInstr), cudaMemcpyHostToDevice, stream));
+    if (!g->match.empty())
+        CUDA_OK(cudaMemcpyAsync(ws + L.match, g->match.data(), g->match.size() * sizeof(MatchNode), cudaMemcpyHostToDevice, stream));
+    if (!g->labels.empty())
+        CUDA_OK(cudaMemcpyAsync(ws + L.labels, g->labels.data(), g->labels.size() * sizeof(LabelInfo), cudaMemcpyHostToDevice, stream));
+    if (!g->consts.empty())
+        CUDA_OK(cudaMemcpyAsync(ws + L.consts, g->consts.data(), g->consts.size() * sizeof(int64_t), cudaMemcpyHostToDevice, stream));
+    rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
+    CUDA_OK(cudaGetLastError());
+    void* args[] = {(void*)&c};
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
+    if (g->has_vector_ops) {
+        rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
+        CUDA_OK(cudaGetLastError());
+    }
+    if (out->trace)
+        CUDA_OK(cudaMemcpyAsync(out->trace_count, &c.ctl->trace_count, sizeof(uint64_t), cudaMemcpyDeviceToDevice, stream));
+    S->last_ctl = c.ctl;
+    S->last_stream = stream;
+    S->ran = true;
+    return RDF_OK;
+}
+
+void rdf_exec_release(rdf_graph* g) {
+    delete static_cast<ExecState*>(g->dev);
+    g->dev = nullptr;
+}
+
+extern "C" int rdf_workspace_bytes(const rdf_graph* g, const rdf_batch* in, const rdf_params* params, int want_grad,
+                                   size_t* bytes) {
+    if (!bytes) return RDF_ERR_BAD_ARG;
+    Layout L;
+    int rc = rdf_make_layout(g, in, params, want_grad, L);
+    if (rc != RDF_OK) return rc;
+    *bytes = L.total;
+    return RDF_OK;
+}
+
+extern "C" int rdf_eval(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    int rc = rdf_check_common(g, in, params, out, workspace);
+    if (rc != RDF_OK) return rc;
+    Layout L;
+    rc = rdf_make_layout(g, in, params, 0, L);
+    if (rc != RDF_OK) return rc;
+    if (workspace_bytes < L.total) return RDF_ERR_WORKSPACE_TOO_SMALL;
+    ExecState* S = rdf_state_of(g);
+    rc = rdf_prepare_device(g, S);
+    if (rc != RDF_OK) return rc;
+    DevCtx c;
+    rdf_fill_ctx(g, in, params, out, static_cast<char*>(workspace), L, S, c);
+    return rdf_launch_forward(g, in, out, static_cast<char*>(workspace), L, S, c, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
+    if (!g || !s) return RDF_ERR_BAD_ARG;
+    ExecState* S = rdf_state_of(g);
+    memset(s, 0, sizeof(*s));
+    if (!S->ran) return RDF_OK;
+    if (cudaStreamSynchronize(S->last_stream) != cudaSuccess) return RDF_ERR_CUDA;
+    Control h;
+    if (cudaMemcpy(&h, S->last_ctl, sizeof(Control), cudaMemcpyDeviceToHost) != cudaSuccess) return RDF_ERR_CUDA;
+    s->status = h.status;
+    s->waves = h.waves; s->waves_backward = h.waves_backward; s->max_wave_tokens = h.max_wave_tokens;
+    s->invocations = h.invocations; s->tokens = h.tokens;
+    s->store_inserts = h.store_inserts; s->store_matches = h.store_matches; s->store_probes = h.store_probes;
+    s->max_probe = h.max_probe; s->max_depth = h.max_depth; s->cells = h.cells; s->leaves = h.leaves;
+    return h.status;
+}

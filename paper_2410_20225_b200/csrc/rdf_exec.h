@@ -1,0 +1,60 @@
+// Shared between the forward executor (rdf_exec.cu) and the gradient pass
+// (rdf_grad.cu): workspace layout, per-graph host state, the fp32 tile step.
+#pragma once
+#include "rdf_device.cuh"
+
+// ---- fp32 tiled contraction: 64 x 64 output tile, 16-deep steps, 256 threads, 4 x 4 per thread
+static const int TM = 64, TN = 64, TK = 16;
+
+struct GemmSmem {
+    float As[TK][TM + 4];     // [k][row of the tile]
+    float Bs[TK][TN + 4];     // [k][column of the tile]
+};
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+
+__device__ __forceinline__ void gemm_tile_step(const GemmSmem& sm, int tx, int ty, float (&acc)[4][4]) {
+#pragma unroll
+    for (int kk = 0; kk < TK; ++kk) {
+        const float4 av = *reinterpret_cast<const float4*>(&sm.As[kk][ty * 4]);
+        const float4 bv = *reinterpret_cast<const float4*>(&sm.Bs[kk][tx * 4]);
+        const float aa[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(aa[i], bb[j], acc[i][j]);
+    }
+}
+
+// ---- host state
+struct ExecState {
+    int device = -1;
+    int grid = 0;
+    int clock_khz = 0;
+    void* last_ctl = nullptr;
+    cudaStream_t last_stream = nullptr;
+    bool ran = false;
+};
+
+struct Layout {
+    size_t ctl, code, match, labels, consts, q0, q1, frames, children, port_val, arrived, table, cell_items,
+        leaf_items, op_l, op_r, arena, ybuf, dhp, dlog, bq0, bq1, all_cells, all_leaves, loss_partial, total;
+    uint32_t qcap, frame_cap, work_cap;
+    uint64_t table_cap;
+    size_t arrived_bytes, table_bytes;
+};
+
+#define CUDA_OK(expr)                                  \
+    do {                                               \
+        cudaError_t e_ = (expr);                       \
+        if (e_ != cudaSuccess) return RDF_ERR_CUDA;    \
+    } while (0)
+
+int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* params, int want_grad, Layout& L);
+ExecState* rdf_state_of(rdf_graph* g);
+int rdf_prepare_device(rdf_graph* g, ExecState* S);
+void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, char* ws,
+                  const Layout& L, ExecState* S, DevCtx& c);
+int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, void* ws);
+int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
+                       DevCtx& c, cudaStream_t stream);

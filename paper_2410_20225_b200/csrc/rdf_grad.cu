@@ -1,0 +1,356 @@
+// Reverse mode (Section 4).  The forward run retains, per invocation, its
+// frame, its state and the operands of the operator that produced the state.
+// The gradient pass re-enters every invocation under the tag (frame) that its
+// forward Call_i created: wave 0 holds the invocations called from `result`,
+// each wave hands the gradients of a cell's operands to the frames of the two
+// calls it made (Call_1 / Call_2 replayed through the children table), until
+// the leaves are reached.  Parameter gradients are sums over all invocations
+// and are formed after the waves as dense contractions over the retained
+// per-invocation values.
+#include <algorithm>
+#include <cstring>
+
+#include "rdf_exec.h"
+
+static const int MAX_CLASSES = 8;
+
+// ---------------------------------------------------------------- loss head
+// per invocation f: z = W_s h + b_s; loss += logsumexp(z) - z[label]; dlog = softmax(z) - onehot
+__global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
+    __shared__ float warp_loss[8];
+    const uint32_t F = c.ctl->frame_count;
+    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
+    const uint32_t warp = blockIdx.x * 8 + wib, n_warps = gridDim.x * 8;
+    const int H = c.H, C = c.n_classes;
+    float my_loss = 0.f;
+    for (uint32_t f = (uint32_t)c.B + warp; f < F; f += n_warps) {
+        const float* h = c.arena + (size_t)f * H;
+        float z[MAX_CLASSES];
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
+        for (int j = lane; j < H; j += 32) {
+            const float hj = h[j];
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) z[k] = fmaf(__ldg(&c.W_s[k * H + j]), hj, z[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            for (int o = 16; o > 0; o >>= 1) z[k] += __shfl_xor_sync(0xffffffffu, z[k], o);
+        const int node = (int)c.frames[f].arg;
+        const int lab = __ldg(&c.label[node]);
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) {
+                z[k] += __ldg(&c.b_s[k]);
+                m = fmaxf(m, z[k]);
+            }
+        float s = 0.f, zl = 0.f;
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) {
+                s += expf(z[k] - m);
+                if (k == lab) zl = z[k];
+            }
+        if (lane == 0) {
+            my_loss += logf(s) + m - zl;
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                c.dlog[(size_t)f * 8 + k] = k < C ? expf(z[k] - m) / s - (k == lab ? 1.f : 0.f) : 0.f;
+        }
+    }
+    if (lane == 0) warp_loss[wib] = my_loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += warp_loss[w];
+        c.loss_partial[blockIdx.x] = t;
+    }
+}
+
+__global__ void rdf_loss_final_kernel(const DevCtx c, int n_partials) {
+    // one thread, fixed order: the same partials always give the same sum
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < n_partials; ++i) t += (double)c.loss_partial[i];
+        c.ctl->loss = (float)t;
+        if (c.loss_out) *c.loss_out = (float)t;
+    }
+}
+
+// ----------------------------------------------------------- backward waves
+__global__ void __launch_bounds__(256) rdf_backward_seed_kernel(const DevCtx c) {
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= c.B) return;
+    // dy enters the gradient of the call made by `result` under that call's own tag
+    c.bq[0][b] = c.children[(size_t)b * c.K + 0];
+    if (b == 0) c.ctl->bq_count[0] = (uint32_t)c.B;
+}
+
+// A: per invocation t of the wave, dh = (gradient from the caller) + W_s^T dlog;
+//    cell: dz = dh * (1 - h^2), queue the two callee frames; leaf: keep dh for dE.
+__device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
+    const int lane = threadIdx.x % 32;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    const int H = c.H, C = c.n_classes;
+    const uint32_t* q = c.bq[wave & 1];
+    for (uint32_t i = warp; i < n; i += n_warps) {
+        const uint32_t t = __ldcg(&q[i]);
+        const uint32_t parent = __ldcg(&c.frames[t].parent);
+        const bool from_result = parent < (uint32_t)c.B;
+        const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
+        const bool leaf = l == LEAF_MARK;
+        float dl[MAX_CLASSES];
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = c.W_s ? __ldcg(&c.dlog[(size_t)t * 8 + k]) : 0.f;
+        float* g = c.dhp + (size_t)t * H;
+        const float* h = c.arena + (size_t)t * H;
+        for (int j = lane; j < H; j += 32) {
+            float dh = from_result ? 0.f : __ldcg(&g[j]);
+            if (c.W_s) {
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
+            }
+            if (!leaf) {
+                const float hj = __ldcg(&h[j]);
+                dh *= 1.f - hj * hj;
+            }
+            g[j] = dh;
+        }
+        if (lane == 0) {
+            if (leaf) {
+                c.all_leaves[atomicAdd(&c.ctl->all_leaves, 1u)] = t;
+            } else {
+                c.all_cells[atomicAdd(&c.ctl->all_cells, 1u)] = t;
+                const uint32_t at = atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u);
+                uint32_t* qn = c.bq[(wave + 1) & 1];
+                qn[at] = l;
+                qn[at + 1] = r;
+            }
+        }
+    }
+}
+
+// B: [dh_l ; dh_r] = W^T dz for the cells all_cells[first, first + n)
+__device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, uint32_t n_items) {
+    const int H = c.H, K2 = 2 * c.H;
+    const int tiles_m = (n_items + TM - 1) / TM, tiles_n = (K2 + TN - 1) / TN;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int arow_l = threadIdx.x / 4, ak = (threadIdx.x % 4) * 4;     // A loader: row, 4 consecutive k
+    const int bk = threadIdx.x / 16, bn = (threadIdx.x % 16) * 4;       // B loader: k, 4 consecutive columns
+    for (int tile = blockIdx.x; tile < tiles_m * tiles_n; tile += gridDim.x) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int row0 = tm * TM, col0 = tn * TN;
+        const int arow = row0 + arow_l;
+        const float* dz = nullptr;
+        if (arow < (int)n_items) dz = c.dhp + (size_t)__ldcg(&c.all_cells[first + arow]) * H;
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int k0 = 0; k0 < H; k0 += TK) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            if (dz && k0 + ak < H) a = ldcg4(dz + k0 + ak);
+            if (k0 + bk < H && col0 + bn < K2) b = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)(k0 + bk) * K2 + col0 + bn));
+            __syncthreads();
+            sm.As[ak + 0][arow_l] = a.x; sm.As[ak + 1][arow_l] = a.y; sm.As[ak + 2][arow_l] = a.z; sm.As[ak + 3][arow_l] = a.w;
+            *reinterpret_cast<float4*>(&sm.Bs[bk][bn]) = b;
+            __syncthreads();
+            gemm_tile_step(sm, tx, ty, acc);
+        }
+        const int col = col0 + tx * 4;
+        if (col < K2) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = row0 + ty * 4 + i;
+                if (row < (int)n_items) {
+                    const uint32_t t = __ldcg(&c.all_cells[first + row]);
+                    const uint32_t child = col < H ? __ldcg(&c.op_l[t]) : __ldcg(&c.op_r[t]);
+                    const int cc = col < H ? col : col - H;
+                    *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + cc) =
+                        make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                }
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ GemmSmem gsm;
+    uint32_t generation = 0, wave = 0, first = 0;
+    for (;; ++wave) {
+        const uint32_t n = ld_volatile_u32(&c.ctl->bq_count[wave % 3]);
+        if (n == 0) break;
+        if (wave >= c.wave_limit) {
+            set_status(c, RDF_ERR_WAVE_LIMIT);
+            break;
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->bq_count[(wave + 2) % 3] = 0;
+        backward_frames(c, wave, n);
+        if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+        const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
+        if (end > first) {
+            backward_operand_tiles(c, gsm, first, end - first);
+            first = end;
+            if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->waves_backward = wave;
+}
+
+// ------------------------------------------- parameter gradients (post pass)
+// dW[j][k] = sum over cells t of dz_t[j] * x_t[k],  x_t = [state(l_t) ; state(r_t)];  split over the cells
+__global__ void __launch_bounds__(256) rdf_dw_kernel(const DevCtx c, int tiles_m, int tiles_n, uint32_t chunk) {
+    __shared__ GemmSmem sm;
+    const uint32_t n_cells = c.ctl->all_cells;
+    const int tile = blockIdx.x % (tiles_m * tiles_n), split = blockIdx.x / (tiles_m * tiles_n);
+    const uint32_t t_begin = (uint32_t)split * chunk, t_end = min(n_cells, t_begin + chunk);
+    if (t_begin >= t_end) return;
+    const int H = c.H, K2 = 2 * c.H;
+    const int tm = tile / tiles_n, tn = tile % tiles_n;
+    const int row0 = tm * TM, col0 = tn * TN;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int lk = threadIdx.x / 16, l4 = (threadIdx.x % 16) * 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (uint32_t t0 = t_begin; t0 < t_end; t0 += TK) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (t0 + lk < t_end) {
+            const uint32_t t = c.all_cells[t0 + lk];
+            if (row0 + l4 < H) a = *reinterpret_cast<const float4*>(c.dhp + (size_t)t * H + row0 + l4);
+            const int col = col0 + l4;
+            if (col < K2) {
+                const uint32_t src = col < H ? c.op_l[t] : c.op_r[t];
+                b = *reinterpret_cast<const float4*>(c.arena + (size_t)src * H + (col < H ? col : col - H));
+            }
+        }
+        __syncthreads();
+        *reinterpret_cast<float4*>(&sm.As[lk][l4]) = a;
+        *reinterpret_cast<float4*>(&sm.Bs[lk][l4]) = b;
+        __syncthreads();
+        gemm_tile_step(sm, tx, ty, acc);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = row0 + ty * 4 + i;
+        if (row >= H) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = col0 + tx * 4 + j;
+            if (col < K2) atomicAdd(&c.dW[(size_t)row * K2 + col], acc[i][j]);
+        }
+    }
+}
+
+// db[j] = sum over cells of dz_t[j]
+__global__ void __launch_bounds__(256) rdf_db_kernel(const DevCtx c) {
+    const uint32_t n_cells = c.ctl->all_cells;
+    const uint32_t per = (n_cells + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = blockIdx.x * per, t1 = min(n_cells, t0 + per);
+    for (int j = threadIdx.x; j < c.H; j += blockDim.x) {
+        float s = 0.f;
+        for (uint32_t i = t0; i < t1; ++i) s += c.dhp[(size_t)c.all_cells[i] * c.H + j];
+        if (t1 > t0) atomicAdd(&c.db[j], s);
+    }
+}
+
+// dW_s[k][j] = sum over invocations of dlog_f[k] * h_f[j];  db_s[k] = sum of dlog_f[k]
+__global__ void __launch_bounds__(256) rdf_dws_kernel(const DevCtx c) {
+    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
+    const uint32_t n = F - B, per = (n + gridDim.x - 1) / gridDim.x;
+    const uint32_t f0 = B + blockIdx.x * per, f1 = min(F, f0 + per);
+    if (f0 >= f1) return;
+    const int H = c.H, C = c.n_classes;
+    for (int j = threadIdx.x; j < H; j += blockDim.x) {
+        float s[MAX_CLASSES];
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) s[k] = 0.f;
+        for (uint32_t f = f0; f < f1; ++f) {
+            const float hj = c.arena[(size_t)f * H + j];
+            const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8);
+            const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8 + 4);
+            s[0] = fmaf(d0.x, hj, s[0]); s[1] = fmaf(d0.y, hj, s[1]); s[2] = fmaf(d0.z, hj, s[2]); s[3] = fmaf(d0.w, hj, s[3]);
+            s[4] = fmaf(d1.x, hj, s[4]); s[5] = fmaf(d1.y, hj, s[5]); s[6] = fmaf(d1.z, hj, s[6]); s[7] = fmaf(d1.w, hj, s[7]);
+        }
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) atomicAdd(&c.dW_s[k * H + j], s[k]);
+    }
+    if (threadIdx.x < C) {
+        float s = 0.f;
+        for (uint32_t f = f0; f < f1; ++f) s += c.dlog[(size_t)f * 8 + threadIdx.x];
+        atomicAdd(&c.db_s[threadIdx.x], s);
+    }
+}
+
+// dE[tok] += dh of every leaf invocation that read row tok
+__global__ void __launch_bounds__(256) rdf_de_kernel(const DevCtx c) {
+    const uint32_t n = c.ctl->all_leaves;
+    const int lane = threadIdx.x % 32;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    for (uint32_t i = warp; i < n; i += n_warps) {
+        const uint32_t t = c.all_leaves[i];
+        const uint32_t tok = c.op_r[t];
+        for (int j = lane; j < c.H; j += 32) atomicAdd(&c.dE[(size_t)tok * c.D + j], c.dhp[(size_t)t * c.H + j]);
+    }
+}
+
+// --------------------------------------------------------------------- host
+extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
+                        rdf_param_grads* grads, void* workspace, size_t workspace_bytes, void* stream_v) {
+    int rc = rdf_check_common(g, in, params, out, workspace);
+    if (rc != RDF_OK) return rc;
+    if (!g->has_vector_ops || !g->has_loss) return RDF_ERR_UNSUPPORTED;
+    if (!grads || !grads->dE || !grads->dW || !grads->db || !grads->dW_s || !grads->db_s) return RDF_ERR_BAD_ARG;
+    if (!params->W_s || !params->b_s || !in->label || !out->loss) return RDF_ERR_BAD_ARG;
+    if (params->n_classes < 1 || params->n_classes > MAX_CLASSES) return RDF_ERR_BAD_ARG;
+    Layout L;
+    rc = rdf_make_layout(g, in, params, 1, L);
+    if (rc != RDF_OK) return rc;
+    if (workspace_bytes < L.total) return RDF_ERR_WORKSPACE_TOO_SMALL;
+    ExecState* S = rdf_state_of(g);
+    rc = rdf_prepare_device(g, S);
+    if (rc != RDF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    char* ws = static_cast<char*>(workspace);
+    DevCtx c;
+    rdf_fill_ctx(g, in, params, out, ws, L, S, c);
+    c.dE = grads->dE; c.dW = grads->dW; c.db = grads->db; c.dW_x = grads->dW_x; c.db_x = grads->db_x;
+    c.dW_s = grads->dW_s; c.db_s = grads->db_s;
+    const int H = params->H;
+    // gradients are sums: start from zero
+    CUDA_OK(cudaMemsetAsync(grads->dE, 0, (size_t)params->V * params->D * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->dW, 0, (size_t)H * 2 * H * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->db, 0, (size_t)H * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->dW_s, 0, (size_t)params->n_classes * H * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->db_s, 0, (size_t)params->n_classes * sizeof(float), stream));
+    rc = rdf_launch_forward(g, in, out, ws, L, S, c, stream);
+    if (rc != RDF_OK) return rc;
+    // loss head over every retained invocation
+    const int loss_blocks = std::min(4096, std::max(1, (int)((in->max_invocations + 63) / 64)));
+    rdf_loss_kernel<<<loss_blocks, 256, 0, stream>>>(c);
+    rdf_loss_final_kernel<<<1, 32, 0, stream>>>(c, loss_blocks);
+    // gradient waves
+    rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
+    CUDA_OK(cudaGetLastError());
+    void* args[] = {(void*)&c};
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
+    // parameter gradients
+    const int tiles_m = (H + TM - 1) / TM, tiles_n = (2 * H + TN - 1) / TN;
+    const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
+    int splits = (int)std::max<long long>(1, std::min<long long>((max_cells + 255) / 256, (4 * S->grid) / (tiles_m * tiles_n) + 1));
+    uint32_t chunk = (uint32_t)((max_cells + splits - 1) / splits);
+    chunk = (chunk + TK - 1) / TK * TK;
+    rdf_dw_kernel<<<tiles_m * tiles_n * splits, 256, 0, stream>>>(c, tiles_m, tiles_n, chunk);
+    rdf_db_kernel<<<S->grid, 256, 0, stream>>>(c);
+    rdf_dws_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+    rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
+    CUDA_OK(cudaGetLastError());
+    return RDF_OK;
+}

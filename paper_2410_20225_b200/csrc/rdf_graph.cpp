@@ -1,0 +1,660 @@
+// Host side of the library: program validation, the graph transformation of
+// Section 3 (recursive definitions -> one static graph with Call_i / Return_i),
+// and the lowering of that graph into segments for the device executor.
+#include <algorithm>
+#include <climits>
+#include <cstring>
+#include <functional>
+#include <map>
+#include <set>
+
+#include "rdf_internal.h"
+
+namespace {
+
+struct Err {
+    int code;
+};
+
+inline void require(bool ok, int code) {
+    if (!ok) throw Err{code};
+}
+
+int arity_of(int op) {
+    switch (op) {
+        case RDF_OP_PARAM: case RDF_OP_CONST: return 0;
+        case RDF_OP_ADD: case RDF_OP_SUB: case RDF_OP_MUL: case RDF_OP_MAX:
+        case RDF_OP_LT: case RDF_OP_EQ: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
+        case RDF_OP_NODE_LOSS: return 2;
+        case RDF_OP_IF: return 3;
+        case RDF_OP_CALL: case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK:
+        case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: return 1;
+        default: return -1;
+    }
+}
+
+struct Prog {
+    const rdf_program* p;
+    const rdf_function& fn(int i) const { return p->functions[i]; }
+    const rdf_expr& ex(int f, int e) const { return p->functions[f].exprs[e]; }
+};
+
+// ---------------------------------------------------------------- validation
+void validate(const Prog& P) {
+    const rdf_program* p = P.p;
+    require(p->n_functions > 0 && p->functions, RDF_ERR_BAD_PROGRAM);
+    require(p->result >= 0 && p->result < p->n_functions, RDF_ERR_BAD_PROGRAM);
+    require(p->tag_mode == RDF_TAGS_PATH || p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_BAD_ARG);
+    for (int f = 0; f < p->n_functions; ++f) {
+        const rdf_function& F = p->functions[f];
+        require(F.exprs && F.n_exprs > 0 && F.n_params >= 0 && F.name, RDF_ERR_BAD_PROGRAM);
+        require(F.root >= 0 && F.root < F.n_exprs, RDF_ERR_BAD_PROGRAM);
+        for (int e = 0; e < F.n_exprs; ++e) {
+            const rdf_expr& x = F.exprs[e];
+            int ar = arity_of(x.op);
+            require(ar >= 0, RDF_ERR_BAD_PROGRAM);
+            int ops[3] = {x.a, x.b, x.c};
+            for (int k = 0; k < ar; ++k) require(ops[k] >= 0 && ops[k] < F.n_exprs, RDF_ERR_BAD_PROGRAM);
+            if (x.op == RDF_OP_PARAM) require(x.imm >= 0 && x.imm < F.n_params, RDF_ERR_BAD_PROGRAM);
+            if (x.op == RDF_OP_CALL) {
+                require(x.imm >= 0 && x.imm < p->n_functions, RDF_ERR_BAD_PROGRAM);   // unknown callee
+                require(x.imm != p->result, RDF_ERR_BAD_PROGRAM);
+                const int m = p->functions[x.imm].n_params;
+                require(m >= 1, RDF_ERR_BAD_PROGRAM);
+                require(m == 1, RDF_ERR_UNSUPPORTED);     // several parameters: valid, not lowered yet
+            }
+        }
+        // no cycles among expressions
+        std::vector<int> state(F.n_exprs, 0);
+        std::function<void(int)> dfs = [&](int e) {
+            require(state[e] != 1, RDF_ERR_BAD_PROGRAM);
+            if (state[e] == 2) return;
+            state[e] = 1;
+            const rdf_expr& x = F.exprs[e];
+            int ops[3] = {x.a, x.b, x.c};
+            for (int k = 0; k < arity_of(x.op); ++k) dfs(ops[k]);
+            state[e] = 2;
+        };
+        dfs(F.root);
+    }
+}
+
+// ------------------------------------------------- literal graph (Section 3)
+const int NODE_FCALL = 100;   // placeholder: "a node labeled with the name of f"
+
+struct Literal {
+    const Prog& P;
+    std::vector<rdf_node>& nodes;
+    std::vector<rdf_edge>& edges;
+    std::vector<int> in_node;    // per function: first IN node
+    std::vector<int> out_node;   // per function: OUT node
+    std::vector<int64_t> callee; // per node: callee of an FCALL placeholder
+
+    int add(int kind, int op, int func, int n_in, int64_t value = 0, int param = 0) {
+        rdf_node n;
+        n.kind = kind; n.op = op; n.label = -1; n.func = func; n.param = param; n.n_in = n_in; n.value = value;
+        nodes.push_back(n);
+        callee.push_back(-1);
+        return (int)nodes.size() - 1;
+    }
+    void connect(int src, int sp, int dst, int dp, int control = 0) {
+        edges.push_back(rdf_edge{src, sp, dst, dp, control});
+    }
+
+    uint32_t params_used(int f, int e, std::map<int, uint32_t>& memo) {
+        auto it = memo.find(e);
+        if (it != memo.end()) return it->second;
+        const rdf_expr& x = P.ex(f, e);
+        uint32_t m = 0;
+        if (x.op == RDF_OP_PARAM) m = 1u << x.imm;
+        int ops[3] = {x.a, x.b, x.c};
+        for (int k = 0; k < arity_of(x.op); ++k) m |= params_used(f, ops[k], memo);
+        memo[e] = m;
+        return m;
+    }
+
+    typedef std::pair<int, int> Val;   // (node, output port)
+    struct Ctx {
+        int id;
+        std::vector<Val> param;
+    };
+
+    void build_function(int f) {
+        const rdf_function& F = P.fn(f);
+        Ctx root{0, {}};
+        in_node[f] = (int)nodes.size();
+        for (int k = 0; k < F.n_params; ++k) root.param.push_back(Val(add(RDF_NODE_IN, -1, f, 0, 0, k), 0));
+        std::map<std::pair<int, int>, Val> memo;
+        std::map<int, uint32_t> used;
+        int next_ctx = 1;
+        std::function<Val(int, const Ctx&)> build = [&](int e, const Ctx& c) -> Val {
+            auto key = std::make_pair(e, c.id);
+            auto it = memo.find(key);
+            if (it != memo.end()) return it->second;
+            const rdf_expr& x = F.exprs[e];
+            Val v;
+            if (x.op == RDF_OP_PARAM) {
+                v = c.param[x.imm];
+            } else if (x.op == RDF_OP_CONST) {
+                v = Val(add(RDF_NODE_CONST, -1, f, 0, x.imm), 0);
+            } else if (x.op == RDF_OP_IF) {
+                // Figure 2: the predicate drives a Switch that routes the parameter to one side
+                Val pred = build(x.a, c);
+                uint32_t m = params_used(f, x.b, used) | params_used(f, x.c, used);
+                Ctx ct{next_ctx++, c.param}, cf{next_ctx++, c.param};
+                for (int k = 0; k < F.n_params; ++k) {
+                    if (!(m >> k & 1)) continue;
+                    int sw = add(RDF_NODE_SWITCH, -1, f, 2);
+                    connect(pred.first, pred.second, sw, 0);
+                    connect(c.param[k].first, c.param[k].second, sw, 1);
+                    ct.param[k] = Val(sw, 0);
+                    cf.param[k] = Val(sw, 1);
+                }
+                Val a = build(x.b, ct), b = build(x.c, cf);
+                // a side that reads no parameter (a bare constant) would fire under every
+                // tag; route its value through a Switch so that only the chosen side is live
+                if (params_used(f, x.b, used) == 0) {
+                    int sw = add(RDF_NODE_SWITCH, -1, f, 2);
+                    connect(pred.first, pred.second, sw, 0);
+                    connect(a.first, a.second, sw, 1);
+                    a = Val(sw, 0);
+                }
+                if (params_used(f, x.c, used) == 0) {
+                    int sw = add(RDF_NODE_SWITCH, -1, f, 2);
+                    connect(pred.first, pred.second, sw, 0);
+                    connect(b.first, b.second, sw, 1);
+                    b = Val(sw, 1);
+                }
+                int mg = add(RDF_NODE_MERGE, -1, f, 2);
+                connect(a.first, a.second, mg, 0);
+                connect(b.first, b.second, mg, 1);
+                v = Val(mg, 0);
+            } else if (x.op == RDF_OP_CALL) {
+                Val a = build(x.a, c);
+                int n = add(NODE_FCALL, -1, f, 1);
+                callee[n] = x.imm;
+                connect(a.first, a.second, n, 0);
+                v = Val(n, 0);
+            } else {
+                int ar = arity_of(x.op);
+                int ops[3] = {x.a, x.b, x.c};
+                Val in[3];
+                for (int k = 0; k < ar; ++k) in[k] = build(ops[k], c);
+                int n = add(RDF_NODE_OP, x.op, f, ar);
+                for (int k = 0; k < ar; ++k) connect(in[k].first, in[k].second, n, k);
+                v = Val(n, 0);
+            }
+            memo[key] = v;
+            return v;
+        };
+        Val r = build(F.root, root);
+        out_node[f] = add(RDF_NODE_OUT, -1, f, 1);
+        connect(r.first, r.second, out_node[f], 0);
+    }
+
+    // The five steps of the general algorithm, per callee f.
+    void transform() {
+        const int nf = P.p->n_functions;
+        std::set<int> removed;
+        for (int f = 0; f < nf; ++f) {
+            if (f == P.p->result) continue;
+            const int m = P.fn(f).n_params;
+            // 1. number the nodes that call f: 0 .. n-1 (callers in `result` first)
+            std::vector<int> calls;
+            for (int n = 0; n < (int)nodes.size(); ++n)
+                if (nodes[n].kind == NODE_FCALL && callee[n] == f) calls.push_back(n);
+            std::stable_sort(calls.begin(), calls.end(), [&](int a, int b) {
+                return (nodes[a].func == P.p->result) > (nodes[b].func == P.p->result);
+            });
+            const int n_calls = (int)calls.size();
+            if (n_calls == 0) continue;
+            // 3. input nodes become Merge nodes with one input per call site
+            for (int k = 0; k < m; ++k) {
+                rdf_node& in = nodes[in_node[f] + k];
+                in.kind = RDF_NODE_ENTRY_MERGE;
+                in.n_in = n_calls;
+            }
+            // the edge into f's output node
+            rdf_edge out_edge{};
+            for (const rdf_edge& e : edges)
+                if (e.dst == out_node[f]) out_edge = e;
+            removed.insert(out_node[f]);
+            for (int i = 0; i < n_calls; ++i) {
+                const int c = calls[i];
+                // 2. m Call_i nodes, one per formal parameter, each with its one input
+                std::vector<int> call_nodes;
+                for (int k = 0; k < m; ++k) {
+                    rdf_edge arg{};
+                    for (const rdf_edge& e : edges)
+                        if (e.dst == c && e.dst_port == k) arg = e;
+                    int cn = add(RDF_NODE_CALL, -1, nodes[c].func, 1, 0, k);
+                    nodes[cn].label = i;
+                    callee[cn] = f;
+                    connect(arg.src, arg.src_port, cn, 0);
+                    connect(cn, 0, in_node[f] + k, i);
+                    call_nodes.push_back(cn);
+                }
+                // 4. Return_i after f's output, feeding the consumers of call node i
+                int rn = add(RDF_NODE_RETURN, -1, nodes[c].func, 1);
+                nodes[rn].label = i;
+                callee[rn] = f;
+                connect(out_edge.src, out_edge.src_port, rn, 0);
+                const size_t n_edges = edges.size();
+                for (size_t j = 0; j < n_edges; ++j)
+                    if (edges[j].src == c) connect(rn, 0, edges[j].dst, edges[j].dst_port, edges[j].control);
+                // 5. control edge Call_i -> Return_i
+                for (int cn : call_nodes) connect(cn, 0, rn, -1, 1);
+                removed.insert(c);
+            }
+            // Figure 3: constants of a called function fire on its entry Merge
+            for (int n = 0; n < (int)nodes.size(); ++n)
+                if (nodes[n].kind == RDF_NODE_CONST && nodes[n].func == f) connect(in_node[f], 0, n, -1, 1);
+        }
+        // drop replaced nodes, renumber
+        std::vector<int> new_id(nodes.size(), -1);
+        std::vector<rdf_node> keep;
+        for (int n = 0; n < (int)nodes.size(); ++n)
+            if (!removed.count(n)) {
+                new_id[n] = (int)keep.size();
+                keep.push_back(nodes[n]);
+            }
+        std::vector<rdf_edge> kept;
+        for (const rdf_edge& e : edges)
+            if (new_id[e.src] >= 0 && new_id[e.dst] >= 0)
+                kept.push_back(rdf_edge{new_id[e.src], e.src_port, new_id[e.dst], e.dst_port, e.control});
+        nodes.swap(keep);
+        edges.swap(kept);
+    }
+};
+
+void build_literal(const Prog& P, rdf_graph* g) {
+    Literal L{P, g->nodes, g->edges, {}, {}, {}};
+    const int nf = P.p->n_functions;
+    L.in_node.assign(nf, -1);
+    L.out_node.assign(nf, -1);
+    L.build_function(P.p->result);          // `result` first, as the paper draws it
+    for (int f = 0; f < nf; ++f)
+        if (f != P.p->result) L.build_function(f);
+    L.transform();
+}
+
+// ------------------------------------------------------------------ lowering
+struct Seg {
+    std::vector<VmInstr> code;
+    int nregs = 0;
+    std::map<int, int> memo;     // expression -> register (only valid in an entry segment)
+    bool entry = false;
+    int base = -1;               // absolute pc after layout
+};
+
+struct Cont {
+    int kind;                    // 0 RET, 1 OUT, 2 PORT, 3 CODE
+    int node = 0, port = 0;
+    std::function<void(int seg, int reg)> fn;
+};
+
+struct Lower {
+    const Prog& P;
+    rdf_graph* g;
+    std::vector<Seg> segs;
+    std::vector<int> entry_seg;          // per function
+    std::vector<int> label_entry_seg;    // per label: callee's entry segment
+    std::vector<int> label_kseg;         // per label: continuation segment (K_SEG) or -1
+    std::vector<int> match_cont_seg;     // per match node
+    std::vector<int> local_count;        // per callee: call sites numbered so far
+    int cur_func = 0;
+    int calls_in_body = 0;
+
+    int new_seg() {
+        segs.emplace_back();
+        return (int)segs.size() - 1;
+    }
+    int reg(int s) {
+        require(segs[s].nregs < RDF_MAX_REGS, RDF_ERR_UNSUPPORTED);
+        return segs[s].nregs++;
+    }
+    void emit(int s, uint8_t op, int dst = 0, int a = 0, int b = 0, int32_t imm = 0) {
+        segs[s].code.push_back(VmInstr{op, (uint8_t)dst, (uint8_t)a, (uint8_t)b, imm});
+    }
+
+    bool call_free(int f, int e) {
+        const rdf_expr& x = P.ex(f, e);
+        switch (x.op) {
+            case RDF_OP_CALL: case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CELL_RNN:
+            case RDF_OP_CELL_LSTM: case RDF_OP_NODE_LOSS: return false;
+            default: break;
+        }
+        int ops[3] = {x.a, x.b, x.c};
+        for (int k = 0; k < arity_of(x.op); ++k)
+            if (!call_free(f, ops[k])) return false;
+        return true;
+    }
+
+    int load_const(int s, int64_t v) {
+        int r = reg(s);
+        if (v >= INT32_MIN && v <= INT32_MAX) {
+            emit(s, VM_MOVI, r, 0, 0, (int32_t)v);
+        } else {
+            require((int)g->consts.size() < RDF_MAX_CONSTS, RDF_ERR_UNSUPPORTED);
+            g->consts.push_back(v);
+            emit(s, VM_MOVC, r, 0, 0, (int32_t)g->consts.size() - 1);
+        }
+        return r;
+    }
+
+    uint8_t vm_binop(int op) {
+        switch (op) {
+            case RDF_OP_ADD: return VM_ADD; case RDF_OP_SUB: return VM_SUB; case RDF_OP_MUL: return VM_MUL;
+            case RDF_OP_MAX: return VM_MAX; case RDF_OP_LT: return VM_LT; case RDF_OP_EQ: return VM_EQ;
+        }
+        throw Err{RDF_ERR_UNSUPPORTED};
+    }
+
+    // value of a call-free expression, computed where the parameters are live
+    int value(int s, int e) {
+        require(segs[s].entry, RDF_ERR_UNSUPPORTED);   // parameters are in registers only in an entry segment
+        auto it = segs[s].memo.find(e);
+        if (it != segs[s].memo.end()) return it->second;
+        const rdf_expr& x = P.ex(cur_func, e);
+        int r;
+        switch (x.op) {
+            case RDF_OP_PARAM: r = (int)x.imm; break;
+            case RDF_OP_CONST: r = load_const(s, x.imm); break;
+            case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK: {
+                int a = value(s, x.a);
+                r = reg(s);
+                g->uses_tree = true;
+                emit(s, x.op == RDF_OP_IS_LEAF ? VM_ISLEAF : x.op == RDF_OP_LEFT ? VM_LEFT
+                        : x.op == RDF_OP_RIGHT ? VM_RIGHT : VM_TOK, r, a);
+                break;
+            }
+            case RDF_OP_IF: {
+                // both sides call-free: an ordinary branch that joins
+                int c = value(s, x.a);
+                r = reg(s);
+                std::map<int, int> saved = segs[s].memo;   // values computed in one arm are not live in the other
+                size_t brz = segs[s].code.size();
+                emit(s, VM_BRZ, 0, c);
+                int a = value(s, x.b);
+                emit(s, VM_MOV, r, a);
+                size_t jmp = segs[s].code.size();
+                emit(s, VM_JMP);
+                segs[s].memo = saved;
+                segs[s].code[brz].imm = (int32_t)segs[s].code.size();
+                int b = value(s, x.c);
+                emit(s, VM_MOV, r, b);
+                segs[s].code[jmp].imm = (int32_t)segs[s].code.size();
+                segs[s].memo = saved;
+                break;
+            }
+            default: {
+                int a = value(s, x.a), b = value(s, x.b);
+                r = reg(s);
+                emit(s, vm_binop(x.op), r, a, b);
+            }
+        }
+        segs[s].memo[e] = r;
+        return r;
+    }
+
+    void apply(const Cont& K, int s, int r) {
+        switch (K.kind) {
+            case 0: emit(s, VM_RET, 0, r); break;
+            case 1: emit(s, VM_OUT, 0, r); break;
+            case 2: emit(s, VM_PORT, 0, r, K.port, K.node); break;
+            default: K.fn(s, r);
+        }
+    }
+
+    // a fresh segment that receives one value in r0 and hands it to K
+    int cont_segment(const Cont& K) {
+        int s = new_seg();
+        int r0 = reg(s);
+        apply(K, s, r0);
+        emit(s, VM_HALT);
+        return s;
+    }
+
+    int new_label(int callee, const Cont& K) {
+        require((int)g->labels.size() < RDF_MAX_LABELS, RDF_ERR_UNSUPPORTED);
+        LabelInfo L{};
+        L.callee = callee;
+        L.local_label = local_count[callee]++;
+        L.child_index = calls_in_body++;
+        int kseg = -1;
+        if (K.kind == 2) {
+            L.k_kind = K_PORT; L.k_node = K.node; L.k_port = K.port;
+        } else if (K.kind == 0) {
+            L.k_kind = K_RET;
+        } else {
+            L.k_kind = K_SEG;
+            kseg = cont_segment(K);
+        }
+        g->labels.push_back(L);
+        label_entry_seg.push_back(entry_seg[callee]);
+        label_kseg.push_back(kseg);
+        return (int)g->labels.size() - 1;
+    }
+
+    int new_match(int n_ports, int kind, int cont_seg) {
+        require((int)g->match.size() < RDF_MAX_MATCH, RDF_ERR_UNSUPPORTED);
+        MatchNode M{n_ports, kind, 0, g->n_ports_total};
+        g->n_ports_total += n_ports;
+        g->match.push_back(M);
+        match_cont_seg.push_back(cont_seg);
+        return (int)g->match.size() - 1;
+    }
+
+    // start the evaluation of expression e in segment s; its value goes to K
+    void cps(int s, int e, const Cont& K) {
+        const int f = cur_func;
+        if (call_free(f, e)) {
+            apply(K, s, value(s, e));
+            return;
+        }
+        const rdf_expr& x = P.ex(f, e);
+        switch (x.op) {
+            case RDF_OP_CALL: {
+                const int callee = (int)x.imm;
+                if (call_free(f, x.a)) {
+                    int r = value(s, x.a);
+                    int label = new_label(callee, K);
+                    emit(s, VM_CALL, 0, r, 0, label);
+                } else {
+                    Cont K2{3};
+                    K2.fn = [this, callee, K](int s2, int r) {
+                        int label = new_label(callee, K);
+                        emit(s2, VM_CALL, 0, r, 0, label);
+                    };
+                    cps(s, x.a, K2);
+                }
+                break;
+            }
+            case RDF_OP_IF: {
+                require(call_free(f, x.a), RDF_ERR_UNSUPPORTED);
+                int c = value(s, x.a);
+                std::map<int, int> saved = segs[s].memo;
+                size_t brz = segs[s].code.size();
+                emit(s, VM_BRZ, 0, c);
+                cps(s, x.b, K);
+                size_t jmp = segs[s].code.size();
+                emit(s, VM_JMP);
+                segs[s].memo = saved;
+                segs[s].code[brz].imm = (int32_t)segs[s].code.size();
+                cps(s, x.c, K);
+                segs[s].code[jmp].imm = (int32_t)segs[s].code.size();
+                segs[s].memo = saved;
+                break;
+            }
+            case RDF_OP_NODE_LOSS: {
+                // identity on the state; the invocation's node index must be the parameter
+                require(P.ex(f, x.b).op == RDF_OP_PARAM, RDF_ERR_UNSUPPORTED);
+                g->has_loss = true;
+                cps(s, x.a, K);
+                break;
+            }
+            case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: {
+                require(call_free(f, x.a), RDF_ERR_UNSUPPORTED);
+                g->has_vector_ops = true;
+                (x.op == RDF_OP_EMBED ? g->has_rnn : g->has_lstm) = true;
+                int r = value(s, x.a);
+                int ks = cont_segment(K);
+                emit(s, x.op == RDF_OP_EMBED ? VM_EMBED : VM_LEAF_LSTM, 0, r, 0, -(ks + 1));   // fixed up at layout
+                break;
+            }
+            case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM: {
+                g->has_vector_ops = true;
+                (x.op == RDF_OP_CELL_RNN ? g->has_rnn : g->has_lstm) = true;
+                int ks = cont_segment(K);
+                int M = new_match(2, x.op == RDF_OP_CELL_RNN ? MATCH_CELL_RNN : MATCH_CELL_LSTM, ks);
+                Cont Ka{2, M, 0}, Kb{2, M, 1};
+                cps(s, x.a, Ka);
+                cps(s, x.b, Kb);
+                break;
+            }
+            default: {
+                // integer operator with at least one operand that depends on a call
+                const int ops[2] = {x.a, x.b};
+                const uint8_t vop = vm_binop(x.op);
+                bool dyn[2];
+                int n_dyn = 0;
+                for (int k = 0; k < 2; ++k) {
+                    dyn[k] = P.ex(f, ops[k]).op != RDF_OP_CONST;
+                    n_dyn += dyn[k];
+                }
+                if (n_dyn == 1) {
+                    // one tagged input: no match needed, the operator runs when that input arrives
+                    const int kd = dyn[0] ? 0 : 1;
+                    const int64_t cv = P.ex(f, ops[1 - kd]).imm;
+                    Cont K2{3};
+                    K2.fn = [this, vop, kd, cv, K](int s2, int r) {
+                        int c = load_const(s2, cv);
+                        int d = reg(s2);
+                        emit(s2, vop, d, kd == 0 ? r : c, kd == 0 ? c : r);
+                        apply(K, s2, d);
+                    };
+                    cps(s, ops[kd], K2);
+                } else {
+                    // two tagged inputs meet in the token store; the continuation gets them as r0, r1
+                    int ks = new_seg();
+                    int r0 = reg(ks), r1 = reg(ks), d = reg(ks);
+                    emit(ks, vop, d, r0, r1);
+                    apply(K, ks, d);
+                    emit(ks, VM_HALT);
+                    int M = new_match(2, MATCH_INT, ks);
+                    Cont Ka{2, M, 0}, Kb{2, M, 1};
+                    cps(s, x.a, Ka);
+                    cps(s, x.b, Kb);
+                }
+            }
+        }
+    }
+
+    void run() {
+        const int nf = P.p->n_functions;
+        entry_seg.assign(nf, -1);
+        local_count.assign(nf, 0);
+        for (int f = 0; f < nf; ++f) {
+            entry_seg[f] = new_seg();
+            segs[entry_seg[f]].entry = true;
+            segs[entry_seg[f]].nregs = std::max(1, P.fn(f).n_params);
+        }
+        std::vector<int> order{P.p->result};
+        for (int f = 0; f < nf; ++f)
+            if (f != P.p->result) order.push_back(f);
+        for (int f : order) {
+            cur_func = f;
+            calls_in_body = 0;
+            Cont K{f == P.p->result ? 1 : 0};
+            cps(entry_seg[f], P.fn(f).root, K);
+            emit(entry_seg[f], VM_HALT);
+            g->max_calls_per_body = std::max(g->max_calls_per_body, calls_in_body);
+        }
+        // layout: concatenate segments, make jump targets absolute
+        int pc = 0;
+        for (Seg& S : segs) {
+            S.base = pc;
+            pc += (int)S.code.size();
+        }
+        require(pc <= RDF_MAX_CODE, RDF_ERR_UNSUPPORTED);
+        for (Seg& S : segs)
+            for (VmInstr in : S.code) {
+                if (in.op == VM_BRZ || in.op == VM_JMP) in.imm += S.base;
+                if (in.op == VM_EMBED || in.op == VM_LEAF_LSTM) in.imm = segs[-in.imm - 1].base;
+                g->code.push_back(in);
+            }
+        for (size_t i = 0; i < g->labels.size(); ++i) {
+            g->labels[i].entry_pc = segs[label_entry_seg[i]].base;
+            if (label_kseg[i] >= 0) g->labels[i].k_pc = segs[label_kseg[i]].base;
+        }
+        for (size_t i = 0; i < g->match.size(); ++i) g->match[i].cont_pc = segs[match_cont_seg[i]].base;
+        g->result_entry_pc = segs[entry_seg[P.p->result]].base;
+        int bits = 1;
+        while ((1 << bits) < (int)g->labels.size()) ++bits;
+        g->label_bits = bits;
+        if (g->has_vector_ops) require(P.p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);
+        require(!(g->has_rnn && g->has_lstm), RDF_ERR_UNSUPPORTED);
+    }
+};
+
+}  // namespace
+
+extern "C" int rdf_graph_build(const rdf_program* prog, rdf_graph** out_graph) {
+    if (!prog || !out_graph) return RDF_ERR_BAD_ARG;
+    *out_graph = nullptr;
+    rdf_graph* g = new rdf_graph();
+    try {
+        Prog P{prog};
+        validate(P);
+        g->tag_mode = prog->tag_mode;
+        for (int f = 0; f < prog->n_functions; ++f) g->func_names.push_back(prog->functions[f].name);
+        build_literal(P, g);
+        Lower L{P, g};
+        L.run();
+    } catch (const Err& e) {
+        delete g;
+        return e.code;
+    } catch (...) {
+        delete g;
+        return RDF_ERR_BAD_PROGRAM;
+    }
+    *out_graph = g;
+    return RDF_OK;
+}
+
+extern "C" void rdf_graph_free(rdf_graph* g) {
+    if (!g) return;
+    rdf_exec_release(g);
+    delete g;
+}
+
+extern "C" int rdf_graph_describe(const rdf_graph* g, rdf_graph_desc* out) {
+    if (!g || !out) return RDF_ERR_BAD_ARG;
+    out->n_nodes = (int32_t)g->nodes.size();
+    out->n_edges = (int32_t)g->edges.size();
+    out->nodes = g->nodes.data();
+    out->edges = g->edges.data();
+    out->n_labels = (int32_t)g->labels.size();
+    out->label_bits = g->label_bits;
+    out->n_match = (int32_t)g->match.size();
+    out->n_code = (int32_t)g->code.size();
+    return RDF_OK;
+}
+
+extern "C" const char* rdf_strerror(int status) {
+    switch (status) {
+        case RDF_OK: return "ok";
+        case RDF_ERR_BAD_PROGRAM: return "malformed program";
+        case RDF_ERR_BAD_ARG: return "bad argument";
+        case RDF_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case RDF_ERR_TAG_OVERFLOW: return "call depth exceeds the packed tag";
+        case RDF_ERR_STORE_FULL: return "token store full";
+        case RDF_ERR_FRAMES_FULL: return "more invocations than max_invocations";
+        case RDF_ERR_QUEUE_FULL: return "wave queue full";
+        case RDF_ERR_WAVE_LIMIT: return "wave limit reached (recursion without base case?)";
+        case RDF_ERR_TIMEOUT: return "bounded device wait expired";
+        case RDF_ERR_CUDA: return "CUDA runtime error";
+        case RDF_ERR_UNSUPPORTED: return "program not supported by the device executor";
+        default: return "unknown status";
+    }
+}
