@@ -1,0 +1,416 @@
+"""ctypes binding of the C boundary declared in include/rdf.h.
+
+Argument marshalling only: every step of the path (tag push/pop, token
+matching, wave scheduling, cells, gradients) runs in the CUDA library.  torch
+is used for device memory and streams.  There is no CPU fallback: a missing
+library or a missing GPU is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+# ---------------------------------------------------------------- constants
+RDF_OK = 0
+ERRORS = {
+    -1: "RDF_ERR_BAD_PROGRAM", -2: "RDF_ERR_BAD_ARG", -3: "RDF_ERR_WORKSPACE_TOO_SMALL", -4: "RDF_ERR_TAG_OVERFLOW",
+    -5: "RDF_ERR_STORE_FULL", -6: "RDF_ERR_FRAMES_FULL", -7: "RDF_ERR_QUEUE_FULL", -8: "RDF_ERR_WAVE_LIMIT",
+    -9: "RDF_ERR_TIMEOUT", -10: "RDF_ERR_CUDA", -11: "RDF_ERR_UNSUPPORTED",
+}
+(OP_PARAM, OP_CONST, OP_ADD, OP_SUB, OP_MUL, OP_MAX, OP_LT, OP_EQ, OP_IF, OP_CALL, OP_IS_LEAF, OP_LEFT, OP_RIGHT,
+ OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS) = range(19)
+TAGS_PATH, TAGS_FRAME = 0, 1
+F32, BF16 = 0, 1
+(NODE_IN, NODE_OUT, NODE_CONST, NODE_OP, NODE_SWITCH, NODE_MERGE, NODE_ENTRY_MERGE, NODE_CALL, NODE_RETURN) = range(9)
+
+PATH_BITS, DEPTH_SHIFT, INST_SHIFT = 38, 38, 44
+
+
+class RdfError(RuntimeError):
+    def __init__(self, code, where=""):
+        self.code = code
+        super().__init__(f"{where}: {ERRORS.get(code, code)}")
+
+
+# ------------------------------------------------------------------ structs
+class rdf_expr(C.Structure):
+    _fields_ = [("op", C.c_int32), ("a", C.c_int32), ("b", C.c_int32), ("c", C.c_int32), ("imm", C.c_int64)]
+
+
+class rdf_function(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("n_params", C.c_int32), ("n_exprs", C.c_int32),
+                ("exprs", C.POINTER(rdf_expr)), ("root", C.c_int32)]
+
+
+class rdf_program(C.Structure):
+    _fields_ = [("n_functions", C.c_int32), ("functions", C.POINTER(rdf_function)), ("result", C.c_int32),
+                ("tag_mode", C.c_int32)]
+
+
+class rdf_node(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("op", C.c_int32), ("label", C.c_int32), ("func", C.c_int32),
+                ("param", C.c_int32), ("n_in", C.c_int32), ("value", C.c_int64)]
+
+
+class rdf_edge(C.Structure):
+    _fields_ = [("src", C.c_int32), ("src_port", C.c_int32), ("dst", C.c_int32), ("dst_port", C.c_int32),
+                ("control", C.c_int32)]
+
+
+class rdf_graph_desc(C.Structure):
+    _fields_ = [("n_nodes", C.c_int32), ("n_edges", C.c_int32), ("nodes", C.POINTER(rdf_node)),
+                ("edges", C.POINTER(rdf_edge)), ("n_labels", C.c_int32), ("label_bits", C.c_int32),
+                ("n_match", C.c_int32), ("n_code", C.c_int32)]
+
+
+class rdf_batch(C.Structure):
+    _fields_ = [("B", C.c_int64), ("x", C.c_void_p), ("tree_root", C.c_void_p), ("N", C.c_int64),
+                ("left", C.c_void_p), ("right", C.c_void_p), ("tok", C.c_void_p), ("label", C.c_void_p),
+                ("max_invocations", C.c_int64), ("max_wave_tokens", C.c_int64)]
+
+
+class rdf_params(C.Structure):
+    _fields_ = [("compute", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("V", C.c_int32),
+                ("n_classes", C.c_int32), ("E", C.c_void_p), ("W", C.c_void_p), ("b", C.c_void_p),
+                ("W_x", C.c_void_p), ("b_x", C.c_void_p), ("W_s", C.c_void_p), ("b_s", C.c_void_p)]
+
+
+class rdf_trace_rec(C.Structure):
+    _fields_ = [("tag", C.c_uint64), ("value", C.c_int64), ("kind", C.c_uint32), ("label", C.c_uint32),
+                ("parent", C.c_uint32), ("instance", C.c_uint32)]
+
+
+TRACE_DTYPE = np.dtype([("tag", "<u8"), ("value", "<i8"), ("kind", "<u4"), ("label", "<u4"), ("parent", "<u4"),
+                        ("instance", "<u4")])
+
+
+class rdf_outputs(C.Structure):
+    _fields_ = [("y", C.c_void_p), ("h_root", C.c_void_p), ("loss", C.c_void_p), ("trace", C.c_void_p),
+                ("trace_capacity", C.c_int64), ("trace_count", C.c_void_p)]
+
+
+class rdf_param_grads(C.Structure):
+    _fields_ = [("dE", C.c_void_p), ("dW", C.c_void_p), ("db", C.c_void_p), ("dW_x", C.c_void_p),
+                ("db_x", C.c_void_p), ("dW_s", C.c_void_p), ("db_s", C.c_void_p)]
+
+
+class rdf_stats(C.Structure):
+    _fields_ = [("status", C.c_int32), ("waves", C.c_uint32), ("waves_backward", C.c_uint32),
+                ("max_wave_tokens", C.c_uint32), ("invocations", C.c_uint64), ("tokens", C.c_uint64),
+                ("store_inserts", C.c_uint64), ("store_matches", C.c_uint64), ("store_probes", C.c_uint64),
+                ("max_probe", C.c_uint32), ("max_depth", C.c_uint32), ("cells", C.c_uint64), ("leaves", C.c_uint64)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
+           "rdf_last_status", "rdf_strerror"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads (building first if the sources are newer) the CUDA library."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        L.rdf_graph_build.argtypes = [C.POINTER(rdf_program), C.POINTER(C.c_void_p)]
+        L.rdf_graph_free.argtypes = [C.c_void_p]
+        L.rdf_graph_free.restype = None
+        L.rdf_graph_describe.argtypes = [C.c_void_p, C.POINTER(rdf_graph_desc)]
+        L.rdf_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params), C.c_int,
+                                          C.POINTER(C.c_size_t)]
+        L.rdf_eval.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params), C.POINTER(rdf_outputs),
+                               C.c_void_p, C.c_size_t, C.c_void_p]
+        L.rdf_grad.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params), C.POINTER(rdf_outputs),
+                               C.POINTER(rdf_param_grads), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
+        L.rdf_strerror.argtypes = [C.c_int]
+        L.rdf_strerror.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+# ------------------------------------------------------- program description
+class Function:
+    """One definition as an expression list; methods return expression indices."""
+
+    def __init__(self, name: str, n_params: int):
+        self.name, self.n_params, self.exprs, self.root = name, n_params, [], -1
+
+    def _add(self, op, a=-1, b=-1, c=-1, imm=0):
+        self.exprs.append((op, a, b, c, imm))
+        return len(self.exprs) - 1
+
+    def param(self, k=0): return self._add(OP_PARAM, imm=k)
+    def const(self, v): return self._add(OP_CONST, imm=int(v))
+    def add(self, a, b): return self._add(OP_ADD, a, b)
+    def sub(self, a, b): return self._add(OP_SUB, a, b)
+    def mul(self, a, b): return self._add(OP_MUL, a, b)
+    def max(self, a, b): return self._add(OP_MAX, a, b)
+    def lt(self, a, b): return self._add(OP_LT, a, b)
+    def eq(self, a, b): return self._add(OP_EQ, a, b)
+    def if_(self, c, a, b): return self._add(OP_IF, c, a, b)
+    def call(self, f_index, arg): return self._add(OP_CALL, arg, imm=f_index)
+    def is_leaf(self, v): return self._add(OP_IS_LEAF, v)
+    def left(self, v): return self._add(OP_LEFT, v)
+    def right(self, v): return self._add(OP_RIGHT, v)
+    def tok(self, v): return self._add(OP_TOK, v)
+    def embed(self, t): return self._add(OP_EMBED, t)
+    def cell_rnn(self, a, b): return self._add(OP_CELL_RNN, a, b)
+    def leaf_lstm(self, t): return self._add(OP_LEAF_LSTM, t)
+    def cell_lstm(self, a, b): return self._add(OP_CELL_LSTM, a, b)
+    def node_loss(self, s, v): return self._add(OP_NODE_LOSS, s, v)
+
+    def ret(self, e):
+        self.root = e
+        return self
+
+
+def fact_program(arg=3, addend=5):
+    """result = addend + fact(arg); fact(n) = if 1 == n then n else n * fact(n-1)."""
+    r = Function("result", 0)
+    r.ret(r.add(r.const(addend), r.call(1, r.const(arg))))
+    f = Function("fact", 1)
+    n = f.param()
+    f.ret(f.if_(f.eq(f.const(1), n), n, f.mul(n, f.call(1, f.sub(n, f.const(1))))))
+    return [r, f], 0
+
+
+def fib_program():
+    """result(x) = fib(x); fib(n) = if n < 2 then n else fib(n-1) + fib(n-2)."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.param()))
+    f = Function("fib", 1)
+    n = f.param()
+    f.ret(f.if_(f.lt(n, f.const(2)), n, f.add(f.call(1, f.sub(n, f.const(1))), f.call(1, f.sub(n, f.const(2))))))
+    return [r, f], 0
+
+
+def tree_fold_program(kind: str):
+    """Integer folds over the input trees: 'sum' of leaf tokens, leaf 'count', 'height'."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.param()))
+    f = Function("fold", 1)
+    v = f.param()
+    a, b = f.call(1, f.left(v)), f.call(1, f.right(v))
+    if kind == "sum":
+        leaf, comb = f.tok(v), f.add(a, b)
+    elif kind == "count":
+        leaf, comb = f.const(1), f.add(a, b)
+    else:
+        leaf, comb = f.const(0), f.add(f.max(a, b), f.const(1))
+    f.ret(f.if_(f.is_leaf(v), leaf, comb))
+    return [r, f], 0
+
+
+def tree_net_program(cell: str = "rnn", with_loss: bool = False):
+    """h(v) = leaf(tok v) if is_leaf(v) else cell(h(left v), h(right v)), optionally under the per-node loss."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.param()))
+    f = Function("h", 1)
+    v = f.param()
+    if cell == "rnn":
+        body = f.if_(f.is_leaf(v), f.embed(f.tok(v)), f.cell_rnn(f.call(1, f.left(v)), f.call(1, f.right(v))))
+    else:
+        body = f.if_(f.is_leaf(v), f.leaf_lstm(f.tok(v)), f.cell_lstm(f.call(1, f.left(v)), f.call(1, f.right(v))))
+    f.ret(f.node_loss(body, v) if with_loss else body)
+    return [r, f], 0
+
+
+# -------------------------------------------------------------------- graph
+def _torch():
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("the recursive-dataflow library needs a CUDA device; there is no CPU path")
+    return torch
+
+
+class Graph:
+    """A program transformed into one static graph and lowered for the device."""
+
+    def __init__(self, functions, result=0, tag_mode=TAGS_PATH):
+        self._keep = []
+        fs = (rdf_function * len(functions))()
+        for i, f in enumerate(functions):
+            ex = (rdf_expr * max(1, len(f.exprs)))(*[rdf_expr(*e) for e in f.exprs])
+            self._keep.append(ex)
+            fs[i] = rdf_function(f.name.encode(), f.n_params, len(f.exprs), ex, f.root)
+        prog = rdf_program(len(functions), fs, result, tag_mode)
+        self.handle = C.c_void_p()
+        self.tag_mode = tag_mode
+        self._ws = None
+        rc = lib().rdf_graph_build(C.byref(prog), C.byref(self.handle))
+        if rc != RDF_OK:
+            self.handle = None
+            raise RdfError(rc, "rdf_graph_build")
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            lib().rdf_graph_free(self.handle)
+            self.handle = None
+
+    def describe(self):
+        d = rdf_graph_desc()
+        rc = lib().rdf_graph_describe(self.handle, C.byref(d))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_graph_describe")
+        nodes = [{k: getattr(d.nodes[i], k) for k, _ in rdf_node._fields_} for i in range(d.n_nodes)]
+        edges = [{k: getattr(d.edges[i], k) for k, _ in rdf_edge._fields_} for i in range(d.n_edges)]
+        return {"nodes": nodes, "edges": edges, "n_labels": d.n_labels, "label_bits": d.label_bits,
+                "n_match": d.n_match, "n_code": d.n_code}
+
+    # ---- workspace (torch owns the memory)
+    def workspace_bytes(self, batch, params, want_grad):
+        n = C.c_size_t()
+        rc = lib().rdf_workspace_bytes(self.handle, C.byref(batch), C.byref(params) if params else None, want_grad,
+                                       C.byref(n))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_workspace_bytes")
+        return n.value
+
+    def _workspace(self, batch, params, want_grad):
+        torch = _torch()
+        n = self.workspace_bytes(batch, params, want_grad)
+        if self._ws is None or self._ws.numel() < n + 256:
+            self._ws = None
+            self._ws = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
+        off = (-self._ws.data_ptr()) % 256
+        return self._ws.data_ptr() + off, n
+
+    def stats(self, check=True):
+        s = rdf_stats()
+        rc = lib().rdf_last_status(self.handle, C.byref(s))
+        if check and rc != RDF_OK:
+            raise RdfError(rc, "device status")
+        return s.as_dict()
+
+    def _outputs(self, trace_capacity, **ptrs):
+        torch = _torch()
+        out = rdf_outputs()
+        keep = None
+        for k, v in ptrs.items():
+            setattr(out, k, v.data_ptr() if v is not None else None)
+        if trace_capacity:
+            buf = torch.empty(trace_capacity * 32, dtype=torch.uint8, device="cuda")
+            cnt = torch.zeros(1, dtype=torch.int64, device="cuda")
+            out.trace, out.trace_capacity, out.trace_count = buf.data_ptr(), trace_capacity, cnt.data_ptr()
+            keep = (buf, cnt)
+        return out, keep
+
+    @staticmethod
+    def _read_trace(keep):
+        if keep is None:
+            return None
+        buf, cnt = keep
+        n = int(cnt.item())
+        assert n * 32 <= buf.numel(), "trace buffer too small"
+        return buf[: n * 32].cpu().numpy().view(TRACE_DTYPE)
+
+    # ---- integer programs
+    def eval_int(self, x, max_invocations, trace_capacity=0, max_wave_tokens=0, check=True, y=None):
+        """x: int64 CUDA tensor [B].  Returns (y int64 CUDA tensor [B], trace ndarray or None)."""
+        torch = _torch()
+        assert x.is_cuda and x.dtype == torch.int64 and x.is_contiguous()
+        B = x.numel()
+        if y is None:
+            y = torch.empty(B, dtype=torch.int64, device="cuda")
+        batch = rdf_batch(B=B, x=x.data_ptr(), N=0, max_invocations=int(max_invocations),
+                          max_wave_tokens=int(max_wave_tokens))
+        out, tr = self._outputs(trace_capacity, y=y)
+        ws, nbytes = self._workspace(batch, None, 0)
+        rc = lib().rdf_eval(self.handle, C.byref(batch), None, C.byref(out), ws, nbytes,
+                            torch.cuda.current_stream().cuda_stream)
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_eval")
+        if check:
+            self.stats()
+        return y, self._read_trace(tr)
+
+    # ---- tree programs
+    @staticmethod
+    def device_trees(tb):
+        """Uploads a workloads.TreeBatch; returns the dict of int32 CUDA tensors."""
+        torch = _torch()
+        return {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).cuda()
+                for k in ("tree_root", "left", "right", "tok", "label")}
+
+    @staticmethod
+    def device_params(params):
+        torch = _torch()
+        return {k: torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).cuda() for k, v in params.items()}
+
+    @staticmethod
+    def _batch(dt):
+        return rdf_batch(B=dt["tree_root"].numel(), x=None, tree_root=dt["tree_root"].data_ptr(),
+                         N=dt["left"].numel(), left=dt["left"].data_ptr(), right=dt["right"].data_ptr(),
+                         tok=dt["tok"].data_ptr(), label=dt["label"].data_ptr(), max_invocations=dt["left"].numel(),
+                         max_wave_tokens=0)
+
+    @staticmethod
+    def _params(dp, compute):
+        g = lambda k: dp[k].data_ptr() if k in dp else None  # noqa: E731
+        H = dp["W"].shape[1] // 2
+        return rdf_params(compute=compute, H=H, D=dp["E"].shape[1], V=dp["E"].shape[0],
+                          n_classes=dp["W_s"].shape[0] if "W_s" in dp else 0, E=g("E"), W=g("W"), b=g("b"),
+                          W_x=g("W_x"), b_x=g("b_x"), W_s=g("W_s"), b_s=g("b_s"))
+
+    def eval_trees(self, dt, dp, compute=F32, trace_capacity=0, check=True, h_root=None):
+        """Forward pass over a batch of trees.  dt/dp: device_trees()/device_params().
+        For integer tree programs (no parameters) pass dp=None: returns (y, trace)."""
+        torch = _torch()
+        batch = self._batch(dt)
+        B = batch.B
+        if dp is None:
+            y = torch.empty(B, dtype=torch.int64, device="cuda")
+            out, tr = self._outputs(trace_capacity, y=y)
+            params = None
+        else:
+            params = self._params(dp, compute)
+            y = h_root if h_root is not None else torch.empty(B, params.H, dtype=torch.float32, device="cuda")
+            out, tr = self._outputs(trace_capacity, h_root=y)
+        ws, nbytes = self._workspace(batch, params, 0)
+        rc = lib().rdf_eval(self.handle, C.byref(batch), C.byref(params) if params else None, C.byref(out), ws,
+                            nbytes, torch.cuda.current_stream().cuda_stream)
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_eval")
+        if check:
+            self.stats()
+        return y, self._read_trace(tr)
+
+    def grad_trees(self, dt, dp, compute=F32, check=True, grads=None, loss=None, h_root=None):
+        """Forward + reverse pass.  Returns (loss tensor [1], h_root, {name: gradient tensor})."""
+        torch = _torch()
+        batch = self._batch(dt)
+        params = self._params(dp, compute)
+        if h_root is None:
+            h_root = torch.empty(batch.B, params.H, dtype=torch.float32, device="cuda")
+        if loss is None:
+            loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+        if grads is None:
+            grads = {k: torch.empty_like(v) for k, v in dp.items()}
+        pg = rdf_param_grads(**{"d" + k: grads[k].data_ptr() for k in grads})
+        out, _ = self._outputs(0, h_root=h_root, loss=loss)
+        ws, nbytes = self._workspace(batch, params, 1)
+        rc = lib().rdf_grad(self.handle, C.byref(batch), C.byref(params), C.byref(out), C.byref(pg), ws, nbytes,
+                            torch.cuda.current_stream().cuda_stream)
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_grad")
+        if check:
+            self.stats()
+        return loss, h_root, grads
+
+
+# --------------------------------------------------------------- tag decode
+def unpack_path_tag(tag: int, label_bits: int):
+    """(instance, labels innermost first) of a packed 64-bit path tag."""
+    tag = int(tag)
+    inst = tag >> INST_SHIFT
+    depth = (tag >> DEPTH_SHIFT) & 63
+    path = tag & ((1 << PATH_BITS) - 1)
+    return inst, tuple((path >> (label_bits * k)) & ((1 << label_bits) - 1) for k in range(depth))

@@ -1,0 +1,183 @@
+"""Host logic of the library, no GPU: the shared object loads and exports every
+declared symbol; rdf_graph_build validates programs; the literal static graph it
+produces (Section 3 transformation) is executed by the oracle's tagged-token
+interpreter -- graph *data* crosses, no code -- and gives the oracle's results."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import workloads
+import paper_2410_20225_b200 as rdf
+from paper_2410_20225_b200 import binding as bd
+from oracle import direct, programs, tagged, transform
+from oracle.graphs import Graph as OGraph
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = rdf.lib()
+    header = open(os.path.join(ROOT, "include", "rdf.h")).read()
+    declared = set(re.findall(r"^(?:int|void|const char\*)\s+(rdf_[a-z_]+)\s*\(", header, flags=re.M))
+    assert {"rdf_graph_build", "rdf_eval", "rdf_grad", "rdf_graph_free", "rdf_strerror"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.rdf_strerror(-4).decode().startswith("call depth")
+    assert set(bd.EXPORTS) <= declared
+
+
+def test_struct_layouts_match_the_header():
+    assert C.sizeof(bd.rdf_expr) == 24 and C.sizeof(bd.rdf_trace_rec) == 32 and bd.TRACE_DTYPE.itemsize == 32
+    assert C.sizeof(bd.rdf_batch) == 10 * 8 and C.sizeof(bd.rdf_node) == 32 and C.sizeof(bd.rdf_edge) == 20
+
+
+# ----------------------------------------------------------------- errors
+def _build(functions, result=0, mode=rdf.TAGS_PATH):
+    return rdf.Graph(functions, result, mode)
+
+
+def test_bad_programs_are_rejected():
+    f = rdf.Function("result", 1)
+    f.ret(f.call(5, f.param()))                       # unknown callee
+    with pytest.raises(rdf.RdfError) as e:
+        _build([f])
+    assert e.value.code == -1
+    fs, r = rdf.fib_program()
+    fs[1].root = 99                                   # root out of range
+    with pytest.raises(rdf.RdfError):
+        _build(fs, r)
+    fs, r = rdf.fib_program()
+    with pytest.raises(rdf.RdfError):
+        _build(fs, 7)                                 # no such `result`
+    # a cycle among expressions
+    g = rdf.Function("result", 1)
+    g.exprs.append((bd.OP_ADD, 0, 0, -1, 0))
+    g.root = 0
+    with pytest.raises(rdf.RdfError):
+        _build([g])
+    # vector programs need frame tags
+    fs, r = rdf.tree_net_program("rnn")
+    with pytest.raises(rdf.RdfError) as e:
+        _build(fs, r, rdf.TAGS_PATH)
+    assert e.value.code == -11
+    # two-parameter callee: valid by the paper, outside this executor
+    a = rdf.Function("result", 1)
+    a.ret(a.call(1, a.param()))
+    b = rdf.Function("g", 2)
+    b.ret(b.param(0))
+    with pytest.raises(rdf.RdfError) as e:
+        _build([a, b])
+    assert e.value.code == -11
+
+
+# ---------------------------------------- literal graph through the oracle
+OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.OP_LT: "<", bd.OP_EQ: "==",
+          bd.OP_IS_LEAF: "is_leaf", bd.OP_LEFT: "left", bd.OP_RIGHT: "right", bd.OP_TOK: "tok",
+          bd.OP_EMBED: "leaf_rnn", bd.OP_CELL_RNN: "cell_rnn", bd.OP_LEAF_LSTM: "leaf_lstm",
+          bd.OP_CELL_LSTM: "cell_lstm", bd.OP_NODE_LOSS: "pass_state"}
+KIND = {bd.NODE_IN: "in", bd.NODE_OUT: "out", bd.NODE_CONST: "const", bd.NODE_OP: "op", bd.NODE_SWITCH: "switch",
+        bd.NODE_MERGE: "merge", bd.NODE_ENTRY_MERGE: "merge", bd.NODE_CALL: "Call", bd.NODE_RETURN: "Return"}
+
+
+def _as_oracle_graph(desc):
+    g = OGraph()
+    for n in desc["nodes"]:
+        kind = KIND[n["kind"]]
+        value = n["value"]
+        if kind in ("Call", "Return"):
+            value = n["label"]
+        elif kind == "in":
+            value = n["param"]
+        g.add(kind, name=OPNAME.get(n["op"], "entry" if n["kind"] == bd.NODE_ENTRY_MERGE else ""), value=value,
+              func=str(n["func"]), n_in=n["n_in"], param=n["param"])
+    for e in desc["edges"]:
+        g.connect(e["src"], e["dst"], e["dst_port"], e["src_port"], bool(e["control"]))
+    return g
+
+
+def test_fact_graph_has_the_structure_of_figure_3():
+    fs, r = rdf.fact_program()
+    d = _build(fs, r).describe()
+    kinds = [n["kind"] for n in d["nodes"]]
+    assert kinds.count(bd.NODE_CALL) == 2 and kinds.count(bd.NODE_RETURN) == 2
+    assert kinds.count(bd.NODE_ENTRY_MERGE) == 1 and kinds.count(bd.NODE_MERGE) == 1 and kinds.count(bd.NODE_SWITCH) == 1
+    ctrl = [e for e in d["edges"] if e["control"]]
+    call_ret = [e for e in ctrl if d["nodes"][e["src"]]["kind"] == bd.NODE_CALL]
+    assert len(call_ret) == 2
+    for e in call_ret:
+        assert d["nodes"][e["dst"]]["kind"] == bd.NODE_RETURN
+        assert d["nodes"][e["dst"]]["label"] == d["nodes"][e["src"]]["label"]
+    assert len(ctrl) - len(call_ret) == 2          # entry Merge -> the two constants 1 (Figure 3)
+    # Call_0 sits in `result`, Call_1 inside fact
+    by_label = {n["label"]: n["func"] for n in d["nodes"] if n["kind"] == bd.NODE_CALL}
+    assert by_label == {0: 0, 1: 1}
+    # same node and edge census as the oracle's own transformation, up to the `id` node that
+    # Figure 2 draws on the then-side
+    og = transform.transform(programs.fact_program())
+    assert len(d["nodes"]) == len(og.nodes) - 1 and len(d["edges"]) == len(og.edges) - 1
+    g = _as_oracle_graph(d)
+    for dead in (True, False):
+        res = tagged.run(g, {}, programs.INT_OPS, dead_tokens=dead)
+        assert res.value == 11
+        assert {t: (a[0], res.returns[t]) for t, a in res.calls.items()} == \
+            {(0,): (3, 6), (1, 0): (2, 2), (1, 1, 0): (1, 1)}
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 7, 12])
+def test_fib_literal_graph_runs_in_the_oracle(n):
+    fs, r = rdf.fib_program()
+    d = _build(fs, r).describe()
+    assert d["n_labels"] == 3 and d["label_bits"] == 2 and d["n_match"] == 1
+    res = tagged.run(_as_oracle_graph(d), {0: n}, programs.INT_OPS)
+    og = tagged.run(transform.transform(programs.fib_program()), {0: n}, programs.INT_OPS)
+    assert res.value == og.value == direct.fib(n)
+    assert res.calls == og.calls and res.returns == og.returns and res.leftover == 0
+
+
+def test_tree_literal_graphs_run_in_the_oracle():
+    tb = workloads.config(2, B=6)["trees"]
+    ops = programs.tree_ops(tb)
+    for kind in ("sum", "count", "height"):
+        fs, r = rdf.tree_fold_program(kind)
+        g = _as_oracle_graph(_build(fs, r, rdf.TAGS_FRAME).describe())
+        for t in range(tb.B):
+            root = int(tb.tree_root[t])
+            want = {"sum": lambda: direct.tree_fold(tb, root, lambda v: int(tb.tok[v]), lambda a, b: a + b),
+                    "count": lambda: direct.tree_fold(tb, root, lambda v: 1, lambda a, b: a + b),
+                    "height": lambda: direct.tree_fold(tb, root, lambda v: 0, lambda a, b: max(a, b) + 1)}[kind]()
+            for dead in (True, False):
+                assert tagged.run(g, {0: root}, ops, dead_tokens=dead).value == want
+
+
+@pytest.mark.parametrize("cell", ["rnn", "lstm"])
+def test_tree_net_literal_graph_runs_in_the_oracle(cell):
+    rng = np.random.default_rng(0)
+    tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, L) for L in (1, 2, 5, 7)], 3, vocab=9)
+    p = (workloads.treernn_params if cell == "rnn" else workloads.treelstm_params)(3, 9, 4, 4)
+    ops = programs.tree_net_ops(tb, p, cell)
+    ops["pass_state"] = lambda s, v: s
+    fs, r = rdf.tree_net_program(cell, with_loss=True)
+    g = _as_oracle_graph(_build(fs, r, rdf.TAGS_FRAME).describe())
+    want = direct.forward(tb, p, cell)
+    for t in range(tb.B):
+        res = tagged.run(g, {0: int(tb.tree_root[t])}, ops)
+        got = res.value if cell == "rnn" else res.value[0]
+        np.testing.assert_allclose(got, want[t], atol=1e-13)
+        assert len(res.calls) == tb.tree_sizes()[t]
+
+
+def test_product_path_has_no_cpu_route():
+    """Without a CUDA device the evaluation entry points refuse to run."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    fs, r = rdf.fib_program()
+    g = _build(fs, r)
+    with pytest.raises(RuntimeError):
+        g.eval_int(torch.zeros(4, dtype=torch.int64), 100)
+    for name in ("binding.py", "__init__.py", "build.py"):
+        src = open(os.path.join(ROOT, "paper_2410_20225_b200", name)).read()
+        assert "import oracle" not in src and "from oracle" not in src
