@@ -1,0 +1,194 @@
+"""GPU parity, integer programs: results and tags of the CUDA executor against
+the CPU oracle, bit for bit, through the C boundary."""
+import collections
+
+import numpy as np
+import pytest
+
+import workloads
+import paper_2410_20225_b200 as rdf
+from oracle import direct, programs, tagged, transform
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def _fib_iter(n):
+    a, b = 0, 1
+    for _ in range(n):
+        a, b = b, a + b
+    return a
+
+
+def pack_path_tag(instance, labels, bits):
+    """The documented packing, written from its definition: instance in bits 63..44, depth in 43..38,
+    labels `bits` wide with the innermost (head of the list) in the lowest bits."""
+    path = 0
+    for k, lab in enumerate(labels):
+        path |= lab << (bits * k)
+    return (instance << 44) | (len(labels) << 38) | path
+
+
+def decode_frame_trace(tr, B):
+    """{frame id: label list (innermost first)} by walking the parent links of the Call records."""
+    calls = tr[tr["kind"] == 0]
+    parent = dict(zip(calls["tag"].tolist(), calls["parent"].tolist()))
+    label = dict(zip(calls["tag"].tolist(), calls["label"].tolist()))
+    tags = {}
+    for f in parent:
+        labs, g = [], f
+        while g >= B:
+            labs.append(label[g])
+            g = parent[g]
+        tags[f] = (g, tuple(labs))        # (instance = root context frame, labels)
+    return tags
+
+
+@pytest.mark.parametrize("mode", [rdf.TAGS_PATH, rdf.TAGS_FRAME])
+def test_fact_example(mode):
+    fs, r = rdf.fact_program()
+    g = rdf.Graph(fs, r, mode)
+    x = torch.zeros(5, dtype=torch.int64, device="cuda")
+    y, tr = g.eval_int(x, max_invocations=64, trace_capacity=256)
+    assert y.tolist() == [11] * 5
+    st = g.stats()
+    assert st["invocations"] == 15 and st["status"] == 0
+    want = {(0,): (3, 6), (1, 0): (2, 2), (1, 1, 0): (1, 1)}
+    calls, rets = tr[tr["kind"] == 0], tr[tr["kind"] == 1]
+    assert len(calls) == 15 and len(rets) == 15
+    if mode == rdf.TAGS_PATH:
+        bits = g.describe()["label_bits"]
+        got = collections.defaultdict(dict)
+        for rec in calls:
+            inst, labs = rdf.unpack_path_tag(rec["tag"], bits)
+            assert int(rec["tag"]) == pack_path_tag(inst, labs, bits)
+            got[inst][labs] = [int(rec["value"]), None]
+        for rec in rets:
+            inst, labs = rdf.unpack_path_tag(rec["tag"], bits)
+            got[inst][labs][1] = int(rec["value"])
+        for inst in range(5):
+            assert {k: tuple(v) for k, v in got[inst].items()} == want
+    else:
+        tags = decode_frame_trace(tr, 5)
+        arg = dict(zip(calls["tag"].tolist(), calls["value"].tolist()))
+        val = dict(zip(rets["tag"].tolist(), rets["value"].tolist()))
+        per = collections.defaultdict(dict)
+        for f, (inst, labs) in tags.items():
+            per[inst][labs] = (arg[f], val[f])
+        assert all(per[i] == want for i in range(5))
+
+
+@pytest.mark.parametrize("mode", [rdf.TAGS_PATH, rdf.TAGS_FRAME])
+def test_fib_batch_full_size_values_and_tags(mode):
+    x = workloads.config(1)["x"]
+    B = len(x)
+    N = sum(2 * _fib_iter(int(n) + 1) - 1 for n in x)
+    fs, r = rdf.fib_program()
+    g = rdf.Graph(fs, r, mode)
+    bits = g.describe()["label_bits"]
+    y, tr = g.eval_int(torch.from_numpy(x).cuda(), max_invocations=N, trace_capacity=2 * N)
+    assert np.array_equal(y.cpu().numpy(), np.array([direct.fib(int(n)) for n in x]))
+    st = g.stats()
+    assert st["invocations"] == N and st["status"] == 0
+    assert st["store_inserts"] == st["store_matches"] == sum(_fib_iter(int(n) + 1) - 1 for n in x)
+    assert st["waves"] <= 2 * 18 + 8
+    calls, rets = tr[tr["kind"] == 0], tr[tr["kind"] == 1]
+    assert len(calls) == N and len(rets) == N
+    # every invocation of every instance: (tag, argument, result) as a set, against direct recursion
+    want = set()
+    for b, n in enumerate(x):
+        for tag, a, v in direct.fib_invocations(int(n))[1]:
+            want.add((b, tag, a, v))
+    if mode == rdf.TAGS_PATH:
+        assert st["max_depth"] == max(1, int(x.max()))
+        key = {}
+        for rec_tag, a in zip(calls["tag"].tolist(), calls["value"].tolist()):
+            key[rec_tag] = a
+        got = set()
+        for rec_tag, v in zip(rets["tag"].tolist(), rets["value"].tolist()):
+            inst, labs = rdf.unpack_path_tag(rec_tag, bits)
+            got.add((inst, labs, key[rec_tag], v))
+        assert got == want
+        # the packed word itself, bit for bit, on a sample
+        for b, tag, a, v in list(want)[:2000]:
+            assert pack_path_tag(b, tag, bits) in key
+    else:
+        tags = decode_frame_trace(tr, B)
+        arg = dict(zip(calls["tag"].tolist(), calls["value"].tolist()))
+        val = dict(zip(rets["tag"].tolist(), rets["value"].tolist()))
+        got = {(inst, labs, arg[f], val[f]) for f, (inst, labs) in tags.items()}
+        assert got == want
+    # the literal interpreter on a sample of instances gives the same records
+    og = transform.transform(programs.fib_program())
+    for b in range(0, B, 97):
+        res = tagged.run(og, {0: int(x[b])}, programs.INT_OPS, dead_tokens=False)
+        assert {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()} == {w for w in want if w[0] == b}
+
+
+def test_edge_cases_single_instance_and_base_cases():
+    fs, r = rdf.fib_program()
+    g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    for xs in ([0], [1], [2], [0, 1, 0, 1], [19]):
+        y, _ = g.eval_int(torch.tensor(xs, dtype=torch.int64, device="cuda"), max_invocations=20000)
+        assert y.tolist() == [direct.fib(n) for n in xs]
+    assert g.stats()["max_depth"] == 19          # 19 labels x 2 bits = 38: the deepest tag that still fits
+
+
+def test_path_tags_overflow_is_reported_and_frames_take_over():
+    fs, r = rdf.fib_program()
+    x = torch.tensor([22], dtype=torch.int64, device="cuda")
+    n_inv = 2 * _fib_iter(23) - 1
+    g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(x, max_invocations=n_inv)
+    assert e.value.code == -4                     # RDF_ERR_TAG_OVERFLOW
+    gf = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    y, _ = gf.eval_int(x, max_invocations=n_inv)
+    assert y.item() == _fib_iter(22) and gf.stats()["invocations"] == n_inv
+    # the context stays usable after a reported error
+    y, _ = g.eval_int(torch.tensor([10], dtype=torch.int64, device="cuda"), max_invocations=1000)
+    assert y.item() == 55
+
+
+def test_capacity_errors_are_status_codes():
+    fs, r = rdf.fib_program()
+    x = torch.tensor([15] * 8, dtype=torch.int64, device="cuda")
+    gf = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    with pytest.raises(rdf.RdfError) as e:
+        gf.eval_int(x, max_invocations=100)
+    assert e.value.code == -6                     # RDF_ERR_FRAMES_FULL
+    gp = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    with pytest.raises(rdf.RdfError) as e:
+        gp.eval_int(x, max_invocations=8 * 1973, max_wave_tokens=64)
+    assert e.value.code == -7                     # RDF_ERR_QUEUE_FULL
+    y, _ = gp.eval_int(x, max_invocations=8 * 1973)
+    assert y.tolist() == [610] * 8
+
+
+def test_bad_arguments():
+    fs, r = rdf.fib_program()
+    g = rdf.Graph(fs, r)
+    with pytest.raises(rdf.RdfError):
+        g.eval_int(torch.zeros(0, dtype=torch.int64, device="cuda"), max_invocations=10)
+    with pytest.raises(rdf.RdfError):
+        g.eval_int(torch.zeros(4, dtype=torch.int64, device="cuda"), max_invocations=0)
+
+
+def test_integer_tree_folds():
+    tb = workloads.config(2)["trees"]
+    dt = rdf.Graph.device_trees(tb)
+    sizes = tb.tree_sizes()
+    leaf_sum = np.array([tb.tok[s:s + n][tb.left[s:s + n] < 0].sum() for s, n in zip(tb.tree_root, sizes)])
+    for kind in ("sum", "count", "height"):
+        fs, r = rdf.tree_fold_program(kind)
+        g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+        y, _ = g.eval_trees(dt, None)
+        y = y.cpu().numpy()
+        if kind == "sum":
+            assert np.array_equal(y, leaf_sum)           # tree-sum identity: flat sum of the leaf tokens
+        elif kind == "count":
+            assert np.array_equal(y, (sizes + 1) // 2)
+        else:
+            want = [direct.tree_fold(tb, int(rt), lambda v: 0, lambda a, b: max(a, b) + 1) for rt in tb.tree_root]
+            assert np.array_equal(y, np.array(want))
+        assert g.stats()["invocations"] == tb.N

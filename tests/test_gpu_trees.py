@@ -1,0 +1,156 @@
+"""GPU parity, recursive tree networks: root states, loss and parameter
+gradients of the CUDA executor against the fp64 CPU oracle, through the C
+boundary.  Tolerance (tensor-normalised max error, per output tensor):
+1e-4 for fp32 arithmetic, 2e-2 for bf16 operands with fp32 accumulation."""
+import os
+
+import numpy as np
+import pytest
+
+import workloads
+import paper_2410_20225_b200 as rdf
+from oracle import direct
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = {rdf.F32: 1e-4, rdf.BF16: 2e-2}
+WORKERS = max(1, min(32, (os.cpu_count() or 2) - 1))
+
+
+def relerr(got, want):
+    want = np.asarray(want, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    return float(np.abs(got - want).max() / max(np.abs(want).max(), 1e-30))
+
+
+def graph(cell="rnn", with_loss=False):
+    fs, r = rdf.tree_net_program(cell, with_loss)
+    return rdf.Graph(fs, r, rdf.TAGS_FRAME)
+
+
+def check_forward(cfg, compute=rdf.F32, trees=None):
+    tb, p = cfg["trees"], cfg["params"]
+    g = graph()
+    h, _ = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), compute)
+    h = h.cpu().numpy()
+    st = g.stats()
+    assert st["invocations"] == tb.N and st["cells"] == tb.n_cells and st["leaves"] == tb.N - tb.n_cells
+    trees = list(range(tb.B)) if trees is None else trees
+    want = direct.forward(tb, p, "rnn", trees=trees)
+    assert relerr(h[trees], want) <= TOL[compute]
+    return st
+
+
+def check_grad(cfg, compute=rdf.F32, workers=1):
+    tb, p = cfg["trees"], cfg["params"]
+    g = graph(with_loss=True)
+    loss, h, grads = g.grad_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), compute)
+    st = g.stats()
+    assert st["status"] == 0 and st["invocations"] == tb.N
+    if workers > 1:
+        want_loss, G, roots = direct.loss_and_grad_pool(tb, p, "rnn", workers=workers)
+    else:
+        want_loss, G, roots = direct.loss_and_grad(tb, p, "rnn")
+    tol = TOL[compute]
+    assert relerr(h.cpu().numpy(), roots) <= tol
+    assert abs(loss.item() - want_loss) <= tol * abs(want_loss)
+    errs = {k: relerr(grads[k].cpu().numpy(), G[k]) for k in G}
+    assert all(e <= tol for e in errs.values()), errs
+    return st, errs
+
+
+def test_treernn_forward_config2_full():
+    st = check_forward(workloads.config(2))
+    assert st["waves"] <= 2 * 32 + 8
+
+
+def test_single_leaf_trees_and_tiny_batches():
+    rng = np.random.default_rng(0)
+    for Ls in ([1], [1, 1, 1], [2], [1, 3, 1, 2]):
+        tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, L) for L in Ls], 7, vocab=50)
+        p = workloads.treernn_params(7, 50, 8, 8)
+        p["b"] = (0.2 * rng.standard_normal(8)).astype(np.float32)
+        cfg = {"trees": tb, "params": p}
+        check_forward(cfg)
+        check_grad(cfg)
+    # a single leaf: the root state is the embedding row, exactly
+    tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, 1)], 7, vocab=50)
+    h, _ = graph().eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p))
+    assert np.array_equal(h.cpu().numpy()[0], p["E"][tb.tok[0]])
+
+
+def test_tags_of_tree_invocations():
+    """Frame ids decode (through the parent links) to the label lists of direct recursion."""
+    tb = workloads.config(2, B=40)["trees"]
+    p = workloads.treernn_params(1, 1000, 64, 64)
+    g = graph()
+    _, tr = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), trace_capacity=2 * tb.N)
+    calls = tr[tr["kind"] == 0]
+    assert len(calls) == tb.N
+    parent = dict(zip(calls["tag"].tolist(), calls["parent"].tolist()))
+    label = dict(zip(calls["tag"].tolist(), calls["label"].tolist()))
+    node = dict(zip(calls["tag"].tolist(), calls["value"].tolist()))
+    got = set()
+    for f in parent:
+        labs, q = [], f
+        while q >= tb.B:
+            labs.append(label[q])
+            q = parent[q]
+        got.add((q, tuple(labs), node[f]))
+    want = set()
+    for t in range(tb.B):
+        for tag, v in direct.deep(direct.tree_invocations, tb, int(tb.tree_root[t])):
+            want.add((t, tag, v))
+    assert got == want
+
+
+def test_treernn_grad_small_fp32():
+    cfg = workloads.config(3, B=96, V=500, H=64)
+    cfg["params"] = workloads.treernn_params(5, 500, 64, 64)
+    rng = np.random.default_rng(1)
+    cfg["params"]["b"] = (0.1 * rng.standard_normal(64)).astype(np.float32)
+    cfg["params"]["b_s"] = (0.1 * rng.standard_normal(5)).astype(np.float32)
+    check_grad(cfg)
+
+
+def test_treernn_grad_ragged_hidden_size():
+    """H = 300 is not a multiple of the tile sizes: ragged tiles in every contraction."""
+    cfg = workloads.config(3, B=64, V=700, H=300)
+    cfg["params"] = workloads.treernn_params(5, 700, 300, 300)
+    check_grad(cfg)
+
+
+def test_depth_stress_reduced():
+    cfg = workloads.config(5, chains=3, chain_depth=300, perfect=2, perfect_height=7, V=400, H=32)
+    st, _ = check_grad(cfg)
+    assert st["waves"] >= 2 * 300 and st["waves_backward"] >= 300
+
+
+def test_frame_tags_required_for_depth():
+    """The packed path form cannot hold a depth-300 tag: the integer fold over a chain
+    reports overflow in path form and runs in frame form."""
+    tb = workloads.tree_batch_from_shapes([workloads.chain_tree_shape(300)], 3, vocab=10)
+    dt = rdf.Graph.device_trees(tb)
+    fs, r = rdf.tree_fold_program("height")
+    with pytest.raises(rdf.RdfError) as e:
+        rdf.Graph(fs, r, rdf.TAGS_PATH).eval_trees(dt, None)
+    assert e.value.code == -4
+    y, _ = rdf.Graph(fs, r, rdf.TAGS_FRAME).eval_trees(dt, None)
+    assert y.item() == 300
+
+
+def test_treernn_config3_full_size():
+    """8192 trees, H = 300, fwd + bwd at full size; the oracle runs over a pool of processes."""
+    cfg = workloads.config(3)
+    compute = rdf.BF16
+    st, errs = check_grad(cfg, compute, workers=WORKERS)
+    print("config 3 errors:", errs, st)
+
+
+def test_depth_stress_config5_forward_sampled():
+    """Full config 5 forward (chains of depth 4096, perfect trees of 2^16 leaves); the oracle
+    evaluates one chain and one perfect tree."""
+    cfg = workloads.config(5)
+    st = check_forward(cfg, trees=[0, 63, 64])
+    assert st["waves"] >= 2 * 4096
