@@ -6,7 +6,8 @@
 // ---- fp32 tiled contraction: 64 x 64 output tile, 16-deep steps, 256 threads, 4 x 4 per thread
 static const int TM = 64, TN = 64, TK = 16;
 
-struct GemmSmem {
+// read and written with 128-bit accesses: rows are 272 bytes, the struct must sit on a 16-byte boundary
+struct __align__(16) GemmSmem {
     float As[TK][TM + 4];     // [k][row of the tile]
     float Bs[TK][TN + 4];     // [k][column of the tile]
 };
