@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark: recursive invocations per second of the tagged-dataflow executor.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl reference]
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+lowered graph -> seed tokens -> all forward waves (tag push/pop, matching, batched
+cells) -> loss head -> gradient waves -> parameter gradients (workloads 3-5), or
+the forward pass alone (workloads 1-2).  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "recursive_invocations_per_sec"
+UNIT = "invocations/s"
+WORKLOAD_NAMES = {
+    1: "config1: fib(n), 1024 calls, n~U[0,18], int64, packed path tags, forward",
+    2: "config2: TreeRNN forward, 512 random binary trees, H=64, fp32",
+    3: "config3: TreeRNN forward+backward, 8192 trees (lognormal leaves, median 18), H=300, vocab 21000, 5-class loss at every node",
+    5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
+}
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11}
+
+
+def fib_iter(n):
+    a, b = 0, 1
+    for _ in range(n):
+        a, b = b, a + b
+    return a
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, p[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- workloads
+def load(k, seed):
+    cfg = workloads.config(k, seed=seed)
+    if cfg["kind"] == "fib":
+        cfg["N"] = int(sum(2 * fib_iter(int(n) + 1) - 1 for n in cfg["x"]))
+    else:
+        cfg["N"] = cfg["trees"].N
+    return cfg
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_step(cfg, sample):
+    """One bounded sample of the workload on the CPU oracle; returns invocations processed."""
+    from oracle import direct
+    if cfg["kind"] == "fib":
+        xs = cfg["x"][:sample]
+        n = 0
+        for v in xs:
+            n += len(direct.fib_invocations(int(v))[1])
+        return n
+    tb = cfg["trees"]
+    trees = list(range(min(sample, tb.B)))
+    if cfg["grad"]:
+        direct.loss_and_grad(tb, cfg["params"], "rnn", trees=trees)
+    else:
+        direct.forward(tb, cfg["params"], "rnn", trees=trees)
+    return int(tb.tree_sizes()[trees].sum())
+
+
+def oracle_sample_size(cfg):
+    if cfg["kind"] == "fib":
+        return 256
+    if cfg["trees"].N > 2_000_000:
+        return 1                       # one chain of depth 4096
+    return 256 if cfg["grad"] else 512
+
+
+def time_oracle(cfg, steps, warmup):
+    try:
+        from threadpoolctl import threadpool_limits
+        ctx = threadpool_limits(limits=1)
+    except Exception:  # pragma: no cover
+        import contextlib
+        ctx = contextlib.nullcontext()
+    sample = oracle_sample_size(cfg)
+    with ctx:
+        for _ in range(warmup):
+            oracle_step(cfg, sample)
+        t0 = time.perf_counter()
+        n = 0
+        for _ in range(steps):
+            n += oracle_step(cfg, sample)
+        dt = time.perf_counter() - t0
+    what = (f"first {sample} instances" if cfg["kind"] == "fib" else f"first {sample} trees") + \
+        f" of the workload per step, {steps} step(s), fp64/int Python+numpy oracle, 1 thread"
+    return n / dt, dt / steps, what
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=3, choices=sorted(WORKLOAD_NAMES))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seed", type=int, default=workloads.DEFAULT_SEED)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        cfg = load(args.workload, args.seed)
+        value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup))
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * s_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAMES[args.workload]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
+
+    import torch
+    import paper_2410_20225_b200 as rdf
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the recursive-dataflow path has no CPU route")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank processes a batch of its own (instances never exchange tokens): weak scaling
+    cfg = load(args.workload, args.seed + rank)
+    N = cfg["N"]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
+
+    if cfg["kind"] == "fib":
+        fs, r = rdf.fib_program()
+        g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+        x_host = torch.from_numpy(cfg["x"]).pin_memory()
+        x_dev = x_host.cuda()
+        y = torch.empty_like(x_dev)
+        kind, compute, dtype = "eval_int", None, "int64"
+
+        def step():
+            g.eval_int(x_dev, N, check=False, y=y)
+
+        def step_e2e():
+            xd = x_host.cuda(non_blocking=True)
+            out, _ = g.eval_int(xd, N, check=False)
+            return out.cpu()
+        h2d, d2h = x_host.numel() * 8, x_host.numel() * 8
+        flops_fwd = 0.0
+    else:
+        tb, p = cfg["trees"], cfg["params"]
+        fs, r = rdf.tree_net_program("rnn", with_loss=cfg["grad"])
+        g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+        compute = rdf.BF16 if cfg["bf16"] else rdf.F32
+        dtype = "f32"                       # arithmetic type of the contractions as built
+        host = {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).pin_memory()
+                for k in ("tree_root", "left", "right", "tok", "label")}
+        dt = {k: v.cuda() for k, v in host.items()}
+        dp = rdf.Graph.device_params(p)
+        H = cfg["H"]
+        h_root = torch.empty(tb.B, H, dtype=torch.float32, device="cuda")
+        flops_fwd = tb.n_cells * 2.0 * (2 * H) * H
+        if cfg["grad"]:
+            kind = "grad"
+            grads = {k: torch.empty_like(v) for k, v in dp.items()}
+            loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+
+            def step():
+                g.grad_trees(dt, dp, compute, check=False, grads=grads, loss=loss, h_root=h_root)
+                if dist is not None:            # data-parallel exchange: one sum of the parameter gradients
+                    for t in grads.values():
+                        dist.all_reduce(t)
+
+            def step_e2e():
+                d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+                l, _, _ = g.grad_trees(d, dp, compute, check=False, grads=grads, h_root=h_root)
+                if dist is not None:
+                    for t in grads.values():
+                        dist.all_reduce(t)
+                return l.item()
+            h2d, d2h = sum(v.numel() * 4 for v in host.values()), 4
+        else:
+            kind = "eval_trees"
+
+            def step():
+                g.eval_trees(dt, dp, compute, check=False, h_root=h_root)
+
+            def step_e2e():
+                d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+                out, _ = g.eval_trees(d, dp, compute, check=False)
+                return out.cpu()
+            h2d, d2h = sum(v.numel() * 4 for v in host.values()), tb.B * H * 4
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    g.set_profiling(True)
+    for _ in range(args.warmup):
+        step()
+    st = g.stats()                                   # also checks the device status word
+
+    # ---- device-timed region: K steps, L2 flushed between steps, one event pair per step
+    clocks = ClockSampler(local)
+    barrier()
+    clocks.start()
+    times, phases = [], {}
+    for _ in range(args.steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+        for k, v in g.phase_ms().items():
+            phases.setdefault(k, []).append(v)
+    barrier()
+    clk = clocks.stop()
+    st = g.stats()
+    total_ms = sum(times)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        n_all = torch.tensor([N], dtype=torch.float64, device="cuda")
+        dist.all_reduce(n_all)
+        N_all = float(n_all.item())
+    else:
+        N_all = float(N)
+    value = N_all * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the public call, host buffers, copies inside the timed region
+    for _ in range(2):
+        step_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step_e2e()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = N_all * args.steps / e2e_s
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel
+    pk = peaks()
+    mean_phase = {k: sum(v) / len(v) for k, v in phases.items()}
+    dominant = max(mean_phase, key=mean_phase.get) if mean_phase else "forward"
+    dom_ms = mean_phase.get(dominant, total_ms / args.steps)
+    if cfg["kind"] == "fib":
+        alg_bytes = 128.0 * N          # 6 token touches x 16 B + one 32 B store slot per invocation
+        achieved = alg_bytes / (dom_ms * 1e-3) / 1e9
+        roof = {"kernel": "rdf_forward_kernel", "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
+    else:
+        H = cfg["H"]
+        C = cfg["trees"].n_cells
+        flops = {"forward": flops_fwd, "backward": flops_fwd, "dW": flops_fwd}.get(dominant, flops_fwd)
+        achieved = flops / (dom_ms * 1e-3) / 1e12
+        kernel = {"forward": "rdf_forward_kernel", "backward": "rdf_backward_kernel", "dW": "rdf_dw_kernel"}.get(
+            dominant, dominant)
+        roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
+                "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                "cells": C, "flops_per_cell": 2.0 * 2 * H * H}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, _, what = time_oracle(cfg, 1, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": dtype, "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.workload], "invocations_per_step": N, "instances": cfg.get("B") or cfg["trees"].B,
+                   "pass": "forward+backward" if cfg.get("grad") else "forward",
+                   "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
+        "clocks": clk,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": KERNELS_PER_STEP[kind] * args.steps,
+        "roofline": roof,
+        "cpu_baseline": cpu,
+        "phase_ms": mean_phase,
+        "waves": {"forward": st["waves"], "backward": st["waves_backward"], "widest": st["max_wave_tokens"]},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

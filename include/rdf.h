@@ -246,6 +246,19 @@ int rdf_last_status(rdf_graph* g, rdf_stats* s);
 
 const char* rdf_strerror(int status);
 
+/* Measurement aid (the paper reports only wall-clock times, Section 6; there is
+ * no counterpart to cite): when enabled, rdf_eval / rdf_grad record CUDA events
+ * on their stream between the phases of a call.  rdf_last_phase_ms synchronises
+ * those events and writes up to `capacity` durations in milliseconds to the
+ * host array `ms`, in this order:
+ *   0 set-up (clears, program upload, seed tokens)   1 forward waves
+ *   2 loss head   3 gradient waves   4 dW   5 db   6 dW_s, db_s   7 dE
+ * (rdf_eval fills 0..1).  *n receives the number written. */
+enum { RDF_PHASE_SETUP = 0, RDF_PHASE_FORWARD, RDF_PHASE_LOSS, RDF_PHASE_BACKWARD, RDF_PHASE_DW, RDF_PHASE_DB,
+       RDF_PHASE_DWS, RDF_PHASE_DE, RDF_PHASE__COUNT };
+int rdf_set_profiling(rdf_graph* g, int enable);
+int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n);
+
 #ifdef __cplusplus
 }
 #endif

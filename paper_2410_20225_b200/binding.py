@@ -108,7 +108,8 @@ class rdf_stats(C.Structure):
 
 
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
-           "rdf_last_status", "rdf_strerror"]
+           "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms"]
+PHASES = ["setup", "forward", "loss", "backward", "dW", "db", "dW_s", "dE"]
 
 _lib = None
 
@@ -130,6 +131,8 @@ def lib() -> C.CDLL:
         L.rdf_grad.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params), C.POINTER(rdf_outputs),
                                C.POINTER(rdf_param_grads), C.c_void_p, C.c_size_t, C.c_void_p]
         L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
+        L.rdf_set_profiling.argtypes = [C.c_void_p, C.c_int]
+        L.rdf_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
         L.rdf_strerror.argtypes = [C.c_int]
         L.rdf_strerror.restype = C.c_char_p
         _lib = L
@@ -282,6 +285,20 @@ class Graph:
             self._ws = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
         off = (-self._ws.data_ptr()) % 256
         return self._ws.data_ptr() + off, n
+
+    def set_profiling(self, on=True):
+        rc = lib().rdf_set_profiling(self.handle, int(on))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_set_profiling")
+
+    def phase_ms(self):
+        """{phase name: milliseconds} of the last call (needs set_profiling(True) before it)."""
+        ms = (C.c_float * len(PHASES))()
+        n = C.c_int()
+        rc = lib().rdf_last_phase_ms(self.handle, ms, len(PHASES), C.byref(n))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_last_phase_ms")
+        return {PHASES[k]: float(ms[k]) for k in range(n.value)}
 
     def stats(self, check=True):
         s = rdf_stats()

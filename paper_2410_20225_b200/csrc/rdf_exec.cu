@@ -490,6 +490,7 @@ int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params
 // zero what must start at zero, upload the program, seed, run all waves
 int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
                        DevCtx& c, cudaStream_t stream) {
+    rdf_mark(S, 0, stream);
     CUDA_OK(cudaMemsetAsync(ws + L.ctl, 0, 4096, stream));
     if (L.arrived_bytes && g->tag_mode == RDF_TAGS_FRAME) CUDA_OK(cudaMemsetAsync(ws + L.arrived, 0, L.arrived_bytes, stream));
     if (L.table_bytes) CUDA_OK(cudaMemsetAsync(ws + L.table, 0xFF, L.table_bytes, stream));
@@ -502,6 +503,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
         CUDA_OK(cudaMemcpyAsync(ws + L.consts, g->consts.data(), g->consts.size() * sizeof(int64_t), cudaMemcpyHostToDevice, stream));
     rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
+    rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
     if (g->has_vector_ops) {
@@ -510,6 +512,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     if (out->trace)
         CUDA_OK(cudaMemcpyAsync(out->trace_count, &c.ctl->trace_count, sizeof(uint64_t), cudaMemcpyDeviceToDevice, stream));
+    rdf_mark(S, 2, stream);
     S->last_ctl = c.ctl;
     S->last_stream = stream;
     S->ran = true;
@@ -517,7 +520,10 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
 }
 
 void rdf_exec_release(rdf_graph* g) {
-    delete static_cast<ExecState*>(g->dev);
+    ExecState* S = static_cast<ExecState*>(g->dev);
+    if (S && S->have_events)
+        for (cudaEvent_t e : S->ev) cudaEventDestroy(e);
+    delete S;
     g->dev = nullptr;
 }
 
@@ -561,4 +567,29 @@ extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
     s->store_inserts = h.store_inserts; s->store_matches = h.store_matches; s->store_probes = h.store_probes;
     s->max_probe = h.max_probe; s->max_depth = h.max_depth; s->cells = h.cells; s->leaves = h.leaves;
     return h.status;
+}
+
+extern "C" int rdf_set_profiling(rdf_graph* g, int enable) {
+    if (!g) return RDF_ERR_BAD_ARG;
+    ExecState* S = rdf_state_of(g);
+    if (enable && !S->have_events) {
+        for (cudaEvent_t& e : S->ev) CUDA_OK(cudaEventCreate(&e));
+        S->have_events = true;
+    }
+    S->profiling = enable != 0;
+    S->n_phases = 0;
+    return RDF_OK;
+}
+
+extern "C" int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n) {
+    if (!g || !ms || !n) return RDF_ERR_BAD_ARG;
+    ExecState* S = rdf_state_of(g);
+    *n = 0;
+    if (!S->profiling || !S->have_events || S->n_phases == 0) return RDF_OK;
+    CUDA_OK(cudaEventSynchronize(S->ev[S->n_phases]));
+    for (int k = 0; k < S->n_phases && k < capacity; ++k) {
+        CUDA_OK(cudaEventElapsedTime(&ms[k], S->ev[k], S->ev[k + 1]));
+        *n = k + 1;
+    }
+    return RDF_OK;
 }

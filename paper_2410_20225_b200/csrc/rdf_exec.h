@@ -35,7 +35,20 @@ struct ExecState {
     void* last_ctl = nullptr;
     cudaStream_t last_stream = nullptr;
     bool ran = false;
+    // optional phase timing
+    bool profiling = false;
+    cudaEvent_t ev[RDF_PHASE__COUNT + 1] = {};
+    bool have_events = false;
+    int n_phases = 0;
 };
+
+// records the boundary after phase `k - 1` (k = 0: start of the call)
+inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
+    if (S->profiling && S->have_events) {
+        cudaEventRecord(S->ev[k], stream);
+        S->n_phases = k;
+    }
+}
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, children, port_val, arrived, table, cell_items,

@@ -336,11 +336,13 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     const int loss_blocks = std::min(4096, std::max(1, (int)((in->max_invocations + 63) / 64)));
     rdf_loss_kernel<<<loss_blocks, 256, 0, stream>>>(c);
     rdf_loss_final_kernel<<<1, 32, 0, stream>>>(c, loss_blocks);
+    rdf_mark(S, 3, stream);
     // gradient waves
     rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
+    rdf_mark(S, 4, stream);
     // parameter gradients
     const int tiles_m = (H + TM - 1) / TM, tiles_n = (2 * H + TN - 1) / TN;
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
@@ -348,9 +350,13 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     uint32_t chunk = (uint32_t)((max_cells + splits - 1) / splits);
     chunk = (chunk + TK - 1) / TK * TK;
     rdf_dw_kernel<<<tiles_m * tiles_n * splits, 256, 0, stream>>>(c, tiles_m, tiles_n, chunk);
+    rdf_mark(S, 5, stream);
     rdf_db_kernel<<<S->grid, 256, 0, stream>>>(c);
+    rdf_mark(S, 6, stream);
     rdf_dws_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+    rdf_mark(S, 7, stream);
     rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
+    rdf_mark(S, 8, stream);
     CUDA_OK(cudaGetLastError());
     return RDF_OK;
 }
