@@ -136,14 +136,14 @@ def oracle_sample_size(cfg):
     return 256 if cfg["grad"] else 512
 
 
-def time_oracle(cfg, steps, warmup):
+def time_oracle(cfg, steps, warmup, scale=1):
     try:
         from threadpoolctl import threadpool_limits
         ctx = threadpool_limits(limits=1)
     except Exception:  # pragma: no cover
         import contextlib
         ctx = contextlib.nullcontext()
-    sample = oracle_sample_size(cfg)
+    sample = oracle_sample_size(cfg) * scale
     with ctx:
         for _ in range(warmup):
             oracle_step(cfg, sample)
@@ -350,7 +350,7 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        v, _, what = time_oracle(cfg, 1, 0)
+        v, _, what = time_oracle(cfg, 1, 0, scale=1 if cfg["trees"].N > 2_000_000 else 4) if cfg["kind"] != "fib" else time_oracle(cfg, 1, 0, scale=4)
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
 
     line = {
