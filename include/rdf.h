@@ -232,6 +232,34 @@ int rdf_workspace_bytes(const rdf_graph* g, const rdf_batch* in, const rdf_param
 int rdf_eval(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
              void* workspace, size_t workspace_bytes, void* stream);
 
+/* rdf_eval for callers that can neither pass a workspace nor allocate one.
+ * (The paper has no counterpart: this is a packaging variant of rdf_eval.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside
+ * a memory pool that has already handed out everything, in a plug-in whose host
+ * forbids cudaMalloc after start-up, or on a latency path where an allocation
+ * (which may synchronise the device) is not acceptable.  Such a caller still
+ * owns and passes the inputs and outputs; only the scratch is taken care of.
+ *
+ * The scratch is a fixed array of RDF_NOALLOC_SCRATCH_BYTES (16 MiB) that is part
+ * of the library image: every GPU that loads the library holds it until the
+ * process ends.  A batch whose rdf_workspace_bytes(.., want_grad = 0, ..) exceeds
+ * that size is refused with RDF_ERR_WORKSPACE_TOO_SMALL and nothing is launched;
+ * use rdf_eval with a workspace of your own for such batches.
+ *
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library
+ * routine.  The first call on each device looks up the array's device address
+ * (a runtime query, done once per device with that device current); make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array, which still holds the previous call's data: the call clears what must
+ * start from zero on `stream` before its kernels run, but two calls that overlap
+ * on the GPU (different streams, or different graphs used concurrently) race on
+ * it -- keep calls to this entry point ordered on one stream per device.
+ * Everything else (arguments, outputs, status reporting) is as for rdf_eval. */
+#define RDF_NOALLOC_SCRATCH_BYTES (16u << 20)
+int rdf_eval_noalloc(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
+                     void* stream);
+
 /* Forward + reverse mode (Section 4): forward values are retained per
  * invocation; the gradient pass re-enters every invocation under the tag its
  * forward Call_i created and accumulates parameter gradients over all

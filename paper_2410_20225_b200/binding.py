@@ -108,7 +108,8 @@ class rdf_stats(C.Structure):
 
 
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
-           "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms"]
+           "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc"]
+NOALLOC_SCRATCH_BYTES = 16 << 20
 PHASES = ["setup", "forward", "loss", "backward", "dW", "db", "dW_s", "dE"]
 
 _lib = None
@@ -130,6 +131,8 @@ def lib() -> C.CDLL:
                                C.c_void_p, C.c_size_t, C.c_void_p]
         L.rdf_grad.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params), C.POINTER(rdf_outputs),
                                C.POINTER(rdf_param_grads), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.rdf_eval_noalloc.argtypes = [C.c_void_p, C.POINTER(rdf_batch), C.POINTER(rdf_params),
+                                       C.POINTER(rdf_outputs), C.c_void_p]
         L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
         L.rdf_set_profiling.argtypes = [C.c_void_p, C.c_int]
         L.rdf_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
@@ -348,6 +351,23 @@ class Graph:
         if check:
             self.stats()
         return y, self._read_trace(tr)
+
+    def eval_int_noalloc(self, x, y, max_invocations, check=True):
+        """rdf_eval_noalloc for an integer program: the caller passes input x and output y (int64
+        CUDA tensors of equal length); scratch is the library's built-in 16 MiB array, so nothing
+        is allocated here -- not even through torch.  Raises RdfError(-3) when the batch needs more."""
+        torch = _torch()
+        assert x.is_cuda and y.is_cuda and x.dtype == y.dtype == torch.int64 and x.numel() == y.numel()
+        batch = rdf_batch(B=x.numel(), x=x.data_ptr(), N=0, max_invocations=int(max_invocations), max_wave_tokens=0)
+        out = rdf_outputs()
+        out.y = y.data_ptr()
+        rc = lib().rdf_eval_noalloc(self.handle, C.byref(batch), None, C.byref(out),
+                                    torch.cuda.current_stream().cuda_stream)
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_eval_noalloc")
+        if check:
+            self.stats()
+        return y
 
     # ---- tree programs
     @staticmethod

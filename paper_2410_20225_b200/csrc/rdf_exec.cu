@@ -593,3 +593,54 @@ extern "C" int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n) 
     }
     return RDF_OK;
 }
+
+// ===========================================================================
+// Evaluation without any caller-supplied or freshly allocated scratch memory
+// ===========================================================================
+// Built-in scratch: lives in the library image, so every GPU that loads the
+// library holds these 16 MiB until the process exits.
+static __device__ __align__(256) unsigned char rdf_builtin_scratch[RDF_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+// Device address of the array above, looked up once per device.  In host code
+// the array's name is only a handle for the runtime; kernels need the address
+// that cudaGetSymbolAddress returns for the device that is current.
+const int kMaxDevices = 64;
+void* g_builtin_scratch[kMaxDevices] = {};
+
+int builtin_scratch(void** out) {
+    int dev = 0;
+    CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return RDF_ERR_BAD_ARG;
+    if (!g_builtin_scratch[dev]) {
+        void* p = nullptr;
+        CUDA_OK(cudaGetSymbolAddress(&p, rdf_builtin_scratch));
+        if (!p) return RDF_ERR_CUDA;
+        g_builtin_scratch[dev] = p;
+    }
+    *out = g_builtin_scratch[dev];
+    return RDF_OK;
+}
+}  // namespace
+
+extern "C" int rdf_eval_noalloc(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
+                                void* stream) {
+    if (!g || !in || !out) return RDF_ERR_BAD_ARG;
+    Layout L;
+    int rc = rdf_make_layout(g, in, params, 0, L);
+    if (rc != RDF_OK) return rc;
+    if (L.total > (size_t)RDF_NOALLOC_SCRATCH_BYTES) return RDF_ERR_WORKSPACE_TOO_SMALL;   // batch too large for the built-in array
+    void* ws = nullptr;
+    rc = builtin_scratch(&ws);
+    if (rc != RDF_OK) return rc;
+    rc = rdf_check_common(g, in, params, out, ws);
+    if (rc != RDF_OK) return rc;
+    ExecState* S = rdf_state_of(g);
+    rc = rdf_prepare_device(g, S);
+    if (rc != RDF_OK) return rc;
+    DevCtx c;
+    rdf_fill_ctx(g, in, params, out, static_cast<char*>(ws), L, S, c);
+    // rdf_launch_forward clears the control block, the arrival counters and the hash tables
+    // on the stream before the first kernel, so nothing of the previous call is read.
+    return rdf_launch_forward(g, in, out, static_cast<char*>(ws), L, S, c, static_cast<cudaStream_t>(stream));
+}
