@@ -31,9 +31,11 @@ WORKLOAD_NAMES = {
     1: "config1: fib(n), 1024 calls, n~U[0,18], int64, packed path tags, forward",
     2: "config2: TreeRNN forward, 512 random binary trees, H=64, fp32",
     3: "config3: TreeRNN forward+backward, 8192 trees (lognormal leaves, median 18), H=300, vocab 21000, 5-class loss at every node",
+    4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11}
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13}
+CELL = {"treernn": "rnn", "treelstm": "lstm"}
 
 
 def fib_iter(n):
@@ -122,9 +124,9 @@ def oracle_step(cfg, sample):
     tb = cfg["trees"]
     trees = list(range(min(sample, tb.B)))
     if cfg["grad"]:
-        direct.loss_and_grad(tb, cfg["params"], "rnn", trees=trees)
+        direct.loss_and_grad(tb, cfg["params"], CELL[cfg["kind"]], trees=trees)
     else:
-        direct.forward(tb, cfg["params"], "rnn", trees=trees)
+        direct.forward(tb, cfg["params"], CELL[cfg["kind"]], trees=trees)
     return int(tb.tree_sizes()[trees].sum())
 
 
@@ -224,7 +226,8 @@ def main():
         flops_fwd = 0.0
     else:
         tb, p = cfg["trees"], cfg["params"]
-        fs, r = rdf.tree_net_program("rnn", with_loss=cfg["grad"])
+        cell = CELL[cfg["kind"]]
+        fs, r = rdf.tree_net_program(cell, with_loss=cfg["grad"])
         g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
         compute = rdf.BF16 if cfg["bf16"] else rdf.F32
         dtype = "f32"                       # arithmetic type of the contractions as built
@@ -235,8 +238,10 @@ def main():
         H = cfg["H"]
         h_root = torch.empty(tb.B, H, dtype=torch.float32, device="cuda")
         flops_fwd = tb.n_cells * 2.0 * (2 * H) * H
+        if cell == "lstm":
+            flops_fwd = tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
         if cfg["grad"]:
-            kind = "grad"
+            kind = "grad" if cell == "rnn" else "grad_lstm"
             grads = {k: torch.empty_like(v) for k, v in dp.items()}
             loss = torch.zeros(1, dtype=torch.float32, device="cuda")
 
@@ -346,7 +351,7 @@ def main():
         roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
                 "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
                 "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
-                "cells": C, "flops_per_cell": 2.0 * 2 * H * H}
+                "cells": C, "flops_forward": flops_fwd}
 
     cpu = None
     if not args.no_cpu_baseline:

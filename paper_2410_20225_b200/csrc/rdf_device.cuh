@@ -96,7 +96,9 @@ struct DevCtx {
     uint32_t  work_cap;
     uint32_t* op_l;               // per frame: operand frames of the operator that made its state
     uint32_t* op_r;               //            (leaf: op_l = LEAF_MARK, op_r = token id)
-    float*    arena;              // [frame_cap, H] fp32 states
+    float*    arena;              // [frame_cap, S] fp32 states: S = H (TreeRNN h) or 2H (TreeLSTM h then c)
+    float*    gates;              // TreeLSTM under rdf_grad: [frame_cap, G] activated gates, later their gradients
+    int       S, G, lstm;
     // parameters
     int H, D, V, n_classes, compute;
     const float *E, *W, *b, *W_x, *b_x, *W_s, *b_s;
@@ -105,7 +107,8 @@ struct DevCtx {
     rdf_trace_rec* trace;
     long long trace_cap;
     // gradient pass
-    float*    dhp;                // [frame_cap, H]: gradient arriving from the parent, then dz (cell) / dh (leaf)
+    float*    dhp;                // [frame_cap, S]: gradient arriving from the caller (dh, and dc for the TreeLSTM);
+                                  //                 TreeRNN: overwritten by dz (cell) / dh (leaf)
     float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
     uint32_t* bq[2];              // backward wave queues (frame ids)
     uint32_t* all_cells;          // every cell frame, in backward wave order

@@ -10,6 +10,7 @@
 #include <cstring>
 
 #include "rdf_exec.h"
+#include "rdf_lstm.cuh"
 
 // ===========================================================================
 // S phase: the segment interpreter
@@ -270,7 +271,8 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
 
 __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_constant__ DevCtx c) {
     __shared__ SharedProgram sp;
-    __shared__ GemmSmem gsm;
+    __shared__ LstmSmem tile_smem;                                   // the TreeRNN tiles use its first part
+    GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     load_program(c, sp);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
@@ -296,8 +298,13 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
         const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
         if (n_leaf | n_cell) {
-            if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
-            if (n_cell) rnn_cell_tiles(c, gsm, min(n_cell, c.work_cap));
+            if (c.lstm) {
+                if (n_leaf) lstm_forward_tiles<3>(c, tile_smem, min(n_leaf, c.work_cap));
+                if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
+            } else {
+                if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
+                if (n_cell) rnn_cell_tiles(c, gsm, min(n_cell, c.work_cap));
+            }
             if (!grid_barrier(c, &c.ctl->bar, generation)) break;
         }
     }
@@ -322,7 +329,7 @@ __global__ void rdf_gather_roots_kernel(const DevCtx c, float* h_root) {
     const int b = blockIdx.x;
     const long long slot = c.y[b];
     if (slot < 0 || slot >= (long long)c.frame_cap) return;
-    for (int k = threadIdx.x; k < c.H; k += blockDim.x) h_root[(size_t)b * c.H + k] = c.arena[(size_t)slot * c.H + k];
+    for (int k = threadIdx.x; k < c.H; k += blockDim.x) h_root[(size_t)b * c.H + k] = c.arena[(size_t)slot * c.S + k];
 }
 
 // ===========================================================================
@@ -382,10 +389,12 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     const size_t vf = g->has_vector_ops ? L.frame_cap : 0;
     L.op_l = P.take<uint32_t>(vf);
     L.op_r = P.take<uint32_t>(vf);
-    L.arena = P.take<float>(vf * H);
+    const size_t S = g->has_lstm ? 2 * (size_t)H : (size_t)H;
+    L.arena = P.take<float>(vf * S);
+    L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
-    L.dhp = P.take<float>(gf * H);
+    L.dhp = P.take<float>(gf * S);
     L.dlog = P.take<float>(gf * 8);
     L.bq0 = P.take<uint32_t>(gf);
     L.bq1 = P.take<uint32_t>(gf);
@@ -451,6 +460,10 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.E = params->E; c.W = params->W; c.b = params->b; c.W_x = params->W_x; c.b_x = params->b_x;
         c.W_s = params->W_s; c.b_s = params->b_s;
         c.y = reinterpret_cast<int64_t*>(ws + L.ybuf);
+        c.lstm = g->has_lstm ? 1 : 0;
+        c.S = g->has_lstm ? 2 * params->H : params->H;
+        c.G = 5 * params->H;
+        c.gates = nullptr;                 // set by rdf_grad for the TreeLSTM
     } else {
         c.y = out->y;
     }
@@ -478,7 +491,7 @@ int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params
     if (g->has_vector_ops) {
         if (!params || !params->E || !params->W || !params->b || !out->h_root) return RDF_ERR_BAD_ARG;
         if (params->D != params->H) return RDF_ERR_UNSUPPORTED;
-        if (g->has_lstm) return RDF_ERR_UNSUPPORTED;
+        if (g->has_lstm && (!params->W_x || !params->b_x)) return RDF_ERR_BAD_ARG;
         if (params->compute != RDF_F32 && params->compute != RDF_BF16) return RDF_ERR_BAD_ARG;
     } else if (!out->y) {
         return RDF_ERR_BAD_ARG;

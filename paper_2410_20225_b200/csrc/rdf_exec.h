@@ -12,6 +12,13 @@ struct __align__(16) GemmSmem {
     float Bs[TK][TN + 4];     // [k][column of the tile]
 };
 
+// TreeLSTM tiles: the same 64 x 64 tile for up to five gate blocks at once, so that all gates of a
+// hidden unit end up in one thread and the gate arithmetic fuses into the epilogue
+struct __align__(16) LstmSmem {
+    float As[TK][TM + 4];
+    float Bs[5][TK][TN + 4];
+};
+
 __device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 __device__ __forceinline__ void gemm_tile_step(const GemmSmem& sm, int tx, int ty, float (&acc)[4][4]) {
@@ -52,7 +59,7 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, children, port_val, arrived, table, cell_items,
-        leaf_items, op_l, op_r, arena, ybuf, dhp, dlog, bq0, bq1, all_cells, all_leaves, loss_partial, total;
+        leaf_items, op_l, op_r, arena, gates, ybuf, dhp, dlog, bq0, bq1, all_cells, all_leaves, loss_partial, total;
     uint32_t qcap, frame_cap, work_cap;
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes;

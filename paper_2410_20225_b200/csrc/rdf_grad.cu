@@ -3,10 +3,10 @@
 // The gradient pass re-enters every invocation under the tag (frame) that its
 // forward Call_i created: wave 0 holds the invocations called from `result`,
 // each wave hands the gradients of a cell's operands to the frames of the two
-// calls it made (Call_1 / Call_2 replayed through the children table), until
-// the leaves are reached.  Parameter gradients are sums over all invocations
-// and are formed after the waves as dense contractions over the retained
-// per-invocation values.
+// calls it made (Call_1 / Call_2 replayed through the retained operand frames),
+// until the leaves are reached.  Parameter gradients are sums over all
+// invocations and are formed after the waves as dense contractions over the
+// retained per-invocation values.
 #include <algorithm>
 #include <cstring>
 
@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
     const int H = c.H, C = c.n_classes;
     float my_loss = 0.f;
     for (uint32_t f = (uint32_t)c.B + warp; f < F; f += n_warps) {
-        const float* h = c.arena + (size_t)f * H;
+        const float* h = c.arena + (size_t)f * c.S;
         float z[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
@@ -88,7 +88,20 @@ __global__ void __launch_bounds__(256) rdf_backward_seed_kernel(const DevCtx c) 
     if (b == 0) c.ctl->bq_count[0] = (uint32_t)c.B;
 }
 
-// A: per invocation t of the wave, dh = (gradient from the caller) + W_s^T dlog;
+__device__ __forceinline__ void backward_enqueue(const DevCtx& c, uint32_t wave, uint32_t t, bool leaf, uint32_t l,
+                                                 uint32_t r) {
+    if (leaf) {
+        c.all_leaves[atomicAdd(&c.ctl->all_leaves, 1u)] = t;
+    } else {
+        c.all_cells[atomicAdd(&c.ctl->all_cells, 1u)] = t;
+        const uint32_t at = atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u);
+        uint32_t* qn = c.bq[(wave + 1) & 1];
+        qn[at] = l;
+        qn[at + 1] = r;
+    }
+}
+
+// A (TreeRNN): per invocation t of the wave, dh = (gradient from the caller) + W_s^T dlog;
 //    cell: dz = dh * (1 - h^2), queue the two callee frames; leaf: keep dh for dE.
 __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
     const int lane = threadIdx.x % 32;
@@ -103,39 +116,78 @@ __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
         const bool leaf = l == LEAF_MARK;
         float dl[MAX_CLASSES];
 #pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = c.W_s ? __ldcg(&c.dlog[(size_t)t * 8 + k]) : 0.f;
+        for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
         float* g = c.dhp + (size_t)t * H;
         const float* h = c.arena + (size_t)t * H;
         for (int j = lane; j < H; j += 32) {
             float dh = from_result ? 0.f : __ldcg(&g[j]);
-            if (c.W_s) {
 #pragma unroll
-                for (int k = 0; k < MAX_CLASSES; ++k)
-                    if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
-            }
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
             if (!leaf) {
                 const float hj = __ldcg(&h[j]);
                 dh *= 1.f - hj * hj;
             }
             g[j] = dh;
         }
-        if (lane == 0) {
-            if (leaf) {
-                c.all_leaves[atomicAdd(&c.ctl->all_leaves, 1u)] = t;
-            } else {
-                c.all_cells[atomicAdd(&c.ctl->all_cells, 1u)] = t;
-                const uint32_t at = atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u);
-                uint32_t* qn = c.bq[(wave + 1) & 1];
-                qn[at] = l;
-                qn[at + 1] = r;
-            }
-        }
+        if (lane == 0) backward_enqueue(c, wave, t, leaf, l, r);
     }
 }
 
-// B: [dh_l ; dh_r] = W^T dz for the cells all_cells[first, first + n)
-__device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, uint32_t n_items) {
-    const int H = c.H, K2 = 2 * c.H;
+// A (TreeLSTM): the gate gradients replace the retained gates; dc goes straight to the callee frames.
+__device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
+    const int lane = threadIdx.x % 32;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    const int H = c.H, C = c.n_classes, S = c.S;
+    const uint32_t* q = c.bq[wave & 1];
+    for (uint32_t i = warp; i < n; i += n_warps) {
+        const uint32_t t = __ldcg(&q[i]);
+        const uint32_t parent = __ldcg(&c.frames[t].parent);
+        const bool from_result = parent < (uint32_t)c.B;
+        const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
+        const bool leaf = l == LEAF_MARK;
+        float dl[MAX_CLASSES];
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
+        const float* g = c.dhp + (size_t)t * S;
+        const float* st = c.arena + (size_t)t * S;
+        float* gt = c.gates + (size_t)t * c.G;
+        for (int j = lane; j < H; j += 32) {
+            float dh = from_result ? 0.f : __ldcg(&g[j]);
+            const float dc_in = from_result ? 0.f : __ldcg(&g[H + j]);
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
+            const float tc = tanhf(__ldcg(&st[H + j]));
+            if (leaf) {
+                const float gi = __ldcg(&gt[j]), go = __ldcg(&gt[H + j]), gu = __ldcg(&gt[2 * H + j]);
+                const float dc = dc_in + dh * go * (1.f - tc * tc);
+                gt[j] = dc * gu * gi * (1.f - gi);
+                gt[H + j] = dh * tc * go * (1.f - go);
+                gt[2 * H + j] = dc * gi * (1.f - gu * gu);
+            } else {
+                const float gi = __ldcg(&gt[j]), fl = __ldcg(&gt[H + j]), fr = __ldcg(&gt[2 * H + j]);
+                const float go = __ldcg(&gt[3 * H + j]), gu = __ldcg(&gt[4 * H + j]);
+                const float cl = __ldcg(&c.arena[(size_t)l * S + H + j]), cr = __ldcg(&c.arena[(size_t)r * S + H + j]);
+                const float dc = dc_in + dh * go * (1.f - tc * tc);
+                gt[j] = dc * gu * gi * (1.f - gi);
+                gt[H + j] = dc * cl * fl * (1.f - fl);
+                gt[2 * H + j] = dc * cr * fr * (1.f - fr);
+                gt[3 * H + j] = dh * tc * go * (1.f - go);
+                gt[4 * H + j] = dc * gi * (1.f - gu * gu);
+                c.dhp[(size_t)l * S + H + j] = dc * fl;
+                c.dhp[(size_t)r * S + H + j] = dc * fr;
+            }
+        }
+        if (lane == 0) backward_enqueue(c, wave, t, leaf, l, r);
+    }
+}
+
+// B: [dh_l ; dh_r] = W^T dg for the cells all_cells[first, first + n).  dg of cell t is the row
+//    A[t * lda .. + Kdim): dz (TreeRNN, Kdim = H) or the five gate gradients (TreeLSTM, Kdim = 5H).
+__device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, uint32_t n_items,
+                                       const float* A, int lda, int Kdim) {
+    const int H = c.H, K2 = 2 * c.H, S = c.S;
     const int tiles_m = (n_items + TM - 1) / TM, tiles_n = (K2 + TN - 1) / TN;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int arow_l = threadIdx.x / 4, ak = (threadIdx.x % 4) * 4;     // A loader: row, 4 consecutive k
@@ -145,16 +197,17 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
         const int row0 = tm * TM, col0 = tn * TN;
         const int arow = row0 + arow_l;
         const float* dz = nullptr;
-        if (arow < (int)n_items) dz = c.dhp + (size_t)__ldcg(&c.all_cells[first + arow]) * H;
+        if (arow < (int)n_items) dz = A + (size_t)__ldcg(&c.all_cells[first + arow]) * lda;
         float acc[4][4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        for (int k0 = 0; k0 < H; k0 += TK) {
+        for (int k0 = 0; k0 < Kdim; k0 += TK) {
             float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-            if (dz && k0 + ak < H) a = ldcg4(dz + k0 + ak);
-            if (k0 + bk < H && col0 + bn < K2) b = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)(k0 + bk) * K2 + col0 + bn));
+            if (dz && k0 + ak < Kdim) a = ldcg4(dz + k0 + ak);
+            if (k0 + bk < Kdim && col0 + bn < K2)
+                b = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)(k0 + bk) * K2 + col0 + bn));
             __syncthreads();
             sm.As[ak + 0][arow_l] = a.x; sm.As[ak + 1][arow_l] = a.y; sm.As[ak + 2][arow_l] = a.z; sm.As[ak + 3][arow_l] = a.w;
             *reinterpret_cast<float4*>(&sm.Bs[bk][bn]) = b;
@@ -170,7 +223,7 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
                     const uint32_t t = __ldcg(&c.all_cells[first + row]);
                     const uint32_t child = col < H ? __ldcg(&c.op_l[t]) : __ldcg(&c.op_r[t]);
                     const int cc = col < H ? col : col - H;
-                    *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + cc) =
+                    *reinterpret_cast<float4*>(c.dhp + (size_t)child * S + cc) =
                         make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
                 }
             }
@@ -189,11 +242,13 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
             break;
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->bq_count[(wave + 2) % 3] = 0;
-        backward_frames(c, wave, n);
+        if (c.lstm) lstm_backward_frames(c, wave, n);
+        else backward_frames(c, wave, n);
         if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
-            backward_operand_tiles(c, gsm, first, end - first);
+            if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
+            else backward_operand_tiles(c, gsm, first, end - first, c.dhp, c.H, c.H);
             first = end;
             if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
         }
@@ -202,15 +257,28 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
 }
 
 // ------------------------------------------- parameter gradients (post pass)
-// dW[j][k] = sum over cells t of dz_t[j] * x_t[k],  x_t = [state(l_t) ; state(r_t)];  split over the cells
-__global__ void __launch_bounds__(256) rdf_dw_kernel(const DevCtx c, int tiles_m, int tiles_n, uint32_t chunk) {
+// out[m][n] = sum over the listed invocations t of A_t[m] * B_t[n]   (split over the list)
+//   A_t = A + t * lda (M values: dz, or gate gradients)
+//   mode 0: B_t = [h(l_t) ; h(r_t)]  (N = 2H)   -> dW
+//   mode 1: B_t = E[tok_t]           (N = D)    -> dW_x (TreeLSTM leaves)
+struct OuterArgs {
+    const uint32_t* list;
+    const uint32_t* count;
+    const float* A;
+    int lda, M, N, mode;
+    float* out;
+    int tiles_m, tiles_n;
+    uint32_t chunk;
+};
+
+__global__ void __launch_bounds__(256) rdf_outer_kernel(const DevCtx c, const OuterArgs a) {
     __shared__ GemmSmem sm;
-    const uint32_t n_cells = c.ctl->all_cells;
-    const int tile = blockIdx.x % (tiles_m * tiles_n), split = blockIdx.x / (tiles_m * tiles_n);
-    const uint32_t t_begin = (uint32_t)split * chunk, t_end = min(n_cells, t_begin + chunk);
+    const uint32_t n_items = *a.count;
+    const int tile = blockIdx.x % (a.tiles_m * a.tiles_n), split = blockIdx.x / (a.tiles_m * a.tiles_n);
+    const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_items, t_begin + a.chunk);
     if (t_begin >= t_end) return;
-    const int H = c.H, K2 = 2 * c.H;
-    const int tm = tile / tiles_n, tn = tile % tiles_n;
+    const int H = c.H, S = c.S;
+    const int tm = tile / a.tiles_n, tn = tile % a.tiles_n;
     const int row0 = tm * TM, col0 = tn * TN;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int lk = threadIdx.x / 16, l4 = (threadIdx.x % 16) * 4;
@@ -220,43 +288,49 @@ __global__ void __launch_bounds__(256) rdf_dw_kernel(const DevCtx c, int tiles_m
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
     for (uint32_t t0 = t_begin; t0 < t_end; t0 += TK) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        float4 av = make_float4(0.f, 0.f, 0.f, 0.f), bv = av;
         if (t0 + lk < t_end) {
-            const uint32_t t = c.all_cells[t0 + lk];
-            if (row0 + l4 < H) a = *reinterpret_cast<const float4*>(c.dhp + (size_t)t * H + row0 + l4);
+            const uint32_t t = a.list[t0 + lk];
+            if (row0 + l4 < a.M) av = *reinterpret_cast<const float4*>(a.A + (size_t)t * a.lda + row0 + l4);
             const int col = col0 + l4;
-            if (col < K2) {
-                const uint32_t src = col < H ? c.op_l[t] : c.op_r[t];
-                b = *reinterpret_cast<const float4*>(c.arena + (size_t)src * H + (col < H ? col : col - H));
+            if (col < a.N) {
+                if (a.mode == 0) {
+                    const uint32_t src = col < H ? c.op_l[t] : c.op_r[t];
+                    bv = *reinterpret_cast<const float4*>(c.arena + (size_t)src * S + (col < H ? col : col - H));
+                } else {
+                    bv = __ldg(reinterpret_cast<const float4*>(c.E + (size_t)c.op_r[t] * c.D + col));
+                }
             }
         }
         __syncthreads();
-        *reinterpret_cast<float4*>(&sm.As[lk][l4]) = a;
-        *reinterpret_cast<float4*>(&sm.Bs[lk][l4]) = b;
+        *reinterpret_cast<float4*>(&sm.As[lk][l4]) = av;
+        *reinterpret_cast<float4*>(&sm.Bs[lk][l4]) = bv;
         __syncthreads();
         gemm_tile_step(sm, tx, ty, acc);
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int row = row0 + ty * 4 + i;
-        if (row >= H) continue;
+        if (row >= a.M) continue;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int col = col0 + tx * 4 + j;
-            if (col < K2) atomicAdd(&c.dW[(size_t)row * K2 + col], acc[i][j]);
+            if (col < a.N) atomicAdd(&a.out[(size_t)row * a.N + col], acc[i][j]);
         }
     }
 }
 
-// db[j] = sum over cells of dz_t[j]
-__global__ void __launch_bounds__(256) rdf_db_kernel(const DevCtx c) {
-    const uint32_t n_cells = c.ctl->all_cells;
-    const uint32_t per = (n_cells + gridDim.x - 1) / gridDim.x;
-    const uint32_t t0 = blockIdx.x * per, t1 = min(n_cells, t0 + per);
-    for (int j = threadIdx.x; j < c.H; j += blockDim.x) {
+// out[m] = sum over the listed invocations of A_t[m]   (bias gradients)
+__global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, const uint32_t* count, const float* A,
+                                                         int lda, int M, float* out) {
+    const uint32_t n = *count;
+    const uint32_t per = (n + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = blockIdx.x * per, t1 = min(n, t0 + per);
+    if (t0 >= t1) return;
+    for (int j = threadIdx.x; j < M; j += blockDim.x) {
         float s = 0.f;
-        for (uint32_t i = t0; i < t1; ++i) s += c.dhp[(size_t)c.all_cells[i] * c.H + j];
-        if (t1 > t0) atomicAdd(&c.db[j], s);
+        for (uint32_t i = t0; i < t1; ++i) s += A[(size_t)list[i] * lda + j];
+        atomicAdd(&out[j], s);
     }
 }
 
@@ -272,7 +346,7 @@ __global__ void __launch_bounds__(256) rdf_dws_kernel(const DevCtx c) {
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) s[k] = 0.f;
         for (uint32_t f = f0; f < f1; ++f) {
-            const float hj = c.arena[(size_t)f * H + j];
+            const float hj = c.arena[(size_t)f * c.S + j];
             const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8);
             const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8 + 4);
             s[0] = fmaf(d0.x, hj, s[0]); s[1] = fmaf(d0.y, hj, s[1]); s[2] = fmaf(d0.z, hj, s[2]); s[3] = fmaf(d0.w, hj, s[3]);
@@ -289,7 +363,7 @@ __global__ void __launch_bounds__(256) rdf_dws_kernel(const DevCtx c) {
     }
 }
 
-// dE[tok] += dh of every leaf invocation that read row tok
+// TreeRNN: dE[tok] += dh of every leaf invocation that read row tok
 __global__ void __launch_bounds__(256) rdf_de_kernel(const DevCtx c) {
     const uint32_t n = c.ctl->all_leaves;
     const int lane = threadIdx.x % 32;
@@ -301,13 +375,76 @@ __global__ void __launch_bounds__(256) rdf_de_kernel(const DevCtx c) {
     }
 }
 
+// TreeLSTM: dE[tok_t] += W_x^T dg_t for every leaf t (dg_t = the 3H gate gradients)
+__global__ void __launch_bounds__(256) rdf_de_lstm_kernel(const DevCtx c, int tiles_n) {
+    __shared__ GemmSmem sm;
+    const uint32_t n_items = c.ctl->all_leaves;
+    const int D = c.D, Kdim = 3 * c.H;
+    const int tiles_m = (n_items + TM - 1) / TM;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int arow_l = threadIdx.x / 4, ak = (threadIdx.x % 4) * 4;
+    const int bk = threadIdx.x / 16, bn = (threadIdx.x % 16) * 4;
+    for (int tile = blockIdx.x; tile < tiles_m * tiles_n; tile += gridDim.x) {
+        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        const int row0 = tm * TM, col0 = tn * TN;
+        const int arow = row0 + arow_l;
+        const float* dg = arow < (int)n_items ? c.gates + (size_t)c.all_leaves[arow] * c.G : nullptr;
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int k0 = 0; k0 < Kdim; k0 += TK) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            if (dg && k0 + ak < Kdim) a = *reinterpret_cast<const float4*>(dg + k0 + ak);
+            if (k0 + bk < Kdim && col0 + bn < D)
+                b = __ldg(reinterpret_cast<const float4*>(c.W_x + (size_t)(k0 + bk) * D + col0 + bn));
+            __syncthreads();
+            sm.As[ak + 0][arow_l] = a.x; sm.As[ak + 1][arow_l] = a.y; sm.As[ak + 2][arow_l] = a.z; sm.As[ak + 3][arow_l] = a.w;
+            *reinterpret_cast<float4*>(&sm.Bs[bk][bn]) = b;
+            __syncthreads();
+            gemm_tile_step(sm, tx, ty, acc);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = row0 + ty * 4 + i;
+            if (row >= (int)n_items) continue;
+            const uint32_t tok = c.op_r[c.all_leaves[row]];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int col = col0 + tx * 4 + j;
+                if (col < D) atomicAdd(&c.dE[(size_t)tok * D + col], acc[i][j]);
+            }
+        }
+    }
+}
+
 // --------------------------------------------------------------------- host
+namespace {
+OuterArgs outer_args(const uint32_t* list, const uint32_t* count, const float* A, int lda, int M, int N, int mode,
+                     float* out, long long max_items, int grid) {
+    OuterArgs a;
+    a.list = list; a.count = count; a.A = A; a.lda = lda; a.M = M; a.N = N; a.mode = mode; a.out = out;
+    a.tiles_m = (M + TM - 1) / TM;
+    a.tiles_n = (N + TN - 1) / TN;
+    const int tiles = a.tiles_m * a.tiles_n;
+    const long long splits = std::max<long long>(1, std::min<long long>((max_items + 255) / 256, (4 * grid) / tiles + 1));
+    uint32_t chunk = (uint32_t)((max_items + splits - 1) / splits);
+    a.chunk = (chunk + TK - 1) / TK * TK;
+    return a;
+}
+int outer_blocks(const OuterArgs& a, long long max_items) {
+    return a.tiles_m * a.tiles_n * (int)((max_items + a.chunk - 1) / a.chunk);
+}
+}  // namespace
+
 extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
                         rdf_param_grads* grads, void* workspace, size_t workspace_bytes, void* stream_v) {
     int rc = rdf_check_common(g, in, params, out, workspace);
     if (rc != RDF_OK) return rc;
     if (!g->has_vector_ops || !g->has_loss) return RDF_ERR_UNSUPPORTED;
     if (!grads || !grads->dE || !grads->dW || !grads->db || !grads->dW_s || !grads->db_s) return RDF_ERR_BAD_ARG;
+    if (g->has_lstm && (!grads->dW_x || !grads->db_x)) return RDF_ERR_BAD_ARG;
     if (!params->W_s || !params->b_s || !in->label || !out->loss) return RDF_ERR_BAD_ARG;
     if (params->n_classes < 1 || params->n_classes > MAX_CLASSES) return RDF_ERR_BAD_ARG;
     Layout L;
@@ -323,13 +460,20 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_fill_ctx(g, in, params, out, ws, L, S, c);
     c.dE = grads->dE; c.dW = grads->dW; c.db = grads->db; c.dW_x = grads->dW_x; c.db_x = grads->db_x;
     c.dW_s = grads->dW_s; c.db_s = grads->db_s;
-    const int H = params->H;
+    const bool lstm = g->has_lstm;
+    if (lstm) c.gates = reinterpret_cast<float*>(ws + L.gates);
+    const int H = params->H, D = params->D;
+    const int MW = lstm ? 5 * H : H;          // rows of W
     // gradients are sums: start from zero
-    CUDA_OK(cudaMemsetAsync(grads->dE, 0, (size_t)params->V * params->D * sizeof(float), stream));
-    CUDA_OK(cudaMemsetAsync(grads->dW, 0, (size_t)H * 2 * H * sizeof(float), stream));
-    CUDA_OK(cudaMemsetAsync(grads->db, 0, (size_t)H * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->dE, 0, (size_t)params->V * D * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->dW, 0, (size_t)MW * 2 * H * sizeof(float), stream));
+    CUDA_OK(cudaMemsetAsync(grads->db, 0, (size_t)MW * sizeof(float), stream));
     CUDA_OK(cudaMemsetAsync(grads->dW_s, 0, (size_t)params->n_classes * H * sizeof(float), stream));
     CUDA_OK(cudaMemsetAsync(grads->db_s, 0, (size_t)params->n_classes * sizeof(float), stream));
+    if (lstm) {
+        CUDA_OK(cudaMemsetAsync(grads->dW_x, 0, (size_t)3 * H * D * sizeof(float), stream));
+        CUDA_OK(cudaMemsetAsync(grads->db_x, 0, (size_t)3 * H * sizeof(float), stream));
+    }
     rc = rdf_launch_forward(g, in, out, ws, L, S, c, stream);
     if (rc != RDF_OK) return rc;
     // loss head over every retained invocation
@@ -344,18 +488,24 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
     rdf_mark(S, 4, stream);
     // parameter gradients
-    const int tiles_m = (H + TM - 1) / TM, tiles_n = (2 * H + TN - 1) / TN;
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
-    int splits = (int)std::max<long long>(1, std::min<long long>((max_cells + 255) / 256, (4 * S->grid) / (tiles_m * tiles_n) + 1));
-    uint32_t chunk = (uint32_t)((max_cells + splits - 1) / splits);
-    chunk = (chunk + TK - 1) / TK * TK;
-    rdf_dw_kernel<<<tiles_m * tiles_n * splits, 256, 0, stream>>>(c, tiles_m, tiles_n, chunk);
+    const long long max_leaves = std::max<long long>(1, in->max_invocations);
+    const float* dgA = lstm ? c.gates : c.dhp;
+    const int lda = lstm ? c.G : H;
+    OuterArgs aw = outer_args(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, 2 * H, 0, grads->dW, max_cells, S->grid);
+    rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw);
+    if (lstm) {
+        OuterArgs ax = outer_args(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, D, 1, grads->dW_x, max_leaves, S->grid);
+        rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
+    }
     rdf_mark(S, 5, stream);
-    rdf_db_kernel<<<S->grid, 256, 0, stream>>>(c);
+    rdf_colsum_kernel<<<S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
+    if (lstm) rdf_colsum_kernel<<<S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
     rdf_mark(S, 6, stream);
     rdf_dws_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
     rdf_mark(S, 7, stream);
-    rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
+    if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
+    else rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
     rdf_mark(S, 8, stream);
     CUDA_OK(cudaGetLastError());
     return RDF_OK;

@@ -29,29 +29,29 @@ def graph(cell="rnn", with_loss=False):
     return rdf.Graph(fs, r, rdf.TAGS_FRAME)
 
 
-def check_forward(cfg, compute=rdf.F32, trees=None):
+def check_forward(cfg, compute=rdf.F32, trees=None, cell="rnn"):
     tb, p = cfg["trees"], cfg["params"]
-    g = graph()
+    g = graph(cell)
     h, _ = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), compute)
     h = h.cpu().numpy()
     st = g.stats()
     assert st["invocations"] == tb.N and st["cells"] == tb.n_cells and st["leaves"] == tb.N - tb.n_cells
     trees = list(range(tb.B)) if trees is None else trees
-    want = direct.forward(tb, p, "rnn", trees=trees)
+    want = direct.forward(tb, p, cell, trees=trees)
     assert relerr(h[trees], want) <= TOL[compute]
     return st
 
 
-def check_grad(cfg, compute=rdf.F32, workers=1):
+def check_grad(cfg, compute=rdf.F32, workers=1, cell="rnn"):
     tb, p = cfg["trees"], cfg["params"]
-    g = graph(with_loss=True)
+    g = graph(cell, with_loss=True)
     loss, h, grads = g.grad_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), compute)
     st = g.stats()
     assert st["status"] == 0 and st["invocations"] == tb.N
     if workers > 1:
-        want_loss, G, roots = direct.loss_and_grad_pool(tb, p, "rnn", workers=workers)
+        want_loss, G, roots = direct.loss_and_grad_pool(tb, p, cell, workers=workers)
     else:
-        want_loss, G, roots = direct.loss_and_grad(tb, p, "rnn")
+        want_loss, G, roots = direct.loss_and_grad(tb, p, cell)
     tol = TOL[compute]
     assert relerr(h.cpu().numpy(), roots) <= tol
     assert abs(loss.item() - want_loss) <= tol * abs(want_loss)
@@ -146,6 +146,37 @@ def test_treernn_config3_full_size():
     compute = rdf.BF16
     st, errs = check_grad(cfg, compute, workers=WORKERS)
     print("config 3 errors:", errs, st)
+
+
+def _lstm_cfg(B, V, H, seed=5):
+    cfg = workloads.config(4, B=B, V=V, H=H)
+    p = workloads.treelstm_params(seed, V, H, H)
+    rng = np.random.default_rng(seed)
+    for k in ("b", "b_x", "b_s"):
+        p[k] = (0.1 * rng.standard_normal(p[k].shape)).astype(np.float32)
+    cfg["params"] = p
+    return cfg
+
+
+def test_treelstm_small_and_tiny():
+    rng = np.random.default_rng(2)
+    for Ls in ([1], [2], [1, 3, 1, 2]):
+        tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, L) for L in Ls], 7, vocab=50)
+        cfg = {"trees": tb, "params": _lstm_cfg(1, 50, 8)["params"]}
+        check_forward(cfg, cell="lstm")
+        check_grad(cfg, cell="lstm")
+    check_forward(_lstm_cfg(96, 500, 64), cell="lstm")
+    check_grad(_lstm_cfg(96, 500, 64), cell="lstm")
+
+
+def test_treelstm_ragged_hidden_size():
+    check_grad(_lstm_cfg(48, 700, 300), cell="lstm")
+
+
+def test_treelstm_config4_full_size():
+    """Binary TreeLSTM, 8192 trees, H = 300, fwd + bwd at full size against the pooled oracle."""
+    st, errs = check_grad(workloads.config(4), rdf.BF16, workers=WORKERS, cell="lstm")
+    print("config 4 errors:", errs, st)
 
 
 def test_depth_stress_config5_forward_sampled():
