@@ -287,7 +287,12 @@ def loss_and_grad(tb, params, cell="rnn", trees=None):
 # --------------------------------------------------------------------------
 def _pool_job(args):
     tb, params, cell, trees = args
-    return loss_and_grad(tb, params, cell, trees)
+    try:                                  # one BLAS thread per worker: the pool already uses every core
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            return loss_and_grad(tb, params, cell, trees)
+    except ImportError:
+        return loss_and_grad(tb, params, cell, trees)
 
 
 def loss_and_grad_pool(tb, params, cell="rnn", workers=8, trees=None):
