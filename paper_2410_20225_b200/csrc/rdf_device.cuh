@@ -7,6 +7,7 @@
 // the non-coherent L1.
 #pragma once
 #include <cooperative_groups.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -99,6 +100,10 @@ struct DevCtx {
     float*    arena;              // [frame_cap, S] fp32 states: S = H (TreeRNN h) or 2H (TreeLSTM h then c)
     float*    gates;              // TreeLSTM under rdf_grad: [frame_cap, G] activated gates, later their gradients
     int       S, G, lstm;
+    // tensor-core path (bf16 operands): bf16 copy of the states with row stride Hp, packed weights
+    __nv_bfloat16* arena_bf;
+    __nv_bfloat16* Wp;
+    int       Hp, use_tc;
     // parameters
     int H, D, V, n_classes, compute;
     const float *E, *W, *b, *W_x, *b_x, *W_s, *b_s;

@@ -11,6 +11,7 @@
 
 #include "rdf_exec.h"
 #include "rdf_lstm.cuh"
+#include "rdf_tc.cuh"
 
 // ===========================================================================
 // S phase: the segment interpreter
@@ -273,7 +274,12 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
     __shared__ SharedProgram sp;
     __shared__ LstmSmem tile_smem;                                   // the TreeRNN tiles use its first part
     GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
+    extern __shared__ unsigned char dyn_smem[];                      // operand stages of the tensor-core path
+    __shared__ uint32_t tmem_slot;
+    __shared__ __align__(8) uint64_t tc_mbars[2];
+    TcState tc;
     load_program(c, sp);
+    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
     for (;; ++wave) {
@@ -298,7 +304,10 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
         const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
         if (n_leaf | n_cell) {
-            if (c.lstm) {
+            if (c.use_tc) {
+                if (n_leaf) tc_leaf_rows(c, min(n_leaf, c.work_cap));
+                if (n_cell) tc_rnn_cell_tiles(c, tc, min(n_cell, c.work_cap));
+            } else if (c.lstm) {
                 if (n_leaf) lstm_forward_tiles<3>(c, tile_smem, min(n_leaf, c.work_cap));
                 if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
             } else {
@@ -308,6 +317,7 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
             if (!grid_barrier(c, &c.ctl->bar, generation)) break;
         }
     }
+    if (c.use_tc) tc_teardown(tc);
     // ---- statistics
     atomicAdd(&c.ctl->invocations, (unsigned long long)st.invocations);
     atomicAdd(&c.ctl->tokens, (unsigned long long)st.tokens);
@@ -392,6 +402,10 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     const size_t S = g->has_lstm ? 2 * (size_t)H : (size_t)H;
     L.arena = P.take<float>(vf * S);
     L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
+    L.Hp = (H + 63) / 64 * 64;
+    L.use_tc = g->has_vector_ops && !g->has_lstm && params->compute == RDF_BF16 && L.Hp <= TC_NMAX;
+    L.arena_bf = P.take<__nv_bfloat16>(L.use_tc ? vf * L.Hp : 0);
+    L.wp = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.Hp * 2 * L.Hp : 0);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
@@ -420,7 +434,8 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     CUDA_OK(cudaDeviceGetAttribute(&S->clock_khz, cudaDevAttrClockRate, dev));
     if (!coop) return RDF_ERR_CUDA;
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, 0));
+    CUDA_OK(cudaFuncSetAttribute(rdf_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, TC_SMEM_BYTES));
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
     S->device = dev;
@@ -464,6 +479,9 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.S = g->has_lstm ? 2 * params->H : params->H;
         c.G = 5 * params->H;
         c.gates = nullptr;                 // set by rdf_grad for the TreeLSTM
+        c.use_tc = L.use_tc; c.Hp = L.Hp;
+        c.arena_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.arena_bf);
+        c.Wp = reinterpret_cast<__nv_bfloat16*>(ws + L.wp);
     } else {
         c.y = out->y;
     }
@@ -516,9 +534,14 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
         CUDA_OK(cudaMemcpyAsync(ws + L.consts, g->consts.data(), g->consts.size() * sizeof(int64_t), cudaMemcpyHostToDevice, stream));
     rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
+    if (c.use_tc) {
+        rdf_pack_w_kernel<<<64, 256, 0, stream>>>(c);
+        CUDA_OK(cudaGetLastError());
+    }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args,
+                                        c.use_tc ? TC_SMEM_BYTES : 0, stream));
     if (g->has_vector_ops) {
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());

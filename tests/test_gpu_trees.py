@@ -121,6 +121,19 @@ def test_treernn_grad_ragged_hidden_size():
     check_grad(cfg)
 
 
+@pytest.mark.parametrize("H", [64, 300])
+def test_treernn_bf16_tensor_core_path(H):
+    """bf16 operands on the tensor cores (fp32 accumulation): parameters are bf16-representable,
+    states are rounded to bf16 after every cell; tolerance 2e-2."""
+    cfg = workloads.config(3, B=200, V=900, H=H)
+    check_forward(cfg, rdf.BF16)
+    check_grad(cfg, rdf.BF16)
+    # more than one 128-row tile per wave and a ragged last tile
+    cfg = workloads.config(3, B=700, V=900, H=H)
+    st = check_forward(cfg, rdf.BF16)
+    assert st["cells"] > 3 * 128
+
+
 def test_depth_stress_reduced():
     cfg = workloads.config(5, chains=3, chain_depth=300, perfect=2, perfect_height=7, V=400, H=32)
     st, _ = check_grad(cfg)
