@@ -372,6 +372,7 @@ def main():
         "cpu_baseline": cpu,
         "phase_ms": mean_phase,
         "waves": {"forward": st["waves"], "backward": st["waves_backward"], "widest": st["max_wave_tokens"]},
+        "block0_ms_at_max_clock": {k[7:]: round(st[k] / 1.965e6, 4) for k in st if k.startswith("cycles_")},
     }
     print(json.dumps(line))
     if dist is not None:

@@ -220,6 +220,10 @@ typedef struct {
     uint32_t max_depth;          /* deepest tag (PATH mode) */
     uint64_t cells;              /* batched cell firings */
     uint64_t leaves;             /* batched leaf firings */
+    /* SM clock cycles spent by thread block 0, forward kernel then gradient kernel:
+       token scheduling / per-frame work, batched operators, waiting at grid barriers */
+    uint64_t cycles_schedule, cycles_batch, cycles_barrier;
+    uint64_t cycles_bwd_frames, cycles_bwd_batch, cycles_bwd_barrier;
 } rdf_stats;
 
 /* Bytes of device scratch rdf_eval (want_grad = 0) or rdf_grad (1) needs for

@@ -101,7 +101,9 @@ class rdf_stats(C.Structure):
     _fields_ = [("status", C.c_int32), ("waves", C.c_uint32), ("waves_backward", C.c_uint32),
                 ("max_wave_tokens", C.c_uint32), ("invocations", C.c_uint64), ("tokens", C.c_uint64),
                 ("store_inserts", C.c_uint64), ("store_matches", C.c_uint64), ("store_probes", C.c_uint64),
-                ("max_probe", C.c_uint32), ("max_depth", C.c_uint32), ("cells", C.c_uint64), ("leaves", C.c_uint64)]
+                ("max_probe", C.c_uint32), ("max_depth", C.c_uint32), ("cells", C.c_uint64), ("leaves", C.c_uint64),
+                ("cycles_schedule", C.c_uint64), ("cycles_batch", C.c_uint64), ("cycles_barrier", C.c_uint64),
+                ("cycles_bwd_frames", C.c_uint64), ("cycles_bwd_batch", C.c_uint64), ("cycles_bwd_barrier", C.c_uint64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

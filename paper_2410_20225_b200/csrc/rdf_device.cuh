@@ -63,6 +63,7 @@ struct Control {
     uint32_t bar2;                // barrier counter of the backward kernel
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
+    unsigned long long cyc[6];    // block 0: forward schedule / batch / barrier, backward frames / batch / barrier
     float    loss;
 };
 
@@ -102,7 +103,9 @@ struct DevCtx {
     int       S, G, lstm;
     // tensor-core path (bf16 operands): bf16 copy of the states with row stride Hp, packed weights
     __nv_bfloat16* arena_bf;
-    __nv_bfloat16* Wp;
+    __nv_bfloat16* Wp;            // [Hp, 2Hp]   forward operand
+    __nv_bfloat16* WTp;           // [2Hp, Hp]   gradient operand
+    __nv_bfloat16* dz_bf;         // [frame_cap, Hp] bf16 copy of dz (rdf_grad)
     int       Hp, use_tc;
     // parameters
     int H, D, V, n_classes, compute;

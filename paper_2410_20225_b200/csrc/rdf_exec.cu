@@ -276,12 +276,19 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
     GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     extern __shared__ unsigned char dyn_smem[];                      // operand stages of the tensor-core path
     __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[2];
+    __shared__ __align__(8) uint64_t tc_mbars[TC_STAGES];
+    __shared__ uint4 tc_items[TC_M];
     TcState tc;
     load_program(c, sp);
-    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars);
+    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Wp, 2 * c.Hp, c.Hp / 4, 4);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
+    long long cyc_s = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
+    auto lap = [&](long long& acc) {
+        const long long now = clock64();
+        acc += now - t_mark;
+        t_mark = now;
+    };
     for (;; ++wave) {
         const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
         if (n == 0) break;
@@ -299,14 +306,17 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         const Token* q = c.q[wave & 1];
         for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
             run_token(c, sp, wave, load_token(&q[i]), st);
+        __syncthreads();
+        lap(cyc_s);
         if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        lap(cyc_b);
         // ---- C: the wave's ready batched operators
         const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
         const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
         if (n_leaf | n_cell) {
             if (c.use_tc) {
                 if (n_leaf) tc_leaf_rows(c, min(n_leaf, c.work_cap));
-                if (n_cell) tc_rnn_cell_tiles(c, tc, min(n_cell, c.work_cap));
+                if (n_cell) tc_tiles<true>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
             } else if (c.lstm) {
                 if (n_leaf) lstm_forward_tiles<3>(c, tile_smem, min(n_leaf, c.work_cap));
                 if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
@@ -314,7 +324,10 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
                 if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
                 if (n_cell) rnn_cell_tiles(c, gsm, min(n_cell, c.work_cap));
             }
+            __syncthreads();
+            lap(cyc_c);
             if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+            lap(cyc_b);
         }
     }
     if (c.use_tc) tc_teardown(tc);
@@ -331,6 +344,7 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->waves = wave;
         c.ctl->max_wave_tokens = widest;
+        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[1] = cyc_c; c.ctl->cyc[2] = cyc_b;
     }
 }
 
@@ -403,9 +417,11 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.arena = P.take<float>(vf * S);
     L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
     L.Hp = (H + 63) / 64 * 64;
-    L.use_tc = g->has_vector_ops && !g->has_lstm && params->compute == RDF_BF16 && L.Hp <= TC_NMAX;
+    L.use_tc = g->has_vector_ops && !g->has_lstm && params->compute == RDF_BF16 && L.Hp <= TC_HP_MAX;
     L.arena_bf = P.take<__nv_bfloat16>(L.use_tc ? vf * L.Hp : 0);
     L.wp = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.Hp * 2 * L.Hp : 0);
+    L.wtp = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.Hp * 2 * L.Hp : 0);
+    L.dz_bf = P.take<__nv_bfloat16>(L.use_tc && want_grad ? vf * L.Hp : 0);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
@@ -482,6 +498,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.use_tc = L.use_tc; c.Hp = L.Hp;
         c.arena_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.arena_bf);
         c.Wp = reinterpret_cast<__nv_bfloat16*>(ws + L.wp);
+        c.WTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wtp);
+        c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
     } else {
         c.y = out->y;
     }
@@ -602,6 +620,8 @@ extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
     s->invocations = h.invocations; s->tokens = h.tokens;
     s->store_inserts = h.store_inserts; s->store_matches = h.store_matches; s->store_probes = h.store_probes;
     s->max_probe = h.max_probe; s->max_depth = h.max_depth; s->cells = h.cells; s->leaves = h.leaves;
+    s->cycles_schedule = h.cyc[0]; s->cycles_batch = h.cyc[1]; s->cycles_barrier = h.cyc[2];
+    s->cycles_bwd_frames = h.cyc[3]; s->cycles_bwd_batch = h.cyc[4]; s->cycles_bwd_barrier = h.cyc[5];
     return h.status;
 }
 

@@ -11,6 +11,7 @@
 #include <cstring>
 
 #include "rdf_exec.h"
+#include "rdf_tc.cuh"
 
 static const int MAX_CLASSES = 8;
 
@@ -28,11 +29,14 @@ __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
         float z[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
-        for (int j = lane; j < H; j += 32) {
-            const float hj = h[j];
+        for (int j = lane * 4; j < H; j += 128) {
+            const float4 h4 = *reinterpret_cast<const float4*>(h + j);
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) z[k] = fmaf(__ldg(&c.W_s[k * H + j]), hj, z[k]);
+                if (k < C) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                    z[k] += w.x * h4.x + w.y * h4.y + w.z * h4.z + w.w * h4.w;
+                }
         }
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k)
@@ -119,17 +123,31 @@ __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
         for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
         float* g = c.dhp + (size_t)t * H;
         const float* h = c.arena + (size_t)t * H;
-        for (int j = lane; j < H; j += 32) {
-            float dh = from_result ? 0.f : __ldcg(&g[j]);
+        for (int j = lane * 4; j < H; j += 128) {
+            float4 dh = from_result ? make_float4(0.f, 0.f, 0.f, 0.f) : ldcg4(g + j);
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
+                if (k < C) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                    dh.x = fmaf(w.x, dl[k], dh.x); dh.y = fmaf(w.y, dl[k], dh.y);
+                    dh.z = fmaf(w.z, dl[k], dh.z); dh.w = fmaf(w.w, dl[k], dh.w);
+                }
             if (!leaf) {
-                const float hj = __ldcg(&h[j]);
-                dh *= 1.f - hj * hj;
+                const float4 hv = ldcg4(h + j);
+                dh.x *= 1.f - hv.x * hv.x; dh.y *= 1.f - hv.y * hv.y;
+                dh.z *= 1.f - hv.z * hv.z; dh.w *= 1.f - hv.w * hv.w;
+                if (c.use_tc) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(dh.x, dh.y), hi = __floats2bfloat162_rn(dh.z, dh.w);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                    *reinterpret_cast<uint2*>(c.dz_bf + (size_t)t * c.Hp + j) = pk;
+                }
             }
-            g[j] = dh;
+            *reinterpret_cast<float4*>(g + j) = dh;
         }
+        if (c.use_tc && !leaf)
+            for (int j = H + lane; j < c.Hp; j += 32) c.dz_bf[(size_t)t * c.Hp + j] = __float2bfloat16_rn(0.f);
         if (lane == 0) backward_enqueue(c, wave, t, leaf, l, r);
     }
 }
@@ -233,7 +251,19 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
 
 __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
     __shared__ GemmSmem gsm;
+    extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
+    __shared__ uint32_t tmem_slot;
+    __shared__ __align__(8) uint64_t tc_mbars[TC_STAGES];
+    __shared__ uint4 tc_items[TC_M];
+    TcState tc;
+    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.WTp, c.Hp, c.Hp / 4, 8);
     uint32_t generation = 0, wave = 0, first = 0;
+    long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
+    auto lap = [&](long long& acc) {
+        const long long now = clock64();
+        acc += now - t_mark;
+        t_mark = now;
+    };
     for (;; ++wave) {
         const uint32_t n = ld_volatile_u32(&c.ctl->bq_count[wave % 3]);
         if (n == 0) break;
@@ -244,16 +274,27 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->bq_count[(wave + 2) % 3] = 0;
         if (c.lstm) lstm_backward_frames(c, wave, n);
         else backward_frames(c, wave, n);
+        __syncthreads();
+        lap(cyc_a);
         if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+        lap(cyc_b);
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
-            if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
+            if (c.use_tc) tc_tiles<false>(c, tc, tc_items, first, end - first);
+            else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
             else backward_operand_tiles(c, gsm, first, end - first, c.dhp, c.H, c.H);
             first = end;
+            __syncthreads();
+            lap(cyc_c);
             if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+            lap(cyc_b);
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->waves_backward = wave;
+    if (c.use_tc) tc_teardown(tc);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        c.ctl->waves_backward = wave;
+        c.ctl->cyc[3] = cyc_a; c.ctl->cyc[4] = cyc_c; c.ctl->cyc[5] = cyc_b;
+    }
 }
 
 // ------------------------------------------- parameter gradients (post pass)
@@ -485,7 +526,9 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args, 0, stream));
+    if (c.use_tc) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args,
+                                        c.use_tc ? TC_SMEM_BYTES : 0, stream));
     rdf_mark(S, 4, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
@@ -499,10 +542,10 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
     }
     rdf_mark(S, 5, stream);
-    rdf_colsum_kernel<<<S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
-    if (lstm) rdf_colsum_kernel<<<S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
+    rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
+    if (lstm) rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
     rdf_mark(S, 6, stream);
-    rdf_dws_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+    rdf_dws_kernel<<<16 * S->grid, 128, 0, stream>>>(c);
     rdf_mark(S, 7, stream);
     if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
     else rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);

@@ -1,33 +1,39 @@
-// Tensor-core path (sm_100a: tcgen05 + tensor memory) for the dense cell
-// contraction of the bf16 workloads:
-//     D[128 cells x Np] = A[128 x Kp] * Wp[Np x Kp]^T,   fp32 accumulation in TMEM
-// A rows are the gathered operand states [h_l ; h_r] of the ready cells, in
-// bf16; Wp is the weight matrix packed to bf16 with each half of K padded to a
-// multiple of 64.  Both operands are K-major; they are staged by all threads
-// into shared memory in the 128-byte-swizzled layout the MMA reads (8-row
-// groups of 1024 bytes, 16-byte chunks XOR-ed with the row index), one elected
-// thread issues the MMAs, completion is signalled on an mbarrier by
-// tcgen05.commit, and the epilogue reads the accumulators back with
-// tcgen05.ld.  Every wait is bounded; on expiry the status word is set.
+// Tensor-core path (sm_100a: tcgen05 + tensor memory) for the dense
+// contractions of the bf16 TreeRNN workloads, forward and operand-gradient:
+//
+//   forward :  D[128 cells x NS] = A[128 x 2Hp] * Wp [NS x 2Hp]^T     A row = [h_l ; h_r] (bf16 states, gathered)
+//   backward:  D[128 cells x NS] = A[128 x  Hp] * WTp[NS x  Hp]^T     A row = dz (bf16),  D = slice of [dh_l ; dh_r]
+//
+// Weight-stationary: the packed weight matrix is split along N into slices of
+// NS = Hp / 4 rows; a thread block owns one slice for the whole kernel and
+// keeps it in shared memory (loaded once, <= 100 KB), so per tile only the
+// gathered operand rows move.  A rows are streamed with cp.async through a
+// 4-stage ring of 128-byte-swizzled [128 x 64] bf16 tiles (8-row groups of
+// 1024 bytes, 16-byte chunks XOR-ed with the row index: the K-major layout the
+// MMA reads); one thread issues the tcgen05.mma instructions, tcgen05.commit
+// signals an mbarrier per stage, accumulators live in tensor memory and the
+// epilogue reads them back with tcgen05.ld.  Every wait is bounded.
 #pragma once
 #include <cuda_bf16.h>
 
 #include "rdf_exec.h"
 
-static const int TC_M = 128;          // cells per tile (TMEM lanes)
-static const int TC_KC = 64;          // bf16 elements per staged K chunk = one 128-byte swizzled row
-static const int TC_NMAX = 320;       // widest packed N (TMEM columns used)
-static const int TC_STAGE_A = TC_M * 128;
-static const int TC_STAGE_B = TC_NMAX * 128;
-static const int TC_STAGE = TC_STAGE_A + TC_STAGE_B;            // 57344 bytes, a multiple of 1024
-static const int TC_SMEM_BYTES = 2 * TC_STAGE + 1024;           // two stages + slack to align to 1024
+static const int TC_M = 128;                 // cells per tile (TMEM lanes)
+static const int TC_KC = 64;                 // bf16 elements per staged K chunk = one 128-byte swizzled row
+static const int TC_STAGES = 4;
+static const int TC_A_STAGE = TC_M * 128;    // 16 KB
+static const int TC_HP_MAX = 320;            // widest padded hidden size the resident slice is sized for
+static const int TC_B_MAX = TC_HP_MAX * TC_HP_MAX;                               // (Hp/4) rows x 2Hp x 2 bytes
+static const int TC_SMEM_BYTES = 1024 + TC_B_MAX + TC_STAGES * TC_A_STAGE;       // + slack to align to 1024
+static const int TC_TMEM_COLS = 128;
 
 struct TcState {
     uint32_t tmem_base;      // TMEM address returned by tcgen05.alloc
-    uint32_t stage_addr;     // shared-space address of stage 0 (1024-byte aligned)
-    uint32_t mbar_addr;      // shared-space address of the two mbarriers
-    uint32_t iter;           // K chunks issued so far (stage = iter & 1)
-    unsigned char* stage_ptr;
+    uint32_t b_addr;         // shared-space address of the resident weight slice (1024-byte aligned)
+    uint32_t a_addr;         // shared-space address of A stage 0
+    uint32_t mbar_addr;      // shared-space address of the per-stage mbarriers
+    uint32_t iter;           // K chunks issued so far (stage = iter % TC_STAGES)
+    int      ns, n_split, n_chunks;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -91,23 +97,50 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// One-time set-up per kernel (all threads call it): TMEM allocation by warp 0, mbarriers.
-__device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, uint32_t* tmem_slot, uint64_t* mbars) {
+// 16-byte asynchronous copy global -> shared through L2; `valid == false` writes zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+    const int n = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// byte offset of 16-byte chunk c16 of row r inside a swizzled [rows x 128 bytes] operand tile
+__device__ __forceinline__ uint32_t swz(int r, int c16) {
+    return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
+}
+
+// One-time set-up per kernel (all threads call it): TMEM allocation by warp 0, mbarriers, and the
+// block's resident slice of the packed weights: rows [slice * ns, +ns) of Bp[. x Kp], chunk by chunk.
+__device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, uint32_t* tmem_slot, uint64_t* mbars,
+                                         const __nv_bfloat16* Bp, int Kp, int ns, int n_split) {
     const uint32_t raw = smem_u32(dyn_smem);
     const uint32_t aligned = (raw + 1023u) & ~1023u;
-    tc.stage_addr = aligned;
-    tc.stage_ptr = dyn_smem + (aligned - raw);
+    tc.b_addr = aligned;
+    tc.a_addr = aligned + TC_B_MAX;
     tc.mbar_addr = smem_u32(mbars);
     tc.iter = 0;
+    tc.ns = ns;
+    tc.n_split = n_split;
+    tc.n_chunks = Kp / TC_KC;
     if (threadIdx.x == 0) {
-        mbar_init(tc.mbar_addr, 1);
-        mbar_init(tc.mbar_addr + 8, 1);
+        for (int s = 0; s < TC_STAGES; ++s) mbar_init(tc.mbar_addr + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < 32) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TC_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    const int slice = blockIdx.x % n_split;
+    unsigned char* bp = dyn_smem + (aligned - raw);
+    const int chunk_bytes = ns * 128;
+    for (int p = threadIdx.x; p < tc.n_chunks * ns * 8; p += blockDim.x) {
+        const int kc = p / (ns * 8), q = p % (ns * 8), r = q >> 3, c16 = q & 7;
+        const uint4 v = *reinterpret_cast<const uint4*>(Bp + (size_t)(slice * ns + r) * Kp + kc * TC_KC + c16 * 8);
+        *reinterpret_cast<uint4*>(bp + kc * chunk_bytes + swz(r, c16)) = v;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -118,99 +151,120 @@ __device__ __forceinline__ void tc_teardown(const TcState& tc) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x < 32)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tc.tmem_base) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tc.tmem_base), "n"(TC_TMEM_COLS) : "memory");
 }
 
-// byte offset of 16-byte chunk c16 of row r inside a swizzled [rows x 128 bytes] operand tile
-__device__ __forceinline__ uint32_t swz(int r, int c16) {
-    return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
-}
-
-// TreeRNN cell on tensor cores: state(out) = tanh(W [state(l); state(r)] + b) for n_items ready cells.
-// arena_bf: bf16 states, row stride Hp (a multiple of 64, pad columns zero); Wp: [Np = Hp][Kp = 2 Hp] bf16.
-__device__ void tc_rnn_cell_tiles(const DevCtx& c, TcState& tc, uint32_t n_items) {
-    const int H = c.H, Hp = c.Hp, Kp = 2 * c.Hp, Np = c.Hp;
-    const int n_chunks = Kp / TC_KC, n_half = Np / 2;            // two MMAs of N = Np / 2 per K step
-    const uint32_t idesc = tc_idesc(n_half);
+// One 128-cell tile loop.  FWD = true : cells cell_items[0, n_items); A row = [state(l) ; state(r)] in bf16;
+//                                         epilogue state(out) = tanh(D + b) into both arenas.
+//                          FWD = false: cells all_cells[first, first + n_items); A row = dz in bf16;
+//                                         epilogue writes D into the incoming-gradient rows of the operand frames.
+// s_items: 128 x uint4 of shared memory for the tile's cell records.
+template <bool FWD>
+__device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t first, uint32_t n_items) {
+    const int H = c.H, Hp = c.Hp, ns = tc.ns, n_chunks = tc.n_chunks;
+    const int slice = blockIdx.x % tc.n_split, rg = blockIdx.x / tc.n_split, n_rg = gridDim.x / tc.n_split;
+    if (rg >= n_rg) return;                                    // blocks beyond the last full group sit this out
+    const uint32_t idesc = tc_idesc(ns);
     const int tiles = (n_items + TC_M - 1) / TC_M;
-    const __nv_bfloat16* arena_bf = c.arena_bf;
+    const __nv_bfloat16* Arows = FWD ? c.arena_bf : c.dz_bf;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+    for (int tile = rg; tile < tiles && ok; tile += n_rg) {
         const int row0 = tile * TC_M;
-        for (int kc = 0; kc < n_chunks && ok; ++kc) {
-            const uint32_t s = tc.iter & 1u;
+        if (threadIdx.x < TC_M) {
+            uint4 it = make_uint4(0u, 0u, 0u, 0u);
+            const int row = row0 + threadIdx.x;
+            if (row < (int)n_items) {
+                if (FWD) {
+                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
+                } else {
+                    const uint32_t t = __ldcg(&c.all_cells[first + row]);
+                    it.x = t; it.y = __ldcg(&c.op_l[t]); it.z = __ldcg(&c.op_r[t]);
+                }
+                it.w = 1u;
+            }
+            s_items[threadIdx.x] = it;
+        }
+        __syncthreads();
+        const uint32_t it0 = tc.iter;
+        auto issue = [&](int kc) {
+            const uint32_t g = it0 + kc, s = g % TC_STAGES;
             // the MMAs that last read this stage must have completed
-            if (tc.iter >= 2) ok = mbar_wait(c, tc.mbar_addr + 8 * s, ((tc.iter >> 1) - 1) & 1u);
-            unsigned char* sa = tc.stage_ptr + s * TC_STAGE;
-            unsigned char* sb = sa + TC_STAGE_A;
-            // A chunk: 128 rows x 8 chunks of 16 bytes, gathered from the operand states
+            if (g >= TC_STAGES) ok = mbar_wait(c, tc.mbar_addr + 8 * s, ((g / TC_STAGES) - 1) & 1u) && ok;
             const int koff = kc * TC_KC;
             for (int p = threadIdx.x; p < TC_M * 8; p += blockDim.x) {
                 const int r = p >> 3, c16 = p & 7;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (row0 + r < (int)n_items) {
-                    const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row0 + r]));   // {out, l, r, -}
-                    const uint32_t src = koff < Hp ? it.y : it.z;
-                    const int kk = (koff < Hp ? koff : koff - Hp) + c16 * 8;
-                    v = __ldcg(reinterpret_cast<const uint4*>(arena_bf + (size_t)src * Hp + kk));
-                }
-                *reinterpret_cast<uint4*>(sa + swz(r, c16)) = v;
+                const uint4 it = s_items[r];
+                size_t src;
+                if (FWD) src = (size_t)(koff < Hp ? it.y : it.z) * Hp + (koff < Hp ? koff : koff - Hp) + c16 * 8;
+                else src = (size_t)it.x * Hp + koff + c16 * 8;
+                cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r, c16), Arows + src, it.w != 0u);
             }
-            // B chunk: Np rows of the packed weights
-            for (int p = threadIdx.x; p < Np * 8; p += blockDim.x) {
-                const int r = p >> 3, c16 = p & 7;
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(c.Wp + (size_t)r * Kp + koff + c16 * 8));
-                *reinterpret_cast<uint4*>(sb + swz(r, c16)) = v;
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy writes -> async proxy reads
+            cp_async_commit();
+        };
+        issue(0);
+        if (n_chunks > 1) issue(1); else cp_async_commit();
+        for (int kc = 0; kc < n_chunks; ++kc) {
+            if (kc + 2 < n_chunks) issue(kc + 2); else cp_async_commit();
+            cp_async_wait<2>();                                          // this thread's copies of chunk kc have landed
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> async-proxy reads
             __syncthreads();
             if (threadIdx.x == 0) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = tc.stage_addr + s * TC_STAGE, b_addr = a_addr + TC_STAGE_A;
+                const uint32_t s = (it0 + kc) % TC_STAGES;
+                const uint32_t a = tc.a_addr + s * TC_A_STAGE, b = tc.b_addr + kc * ns * 128;
 #pragma unroll
-                for (int ks = 0; ks < TC_KC / 16; ++ks) {
-                    const uint32_t acc = (kc > 0 || ks > 0) ? 1u : 0u;
-                    const uint64_t ad = tc_desc(a_addr + ks * 32);
-                    tc_mma(tc.tmem_base, ad, tc_desc(b_addr + ks * 32), idesc, acc);
-                    tc_mma(tc.tmem_base + n_half, ad, tc_desc(b_addr + n_half * 128 + ks * 32), idesc, acc);
-                }
+                for (int ks = 0; ks < TC_KC / 16; ++ks)
+                    tc_mma(tc.tmem_base, tc_desc(a + ks * 32), tc_desc(b + ks * 32), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(tc.mbar_addr + 8 * s);
             }
-            ++tc.iter;
         }
-        // accumulators complete when the last commit has arrived
-        if (ok) ok = mbar_wait(c, tc.mbar_addr + 8 * ((tc.iter - 1) & 1u), ((tc.iter - 1) >> 1) & 1u);
+        tc.iter = it0 + n_chunks;
+        // accumulators are complete when the last commit has arrived
+        {
+            const uint32_t g = tc.iter - 1;
+            if (ok) ok = mbar_wait(c, tc.mbar_addr + 8 * (g % TC_STAGES), (g / TC_STAGES) & 1u);
+        }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
-            // epilogue: warp w reads TMEM lanes 32 (w % 4) ..; warps 0-3 take the low half of the columns, 4-7 the high half
+            // warp w reads TMEM lanes 32 (w % 4) ..; warps 0-3 take the first 16-column groups, warps 4-7 the rest
             const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
             const int row = (warp & 3) * 32 + lane;
-            const int cbase = (warp >> 2) * n_half;
-            const bool live = row0 + row < (int)n_items;
-            const uint32_t out = live ? __ldcg(&c.cell_items[row0 + row].out) : 0u;
-            for (int cc = 0; cc < n_half; cc += 16) {
+            const int groups = ns / 16, g_lo = (groups + 1) / 2;
+            const int g_begin = warp < 4 ? 0 : g_lo, g_end = warp < 4 ? g_lo : groups;
+            const uint4 it = s_items[row];
+            const bool live = it.w != 0u;
+            for (int gi = g_begin; gi < g_end; ++gi) {
                 float v[16];
-                tc_ld16(tc.tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cbase + cc), v);
+                tc_ld16(tc.tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(gi * 16), v);
                 if (!live) continue;
-                const int col = cbase + cc;
-                __align__(16) __nv_bfloat16 hb[16];
+                const int col = slice * ns + gi * 16;                       // column of the padded N range
+                if (FWD) {
+                    __align__(16) __nv_bfloat16 hb[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float h = 0.f;
-                    if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
-                    hb[i] = __float2bfloat16_rn(h);
-                    v[i] = __bfloat162float(hb[i]);          // the state every consumer sees is the bf16 value
+                    for (int i = 0; i < 16; ++i) {
+                        float h = 0.f;
+                        if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
+                        hb[i] = __float2bfloat16_rn(h);
+                        v[i] = __bfloat162float(hb[i]);      // the state every consumer sees is the bf16 value
+                    }
+                    uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
+                    dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
+                    dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
+                    float* dstf = c.arena + (size_t)it.x * H + col;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                } else {
+                    const uint32_t child = col < Hp ? it.y : it.z;
+                    const int cc = col < Hp ? col : col - Hp;
+                    float* dst = c.dhp + (size_t)child * H + cc;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        if (cc + i < H) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                 }
-                uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)out * Hp + col);
-                dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
-                dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
-                float* dstf = c.arena + (size_t)out * H + col;
-#pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
             }
         }
-        // TMEM and the stages may be overwritten by the next tile only after everybody has read them
+        // TMEM, the stages and s_items may be overwritten by the next tile only after everybody has read them
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
     }
@@ -226,23 +280,40 @@ __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
         const float* src = c.E + (size_t)it.y * c.D;
         float* dst = c.arena + (size_t)it.x * H;
         __nv_bfloat16* dstb = c.arena_bf + (size_t)it.x * Hp;
-        for (int k = lane; k < Hp; k += 32) {
-            const float v = k < H ? __ldg(src + k) : 0.f;
-            const __nv_bfloat16 b = __float2bfloat16_rn(v);
-            dstb[k] = b;
-            if (k < H) dst[k] = __bfloat162float(b);
+        for (int k = lane * 8; k < Hp; k += 256) {             // 8 elements per lane: 32 bytes in, 16 + 32 bytes out
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; i += 4) {
+                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (k + i < H) t = __ldg(reinterpret_cast<const float4*>(src + k + i));
+                v[i] = t.x; v[i + 1] = t.y; v[i + 2] = t.z; v[i + 3] = t.w;
+            }
+            __align__(16) __nv_bfloat16 hb[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                hb[i] = __float2bfloat16_rn(v[i]);
+                v[i] = __bfloat162float(hb[i]);
+            }
+            *reinterpret_cast<uint4*>(dstb + k) = *reinterpret_cast<const uint4*>(hb);
+#pragma unroll
+            for (int i = 0; i < 8; i += 4)
+                if (k + i < H) *reinterpret_cast<float4*>(dst + k + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
         }
     }
 }
 
-// Wp[j][k'] (bf16): rows j < H are W[j], with the left half of K at k' = k and the right half at k' = Hp + (k - H).
-__global__ void __launch_bounds__(256) rdf_pack_w_kernel(const DevCtx c) {
+// Packed weights (bf16), K halves padded to Hp:
+//   Wp [j][k']  (Hp x 2Hp): forward operand,  Wp[j][half*Hp + kk]  = W[j][half*H + kk]
+//   WTp[c'][j]  (2Hp x Hp): gradient operand, WTp[half*Hp + kk][j] = W[j][half*H + kk]
+static __global__ void __launch_bounds__(256) rdf_pack_w_kernel(const DevCtx c) {
     const int Hp = c.Hp, Kp = 2 * c.Hp, H = c.H;
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < Hp * Kp; idx += gridDim.x * blockDim.x) {
         const int j = idx / Kp, kp = idx % Kp;
         const int half = kp >= Hp, kk = kp - half * Hp;
         float v = 0.f;
         if (j < H && kk < H) v = c.W[(size_t)j * 2 * H + half * H + kk];
-        c.Wp[idx] = __float2bfloat16_rn(v);
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        c.Wp[idx] = b;
+        c.WTp[(size_t)kp * Hp + j] = b;
     }
 }
