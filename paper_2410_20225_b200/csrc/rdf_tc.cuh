@@ -271,7 +271,7 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
 }
 
 // Leaves in bf16 mode: state(slot) = E[tok] in both arenas (pad columns of the bf16 row are zero).
-__device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
+static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
     const int H = c.H, Hp = c.Hp;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
     const int n_warps = gridDim.x * blockDim.x / 32;
