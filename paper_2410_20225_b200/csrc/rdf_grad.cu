@@ -12,6 +12,7 @@
 
 #include "rdf_exec.h"
 #include "rdf_tc.cuh"
+#include "rdf_tc_dw.cuh"
 
 static const int MAX_CLASSES = 8;
 
@@ -97,7 +98,9 @@ __device__ __forceinline__ void backward_enqueue(const DevCtx& c, uint32_t wave,
     if (leaf) {
         c.all_leaves[atomicAdd(&c.ctl->all_leaves, 1u)] = t;
     } else {
-        c.all_cells[atomicAdd(&c.ctl->all_cells, 1u)] = t;
+        const uint32_t idx = atomicAdd(&c.ctl->all_cells, 1u);
+        c.all_cells[idx] = t;
+        if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
         const uint32_t at = atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u);
         uint32_t* qn = c.bq[(wave + 1) & 1];
         qn[at] = l;
@@ -535,8 +538,19 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     const long long max_leaves = std::max<long long>(1, in->max_invocations);
     const float* dgA = lstm ? c.gates : c.dhp;
     const int lda = lstm ? c.G : H;
-    OuterArgs aw = outer_args(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, 2 * H, 0, grads->dW, max_cells, S->grid);
-    rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw);
+    if (c.use_tc) {
+        // 128 x 128 tiles of the padded [Hp x 2Hp] gradient, the cells split over the remaining blocks
+        const int tiles_m = (c.Hp + 127) / 128, tiles_n = (2 * c.Hp + 127) / 128, n_tiles = tiles_m * tiles_n;
+        const int splits = std::max(1, S->grid / n_tiles);
+        uint32_t chunk = (uint32_t)((max_cells + splits - 1) / splits);
+        chunk = (chunk + DW_KT - 1) / DW_KT * DW_KT;
+        const int blocks = n_tiles * (int)((max_cells + chunk - 1) / chunk);
+        CUDA_OK(cudaFuncSetAttribute(rdf_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BYTES));
+        rdf_dw_tc_kernel<<<blocks, 256, DW_SMEM_BYTES, stream>>>(c, tiles_n, n_tiles, chunk, 8192u, 1024u);
+    } else {
+        OuterArgs aw = outer_args(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, 2 * H, 0, grads->dW, max_cells, S->grid);
+        rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw);
+    }
     if (lstm) {
         OuterArgs ax = outer_args(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, D, 1, grads->dW_x, max_leaves, S->grid);
         rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);

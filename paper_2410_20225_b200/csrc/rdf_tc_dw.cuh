@@ -1,0 +1,131 @@
+// Weight gradient of the TreeRNN cell on tensor cores:
+//     dW[j][k] = sum over cells t of dz_t[j] * x_t[k],      x_t = [h(l_t) ; h(r_t)]
+// The contraction runs over the cells, and both operands are stored with the
+// contracted index outermost (dz_bf[t][j], arena_bf[.][k]): the "MN-major"
+// operand form.  A stage holds 64 cells: for A, two 64-wide groups of j, for B
+// two 64-wide groups of k, each as 8 atoms of (8 cells x 128 bytes) with the
+// 128-byte swizzle.  Each thread block owns one 128 x 128 tile of dW and a
+// range of the cells (split-K); partial tiles are added to dW with atomics.
+#pragma once
+#include "rdf_tc.cuh"
+
+static const int DW_KT = 64;                          // cells per stage
+static const int DW_HALF = DW_KT * 256;               // 16 KB: one operand of a stage
+static const int DW_STAGE = 2 * DW_HALF;
+static const int DW_STAGES = 4;
+static const int DW_SMEM_BYTES = 1024 + DW_STAGES * DW_STAGE;
+
+// MN-major operand descriptor: atoms of 64 elements (128 bytes) along M/N by 8 along K;
+// lbo = byte distance between atoms along M/N, sbo = between atoms along K.
+__device__ __forceinline__ uint64_t tc_desc_mn(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int tiles_n, int n_tiles, uint32_t chunk,
+                                                           uint32_t lbo, uint32_t sbo) {
+    extern __shared__ unsigned char dyn_smem[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ __align__(8) uint64_t mbars[DW_STAGES];
+    __shared__ uint4 s_ops[DW_STAGES][DW_KT];
+    const uint32_t n_cells = c.ctl->all_cells;
+    const int tile = blockIdx.x % n_tiles, split = blockIdx.x / n_tiles;
+    const uint32_t t_begin = (uint32_t)split * chunk, t_end = min(n_cells, t_begin + chunk);
+    if (t_begin >= t_end) return;                                  // the whole block leaves before any set-up
+    const int H = c.H, Hp = c.Hp, K2p = 2 * c.Hp;
+    const int m0 = (tile / tiles_n) * 128, n0 = (tile % tiles_n) * 128;
+    const int n_chunks = (int)((t_end - t_begin + DW_KT - 1) / DW_KT);
+
+    const uint32_t raw = smem_u32(dyn_smem);
+    const uint32_t stage0 = (raw + 1023u) & ~1023u;
+    const uint32_t mbar = smem_u32(mbars);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < DW_STAGES; ++s) mbar_init(mbar + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;" ::"r"(smem_u32(&tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    auto load_ops = [&](int kc) {
+        if (threadIdx.x < DW_KT) {
+            const uint32_t idx = t_begin + kc * DW_KT + threadIdx.x;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (idx < t_end) v = *reinterpret_cast<const uint4*>(&c.cell_ops[idx]);     // {t, l, r, 1}
+            s_ops[kc % DW_STAGES][threadIdx.x] = v;
+        }
+    };
+    for (int kc = 0; kc < 3 && kc < n_chunks; ++kc) load_ops(kc);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+    const uint32_t idesc = tc_idesc(128) | (1u << 15) | (1u << 16);        // both operands MN-major
+
+    bool ok = true;
+    auto issue = [&](int kc) {
+        const uint32_t s = kc % DW_STAGES;
+        if (kc >= DW_STAGES) ok = mbar_wait(c, mbar + 8 * s, ((kc / DW_STAGES) - 1) & 1u) && ok;
+        const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
+        for (int p = threadIdx.x; p < DW_KT * 16; p += blockDim.x) {
+            const int tr = p >> 4, q = p & 15, atom = q >> 3, c16 = q & 7;
+            const uint4 it = s_ops[s][tr];
+            const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
+            const int m = m0 + atom * 64 + c16 * 8;
+            cp_async16(a_st + off, c.dz_bf + (size_t)it.x * Hp + (m < Hp ? m : 0), it.w != 0u && m < Hp);
+            const int n = n0 + atom * 64 + c16 * 8;
+            const bool nv = it.w != 0u && n < K2p;
+            const size_t src = n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (nv ? n - Hp : 0);
+            cp_async16(b_st + off, c.arena_bf + src, nv);
+        }
+        cp_async_commit();
+    };
+    issue(0);
+    if (n_chunks > 1) issue(1); else cp_async_commit();
+    for (int kc = 0; kc < n_chunks; ++kc) {
+        if (kc + 3 < n_chunks) load_ops(kc + 3);
+        if (kc + 2 < n_chunks) issue(kc + 2); else cp_async_commit();
+        cp_async_wait<2>();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t s = kc % DW_STAGES;
+            const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
+#pragma unroll
+            for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 cells = two K atoms = 2048 bytes per step
+                tc_mma(tmem, tc_desc_mn(a_st + ks * 2048, lbo, sbo), tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc,
+                       (kc > 0 || ks > 0) ? 1u : 0u);
+            tc_commit(mbar + 8 * s);
+        }
+    }
+    {
+        const uint32_t g = n_chunks - 1;
+        if (ok) ok = mbar_wait(c, mbar + 8 * (g % DW_STAGES), (g / DW_STAGES) & 1u);
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        const int m = m0 + (warp & 3) * 32 + lane;
+        for (int gi = 0; gi < 4; ++gi) {
+            float v[16];
+            const int cl = (warp >> 2) * 64 + gi * 16;
+            tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)cl, v);
+            if (m >= H) continue;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int n = n0 + cl + i;
+                const int k = n < Hp ? n : n - Hp;
+                if (n < K2p && k < H) atomicAdd(&c.dW[(size_t)m * 2 * H + (n < Hp ? k : H + k)], v[i]);
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;" ::"r"(tmem) : "memory");
+}
