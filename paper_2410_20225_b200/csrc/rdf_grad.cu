@@ -19,18 +19,21 @@ static const int MAX_CLASSES = 8;
 // ---------------------------------------------------------------- loss head
 // per invocation f: z = W_s h + b_s; loss += logsumexp(z) - z[label]; dlog = softmax(z) - onehot
 __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
+    // four invocations per warp (8 lanes each) so that four rows are in flight at a time
     __shared__ float warp_loss[8];
     const uint32_t F = c.ctl->frame_count;
-    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
+    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, sub = lane / 8, sl = lane % 8;
     const uint32_t warp = blockIdx.x * 8 + wib, n_warps = gridDim.x * 8;
     const int H = c.H, C = c.n_classes;
     float my_loss = 0.f;
-    for (uint32_t f = (uint32_t)c.B + warp; f < F; f += n_warps) {
-        const float* h = c.arena + (size_t)f * c.S;
+    for (uint32_t base = (uint32_t)c.B + warp * 4; base < F; base += n_warps * 4) {
+        const uint32_t f = base + sub;
+        const bool act = f < F;
+        const float* h = c.arena + (size_t)(act ? f : base) * c.S;
         float z[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
-        for (int j = lane * 4; j < H; j += 128) {
+        for (int j = sl * 4; j < H; j += 32) {
             const float4 h4 = *reinterpret_cast<const float4*>(h + j);
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
@@ -41,30 +44,35 @@ __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
         }
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k)
-            for (int o = 16; o > 0; o >>= 1) z[k] += __shfl_xor_sync(0xffffffffu, z[k], o);
-        const int node = (int)c.frames[f].arg;
-        const int lab = __ldg(&c.label[node]);
-        float m = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            if (k < C) {
-                z[k] += __ldg(&c.b_s[k]);
-                m = fmaxf(m, z[k]);
-            }
-        float s = 0.f, zl = 0.f;
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            if (k < C) {
-                s += expf(z[k] - m);
-                if (k == lab) zl = z[k];
-            }
-        if (lane == 0) {
-            my_loss += logf(s) + m - zl;
+            for (int o = 4; o > 0; o >>= 1) z[k] += __shfl_xor_sync(0xffffffffu, z[k], o);
+        if (act && sl == 0) {
+            const int node = (int)c.frames[f].arg;
+            const int lab = __ldg(&c.label[node]);
+            float m = -INFINITY;
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
-                c.dlog[(size_t)f * 8 + k] = k < C ? expf(z[k] - m) / s - (k == lab ? 1.f : 0.f) : 0.f;
+                if (k < C) {
+                    z[k] += __ldg(&c.b_s[k]);
+                    m = fmaxf(m, z[k]);
+                }
+            float s = 0.f, zl = 0.f;
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) {
+                    s += expf(z[k] - m);
+                    if (k == lab) zl = z[k];
+                }
+            my_loss += logf(s) + m - zl;
+            float d[MAX_CLASSES];
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k) d[k] = k < C ? expf(z[k] - m) / s - (k == lab ? 1.f : 0.f) : 0.f;
+            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8) = make_float4(d[0], d[1], d[2], d[3]);
+            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8 + 4) = make_float4(d[4], d[5], d[6], d[7]);
         }
     }
+    // fixed-order sum of the four group leaders, then of the warps
+    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 16);
+    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 8);
     if (lane == 0) warp_loss[wib] = my_loss;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -111,22 +119,23 @@ __device__ __forceinline__ void backward_enqueue(const DevCtx& c, uint32_t wave,
 // A (TreeRNN): per invocation t of the wave, dh = (gradient from the caller) + W_s^T dlog;
 //    cell: dz = dh * (1 - h^2), queue the two callee frames; leaf: keep dh for dE.
 __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
-    const int lane = threadIdx.x % 32;
+    // four invocations per warp (8 lanes each): four independent chains of loads in flight
+    const int lane = threadIdx.x % 32, sub = lane / 8, sl = lane % 8;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
     const int H = c.H, C = c.n_classes;
     const uint32_t* q = c.bq[wave & 1];
-    for (uint32_t i = warp; i < n; i += n_warps) {
+    for (uint32_t i = warp * 4 + sub; i < n; i += n_warps * 4) {
         const uint32_t t = __ldcg(&q[i]);
         const uint32_t parent = __ldcg(&c.frames[t].parent);
         const bool from_result = parent < (uint32_t)c.B;
         const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
         const bool leaf = l == LEAF_MARK;
-        float dl[MAX_CLASSES];
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
+        const float4 d0 = ldcg4(c.dlog + (size_t)t * 8), d1 = ldcg4(c.dlog + (size_t)t * 8 + 4);
+        const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
         float* g = c.dhp + (size_t)t * H;
         const float* h = c.arena + (size_t)t * H;
-        for (int j = lane * 4; j < H; j += 128) {
+#pragma unroll 2
+        for (int j = sl * 4; j < H; j += 32) {
             float4 dh = from_result ? make_float4(0.f, 0.f, 0.f, 0.f) : ldcg4(g + j);
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
@@ -150,8 +159,8 @@ __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
             *reinterpret_cast<float4*>(g + j) = dh;
         }
         if (c.use_tc && !leaf)
-            for (int j = H + lane; j < c.Hp; j += 32) c.dz_bf[(size_t)t * c.Hp + j] = __float2bfloat16_rn(0.f);
-        if (lane == 0) backward_enqueue(c, wave, t, leaf, l, r);
+            for (int j = H + sl; j < c.Hp; j += 8) c.dz_bf[(size_t)t * c.Hp + j] = __float2bfloat16_rn(0.f);
+        if (sl == 0) backward_enqueue(c, wave, t, leaf, l, r);
     }
 }
 
@@ -373,6 +382,7 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, c
     if (t0 >= t1) return;
     for (int j = threadIdx.x; j < M; j += blockDim.x) {
         float s = 0.f;
+#pragma unroll 4
         for (uint32_t i = t0; i < t1; ++i) s += A[(size_t)list[i] * lda + j];
         atomicAdd(&out[j], s);
     }
@@ -389,6 +399,7 @@ __global__ void __launch_bounds__(256) rdf_dws_kernel(const DevCtx c) {
         float s[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) s[k] = 0.f;
+#pragma unroll 4
         for (uint32_t f = f0; f < f1; ++f) {
             const float hj = c.arena[(size_t)f * c.S + j];
             const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8);
