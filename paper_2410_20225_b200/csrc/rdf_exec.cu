@@ -233,6 +233,40 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) 
     }
 }
 
+// Narrow waves (a few dozen ready cells, e.g. the tail of a deep chain): the 64 x 64 tiles would keep
+// a handful of blocks busy with a long dependent k-loop.  Here one block step computes an 8 cell x 16
+// column patch with the whole contraction spread over its threads: thread = (cell, column, half of k),
+// streaming its operand row and weight row with independent 128-bit loads.
+__device__ void rnn_cell_thin(const DevCtx& c, float* red, uint32_t n_items) {
+    const int H = c.H, K2 = 2 * c.H;
+    const int units_n = (H + 15) / 16, units = ((n_items + 7) / 8) * units_n;
+    const int o = threadIdx.x & 127, kh = threadIdx.x >> 7, rr = o >> 4, cc = o & 15;
+    for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+        const int row = (unit / units_n) * 8 + rr, col = (unit % units_n) * 16 + cc;
+        const bool live = row < (int)n_items && col < H;
+        float acc = 0.f;
+        uint32_t out = 0;
+        if (live) {
+            const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
+            out = it.x;
+            const float4* x = reinterpret_cast<const float4*>(c.arena + (size_t)(kh == 0 ? it.y : it.z) * H);
+            const float4* w = reinterpret_cast<const float4*>(c.W + (size_t)col * K2 + kh * H);
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+            for (int k4 = 0; k4 < H / 4; ++k4) {
+                const float4 xv = __ldcg(x + k4), wv = __ldg(w + k4);
+                a0 = fmaf(xv.x, wv.x, a0); a1 = fmaf(xv.y, wv.y, a1);
+                a2 = fmaf(xv.z, wv.z, a2); a3 = fmaf(xv.w, wv.w, a3);
+            }
+            acc = (a0 + a1) + (a2 + a3);
+        }
+        if (kh == 1) red[o] = acc;
+        __syncthreads();
+        if (kh == 0 && live) c.arena[(size_t)out * H + col] = tanhf(acc + red[o] + __ldg(&c.b[col]));
+        __syncthreads();
+    }
+}
+
 __device__ void rnn_leaf_rows(const DevCtx& c, uint32_t n_items) {
     // one warp per leaf: state(slot) = E[tok]
     const int H = c.H;
@@ -322,7 +356,12 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
                 if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
             } else {
                 if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
-                if (n_cell) rnn_cell_tiles(c, gsm, min(n_cell, c.work_cap));
+                if (n_cell) {
+                    const uint32_t nc = min(n_cell, c.work_cap);
+                    // thin patches while they fit in two rounds over the grid, tiles for wide waves
+                    if (((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x) rnn_cell_thin(c, &gsm.As[0][0], nc);
+                    else rnn_cell_tiles(c, gsm, nc);
+                }
             }
             __syncthreads();
             lap(cyc_c);

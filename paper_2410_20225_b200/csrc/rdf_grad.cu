@@ -101,18 +101,34 @@ __global__ void __launch_bounds__(256) rdf_backward_seed_kernel(const DevCtx c) 
     if (b == 0) c.ctl->bq_count[0] = (uint32_t)c.B;
 }
 
-__device__ __forceinline__ void backward_enqueue(const DevCtx& c, uint32_t wave, uint32_t t, bool leaf, uint32_t l,
-                                                 uint32_t r) {
-    if (leaf) {
-        c.all_leaves[atomicAdd(&c.ctl->all_leaves, 1u)] = t;
-    } else {
-        const uint32_t idx = atomicAdd(&c.ctl->all_cells, 1u);
-        c.all_cells[idx] = t;
-        if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
-        const uint32_t at = atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u);
-        uint32_t* qn = c.bq[(wave + 1) & 1];
-        qn[at] = l;
-        qn[at + 1] = r;
+// Appends this block's cells / leaves of one lock-step iteration to the global lists with one
+// global atomic per list per block (thousands of same-address atomics per wave would serialise in
+// L2).  Called by every thread of the block; `mine` marks the one thread that speaks for a frame.
+__device__ __forceinline__ void backward_enqueue_block(const DevCtx& c, uint32_t wave, bool mine, uint32_t t, bool leaf,
+                                                       uint32_t l, uint32_t r) {
+    __shared__ uint32_t cnt[2], base[3];
+    if (threadIdx.x == 0) cnt[0] = cnt[1] = 0;
+    __syncthreads();
+    uint32_t local = 0;
+    if (mine) local = atomicAdd(&cnt[leaf ? 1 : 0], 1u);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        base[0] = cnt[0] ? atomicAdd(&c.ctl->all_cells, cnt[0]) : 0u;
+        base[1] = cnt[1] ? atomicAdd(&c.ctl->all_leaves, cnt[1]) : 0u;
+        base[2] = cnt[0] ? atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u * cnt[0]) : 0u;
+    }
+    __syncthreads();
+    if (mine) {
+        if (leaf) {
+            c.all_leaves[base[1] + local] = t;
+        } else {
+            const uint32_t idx = base[0] + local;
+            c.all_cells[idx] = t;
+            if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
+            uint32_t* qn = c.bq[(wave + 1) & 1];
+            qn[base[2] + 2 * local] = l;
+            qn[base[2] + 2 * local + 1] = r;
+        }
     }
 }
 
@@ -121,15 +137,20 @@ __device__ __forceinline__ void backward_enqueue(const DevCtx& c, uint32_t wave,
 __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
     // four invocations per warp (8 lanes each): four independent chains of loads in flight
     const int lane = threadIdx.x % 32, sub = lane / 8, sl = lane % 8;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    const int wib = threadIdx.x / 32;
     const int H = c.H, C = c.n_classes;
     const uint32_t* q = c.bq[wave & 1];
-    for (uint32_t i = warp * 4 + sub; i < n; i += n_warps * 4) {
-        const uint32_t t = __ldcg(&q[i]);
+    for (uint32_t base = blockIdx.x * 32; base < n; base += gridDim.x * 32) {      // 32 frames per block per step
+        const uint32_t i = base + wib * 4 + sub;
+        const bool act = i < n;
+        uint32_t t = 0, l = 0, r = 0;
+        bool leaf = false;
+        if (act) {
+        t = __ldcg(&q[i]);
         const uint32_t parent = __ldcg(&c.frames[t].parent);
         const bool from_result = parent < (uint32_t)c.B;
-        const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
-        const bool leaf = l == LEAF_MARK;
+        l = __ldcg(&c.op_l[t]); r = __ldcg(&c.op_r[t]);
+        leaf = l == LEAF_MARK;
         const float4 d0 = ldcg4(c.dlog + (size_t)t * 8), d1 = ldcg4(c.dlog + (size_t)t * 8 + 4);
         const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
         float* g = c.dhp + (size_t)t * H;
@@ -160,22 +181,28 @@ __device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
         }
         if (c.use_tc && !leaf)
             for (int j = H + sl; j < c.Hp; j += 8) c.dz_bf[(size_t)t * c.Hp + j] = __float2bfloat16_rn(0.f);
-        if (sl == 0) backward_enqueue(c, wave, t, leaf, l, r);
+        }
+        backward_enqueue_block(c, wave, act && sl == 0, t, leaf, l, r);
     }
 }
 
 // A (TreeLSTM): the gate gradients replace the retained gates; dc goes straight to the callee frames.
 __device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
     const int lane = threadIdx.x % 32;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    const int wib = threadIdx.x / 32;
     const int H = c.H, C = c.n_classes, S = c.S;
     const uint32_t* q = c.bq[wave & 1];
-    for (uint32_t i = warp; i < n; i += n_warps) {
-        const uint32_t t = __ldcg(&q[i]);
+    for (uint32_t base = blockIdx.x * 8; base < n; base += gridDim.x * 8) {        // 8 frames per block per step
+        const uint32_t i = base + wib;
+        const bool act = i < n;
+        uint32_t t = 0, l = 0, r = 0;
+        bool leaf = false;
+        if (act) {
+        t = __ldcg(&q[i]);
         const uint32_t parent = __ldcg(&c.frames[t].parent);
         const bool from_result = parent < (uint32_t)c.B;
-        const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
-        const bool leaf = l == LEAF_MARK;
+        l = __ldcg(&c.op_l[t]); r = __ldcg(&c.op_r[t]);
+        leaf = l == LEAF_MARK;
         float dl[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
@@ -209,7 +236,8 @@ __device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n)
                 c.dhp[(size_t)r * S + H + j] = dc * fr;
             }
         }
-        if (lane == 0) backward_enqueue(c, wave, t, leaf, l, r);
+        }
+        backward_enqueue_block(c, wave, act && lane == 0, t, leaf, l, r);
     }
 }
 
@@ -261,6 +289,45 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
     }
 }
 
+// Narrow waves: an 8 cell x 32 column patch of [dh_l ; dh_r] = W^T dz per block step;
+// thread = (cell, 4 columns, quarter of the contraction over j).
+__device__ void backward_operand_thin(const DevCtx& c, float* red, uint32_t first, uint32_t n_items) {
+    const int H = c.H, K2 = 2 * c.H;
+    const int units_n = (K2 + 31) / 32, units = ((n_items + 7) / 8) * units_n;
+    const int o = threadIdx.x & 63, jq = threadIdx.x >> 6, rr = o >> 3, c4 = o & 7;
+    const int jlen = (H + 3) / 4;
+    for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+        const int row = (unit / units_n) * 8 + rr, col = (unit % units_n) * 32 + c4 * 4;
+        const bool live = row < (int)n_items && col < K2;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        uint32_t t = 0;
+        if (live) {
+            t = __ldcg(&c.all_cells[first + row]);
+            const float* dz = c.dhp + (size_t)t * H;
+            const int j0 = jq * jlen, j1 = min(H, j0 + jlen);
+#pragma unroll 4
+            for (int j = j0; j < j1; ++j) {
+                const float d = __ldcg(dz + j);
+                const float4 w = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col));
+                acc.x = fmaf(d, w.x, acc.x); acc.y = fmaf(d, w.y, acc.y);
+                acc.z = fmaf(d, w.z, acc.z); acc.w = fmaf(d, w.w, acc.w);
+            }
+        }
+        if (jq > 0) *reinterpret_cast<float4*>(red + ((jq - 1) * 64 + o) * 4) = acc;
+        __syncthreads();
+        if (jq == 0 && live) {
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+                const float4 p = *reinterpret_cast<const float4*>(red + (q * 64 + o) * 4);
+                acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+            }
+            const uint32_t child = col < H ? __ldcg(&c.op_l[t]) : __ldcg(&c.op_r[t]);
+            *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + (col < H ? col : col - H)) = acc;
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
     __shared__ GemmSmem gsm;
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
@@ -294,6 +361,8 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         if (end > first) {
             if (c.use_tc) tc_tiles<false>(c, tc, tc_items, first, end - first);
             else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
+            else if (((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
+                backward_operand_thin(c, &gsm.As[0][0], first, end - first);
             else backward_operand_tiles(c, gsm, first, end - first, c.dhp, c.H, c.H);
             first = end;
             __syncthreads();
