@@ -237,24 +237,35 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) 
 // a handful of blocks busy with a long dependent k-loop.  Here one block step computes an 8 cell x 16
 // column patch with the whole contraction spread over its threads: thread = (cell, column, half of k),
 // streaming its operand row and weight row with independent 128-bit loads.
-__device__ void rnn_cell_thin(const DevCtx& c, float* red, uint32_t n_items) {
+__device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t n_items) {
+    // xs: shared staging for the 8 operand rows [h_l ; h_r] of the patch (8 x 2H floats) + 128 floats
     const int H = c.H, K2 = 2 * c.H;
+    float* red = xs + 8 * K2;
     const int units_n = (H + 15) / 16, units = ((n_items + 7) / 8) * units_n;
     const int o = threadIdx.x & 127, kh = threadIdx.x >> 7, rr = o >> 4, cc = o & 15;
     for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
-        const int row = (unit / units_n) * 8 + rr, col = (unit % units_n) * 16 + cc;
+        const int row0 = (unit / units_n) * 8;
+        // all operand rows of the patch in one round of independent 128-bit loads
+        for (int p = threadIdx.x; p < 8 * (K2 / 4); p += blockDim.x) {
+            const int r = p / (K2 / 4), k = (p % (K2 / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (row0 + r < (int)n_items) {
+                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row0 + r]));   // {out, l, r, -}
+                v = k < H ? ldcg4(c.arena + (size_t)it.y * H + k) : ldcg4(c.arena + (size_t)it.z * H + (k - H));
+            }
+            *reinterpret_cast<float4*>(xs + r * K2 + k) = v;
+        }
+        __syncthreads();
+        const int row = row0 + rr, col = (unit % units_n) * 16 + cc;
         const bool live = row < (int)n_items && col < H;
         float acc = 0.f;
-        uint32_t out = 0;
         if (live) {
-            const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
-            out = it.x;
-            const float4* x = reinterpret_cast<const float4*>(c.arena + (size_t)(kh == 0 ? it.y : it.z) * H);
-            const float4* w = reinterpret_cast<const float4*>(c.W + (size_t)col * K2 + kh * H);
+            const float4* x = reinterpret_cast<const float4*>(xs + rr * K2 + kh * H);
+            const float4* w = reinterpret_cast<const float4*>(c.W + (size_t)col * K2 + kh * H);   // L1-resident across waves
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 4
+#pragma unroll 8
             for (int k4 = 0; k4 < H / 4; ++k4) {
-                const float4 xv = __ldcg(x + k4), wv = __ldg(w + k4);
+                const float4 xv = x[k4], wv = __ldg(w + k4);
                 a0 = fmaf(xv.x, wv.x, a0); a1 = fmaf(xv.y, wv.y, a1);
                 a2 = fmaf(xv.z, wv.z, a2); a3 = fmaf(xv.w, wv.w, a3);
             }
@@ -262,7 +273,8 @@ __device__ void rnn_cell_thin(const DevCtx& c, float* red, uint32_t n_items) {
         }
         if (kh == 1) red[o] = acc;
         __syncthreads();
-        if (kh == 0 && live) c.arena[(size_t)out * H + col] = tanhf(acc + red[o] + __ldg(&c.b[col]));
+        if (kh == 0 && live)
+            c.arena[(size_t)__ldcg(&c.cell_items[row].out) * H + col] = tanhf(acc + red[o] + __ldg(&c.b[col]));
         __syncthreads();
     }
 }
@@ -359,7 +371,8 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
                 if (n_cell) {
                     const uint32_t nc = min(n_cell, c.work_cap);
                     // thin patches while they fit in two rounds over the grid, tiles for wide waves
-                    if (((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x) rnn_cell_thin(c, &gsm.As[0][0], nc);
+                    if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
+                        rnn_cell_thin(c, reinterpret_cast<float*>(&tile_smem), nc);      // 8 x 2H + 128 floats <= 26 KB
                     else rnn_cell_tiles(c, gsm, nc);
                 }
             }

@@ -112,11 +112,10 @@ __device__ __forceinline__ void backward_enqueue_block(const DevCtx& c, uint32_t
     uint32_t local = 0;
     if (mine) local = atomicAdd(&cnt[leaf ? 1 : 0], 1u);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        base[0] = cnt[0] ? atomicAdd(&c.ctl->all_cells, cnt[0]) : 0u;
-        base[1] = cnt[1] ? atomicAdd(&c.ctl->all_leaves, cnt[1]) : 0u;
-        base[2] = cnt[0] ? atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u * cnt[0]) : 0u;
-    }
+    // three threads, three independent round trips at once
+    if (threadIdx.x == 0) base[0] = cnt[0] ? atomicAdd(&c.ctl->all_cells, cnt[0]) : 0u;
+    if (threadIdx.x == 32) base[1] = cnt[1] ? atomicAdd(&c.ctl->all_leaves, cnt[1]) : 0u;
+    if (threadIdx.x == 64) base[2] = cnt[0] ? atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u * cnt[0]) : 0u;
     __syncthreads();
     if (mine) {
         if (leaf) {
@@ -291,24 +290,32 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
 
 // Narrow waves: an 8 cell x 32 column patch of [dh_l ; dh_r] = W^T dz per block step;
 // thread = (cell, 4 columns, quarter of the contraction over j).
-__device__ void backward_operand_thin(const DevCtx& c, float* red, uint32_t first, uint32_t n_items) {
+__device__ void backward_operand_thin(const DevCtx& c, float* zs, uint32_t first, uint32_t n_items) {
+    // zs: shared staging for the 8 dz rows of the patch (8 x H floats) followed by 768 floats of partial sums
     const int H = c.H, K2 = 2 * c.H;
+    float* red = zs + 8 * H;
     const int units_n = (K2 + 31) / 32, units = ((n_items + 7) / 8) * units_n;
     const int o = threadIdx.x & 63, jq = threadIdx.x >> 6, rr = o >> 3, c4 = o & 7;
     const int jlen = (H + 3) / 4;
     for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
-        const int row = (unit / units_n) * 8 + rr, col = (unit % units_n) * 32 + c4 * 4;
+        const int row0 = (unit / units_n) * 8;
+        for (int p = threadIdx.x; p < 8 * (H / 4); p += blockDim.x) {
+            const int r = p / (H / 4), k = (p % (H / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (row0 + r < (int)n_items) v = ldcg4(c.dhp + (size_t)__ldcg(&c.all_cells[first + row0 + r]) * H + k);
+            *reinterpret_cast<float4*>(zs + r * H + k) = v;
+        }
+        __syncthreads();
+        const int row = row0 + rr, col = (unit % units_n) * 32 + c4 * 4;
         const bool live = row < (int)n_items && col < K2;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        uint32_t t = 0;
         if (live) {
-            t = __ldcg(&c.all_cells[first + row]);
-            const float* dz = c.dhp + (size_t)t * H;
+            const float* dz = zs + rr * H;
             const int j0 = jq * jlen, j1 = min(H, j0 + jlen);
-#pragma unroll 4
+#pragma unroll 8
             for (int j = j0; j < j1; ++j) {
-                const float d = __ldcg(dz + j);
-                const float4 w = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col));
+                const float d = dz[j];
+                const float4 w = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col));   // L1-resident across waves
                 acc.x = fmaf(d, w.x, acc.x); acc.y = fmaf(d, w.y, acc.y);
                 acc.z = fmaf(d, w.z, acc.z); acc.w = fmaf(d, w.w, acc.w);
             }
@@ -321,6 +328,7 @@ __device__ void backward_operand_thin(const DevCtx& c, float* red, uint32_t firs
                 const float4 p = *reinterpret_cast<const float4*>(red + (q * 64 + o) * 4);
                 acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
             }
+            const uint32_t t = __ldcg(&c.all_cells[first + row]);
             const uint32_t child = col < H ? __ldcg(&c.op_l[t]) : __ldcg(&c.op_r[t]);
             *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + (col < H ? col : col - H)) = acc;
         }
@@ -329,7 +337,8 @@ __device__ void backward_operand_thin(const DevCtx& c, float* red, uint32_t firs
 }
 
 __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
-    __shared__ GemmSmem gsm;
+    __shared__ LstmSmem tile_smem;                                   // tiles use its first part; thin patches stage rows in it
+    GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(8) uint64_t tc_mbars[TC_STAGES];
@@ -361,8 +370,8 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         if (end > first) {
             if (c.use_tc) tc_tiles<false>(c, tc, tc_items, first, end - first);
             else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
-            else if (((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
-                backward_operand_thin(c, &gsm.As[0][0], first, end - first);
+            else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
+                backward_operand_thin(c, reinterpret_cast<float*>(&tile_smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
             else backward_operand_tiles(c, gsm, first, end - first, c.dhp, c.H, c.H);
             first = end;
             __syncthreads();
