@@ -34,7 +34,7 @@ WORKLOAD_NAMES = {
     4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13}
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13, "grad_tc": 12}
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
 
 
@@ -230,7 +230,10 @@ def main():
         fs, r = rdf.tree_net_program(cell, with_loss=cfg["grad"])
         g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
         compute = rdf.BF16 if cfg["bf16"] else rdf.F32
-        dtype = "f32"                       # arithmetic type of the contractions as built
+        # arithmetic type of the contractions: bf16 operands on the tensor cores (fp32 accumulate) for the
+        # bf16 TreeRNN workload, fp32 FMA otherwise (the TreeLSTM contractions are fp32 as built)
+        use_tc = cfg["bf16"] and CELL[cfg["kind"]] == "rnn"
+        dtype = "bf16" if use_tc else "f32"
         host = {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).pin_memory()
                 for k in ("tree_root", "left", "right", "tok", "label")}
         dt = {k: v.cuda() for k, v in host.items()}
@@ -241,7 +244,7 @@ def main():
         if cell == "lstm":
             flops_fwd = tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
         if cfg["grad"]:
-            kind = "grad" if cell == "rnn" else "grad_lstm"
+            kind = "grad_lstm" if cell == "lstm" else ("grad_tc" if use_tc else "grad")
             grads = {k: torch.empty_like(v) for k, v in dp.items()}
             loss = torch.zeros(1, dtype=torch.float32, device="cuda")
 
@@ -344,14 +347,23 @@ def main():
     else:
         H = cfg["H"]
         C = cfg["trees"].n_cells
+        # algorithmic flops of the contraction in each phase: 2 * 2H * (rows of W) per cell
         flops = {"forward": flops_fwd, "backward": flops_fwd, "dW": flops_fwd}.get(dominant, flops_fwd)
         achieved = flops / (dom_ms * 1e-3) / 1e12
-        kernel = {"forward": "rdf_forward_kernel", "backward": "rdf_backward_kernel", "dW": "rdf_dw_kernel"}.get(
-            dominant, dominant)
-        roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
-                "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
-                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
-                "cells": C, "flops_forward": flops_fwd}
+        kernel = {"forward": "rdf_forward_kernel", "backward": "rdf_backward_kernel",
+                  "dW": "rdf_dw_tc_kernel" if use_tc else "rdf_outer_kernel"}.get(dominant, dominant)
+        if use_tc:
+            peak = pk["bf16_tflops_sustained"]
+            roof = {"kernel": kernel, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": None,
+                    "peak_source": pk["source"] + " (bf16 dense, sustained)", "cells": C, "flops_phase": flops,
+                    "note": "the persistent kernel also runs token scheduling and grid barriers of every wave; "
+                            "see block0_ms_at_max_clock for the split"}
+        else:
+            roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
+                    "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
+                    "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                    "cells": C, "flops_phase": flops}
 
     cpu = None
     if not args.no_cpu_baseline:
