@@ -107,6 +107,10 @@ def peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
+# (profiles/rdf_forward_kernel_config3.md); None where no capture of the current kernel exists
+NCU_TRAFFIC_BYTES = {("rdf_forward_kernel", 3): 921.46e6}
+
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
@@ -365,6 +369,7 @@ def main():
                     "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
                     "cells": C, "flops_phase": flops}
 
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((roof["kernel"], args.workload))
     cpu = None
     if not args.no_cpu_baseline:
         v, _, what = time_oracle(cfg, 1, 0, scale=1 if cfg["trees"].N > 2_000_000 else 4) if cfg["kind"] != "fib" else time_oracle(cfg, 1, 0, scale=4)
