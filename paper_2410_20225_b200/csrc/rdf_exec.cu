@@ -322,11 +322,14 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
     GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     extern __shared__ unsigned char dyn_smem[];                      // operand stages of the tensor-core path
     __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[TC_STAGES];
+    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
     __shared__ uint4 tc_items[TC_M];
     TcState tc;
     load_program(c, sp);
-    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Wp, 2 * c.Hp, c.Hp / 4, 4);
+    if (c.use_tc) {
+        if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Hp / 16, 3, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
+        else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 4, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
+    }
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
     long long cyc_s = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
@@ -360,9 +363,12 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
         const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
         if (n_leaf | n_cell) {
-            if (c.use_tc) {
+            if (c.use_tc && c.lstm) {
+                if (n_leaf) tc_tiles<TC_LSTM_LEAF>(c, tc, tc_items, 0, min(n_leaf, c.work_cap));
+                if (n_cell) tc_tiles<TC_LSTM_CELL>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
+            } else if (c.use_tc) {
                 if (n_leaf) tc_leaf_rows(c, min(n_leaf, c.work_cap));
-                if (n_cell) tc_tiles<true>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
+                if (n_cell) tc_tiles<TC_RNN_FWD>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
             } else if (c.lstm) {
                 if (n_leaf) lstm_forward_tiles<3>(c, tile_smem, min(n_leaf, c.work_cap));
                 if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
@@ -469,11 +475,18 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.arena = P.take<float>(vf * S);
     L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
     L.Hp = (H + 63) / 64 * 64;
-    L.use_tc = g->has_vector_ops && !g->has_lstm && params->compute == RDF_BF16 && L.Hp <= TC_HP_MAX;
+    L.use_tc = g->has_vector_ops && params->compute == RDF_BF16 && L.Hp <= TC_HP_MAX && params->D == params->H;
+    const bool tcl = L.use_tc && g->has_lstm, tcr = L.use_tc && !g->has_lstm;
+    const size_t wcount = (size_t)L.Hp * 2 * L.Hp * (tcl ? 5 : 1);
     L.arena_bf = P.take<__nv_bfloat16>(L.use_tc ? vf * L.Hp : 0);
-    L.wp = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.Hp * 2 * L.Hp : 0);
-    L.wtp = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.Hp * 2 * L.Hp : 0);
-    L.dz_bf = P.take<__nv_bfloat16>(L.use_tc && want_grad ? vf * L.Hp : 0);
+    L.wp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
+    L.wtp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
+    L.dz_bf = P.take<__nv_bfloat16>(tcr && want_grad ? vf * L.Hp : 0);
+    L.wxp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
+    L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
+    L.dg_bf = P.take<__nv_bfloat16>(tcl && want_grad ? vf * 5 * L.Hp : 0);
+    L.tc_smem_fwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(80, 2 * L.Hp, 48, L.Hp, 3) : tc_smem_bytes(L.Hp / 4, 2 * L.Hp, 0, 0, 4);
+    L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(32, 5 * L.Hp, 0, 0, 4) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, 4);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
@@ -503,8 +516,9 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     CUDA_OK(cudaDeviceGetAttribute(&S->clock_khz, cudaDevAttrClockRate, dev));
     if (!coop) return RDF_ERR_CUDA;
-    CUDA_OK(cudaFuncSetAttribute(rdf_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, TC_SMEM_BYTES));
+    const int max_dyn = tc_smem_bytes(80, 2 * TC_HP_MAX, 48, TC_HP_MAX, 3);       // the largest configuration
+    CUDA_OK(cudaFuncSetAttribute(rdf_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, max_dyn));
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
     S->device = dev;
@@ -553,6 +567,9 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.Wp = reinterpret_cast<__nv_bfloat16*>(ws + L.wp);
         c.WTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wtp);
         c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
+        c.Wxp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxp);
+        c.E_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.e_bf);
+        c.dg_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dg_bf);
     } else {
         c.y = out->y;
     }
@@ -607,13 +624,18 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     if (c.use_tc) {
-        rdf_pack_w_kernel<<<64, 256, 0, stream>>>(c);
+        if (c.lstm) {
+            rdf_pack_lstm_kernel<<<256, 256, 0, stream>>>(c);
+            rdf_pack_e_kernel<<<1024, 256, 0, stream>>>(c);
+        } else {
+            rdf_pack_w_kernel<<<64, 256, 0, stream>>>(c);
+        }
         CUDA_OK(cudaGetLastError());
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args,
-                                        c.use_tc ? TC_SMEM_BYTES : 0, stream));
+                                        (size_t)L.tc_smem_fwd, stream));
     if (g->has_vector_ops) {
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());

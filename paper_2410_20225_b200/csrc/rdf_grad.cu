@@ -341,10 +341,11 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
     GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
     __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[TC_STAGES];
+    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
     __shared__ uint4 tc_items[TC_M];
     TcState tc;
-    if (c.use_tc) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.WTp, c.Hp, c.Hp / 4, 8);
+    const bool tc_on = c.use_tc && !c.lstm;        // the TreeLSTM gradient contractions run on the FMA tiles
+    if (tc_on) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 8, 4, c.WTp, c.Hp, c.Hp / 4);
     uint32_t generation = 0, wave = 0, first = 0;
     long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
@@ -368,7 +369,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         lap(cyc_b);
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
-            if (c.use_tc) tc_tiles<false>(c, tc, tc_items, first, end - first);
+            if (tc_on) tc_tiles<TC_RNN_BWD>(c, tc, tc_items, first, end - first);
             else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
             else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
                 backward_operand_thin(c, reinterpret_cast<float*>(&tile_smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
@@ -380,7 +381,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
             lap(cyc_b);
         }
     }
-    if (c.use_tc) tc_teardown(tc);
+    if (tc_on) tc_teardown(tc);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->waves_backward = wave;
         c.ctl->cyc[3] = cyc_a; c.ctl->cyc[4] = cyc_c; c.ctl->cyc[5] = cyc_b;
@@ -618,16 +619,17 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
-    if (c.use_tc) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    const bool tc_rnn = c.use_tc && !lstm;
+    if (tc_rnn) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args,
-                                        c.use_tc ? TC_SMEM_BYTES : 0, stream));
+                                        tc_rnn ? (size_t)L.tc_smem_bwd : 0, stream));
     rdf_mark(S, 4, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
     const long long max_leaves = std::max<long long>(1, in->max_invocations);
     const float* dgA = lstm ? c.gates : c.dhp;
     const int lda = lstm ? c.G : H;
-    if (c.use_tc) {
+    if (tc_rnn) {
         // 128 x 128 tiles of the padded [Hp x 2Hp] gradient, the cells split over the remaining blocks
         const int tiles_m = (c.Hp + 127) / 128, tiles_n = (2 * c.Hp + 127) / 128, n_tiles = tiles_m * tiles_n;
         const int splits = std::max(1, S->grid / n_tiles);

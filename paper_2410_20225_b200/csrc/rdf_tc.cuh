@@ -20,21 +20,36 @@
 
 static const int TC_M = 128;                 // cells per tile (TMEM lanes)
 static const int TC_KC = 64;                 // bf16 elements per staged K chunk = one 128-byte swizzled row
-static const int TC_STAGES = 4;
+static const int TC_MAX_STAGES = 4;
 static const int TC_A_STAGE = TC_M * 128;    // 16 KB
-static const int TC_HP_MAX = 320;            // widest padded hidden size the resident slice is sized for
-static const int TC_B_MAX = TC_HP_MAX * TC_HP_MAX;                               // (Hp/4) rows x 2Hp x 2 bytes
-static const int TC_SMEM_BYTES = 1024 + TC_B_MAX + TC_STAGES * TC_A_STAGE;       // + slack to align to 1024
+static const int TC_HP_MAX = 320;            // widest padded hidden size the resident slices are sized for
 static const int TC_TMEM_COLS = 128;
+
+// tile loops (template parameter of tc_tiles)
+enum TcMode {
+    TC_RNN_FWD = 0,     // A = [h_l ; h_r] (bf16 states), B = Wp slice;           epilogue: tanh, both arenas
+    TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: operand gradients
+    TC_LSTM_CELL = 2,   // A = [h_l ; h_r],                B = W5p slice (5 gates x 16 units); epilogue: gates, c, h
+    TC_LSTM_LEAF = 3,   // A = E_bf[tok],                  B = Wxp slice (3 gates x 16 units); epilogue: gates, c, h
+    TC_LSTM_BWD = 4     // A = gate gradients (5 Hp),      B = WT5p slice;         epilogue: operand gradients (dh)
+};
 
 struct TcState {
     uint32_t tmem_base;      // TMEM address returned by tcgen05.alloc
-    uint32_t b_addr;         // shared-space address of the resident weight slice (1024-byte aligned)
     uint32_t a_addr;         // shared-space address of A stage 0
     uint32_t mbar_addr;      // shared-space address of the per-stage mbarriers
-    uint32_t iter;           // K chunks issued so far (stage = iter % TC_STAGES)
-    int      ns, n_split, n_chunks;
+    uint32_t iter;           // K chunks issued so far (stage = iter % stages)
+    uint32_t stages;         // depth of the A ring (3 or 4)
+    int      n_split;        // N slices = blocks per row group
+    // up to two resident weight slices (the TreeLSTM forward keeps the cell and the leaf weights)
+    uint32_t b_addr[2];
+    int      ns[2], n_chunks[2];
 };
+
+// dynamic shared memory a kernel needs for the given resident slices and ring depth
+inline int tc_smem_bytes(int ns0, int k0, int ns1, int k1, int stages) {
+    return 1024 + (k0 / TC_KC) * ns0 * 128 + (ns1 ? (k1 / TC_KC) * ns1 * 128 : 0) + stages * TC_A_STAGE;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -112,20 +127,25 @@ __device__ __forceinline__ uint32_t swz(int r, int c16) {
 }
 
 // One-time set-up per kernel (all threads call it): TMEM allocation by warp 0, mbarriers, and the
-// block's resident slice of the packed weights: rows [slice * ns, +ns) of Bp[. x Kp], chunk by chunk.
+// block's resident slices of the packed weights: rows [slice * ns, +ns) of B[. x K], chunk by chunk.
 __device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, uint32_t* tmem_slot, uint64_t* mbars,
-                                         const __nv_bfloat16* Bp, int Kp, int ns, int n_split) {
+                                         int n_split, int stages, const __nv_bfloat16* B0, int K0, int ns0,
+                                         const __nv_bfloat16* B1 = nullptr, int K1 = 0, int ns1 = 0) {
     const uint32_t raw = smem_u32(dyn_smem);
     const uint32_t aligned = (raw + 1023u) & ~1023u;
-    tc.b_addr = aligned;
-    tc.a_addr = aligned + TC_B_MAX;
+    unsigned char* base = dyn_smem + (aligned - raw);
+    const int bytes0 = (K0 / TC_KC) * ns0 * 128, bytes1 = B1 ? (K1 / TC_KC) * ns1 * 128 : 0;
+    tc.b_addr[0] = aligned;
+    tc.b_addr[1] = aligned + bytes0;
+    tc.a_addr = aligned + bytes0 + bytes1;
+    tc.ns[0] = ns0; tc.ns[1] = ns1;
+    tc.n_chunks[0] = K0 / TC_KC; tc.n_chunks[1] = B1 ? K1 / TC_KC : 0;
     tc.mbar_addr = smem_u32(mbars);
     tc.iter = 0;
-    tc.ns = ns;
+    tc.stages = stages;
     tc.n_split = n_split;
-    tc.n_chunks = Kp / TC_KC;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) mbar_init(tc.mbar_addr + 8 * s, 1);
+        for (int s = 0; s < TC_MAX_STAGES; ++s) mbar_init(tc.mbar_addr + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < 32) {
@@ -133,12 +153,16 @@ __device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, u
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const int slice = blockIdx.x % n_split;
-    unsigned char* bp = dyn_smem + (aligned - raw);
-    const int chunk_bytes = ns * 128;
-    for (int p = threadIdx.x; p < tc.n_chunks * ns * 8; p += blockDim.x) {
-        const int kc = p / (ns * 8), q = p % (ns * 8), r = q >> 3, c16 = q & 7;
-        const uint4 v = *reinterpret_cast<const uint4*>(Bp + (size_t)(slice * ns + r) * Kp + kc * TC_KC + c16 * 8);
-        *reinterpret_cast<uint4*>(bp + kc * chunk_bytes + swz(r, c16)) = v;
+    for (int which = 0; which < 2; ++which) {
+        const __nv_bfloat16* Bp = which ? B1 : B0;
+        if (!Bp) continue;
+        const int ns = which ? ns1 : ns0, Kp = which ? K1 : K0;
+        unsigned char* bp = base + (which ? bytes0 : 0);
+        for (int p = threadIdx.x; p < (Kp / TC_KC) * ns * 8; p += blockDim.x) {
+            const int kc = p / (ns * 8), q = p % (ns * 8), r = q >> 3, c16 = q & 7;
+            const uint4 v = *reinterpret_cast<const uint4*>(Bp + (size_t)(slice * ns + r) * Kp + kc * TC_KC + c16 * 8);
+            *reinterpret_cast<uint4*>(bp + kc * ns * 128 + swz(r, c16)) = v;
+        }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -154,19 +178,34 @@ __device__ __forceinline__ void tc_teardown(const TcState& tc) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tc.tmem_base), "n"(TC_TMEM_COLS) : "memory");
 }
 
-// One 128-cell tile loop.  FWD = true : cells cell_items[0, n_items); A row = [state(l) ; state(r)] in bf16;
-//                                         epilogue state(out) = tanh(D + b) into both arenas.
-//                          FWD = false: cells all_cells[first, first + n_items); A row = dz in bf16;
-//                                         epilogue writes D into the incoming-gradient rows of the operand frames.
-// s_items: 128 x uint4 of shared memory for the tile's cell records.
-template <bool FWD>
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float tc_sigmoid(float x) { return 1.f / (1.f + expf(-x)); }
+
+// One 128-row tile loop over n_items ready operators (see TcMode).  Rows come from cell_items /
+// leaf_items (forward modes) or from all_cells[first ..] (gradient modes).
+// s_items: 128 x uint4 of shared memory for the tile's records {frame, left, right / token, valid}.
+template <int MODE>
 __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t first, uint32_t n_items) {
-    const int H = c.H, Hp = c.Hp, ns = tc.ns, n_chunks = tc.n_chunks;
+    constexpr int RGN = MODE == TC_LSTM_LEAF ? 1 : 0;
+    constexpr bool GRAD = MODE == TC_RNN_BWD || MODE == TC_LSTM_BWD;
+    const int H = c.H, Hp = c.Hp, S = c.S, ns = tc.ns[RGN], n_chunks = tc.n_chunks[RGN];
+    const uint32_t stages = tc.stages;
     const int slice = blockIdx.x % tc.n_split, rg = blockIdx.x / tc.n_split, n_rg = gridDim.x / tc.n_split;
     if (rg >= n_rg) return;                                    // blocks beyond the last full group sit this out
     const uint32_t idesc = tc_idesc(ns);
     const int tiles = (n_items + TC_M - 1) / TC_M;
-    const __nv_bfloat16* Arows = FWD ? c.arena_bf : c.dz_bf;
+    const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : MODE == TC_LSTM_BWD ? c.dg_bf
+                                 : MODE == TC_LSTM_LEAF ? c.E_bf : c.arena_bf;
     bool ok = true;
     for (int tile = rg; tile < tiles && ok; tile += n_rg) {
         const int row0 = tile * TC_M;
@@ -174,11 +213,14 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
             uint4 it = make_uint4(0u, 0u, 0u, 0u);
             const int row = row0 + threadIdx.x;
             if (row < (int)n_items) {
-                if (FWD) {
-                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
-                } else {
+                if (GRAD) {
                     const uint32_t t = __ldcg(&c.all_cells[first + row]);
                     it.x = t; it.y = __ldcg(&c.op_l[t]); it.z = __ldcg(&c.op_r[t]);
+                } else if (MODE == TC_LSTM_LEAF) {
+                    const uint2 lf = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[row]));   // {slot, tok}
+                    it.x = lf.x; it.y = lf.y;
+                } else {
+                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
                 }
                 it.w = 1u;
             }
@@ -187,16 +229,19 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
         __syncthreads();
         const uint32_t it0 = tc.iter;
         auto issue = [&](int kc) {
-            const uint32_t g = it0 + kc, s = g % TC_STAGES;
+            const uint32_t g = it0 + kc, s = g % stages;
             // the MMAs that last read this stage must have completed
-            if (g >= TC_STAGES) ok = mbar_wait(c, tc.mbar_addr + 8 * s, ((g / TC_STAGES) - 1) & 1u) && ok;
+            if (g >= stages) ok = mbar_wait(c, tc.mbar_addr + 8 * s, ((g / stages) - 1) & 1u) && ok;
             const int koff = kc * TC_KC;
             for (int p = threadIdx.x; p < TC_M * 8; p += blockDim.x) {
                 const int r = p >> 3, c16 = p & 7;
                 const uint4 it = s_items[r];
                 size_t src;
-                if (FWD) src = (size_t)(koff < Hp ? it.y : it.z) * Hp + (koff < Hp ? koff : koff - Hp) + c16 * 8;
-                else src = (size_t)it.x * Hp + koff + c16 * 8;
+                if (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL)
+                    src = (size_t)(koff < Hp ? it.y : it.z) * Hp + (koff < Hp ? koff : koff - Hp) + c16 * 8;
+                else if (MODE == TC_RNN_BWD) src = (size_t)it.x * Hp + koff + c16 * 8;
+                else if (MODE == TC_LSTM_BWD) src = (size_t)it.x * 5 * Hp + koff + c16 * 8;
+                else src = (size_t)it.y * Hp + koff + c16 * 8;                       // leaf: E_bf[tok]
                 cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r, c16), Arows + src, it.w != 0u);
             }
             cp_async_commit();
@@ -204,14 +249,16 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
         issue(0);
         if (n_chunks > 1) issue(1); else cp_async_commit();
         for (int kc = 0; kc < n_chunks; ++kc) {
+            // with a ring of 3 the stage of chunk kc + 2 is the one chunk kc - 1 used: its MMAs were
+            // committed one step ago, issue() waits for them
             if (kc + 2 < n_chunks) issue(kc + 2); else cp_async_commit();
             cp_async_wait<2>();                                          // this thread's copies of chunk kc have landed
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> async-proxy reads
             __syncthreads();
             if (threadIdx.x == 0) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t s = (it0 + kc) % TC_STAGES;
-                const uint32_t a = tc.a_addr + s * TC_A_STAGE, b = tc.b_addr + kc * ns * 128;
+                const uint32_t s = (it0 + kc) % stages;
+                const uint32_t a = tc.a_addr + s * TC_A_STAGE, b = tc.b_addr[RGN] + kc * ns * 128;
 #pragma unroll
                 for (int ks = 0; ks < TC_KC / 16; ++ks)
                     tc_mma(tc.tmem_base, tc_desc(a + ks * 32), tc_desc(b + ks * 32), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
@@ -222,45 +269,115 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
         // accumulators are complete when the last commit has arrived
         {
             const uint32_t g = tc.iter - 1;
-            if (ok) ok = mbar_wait(c, tc.mbar_addr + 8 * (g % TC_STAGES), (g / TC_STAGES) & 1u);
+            if (ok) ok = mbar_wait(c, tc.mbar_addr + 8 * (g % stages), (g / stages) & 1u);
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
-            // warp w reads TMEM lanes 32 (w % 4) ..; warps 0-3 take the first 16-column groups, warps 4-7 the rest
             const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-            const int row = (warp & 3) * 32 + lane;
-            const int groups = ns / 16, g_lo = (groups + 1) / 2;
-            const int g_begin = warp < 4 ? 0 : g_lo, g_end = warp < 4 ? g_lo : groups;
+            const int row = (warp & 3) * 32 + lane;                       // warp w reads TMEM lanes 32 (w % 4) ..
+            const uint32_t lane_base = tc.tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
             const uint4 it = s_items[row];
             const bool live = it.w != 0u;
-            for (int gi = g_begin; gi < g_end; ++gi) {
-                float v[16];
-                tc_ld16(tc.tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(gi * 16), v);
-                if (!live) continue;
-                const int col = slice * ns + gi * 16;                       // column of the padded N range
-                if (FWD) {
-                    __align__(16) __nv_bfloat16 hb[16];
+            if (MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) {
+                // slice = 16 hidden units, columns gate * 16 + unit; warps 0-3 take units 0-7, warps 4-7 units 8-15
+                constexpr int NG = MODE == TC_LSTM_CELL ? 5 : 3;
+                const int wg = warp >> 2, u0 = slice * 16 + wg * 8;
+                float v[NG][8];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float h = 0.f;
-                        if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
-                        hb[i] = __float2bfloat16_rn(h);
-                        v[i] = __bfloat162float(hb[i]);      // the state every consumer sees is the bf16 value
+                for (int g = 0; g < NG; ++g) tc_ld8(lane_base + (uint32_t)(g * 16 + wg * 8), v[g]);
+                if (live) {
+                    const float* bias = MODE == TC_LSTM_CELL ? c.b : c.b_x;
+                    float cl[8], cr[8], hv[8], cv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) cl[i] = cr[i] = 0.f;
+                    if (MODE == TC_LSTM_CELL) {
+#pragma unroll
+                        for (int i = 0; i < 8; i += 4)
+                            if (u0 + i < H) {
+                                const float4 a = ldcg4(c.arena + (size_t)it.y * S + H + u0 + i);
+                                const float4 b = ldcg4(c.arena + (size_t)it.z * S + H + u0 + i);
+                                cl[i] = a.x; cl[i + 1] = a.y; cl[i + 2] = a.z; cl[i + 3] = a.w;
+                                cr[i] = b.x; cr[i + 1] = b.y; cr[i + 2] = b.z; cr[i + 3] = b.w;
+                            }
                     }
-                    uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
-                    dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
-                    dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
-                    float* dstf = c.arena + (size_t)it.x * H + col;
+                    __align__(16) __nv_bfloat16 hb[8];
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4)
-                        if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                } else {
-                    const uint32_t child = col < Hp ? it.y : it.z;
-                    const int cc = col < Hp ? col : col - Hp;
-                    float* dst = c.dhp + (size_t)child * H + cc;
+                    for (int i = 0; i < 8; ++i) {
+                        const int u = u0 + i;
+                        float h = 0.f, cc = 0.f;
+                        if (u < H) {
+                            if (MODE == TC_LSTM_CELL) {
+                                const float gi = tc_sigmoid(v[0][i] + __ldg(&bias[u]));
+                                const float fl = tc_sigmoid(v[1][i] + __ldg(&bias[H + u]));
+                                const float fr = tc_sigmoid(v[2][i] + __ldg(&bias[2 * H + u]));
+                                const float go = tc_sigmoid(v[3 % NG][i] + __ldg(&bias[3 * H + u]));
+                                const float gu = tanhf(v[4 % NG][i] + __ldg(&bias[4 * H + u]));
+                                cc = gi * gu + fl * cl[i] + fr * cr[i];
+                                h = go * tanhf(cc);
+                                v[0][i] = gi; v[1][i] = fl; v[2][i] = fr; v[3 % NG][i] = go; v[4 % NG][i] = gu;
+                            } else {
+                                const float gi = tc_sigmoid(v[0][i] + __ldg(&bias[u]));
+                                const float go = tc_sigmoid(v[1][i] + __ldg(&bias[H + u]));
+                                const float gu = tanhf(v[2][i] + __ldg(&bias[2 * H + u]));
+                                cc = gi * gu;
+                                h = go * tanhf(cc);
+                                v[0][i] = gi; v[1][i] = go; v[2][i] = gu;
+                            }
+                        }
+                        hb[i] = __float2bfloat16_rn(h);
+                        hv[i] = __bfloat162float(hb[i]);        // the h every consumer sees is the bf16 value
+                        cv[i] = cc;
+                    }
+                    *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + u0) = *reinterpret_cast<const uint4*>(hb);
+                    float* st = c.arena + (size_t)it.x * S;
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4)
-                        if (cc + i < H) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    for (int i = 0; i < 8; i += 4)
+                        if (u0 + i < H) {
+                            *reinterpret_cast<float4*>(st + u0 + i) = make_float4(hv[i], hv[i + 1], hv[i + 2], hv[i + 3]);
+                            *reinterpret_cast<float4*>(st + H + u0 + i) = make_float4(cv[i], cv[i + 1], cv[i + 2], cv[i + 3]);
+                            if (c.gates) {
+                                float* gt = c.gates + (size_t)it.x * c.G;
+#pragma unroll
+                                for (int g = 0; g < NG; ++g)
+                                    *reinterpret_cast<float4*>(gt + g * H + u0 + i) =
+                                        make_float4(v[g][i], v[g][i + 1], v[g][i + 2], v[g][i + 3]);
+                            }
+                        }
+                }
+            } else {
+                // warps 0-3 take the first 16-column groups, warps 4-7 the rest
+                const int groups = ns / 16, g_lo = (groups + 1) / 2;
+                const int g_begin = warp < 4 ? 0 : g_lo, g_end = warp < 4 ? g_lo : groups;
+                for (int gi = g_begin; gi < g_end; ++gi) {
+                    float v[16];
+                    tc_ld16(lane_base + (uint32_t)(gi * 16), v);
+                    if (!live) continue;
+                    const int col = slice * ns + gi * 16;                       // column of the padded N range
+                    if (MODE == TC_RNN_FWD) {
+                        __align__(16) __nv_bfloat16 hb[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float h = 0.f;
+                            if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
+                            hb[i] = __float2bfloat16_rn(h);
+                            v[i] = __bfloat162float(hb[i]);      // the state every consumer sees is the bf16 value
+                        }
+                        uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
+                        dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
+                        dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
+                        float* dstf = c.arena + (size_t)it.x * H + col;
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else {
+                        // operand gradients: columns [0, Hp) belong to the left callee frame, [Hp, 2Hp) to the right
+                        const uint32_t child = col < Hp ? it.y : it.z;
+                        const int cc = col < Hp ? col : col - Hp;
+                        float* dst = c.dhp + (size_t)child * S + cc;
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            if (cc + i < H) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    }
                 }
             }
         }
@@ -315,5 +432,41 @@ static __global__ void __launch_bounds__(256) rdf_pack_w_kernel(const DevCtx c) 
         const __nv_bfloat16 b = __float2bfloat16_rn(v);
         c.Wp[idx] = b;
         c.WTp[(size_t)kp * Hp + j] = b;
+    }
+}
+
+// TreeLSTM packings (bf16).  Slice-major row order puts everything one block needs in consecutive rows:
+//   W5p [(ub*5 + g)*16 + i][k']  (5Hp x 2Hp): gate g of hidden unit u = ub*16 + i, K halves padded to Hp
+//   Wxp [(ub*3 + g)*16 + i][k]   (3Hp x Hp) : leaf projection, gates (i, o, u)
+//   WT5p[half*Hp + cc][g*Hp + j] (2Hp x 5Hp): gradient operand, = W[g*H + j][half*H + cc]
+static __global__ void __launch_bounds__(256) rdf_pack_lstm_kernel(const DevCtx c) {
+    const int Hp = c.Hp, Kp = 2 * c.Hp, H = c.H, D = c.D;
+    const int stride = gridDim.x * blockDim.x, tid = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int idx = tid; idx < 5 * Hp * Kp; idx += stride) {
+        const int R = idx / Kp, kp = idx % Kp;
+        const int ub = R / 80, g = (R % 80) / 16, u = ub * 16 + R % 16;
+        const int half = kp >= Hp, kk = kp - half * Hp;
+        float v = 0.f;
+        if (u < H && kk < H) v = c.W[(size_t)(g * H + u) * 2 * H + half * H + kk];
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        c.Wp[idx] = b;
+        c.WTp[(size_t)kp * 5 * Hp + g * Hp + u] = b;
+    }
+    for (int idx = tid; idx < 3 * Hp * Hp; idx += stride) {
+        const int R = idx / Hp, k = idx % Hp;
+        const int ub = R / 48, g = (R % 48) / 16, u = ub * 16 + R % 16;
+        float v = 0.f;
+        if (u < H && k < D) v = c.W_x[(size_t)(g * H + u) * D + k];
+        c.Wxp[idx] = __float2bfloat16_rn(v);
+    }
+}
+
+// E_bf[v][k] (V x Hp): the embedding table in bf16 with zero pad columns (operand rows of the leaf projection)
+static __global__ void __launch_bounds__(256) rdf_pack_e_kernel(const DevCtx c) {
+    const size_t total = (size_t)c.V * c.Hp;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const size_t v = idx / c.Hp;
+        const int k = (int)(idx % c.Hp);
+        c.E_bf[idx] = __float2bfloat16_rn(k < c.D ? c.E[v * c.D + k] : 0.f);
     }
 }

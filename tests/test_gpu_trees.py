@@ -186,6 +186,17 @@ def test_treelstm_ragged_hidden_size():
     check_grad(_lstm_cfg(48, 700, 300), cell="lstm")
 
 
+@pytest.mark.parametrize("H", [64, 300])
+def test_treelstm_bf16_tensor_core_path(H):
+    """TreeLSTM with bf16 operands on the tensor cores: weights are bf16-representable, h is rounded to
+    bf16 after every cell (c stays fp32); tolerance 2e-2."""
+    cfg = workloads.config(4, B=200, V=900, H=H)
+    check_forward(cfg, rdf.BF16, cell="lstm")
+    check_grad(cfg, rdf.BF16, cell="lstm")
+    st = check_forward(workloads.config(4, B=700, V=900, H=H), rdf.BF16, cell="lstm")
+    assert st["cells"] > 3 * 128
+
+
 def test_treelstm_config4_full_size():
     """Binary TreeLSTM, 8192 trees, H = 300, fwd + bwd in the benchmark's launch configuration.
     The fp64 oracle needs ~3 ms per node for this gradient, so at full size it checks what it can
