@@ -125,6 +125,7 @@ struct DevCtx {
     uint32_t* bq[2];              // backward wave queues (frame ids)
     uint32_t* all_cells;          // every cell frame, in backward wave order
     uint4*    cell_ops;           // {cell frame, left operand frame, right operand frame, 1} in all_cells order
+    uint4*    leaf_ops;           // {leaf frame, token id, 0, 1} in all_leaves order
     uint32_t* all_leaves;         // every leaf frame
     float*    loss_partial;       // per-block partial sums of the loss
     float    *dE, *dW, *db, *dW_x, *db_x, *dW_s, *db_s;

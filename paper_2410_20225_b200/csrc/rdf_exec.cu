@@ -495,6 +495,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.bq1 = P.take<uint32_t>(gf);
     L.all_cells = P.take<uint32_t>(gf);
     L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
+    L.leaf_ops = P.take<uint4>(tcl ? gf : 0);
     L.all_leaves = P.take<uint32_t>(gf);
     L.loss_partial = P.take<float>(want_grad ? 4096 : 0);
     L.total = (P.off + 255) & ~(size_t)255;
@@ -579,6 +580,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.bq[0] = reinterpret_cast<uint32_t*>(ws + L.bq0); c.bq[1] = reinterpret_cast<uint32_t*>(ws + L.bq1);
     c.all_cells = reinterpret_cast<uint32_t*>(ws + L.all_cells);
     c.cell_ops = L.use_tc ? reinterpret_cast<uint4*>(ws + L.cell_ops) : nullptr;
+    c.leaf_ops = L.use_tc && g->has_lstm ? reinterpret_cast<uint4*>(ws + L.leaf_ops) : nullptr;
     c.all_leaves = reinterpret_cast<uint32_t*>(ws + L.all_leaves);
     c.loss_partial = reinterpret_cast<float*>(ws + L.loss_partial);
     c.loss_out = out->loss;

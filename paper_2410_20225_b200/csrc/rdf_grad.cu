@@ -120,6 +120,7 @@ __device__ __forceinline__ void backward_enqueue_block(const DevCtx& c, uint32_t
     if (mine) {
         if (leaf) {
             c.all_leaves[base[1] + local] = t;
+            if (c.leaf_ops) c.leaf_ops[base[1] + local] = make_uint4(t, r, 0u, 1u);      // r = token id of a leaf
         } else {
             const uint32_t idx = base[0] + local;
             c.all_cells[idx] = t;
@@ -218,23 +219,33 @@ __device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n)
             if (leaf) {
                 const float gi = __ldcg(&gt[j]), go = __ldcg(&gt[H + j]), gu = __ldcg(&gt[2 * H + j]);
                 const float dc = dc_in + dh * go * (1.f - tc * tc);
-                gt[j] = dc * gu * gi * (1.f - gi);
-                gt[H + j] = dh * tc * go * (1.f - go);
-                gt[2 * H + j] = dc * gi * (1.f - gu * gu);
+                const float g0 = dc * gu * gi * (1.f - gi), g1 = dh * tc * go * (1.f - go), g2 = dc * gi * (1.f - gu * gu);
+                gt[j] = g0; gt[H + j] = g1; gt[2 * H + j] = g2;
+                if (c.dg_bf) {
+                    __nv_bfloat16* gb = c.dg_bf + (size_t)t * 5 * c.Hp;
+                    gb[j] = __float2bfloat16_rn(g0); gb[c.Hp + j] = __float2bfloat16_rn(g1); gb[2 * c.Hp + j] = __float2bfloat16_rn(g2);
+                }
             } else {
                 const float gi = __ldcg(&gt[j]), fl = __ldcg(&gt[H + j]), fr = __ldcg(&gt[2 * H + j]);
                 const float go = __ldcg(&gt[3 * H + j]), gu = __ldcg(&gt[4 * H + j]);
                 const float cl = __ldcg(&c.arena[(size_t)l * S + H + j]), cr = __ldcg(&c.arena[(size_t)r * S + H + j]);
                 const float dc = dc_in + dh * go * (1.f - tc * tc);
-                gt[j] = dc * gu * gi * (1.f - gi);
-                gt[H + j] = dc * cl * fl * (1.f - fl);
-                gt[2 * H + j] = dc * cr * fr * (1.f - fr);
-                gt[3 * H + j] = dh * tc * go * (1.f - go);
-                gt[4 * H + j] = dc * gi * (1.f - gu * gu);
+                const float g0 = dc * gu * gi * (1.f - gi), g1 = dc * cl * fl * (1.f - fl), g2 = dc * cr * fr * (1.f - fr);
+                const float g3 = dh * tc * go * (1.f - go), g4 = dc * gi * (1.f - gu * gu);
+                gt[j] = g0; gt[H + j] = g1; gt[2 * H + j] = g2; gt[3 * H + j] = g3; gt[4 * H + j] = g4;
+                if (c.dg_bf) {
+                    __nv_bfloat16* gb = c.dg_bf + (size_t)t * 5 * c.Hp;
+                    gb[j] = __float2bfloat16_rn(g0); gb[c.Hp + j] = __float2bfloat16_rn(g1);
+                    gb[2 * c.Hp + j] = __float2bfloat16_rn(g2); gb[3 * c.Hp + j] = __float2bfloat16_rn(g3);
+                    gb[4 * c.Hp + j] = __float2bfloat16_rn(g4);
+                }
                 c.dhp[(size_t)l * S + H + j] = dc * fl;
                 c.dhp[(size_t)r * S + H + j] = dc * fr;
             }
         }
+        if (c.dg_bf)                      // pad columns of every gate block are zero
+            for (int q = lane; q < (leaf ? 3 : 5) * (c.Hp - H); q += 32)
+                c.dg_bf[(size_t)t * 5 * c.Hp + (q / (c.Hp - H)) * c.Hp + H + q % (c.Hp - H)] = __float2bfloat16_rn(0.f);
         }
         backward_enqueue_block(c, wave, act && lane == 0, t, leaf, l, r);
     }
@@ -344,8 +355,11 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
     __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
     __shared__ uint4 tc_items[TC_M];
     TcState tc;
-    const bool tc_on = c.use_tc && !c.lstm;        // the TreeLSTM gradient contractions run on the FMA tiles
-    if (tc_on) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 8, 4, c.WTp, c.Hp, c.Hp / 4);
+    const bool tc_on = c.use_tc;
+    if (tc_on) {
+        if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 2 * c.Hp / 32, 4, c.WTp, 5 * c.Hp, 32);
+        else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 8, 4, c.WTp, c.Hp, c.Hp / 4);
+    }
     uint32_t generation = 0, wave = 0, first = 0;
     long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
@@ -369,7 +383,8 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         lap(cyc_b);
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
-            if (tc_on) tc_tiles<TC_RNN_BWD>(c, tc, tc_items, first, end - first);
+            if (tc_on && c.lstm) tc_tiles<TC_LSTM_BWD>(c, tc, tc_items, first, end - first);
+            else if (tc_on) tc_tiles<TC_RNN_BWD>(c, tc, tc_items, first, end - first);
             else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
             else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
                 backward_operand_thin(c, reinterpret_cast<float*>(&tile_smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
@@ -619,32 +634,46 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
-    const bool tc_rnn = c.use_tc && !lstm;
-    if (tc_rnn) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
+    const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
+    if (c.use_tc) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args,
-                                        tc_rnn ? (size_t)L.tc_smem_bwd : 0, stream));
+                                        c.use_tc ? (size_t)L.tc_smem_bwd : 0, stream));
     rdf_mark(S, 4, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
     const long long max_leaves = std::max<long long>(1, in->max_invocations);
     const float* dgA = lstm ? c.gates : c.dhp;
     const int lda = lstm ? c.G : H;
-    if (tc_rnn) {
-        // 128 x 128 tiles of the padded [Hp x 2Hp] gradient, the cells split over the remaining blocks
-        const int tiles_m = (c.Hp + 127) / 128, tiles_n = (2 * c.Hp + 127) / 128, n_tiles = tiles_m * tiles_n;
-        const int splits = std::max(1, S->grid / n_tiles);
-        uint32_t chunk = (uint32_t)((max_cells + splits - 1) / splits);
-        chunk = (chunk + DW_KT - 1) / DW_KT * DW_KT;
-        const int blocks = n_tiles * (int)((max_cells + chunk - 1) / chunk);
+    if (c.use_tc) {
+        // 128 x 128 tiles of the padded gradient, the invocations split over the remaining blocks
         CUDA_OK(cudaFuncSetAttribute(rdf_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BYTES));
-        rdf_dw_tc_kernel<<<blocks, 256, DW_SMEM_BYTES, stream>>>(c, tiles_n, n_tiles, chunk, 8192u, 1024u);
+        auto launch_dw = [&](DwArgs a, long long max_items) {
+            a.tiles_n = (a.Np + 127) / 128;
+            a.n_tiles = ((a.Mp + 127) / 128) * a.tiles_n;
+            const int splits = std::max(1, S->grid / a.n_tiles);
+            uint32_t chunk = (uint32_t)((max_items + splits - 1) / splits);
+            a.chunk = (chunk + DW_KT - 1) / DW_KT * DW_KT;
+            const int blocks = a.n_tiles * (int)((max_items + a.chunk - 1) / a.chunk);
+            rdf_dw_tc_kernel<<<blocks, 256, DW_SMEM_BYTES, stream>>>(c, a);
+        };
+        DwArgs a{};
+        a.ops = c.cell_ops; a.count = &c.ctl->all_cells;
+        a.A = tc_lstm ? c.dg_bf : c.dz_bf; a.lda = tc_lstm ? 5 * c.Hp : c.Hp; a.Mp = tc_lstm ? 5 * c.Hp : c.Hp;
+        a.Np = 2 * c.Hp; a.mode = 0; a.out = grads->dW; a.ldo = 2 * H;
+        launch_dw(a, max_cells);
+        if (tc_lstm) {
+            DwArgs x{};
+            x.ops = c.leaf_ops; x.count = &c.ctl->all_leaves;
+            x.A = c.dg_bf; x.lda = 5 * c.Hp; x.Mp = 3 * c.Hp; x.Np = c.Hp; x.mode = 1; x.out = grads->dW_x; x.ldo = D;
+            launch_dw(x, max_leaves);
+        }
     } else {
         OuterArgs aw = outer_args(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, 2 * H, 0, grads->dW, max_cells, S->grid);
         rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw);
-    }
-    if (lstm) {
-        OuterArgs ax = outer_args(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, D, 1, grads->dW_x, max_leaves, S->grid);
-        rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
+        if (lstm) {
+            OuterArgs ax = outer_args(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, D, 1, grads->dW_x, max_leaves, S->grid);
+            rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
+        }
     }
     rdf_mark(S, 5, stream);
     rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);

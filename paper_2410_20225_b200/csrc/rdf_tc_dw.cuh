@@ -27,18 +27,33 @@ __device__ __forceinline__ uint64_t tc_desc_mn(uint32_t smem_addr, uint32_t lbo,
     return d;
 }
 
-__global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int tiles_n, int n_tiles, uint32_t chunk,
-                                                           uint32_t lbo, uint32_t sbo) {
+// What to contract:  out[row(m)][col(n)] += sum over the listed invocations t of A_t[m] * B_t[n]
+//   A_t = A + t * lda, Mp padded rows in blocks of Hp (block g, unit j -> output row g * H + j, j < H)
+//   mode 0: B_t = [h(l_t) ; h(r_t)] from arena_bf (Np = 2 Hp; column half * Hp + k -> output column half * H + k)
+//   mode 1: B_t = E_bf[tok_t]                     (Np = Hp;  column k -> output column k, k < D)
+struct DwArgs {
+    const uint4* ops;            // {frame, left / token, right, valid} per listed invocation
+    const uint32_t* count;
+    const __nv_bfloat16* A;
+    int lda, Mp, Np, mode;
+    float* out;
+    int ldo;
+    int tiles_n, n_tiles;
+    uint32_t chunk;
+};
+
+__global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const DwArgs a) {
+    const uint32_t lbo = 8192u, sbo = 1024u;       // next atom along M/N, next atom along K
     extern __shared__ unsigned char dyn_smem[];
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(8) uint64_t mbars[DW_STAGES];
     __shared__ uint4 s_ops[DW_STAGES][DW_KT];
-    const uint32_t n_cells = c.ctl->all_cells;
-    const int tile = blockIdx.x % n_tiles, split = blockIdx.x / n_tiles;
-    const uint32_t t_begin = (uint32_t)split * chunk, t_end = min(n_cells, t_begin + chunk);
+    const uint32_t n_cells = *a.count;
+    const int tile = blockIdx.x % a.n_tiles, split = blockIdx.x / a.n_tiles;
+    const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_cells, t_begin + a.chunk);
     if (t_begin >= t_end) return;                                  // the whole block leaves before any set-up
-    const int H = c.H, Hp = c.Hp, K2p = 2 * c.Hp;
-    const int m0 = (tile / tiles_n) * 128, n0 = (tile % tiles_n) * 128;
+    const int H = c.H, Hp = c.Hp;
+    const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
     const int n_chunks = (int)((t_end - t_begin + DW_KT - 1) / DW_KT);
 
     const uint32_t raw = smem_u32(dyn_smem);
@@ -56,7 +71,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int t
         if (threadIdx.x < DW_KT) {
             const uint32_t idx = t_begin + kc * DW_KT + threadIdx.x;
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (idx < t_end) v = *reinterpret_cast<const uint4*>(&c.cell_ops[idx]);     // {t, l, r, 1}
+            if (idx < t_end) v = a.ops[idx];
             s_ops[kc % DW_STAGES][threadIdx.x] = v;
         }
     };
@@ -77,11 +92,13 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int t
             const uint4 it = s_ops[s][tr];
             const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
             const int m = m0 + atom * 64 + c16 * 8;
-            cp_async16(a_st + off, c.dz_bf + (size_t)it.x * Hp + (m < Hp ? m : 0), it.w != 0u && m < Hp);
+            const bool mv = it.w != 0u && m < a.Mp;
+            cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
             const int n = n0 + atom * 64 + c16 * 8;
-            const bool nv = it.w != 0u && n < K2p;
-            const size_t src = n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (nv ? n - Hp : 0);
-            cp_async16(b_st + off, c.arena_bf + src, nv);
+            const bool nv = it.w != 0u && n < a.Np;
+            size_t src = 0;
+            if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
+            cp_async16(b_st + off, (a.mode == 0 ? c.arena_bf : c.E_bf) + src, nv);
         }
         cp_async_commit();
     };
@@ -98,7 +115,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int t
             const uint32_t s = kc % DW_STAGES;
             const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
 #pragma unroll
-            for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 cells = two K atoms = 2048 bytes per step
+            for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 invocations = two K atoms = 2048 bytes per step
                 tc_mma(tmem, tc_desc_mn(a_st + ks * 2048, lbo, sbo), tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc,
                        (kc > 0 || ks > 0) ? 1u : 0u);
             tc_commit(mbar + 8 * s);
@@ -112,16 +129,18 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, int t
     if (ok) {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
         const int m = m0 + (warp & 3) * 32 + lane;
+        const int mj = m % Hp, row = (m / Hp) * H + mj;              // gate block, unit
+        const int n_limit = a.mode == 0 ? H : c.D;
         for (int gi = 0; gi < 4; ++gi) {
             float v[16];
             const int cl = (warp >> 2) * 64 + gi * 16;
             tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)cl, v);
-            if (m >= H) continue;
+            if (m >= a.Mp || mj >= H) continue;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int n = n0 + cl + i;
                 const int k = n < Hp ? n : n - Hp;
-                if (n < K2p && k < H) atomicAdd(&c.dW[(size_t)m * 2 * H + (n < Hp ? k : H + k)], v[i]);
+                if (n < a.Np && k < n_limit) atomicAdd(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)], v[i]);
             }
         }
     }
