@@ -570,7 +570,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
         c.Wxp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxp);
         c.E_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.e_bf);
-        c.dg_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dg_bf);
+        // only present (and only non-null) for the TreeLSTM on the tensor-core path
+        c.dg_bf = L.use_tc && g->has_lstm ? reinterpret_cast<__nv_bfloat16*>(ws + L.dg_bf) : nullptr;
     } else {
         c.y = out->y;
     }
