@@ -34,7 +34,7 @@ WORKLOAD_NAMES = {
     4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13, "grad_tc": 12}
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13, "grad_tc": 12, "grad_lstm_tc": 15}
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
 
 
@@ -163,6 +163,31 @@ def time_oracle(cfg, steps, warmup, scale=1):
     return n / dt, dt / steps, what
 
 
+# --------------------------------------------------------------------------- multi-rank host logic
+def rank_seed(seed, rank):
+    """Every rank draws a batch of its own: instances never exchange tokens (weak scaling)."""
+    return seed + rank
+
+
+def reduce_job(dist, device, elapsed, units):
+    """Whole-job figures from per-rank ones: time = max over ranks, units = sum over ranks."""
+    import torch
+    if dist is None:
+        return float(elapsed), float(units)
+    t = torch.tensor([elapsed], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(n)
+    return float(t.item()), float(n.item())
+
+
+def sum_gradients(dist, grads):
+    """The one exchange step of data-parallel rdf_grad: parameter gradients are summed over ranks."""
+    if dist is not None:
+        for t in grads.values():
+            dist.all_reduce(t)
+
+
 # --------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -207,7 +232,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # every rank processes a batch of its own (instances never exchange tokens): weak scaling
-    cfg = load(args.workload, args.seed + rank)
+    cfg = load(args.workload, rank_seed(args.seed, rank))
     N = cfg["N"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
 
@@ -235,8 +260,8 @@ def main():
         g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
         compute = rdf.BF16 if cfg["bf16"] else rdf.F32
         # arithmetic type of the contractions: bf16 operands on the tensor cores (fp32 accumulate) for the
-        # bf16 TreeRNN workload, fp32 FMA otherwise (the TreeLSTM contractions are fp32 as built)
-        use_tc = cfg["bf16"] and CELL[cfg["kind"]] == "rnn"
+        # bf16 workloads, fp32 FMA otherwise
+        use_tc = bool(cfg["bf16"])
         dtype = "bf16" if use_tc else "f32"
         host = {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).pin_memory()
                 for k in ("tree_root", "left", "right", "tok", "label")}
@@ -248,22 +273,18 @@ def main():
         if cell == "lstm":
             flops_fwd = tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
         if cfg["grad"]:
-            kind = "grad_lstm" if cell == "lstm" else ("grad_tc" if use_tc else "grad")
+            kind = ("grad_lstm_tc" if use_tc else "grad_lstm") if cell == "lstm" else ("grad_tc" if use_tc else "grad")
             grads = {k: torch.empty_like(v) for k, v in dp.items()}
             loss = torch.zeros(1, dtype=torch.float32, device="cuda")
 
             def step():
                 g.grad_trees(dt, dp, compute, check=False, grads=grads, loss=loss, h_root=h_root)
-                if dist is not None:            # data-parallel exchange: one sum of the parameter gradients
-                    for t in grads.values():
-                        dist.all_reduce(t)
+                sum_gradients(dist, grads)      # data-parallel exchange: one sum of the parameter gradients
 
             def step_e2e():
                 d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
                 l, _, _ = g.grad_trees(d, dp, compute, check=False, grads=grads, h_root=h_root)
-                if dist is not None:
-                    for t in grads.values():
-                        dist.all_reduce(t)
+                sum_gradients(dist, grads)
                 return l.item()
             h2d, d2h = sum(v.numel() * 4 for v in host.values()), 4
         else:
@@ -306,16 +327,7 @@ def main():
     barrier()
     clk = clocks.stop()
     st = g.stats()
-    total_ms = sum(times)
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        n_all = torch.tensor([N], dtype=torch.float64, device="cuda")
-        dist.all_reduce(n_all)
-        N_all = float(n_all.item())
-    else:
-        N_all = float(N)
+    total_ms, N_all = reduce_job(dist, "cuda", sum(times), N)
     value = N_all * args.steps / (total_ms * 1e-3)
 
     # ---- end to end through the public call, host buffers, copies inside the timed region
@@ -327,10 +339,7 @@ def main():
         step_e2e()
     barrier()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s, _ = reduce_job(dist, "cuda", e2e_s, N)
     e2e_value = N_all * args.steps / e2e_s
 
     if rank != 0:
