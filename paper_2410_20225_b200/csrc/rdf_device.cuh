@@ -108,6 +108,7 @@ struct DevCtx {
     __nv_bfloat16* dz_bf;         // [frame_cap, Hp] bf16 copy of dz (rdf_grad)
     // TreeLSTM on tensor cores: Wp / WTp hold the slice-major W5p [5Hp, 2Hp] and WT5p [2Hp, 5Hp]
     __nv_bfloat16* Wxp;           // [3Hp, Hp] leaf projection, slice-major
+    __nv_bfloat16* WxTp;          // [Hp, 3Hp] its transpose (operand of the embedding gradient)
     __nv_bfloat16* E_bf;          // [V, Hp] embedding table in bf16
     __nv_bfloat16* dg_bf;         // [frame_cap, 5Hp] bf16 gate gradients (rdf_grad)
     int       Hp, use_tc;

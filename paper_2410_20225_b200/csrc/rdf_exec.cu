@@ -483,6 +483,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.wtp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
     L.dz_bf = P.take<__nv_bfloat16>(tcr && want_grad ? vf * L.Hp : 0);
     L.wxp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
+    L.wxtp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
     L.dg_bf = P.take<__nv_bfloat16>(tcl && want_grad ? vf * 5 * L.Hp : 0);
     L.tc_smem_fwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(80, 2 * L.Hp, 48, L.Hp, 3) : tc_smem_bytes(L.Hp / 4, 2 * L.Hp, 0, 0, 4);
@@ -569,6 +570,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.WTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wtp);
         c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
         c.Wxp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxp);
+        c.WxTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxtp);
         c.E_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.e_bf);
         // only present (and only non-null) for the TreeLSTM on the tensor-core path
         c.dg_bf = L.use_tc && g->has_lstm ? reinterpret_cast<__nv_bfloat16*>(ws + L.dg_bf) : nullptr;

@@ -209,38 +209,66 @@ __device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n)
         const float* g = c.dhp + (size_t)t * S;
         const float* st = c.arena + (size_t)t * S;
         float* gt = c.gates + (size_t)t * c.G;
-        for (int j = lane; j < H; j += 32) {
-            float dh = from_result ? 0.f : __ldcg(&g[j]);
-            const float dc_in = from_result ? 0.f : __ldcg(&g[H + j]);
+        // 128-bit accesses: four hidden units per lane and step
+        auto ld = [](const float* p) { const float4 v = ldcg4(p); return v; };
+        auto st4 = [](float* p, const float (&v)[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); };
+        auto stb = [&](int gate, int j, const float (&v)[4]) {
+            if (!c.dg_bf) return;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(c.dg_bf + (size_t)t * 5 * c.Hp + gate * c.Hp + j) = pk;
+        };
+        for (int j = lane * 4; j < H; j += 128) {
+            const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 dh4 = from_result ? z4 : ld(g + j), dc4 = from_result ? z4 : ld(g + H + j), c4 = ld(st + H + j);
+            float dh[4] = {dh4.x, dh4.y, dh4.z, dh4.w};
+            const float dci[4] = {dc4.x, dc4.y, dc4.z, dc4.w}, cc[4] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) dh = fmaf(__ldg(&c.W_s[k * H + j]), dl[k], dh);
-            const float tc = tanhf(__ldcg(&st[H + j]));
+                if (k < C) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                    dh[0] = fmaf(w.x, dl[k], dh[0]); dh[1] = fmaf(w.y, dl[k], dh[1]);
+                    dh[2] = fmaf(w.z, dl[k], dh[2]); dh[3] = fmaf(w.w, dl[k], dh[3]);
+                }
             if (leaf) {
-                const float gi = __ldcg(&gt[j]), go = __ldcg(&gt[H + j]), gu = __ldcg(&gt[2 * H + j]);
-                const float dc = dc_in + dh * go * (1.f - tc * tc);
-                const float g0 = dc * gu * gi * (1.f - gi), g1 = dh * tc * go * (1.f - go), g2 = dc * gi * (1.f - gu * gu);
-                gt[j] = g0; gt[H + j] = g1; gt[2 * H + j] = g2;
-                if (c.dg_bf) {
-                    __nv_bfloat16* gb = c.dg_bf + (size_t)t * 5 * c.Hp;
-                    gb[j] = __float2bfloat16_rn(g0); gb[c.Hp + j] = __float2bfloat16_rn(g1); gb[2 * c.Hp + j] = __float2bfloat16_rn(g2);
+                const float4 a4 = ld(gt + j), o4 = ld(gt + H + j), u4 = ld(gt + 2 * H + j);
+                const float gi[4] = {a4.x, a4.y, a4.z, a4.w}, go[4] = {o4.x, o4.y, o4.z, o4.w}, gu[4] = {u4.x, u4.y, u4.z, u4.w};
+                float g0[4], g1[4], g2[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float tc = tanhf(cc[e]);
+                    const float dc = dci[e] + dh[e] * go[e] * (1.f - tc * tc);
+                    g0[e] = dc * gu[e] * gi[e] * (1.f - gi[e]);
+                    g1[e] = dh[e] * tc * go[e] * (1.f - go[e]);
+                    g2[e] = dc * gi[e] * (1.f - gu[e] * gu[e]);
                 }
+                st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2);
+                stb(0, j, g0); stb(1, j, g1); stb(2, j, g2);
             } else {
-                const float gi = __ldcg(&gt[j]), fl = __ldcg(&gt[H + j]), fr = __ldcg(&gt[2 * H + j]);
-                const float go = __ldcg(&gt[3 * H + j]), gu = __ldcg(&gt[4 * H + j]);
-                const float cl = __ldcg(&c.arena[(size_t)l * S + H + j]), cr = __ldcg(&c.arena[(size_t)r * S + H + j]);
-                const float dc = dc_in + dh * go * (1.f - tc * tc);
-                const float g0 = dc * gu * gi * (1.f - gi), g1 = dc * cl * fl * (1.f - fl), g2 = dc * cr * fr * (1.f - fr);
-                const float g3 = dh * tc * go * (1.f - go), g4 = dc * gi * (1.f - gu * gu);
-                gt[j] = g0; gt[H + j] = g1; gt[2 * H + j] = g2; gt[3 * H + j] = g3; gt[4 * H + j] = g4;
-                if (c.dg_bf) {
-                    __nv_bfloat16* gb = c.dg_bf + (size_t)t * 5 * c.Hp;
-                    gb[j] = __float2bfloat16_rn(g0); gb[c.Hp + j] = __float2bfloat16_rn(g1);
-                    gb[2 * c.Hp + j] = __float2bfloat16_rn(g2); gb[3 * c.Hp + j] = __float2bfloat16_rn(g3);
-                    gb[4 * c.Hp + j] = __float2bfloat16_rn(g4);
+                const float4 a4 = ld(gt + j), l4 = ld(gt + H + j), r4 = ld(gt + 2 * H + j), o4 = ld(gt + 3 * H + j), u4 = ld(gt + 4 * H + j);
+                const float4 cl4 = ld(c.arena + (size_t)l * S + H + j), cr4 = ld(c.arena + (size_t)r * S + H + j);
+                const float gi[4] = {a4.x, a4.y, a4.z, a4.w}, fl[4] = {l4.x, l4.y, l4.z, l4.w}, fr[4] = {r4.x, r4.y, r4.z, r4.w};
+                const float go[4] = {o4.x, o4.y, o4.z, o4.w}, gu[4] = {u4.x, u4.y, u4.z, u4.w};
+                const float cl[4] = {cl4.x, cl4.y, cl4.z, cl4.w}, cr[4] = {cr4.x, cr4.y, cr4.z, cr4.w};
+                float g0[4], g1[4], g2[4], g3[4], g4[4], dl_[4], dr_[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float tc = tanhf(cc[e]);
+                    const float dc = dci[e] + dh[e] * go[e] * (1.f - tc * tc);
+                    g0[e] = dc * gu[e] * gi[e] * (1.f - gi[e]);
+                    g1[e] = dc * cl[e] * fl[e] * (1.f - fl[e]);
+                    g2[e] = dc * cr[e] * fr[e] * (1.f - fr[e]);
+                    g3[e] = dh[e] * tc * go[e] * (1.f - go[e]);
+                    g4[e] = dc * gi[e] * (1.f - gu[e] * gu[e]);
+                    dl_[e] = dc * fl[e];
+                    dr_[e] = dc * fr[e];
                 }
-                c.dhp[(size_t)l * S + H + j] = dc * fl;
-                c.dhp[(size_t)r * S + H + j] = dc * fr;
+                st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2); st4(gt + 3 * H + j, g3); st4(gt + 4 * H + j, g4);
+                stb(0, j, g0); stb(1, j, g1); stb(2, j, g2); stb(3, j, g3); stb(4, j, g4);
+                st4(c.dhp + (size_t)l * S + H + j, dl_);
+                st4(c.dhp + (size_t)r * S + H + j, dr_);
             }
         }
         if (c.dg_bf)                      // pad columns of every gate block are zero
@@ -681,7 +709,11 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_mark(S, 6, stream);
     rdf_dws_kernel<<<16 * S->grid, 128, 0, stream>>>(c);
     rdf_mark(S, 7, stream);
-    if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
+    if (tc_lstm) {
+        const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 4);
+        CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));
+        rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, 256, de_smem, stream>>>(c);
+    } else if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
     else rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
     rdf_mark(S, 8, stream);
     CUDA_OK(cudaGetLastError());

@@ -31,7 +31,8 @@ enum TcMode {
     TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: operand gradients
     TC_LSTM_CELL = 2,   // A = [h_l ; h_r],                B = W5p slice (5 gates x 16 units); epilogue: gates, c, h
     TC_LSTM_LEAF = 3,   // A = E_bf[tok],                  B = Wxp slice (3 gates x 16 units); epilogue: gates, c, h
-    TC_LSTM_BWD = 4     // A = gate gradients (5 Hp),      B = WT5p slice;         epilogue: operand gradients (dh)
+    TC_LSTM_BWD = 4,    // A = gate gradients (5 Hp),      B = WT5p slice;         epilogue: operand gradients (dh)
+    TC_LSTM_DE = 5      // A = leaf gate gradients (3 Hp), B = WxTp slice;         epilogue: dE[tok] += W_x^T dg
 };
 
 struct TcState {
@@ -204,7 +205,7 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
     if (rg >= n_rg) return;                                    // blocks beyond the last full group sit this out
     const uint32_t idesc = tc_idesc(ns);
     const int tiles = (n_items + TC_M - 1) / TC_M;
-    const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : MODE == TC_LSTM_BWD ? c.dg_bf
+    const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? c.dg_bf
                                  : MODE == TC_LSTM_LEAF ? c.E_bf : c.arena_bf;
     bool ok = true;
     for (int tile = rg; tile < tiles && ok; tile += n_rg) {
@@ -213,7 +214,9 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
             uint4 it = make_uint4(0u, 0u, 0u, 0u);
             const int row = row0 + threadIdx.x;
             if (row < (int)n_items) {
-                if (GRAD) {
+                if (MODE == TC_LSTM_DE) {
+                    it = c.leaf_ops[first + row];                                    // {leaf frame, token id, -, 1}
+                } else if (GRAD) {
                     const uint32_t t = __ldcg(&c.all_cells[first + row]);
                     it.x = t; it.y = __ldcg(&c.op_l[t]); it.z = __ldcg(&c.op_r[t]);
                 } else if (MODE == TC_LSTM_LEAF) {
@@ -240,7 +243,7 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
                 if (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL)
                     src = (size_t)(koff < Hp ? it.y : it.z) * Hp + (koff < Hp ? koff : koff - Hp) + c16 * 8;
                 else if (MODE == TC_RNN_BWD) src = (size_t)it.x * Hp + koff + c16 * 8;
-                else if (MODE == TC_LSTM_BWD) src = (size_t)it.x * 5 * Hp + koff + c16 * 8;
+                else if (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) src = (size_t)it.x * 5 * Hp + koff + c16 * 8;
                 else src = (size_t)it.y * Hp + koff + c16 * 8;                       // leaf: E_bf[tok]
                 cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r, c16), Arows + src, it.w != 0u);
             }
@@ -369,6 +372,11 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
 #pragma unroll
                         for (int i = 0; i < 16; i += 4)
                             if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else if (MODE == TC_LSTM_DE) {
+                        // embedding gradient: row tok of dE gathers the contribution of this leaf
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (col + i < c.D) atomicAdd(&c.dE[(size_t)it.y * c.D + col + i], v[i]);
                     } else {
                         // operand gradients: columns [0, Hp) belong to the left callee frame, [Hp, 2Hp) to the right
                         const uint32_t child = col < Hp ? it.y : it.z;
@@ -457,8 +465,22 @@ static __global__ void __launch_bounds__(256) rdf_pack_lstm_kernel(const DevCtx 
         const int ub = R / 48, g = (R % 48) / 16, u = ub * 16 + R % 16;
         float v = 0.f;
         if (u < H && k < D) v = c.W_x[(size_t)(g * H + u) * D + k];
-        c.Wxp[idx] = __float2bfloat16_rn(v);
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        c.Wxp[idx] = b;
+        if (k < Hp) c.WxTp[(size_t)k * 3 * Hp + g * Hp + u] = b;       // WxTp[d][g*Hp + j] = W_x[g*H + j][d]
     }
+}
+
+// dE of the TreeLSTM on tensor cores: one launch after the gradient waves, blocks = (row group, 64-column slice of D)
+static __global__ void __launch_bounds__(256, 1) rdf_de_tc_kernel(const DevCtx c) {
+    extern __shared__ unsigned char dyn_smem[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
+    __shared__ uint4 tc_items[TC_M];
+    TcState tc;
+    tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Hp / 64, 4, c.WxTp, 3 * c.Hp, 64);
+    tc_tiles<TC_LSTM_DE>(c, tc, tc_items, 0, c.ctl->all_leaves);
+    tc_teardown(tc);
 }
 
 // E_bf[v][k] (V x Hp): the embedding table in bf16 with zero pad columns (operand rows of the leaf projection)
