@@ -234,3 +234,11 @@ def test_depth_stress_config5_forward_sampled():
     cfg = workloads.config(5)
     st = check_forward(cfg, trees=[0, 63, 64])
     assert st["waves"] >= 2 * 4096
+
+
+def test_depth_stress_config5_full_size_gradients():
+    """Config 5 at full size, forward + backward in fp32: 64 chains of depth 4096 and 16 perfect trees of
+    2^16 leaves (2.6 M invocations); every output against the fp64 oracle run over a pool of processes."""
+    st, errs = check_grad(workloads.config(5), rdf.F32, workers=WORKERS)
+    print("config 5 errors:", errs)
+    assert st["waves_backward"] >= 4096
