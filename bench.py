@@ -89,8 +89,8 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- workloads
-def load(k, seed):
-    cfg = workloads.config(k, seed=seed)
+def load(k, seed, fib_batch=None):
+    cfg = workloads.config(k, seed=seed, B=fib_batch) if (k == 1 and fib_batch) else workloads.config(k, seed=seed)
     if cfg["kind"] == "fib":
         cfg["N"] = int(sum(2 * fib_iter(int(n) + 1) - 1 for n in cfg["x"]))
     else:
@@ -198,6 +198,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=workloads.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fib-batch", type=int, default=None,
+                    help="workload 1 only: number of independent fib calls (default 1024, the named configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -208,7 +210,7 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        cfg = load(args.workload, args.seed)
+        cfg = load(args.workload, args.seed, args.fib_batch)
         value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup))
         print(json.dumps({
             "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -232,7 +234,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # every rank processes a batch of its own (instances never exchange tokens): weak scaling
-    cfg = load(args.workload, rank_seed(args.seed, rank))
+    cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch)
     N = cfg["N"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
 
@@ -244,12 +246,15 @@ def main():
         y = torch.empty_like(x_dev)
         kind, compute, dtype = "eval_int", None, "int64"
 
+        # the widest wave of fib(18) holds 2048 calls + their continuations per instance: 4096 tokens bound it
+        wave_cap = min(N + len(cfg["x"]), 4096 * len(cfg["x"]))
+
         def step():
-            g.eval_int(x_dev, N, check=False, y=y)
+            g.eval_int(x_dev, N, check=False, y=y, max_wave_tokens=wave_cap)
 
         def step_e2e():
             xd = x_host.cuda(non_blocking=True)
-            out, _ = g.eval_int(xd, N, check=False)
+            out, _ = g.eval_int(xd, N, check=False, max_wave_tokens=wave_cap)
             return out.cpu()
         h2d, d2h = x_host.numel() * 8, x_host.numel() * 8
         flops_fwd = 0.0
@@ -388,7 +393,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": dtype, "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAMES[args.workload], "invocations_per_step": N, "instances": cfg.get("B") or cfg["trees"].B,
+        "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else ""),
+                   "invocations_per_step": N, "instances": cfg.get("B") or cfg["trees"].B,
                    "pass": "forward+backward" if cfg.get("grad") else "forward",
                    "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
         "clocks": clk,
