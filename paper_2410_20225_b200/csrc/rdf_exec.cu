@@ -295,6 +295,65 @@ __device__ void rnn_leaf_rows(const DevCtx& c, uint32_t n_items) {
 // ===========================================================================
 // the persistent forward kernel
 // ===========================================================================
+// per-thread counters -> one set of atomics per warp
+__device__ __forceinline__ void flush_stats(const DevCtx& c, const ThreadStats& st) {
+    unsigned long long v[7] = {st.invocations, st.tokens, st.cells, st.leaves, st.sc.inserts, st.sc.matches, st.sc.probes};
+    uint32_t mp = st.sc.max_probe, md = st.max_depth;
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int k = 0; k < 7; ++k) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
+        mp = max(mp, __shfl_xor_sync(0xffffffffu, mp, o));
+        md = max(md, __shfl_xor_sync(0xffffffffu, md, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&c.ctl->invocations, v[0]); atomicAdd(&c.ctl->tokens, v[1]); atomicAdd(&c.ctl->cells, v[2]);
+        atomicAdd(&c.ctl->leaves, v[3]); atomicAdd(&c.ctl->store_inserts, v[4]); atomicAdd(&c.ctl->store_matches, v[5]);
+        atomicAdd(&c.ctl->store_probes, v[6]);
+        atomicMax(&c.ctl->max_probe, mp);
+        atomicMax(&c.ctl->max_depth, md);
+    }
+}
+
+// Lean variant of the persistent kernel for programs without vector operators (integer recursion):
+// only the S phase exists, so the block can be four times as wide and hide four times as much of the
+// latency of the dependent L2 round trips (queue, frame table, store) that a token makes.
+__global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ SharedProgram sp;
+    load_program(c, sp);
+    ThreadStats st;
+    uint32_t generation = 0, wave = 0, widest = 0;
+    long long cyc_s = 0, cyc_b = 0, t_mark = clock64();
+    auto lap = [&](long long& acc) {
+        const long long now = clock64();
+        acc += now - t_mark;
+        t_mark = now;
+    };
+    for (;; ++wave) {
+        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
+        if (n == 0) break;
+        if (wave >= c.wave_limit) {
+            set_status(c, RDF_ERR_WAVE_LIMIT);
+            break;
+        }
+        widest = max(widest, n);
+        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
+        const Token* q = c.q[wave & 1];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+            run_token(c, sp, wave, load_token(&q[i]), st);
+        __syncthreads();
+        lap(cyc_s);
+        if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        lap(cyc_b);
+    }
+    flush_stats(c, st);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        c.ctl->waves = wave;
+        c.ctl->max_wave_tokens = widest;
+        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[1] = 0; c.ctl->cyc[2] = cyc_b;
+    }
+}
+
+
 __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= c.B) return;
@@ -389,16 +448,7 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         }
     }
     if (c.use_tc) tc_teardown(tc);
-    // ---- statistics
-    atomicAdd(&c.ctl->invocations, (unsigned long long)st.invocations);
-    atomicAdd(&c.ctl->tokens, (unsigned long long)st.tokens);
-    atomicAdd(&c.ctl->cells, (unsigned long long)st.cells);
-    atomicAdd(&c.ctl->leaves, (unsigned long long)st.leaves);
-    atomicAdd(&c.ctl->store_inserts, (unsigned long long)st.sc.inserts);
-    atomicAdd(&c.ctl->store_matches, (unsigned long long)st.sc.matches);
-    atomicAdd(&c.ctl->store_probes, (unsigned long long)st.sc.probes);
-    atomicMax(&c.ctl->max_probe, st.sc.max_probe);
-    atomicMax(&c.ctl->max_depth, st.max_depth);
+    flush_stats(c, st);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->waves = wave;
         c.ctl->max_wave_tokens = widest;
@@ -639,8 +689,11 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args,
-                                        (size_t)L.tc_smem_fwd, stream));
+    if (g->has_vector_ops)
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args,
+                                            (size_t)L.tc_smem_fwd, stream));
+    else
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_int_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
     if (g->has_vector_ops) {
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());
