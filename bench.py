@@ -109,7 +109,8 @@ def peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
 # (profiles/rdf_forward_kernel_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {("rdf_forward_kernel", 3): 921.46e6}
+NCU_TRAFFIC_BYTES = {("rdf_forward_kernel", 3, None): 924.30e6,             # profiles/rdf_forward_kernel_config3.md
+                     ("rdf_forward_int_kernel", 1, 131072): 37.04e9}      # profiles/rdf_forward_int_kernel_fib_scaled.md
 
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
@@ -360,7 +361,7 @@ def main():
     if cfg["kind"] == "fib":
         alg_bytes = 128.0 * N          # 6 token touches x 16 B + one 32 B store slot per invocation
         achieved = alg_bytes / (dom_ms * 1e-3) / 1e9
-        roof = {"kernel": "rdf_forward_kernel", "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"],
+        roof = {"kernel": "rdf_forward_int_kernel", "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
     else:
         H = cfg["H"]
@@ -383,7 +384,7 @@ def main():
                     "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
                     "cells": C, "flops_phase": flops}
 
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((roof["kernel"], args.workload))
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((roof["kernel"], args.workload, args.fib_batch if args.workload == 1 else None))
     cpu = None
     if not args.no_cpu_baseline:
         v, _, what = time_oracle(cfg, 1, 0, scale=1 if cfg["trees"].N > 2_000_000 else 4) if cfg["kind"] != "fib" else time_oracle(cfg, 1, 0, scale=4)
