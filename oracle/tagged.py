@@ -19,7 +19,7 @@ time, following the paper's semantic equations:
   * nodes wait in a pending table keyed by (node, tag) and tokens are taken
     from a FIFO queue until it is empty (Section 5.1).
 
-Readings where the text is silent (kept in step with the list in the design doc):
+Readings where the text is silent:
   * the entry Merge of a function has one input per call site; tokens from
     different call sites carry different tags, so at most one live token per
     tag ever arrives and it is forwarded as it arrives;
