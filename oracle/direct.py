@@ -61,6 +61,26 @@ def fib(n):
     return n if n < 2 else fib(n - 1) + fib(n - 2)
 
 
+def ack(m, n, count=None):
+    """Textbook Ackermann function; `count` (a one-element list) counts the invocations."""
+    if count is not None:
+        count[0] += 1
+    if m == 0:
+        return n + 1
+    if n == 0:
+        return ack(m - 1, 1, count)
+    return ack(m - 1, ack(m, n - 1, count), count)
+
+
+def tak(x, y, z, count=None):
+    """Textbook Takeuchi function."""
+    if count is not None:
+        count[0] += 1
+    if y < x:
+        return tak(tak(x - 1, y, z, count), tak(y - 1, z, x, count), tak(z - 1, x, y, count), count)
+    return z
+
+
 def fib_invocations(n, tag=(0,), out=None):
     """Every invocation of fib below the call `result = fib(n)` as
     (tag, argument, result); the call in `result` is call site 0, the two

@@ -36,6 +36,7 @@ INT_OPS = {
     "==": lambda a, b: a == b,
     "id": lambda a: a,
     "max": lambda a, b: a if a > b else b,
+    "one": lambda a: 1,
 }
 
 
@@ -60,6 +61,50 @@ def fib_program():
     a = f.call("fib", f.op("-", e, f.const(1)))
     b = f.call("fib", f.op("-", e, f.const(2)))
     f.output(f.merge(f.op("id", t), f.op("+", a, b)))
+    return [r, f]
+
+
+def ack_program(m_const=2):
+    """result(x) = ack(m_const, x);
+    ack(m, n) = if m == 0 then n + 1 else if n == 0 then ack(m - 1, 1) else ack(m - 1, ack(m, n - 1)).
+    Table 1 names the Ackermann function without printing it: this is the textbook two-argument form.
+    Every value a branch uses is routed through that branch's Switch (Figure 2), including the
+    constant 1 of the second call, which is derived from the routed n ("one")."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("ack", r.const(m_const), r.param(0)))
+    f = FunctionGraph("ack", 2)
+    m, n = f.param(0), f.param(1)
+    p1 = f.op("==", m, f.const(0))
+    _, m_e = f.switch(p1, m)
+    n_t, n_e = f.switch(p1, n)
+    base = f.op("+", n_t, f.const(1))
+    p2 = f.op("==", n_e, f.const(0))
+    m_t2, m_e2 = f.switch(p2, m_e)
+    n_t2, n_e2 = f.switch(p2, n_e)
+    second = f.call("ack", f.op("-", m_t2, f.const(1)), f.op("one", n_t2))
+    inner = f.call("ack", m_e2, f.op("-", n_e2, f.const(1)))
+    third = f.call("ack", f.op("-", m_e2, f.const(1)), inner)
+    f.output(f.merge(base, f.merge(second, third)))
+    return [r, f]
+
+
+def tak_program(y_const=12, z_const=6):
+    """result(x) = tak(x, y_const, z_const);
+    tak(x, y, z) = if y < x then tak(tak(x-1, y, z), tak(y-1, z, x), tak(z-1, x, y)) else z.
+    Table 1 names the Takeuchi function without printing it: this is the textbook form."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("tak", r.param(0), r.const(y_const), r.const(z_const)))
+    f = FunctionGraph("tak", 3)
+    x, y, z = f.param(0), f.param(1), f.param(2)
+    p = f.op("<", y, x)
+    x_t, _ = f.switch(p, x)
+    y_t, _ = f.switch(p, y)
+    z_t, z_e = f.switch(p, z)
+    one = f.const(1)
+    a = f.call("tak", f.op("-", x_t, one), y_t, z_t)
+    b = f.call("tak", f.op("-", y_t, one), z_t, x_t)
+    c = f.call("tak", f.op("-", z_t, one), x_t, y_t)
+    f.output(f.merge(f.call("tak", a, b, c), f.op("id", z_e)))
     return [r, f]
 
 

@@ -73,7 +73,8 @@ def transform(functions, result_name: str = "result") -> Graph:
             # step 2: m nodes Call_i, each with the one input of its parameter
             call_nodes = []
             for k in range(m):
-                (arg_edge,) = [e for e in g.in_edges(c) if e.dst_port == k]
+                # (an argument that is itself a call was re-wired to that call's Return_j already)
+                (arg_edge,) = [e for e in g.in_edges(c) if e.dst_port == k and e.src not in removed]
                 cid = g.add("Call", name=f.name, value=i, func=g.nodes[c].func, n_in=1, param=k)
                 g.connect(arg_edge.src, cid, 0, src_port=arg_edge.src_port)
                 # step 3 (edge part)

@@ -277,3 +277,58 @@ def test_chain_and_perfect_shapes():
     # every right child of the chain is a leaf
     chain_int = [v for v in range(81) if tb.left[v] >= 0]
     assert all(tb.left[tb.right[v]] < 0 for v in chain_int)
+
+
+# --------------------------------------------------------------------------
+# multi-parameter and nested recursion (Table 1's ack and tak)
+# --------------------------------------------------------------------------
+def test_ackermann_closed_forms():
+    """ack(1, n) = n + 2, ack(2, n) = 2n + 3, ack(3, n) = 2^(n+3) - 3."""
+    for n in range(0, 7):
+        assert direct.deep(direct.ack, 1, n) == n + 2
+        assert direct.deep(direct.ack, 2, n) == 2 * n + 3
+    for n in range(0, 5):
+        assert direct.deep(direct.ack, 3, n) == 2 ** (n + 3) - 3
+
+
+def test_takeuchi_known_values():
+    """tak(x, y, z) with y >= x is z; tak(18, 12, 6) = 7 after 63 609 calls (the classic benchmark figures)."""
+    assert direct.tak(3, 5, 9) == 9
+    count = [0]
+    assert direct.deep(direct.tak, 18, 12, 6, count) == 7 and count[0] == 63609
+
+
+def test_transform_of_multi_parameter_functions():
+    g = transform.transform(programs.tak_program())
+    # 5 call sites of a 3-parameter function: 15 Call nodes, 5 Returns, 3 entry Merges with 5 inputs each
+    assert g.count("Call") == 15 and g.count("Return") == 5
+    entry = [n for n in g.nodes if n.kind == "merge" and n.name == "entry"]
+    assert len(entry) == 3 and all(n.n_in == 5 for n in entry)
+    ctrl = [e for e in g.edges if e.control and g.nodes[e.src].kind == "Call"]
+    assert len(ctrl) == 15
+
+
+@pytest.mark.parametrize("m,n", [(0, 3), (1, 2), (2, 0), (2, 3), (3, 2)])
+def test_ack_tagged_equals_direct(m, n):
+    g = transform.transform(programs.ack_program(m))
+    count = [0]
+    want = direct.deep(direct.ack, m, n, count)
+    for dead in (True, False):
+        r = tagged.run(g, {0: n}, programs.INT_OPS, dead_tokens=dead)
+        assert r.value == want and len(r.calls) == count[0]
+        # every invocation has both of its parameters, delivered by the two Call_i nodes of its call site
+        assert all(sorted(a) == [0, 1] for a in r.calls.values())
+        for tag, args in r.calls.items():
+            assert r.returns[tag] == direct.deep(direct.ack, args[0], args[1])
+    assert tagged.run(g, {0: n}, programs.INT_OPS, dead_tokens=True).leftover == 0
+
+
+@pytest.mark.parametrize("x", [2, 5, 7, 9])
+def test_tak_tagged_equals_direct(x):
+    g = transform.transform(programs.tak_program(4, 2))
+    count = [0]
+    want = direct.tak(x, 4, 2, count)
+    r = tagged.run(g, {0: x}, programs.INT_OPS, dead_tokens=False)
+    assert r.value == want and len(r.calls) == count[0]
+    for tag, args in r.calls.items():
+        assert r.returns[tag] == direct.tak(args[0], args[1], args[2])
