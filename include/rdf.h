@@ -62,7 +62,8 @@ typedef enum {
     RDF_OP_ADD, RDF_OP_SUB, RDF_OP_MUL, RDF_OP_MAX,   /* a, b                       */
     RDF_OP_LT, RDF_OP_EQ,                             /* a, b -> 0/1                */
     RDF_OP_IF,           /* a = condition, b = then, c = else                       */
-    RDF_OP_CALL,         /* imm = callee function index, a = argument expression    */
+    RDF_OP_CALL,         /* imm = callee function index; a, b, c = one argument expression per formal
+                            parameter of the callee (up to three); an argument may itself be a call */
     /* accessors on the batch's flat tree arrays; operand = node index           */
     RDF_OP_IS_LEAF, RDF_OP_LEFT, RDF_OP_RIGHT, RDF_OP_TOK,
     /* vector-valued operators of the tree networks                               */
@@ -84,7 +85,8 @@ typedef struct {
 
 typedef struct {
     const char*     name;        /* host, NUL-terminated, copied by rdf_graph_build */
-    int32_t         n_params;    /* m >= 0 formal parameters */
+    int32_t         n_params;    /* m formal parameters: 1 for `result`, 1..3 for the others; m > 1 needs
+                                    RDF_TAGS_FRAME (UNSUPPORTED otherwise) */
     int32_t         n_exprs;
     const rdf_expr* exprs;       /* host, [n_exprs]; a DAG (no cycles) */
     int32_t         root;        /* index of the expression that is the function's output */
@@ -101,8 +103,8 @@ typedef struct {
      *                 [63:44] instance | [43:38] depth | [37:0] labels, `label_bits` each, innermost lowest.
      *                 Matching uses an open-addressing hash table keyed by the packed tag.
      * RDF_TAGS_FRAME: an interned frame id; a frame record holds the parent frame and the label
-     *                 (the paper's own representation, Section 5.1).  Needed for deep recursion
-     *                 and for vector-valued programs. */
+     *                 (the paper's own representation, Section 5.1).  Needed for deep recursion,
+     *                 for vector-valued programs and for functions of several parameters. */
     int32_t             tag_mode;
 } rdf_program;
 

@@ -164,7 +164,7 @@ class Function:
     def lt(self, a, b): return self._add(OP_LT, a, b)
     def eq(self, a, b): return self._add(OP_EQ, a, b)
     def if_(self, c, a, b): return self._add(OP_IF, c, a, b)
-    def call(self, f_index, arg): return self._add(OP_CALL, arg, imm=f_index)
+    def call(self, f_index, *args): return self._add(OP_CALL, *(list(args) + [-1] * (3 - len(args))), imm=f_index)
     def is_leaf(self, v): return self._add(OP_IS_LEAF, v)
     def left(self, v): return self._add(OP_LEFT, v)
     def right(self, v): return self._add(OP_RIGHT, v)
@@ -197,6 +197,33 @@ def fib_program():
     f = Function("fib", 1)
     n = f.param()
     f.ret(f.if_(f.lt(n, f.const(2)), n, f.add(f.call(1, f.sub(n, f.const(1))), f.call(1, f.sub(n, f.const(2))))))
+    return [r, f], 0
+
+
+def ack_program(m_const=2):
+    """result(x) = ack(m_const, x); ack(m, n) = n+1 if m == 0, ack(m-1, 1) if n == 0, else ack(m-1, ack(m, n-1))."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.const(m_const), r.param()))
+    f = Function("ack", 2)
+    m, n = f.param(0), f.param(1)
+    zero, one = f.const(0), f.const(1)
+    m1 = f.sub(m, one)
+    inner = f.call(1, m, f.sub(n, one))
+    f.ret(f.if_(f.eq(m, zero), f.add(n, one), f.if_(f.eq(n, zero), f.call(1, m1, one), f.call(1, m1, inner))))
+    return [r, f], 0
+
+
+def tak_program(y_const=12, z_const=6):
+    """result(x) = tak(x, y, z); tak(x, y, z) = tak(tak(x-1, y, z), tak(y-1, z, x), tak(z-1, x, y)) if y < x else z."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.param(), r.const(y_const), r.const(z_const)))
+    f = Function("tak", 3)
+    x, y, z = f.param(0), f.param(1), f.param(2)
+    one = f.const(1)
+    a = f.call(1, f.sub(x, one), y, z)
+    b = f.call(1, f.sub(y, one), z, x)
+    c = f.call(1, f.sub(z, one), x, y)
+    f.ret(f.if_(f.lt(y, x), f.call(1, a, b, c), z))
     return [r, f], 0
 
 

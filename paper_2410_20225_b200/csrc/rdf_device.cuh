@@ -86,6 +86,7 @@ struct DevCtx {
     Frame*    frames;
     uint32_t* children;           // [frame_cap * K]: frame created by call site k of this frame's body
     uint32_t  frame_cap;
+    int64_t*  frame_args;         // [frame_cap * 2]: parameters 1 and 2 of invocations of multi-parameter functions
     // token store, dense form: one cell per (frame, port) and an arrival counter per (frame, match node)
     int64_t*  port_val;
     uint32_t* arrived;

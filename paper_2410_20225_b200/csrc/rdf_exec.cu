@@ -90,9 +90,14 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
                     const uint32_t d = (uint32_t)(nt >> RDF_DEPTH_SHIFT) & 63u;
                     if (d > st.max_depth) st.max_depth = d;
                 }
+                if (sp.labels[in.imm].n_args > 1) {             // the other Call_i nodes of this call site
+                    c.frame_args[(size_t)nt * 2] = r[in.b];
+                    c.frame_args[(size_t)nt * 2 + 1] = r[in.dst];
+                }
                 push_token(c, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
                 break;
             }
+            case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)tag * 2 + in.imm - 1])); break;
             case VM_RET:
             case VM_PORT: {
                 const int64_t val = r[in.a];
@@ -509,6 +514,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.q0 = P.take<Token>(L.qcap);
     L.q1 = P.take<Token>(L.qcap);
     L.frames = P.take<Frame>(L.frame_cap);
+    L.frame_args = P.take<int64_t>(g->max_params > 1 ? (size_t)L.frame_cap * 2 : 0);
     L.children = P.take<uint32_t>((size_t)L.frame_cap * g->max_calls_per_body);
     L.port_val = P.take<int64_t>((size_t)L.frame_cap * g->n_ports_total);
     L.arrived_bytes = (size_t)L.frame_cap * std::max<size_t>(1, g->match.size()) * sizeof(uint32_t);
@@ -594,6 +600,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.qcap = L.qcap;
     c.frames = reinterpret_cast<Frame*>(ws + L.frames);
     c.children = reinterpret_cast<uint32_t*>(ws + L.children);
+    c.frame_args = reinterpret_cast<int64_t*>(ws + L.frame_args);
     c.frame_cap = L.frame_cap;
     c.port_val = reinterpret_cast<int64_t*>(ws + L.port_val);
     c.arrived = reinterpret_cast<uint32_t*>(ws + L.arrived);

@@ -37,6 +37,11 @@ struct Prog {
     const rdf_program* p;
     const rdf_function& fn(int i) const { return p->functions[i]; }
     const rdf_expr& ex(int f, int e) const { return p->functions[f].exprs[e]; }
+    // number of operand expressions: a call has one per formal parameter of its callee
+    int n_ops(const rdf_expr& x) const {
+        if (x.op == RDF_OP_CALL) return (x.imm >= 0 && x.imm < p->n_functions) ? p->functions[x.imm].n_params : 0;
+        return arity_of(x.op);
+    }
 };
 
 // ---------------------------------------------------------------- validation
@@ -45,24 +50,27 @@ void validate(const Prog& P) {
     require(p->n_functions > 0 && p->functions, RDF_ERR_BAD_PROGRAM);
     require(p->result >= 0 && p->result < p->n_functions, RDF_ERR_BAD_PROGRAM);
     require(p->tag_mode == RDF_TAGS_PATH || p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_BAD_ARG);
+    require(p->functions[p->result].n_params <= 1, RDF_ERR_UNSUPPORTED);    // one input per instance
     for (int f = 0; f < p->n_functions; ++f) {
         const rdf_function& F = p->functions[f];
         require(F.exprs && F.n_exprs > 0 && F.n_params >= 0 && F.name, RDF_ERR_BAD_PROGRAM);
         require(F.root >= 0 && F.root < F.n_exprs, RDF_ERR_BAD_PROGRAM);
         for (int e = 0; e < F.n_exprs; ++e) {
             const rdf_expr& x = F.exprs[e];
-            int ar = arity_of(x.op);
-            require(ar >= 0, RDF_ERR_BAD_PROGRAM);
-            int ops[3] = {x.a, x.b, x.c};
-            for (int k = 0; k < ar; ++k) require(ops[k] >= 0 && ops[k] < F.n_exprs, RDF_ERR_BAD_PROGRAM);
-            if (x.op == RDF_OP_PARAM) require(x.imm >= 0 && x.imm < F.n_params, RDF_ERR_BAD_PROGRAM);
+            require(arity_of(x.op) >= 0, RDF_ERR_BAD_PROGRAM);
             if (x.op == RDF_OP_CALL) {
                 require(x.imm >= 0 && x.imm < p->n_functions, RDF_ERR_BAD_PROGRAM);   // unknown callee
                 require(x.imm != p->result, RDF_ERR_BAD_PROGRAM);
                 const int m = p->functions[x.imm].n_params;
                 require(m >= 1, RDF_ERR_BAD_PROGRAM);
-                require(m == 1, RDF_ERR_UNSUPPORTED);     // several parameters: valid, not lowered yet
+                require(m <= 3, RDF_ERR_UNSUPPORTED);     // an expression node carries at most three operands
+                // several parameters live in the invocation's frame: frame-form tags only
+                require(m == 1 || p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);
             }
+            const int ar = P.n_ops(x);
+            int ops[3] = {x.a, x.b, x.c};
+            for (int k = 0; k < ar; ++k) require(ops[k] >= 0 && ops[k] < F.n_exprs, RDF_ERR_BAD_PROGRAM);   // arity mismatch too
+            if (x.op == RDF_OP_PARAM) require(x.imm >= 0 && x.imm < F.n_params, RDF_ERR_BAD_PROGRAM);
         }
         // no cycles among expressions
         std::vector<int> state(F.n_exprs, 0);
@@ -72,7 +80,7 @@ void validate(const Prog& P) {
             state[e] = 1;
             const rdf_expr& x = F.exprs[e];
             int ops[3] = {x.a, x.b, x.c};
-            for (int k = 0; k < arity_of(x.op); ++k) dfs(ops[k]);
+            for (int k = 0; k < P.n_ops(x); ++k) dfs(ops[k]);
             state[e] = 2;
         };
         dfs(F.root);
@@ -108,20 +116,26 @@ struct Literal {
         uint32_t m = 0;
         if (x.op == RDF_OP_PARAM) m = 1u << x.imm;
         int ops[3] = {x.a, x.b, x.c};
-        for (int k = 0; k < arity_of(x.op); ++k) m |= params_used(f, ops[k], memo);
+        for (int k = 0; k < P.n_ops(x); ++k) m |= params_used(f, ops[k], memo);
         memo[e] = m;
         return m;
     }
 
     typedef std::pair<int, int> Val;   // (node, output port)
+    struct Gate {
+        Val pred;
+        int side;          // Switch output that is live in this context
+        bool conditional;  // the predicate reads a parameter, so it is itself live only in its own context
+    };
     struct Ctx {
         int id;
         std::vector<Val> param;
+        std::vector<Gate> gates;   // enclosing conditionals, outermost first
     };
 
     void build_function(int f) {
         const rdf_function& F = P.fn(f);
-        Ctx root{0, {}};
+        Ctx root{0, {}, {}};
         in_node[f] = (int)nodes.size();
         for (int k = 0; k < F.n_params; ++k) root.param.push_back(Val(add(RDF_NODE_IN, -1, f, 0, 0, k), 0));
         std::map<std::pair<int, int>, Val> memo;
@@ -141,7 +155,10 @@ struct Literal {
                 // Figure 2: the predicate drives a Switch that routes the parameter to one side
                 Val pred = build(x.a, c);
                 uint32_t m = params_used(f, x.b, used) | params_used(f, x.c, used);
-                Ctx ct{next_ctx++, c.param}, cf{next_ctx++, c.param};
+                Ctx ct{next_ctx++, c.param, c.gates}, cf{next_ctx++, c.param, c.gates};
+                const bool conditional = params_used(f, x.a, used) != 0;
+                ct.gates.push_back(Gate{pred, 0, conditional});
+                cf.gates.push_back(Gate{pred, 1, conditional});
                 for (int k = 0; k < F.n_params; ++k) {
                     if (!(m >> k & 1)) continue;
                     int sw = add(RDF_NODE_SWITCH, -1, f, 2);
@@ -170,10 +187,26 @@ struct Literal {
                 connect(b.first, b.second, mg, 1);
                 v = Val(mg, 0);
             } else if (x.op == RDF_OP_CALL) {
-                Val a = build(x.a, c);
-                int n = add(NODE_FCALL, -1, f, 1);
+                const int m = P.n_ops(x);
+                const int ops[3] = {x.a, x.b, x.c};
+                Val in[3];
+                for (int k = 0; k < m; ++k) {
+                    in[k] = build(ops[k], c);
+                    // an argument that reads no parameter would feed its Call_i under every tag of
+                    // this function: let the enclosing conditionals' Switches pass it on instead
+                    if (params_used(f, ops[k], used) != 0) continue;
+                    for (int gi = (int)c.gates.size() - 1; gi >= 0; --gi) {
+                        const Gate& gt = c.gates[gi];
+                        int sw = add(RDF_NODE_SWITCH, -1, f, 2);
+                        connect(gt.pred.first, gt.pred.second, sw, 0);
+                        connect(in[k].first, in[k].second, sw, 1);
+                        in[k] = Val(sw, gt.side);
+                        if (gt.conditional) break;
+                    }
+                }
+                int n = add(NODE_FCALL, -1, f, m);
                 callee[n] = x.imm;
-                connect(a.first, a.second, n, 0);
+                for (int k = 0; k < m; ++k) connect(in[k].first, in[k].second, n, k);
                 v = Val(n, 0);
             } else {
                 int ar = arity_of(x.op);
@@ -325,7 +358,7 @@ struct Lower {
             default: break;
         }
         int ops[3] = {x.a, x.b, x.c};
-        for (int k = 0; k < arity_of(x.op); ++k)
+        for (int k = 0; k < P.n_ops(x); ++k)
             if (!call_free(f, ops[k])) return false;
         return true;
     }
@@ -352,13 +385,15 @@ struct Lower {
 
     // value of a call-free expression, computed where the parameters are live
     int value(int s, int e) {
-        require(segs[s].entry, RDF_ERR_UNSUPPORTED);   // parameters are in registers only in an entry segment
         auto it = segs[s].memo.find(e);
         if (it != segs[s].memo.end()) return it->second;
         const rdf_expr& x = P.ex(cur_func, e);
         int r;
         switch (x.op) {
-            case RDF_OP_PARAM: r = (int)x.imm; break;
+            case RDF_OP_PARAM:
+                require(segs[s].entry, RDF_ERR_UNSUPPORTED);   // parameters are in registers only in an entry segment
+                r = (int)x.imm;
+                break;
             case RDF_OP_CONST: r = load_const(s, x.imm); break;
             case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK: {
                 int a = value(s, x.a);
@@ -421,6 +456,7 @@ struct Lower {
         L.callee = callee;
         L.local_label = local_count[callee]++;
         L.child_index = calls_in_body++;
+        L.n_args = P.fn(callee).n_params;
         int kseg = -1;
         if (K.kind == 2) {
             L.k_kind = K_PORT; L.k_node = K.node; L.k_port = K.port;
@@ -456,17 +492,38 @@ struct Lower {
         switch (x.op) {
             case RDF_OP_CALL: {
                 const int callee = (int)x.imm;
-                if (call_free(f, x.a)) {
-                    int r = value(s, x.a);
+                const int m = P.n_ops(x);
+                const int ops[3] = {x.a, x.b, x.c};
+                bool all_free = true;
+                for (int k = 0; k < m; ++k) all_free = all_free && call_free(f, ops[k]);
+                if (all_free) {
+                    // the m Call_i nodes of this call site fire together: all arguments are at hand
+                    int r[3] = {0, 0, 0};
+                    for (int k = 0; k < m; ++k) r[k] = value(s, ops[k]);
                     int label = new_label(callee, K);
-                    emit(s, VM_CALL, 0, r, 0, label);
-                } else {
+                    emit(s, VM_CALL, r[2], r[0], r[1], label);
+                } else if (m == 1) {
                     Cont K2{3};
                     K2.fn = [this, callee, K](int s2, int r) {
                         int label = new_label(callee, K);
                         emit(s2, VM_CALL, 0, r, 0, label);
                     };
                     cps(s, x.a, K2);
+                } else {
+                    // some argument is itself the result of a call: the arguments meet in the token store
+                    // under the caller's tag, and the call fires when the last one has arrived
+                    int ks = new_seg();
+                    int r[3] = {0, 0, 0};
+                    for (int k = 0; k < m; ++k) r[k] = reg(ks);
+                    int M = new_match(m, MATCH_INT, ks);
+                    for (int k = 0; k < m; ++k) {
+                        Cont Kk{2, M, k};
+                        cps(s, ops[k], Kk);
+                    }
+                    // numbered after the call sites inside its arguments, as in the literal graph
+                    int label = new_label(callee, K);
+                    emit(ks, VM_CALL, r[2], r[0], r[1], label);
+                    emit(ks, VM_HALT);
                 }
                 break;
             }
@@ -565,6 +622,8 @@ struct Lower {
         for (int f : order) {
             cur_func = f;
             calls_in_body = 0;
+            g->max_params = std::max(g->max_params, P.fn(f).n_params);
+            for (int k = 1; k < P.fn(f).n_params; ++k) emit(entry_seg[f], VM_LDARG, k, 0, 0, k);   // parameter k from the frame
             Cont K{f == P.p->result ? 1 : 0};
             cps(entry_seg[f], P.fn(f).root, K);
             emit(entry_seg[f], VM_HALT);

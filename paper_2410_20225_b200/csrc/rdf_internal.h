@@ -24,7 +24,8 @@ enum VmOp : uint8_t {
     VM_ISLEAF, VM_LEFT, VM_RIGHT, VM_TOK,           // r[dst] = tree accessor(r[a])
     VM_BRZ,        // Switch: if r[a] == 0 jump to imm (segment-relative before layout, absolute after)
     VM_JMP,        // jump to imm
-    VM_CALL,       // Call_i: push label imm on the tag, send <i:t, r[a]> to the callee's entry segment
+    VM_CALL,       // Call_i: push label imm on the tag, send <i:t, r[a]> (further parameters r[b], r[dst]) to the callee
+    VM_LDARG,      // r[dst] = parameter imm (> 0) of this invocation, kept in its frame
     VM_PORT,       // deliver r[a] to input port b of match node imm under the current tag
     VM_RET,        // the function's output r[a]: Return_i pops the tag and continues in the caller
     VM_OUT,        // r[a] is the program's output for this instance
@@ -58,6 +59,7 @@ struct LabelInfo {
     int32_t child_index; // position of this call site among the call sites of its caller's body
     int32_t callee;      // function index
     int32_t local_label; // i of Call_i in the per-callee numbering of Section 3
+    int32_t n_args;      // formal parameters of the callee (one Call_i node per parameter)
 };
 
 static const int RDF_MAX_REGS = 16;
@@ -81,6 +83,7 @@ struct rdf_graph {
     int32_t result_entry_pc = 0;
     int32_t n_ports_total = 0;
     int32_t max_calls_per_body = 1;
+    int32_t max_params = 1;
     int32_t label_bits = 1;
     int32_t tag_mode = RDF_TAGS_PATH;
     bool has_vector_ops = false;

@@ -192,3 +192,84 @@ def test_integer_tree_folds():
             want = [direct.tree_fold(tb, int(rt), lambda v: 0, lambda a, b: max(a, b) + 1) for rt in tb.tree_root]
             assert np.array_equal(y, np.array(want))
         assert g.stats()["invocations"] == tb.N
+
+
+# ---------------------------------------- several parameters, calls nested in arguments
+def _frame_records(g, x, max_invocations):
+    """(instance, tag, first argument, result) of every invocation, from the frame-mode trace."""
+    y, tr = g.eval_int(x, max_invocations=max_invocations, trace_capacity=2 * max_invocations + 16)
+    calls, rets = tr[tr["kind"] == 0], tr[tr["kind"] == 1]
+    tags = decode_frame_trace(tr, x.numel())
+    arg = dict(zip(calls["tag"].tolist(), calls["value"].tolist()))
+    val = dict(zip(rets["tag"].tolist(), rets["value"].tolist()))
+    return y, {(inst, labs, arg[f], val[f]) for f, (inst, labs) in tags.items()}
+
+
+@pytest.mark.parametrize("m,ns", [(0, range(0, 6)), (1, range(0, 12)), (2, range(0, 40)), (3, range(0, 6))])
+def test_ackermann(m, ns):
+    """ack(m, n) over a batch of n: two parameters, a call as the second argument of another call."""
+    ns = list(ns)
+    counts = []
+    for n in ns:
+        c = [0]
+        direct.ack(m, n, c)
+        counts.append(c[0])
+    fs, r = rdf.ack_program(m)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    x = torch.tensor(ns, dtype=torch.int64, device="cuda")
+    y, _ = g.eval_int(x, max_invocations=sum(counts))
+    assert y.tolist() == [direct.ack(m, n) for n in ns]
+    st = g.stats()
+    assert st["status"] == 0 and st["invocations"] == sum(counts)
+    # closed forms: ack(1, n) = n + 2, ack(2, n) = 2n + 3, ack(3, n) = 2^(n+3) - 3
+    closed = {0: lambda n: n + 1, 1: lambda n: n + 2, 2: lambda n: 2 * n + 3, 3: lambda n: 2 ** (n + 3) - 3}[m]
+    assert y.tolist() == [closed(n) for n in ns]
+    # one frame too few is a status code, not a fault
+    if sum(counts) > len(ns):
+        with pytest.raises(rdf.RdfError) as e:
+            g.eval_int(x, max_invocations=sum(counts) - 1)
+        assert e.value.code == -6
+
+
+def test_ackermann_every_invocation_against_the_literal_interpreter():
+    fs, r = rdf.ack_program(2)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    ns = [0, 1, 3, 4]
+    x = torch.tensor(ns, dtype=torch.int64, device="cuda")
+    y, got = _frame_records(g, x, 256)
+    og = transform.transform(programs.ack_program(2))
+    want = set()
+    for b, n in enumerate(ns):
+        res = tagged.run(og, {0: n}, programs.INT_OPS, dead_tokens=False)
+        assert res.value == y[b].item()
+        want |= {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()}
+    assert got == want
+
+
+@pytest.mark.parametrize("yz", [(12, 6), (6, 2), (0, 0)])
+def test_takeuchi(yz):
+    """tak(x, y, z) over a batch of x: three parameters, every argument of the outer call a call."""
+    yc, zc = yz
+    xs = list(range(0, 19)) if yz == (12, 6) else list(range(0, 12))
+    counts = []
+    for v in xs:
+        c = [0]
+        direct.tak(v, yc, zc, c)
+        counts.append(c[0])
+    fs, r = rdf.tak_program(yc, zc)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    x = torch.tensor(xs, dtype=torch.int64, device="cuda")
+    y, got = _frame_records(g, x, sum(counts))
+    assert y.tolist() == [direct.tak(v, yc, zc) for v in xs]
+    st = g.stats()
+    assert st["status"] == 0 and st["invocations"] == sum(counts)
+    # the three inner calls of one invocation run in the same wave: fewer waves than invocations
+    if yz == (12, 6):
+        print("tak waves", st["waves"], "invocations", st["invocations"])
+        assert st["waves"] * 2 < st["invocations"]
+    og = transform.transform(programs.tak_program(yc, zc))
+    for b in range(0, len(xs), 5):
+        if counts[b] > 3000:
+            continue
+        res = tagged.run(og, {0: xs[b]}, programs.INT_OPS, dead_tokens=False)
+        assert {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()} == {w for w in got if w[0] == b}

@@ -63,14 +63,20 @@ def test_bad_programs_are_rejected():
     with pytest.raises(rdf.RdfError) as e:
         _build(fs, r, rdf.TAGS_PATH)
     assert e.value.code == -11
-    # two-parameter callee: valid by the paper, outside this executor
+    # several formal parameters live in the invocation's frame: packed path tags have no room for them
     a = rdf.Function("result", 1)
-    a.ret(a.call(1, a.param()))
+    a.ret(a.call(1, a.param(), a.const(3)))
     b = rdf.Function("g", 2)
-    b.ret(b.param(0))
+    b.ret(b.param(1))
     with pytest.raises(rdf.RdfError) as e:
-        _build([a, b])
+        _build([a, b], 0, rdf.TAGS_PATH)
     assert e.value.code == -11
+    _build([a, b], 0, rdf.TAGS_FRAME)
+    # a call site must give one argument per formal parameter
+    a2 = rdf.Function("result", 1)
+    a2.ret(a2.call(1, a2.param()))
+    with pytest.raises(rdf.RdfError):
+        _build([a2, b], 0, rdf.TAGS_FRAME)
 
 
 # ---------------------------------------- literal graph through the oracle
@@ -134,6 +140,24 @@ def test_fib_literal_graph_runs_in_the_oracle(n):
     res = tagged.run(_as_oracle_graph(d), {0: n}, programs.INT_OPS)
     og = tagged.run(transform.transform(programs.fib_program()), {0: n}, programs.INT_OPS)
     assert res.value == og.value == direct.fib(n)
+    assert res.calls == og.calls and res.returns == og.returns and res.leftover == 0
+
+
+@pytest.mark.parametrize("name,arg", [("ack", 0), ("ack", 3), ("tak", 3), ("tak", 9)])
+def test_multi_parameter_literal_graphs_run_in_the_oracle(name, arg):
+    """One Call_i node per formal parameter and one Return_i per call site; calls nested in arguments."""
+    if name == "ack":
+        (fs, r), oprog, want = rdf.ack_program(2), programs.ack_program(2), direct.ack(2, arg)
+    else:
+        (fs, r), oprog, want = rdf.tak_program(6, 2), programs.tak_program(6, 2), direct.tak(arg, 6, 2)
+    d = _build(fs, r, rdf.TAGS_FRAME).describe()
+    n_par = 2 if name == "ack" else 3
+    sites = d["n_labels"]
+    kinds = [n["kind"] for n in d["nodes"]]
+    assert kinds.count(bd.NODE_RETURN) == sites and kinds.count(bd.NODE_CALL) == sites * n_par
+    res = tagged.run(_as_oracle_graph(d), {0: arg}, programs.INT_OPS)
+    og = tagged.run(transform.transform(oprog), {0: arg}, programs.INT_OPS)
+    assert res.value == og.value == want
     assert res.calls == og.calls and res.returns == og.returns and res.leftover == 0
 
 
