@@ -81,6 +81,25 @@ def tak(x, y, z, count=None):
     return z
 
 
+def primes(n, count=None):
+    """How many primes are <= n: every i in 2..n is tried against d = 2, 3, ... while d * d <= i.
+    `count` (a one-element list) receives the number of invocations the recursive definition
+    count/isprime makes: one `count` per i in 2..n+1 and one `isprime` per divisor tried."""
+    found = 0
+    calls = 0
+    for i in range(2, n + 1):
+        d = 2
+        calls += 1
+        while d * d <= i and i % d != 0:
+            d += 1
+            calls += 1
+        if d * d > i:
+            found += 1
+    if count is not None:
+        count[0] += calls + max(n, 1)      # count(2..n+1, n): n invocations (one when n < 2)
+    return found
+
+
 def fib_invocations(n, tag=(0,), out=None):
     """Every invocation of fib below the call `result = fib(n)` as
     (tag, argument, result); the call in `result` is call site 0, the two

@@ -37,6 +37,8 @@ INT_OPS = {
     "id": lambda a: a,
     "max": lambda a, b: a if a > b else b,
     "one": lambda a: 1,
+    # remainder of truncating division (sign of the dividend); 0 for a zero divisor
+    "%": lambda a, b: 0 if b == 0 else (abs(a) % abs(b)) * (1 if a >= 0 else -1),
 }
 
 
@@ -86,6 +88,40 @@ def ack_program(m_const=2):
     third = f.call("ack", f.op("-", m_e2, f.const(1)), inner)
     f.output(f.merge(base, f.merge(second, third)))
     return [r, f]
+
+
+def primes_program():
+    """result(x) = count(2, x): how many primes are <= x, by trial division;
+    count(i, n)   = if n < i then 0 else isprime(i, 2) + count(i + 1, n)
+    isprime(i, d) = if i < d * d then 1 else if i % d == 0 then 0 else isprime(i, d + 1).
+    Table 1 names `primes` without printing it: this is a textbook form that needs two functions of
+    two parameters each, linear recursion as deep as x and a call next to another call's result.
+    Constants used on one side of a conditional pass through that conditional's Switch."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("count", r.const(2), r.param(0)))
+    c = FunctionGraph("count", 2)
+    i, n = c.param(0), c.param(1)
+    p = c.op("<", n, i)
+    _, i_e = c.switch(p, i)
+    _, n_e = c.switch(p, n)
+    zero_t, _ = c.switch(p, c.const(0))
+    _, two_e = c.switch(p, c.const(2))
+    here = c.call("isprime", i_e, two_e)
+    rest = c.call("count", c.op("+", i_e, c.const(1)), n_e)
+    c.output(c.merge(c.op("id", zero_t), c.op("+", here, rest)))
+    q = FunctionGraph("isprime", 2)
+    i, d = q.param(0), q.param(1)
+    p1 = q.op("<", i, q.op("*", d, d))
+    _, i_e = q.switch(p1, i)
+    _, d_e = q.switch(p1, d)
+    one_t, _ = q.switch(p1, q.const(1))
+    p2 = q.op("==", q.op("%", i_e, d_e), q.const(0))
+    _, i_e2 = q.switch(p2, i_e)
+    _, d_e2 = q.switch(p2, d_e)
+    zero_t2, _ = q.switch(p2, q.const(0))
+    again = q.call("isprime", i_e2, q.op("+", d_e2, q.const(1)))
+    q.output(q.merge(q.op("id", one_t), q.merge(q.op("id", zero_t2), again)))
+    return [r, c, q]
 
 
 def tak_program(y_const=12, z_const=6):

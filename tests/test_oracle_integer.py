@@ -332,3 +332,58 @@ def test_tak_tagged_equals_direct(x):
     assert r.value == want and len(r.calls) == count[0]
     for tag, args in r.calls.items():
         assert r.returns[tag] == direct.tak(args[0], args[1], args[2])
+
+
+# ---------------------------------------------------------------------------
+# primes: two mutually nested functions of two parameters, linear recursion
+# ---------------------------------------------------------------------------
+def _sieve_count(n):
+    if n < 2:
+        return 0
+    mark = np.ones(n + 1, dtype=bool)
+    mark[:2] = False
+    for p in range(2, int(n ** 0.5) + 1):
+        if mark[p]:
+            mark[p * p::p] = False
+    return int(mark.sum())
+
+
+def test_primes_known_values():
+    """pi(100) = 25, pi(1000) = 168, pi(10000) = 1229; 7919 is the 1000th prime."""
+    assert [direct.primes(n) for n in (0, 1, 2, 3, 4, 100, 1000)] == [0, 0, 1, 2, 2, 25, 168]
+    assert direct.primes(10000) == 1229
+    assert direct.primes(7919) == 1000 and direct.primes(7918) == 999
+    for n in (17, 289, 290, 2000, 7500):
+        assert direct.primes(n) == _sieve_count(n)      # a sieve shares nothing with trial division
+
+
+def test_remainder_operator():
+    rem = programs.INT_OPS["%"]
+    assert [rem(7, 3), rem(-7, 3), rem(7, -3), rem(-7, -3), rem(6, 3), rem(5, 0)] == [1, -1, 1, -1, 0, 0]
+    assert rem(2 ** 62 + 5, 2 ** 31) == 5
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 10, 49, 120])
+def test_primes_tagged_equals_direct(n):
+    g = transform.transform(programs.primes_program())
+    # 2 call sites of `count`, 2 of `isprime`, two parameters each
+    assert g.count("Call") == 8 and g.count("Return") == 4
+    count = [0]
+    want = direct.primes(n, count)
+    assert want == _sieve_count(n)
+    for dead in (True, False):
+        r = tagged.run(g, {0: n}, programs.INT_OPS, dead_tokens=dead)
+        assert r.value == want and len(r.calls) == count[0]
+        assert all(sorted(a) == [0, 1] for a in r.calls.values())
+    r = tagged.run(g, {0: n}, programs.INT_OPS)
+    assert r.leftover == 0
+    # every invocation, as (arguments -> result): a `count(i, n)` returns pi(n) - pi(i - 1), an
+    # `isprime(i, d)` whether i has no divisor in d .. sqrt(i); the two are told apart by the second
+    # argument, which is n for count and at most sqrt(n) + 1 for isprime (n >= 5 makes them disjoint)
+    if n >= 5:
+        for tag, a in r.calls.items():
+            if a[1] == n:
+                assert r.returns[tag] == _sieve_count(n) - _sieve_count(a[0] - 1)
+            else:
+                no_divisor = all(a[0] % d for d in range(a[1], int(a[0] ** 0.5) + 1))
+                assert r.returns[tag] == int(no_divisor)
