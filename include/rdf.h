@@ -74,6 +74,7 @@ typedef enum {
     RDF_OP_NODE_LOSS,    /* a = state, b = node index; passes the state through and
                             marks the invocation as a term of the summed per-node
                             softmax cross-entropy loss that rdf_grad differentiates */
+    RDF_OP_REM,          /* a, b -> remainder of the truncating division a / b (sign of a); 0 when b == 0 */
     RDF_OP__COUNT
 } rdf_opcode;
 
@@ -149,6 +150,10 @@ typedef struct {
     int32_t         label_bits;  /* bits per label in the packed path tag */
     int32_t         n_match;     /* operators with more than one tagged input (token-store users) */
     int32_t         n_code;      /* instructions in the lowered device program */
+    /* host [n_labels], owned by the graph: for device label id g, the function it calls and the i of
+     * its Call_i / Return_i in the per-callee numbering of Section 3 (a tag of the paper lists these i) */
+    const int32_t*  label_callee;
+    const int32_t*  label_local;
 } rdf_graph_desc;
 
 int rdf_graph_describe(const rdf_graph* g, rdf_graph_desc* out);

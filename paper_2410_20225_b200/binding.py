@@ -21,7 +21,7 @@ ERRORS = {
     -9: "RDF_ERR_TIMEOUT", -10: "RDF_ERR_CUDA", -11: "RDF_ERR_UNSUPPORTED",
 }
 (OP_PARAM, OP_CONST, OP_ADD, OP_SUB, OP_MUL, OP_MAX, OP_LT, OP_EQ, OP_IF, OP_CALL, OP_IS_LEAF, OP_LEFT, OP_RIGHT,
- OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS) = range(19)
+ OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS, OP_REM) = range(20)
 TAGS_PATH, TAGS_FRAME = 0, 1
 F32, BF16 = 0, 1
 (NODE_IN, NODE_OUT, NODE_CONST, NODE_OP, NODE_SWITCH, NODE_MERGE, NODE_ENTRY_MERGE, NODE_CALL, NODE_RETURN) = range(9)
@@ -63,7 +63,8 @@ class rdf_edge(C.Structure):
 class rdf_graph_desc(C.Structure):
     _fields_ = [("n_nodes", C.c_int32), ("n_edges", C.c_int32), ("nodes", C.POINTER(rdf_node)),
                 ("edges", C.POINTER(rdf_edge)), ("n_labels", C.c_int32), ("label_bits", C.c_int32),
-                ("n_match", C.c_int32), ("n_code", C.c_int32)]
+                ("n_match", C.c_int32), ("n_code", C.c_int32), ("label_callee", C.POINTER(C.c_int32)),
+                ("label_local", C.POINTER(C.c_int32))]
 
 
 class rdf_batch(C.Structure):
@@ -161,6 +162,7 @@ class Function:
     def sub(self, a, b): return self._add(OP_SUB, a, b)
     def mul(self, a, b): return self._add(OP_MUL, a, b)
     def max(self, a, b): return self._add(OP_MAX, a, b)
+    def rem(self, a, b): return self._add(OP_REM, a, b)
     def lt(self, a, b): return self._add(OP_LT, a, b)
     def eq(self, a, b): return self._add(OP_EQ, a, b)
     def if_(self, c, a, b): return self._add(OP_IF, c, a, b)
@@ -211,6 +213,22 @@ def ack_program(m_const=2):
     inner = f.call(1, m, f.sub(n, one))
     f.ret(f.if_(f.eq(m, zero), f.add(n, one), f.if_(f.eq(n, zero), f.call(1, m1, one), f.call(1, m1, inner))))
     return [r, f], 0
+
+
+def primes_program():
+    """result(x) = count(2, x), the number of primes <= x by trial division;
+    count(i, n) = 0 if n < i else isprime(i, 2) + count(i + 1, n);
+    isprime(i, d) = 1 if i < d * d, 0 if i % d == 0, else isprime(i, d + 1)."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.const(2), r.param()))
+    c = Function("count", 2)
+    i, n = c.param(0), c.param(1)
+    c.ret(c.if_(c.lt(n, i), c.const(0), c.add(c.call(2, i, c.const(2)), c.call(1, c.add(i, c.const(1)), n))))
+    q = Function("isprime", 2)
+    i, d = q.param(0), q.param(1)
+    q.ret(q.if_(q.lt(i, q.mul(d, d)), q.const(1),
+                q.if_(q.eq(q.rem(i, d), q.const(0)), q.const(0), q.call(2, i, q.add(d, q.const(1))))))
+    return [r, c, q], 0
 
 
 def tak_program(y_const=12, z_const=6):
@@ -298,7 +316,9 @@ class Graph:
         nodes = [{k: getattr(d.nodes[i], k) for k, _ in rdf_node._fields_} for i in range(d.n_nodes)]
         edges = [{k: getattr(d.edges[i], k) for k, _ in rdf_edge._fields_} for i in range(d.n_edges)]
         return {"nodes": nodes, "edges": edges, "n_labels": d.n_labels, "label_bits": d.label_bits,
-                "n_match": d.n_match, "n_code": d.n_code}
+                "n_match": d.n_match, "n_code": d.n_code,
+                "label_callee": [d.label_callee[i] for i in range(d.n_labels)],
+                "label_local": [d.label_local[i] for i in range(d.n_labels)]}
 
     # ---- workspace (torch owns the memory)
     def workspace_bytes(self, batch, params, want_grad):

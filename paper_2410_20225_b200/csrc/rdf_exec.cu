@@ -74,6 +74,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
             case VM_SUB: r[in.dst] = r[in.a] - r[in.b]; break;
             case VM_MUL: r[in.dst] = r[in.a] * r[in.b]; break;
             case VM_MAX: r[in.dst] = r[in.a] > r[in.b] ? r[in.a] : r[in.b]; break;
+            case VM_REM: r[in.dst] = r[in.b] == 0 ? 0 : r[in.a] % r[in.b]; break;
             case VM_LT: r[in.dst] = r[in.a] < r[in.b]; break;
             case VM_EQ: r[in.dst] = r[in.a] == r[in.b]; break;
             case VM_ISLEAF: r[in.dst] = __ldg(&c.left[r[in.a]]) < 0; break;

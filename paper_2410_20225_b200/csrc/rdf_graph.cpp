@@ -24,7 +24,7 @@ int arity_of(int op) {
     switch (op) {
         case RDF_OP_PARAM: case RDF_OP_CONST: return 0;
         case RDF_OP_ADD: case RDF_OP_SUB: case RDF_OP_MUL: case RDF_OP_MAX:
-        case RDF_OP_LT: case RDF_OP_EQ: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
+        case RDF_OP_LT: case RDF_OP_EQ: case RDF_OP_REM: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
         case RDF_OP_NODE_LOSS: return 2;
         case RDF_OP_IF: return 3;
         case RDF_OP_CALL: case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK:
@@ -379,6 +379,7 @@ struct Lower {
         switch (op) {
             case RDF_OP_ADD: return VM_ADD; case RDF_OP_SUB: return VM_SUB; case RDF_OP_MUL: return VM_MUL;
             case RDF_OP_MAX: return VM_MAX; case RDF_OP_LT: return VM_LT; case RDF_OP_EQ: return VM_EQ;
+            case RDF_OP_REM: return VM_REM;
         }
         throw Err{RDF_ERR_UNSUPPORTED};
     }
@@ -651,6 +652,10 @@ struct Lower {
         int bits = 1;
         while ((1 << bits) < (int)g->labels.size()) ++bits;
         g->label_bits = bits;
+        for (const LabelInfo& L : g->labels) {
+            g->label_callee.push_back(L.callee);
+            g->label_local.push_back(L.local_label);
+        }
         if (g->has_vector_ops) require(P.p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);
         require(!(g->has_rnn && g->has_lstm), RDF_ERR_UNSUPPORTED);
     }
@@ -697,6 +702,8 @@ extern "C" int rdf_graph_describe(const rdf_graph* g, rdf_graph_desc* out) {
     out->label_bits = g->label_bits;
     out->n_match = (int32_t)g->match.size();
     out->n_code = (int32_t)g->code.size();
+    out->label_callee = g->label_callee.data();
+    out->label_local = g->label_local.data();
     return RDF_OK;
 }
 

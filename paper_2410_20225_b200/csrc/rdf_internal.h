@@ -20,7 +20,7 @@ enum VmOp : uint8_t {
     VM_MOVI = 0,   // r[dst] = imm
     VM_MOVC,       // r[dst] = const_pool[imm]
     VM_MOV,        // r[dst] = r[a]
-    VM_ADD, VM_SUB, VM_MUL, VM_MAX, VM_LT, VM_EQ,   // r[dst] = r[a] op r[b]
+    VM_ADD, VM_SUB, VM_MUL, VM_MAX, VM_LT, VM_EQ, VM_REM,   // r[dst] = r[a] op r[b]
     VM_ISLEAF, VM_LEFT, VM_RIGHT, VM_TOK,           // r[dst] = tree accessor(r[a])
     VM_BRZ,        // Switch: if r[a] == 0 jump to imm (segment-relative before layout, absolute after)
     VM_JMP,        // jump to imm
@@ -80,6 +80,7 @@ struct rdf_graph {
     std::vector<MatchNode> match;
     std::vector<LabelInfo> labels;
     std::vector<int64_t> consts;
+    std::vector<int32_t> label_callee, label_local;   // the same two fields of `labels`, as plain arrays for rdf_graph_describe
     int32_t result_entry_pc = 0;
     int32_t n_ports_total = 0;
     int32_t max_calls_per_body = 1;

@@ -196,10 +196,13 @@ def test_integer_tree_folds():
 
 # ---------------------------------------- several parameters, calls nested in arguments
 def _frame_records(g, x, max_invocations):
-    """(instance, tag, first argument, result) of every invocation, from the frame-mode trace."""
+    """(instance, tag, first argument, result) of every invocation, from the frame-mode trace; the
+    tag lists the per-callee call-site numbers i of Section 3, which the graph description gives
+    for every device label."""
     y, tr = g.eval_int(x, max_invocations=max_invocations, trace_capacity=2 * max_invocations + 16)
     calls, rets = tr[tr["kind"] == 0], tr[tr["kind"] == 1]
-    tags = decode_frame_trace(tr, x.numel())
+    local = g.describe()["label_local"]
+    tags = {f: (inst, tuple(local[l] for l in labs)) for f, (inst, labs) in decode_frame_trace(tr, x.numel()).items()}
     arg = dict(zip(calls["tag"].tolist(), calls["value"].tolist()))
     val = dict(zip(rets["tag"].tolist(), rets["value"].tolist()))
     return y, {(inst, labs, arg[f], val[f]) for f, (inst, labs) in tags.items()}
@@ -273,3 +276,46 @@ def test_takeuchi(yz):
             continue
         res = tagged.run(og, {0: xs[b]}, programs.INT_OPS, dead_tokens=False)
         assert {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()} == {w for w in got if w[0] == b}
+
+
+def test_primes():
+    """count/isprime: two callees of two parameters, the remainder operator, recursion as deep as x."""
+    xs = [0, 1, 2, 3, 4, 10, 100, 289, 1000, 2000, 7500]
+    counts = []
+    for v in xs:
+        c = [0]
+        direct.primes(v, c)
+        counts.append(c[0])
+    fs, r = rdf.primes_program()
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    x = torch.tensor(xs, dtype=torch.int64, device="cuda")
+    y, _ = g.eval_int(x, max_invocations=sum(counts))
+    assert y.tolist() == [direct.primes(v) for v in xs]
+    assert y.tolist()[-5:] == [25, 61, 168, 303, 950]
+    st = g.stats()
+    assert st["status"] == 0 and st["invocations"] == sum(counts)
+    assert st["waves"] >= 7500              # the chain count(2, x) .. count(x + 1, x) descends one call per wave
+    # every invocation of a small batch against the literal interpreter
+    small = [0, 2, 11, 30]
+    x = torch.tensor(small, dtype=torch.int64, device="cuda")
+    _, got = _frame_records(g, x, 512)
+    og = transform.transform(programs.primes_program())
+    want = set()
+    for b, n in enumerate(small):
+        res = tagged.run(og, {0: n}, programs.INT_OPS, dead_tokens=False)
+        want |= {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()}
+    assert got == want
+
+
+def test_remainder_semantics():
+    """result(x) = (x % 7) + ((0 - x) % 7) * 100 + (x % 0) * 10000: truncating division, zero divisor gives 0."""
+    f = rdf.Function("result", 1)
+    x = f.param()
+    seven, zero = f.const(7), f.const(0)
+    f.ret(f.add(f.add(f.rem(x, seven), f.mul(f.rem(f.sub(zero, x), seven), f.const(100))),
+                f.mul(f.rem(x, zero), f.const(10000))))
+    g = rdf.Graph([f], 0, rdf.TAGS_PATH)
+    xs = [0, 1, 6, 7, 8, 20, 2 ** 40 + 3]
+    y, _ = g.eval_int(torch.tensor(xs, dtype=torch.int64, device="cuda"), max_invocations=8)
+    rem = programs.INT_OPS["%"]
+    assert y.tolist() == [rem(v, 7) + rem(-v, 7) * 100 for v in xs]

@@ -80,7 +80,7 @@ def test_bad_programs_are_rejected():
 
 
 # ---------------------------------------- literal graph through the oracle
-OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.OP_LT: "<", bd.OP_EQ: "==",
+OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.OP_REM: "%", bd.OP_LT: "<", bd.OP_EQ: "==",
           bd.OP_IS_LEAF: "is_leaf", bd.OP_LEFT: "left", bd.OP_RIGHT: "right", bd.OP_TOK: "tok",
           bd.OP_EMBED: "leaf_rnn", bd.OP_CELL_RNN: "cell_rnn", bd.OP_LEAF_LSTM: "leaf_lstm",
           bd.OP_CELL_LSTM: "cell_lstm", bd.OP_NODE_LOSS: "pass_state"}
@@ -143,16 +143,23 @@ def test_fib_literal_graph_runs_in_the_oracle(n):
     assert res.calls == og.calls and res.returns == og.returns and res.leftover == 0
 
 
-@pytest.mark.parametrize("name,arg", [("ack", 0), ("ack", 3), ("tak", 3), ("tak", 9)])
+@pytest.mark.parametrize("name,arg", [("ack", 0), ("ack", 3), ("tak", 3), ("tak", 9), ("primes", 1), ("primes", 30)])
 def test_multi_parameter_literal_graphs_run_in_the_oracle(name, arg):
     """One Call_i node per formal parameter and one Return_i per call site; calls nested in arguments."""
     if name == "ack":
         (fs, r), oprog, want = rdf.ack_program(2), programs.ack_program(2), direct.ack(2, arg)
-    else:
+    elif name == "tak":
         (fs, r), oprog, want = rdf.tak_program(6, 2), programs.tak_program(6, 2), direct.tak(arg, 6, 2)
+    else:
+        (fs, r), oprog, want = rdf.primes_program(), programs.primes_program(), direct.primes(arg)
     d = _build(fs, r, rdf.TAGS_FRAME).describe()
-    n_par = 2 if name == "ack" else 3
+    n_par = 3 if name == "tak" else 2
     sites = d["n_labels"]
+    # per callee, the local call-site numbers are 0 .. (sites of that callee) - 1, `result`'s site first
+    by_callee = {}
+    for callee, local in zip(d["label_callee"], d["label_local"]):
+        by_callee.setdefault(callee, []).append(local)
+    assert all(sorted(v) == list(range(len(v))) for v in by_callee.values()) and d["label_local"][0] == 0
     kinds = [n["kind"] for n in d["nodes"]]
     assert kinds.count(bd.NODE_RETURN) == sites and kinds.count(bd.NODE_CALL) == sites * n_par
     res = tagged.run(_as_oracle_graph(d), {0: arg}, programs.INT_OPS)
