@@ -61,6 +61,7 @@ struct Control {
     uint32_t all_leaves;          // backward: leaves seen so far
     uint32_t bq_count[3];         // backward wave queues
     uint32_t bar2;                // barrier counter of the backward kernel
+    uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
     unsigned long long cyc[6];    // block 0: forward schedule / batch / barrier, backward frames / batch / barrier

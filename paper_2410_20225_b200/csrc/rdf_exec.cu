@@ -320,6 +320,8 @@ __device__ __forceinline__ void flush_stats(const DevCtx& c, const ThreadStats& 
     }
 }
 
+static const uint32_t INT_NARROW_STRETCH = 4096;   // waves block 0 runs alone before it meets the grid again
+
 // Lean variant of the persistent kernel for programs without vector operators (integer recursion):
 // only the S phase exists, so the block can be four times as wide and hide four times as much of the
 // latency of the dependent L2 round trips (queue, frame table, store) that a token makes.
@@ -342,6 +344,32 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
             break;
         }
         widest = max(widest, n);
+        if (n <= blockDim.x) {
+            // A stretch of narrow waves (deep, thin recursion): one block has a thread for every token,
+            // so block 0 runs wave after wave with a block barrier between them while the other blocks
+            // wait at the grid barrier below.  It comes back to the grid when a wave is wider than the
+            // block, when the queue is empty, or after INT_NARROW_STRETCH waves (so that the bounded
+            // wait of the other blocks never expires on a long stretch).
+            if (blockIdx.x == 0) {
+                uint32_t m = n, k = 0;
+                do {
+                    if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
+                    if (threadIdx.x < m) run_token(c, sp, wave, load_token(&c.q[wave & 1][threadIdx.x]), st);
+                    __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
+                    ++wave;
+                    ++k;
+                    m = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
+                    widest = max(widest, m);
+                } while (m != 0 && m <= blockDim.x && k < INT_NARROW_STRETCH && wave < c.wave_limit &&
+                         ld_volatile_i32(&c.ctl->status) == 0);
+                if (threadIdx.x == 0) c.ctl->resume_wave = wave;
+            }
+            lap(cyc_s);
+            if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+            lap(cyc_b);
+            wave = ld_volatile_u32(&c.ctl->resume_wave) - 1;      // the loop header adds the one back
+            continue;
+        }
         if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
         const Token* q = c.q[wave & 1];
         for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
