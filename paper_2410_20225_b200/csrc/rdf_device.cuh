@@ -59,13 +59,13 @@ struct Control {
     uint32_t waves, waves_backward, max_wave_tokens, max_probe, max_depth;
     uint32_t all_cells;           // backward: cells seen so far (length of the all-cells list)
     uint32_t all_leaves;          // backward: leaves seen so far
-    uint32_t bq_count[3];         // backward wave queues
     uint32_t bar2;                // barrier counter of the backward kernel
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
     unsigned long long cyc[6];    // block 0: forward schedule / batch / barrier, backward frames / batch / barrier
     float    loss;
+    int32_t  forward_status;      // status word at the end of the forward pass and the loss head
 };
 
 struct DevCtx {
@@ -125,7 +125,10 @@ struct DevCtx {
     float*    dhp;                // [frame_cap, S]: gradient arriving from the caller (dh, and dc for the TreeLSTM);
                                   //                 TreeRNN: overwritten by dz (cell) / dh (leaf)
     float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
-    uint32_t* bq[2];              // backward wave queues (frame ids)
+    uint32_t* wave_frames;        // [wave_cap]: frames allocated up to the end of forward wave w.  Frame ids are
+                                  // handed out in wave order, so the invocations that Call_i created in wave w are
+                                  // the id range [wave_frames[w-1], wave_frames[w]) -- one wave of the gradient pass
+    uint32_t  wave_cap;
     uint32_t* all_cells;          // every cell frame, in backward wave order
     uint4*    cell_ops;           // {cell frame, left operand frame, right operand frame, 1} in all_cells order
     uint4*    leaf_ops;           // {leaf frame, token id, 0, 1} in all_leaves order

@@ -452,6 +452,8 @@ __global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_consta
         lap(cyc_s);
         if (!grid_barrier(c, &c.ctl->bar, generation)) break;
         lap(cyc_b);
+        // every frame of this wave has its id now: the gradient pass walks these ranges
+        if (c.wave_frames && blockIdx.x == 0 && threadIdx.x == 0) c.wave_frames[wave] = ld_volatile_u32(&c.ctl->frame_count);
         // ---- C: the wave's ready batched operators
         const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
         const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
@@ -495,7 +497,9 @@ __global__ void rdf_gather_roots_kernel(const DevCtx c, float* h_root) {
     const int b = blockIdx.x;
     const long long slot = c.y[b];
     if (slot < 0 || slot >= (long long)c.frame_cap) return;
-    for (int k = threadIdx.x; k < c.H; k += blockDim.x) h_root[(size_t)b * c.H + k] = c.arena[(size_t)slot * c.S + k];
+    for (int k = threadIdx.x; k < c.H; k += blockDim.x)
+        h_root[(size_t)b * c.H + k] = c.arena ? c.arena[(size_t)slot * c.S + k]
+                                              : __bfloat162float(c.arena_bf[(size_t)slot * c.Hp + k]);
 }
 
 // ===========================================================================
@@ -557,11 +561,11 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.op_l = P.take<uint32_t>(vf);
     L.op_r = P.take<uint32_t>(vf);
     const size_t S = g->has_lstm ? 2 * (size_t)H : (size_t)H;
-    L.arena = P.take<float>(vf * S);
-    L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
     L.Hp = (H + 63) / 64 * 64;
     L.use_tc = g->has_vector_ops && params->compute == RDF_BF16 && L.Hp <= TC_HP_MAX && params->D == params->H;
     const bool tcl = L.use_tc && g->has_lstm, tcr = L.use_tc && !g->has_lstm;
+    L.arena = P.take<float>(tcr ? 0 : vf * S);          // the bf16 TreeRNN keeps its states in arena_bf only
+    L.gates = P.take<float>(g->has_lstm && want_grad ? vf * 5 * H : 0);
     const size_t wcount = (size_t)L.Hp * 2 * L.Hp * (tcl ? 5 : 1);
     L.arena_bf = P.take<__nv_bfloat16>(L.use_tc ? vf * L.Hp : 0);
     L.wp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
@@ -577,8 +581,9 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
     L.dlog = P.take<float>(gf * 8);
-    L.bq0 = P.take<uint32_t>(gf);
-    L.bq1 = P.take<uint32_t>(gf);
+    // a wave of a tree program holds at least one token of an invocation on its way down or up
+    L.wave_cap = want_grad ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
+    L.wave_frames = P.take<uint32_t>(L.wave_cap);
     L.all_cells = P.take<uint32_t>(gf);
     L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
     L.leaf_ops = P.take<uint4>(tcl ? gf : 0);
@@ -640,7 +645,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.work_cap = L.work_cap;
     c.op_l = reinterpret_cast<uint32_t*>(ws + L.op_l);
     c.op_r = reinterpret_cast<uint32_t*>(ws + L.op_r);
-    c.arena = reinterpret_cast<float*>(ws + L.arena);
+    c.arena = L.use_tc && !g->has_lstm ? nullptr : reinterpret_cast<float*>(ws + L.arena);
     if (g->has_vector_ops) {
         c.H = params->H; c.D = params->D; c.V = params->V; c.n_classes = params->n_classes; c.compute = params->compute;
         c.E = params->E; c.W = params->W; c.b = params->b; c.W_x = params->W_x; c.b_x = params->b_x;
@@ -666,7 +671,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.trace = out->trace; c.trace_cap = out->trace ? out->trace_capacity : 0;
     c.dhp = reinterpret_cast<float*>(ws + L.dhp);
     c.dlog = reinterpret_cast<float*>(ws + L.dlog);
-    c.bq[0] = reinterpret_cast<uint32_t*>(ws + L.bq0); c.bq[1] = reinterpret_cast<uint32_t*>(ws + L.bq1);
+    c.wave_frames = L.wave_cap ? reinterpret_cast<uint32_t*>(ws + L.wave_frames) : nullptr;
+    c.wave_cap = L.wave_cap;
     c.all_cells = reinterpret_cast<uint32_t*>(ws + L.all_cells);
     c.cell_ops = L.use_tc ? reinterpret_cast<uint4*>(ws + L.cell_ops) : nullptr;
     c.leaf_ops = L.use_tc && g->has_lstm ? reinterpret_cast<uint4*>(ws + L.leaf_ops) : nullptr;
@@ -674,7 +680,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.loss_partial = reinterpret_cast<float*>(ws + L.loss_partial);
     c.loss_out = out->loss;
     c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
-    c.wave_limit = 1u << 24;
+    c.wave_limit = L.wave_cap ? L.wave_cap : 1u << 24;
     c.spin_limit = (long long)S->clock_khz * 2000ll;       // about two seconds of SM clock
 }
 

@@ -17,9 +17,21 @@
 static const int MAX_CLASSES = 8;
 
 // ---------------------------------------------------------------- loss head
+// Eight hidden units of a state row as floats: from the fp32 arena (row stride S) or, for the bf16
+// TreeRNN, from the bf16 arena (row stride Hp, pad columns zero).
+__device__ __forceinline__ void unpack_bf8(const uint4& v, float (&x)[8]) {
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(p[i]);
+        x[2 * i] = f.x; x[2 * i + 1] = f.y;
+    }
+}
+
 // per invocation f: z = W_s h + b_s; loss += logsumexp(z) - z[label]; dlog = softmax(z) - onehot
+template <bool BF>
 __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
-    // four invocations per warp (8 lanes each) so that four rows are in flight at a time
+    // four invocations per warp (8 lanes each); a lane loads all its pieces of the row before it uses them
     __shared__ float warp_loss[8];
     const uint32_t F = c.ctl->frame_count;
     const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, sub = lane / 8, sl = lane % 8;
@@ -29,18 +41,46 @@ __global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
     for (uint32_t base = (uint32_t)c.B + warp * 4; base < F; base += n_warps * 4) {
         const uint32_t f = base + sub;
         const bool act = f < F;
-        const float* h = c.arena + (size_t)(act ? f : base) * c.S;
         float z[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
-        for (int j = sl * 4; j < H; j += 32) {
-            const float4 h4 = *reinterpret_cast<const float4*>(h + j);
+        if (BF) {
+            const __nv_bfloat16* h = c.arena_bf + (size_t)(act ? f : base) * c.Hp;
+            uint4 hv[TC_HP_MAX / 64];
 #pragma unroll
-            for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) {
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                    z[k] += w.x * h4.x + w.y * h4.y + w.z * h4.z + w.w * h4.w;
-                }
+            for (int q = 0; q < TC_HP_MAX / 64; ++q) {
+                const int j = sl * 8 + 64 * q;
+                hv[q] = j < c.Hp ? *reinterpret_cast<const uint4*>(h + j) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int q = 0; q < TC_HP_MAX / 64; ++q) {
+                const int j = sl * 8 + 64 * q;
+                if (j >= H) continue;
+                float x[8];
+                unpack_bf8(hv[q], x);
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        const float4 w0 = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                        z[k] += w0.x * x[0] + w0.y * x[1] + w0.z * x[2] + w0.w * x[3];
+                        if (j + 4 < H) {
+                            const float4 w1 = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j + 4]));
+                            z[k] += w1.x * x[4] + w1.y * x[5] + w1.z * x[6] + w1.w * x[7];
+                        }
+                    }
+            }
+        } else {
+            const float* h = c.arena + (size_t)(act ? f : base) * c.S;
+#pragma unroll 4
+            for (int j = sl * 4; j < H; j += 32) {
+                const float4 h4 = *reinterpret_cast<const float4*>(h + j);
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                        z[k] += w.x * h4.x + w.y * h4.y + w.z * h4.z + w.w * h4.w;
+                    }
+            }
         }
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k)
@@ -89,120 +129,162 @@ __global__ void rdf_loss_final_kernel(const DevCtx c, int n_partials) {
         for (int i = 0; i < n_partials; ++i) t += (double)c.loss_partial[i];
         c.ctl->loss = (float)t;
         if (c.loss_out) *c.loss_out = (float)t;
+        c.ctl->forward_status = c.ctl->status;      // what the gradient kernel checks before it starts
     }
 }
 
 // ----------------------------------------------------------- backward waves
-__global__ void __launch_bounds__(256) rdf_backward_seed_kernel(const DevCtx c) {
-    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= c.B) return;
-    // dy enters the gradient of the call made by `result` under that call's own tag
-    c.bq[0][b] = c.children[(size_t)b * c.K + 0];
-    if (b == 0) c.ctl->bq_count[0] = (uint32_t)c.B;
+// The cells (and, for the TreeLSTM, the leaves) among the up to 256 frames [base, end) of this block
+// are appended to the global lists with one atomic per list.  The cells of a wave, in list order, are
+// the rows of the wave's operand-gradient contraction.  Called by every thread of the block.
+struct FrameLists {
+    uint32_t wcnt[2][8], gbase[2];
+};
+
+__device__ __forceinline__ void backward_list_frames(const DevCtx& c, FrameLists& fl, uint32_t base, uint32_t end) {
+    const uint32_t t = base + threadIdx.x;
+    const bool valid = t < end;
+    uint32_t l = LEAF_MARK, r = 0;
+    if (valid) {
+        l = __ldcg(&c.op_l[t]);
+        r = __ldcg(&c.op_r[t]);
+    }
+    const bool cell = valid && l != LEAF_MARK, leaf = valid && l == LEAF_MARK && c.lstm;
+    const uint32_t mc = __ballot_sync(0xffffffffu, cell), ml = __ballot_sync(0xffffffffu, leaf);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) {
+        fl.wcnt[0][warp] = __popc(mc);
+        fl.wcnt[1][warp] = __popc(ml);
+    }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        uint32_t tot = 0;
+        for (int w = 0; w < 8; ++w) tot += fl.wcnt[threadIdx.x][w];
+        fl.gbase[threadIdx.x] = tot ? atomicAdd(threadIdx.x ? &c.ctl->all_leaves : &c.ctl->all_cells, tot) : 0u;
+    }
+    __syncthreads();
+    uint32_t pre_c = fl.gbase[0], pre_l = fl.gbase[1];
+    for (int w = 0; w < warp; ++w) {
+        pre_c += fl.wcnt[0][w];
+        pre_l += fl.wcnt[1][w];
+    }
+    const uint32_t below = (1u << lane) - 1u;
+    if (cell) {
+        const uint32_t idx = pre_c + __popc(mc & below);
+        c.all_cells[idx] = t;
+        if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
+    }
+    if (leaf) {
+        const uint32_t idx = pre_l + __popc(ml & below);
+        c.all_leaves[idx] = t;
+        if (c.leaf_ops) c.leaf_ops[idx] = make_uint4(t, r, 0u, 1u);       // r = token id of a leaf
+    }
+    __syncthreads();                                   // fl is reused by the next round
 }
 
-// Appends this block's cells / leaves of one lock-step iteration to the global lists with one
-// global atomic per list per block (thousands of same-address atomics per wave would serialise in
-// L2).  Called by every thread of the block; `mine` marks the one thread that speaks for a frame.
-__device__ __forceinline__ void backward_enqueue_block(const DevCtx& c, uint32_t wave, bool mine, uint32_t t, bool leaf,
-                                                       uint32_t l, uint32_t r) {
-    __shared__ uint32_t cnt[2], base[3];
-    if (threadIdx.x == 0) cnt[0] = cnt[1] = 0;
-    __syncthreads();
-    uint32_t local = 0;
-    if (mine) local = atomicAdd(&cnt[leaf ? 1 : 0], 1u);
-    __syncthreads();
-    // three threads, three independent round trips at once
-    if (threadIdx.x == 0) base[0] = cnt[0] ? atomicAdd(&c.ctl->all_cells, cnt[0]) : 0u;
-    if (threadIdx.x == 32) base[1] = cnt[1] ? atomicAdd(&c.ctl->all_leaves, cnt[1]) : 0u;
-    if (threadIdx.x == 64) base[2] = cnt[0] ? atomicAdd(&c.ctl->bq_count[(wave + 1) % 3], 2u * cnt[0]) : 0u;
-    __syncthreads();
-    if (mine) {
+// A (bf16 TreeRNN), one invocation t per 8 lanes: dh = (gradient from the caller) + W_s^T dlog;
+//    cell: dz = dh * (1 - h^2) as the bf16 operand row of the contractions; leaf: dE[tok] += dh.
+// A lane owns 8 consecutive hidden units per 64 and loads all its pieces of the rows before it uses them.
+__device__ __forceinline__ void backward_frame_tc(const DevCtx& c, uint32_t t, int sl) {
+    const int H = c.H, Hp = c.Hp, C = c.n_classes;
+    const uint32_t parent = __ldcg(&c.frames[t].parent);
+    const uint32_t l = __ldcg(&c.op_l[t]);
+    const bool from_result = parent < (uint32_t)c.B, leaf = l == LEAF_MARK;
+    const uint32_t tok = leaf ? __ldcg(&c.op_r[t]) : 0u;
+    const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8);
+    const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8 + 4);
+    const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+    const float* g = c.dhp + (size_t)t * H;
+    constexpr int NQ = TC_HP_MAX / 64;
+    float4 gv[NQ][2];
+    uint4 hv[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int j = sl * 8 + 64 * q;
+        gv[q][0] = gv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        hv[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (!from_result && j < H) gv[q][0] = ldcg4(g + j);
+        if (!from_result && j + 4 < H) gv[q][1] = ldcg4(g + j + 4);
+        if (!leaf && j < Hp) hv[q] = *reinterpret_cast<const uint4*>(c.arena_bf + (size_t)t * Hp + j);
+    }
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int j = sl * 8 + 64 * q;
+        if (j >= Hp) continue;
+        float dh[8] = {gv[q][0].x, gv[q][0].y, gv[q][0].z, gv[q][0].w, gv[q][1].x, gv[q][1].y, gv[q][1].z, gv[q][1].w};
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) {
+                if (j < H) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                    dh[0] = fmaf(w.x, dl[k], dh[0]); dh[1] = fmaf(w.y, dl[k], dh[1]);
+                    dh[2] = fmaf(w.z, dl[k], dh[2]); dh[3] = fmaf(w.w, dl[k], dh[3]);
+                }
+                if (j + 4 < H) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j + 4]));
+                    dh[4] = fmaf(w.x, dl[k], dh[4]); dh[5] = fmaf(w.y, dl[k], dh[5]);
+                    dh[6] = fmaf(w.z, dl[k], dh[6]); dh[7] = fmaf(w.w, dl[k], dh[7]);
+                }
+            }
         if (leaf) {
-            c.all_leaves[base[1] + local] = t;
-            if (c.leaf_ops) c.leaf_ops[base[1] + local] = make_uint4(t, r, 0u, 1u);      // r = token id of a leaf
+            float* de = c.dE + (size_t)tok * c.D + j;
+            if (j < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(dh[0], dh[1], dh[2], dh[3]));
+            if (j + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(dh[4], dh[5], dh[6], dh[7]));
         } else {
-            const uint32_t idx = base[0] + local;
-            c.all_cells[idx] = t;
-            if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
-            uint32_t* qn = c.bq[(wave + 1) & 1];
-            qn[base[2] + 2 * local] = l;
-            qn[base[2] + 2 * local + 1] = r;
+            float x[8];
+            unpack_bf8(hv[q], x);
+            __align__(16) __nv_bfloat162 pk[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)                 // pad columns: dh = 0 and h = 0, so dz = 0
+                pk[i] = __floats2bfloat162_rn(dh[2 * i] * (1.f - x[2 * i] * x[2 * i]),
+                                              dh[2 * i + 1] * (1.f - x[2 * i + 1] * x[2 * i + 1]));
+            *reinterpret_cast<uint4*>(c.dz_bf + (size_t)t * Hp + j) = *reinterpret_cast<const uint4*>(pk);
         }
     }
 }
 
-// A (TreeRNN): per invocation t of the wave, dh = (gradient from the caller) + W_s^T dlog;
-//    cell: dz = dh * (1 - h^2), queue the two callee frames; leaf: keep dh for dE.
-__device__ void backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
-    // four invocations per warp (8 lanes each): four independent chains of loads in flight
-    const int lane = threadIdx.x % 32, sub = lane / 8, sl = lane % 8;
-    const int wib = threadIdx.x / 32;
+// A (fp32 TreeRNN), one invocation t per 8 lanes; dz (cell) / dh (leaf) replaces the incoming gradient.
+__device__ __forceinline__ void backward_frame_f32(const DevCtx& c, uint32_t t, int sl) {
     const int H = c.H, C = c.n_classes;
-    const uint32_t* q = c.bq[wave & 1];
-    for (uint32_t base = blockIdx.x * 32; base < n; base += gridDim.x * 32) {      // 32 frames per block per step
-        const uint32_t i = base + wib * 4 + sub;
-        const bool act = i < n;
-        uint32_t t = 0, l = 0, r = 0;
-        bool leaf = false;
-        if (act) {
-        t = __ldcg(&q[i]);
-        const uint32_t parent = __ldcg(&c.frames[t].parent);
-        const bool from_result = parent < (uint32_t)c.B;
-        l = __ldcg(&c.op_l[t]); r = __ldcg(&c.op_r[t]);
-        leaf = l == LEAF_MARK;
-        const float4 d0 = ldcg4(c.dlog + (size_t)t * 8), d1 = ldcg4(c.dlog + (size_t)t * 8 + 4);
-        const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-        float* g = c.dhp + (size_t)t * H;
-        const float* h = c.arena + (size_t)t * H;
-#pragma unroll 2
-        for (int j = sl * 4; j < H; j += 32) {
-            float4 dh = from_result ? make_float4(0.f, 0.f, 0.f, 0.f) : ldcg4(g + j);
+    const uint32_t parent = __ldcg(&c.frames[t].parent);
+    const uint32_t l = __ldcg(&c.op_l[t]);
+    const bool from_result = parent < (uint32_t)c.B, leaf = l == LEAF_MARK;
+    const uint32_t tok = leaf ? __ldcg(&c.op_r[t]) : 0u;
+    const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8);
+    const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8 + 4);
+    const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+    float* g = c.dhp + (size_t)t * H;
+    const float* h = c.arena + (size_t)t * H;
+#pragma unroll 4
+    for (int j = sl * 4; j < H; j += 32) {
+        float4 dh = from_result ? make_float4(0.f, 0.f, 0.f, 0.f) : ldcg4(g + j);
 #pragma unroll
-            for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) {
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                    dh.x = fmaf(w.x, dl[k], dh.x); dh.y = fmaf(w.y, dl[k], dh.y);
-                    dh.z = fmaf(w.z, dl[k], dh.z); dh.w = fmaf(w.w, dl[k], dh.w);
-                }
-            if (!leaf) {
-                const float4 hv = ldcg4(h + j);
-                dh.x *= 1.f - hv.x * hv.x; dh.y *= 1.f - hv.y * hv.y;
-                dh.z *= 1.f - hv.z * hv.z; dh.w *= 1.f - hv.w * hv.w;
-                if (c.use_tc) {
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(dh.x, dh.y), hi = __floats2bfloat162_rn(dh.z, dh.w);
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-                    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                    *reinterpret_cast<uint2*>(c.dz_bf + (size_t)t * c.Hp + j) = pk;
-                }
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) {
+                const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                dh.x = fmaf(w.x, dl[k], dh.x); dh.y = fmaf(w.y, dl[k], dh.y);
+                dh.z = fmaf(w.z, dl[k], dh.z); dh.w = fmaf(w.w, dl[k], dh.w);
             }
+        if (leaf) {
+            atomicAdd(reinterpret_cast<float4*>(c.dE + (size_t)tok * c.D + j), dh);
+        } else {
+            const float4 hv = *reinterpret_cast<const float4*>(h + j);
+            dh.x *= 1.f - hv.x * hv.x; dh.y *= 1.f - hv.y * hv.y;
+            dh.z *= 1.f - hv.z * hv.z; dh.w *= 1.f - hv.w * hv.w;
             *reinterpret_cast<float4*>(g + j) = dh;
         }
-        if (c.use_tc && !leaf)
-            for (int j = H + sl; j < c.Hp; j += 8) c.dz_bf[(size_t)t * c.Hp + j] = __float2bfloat16_rn(0.f);
-        }
-        backward_enqueue_block(c, wave, act && sl == 0, t, leaf, l, r);
     }
 }
 
 // A (TreeLSTM): the gate gradients replace the retained gates; dc goes straight to the callee frames.
-__device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n) {
-    const int lane = threadIdx.x % 32;
-    const int wib = threadIdx.x / 32;
+// One invocation t per warp.
+__device__ __forceinline__ void lstm_backward_frame(const DevCtx& c, uint32_t t, int lane) {
     const int H = c.H, C = c.n_classes, S = c.S;
-    const uint32_t* q = c.bq[wave & 1];
-    for (uint32_t base = blockIdx.x * 8; base < n; base += gridDim.x * 8) {        // 8 frames per block per step
-        const uint32_t i = base + wib;
-        const bool act = i < n;
-        uint32_t t = 0, l = 0, r = 0;
-        bool leaf = false;
-        if (act) {
-        t = __ldcg(&q[i]);
+    {
         const uint32_t parent = __ldcg(&c.frames[t].parent);
         const bool from_result = parent < (uint32_t)c.B;
-        l = __ldcg(&c.op_l[t]); r = __ldcg(&c.op_r[t]);
-        leaf = l == LEAF_MARK;
+        const uint32_t l = __ldcg(&c.op_l[t]), r = __ldcg(&c.op_r[t]);
+        const bool leaf = l == LEAF_MARK;
         float dl[MAX_CLASSES];
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) dl[k] = __ldcg(&c.dlog[(size_t)t * 8 + k]);
@@ -274,8 +356,6 @@ __device__ void lstm_backward_frames(const DevCtx& c, uint32_t wave, uint32_t n)
         if (c.dg_bf)                      // pad columns of every gate block are zero
             for (int q = lane; q < (leaf ? 3 : 5) * (c.Hp - H); q += 32)
                 c.dg_bf[(size_t)t * 5 * c.Hp + (q / (c.Hp - H)) * c.Hp + H + q % (c.Hp - H)] = __float2bfloat16_rn(0.f);
-        }
-        backward_enqueue_block(c, wave, act && lane == 0, t, leaf, l, r);
     }
 }
 
@@ -382,12 +462,15 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
     __shared__ uint4 tc_items[TC_M];
+    __shared__ FrameLists lists;
+    if (c.ctl->forward_status != 0) return;                          // the forward pass failed: nothing to differentiate
     TcState tc;
     const bool tc_on = c.use_tc;
     if (tc_on) {
         if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 2 * c.Hp / 32, 4, c.WTp, 5 * c.Hp, 32);
         else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 8, 4, c.WTp, c.Hp, c.Hp / 4);
     }
+    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
     uint32_t generation = 0, wave = 0, first = 0;
     long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
@@ -395,20 +478,37 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         acc += now - t_mark;
         t_mark = now;
     };
-    for (;; ++wave) {
-        const uint32_t n = ld_volatile_u32(&c.ctl->bq_count[wave % 3]);
-        if (n == 0) break;
-        if (wave >= c.wave_limit) {
-            set_status(c, RDF_ERR_WAVE_LIMIT);
-            break;
+    // Gradient wave d re-enters the invocations that Call_i created in forward wave d: frame ids are
+    // handed out in wave order, so they are the range [f0, f1) and their rows are consecutive in memory.
+    const uint32_t n_fwd = min(c.ctl->waves, c.wave_cap);
+    uint32_t f1 = (uint32_t)c.B;
+    for (uint32_t d = 0; d < n_fwd; ++d) {
+        const uint32_t f0 = f1;
+        f1 = max(f0, min(c.wave_frames[d], c.frame_cap));
+        if (f1 == f0) continue;                                      // a wave without calls
+        ++wave;
+        // ---- A: per-invocation work, a contiguous piece of the range per block, 256 frames per round
+        const uint32_t n = f1 - f0;
+        const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
+        const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
+        const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
+        for (uint32_t base = c0; base < c1; base += 256) {
+            const uint32_t end = min(c1, base + 256);
+            if (c.lstm) {
+                for (uint32_t t = base + wib; t < end; t += 8) lstm_backward_frame(c, t, lane);
+            } else {
+                for (uint32_t t = base + wib * 4 + lane / 8; t < end; t += 32) {
+                    if (tc_on) backward_frame_tc(c, t, lane % 8);
+                    else backward_frame_f32(c, t, lane % 8);
+                }
+            }
+            backward_list_frames(c, lists, base, end);
         }
-        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->bq_count[(wave + 2) % 3] = 0;
-        if (c.lstm) lstm_backward_frames(c, wave, n);
-        else backward_frames(c, wave, n);
         __syncthreads();
         lap(cyc_a);
         if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
         lap(cyc_b);
+        // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
             if (tc_on && c.lstm) tc_tiles<TC_LSTM_BWD>(c, tc, tc_items, first, end - first);
@@ -510,45 +610,40 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, c
     }
 }
 
-// dW_s[k][j] = sum over invocations of dlog_f[k] * h_f[j];  db_s[k] = sum of dlog_f[k]
-__global__ void __launch_bounds__(256) rdf_dws_kernel(const DevCtx c) {
+// Column sums over all invocations, one thread per hidden unit j:
+//   dW_s[k][j] = sum_f dlog_f[k] * h_f[j];   db_s[k] = sum_f dlog_f[k];
+//   WITH_DB (TreeRNN): db[j] = sum over the cells of dz_f[j]
+// BF: states and dz are the bf16 rows (stride Hp) of the bf16 TreeRNN, else fp32 rows (stride S; dz in dhp).
+template <bool BF, bool WITH_DB>
+__global__ void __launch_bounds__(128) rdf_heads_kernel(const DevCtx c) {
     const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
     const uint32_t n = F - B, per = (n + gridDim.x - 1) / gridDim.x;
     const uint32_t f0 = B + blockIdx.x * per, f1 = min(F, f0 + per);
     if (f0 >= f1) return;
     const int H = c.H, C = c.n_classes;
     for (int j = threadIdx.x; j < H; j += blockDim.x) {
-        float s[MAX_CLASSES];
+        float s[MAX_CLASSES], db = 0.f;
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k) s[k] = 0.f;
-#pragma unroll 4
+#pragma unroll 8
         for (uint32_t f = f0; f < f1; ++f) {
-            const float hj = c.arena[(size_t)f * c.S + j];
+            const float hj = BF ? __bfloat162float(c.arena_bf[(size_t)f * c.Hp + j]) : c.arena[(size_t)f * c.S + j];
             const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8);
             const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8 + 4);
             s[0] = fmaf(d0.x, hj, s[0]); s[1] = fmaf(d0.y, hj, s[1]); s[2] = fmaf(d0.z, hj, s[2]); s[3] = fmaf(d0.w, hj, s[3]);
             s[4] = fmaf(d1.x, hj, s[4]); s[5] = fmaf(d1.y, hj, s[5]); s[6] = fmaf(d1.z, hj, s[6]); s[7] = fmaf(d1.w, hj, s[7]);
+            if (WITH_DB && c.op_l[f] != LEAF_MARK)
+                db += BF ? __bfloat162float(c.dz_bf[(size_t)f * c.Hp + j]) : c.dhp[(size_t)f * c.S + j];
         }
 #pragma unroll
         for (int k = 0; k < MAX_CLASSES; ++k)
             if (k < C) atomicAdd(&c.dW_s[k * H + j], s[k]);
+        if (WITH_DB) atomicAdd(&c.db[j], db);
     }
     if (threadIdx.x < C) {
         float s = 0.f;
         for (uint32_t f = f0; f < f1; ++f) s += c.dlog[(size_t)f * 8 + threadIdx.x];
         atomicAdd(&c.db_s[threadIdx.x], s);
-    }
-}
-
-// TreeRNN: dE[tok] += dh of every leaf invocation that read row tok
-__global__ void __launch_bounds__(256) rdf_de_kernel(const DevCtx c) {
-    const uint32_t n = c.ctl->all_leaves;
-    const int lane = threadIdx.x % 32;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
-    for (uint32_t i = warp; i < n; i += n_warps) {
-        const uint32_t t = c.all_leaves[i];
-        const uint32_t tok = c.op_r[t];
-        for (int j = lane; j < c.H; j += 32) atomicAdd(&c.dE[(size_t)tok * c.D + j], c.dhp[(size_t)t * c.H + j]);
     }
 }
 
@@ -655,14 +750,14 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     if (rc != RDF_OK) return rc;
     // loss head over every retained invocation
     const int loss_blocks = std::min(4096, std::max(1, (int)((in->max_invocations + 63) / 64)));
-    rdf_loss_kernel<<<loss_blocks, 256, 0, stream>>>(c);
+    const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
+    if (tc_rnn) rdf_loss_kernel<true><<<loss_blocks, 256, 0, stream>>>(c);
+    else rdf_loss_kernel<false><<<loss_blocks, 256, 0, stream>>>(c);
     rdf_loss_final_kernel<<<1, 32, 0, stream>>>(c, loss_blocks);
     rdf_mark(S, 3, stream);
     // gradient waves
-    rdf_backward_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
-    const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
     if (c.use_tc) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args,
                                         c.use_tc ? (size_t)L.tc_smem_bwd : 0, stream));
@@ -704,17 +799,22 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 5, stream);
-    rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
-    if (lstm) rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
+    if (lstm) {
+        rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
+        rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
+    }
     rdf_mark(S, 6, stream);
-    rdf_dws_kernel<<<16 * S->grid, 128, 0, stream>>>(c);
+    // dW_s, db_s (and the TreeRNN's db) in one pass over the retained states
+    if (lstm) rdf_heads_kernel<false, false><<<16 * S->grid, 128, 0, stream>>>(c);
+    else if (tc_rnn) rdf_heads_kernel<true, true><<<16 * S->grid, 128, 0, stream>>>(c);
+    else rdf_heads_kernel<false, true><<<16 * S->grid, 128, 0, stream>>>(c);
     rdf_mark(S, 7, stream);
     if (tc_lstm) {
         const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 4);
         CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));
         rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, 256, de_smem, stream>>>(c);
     } else if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
-    else rdf_de_kernel<<<4 * S->grid, 256, 0, stream>>>(c);
+    // (TreeRNN: the leaves added their dh to dE during the gradient waves)
     rdf_mark(S, 8, stream);
     CUDA_OK(cudaGetLastError());
     return RDF_OK;

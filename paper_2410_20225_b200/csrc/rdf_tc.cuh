@@ -357,21 +357,17 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
                     if (!live) continue;
                     const int col = slice * ns + gi * 16;                       // column of the padded N range
                     if (MODE == TC_RNN_FWD) {
+                        // the state lives in bf16 only: every consumer reads the rounded value
                         __align__(16) __nv_bfloat16 hb[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float h = 0.f;
                             if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
                             hb[i] = __float2bfloat16_rn(h);
-                            v[i] = __bfloat162float(hb[i]);      // the state every consumer sees is the bf16 value
                         }
                         uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
                         dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
                         dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
-                        float* dstf = c.arena + (size_t)it.x * H + col;
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4)
-                            if (col + i < H) *reinterpret_cast<float4*>(dstf + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                     } else if (MODE == TC_LSTM_DE) {
                         // embedding gradient: row tok of dE gathers the contribution of this leaf
 #pragma unroll
@@ -395,34 +391,35 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
     }
 }
 
-// Leaves in bf16 mode: state(slot) = E[tok] in both arenas (pad columns of the bf16 row are zero).
+// Leaves in bf16 mode: state(slot) = bf16(E[tok]), pad columns of the row zero.  Each warp takes four
+// leaves at a time, so that four rows are in flight per warp.
 static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
     const int H = c.H, Hp = c.Hp;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
     const int n_warps = gridDim.x * blockDim.x / 32;
-    for (uint32_t i = warp; i < n_items; i += n_warps) {
-        const uint2 it = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[i]));          // {slot, tok}
-        const float* src = c.E + (size_t)it.y * c.D;
-        float* dst = c.arena + (size_t)it.x * H;
-        __nv_bfloat16* dstb = c.arena_bf + (size_t)it.x * Hp;
-        for (int k = lane * 8; k < Hp; k += 256) {             // 8 elements per lane: 32 bytes in, 16 + 32 bytes out
-            float v[8];
+    for (uint32_t i0 = warp * 4; i0 < n_items; i0 += n_warps * 4) {
+        uint2 it[4];
 #pragma unroll
-            for (int i = 0; i < 8; i += 4) {
-                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (k + i < H) t = __ldg(reinterpret_cast<const float4*>(src + k + i));
-                v[i] = t.x; v[i + 1] = t.y; v[i + 2] = t.z; v[i + 3] = t.w;
+        for (int q = 0; q < 4; ++q)
+            it[q] = i0 + q < n_items ? __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[i0 + q])) : make_uint2(0u, 0u);   // {slot, tok}
+        for (int k = lane * 8; k < Hp; k += 256) {             // 8 elements per lane: 32 bytes in, 16 bytes out
+            float4 v[4][2];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    v[q][e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i0 + q < n_items && k + 4 * e < H)
+                        v[q][e] = __ldg(reinterpret_cast<const float4*>(c.E + (size_t)it[q].y * c.D + k + 4 * e));
+                }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (i0 + q >= n_items) continue;
+                __align__(16) __nv_bfloat162 hb[4];
+                hb[0] = __floats2bfloat162_rn(v[q][0].x, v[q][0].y); hb[1] = __floats2bfloat162_rn(v[q][0].z, v[q][0].w);
+                hb[2] = __floats2bfloat162_rn(v[q][1].x, v[q][1].y); hb[3] = __floats2bfloat162_rn(v[q][1].z, v[q][1].w);
+                *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it[q].x * Hp + k) = *reinterpret_cast<const uint4*>(hb);
             }
-            __align__(16) __nv_bfloat16 hb[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                hb[i] = __float2bfloat16_rn(v[i]);
-                v[i] = __bfloat162float(hb[i]);
-            }
-            *reinterpret_cast<uint4*>(dstb + k) = *reinterpret_cast<const uint4*>(hb);
-#pragma unroll
-            for (int i = 0; i < 8; i += 4)
-                if (k + i < H) *reinterpret_cast<float4*>(dst + k + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
         }
     }
 }
