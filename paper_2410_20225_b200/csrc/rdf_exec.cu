@@ -356,6 +356,31 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
                     if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
                     if (threadIdx.x < m) run_token(c, sp, wave, load_token(&c.q[wave & 1][threadIdx.x]), st);
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
+                    if (k == 0) {
+                        // The next wave clears the counter that the other blocks read to take this branch:
+                        // carry on only when all of them have arrived at the grid barrier below (they
+                        // read the counter before they arrive).  Bounded like every other wait.
+                        __shared__ int others_in;
+                        if (threadIdx.x == 0) {
+                            const uint32_t target = generation * gridDim.x + gridDim.x - 1;
+                            const long long t0 = clock64();
+                            int good = 1;
+                            while (ld_volatile_u32(&c.ctl->bar) < target) {
+                                if (clock64() - t0 > c.spin_limit) {
+                                    set_status(c, RDF_ERR_TIMEOUT);
+                                    good = 0;
+                                    break;
+                                }
+                                __nanosleep(32);
+                            }
+                            others_in = good;
+                        }
+                        __syncthreads();
+                        if (!others_in) {
+                            ++wave;
+                            break;
+                        }
+                    }
                     ++wave;
                     ++k;
                     m = ld_volatile_u32(&c.ctl->qcount[wave % 3]);

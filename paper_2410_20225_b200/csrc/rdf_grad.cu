@@ -28,107 +28,201 @@ __device__ __forceinline__ void unpack_bf8(const uint4& v, float (&x)[8]) {
     }
 }
 
-// per invocation f: z = W_s h + b_s; loss += logsumexp(z) - z[label]; dlog = softmax(z) - onehot
+// Loss head and its parameter gradients in one streaming pass over the retained states:
+//   per invocation f:  z = W_s h_f + b_s;  loss += logsumexp(z) - z[label];  dlog_f = softmax(z) - onehot
+//   dW_s[k][j] = sum_f dlog_f[k] * h_f[j];   db_s[k] = sum_f dlog_f[k]
+// A block owns a contiguous range of invocations (consecutive frame ids = consecutive rows) and moves
+// it through shared memory in slabs of `fr` rows with bulk asynchronous copies, two slabs in flight.
+// BF: rows of the bf16 arena (Hp bf16, pad columns zero); else rows of the fp32 arena (S floats).
+static const int LH_MAX_ROWS = 64;          // rows per slab
+static const int LH_SLAB_BYTES = 48 * 1024;
+static const int GRAD_MAX_H = 1024;         // widest hidden size of the gradient pass
+
 template <bool BF>
-__global__ void __launch_bounds__(256) rdf_loss_kernel(const DevCtx c) {
-    // four invocations per warp (8 lanes each); a lane loads all its pieces of the row before it uses them
+__global__ void __launch_bounds__(256) rdf_loss_heads_kernel(const DevCtx c, int fr, int rowbytes) {
+    extern __shared__ __align__(128) unsigned char slab_smem[];
+    __shared__ __align__(8) uint64_t mbars[2];
+    __shared__ __align__(16) float s_dl[LH_MAX_ROWS][8];
+    __shared__ int s_lab[2][LH_MAX_ROWS];
     __shared__ float warp_loss[8];
-    const uint32_t F = c.ctl->frame_count;
-    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, sub = lane / 8, sl = lane % 8;
-    const uint32_t warp = blockIdx.x * 8 + wib, n_warps = gridDim.x * 8;
+    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
+    const uint32_t n = F > B ? F - B : 0u, per = (n + gridDim.x - 1) / gridDim.x;
+    const uint32_t f0 = min(F, B + blockIdx.x * per), f1 = min(F, f0 + per);
+    const int n_slabs = (int)((f1 - f0 + fr - 1) / fr);
+    const int tid = threadIdx.x, lane = tid % 32, wib = tid / 32;
     const int H = c.H, C = c.n_classes;
-    float my_loss = 0.f;
-    for (uint32_t base = (uint32_t)c.B + warp * 4; base < F; base += n_warps * 4) {
-        const uint32_t f = base + sub;
-        const bool act = f < F;
-        float z[MAX_CLASSES];
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k) z[k] = 0.f;
-        if (BF) {
-            const __nv_bfloat16* h = c.arena_bf + (size_t)(act ? f : base) * c.Hp;
-            uint4 hv[TC_HP_MAX / 64];
-#pragma unroll
-            for (int q = 0; q < TC_HP_MAX / 64; ++q) {
-                const int j = sl * 8 + 64 * q;
-                hv[q] = j < c.Hp ? *reinterpret_cast<const uint4*>(h + j) : make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll
-            for (int q = 0; q < TC_HP_MAX / 64; ++q) {
-                const int j = sl * 8 + 64 * q;
-                if (j >= H) continue;
-                float x[8];
-                unpack_bf8(hv[q], x);
-#pragma unroll
-                for (int k = 0; k < MAX_CLASSES; ++k)
-                    if (k < C) {
-                        const float4 w0 = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                        z[k] += w0.x * x[0] + w0.y * x[1] + w0.z * x[2] + w0.w * x[3];
-                        if (j + 4 < H) {
-                            const float4 w1 = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j + 4]));
-                            z[k] += w1.x * x[4] + w1.y * x[5] + w1.z * x[6] + w1.w * x[7];
-                        }
-                    }
-            }
-        } else {
-            const float* h = c.arena + (size_t)(act ? f : base) * c.S;
-#pragma unroll 4
-            for (int j = sl * 4; j < H; j += 32) {
-                const float4 h4 = *reinterpret_cast<const float4*>(h + j);
-#pragma unroll
-                for (int k = 0; k < MAX_CLASSES; ++k)
-                    if (k < C) {
-                        const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                        z[k] += w.x * h4.x + w.y * h4.y + w.z * h4.z + w.w * h4.w;
-                    }
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            for (int o = 4; o > 0; o >>= 1) z[k] += __shfl_xor_sync(0xffffffffu, z[k], o);
-        if (act && sl == 0) {
-            const int node = (int)c.frames[f].arg;
-            const int lab = __ldg(&c.label[node]);
-            float m = -INFINITY;
-#pragma unroll
-            for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) {
-                    z[k] += __ldg(&c.b_s[k]);
-                    m = fmaxf(m, z[k]);
-                }
-            float s = 0.f, zl = 0.f;
-#pragma unroll
-            for (int k = 0; k < MAX_CLASSES; ++k)
-                if (k < C) {
-                    s += expf(z[k] - m);
-                    if (k == lab) zl = z[k];
-                }
-            my_loss += logf(s) + m - zl;
-            float d[MAX_CLASSES];
-#pragma unroll
-            for (int k = 0; k < MAX_CLASSES; ++k) d[k] = k < C ? expf(z[k] - m) / s - (k == lab ? 1.f : 0.f) : 0.f;
-            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8) = make_float4(d[0], d[1], d[2], d[3]);
-            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8 + 4) = make_float4(d[4], d[5], d[6], d[7]);
-        }
+    const uint32_t mbar = smem_u32(mbars), stage0 = smem_u32(slab_smem);
+    const uint32_t stage_bytes = (uint32_t)fr * rowbytes;
+    const unsigned char* rows = BF ? reinterpret_cast<const unsigned char*>(c.arena_bf)
+                                   : reinterpret_cast<const unsigned char*>(c.arena);
+    if (tid == 0) {
+        mbar_init(mbar, 1);
+        mbar_init(mbar + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // fixed-order sum of the four group leaders, then of the warps
-    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 16);
-    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 8);
+    __syncthreads();
+    auto issue = [&](int i) {
+        const uint32_t fs = f0 + (uint32_t)i * fr, cnt = min((uint32_t)fr, f1 - fs);
+        if (tid == 0) {
+            const uint32_t bytes = cnt * rowbytes, mb = mbar + 8 * (i & 1);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mb), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(stage0 + (i & 1) * stage_bytes), "l"(rows + (size_t)fs * rowbytes), "r"(bytes), "r"(mb) : "memory");
+        }
+        if (tid < (int)cnt) s_lab[i & 1][tid] = __ldg(&c.label[(int)c.frames[fs + tid].arg]);
+    };
+    // W_s in shared memory, behind the two slab stages
+    float* s_ws = reinterpret_cast<float*>(slab_smem + 2 * (size_t)stage_bytes);
+    for (int q = tid; q < C * H; q += 256) s_ws[q] = __ldg(&c.W_s[q]);
+    // dW_s: G groups of four hidden units, n_sets threads per group (GRAD_MAX_H / 4 = 256 threads at most per set)
+    const int G = (H + 3) / 4, n_sets = 256 / G, cg = tid % G, set = tid / G;
+    float acc[4][MAX_CLASSES];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) acc[e][k] = 0.f;
+    float my_loss = 0.f, my_dbs = 0.f;
+    bool ok = true;
+    if (n_slabs > 0) issue(0);
+    for (int i = 0; i < n_slabs && ok; ++i) {
+        if (i + 1 < n_slabs) issue(i + 1);             // its stage was released by the barrier that ended slab i - 1
+        const uint32_t fs = f0 + (uint32_t)i * fr, cnt = min((uint32_t)fr, f1 - fs);
+        ok = __syncthreads_and(mbar_wait(c, mbar + 8 * (i & 1), (uint32_t)(i >> 1) & 1u)) != 0;
+        if (!ok) break;                                // the whole block agrees
+        const unsigned char* st = slab_smem + (size_t)(i & 1) * stage_bytes;
+        // ---- logits, loss, dlog: a warp takes four rows at a time, a lane 8 hidden units per 256;
+        //      a piece of W_s (from shared memory) serves all four rows
+        for (uint32_t fb = wib * 4; fb < cnt; fb += 32) {
+            float z[4][MAX_CLASSES];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k) z[r][k] = 0.f;
+            for (int j = lane * 8; j < H; j += 256) {
+                float x[4][8];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const unsigned char* row = st + (size_t)min(fb + r, cnt - 1) * rowbytes;
+                    if (BF) {
+                        unpack_bf8(*reinterpret_cast<const uint4*>(row + 2 * j), x[r]);
+                    } else {
+                        const float4 a = *reinterpret_cast<const float4*>(row + 4 * j);
+                        const float4 b = j + 4 < H ? *reinterpret_cast<const float4*>(row + 4 * j + 16) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        x[r][0] = a.x; x[r][1] = a.y; x[r][2] = a.z; x[r][3] = a.w;
+                        x[r][4] = b.x; x[r][5] = b.y; x[r][6] = b.z; x[r][7] = b.w;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        const float4 w0 = *reinterpret_cast<const float4*>(&s_ws[k * H + j]);
+                        const float4 w1 = j + 4 < H ? *reinterpret_cast<const float4*>(&s_ws[k * H + j + 4]) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int r = 0; r < 4; ++r)
+                            z[r][k] += w0.x * x[r][0] + w0.y * x[r][1] + w0.z * x[r][2] + w0.w * x[r][3] +
+                                       w1.x * x[r][4] + w1.y * x[r][5] + w1.z * x[r][6] + w1.w * x[r][7];
+                    }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C)
+                        for (int o = 16; o > 0; o >>= 1) z[r][k] += __shfl_xor_sync(0xffffffffu, z[r][k], o);
+            // lane r finishes row fb + r
+            float zr[MAX_CLASSES];
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k) zr[k] = lane == 0 ? z[0][k] : lane == 1 ? z[1][k] : lane == 2 ? z[2][k] : z[3][k];
+            const uint32_t fi = fb + lane;
+            if (lane < 4 && fi < cnt) {
+                const int lab = s_lab[i & 1][fi];
+                float m = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        zr[k] += __ldg(&c.b_s[k]);
+                        m = fmaxf(m, zr[k]);
+                    }
+                float sum = 0.f, zl = 0.f;
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        sum += expf(zr[k] - m);
+                        if (k == lab) zl = zr[k];
+                    }
+                my_loss += logf(sum) + m - zl;
+                float d[MAX_CLASSES];
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k) d[k] = k < C ? expf(zr[k] - m) / sum - (k == lab ? 1.f : 0.f) : 0.f;
+                const float4 lo = make_float4(d[0], d[1], d[2], d[3]), hi = make_float4(d[4], d[5], d[6], d[7]);
+                *reinterpret_cast<float4*>(c.dlog + (size_t)(fs + fi) * 8) = lo;
+                *reinterpret_cast<float4*>(c.dlog + (size_t)(fs + fi) * 8 + 4) = hi;
+                *reinterpret_cast<float4*>(&s_dl[fi][0]) = lo;
+                *reinterpret_cast<float4*>(&s_dl[fi][4]) = hi;
+            }
+        }
+        __syncthreads();
+        // ---- dW_s, db_s: a thread owns four hidden units and every n_sets-th row; sums stay in registers
+        if (tid < n_sets * G) {
+            for (uint32_t fi = set; fi < cnt; fi += n_sets) {
+                const unsigned char* row = st + (size_t)fi * rowbytes;
+                float hx[4];
+                if (BF) {
+                    const uint2 v = *reinterpret_cast<const uint2*>(row + 8 * cg);
+                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+                    hx[0] = a.x; hx[1] = a.y; hx[2] = b.x; hx[3] = b.y;
+                } else {
+                    const float4 v = *reinterpret_cast<const float4*>(row + 16 * cg);
+                    hx[0] = v.x; hx[1] = v.y; hx[2] = v.z; hx[3] = v.w;
+                }
+                const float4 d0 = *reinterpret_cast<const float4*>(&s_dl[fi][0]);
+                const float4 d1 = *reinterpret_cast<const float4*>(&s_dl[fi][4]);
+                const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int k = 0; k < MAX_CLASSES; ++k) acc[e][k] = fmaf(dl[k], hx[e], acc[e][k]);
+            }
+        }
+        if (tid < C)
+            for (uint32_t fi = 0; fi < cnt; ++fi) my_dbs += s_dl[fi][tid];
+        __syncthreads();                               // the stage and s_dl are free again
+    }
+    if (tid < n_sets * G && n_slabs > 0) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C && 4 * cg + e < H) atomicAdd(&c.dW_s[k * H + 4 * cg + e], acc[e][k]);
+    }
+    if (tid < C && n_slabs > 0) atomicAdd(&c.db_s[tid], my_dbs);
+    // lanes 0..3 of every warp hold row losses: fixed-order sum inside the warp, then over the warps
+    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 2);
+    my_loss += __shfl_down_sync(0xffffffffu, my_loss, 1);
     if (lane == 0) warp_loss[wib] = my_loss;
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         float t = 0.f;
         for (int w = 0; w < 8; ++w) t += warp_loss[w];
         c.loss_partial[blockIdx.x] = t;
     }
 }
 
-__global__ void rdf_loss_final_kernel(const DevCtx c, int n_partials) {
-    // one thread, fixed order: the same partials always give the same sum
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        double t = 0.0;
-        for (int i = 0; i < n_partials; ++i) t += (double)c.loss_partial[i];
-        c.ctl->loss = (float)t;
-        if (c.loss_out) *c.loss_out = (float)t;
+// Sum of the per-block partial losses in a fixed order (the same partials always give the same sum).
+__global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int n_partials) {
+    __shared__ double part[256];
+    double t = 0.0;
+    for (int i = threadIdx.x; i < n_partials; i += 256) t += (double)c.loss_partial[i];
+    part[threadIdx.x] = t;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        c.ctl->loss = (float)part[0];
+        if (c.loss_out) *c.loss_out = (float)part[0];
         c.ctl->forward_status = c.ctl->status;      // what the gradient kernel checks before it starts
     }
 }
@@ -233,11 +327,11 @@ __device__ __forceinline__ void backward_frame_tc(const DevCtx& c, uint32_t t, i
         } else {
             float x[8];
             unpack_bf8(hv[q], x);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dh[i] *= 1.f - x[i] * x[i];      // pad columns: dh = 0 and h = 0, so dz = 0
             __align__(16) __nv_bfloat162 pk[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)                 // pad columns: dh = 0 and h = 0, so dz = 0
-                pk[i] = __floats2bfloat162_rn(dh[2 * i] * (1.f - x[2 * i] * x[2 * i]),
-                                              dh[2 * i + 1] * (1.f - x[2 * i + 1] * x[2 * i + 1]));
+            for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(dh[2 * i], dh[2 * i + 1]);
             *reinterpret_cast<uint4*>(c.dz_bf + (size_t)t * Hp + j) = *reinterpret_cast<const uint4*>(pk);
         }
     }
@@ -596,7 +690,11 @@ __global__ void __launch_bounds__(256) rdf_outer_kernel(const DevCtx c, const Ou
 }
 
 // out[m] = sum over the listed invocations of A_t[m]   (bias gradients)
-__global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, const uint32_t* count, const float* A,
+__device__ __forceinline__ float as_float(float v) { return v; }
+__device__ __forceinline__ float as_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T>
+__global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, const uint32_t* count, const T* A,
                                                          int lda, int M, float* out) {
     const uint32_t n = *count;
     const uint32_t per = (n + gridDim.x - 1) / gridDim.x;
@@ -604,46 +702,9 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, c
     if (t0 >= t1) return;
     for (int j = threadIdx.x; j < M; j += blockDim.x) {
         float s = 0.f;
-#pragma unroll 4
-        for (uint32_t i = t0; i < t1; ++i) s += A[(size_t)list[i] * lda + j];
-        atomicAdd(&out[j], s);
-    }
-}
-
-// Column sums over all invocations, one thread per hidden unit j:
-//   dW_s[k][j] = sum_f dlog_f[k] * h_f[j];   db_s[k] = sum_f dlog_f[k];
-//   WITH_DB (TreeRNN): db[j] = sum over the cells of dz_f[j]
-// BF: states and dz are the bf16 rows (stride Hp) of the bf16 TreeRNN, else fp32 rows (stride S; dz in dhp).
-template <bool BF, bool WITH_DB>
-__global__ void __launch_bounds__(128) rdf_heads_kernel(const DevCtx c) {
-    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
-    const uint32_t n = F - B, per = (n + gridDim.x - 1) / gridDim.x;
-    const uint32_t f0 = B + blockIdx.x * per, f1 = min(F, f0 + per);
-    if (f0 >= f1) return;
-    const int H = c.H, C = c.n_classes;
-    for (int j = threadIdx.x; j < H; j += blockDim.x) {
-        float s[MAX_CLASSES], db = 0.f;
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k) s[k] = 0.f;
 #pragma unroll 8
-        for (uint32_t f = f0; f < f1; ++f) {
-            const float hj = BF ? __bfloat162float(c.arena_bf[(size_t)f * c.Hp + j]) : c.arena[(size_t)f * c.S + j];
-            const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8);
-            const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)f * 8 + 4);
-            s[0] = fmaf(d0.x, hj, s[0]); s[1] = fmaf(d0.y, hj, s[1]); s[2] = fmaf(d0.z, hj, s[2]); s[3] = fmaf(d0.w, hj, s[3]);
-            s[4] = fmaf(d1.x, hj, s[4]); s[5] = fmaf(d1.y, hj, s[5]); s[6] = fmaf(d1.z, hj, s[6]); s[7] = fmaf(d1.w, hj, s[7]);
-            if (WITH_DB && c.op_l[f] != LEAF_MARK)
-                db += BF ? __bfloat162float(c.dz_bf[(size_t)f * c.Hp + j]) : c.dhp[(size_t)f * c.S + j];
-        }
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            if (k < C) atomicAdd(&c.dW_s[k * H + j], s[k]);
-        if (WITH_DB) atomicAdd(&c.db[j], db);
-    }
-    if (threadIdx.x < C) {
-        float s = 0.f;
-        for (uint32_t f = f0; f < f1; ++f) s += c.dlog[(size_t)f * 8 + threadIdx.x];
-        atomicAdd(&c.db_s[threadIdx.x], s);
+        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)list[i] * lda + j]);
+        atomicAdd(&out[j], s);
     }
 }
 
@@ -719,6 +780,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     if (g->has_lstm && (!grads->dW_x || !grads->db_x)) return RDF_ERR_BAD_ARG;
     if (!params->W_s || !params->b_s || !in->label || !out->loss) return RDF_ERR_BAD_ARG;
     if (params->n_classes < 1 || params->n_classes > MAX_CLASSES) return RDF_ERR_BAD_ARG;
+    if (params->H > GRAD_MAX_H) return RDF_ERR_UNSUPPORTED;
     Layout L;
     rc = rdf_make_layout(g, in, params, 1, L);
     if (rc != RDF_OK) return rc;
@@ -749,11 +811,21 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rc = rdf_launch_forward(g, in, out, ws, L, S, c, stream);
     if (rc != RDF_OK) return rc;
     // loss head over every retained invocation
-    const int loss_blocks = std::min(4096, std::max(1, (int)((in->max_invocations + 63) / 64)));
     const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
-    if (tc_rnn) rdf_loss_kernel<true><<<loss_blocks, 256, 0, stream>>>(c);
-    else rdf_loss_kernel<false><<<loss_blocks, 256, 0, stream>>>(c);
-    rdf_loss_final_kernel<<<1, 32, 0, stream>>>(c, loss_blocks);
+    {
+        const int rowbytes = tc_rnn ? c.Hp * 2 : c.S * 4;
+        const int fr = std::max(1, std::min(LH_MAX_ROWS, LH_SLAB_BYTES / rowbytes));
+        const int smem = 2 * fr * rowbytes + params->n_classes * H * (int)sizeof(float);
+        const int loss_blocks = std::min(4096, 2 * S->grid);
+        if (tc_rnn) {
+            CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            rdf_loss_heads_kernel<true><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes);
+        } else {
+            CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            rdf_loss_heads_kernel<false><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes);
+        }
+        rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks);
+    }
     rdf_mark(S, 3, stream);
     // gradient waves
     CUDA_OK(cudaGetLastError());
@@ -799,16 +871,11 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 5, stream);
-    if (lstm) {
-        rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
-        rdf_colsum_kernel<<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
-    }
+    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, grads->db);
+    else rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
+    if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
     rdf_mark(S, 6, stream);
-    // dW_s, db_s (and the TreeRNN's db) in one pass over the retained states
-    if (lstm) rdf_heads_kernel<false, false><<<16 * S->grid, 128, 0, stream>>>(c);
-    else if (tc_rnn) rdf_heads_kernel<true, true><<<16 * S->grid, 128, 0, stream>>>(c);
-    else rdf_heads_kernel<false, true><<<16 * S->grid, 128, 0, stream>>>(c);
-    rdf_mark(S, 7, stream);
+    rdf_mark(S, 7, stream);       // (dW_s and db_s come from the loss-head pass)
     if (tc_lstm) {
         const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 4);
         CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));
