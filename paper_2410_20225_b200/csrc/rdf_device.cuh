@@ -53,13 +53,14 @@ struct Control {
     int32_t  status;
     uint32_t bar;                 // grid barrier arrivals (monotone)
     uint32_t qcount[3];           // tokens in the queue of wave w at [w % 3]
-    uint32_t cell_count[2];       // ready cells of wave w at [w % 2]
-    uint32_t leaf_count[2];
+    uint32_t cell_count;          // ready cells queued so far, all waves (length of cell_items)
+    uint32_t leaf_count;          // ready leaves queued so far (length of leaf_items)
     uint32_t frame_count;
     uint32_t waves, waves_backward, max_wave_tokens, max_probe, max_depth;
     uint32_t all_cells;           // backward: cells seen so far (length of the all-cells list)
     uint32_t all_leaves;          // backward: leaves seen so far
     uint32_t bar2;                // barrier counter of the backward kernel
+    uint32_t bar_ops;             // barrier counter of the operator kernel
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
@@ -95,8 +96,8 @@ struct DevCtx {
     Slot*     table;
     uint64_t  table_cap;          // slots per match node, power of two
     // batched operators
-    CellItem* cell_items;
-    LeafItem* leaf_items;
+    CellItem* cell_items;         // every cell in the order it became ready (wave after wave)
+    LeafItem* leaf_items;         // every leaf in the order it was reached
     uint32_t  work_cap;
     uint32_t* op_l;               // per frame: operand frames of the operator that made its state
     uint32_t* op_r;               //            (leaf: op_l = LEAF_MARK, op_r = token id)
@@ -125,9 +126,10 @@ struct DevCtx {
     float*    dhp;                // [frame_cap, S]: gradient arriving from the caller (dh, and dc for the TreeLSTM);
                                   //                 TreeRNN: overwritten by dz (cell) / dh (leaf)
     float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
-    uint32_t* wave_frames;        // [wave_cap]: frames allocated up to the end of forward wave w.  Frame ids are
-                                  // handed out in wave order, so the invocations that Call_i created in wave w are
-                                  // the id range [wave_frames[w-1], wave_frames[w]) -- one wave of the gradient pass
+    uint4*    wave_marks;         // [wave_cap]: {frames, cells, leaves} counted up to the end of scheduler wave w.
+                                  // Frame ids are handed out in wave order, so the invocations that Call_i created
+                                  // in wave w are the id range [marks[w-1].x, marks[w].x) -- one wave of the gradient
+                                  // pass; the cells that became ready in wave w are cell_items[marks[w-1].y, marks[w].y)
     uint32_t  wave_cap;
     uint32_t* all_cells;          // every cell frame, in backward wave order
     uint4*    cell_ops;           // {cell frame, left operand frame, right operand frame, 1} in all_cells order
@@ -162,19 +164,33 @@ __device__ __forceinline__ uint32_t aggregated_inc(uint32_t* counter) {
     return g.shfl(base, 0) + g.thread_rank();
 }
 
+// What the operator kernel and the gradient pass need to know about scheduler wave w: how many
+// frames, ready cells and ready leaves existed at its end.  Written by one thread at a moment when
+// every block has finished wave w and none has begun wave w + 1.
+__device__ __forceinline__ void mark_wave(const DevCtx& c, uint32_t wave) {
+    if (c.wave_marks && wave < c.wave_cap)
+        c.wave_marks[wave] = make_uint4(ld_volatile_u32(&c.ctl->frame_count), ld_volatile_u32(&c.ctl->cell_count),
+                                        ld_volatile_u32(&c.ctl->leaf_count), 0u);
+}
+static const uint32_t NO_MARK = 0xFFFFFFFFu;
+
 // Grid-wide barrier with a bounded wait.  All blocks of the (cooperatively
 // launched, hence co-resident) grid call it the same number of times.  The
 // counter only grows; generation k is complete when it reaches k * gridDim.x.
 // Returns false when the wait expired or any block reported an error; the
-// caller then leaves the kernel.
-__device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter, uint32_t& generation) {
+// caller then leaves the kernel.  With mark != NO_MARK the last block to arrive
+// (all others have finished their work, none has left the barrier) records the
+// counts of scheduler wave `mark`.
+__device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter, uint32_t& generation,
+                                             uint32_t mark = NO_MARK) {
     __shared__ int ok;
     __syncthreads();
     if (threadIdx.x == 0) {
         ++generation;
         const uint32_t target = generation * gridDim.x;
         __threadfence();
-        atomicAdd(counter, 1u);
+        const uint32_t before = atomicAdd(counter, 1u);
+        if (mark != NO_MARK && before + 1 == target) mark_wave(c, mark);
         const long long t0 = clock64();
         int good = 1;
         while (ld_volatile_u32(counter) < target) {

@@ -1,10 +1,12 @@
-// Device executor, forward: a persistent, cooperatively launched kernel runs
-// all waves of the tagged dataflow graph without returning to the host.  Each
-// wave
-//   S) takes the wave's tokens, runs their segments (tag push / pop, Switch,
-//      token-store insert or match), emits the next wave's tokens and the lists
-//      of ready batched operators;
-//   C) fires every ready leaf / cell operator of the wave as one batch.
+// Device executor, forward: persistent, cooperatively launched kernels run all
+// waves of the tagged dataflow graph without returning to the host.
+//   Scheduler kernel: every wave takes its tokens, runs their segments (tag
+//      push / pop, Switch, token-store insert or match) and emits the next
+//      wave's tokens.  A vector value travels by reference (the frame that
+//      holds it), so a ready leaf / cell operator is queued, not computed: the
+//      kernel leaves behind, wave by wave, the lists of ready operators.
+//   Operator kernel: fires the ready operators of each wave as one batch, the
+//      waves in the order in which the scheduler formed them.
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
@@ -40,7 +42,7 @@ __device__ __forceinline__ void load_program(const DevCtx& c, SharedProgram& sp)
 // that carries its state onwards in the next wave.
 __device__ __forceinline__ void fire_cell(const DevCtx& c, const MatchNode& M, uint32_t wave, uint64_t tag,
                                           const int64_t* regs, ThreadStats& st) {
-    const uint32_t i = aggregated_inc(&c.ctl->cell_count[wave & 1]);
+    const uint32_t i = aggregated_inc(&c.ctl->cell_count);
     if (i >= c.work_cap) {
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
@@ -161,7 +163,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
             }
             case VM_EMBED:
             case VM_LEAF_LSTM: {
-                const uint32_t i = aggregated_inc(&c.ctl->leaf_count[wave & 1]);
+                const uint32_t i = aggregated_inc(&c.ctl->leaf_count);
                 if (i >= c.work_cap) {
                     set_status(c, RDF_ERR_QUEUE_FULL);
                     return;
@@ -187,7 +189,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
 // C phase, fp32: leaf gather and the TreeRNN cell as a tiled FFMA contraction
 // ===========================================================================
 // out[i][j] = tanh( sum_k W[j][k] * x_i[k] + b[j] ),  x_i = [state(l_i) ; state(r_i)]
-__device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) {
+__device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, uint32_t n_items) {
     const int H = c.H, K2 = 2 * c.H;
     const int tiles_m = (n_items + TM - 1) / TM, tiles_n = (H + TN - 1) / TN;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
@@ -199,7 +201,7 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) 
         const int arow = row0 + lrow;
         const float *xl = nullptr, *xr = nullptr;
         if (arow < (int)n_items) {
-            const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[arow]));   // {out, l, r, -}
+            const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + arow]));   // {out, l, r, -}
             xl = c.arena + (size_t)it.y * H;
             xr = c.arena + (size_t)it.z * H;
         }
@@ -228,7 +230,7 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) 
             for (int i = 0; i < 4; ++i) {
                 const int row = row0 + ty * 4 + i;
                 if (row < (int)n_items) {
-                    const uint32_t out = __ldcg(&c.cell_items[row].out);
+                    const uint32_t out = __ldcg(&c.cell_items[first + row].out);
                     float4 v;
                     v.x = tanhf(acc[i][0] + bias.x); v.y = tanhf(acc[i][1] + bias.y);
                     v.z = tanhf(acc[i][2] + bias.z); v.w = tanhf(acc[i][3] + bias.w);
@@ -243,7 +245,7 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t n_items) 
 // a handful of blocks busy with a long dependent k-loop.  Here one block step computes an 8 cell x 16
 // column patch with the whole contraction spread over its threads: thread = (cell, column, half of k),
 // streaming its operand row and weight row with independent 128-bit loads.
-__device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t n_items) {
+__device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t first, uint32_t n_items) {
     // xs: shared staging for the 8 operand rows [h_l ; h_r] of the patch (8 x 2H floats) + 128 floats
     const int H = c.H, K2 = 2 * c.H;
     float* red = xs + 8 * K2;
@@ -256,7 +258,7 @@ __device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t n_items) {
             const int r = p / (K2 / 4), k = (p % (K2 / 4)) * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             if (row0 + r < (int)n_items) {
-                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row0 + r]));   // {out, l, r, -}
+                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row0 + r]));   // {out, l, r, -}
                 v = k < H ? ldcg4(c.arena + (size_t)it.y * H + k) : ldcg4(c.arena + (size_t)it.z * H + (k - H));
             }
             *reinterpret_cast<float4*>(xs + r * K2 + k) = v;
@@ -280,7 +282,7 @@ __device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t n_items) {
         if (kh == 1) red[o] = acc;
         __syncthreads();
         if (kh == 0 && live)
-            c.arena[(size_t)__ldcg(&c.cell_items[row].out) * H + col] = tanhf(acc + red[o] + __ldg(&c.b[col]));
+            c.arena[(size_t)__ldcg(&c.cell_items[first + row].out) * H + col] = tanhf(acc + red[o] + __ldg(&c.b[col]));
         __syncthreads();
     }
 }
@@ -320,12 +322,12 @@ __device__ __forceinline__ void flush_stats(const DevCtx& c, const ThreadStats& 
     }
 }
 
-static const uint32_t INT_NARROW_STRETCH = 4096;   // waves block 0 runs alone before it meets the grid again
+static const uint32_t NARROW_STRETCH = 4096;   // waves block 0 runs alone before it meets the grid again
 
-// Lean variant of the persistent kernel for programs without vector operators (integer recursion):
-// only the S phase exists, so the block can be four times as wide and hide four times as much of the
-// latency of the dependent L2 round trips (queue, frame table, store) that a token makes.
-__global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_constant__ DevCtx c) {
+// The scheduler: all waves of token processing, for integer and for vector programs.  Only tokens are
+// handled here, so the block is 1024 threads wide: the dependent L2 round trips of a token (queue,
+// frame table, store) are hidden by the number of tokens in flight.
+__global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_constant__ DevCtx c) {
     __shared__ SharedProgram sp;
     load_program(c, sp);
     ThreadStats st;
@@ -348,7 +350,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
             // A stretch of narrow waves (deep, thin recursion): one block has a thread for every token,
             // so block 0 runs wave after wave with a block barrier between them while the other blocks
             // wait at the grid barrier below.  It comes back to the grid when a wave is wider than the
-            // block, when the queue is empty, or after INT_NARROW_STRETCH waves (so that the bounded
+            // block, when the queue is empty, or after NARROW_STRETCH waves (so that the bounded
             // wait of the other blocks never expires on a long stretch).
             if (blockIdx.x == 0) {
                 uint32_t m = n, k = 0;
@@ -356,6 +358,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
                     if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
                     if (threadIdx.x < m) run_token(c, sp, wave, load_token(&c.q[wave & 1][threadIdx.x]), st);
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
+                    if (threadIdx.x == 0) mark_wave(c, wave);
                     if (k == 0) {
                         // The next wave clears the counter that the other blocks read to take this branch:
                         // carry on only when all of them have arrived at the grid barrier below (they
@@ -385,7 +388,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
                     ++k;
                     m = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
                     widest = max(widest, m);
-                } while (m != 0 && m <= blockDim.x && k < INT_NARROW_STRETCH && wave < c.wave_limit &&
+                } while (m != 0 && m <= blockDim.x && k < NARROW_STRETCH && wave < c.wave_limit &&
                          ld_volatile_i32(&c.ctl->status) == 0);
                 if (threadIdx.x == 0) c.ctl->resume_wave = wave;
             }
@@ -401,14 +404,15 @@ __global__ void __launch_bounds__(1024, 1) rdf_forward_int_kernel(const __grid_c
             run_token(c, sp, wave, load_token(&q[i]), st);
         __syncthreads();
         lap(cyc_s);
-        if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        if (!grid_barrier(c, &c.ctl->bar, generation, wave)) break;
         lap(cyc_b);
     }
     flush_stats(c, st);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->waves = wave;
         c.ctl->max_wave_tokens = widest;
-        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[1] = 0; c.ctl->cyc[2] = cyc_b;
+        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[2] = cyc_b;
+        c.ctl->forward_status = c.ctl->status;      // what the operator kernel checks before it starts
     }
 }
 
@@ -434,86 +438,63 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     }
 }
 
-__global__ void __launch_bounds__(256, 1) rdf_forward_kernel(const __grid_constant__ DevCtx c) {
-    __shared__ SharedProgram sp;
+// The operator kernel: the leaves first (they wait for nothing), then, wave by wave, the cells that
+// became ready in that wave; a grid barrier separates the waves (a cell reads states of earlier waves).
+__global__ void __launch_bounds__(256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
     __shared__ LstmSmem tile_smem;                                   // the TreeRNN tiles use its first part
     GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
     extern __shared__ unsigned char dyn_smem[];                      // operand stages of the tensor-core path
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
     __shared__ uint4 tc_items[TC_M];
+    if (c.ctl->forward_status != 0) return;                          // the scheduler failed: the lists are not to be trusted
     TcState tc;
-    load_program(c, sp);
     if (c.use_tc) {
         if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Hp / 16, 3, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
         else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 4, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
     }
-    ThreadStats st;
-    uint32_t generation = 0, wave = 0, widest = 0;
-    long long cyc_s = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
+    uint32_t generation = 0;
+    long long cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
         const long long now = clock64();
         acc += now - t_mark;
         t_mark = now;
     };
-    for (;; ++wave) {
-        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
-        if (n == 0) break;
-        if (wave >= c.wave_limit) {
-            set_status(c, RDF_ERR_WAVE_LIMIT);
-            break;
-        }
-        widest = max(widest, n);
-        if (blockIdx.x == 0 && threadIdx.x == 0) {
-            c.ctl->qcount[(wave + 2) % 3] = 0;       // the counter the next wave appends to
-            c.ctl->cell_count[(wave + 1) & 1] = 0;
-            c.ctl->leaf_count[(wave + 1) & 1] = 0;
-        }
-        // ---- S: every token of this wave, one per thread
-        const Token* q = c.q[wave & 1];
-        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-            run_token(c, sp, wave, load_token(&q[i]), st);
+    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
+    const uint32_t n_leaf = min(c.ctl->leaf_count, c.work_cap);
+    bool alive = true;
+    if (n_leaf) {
+        if (c.use_tc && c.lstm) tc_tiles<TC_LSTM_LEAF>(c, tc, tc_items, 0, n_leaf);
+        else if (c.use_tc) tc_leaf_rows(c, n_leaf);
+        else if (c.lstm) lstm_forward_tiles<3>(c, tile_smem, 0, n_leaf);
+        else rnn_leaf_rows(c, n_leaf);
         __syncthreads();
-        lap(cyc_s);
-        if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+        lap(cyc_c);
+        alive = grid_barrier(c, &c.ctl->bar_ops, generation);
         lap(cyc_b);
-        // every frame of this wave has its id now: the gradient pass walks these ranges
-        if (c.wave_frames && blockIdx.x == 0 && threadIdx.x == 0) c.wave_frames[wave] = ld_volatile_u32(&c.ctl->frame_count);
-        // ---- C: the wave's ready batched operators
-        const uint32_t n_leaf = ld_volatile_u32(&c.ctl->leaf_count[wave & 1]);
-        const uint32_t n_cell = ld_volatile_u32(&c.ctl->cell_count[wave & 1]);
-        if (n_leaf | n_cell) {
-            if (c.use_tc && c.lstm) {
-                if (n_leaf) tc_tiles<TC_LSTM_LEAF>(c, tc, tc_items, 0, min(n_leaf, c.work_cap));
-                if (n_cell) tc_tiles<TC_LSTM_CELL>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
-            } else if (c.use_tc) {
-                if (n_leaf) tc_leaf_rows(c, min(n_leaf, c.work_cap));
-                if (n_cell) tc_tiles<TC_RNN_FWD>(c, tc, tc_items, 0, min(n_cell, c.work_cap));
-            } else if (c.lstm) {
-                if (n_leaf) lstm_forward_tiles<3>(c, tile_smem, min(n_leaf, c.work_cap));
-                if (n_cell) lstm_forward_tiles<5>(c, tile_smem, min(n_cell, c.work_cap));
-            } else {
-                if (n_leaf) rnn_leaf_rows(c, min(n_leaf, c.work_cap));
-                if (n_cell) {
-                    const uint32_t nc = min(n_cell, c.work_cap);
-                    // thin patches while they fit in two rounds over the grid, tiles for wide waves
-                    if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
-                        rnn_cell_thin(c, reinterpret_cast<float*>(&tile_smem), nc);      // 8 x 2H + 128 floats <= 26 KB
-                    else rnn_cell_tiles(c, gsm, nc);
-                }
-            }
-            __syncthreads();
-            lap(cyc_c);
-            if (!grid_barrier(c, &c.ctl->bar, generation)) break;
-            lap(cyc_b);
-        }
+    }
+    uint32_t first = 0;
+    for (uint32_t w = 0; w < n_waves && alive; ++w) {
+        const uint32_t end = min(c.wave_marks[w].y, c.work_cap);
+        if (end <= first) continue;                                  // no cell became ready in this wave
+        const uint32_t nc = end - first;
+        if (c.use_tc && c.lstm) tc_tiles<TC_LSTM_CELL>(c, tc, tc_items, first, nc);
+        else if (c.use_tc) tc_tiles<TC_RNN_FWD>(c, tc, tc_items, first, nc);
+        else if (c.lstm) lstm_forward_tiles<5>(c, tile_smem, first, nc);
+        // thin patches while they fit in two rounds over the grid, tiles for wide waves
+        else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
+            rnn_cell_thin(c, reinterpret_cast<float*>(&tile_smem), first, nc);      // 8 x 2H + 128 floats <= 26 KB
+        else rnn_cell_tiles(c, gsm, first, nc);
+        first = end;
+        __syncthreads();
+        lap(cyc_c);
+        alive = grid_barrier(c, &c.ctl->bar_ops, generation);
+        lap(cyc_b);
     }
     if (c.use_tc) tc_teardown(tc);
-    flush_stats(c, st);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        c.ctl->waves = wave;
-        c.ctl->max_wave_tokens = widest;
-        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[1] = cyc_c; c.ctl->cyc[2] = cyc_b;
+        c.ctl->cyc[1] = cyc_c;
+        c.ctl->cyc[2] += cyc_b;
     }
 }
 
@@ -563,7 +544,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
                                            0x7FFFFFFFll);
     L.qcap = std::max<uint32_t>(L.qcap, (uint32_t)in->B);
     L.frame_cap = g->tag_mode == RDF_TAGS_FRAME ? (uint32_t)(in->B + in->max_invocations) : 0;
-    L.work_cap = g->has_vector_ops ? L.qcap : 0;
+    L.work_cap = g->has_vector_ops ? L.frame_cap : 0;       // the operator lists hold every invocation of the run
     L.ctl = P.take<char>(4096);
     L.code = P.take<VmInstr>(g->code.size());
     L.match = P.take<MatchNode>(std::max<size_t>(1, g->match.size()));
@@ -606,9 +587,9 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
     L.dlog = P.take<float>(gf * 8);
-    // a wave of a tree program holds at least one token of an invocation on its way down or up
-    L.wave_cap = want_grad ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
-    L.wave_frames = P.take<uint32_t>(L.wave_cap);
+    // every wave of a vector program holds at least one token of an invocation on its way down or up
+    L.wave_cap = g->has_vector_ops ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
+    L.wave_marks = P.take<uint4>(L.wave_cap);
     L.all_cells = P.take<uint32_t>(gf);
     L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
     L.leaf_ops = P.take<uint4>(tcl ? gf : 0);
@@ -634,8 +615,10 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaDeviceGetAttribute(&S->clock_khz, cudaDevAttrClockRate, dev));
     if (!coop) return RDF_ERR_CUDA;
     const int max_dyn = tc_smem_bytes(80, 2 * TC_HP_MAX, 48, TC_HP_MAX, 3);       // the largest configuration
-    CUDA_OK(cudaFuncSetAttribute(rdf_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_forward_kernel, 256, max_dyn));
+    CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel, 256, max_dyn));
+    if (per_sm < 1) return RDF_ERR_CUDA;
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 0));
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
     S->device = dev;
@@ -696,7 +679,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.trace = out->trace; c.trace_cap = out->trace ? out->trace_capacity : 0;
     c.dhp = reinterpret_cast<float*>(ws + L.dhp);
     c.dlog = reinterpret_cast<float*>(ws + L.dlog);
-    c.wave_frames = L.wave_cap ? reinterpret_cast<uint32_t*>(ws + L.wave_frames) : nullptr;
+    c.wave_marks = L.wave_cap ? reinterpret_cast<uint4*>(ws + L.wave_marks) : nullptr;
     c.wave_cap = L.wave_cap;
     c.all_cells = reinterpret_cast<uint32_t*>(ws + L.all_cells);
     c.cell_ops = L.use_tc ? reinterpret_cast<uint4*>(ws + L.cell_ops) : nullptr;
@@ -756,12 +739,10 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    if (g->has_vector_ops)
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_kernel, dim3(S->grid), dim3(256), args,
-                                            (size_t)L.tc_smem_fwd, stream));
-    else
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_forward_int_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
     if (g->has_vector_ops) {
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel, dim3(S->grid), dim3(256), args,
+                                            (size_t)L.tc_smem_fwd, stream));
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());
     }

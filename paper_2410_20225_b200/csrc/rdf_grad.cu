@@ -578,7 +578,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
     uint32_t f1 = (uint32_t)c.B;
     for (uint32_t d = 0; d < n_fwd; ++d) {
         const uint32_t f0 = f1;
-        f1 = max(f0, min(c.wave_frames[d], c.frame_cap));
+        f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
         if (f1 == f0) continue;                                      // a wave without calls
         ++wave;
         // ---- A: per-invocation work, a contiguous piece of the range per block, 256 frames per round

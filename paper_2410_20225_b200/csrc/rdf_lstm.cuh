@@ -8,7 +8,7 @@
 __device__ __forceinline__ float sigmoid_f(float x) { return 1.f / (1.f + expf(-x)); }
 
 template <int NG>
-__device__ void lstm_forward_tiles(const DevCtx& c, LstmSmem& sm, uint32_t n_items) {
+__device__ void lstm_forward_tiles(const DevCtx& c, LstmSmem& sm, uint32_t first, uint32_t n_items) {
     constexpr bool CELL = NG == 5;
     const int H = c.H, S = c.S, G = c.G;
     const int Kdim = CELL ? 2 * H : c.D;
@@ -25,7 +25,7 @@ __device__ void lstm_forward_tiles(const DevCtx& c, LstmSmem& sm, uint32_t n_ite
         const float *xl = nullptr, *xr = nullptr;
         if (arow < (int)n_items) {
             if constexpr (CELL) {
-                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[arow]));   // {out, l, r, -}
+                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + arow]));   // {out, l, r, -}
                 xl = c.arena + (size_t)it.y * S;
                 xr = c.arena + (size_t)it.z * S;
             } else {
@@ -90,7 +90,7 @@ __device__ void lstm_forward_tiles(const DevCtx& c, LstmSmem& sm, uint32_t n_ite
                 float hv[4], cv[4], gv[NG][4];
                 uint32_t out;
                 if constexpr (CELL) {
-                    const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));
+                    const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row]));
                     out = it.x;
                     const float4 cl4 = ldcg4(c.arena + (size_t)it.y * S + H + col);
                     const float4 cr4 = ldcg4(c.arena + (size_t)it.z * S + H + col);

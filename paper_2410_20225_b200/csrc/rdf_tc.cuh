@@ -223,7 +223,7 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
                     const uint2 lf = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[row]));   // {slot, tok}
                     it.x = lf.x; it.y = lf.y;
                 } else {
-                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[row]));   // {out, l, r, -}
+                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row]));   // {out, l, r, -}
                 }
                 it.w = 1u;
             }
