@@ -10,6 +10,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <type_traits>
 
 #include "rdf_exec.h"
 #include "rdf_lstm.cuh"
@@ -440,18 +441,16 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
 
 // The operator kernel: the leaves first (they wait for nothing), then, wave by wave, the cells that
 // became ready in that wave; a grid barrier separates the waves (a cell reads states of earlier waves).
-__global__ void __launch_bounds__(256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
-    __shared__ LstmSmem tile_smem;                                   // the TreeRNN tiles use its first part
-    GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
-    extern __shared__ unsigned char dyn_smem[];                      // operand stages of the tensor-core path
-    __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
-    __shared__ uint4 tc_items[TC_M];
+// TC: bf16 operands on the tensor cores (the tile pipeline of rdf_tc.cuh); otherwise fp32 FMA tiles.
+template <bool TC>
+__global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // (the TreeRNN tiles use the first part of LstmSmem)
+    extern __shared__ unsigned char dyn_smem[];                      // TC: resident weight slices + operand stages
     if (c.ctl->forward_status != 0) return;                          // the scheduler failed: the lists are not to be trusted
     TcState tc;
-    if (c.use_tc) {
-        if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Hp / 16, 3, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
-        else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 4, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
+    if constexpr (TC) {
+        if (c.lstm) tc_setup(tc, smem, dyn_smem, c.Hp / 16, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
+        else tc_setup(tc, smem, dyn_smem, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
     }
     uint32_t generation = 0;
     long long cyc_c = 0, cyc_b = 0, t_mark = clock64();
@@ -464,10 +463,13 @@ __global__ void __launch_bounds__(256, 1) rdf_operator_kernel(const __grid_const
     const uint32_t n_leaf = min(c.ctl->leaf_count, c.work_cap);
     bool alive = true;
     if (n_leaf) {
-        if (c.use_tc && c.lstm) tc_tiles<TC_LSTM_LEAF>(c, tc, tc_items, 0, n_leaf);
-        else if (c.use_tc) tc_leaf_rows(c, n_leaf);
-        else if (c.lstm) lstm_forward_tiles<3>(c, tile_smem, 0, n_leaf);
-        else rnn_leaf_rows(c, n_leaf);
+        if constexpr (TC) {
+            if (c.lstm) tc_pipe<TC_LSTM_LEAF, TC_STAGES_LSTM_FWD>(c, tc, smem, 0, n_leaf);
+            else tc_leaf_rows(c, n_leaf);
+        } else {
+            if (c.lstm) lstm_forward_tiles<3>(c, smem, 0, n_leaf);
+            else rnn_leaf_rows(c, n_leaf);
+        }
         __syncthreads();
         lap(cyc_c);
         alive = grid_barrier(c, &c.ctl->bar_ops, generation);
@@ -478,20 +480,23 @@ __global__ void __launch_bounds__(256, 1) rdf_operator_kernel(const __grid_const
         const uint32_t end = min(c.wave_marks[w].y, c.work_cap);
         if (end <= first) continue;                                  // no cell became ready in this wave
         const uint32_t nc = end - first;
-        if (c.use_tc && c.lstm) tc_tiles<TC_LSTM_CELL>(c, tc, tc_items, first, nc);
-        else if (c.use_tc) tc_tiles<TC_RNN_FWD>(c, tc, tc_items, first, nc);
-        else if (c.lstm) lstm_forward_tiles<5>(c, tile_smem, first, nc);
-        // thin patches while they fit in two rounds over the grid, tiles for wide waves
-        else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
-            rnn_cell_thin(c, reinterpret_cast<float*>(&tile_smem), first, nc);      // 8 x 2H + 128 floats <= 26 KB
-        else rnn_cell_tiles(c, gsm, first, nc);
+        if constexpr (TC) {
+            if (c.lstm) tc_pipe<TC_LSTM_CELL, TC_STAGES_LSTM_FWD>(c, tc, smem, first, nc);
+            else tc_pipe<TC_RNN_FWD, TC_STAGES_RNN_FWD>(c, tc, smem, first, nc);
+        } else {
+            if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
+            // thin patches while they fit in two rounds over the grid, tiles for wide waves
+            else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
+                rnn_cell_thin(c, reinterpret_cast<float*>(&smem), first, nc);      // 8 x 2H + 128 floats <= 26 KB
+            else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
+        }
         first = end;
         __syncthreads();
         lap(cyc_c);
         alive = grid_barrier(c, &c.ctl->bar_ops, generation);
         lap(cyc_b);
     }
-    if (c.use_tc) tc_teardown(tc);
+    if constexpr (TC) tc_teardown(tc);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->cyc[1] = cyc_c;
         c.ctl->cyc[2] += cyc_b;
@@ -581,8 +586,8 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.wxtp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
     L.dg_bf = P.take<__nv_bfloat16>(tcl && want_grad ? vf * 5 * L.Hp : 0);
-    L.tc_smem_fwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(80, 2 * L.Hp, 48, L.Hp, 3) : tc_smem_bytes(L.Hp / 4, 2 * L.Hp, 0, 0, 4);
-    L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(32, 5 * L.Hp, 0, 0, 4) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, 4);
+    L.tc_smem_fwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(80, 2 * L.Hp, 48, L.Hp, TC_STAGES_LSTM_FWD) : tc_smem_bytes(L.Hp / 4, 2 * L.Hp, 0, 0, TC_STAGES_RNN_FWD);
+    L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(32, 5 * L.Hp, 0, 0, TC_STAGES_LSTM_BWD) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, TC_STAGES_RNN_BWD);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(gf * S);
@@ -614,9 +619,12 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     CUDA_OK(cudaDeviceGetAttribute(&S->clock_khz, cudaDevAttrClockRate, dev));
     if (!coop) return RDF_ERR_CUDA;
-    const int max_dyn = tc_smem_bytes(80, 2 * TC_HP_MAX, 48, TC_HP_MAX, 3);       // the largest configuration
-    CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel, 256, max_dyn));
+    const int max_dyn = std::max(tc_smem_bytes(80, 2 * TC_HP_MAX, 48, TC_HP_MAX, TC_STAGES_LSTM_FWD),
+                                 tc_smem_bytes(TC_HP_MAX / 4, 2 * TC_HP_MAX, 0, 0, TC_STAGES_RNN_FWD));   // the largest configurations
+    CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<true>, TC_THREADS, max_dyn));
+    if (per_sm < 1) return RDF_ERR_CUDA;
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 0));
     if (per_sm < 1) return RDF_ERR_CUDA;
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 0));
     if (per_sm < 1) return RDF_ERR_CUDA;
@@ -741,8 +749,11 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     void* args[] = {(void*)&c};
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
     if (g->has_vector_ops) {
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel, dim3(S->grid), dim3(256), args,
-                                            (size_t)L.tc_smem_fwd, stream));
+        if (c.use_tc)
+            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
+                                                (size_t)L.tc_smem_fwd, stream));
+        else
+            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), args, 0, stream));
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());
     }

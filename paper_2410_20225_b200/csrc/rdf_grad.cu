@@ -9,6 +9,7 @@
 // retained per-invocation values.
 #include <algorithm>
 #include <cstring>
+#include <type_traits>
 
 #include "rdf_exec.h"
 #include "rdf_tc.cuh"
@@ -228,11 +229,11 @@ __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int
 }
 
 // ----------------------------------------------------------- backward waves
-// The cells (and, for the TreeLSTM, the leaves) among the up to 256 frames [base, end) of this block
+// The cells (and, for the TreeLSTM, the leaves) among the up to blockDim.x frames [base, end) of this block
 // are appended to the global lists with one atomic per list.  The cells of a wave, in list order, are
 // the rows of the wave's operand-gradient contraction.  Called by every thread of the block.
 struct FrameLists {
-    uint32_t wcnt[2][8], gbase[2];
+    uint32_t wcnt[2][16], gbase[2];          // up to 16 warps per block
 };
 
 __device__ __forceinline__ void backward_list_frames(const DevCtx& c, FrameLists& fl, uint32_t base, uint32_t end) {
@@ -253,7 +254,7 @@ __device__ __forceinline__ void backward_list_frames(const DevCtx& c, FrameLists
     __syncthreads();
     if (threadIdx.x < 2) {
         uint32_t tot = 0;
-        for (int w = 0; w < 8; ++w) tot += fl.wcnt[threadIdx.x][w];
+        for (int w = 0; w < (int)(blockDim.x / 32); ++w) tot += fl.wcnt[threadIdx.x][w];
         fl.gbase[threadIdx.x] = tot ? atomicAdd(threadIdx.x ? &c.ctl->all_leaves : &c.ctl->all_cells, tot) : 0u;
     }
     __syncthreads();
@@ -549,22 +550,18 @@ __device__ void backward_operand_thin(const DevCtx& c, float* zs, uint32_t first
     }
 }
 
-__global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
-    __shared__ LstmSmem tile_smem;                                   // tiles use its first part; thin patches stage rows in it
-    GemmSmem& gsm = *reinterpret_cast<GemmSmem*>(&tile_smem);
+template <bool TC>
+__global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // fp32: tiles use the first part; thin patches stage rows in it
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
-    __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
-    __shared__ uint4 tc_items[TC_M];
     __shared__ FrameLists lists;
     if (c.ctl->forward_status != 0) return;                          // the forward pass failed: nothing to differentiate
     TcState tc;
-    const bool tc_on = c.use_tc;
-    if (tc_on) {
-        if (c.lstm) tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 2 * c.Hp / 32, 4, c.WTp, 5 * c.Hp, 32);
-        else tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, 8, 4, c.WTp, c.Hp, c.Hp / 4);
+    if constexpr (TC) {
+        if (c.lstm) tc_setup(tc, smem, dyn_smem, 2 * c.Hp / 32, c.WTp, 5 * c.Hp, 32);
+        else tc_setup(tc, smem, dyn_smem, 8, c.WTp, c.Hp, c.Hp / 4);
     }
-    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32;
+    const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, n_warps = blockDim.x / 32;
     uint32_t generation = 0, wave = 0, first = 0;
     long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
@@ -581,18 +578,18 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
         if (f1 == f0) continue;                                      // a wave without calls
         ++wave;
-        // ---- A: per-invocation work, a contiguous piece of the range per block, 256 frames per round
+        // ---- A: per-invocation work, a contiguous piece of the range per block, one frame per thread and round
         const uint32_t n = f1 - f0;
         const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
         const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
         const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
-        for (uint32_t base = c0; base < c1; base += 256) {
-            const uint32_t end = min(c1, base + 256);
+        for (uint32_t base = c0; base < c1; base += blockDim.x) {
+            const uint32_t end = min(c1, base + blockDim.x);
             if (c.lstm) {
-                for (uint32_t t = base + wib; t < end; t += 8) lstm_backward_frame(c, t, lane);
+                for (uint32_t t = base + wib; t < end; t += n_warps) lstm_backward_frame(c, t, lane);
             } else {
-                for (uint32_t t = base + wib * 4 + lane / 8; t < end; t += 32) {
-                    if (tc_on) backward_frame_tc(c, t, lane % 8);
+                for (uint32_t t = base + wib * 4 + lane / 8; t < end; t += 4 * n_warps) {
+                    if constexpr (TC) backward_frame_tc(c, t, lane % 8);
                     else backward_frame_f32(c, t, lane % 8);
                 }
             }
@@ -605,12 +602,15 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
         const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
         if (end > first) {
-            if (tc_on && c.lstm) tc_tiles<TC_LSTM_BWD>(c, tc, tc_items, first, end - first);
-            else if (tc_on) tc_tiles<TC_RNN_BWD>(c, tc, tc_items, first, end - first);
-            else if (c.lstm) backward_operand_tiles(c, gsm, first, end - first, c.gates, c.G, 5 * c.H);
-            else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
-                backward_operand_thin(c, reinterpret_cast<float*>(&tile_smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
-            else backward_operand_tiles(c, gsm, first, end - first, c.dhp, c.H, c.H);
+            if constexpr (TC) {
+                if (c.lstm) tc_pipe<TC_LSTM_BWD, TC_STAGES_LSTM_BWD>(c, tc, smem, first, end - first);
+                else tc_pipe<TC_RNN_BWD, TC_STAGES_RNN_BWD>(c, tc, smem, first, end - first);
+            } else {
+                if (c.lstm) backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.gates, c.G, 5 * c.H);
+                else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
+                    backward_operand_thin(c, reinterpret_cast<float*>(&smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
+                else backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.dhp, c.H, c.H);
+            }
             first = end;
             __syncthreads();
             lap(cyc_c);
@@ -618,7 +618,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_kernel(const __grid_const
             lap(cyc_b);
         }
     }
-    if (tc_on) tc_teardown(tc);
+    if constexpr (TC) tc_teardown(tc);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->waves_backward = wave;
         c.ctl->cyc[3] = cyc_a; c.ctl->cyc[4] = cyc_c; c.ctl->cyc[5] = cyc_b;
@@ -830,9 +830,13 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     // gradient waves
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
-    if (c.use_tc) CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel, dim3(S->grid), dim3(256), args,
-                                        c.use_tc ? (size_t)L.tc_smem_bwd : 0, stream));
+    if (c.use_tc) {
+        CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
+                                            (size_t)L.tc_smem_bwd, stream));
+    } else {
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args, 0, stream));
+    }
     rdf_mark(S, 4, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
@@ -877,9 +881,9 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     rdf_mark(S, 6, stream);
     rdf_mark(S, 7, stream);       // (dW_s and db_s come from the loss-head pass)
     if (tc_lstm) {
-        const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 4);
+        const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 5);
         CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));
-        rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, 256, de_smem, stream>>>(c);
+        rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, TC_THREADS, de_smem, stream>>>(c);
     } else if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
     // (TreeRNN: the leaves added their dh to dE during the gradient waves)
     rdf_mark(S, 8, stream);

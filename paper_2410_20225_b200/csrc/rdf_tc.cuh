@@ -1,18 +1,21 @@
 // Tensor-core path (sm_100a: tcgen05 + tensor memory) for the dense
-// contractions of the bf16 TreeRNN workloads, forward and operand-gradient:
+// contractions of the bf16 workloads, forward and operand-gradient:
 //
 //   forward :  D[128 cells x NS] = A[128 x 2Hp] * Wp [NS x 2Hp]^T     A row = [h_l ; h_r] (bf16 states, gathered)
 //   backward:  D[128 cells x NS] = A[128 x  Hp] * WTp[NS x  Hp]^T     A row = dz (bf16),  D = slice of [dh_l ; dh_r]
 //
-// Weight-stationary: the packed weight matrix is split along N into slices of
-// NS = Hp / 4 rows; a thread block owns one slice for the whole kernel and
-// keeps it in shared memory (loaded once, <= 100 KB), so per tile only the
-// gathered operand rows move.  A rows are streamed with cp.async through a
-// 4-stage ring of 128-byte-swizzled [128 x 64] bf16 tiles (8-row groups of
-// 1024 bytes, 16-byte chunks XOR-ed with the row index: the K-major layout the
-// MMA reads); one thread issues the tcgen05.mma instructions, tcgen05.commit
-// signals an mbarrier per stage, accumulators live in tensor memory and the
-// epilogue reads them back with tcgen05.ld.  Every wait is bounded.
+// Weight-stationary: the packed weight matrix is split along N into slices; a
+// thread block owns one slice for the whole kernel and keeps it in shared
+// memory (loaded once, <= 130 KB), so per tile only the gathered operand rows
+// move.  The tile loop is a pipeline of three roles inside the 416-thread block:
+//   producers (4 warps): gather the operand rows with cp.async into a ring of 128-byte-swizzled
+//       [128 x 64] bf16 stages (8-row groups of 1024 bytes, 16-byte chunks XOR-ed with the row index:
+//       the K-major layout the MMA reads), several stages ahead and across tile boundaries;
+//   MMA issuer (1 thread): tcgen05.mma per stage into one of two accumulator buffers in tensor
+//       memory; tcgen05.commit frees the stage and, after a tile's last stage, publishes the buffer;
+//   epilogue (8 warps): tcgen05.ld of a finished buffer, bias / activations, stores -- while the
+//       MMAs of the next tile fill the other buffer.
+// The roles meet only through mbarriers, and every wait is bounded.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -20,14 +23,19 @@
 
 static const int TC_M = 128;                 // cells per tile (TMEM lanes)
 static const int TC_KC = 64;                 // bf16 elements per staged K chunk = one 128-byte swizzled row
-static const int TC_MAX_STAGES = 4;
+static const int TC_MAX_STAGES = 8;
 static const int TC_A_STAGE = TC_M * 128;    // 16 KB
 static const int TC_HP_MAX = 320;            // widest padded hidden size the resident slices are sized for
-static const int TC_TMEM_COLS = 128;
+static const int TC_ACC_COLS = 128;          // TMEM columns per accumulator buffer
+static const int TC_TMEM_COLS = 2 * TC_ACC_COLS;
+static const int TC_THREADS = 416;           // warps 0-7 epilogue, warp 8 MMA issuer, warps 9-12 producers
+static const int TC_EPI_THREADS = 256, TC_MMA_WARP = 8, TC_PROD_WARP0 = 9, TC_PRODUCERS = 128;
+// ring depth per kernel: what is left of the shared memory beside the resident weight slices
+static const int TC_STAGES_RNN_FWD = 7, TC_STAGES_LSTM_FWD = 5, TC_STAGES_RNN_BWD = 8, TC_STAGES_LSTM_BWD = 7;
 
-// tile loops (template parameter of tc_tiles)
+// tile loops (template parameter of tc_pipe)
 enum TcMode {
-    TC_RNN_FWD = 0,     // A = [h_l ; h_r] (bf16 states), B = Wp slice;           epilogue: tanh, both arenas
+    TC_RNN_FWD = 0,     // A = [h_l ; h_r] (bf16 states), B = Wp slice;           epilogue: tanh, bf16 state
     TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: operand gradients
     TC_LSTM_CELL = 2,   // A = [h_l ; h_r],                B = W5p slice (5 gates x 16 units); epilogue: gates, c, h
     TC_LSTM_LEAF = 3,   // A = E_bf[tok],                  B = Wxp slice (3 gates x 16 units); epilogue: gates, c, h
@@ -35,12 +43,21 @@ enum TcMode {
     TC_LSTM_DE = 5      // A = leaf gate gradients (3 Hp), B = WxTp slice;         epilogue: dE[tok] += W_x^T dg
 };
 
+// mbarriers and tile records of the pipeline (static shared memory of the kernel)
+struct __align__(16) TcShared {
+    uint4    items[2][TC_M];                 // per accumulator buffer: {frame, left, right / token, valid} of the tile's rows
+    uint64_t full[TC_MAX_STAGES];            // stage filled (all producer threads arrived)
+    uint64_t empty[TC_MAX_STAGES];           // stage consumed (tcgen05.commit)
+    uint64_t acc_full[2], acc_empty[2];      // accumulator buffer complete / read out by the epilogue
+    uint64_t items_full[2];                  // tile records written
+    uint32_t tmem_slot;
+};
+
 struct TcState {
     uint32_t tmem_base;      // TMEM address returned by tcgen05.alloc
     uint32_t a_addr;         // shared-space address of A stage 0
-    uint32_t mbar_addr;      // shared-space address of the per-stage mbarriers
-    uint32_t iter;           // K chunks issued so far (stage = iter % stages)
-    uint32_t stages;         // depth of the A ring (3 or 4)
+    uint32_t g;              // K chunks that went through the ring so far (stage = g % stages)
+    uint32_t T;              // tiles this block has run so far (accumulator buffer = T % 2)
     int      n_split;        // N slices = blocks per row group
     // up to two resident weight slices (the TreeLSTM forward keeps the cell and the leaf weights)
     uint32_t b_addr[2];
@@ -121,16 +138,32 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool v
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// the same with a run-time count (the instruction takes an immediate)
+__device__ __forceinline__ void cp_async_wait_upto(uint32_t n) {
+    switch (n) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        default: cp_async_wait<6>(); break;
+    }
+}
 
 // byte offset of 16-byte chunk c16 of row r inside a swizzled [rows x 128 bytes] operand tile
 __device__ __forceinline__ uint32_t swz(int r, int c16) {
     return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t addr) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+
 // One-time set-up per kernel (all threads call it): TMEM allocation by warp 0, mbarriers, and the
 // block's resident slices of the packed weights: rows [slice * ns, +ns) of B[. x K], chunk by chunk.
-__device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, uint32_t* tmem_slot, uint64_t* mbars,
-                                         int n_split, int stages, const __nv_bfloat16* B0, int K0, int ns0,
+__device__ __forceinline__ void tc_setup(TcState& tc, TcShared& sh, unsigned char* dyn_smem, int n_split,
+                                         const __nv_bfloat16* B0, int K0, int ns0,
                                          const __nv_bfloat16* B1 = nullptr, int K1 = 0, int ns1 = 0) {
     const uint32_t raw = smem_u32(dyn_smem);
     const uint32_t aligned = (raw + 1023u) & ~1023u;
@@ -141,16 +174,23 @@ __device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, u
     tc.a_addr = aligned + bytes0 + bytes1;
     tc.ns[0] = ns0; tc.ns[1] = ns1;
     tc.n_chunks[0] = K0 / TC_KC; tc.n_chunks[1] = B1 ? K1 / TC_KC : 0;
-    tc.mbar_addr = smem_u32(mbars);
-    tc.iter = 0;
-    tc.stages = stages;
+    tc.g = 0;
+    tc.T = 0;
     tc.n_split = n_split;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_MAX_STAGES; ++s) mbar_init(tc.mbar_addr + 8 * s, 1);
+        for (int s = 0; s < TC_MAX_STAGES; ++s) {
+            mbar_init(smem_u32(&sh.full[s]), TC_PRODUCERS);
+            mbar_init(smem_u32(&sh.empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh.acc_full[b]), 1);
+            mbar_init(smem_u32(&sh.acc_empty[b]), TC_EPI_THREADS);
+            mbar_init(smem_u32(&sh.items_full[b]), TC_PRODUCERS);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < 32) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_slot)), "n"(TC_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const int slice = blockIdx.x % n_split;
@@ -169,7 +209,7 @@ __device__ __forceinline__ void tc_setup(TcState& tc, unsigned char* dyn_smem, u
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    tc.tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+    tc.tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_slot);
 }
 
 __device__ __forceinline__ void tc_teardown(const TcState& tc) {
@@ -192,94 +232,133 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8]) {
 
 __device__ __forceinline__ float tc_sigmoid(float x) { return 1.f / (1.f + expf(-x)); }
 
-// One 128-row tile loop over n_items ready operators (see TcMode).  Rows come from cell_items /
-// leaf_items (forward modes) or from all_cells[first ..] (gradient modes).
-// s_items: 128 x uint4 of shared memory for the tile's records {frame, left, right / token, valid}.
-template <int MODE>
-__device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t first, uint32_t n_items) {
+// The tile loop over n_items ready operators (see TcMode), 128 rows per tile.  Rows come from
+// cell_items / leaf_items (forward modes) or from cell_ops / leaf_ops at [first ..] (gradient modes).
+// Called by all TC_THREADS threads of the block; returns when every tile has been written out.
+template <int MODE, int STAGES>
+__device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t first, uint32_t n_items) {
+    static_assert(STAGES >= 3 && STAGES <= TC_MAX_STAGES, "ring depth");
     constexpr int RGN = MODE == TC_LSTM_LEAF ? 1 : 0;
-    constexpr bool GRAD = MODE == TC_RNN_BWD || MODE == TC_LSTM_BWD;
+    constexpr int D = STAGES - 2;                              // chunks a producer thread keeps in flight
     const int H = c.H, Hp = c.Hp, S = c.S, ns = tc.ns[RGN], n_chunks = tc.n_chunks[RGN];
-    const uint32_t stages = tc.stages;
     const int slice = blockIdx.x % tc.n_split, rg = blockIdx.x / tc.n_split, n_rg = gridDim.x / tc.n_split;
-    if (rg >= n_rg) return;                                    // blocks beyond the last full group sit this out
-    const uint32_t idesc = tc_idesc(ns);
     const int tiles = (n_items + TC_M - 1) / TC_M;
-    const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? c.dg_bf
-                                 : MODE == TC_LSTM_LEAF ? c.E_bf : c.arena_bf;
+    // blocks beyond the last full group of slices have no tiles
+    const int my_tiles = rg < n_rg && tiles > rg ? (tiles - rg + n_rg - 1) / n_rg : 0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(&sh.full[0]), empty0 = smem_u32(&sh.empty[0]);
+    const uint32_t acc_full0 = smem_u32(&sh.acc_full[0]), acc_empty0 = smem_u32(&sh.acc_empty[0]);
+    const uint32_t items_full0 = smem_u32(&sh.items_full[0]);
     bool ok = true;
-    for (int tile = rg; tile < tiles && ok; tile += n_rg) {
-        const int row0 = tile * TC_M;
-        if (threadIdx.x < TC_M) {
+    if (warp >= TC_PROD_WARP0) {
+        // ------------------------------------------------------------ producers
+        const int p = threadIdx.x - TC_PROD_WARP0 * 32, r8 = p >> 3, c16 = p & 7;
+        const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? c.dg_bf
+                                     : MODE == TC_LSTM_LEAF ? c.E_bf : c.arena_bf;
+        auto load_item = [&](int tile) {                     // the record of row p of the tile
             uint4 it = make_uint4(0u, 0u, 0u, 0u);
-            const int row = row0 + threadIdx.x;
-            if (row < (int)n_items) {
-                if (MODE == TC_LSTM_DE) {
-                    it = c.leaf_ops[first + row];                                    // {leaf frame, token id, -, 1}
-                } else if (GRAD) {
-                    const uint32_t t = __ldcg(&c.all_cells[first + row]);
-                    it.x = t; it.y = __ldcg(&c.op_l[t]); it.z = __ldcg(&c.op_r[t]);
-                } else if (MODE == TC_LSTM_LEAF) {
-                    const uint2 lf = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[row]));   // {slot, tok}
+            const uint32_t row = (uint32_t)tile * TC_M + p;
+            if (row < n_items) {
+                if (MODE == TC_LSTM_DE) it = __ldcg(&c.leaf_ops[first + row]);                   // {leaf frame, token id, -, 1}
+                else if (MODE == TC_RNN_BWD || MODE == TC_LSTM_BWD) it = __ldcg(&c.cell_ops[first + row]);   // {cell, left, right, 1}
+                else if (MODE == TC_LSTM_LEAF) {
+                    const uint2 lf = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[first + row]));     // {slot, tok}
                     it.x = lf.x; it.y = lf.y;
-                } else {
-                    it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row]));   // {out, l, r, -}
-                }
+                } else it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row]));  // {out, l, r, -}
                 it.w = 1u;
             }
-            s_items[threadIdx.x] = it;
-        }
-        __syncthreads();
-        const uint32_t it0 = tc.iter;
-        auto issue = [&](int kc) {
-            const uint32_t g = it0 + kc, s = g % stages;
-            // the MMAs that last read this stage must have completed
-            if (g >= stages) ok = mbar_wait(c, tc.mbar_addr + 8 * s, ((g / stages) - 1) & 1u) && ok;
-            const int koff = kc * TC_KC;
-            for (int p = threadIdx.x; p < TC_M * 8; p += blockDim.x) {
-                const int r = p >> 3, c16 = p & 7;
-                const uint4 it = s_items[r];
-                size_t src;
-                if (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL)
-                    src = (size_t)(koff < Hp ? it.y : it.z) * Hp + (koff < Hp ? koff : koff - Hp) + c16 * 8;
-                else if (MODE == TC_RNN_BWD) src = (size_t)it.x * Hp + koff + c16 * 8;
-                else if (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) src = (size_t)it.x * 5 * Hp + koff + c16 * 8;
-                else src = (size_t)it.y * Hp + koff + c16 * 8;                       // leaf: E_bf[tok]
-                cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r, c16), Arows + src, it.w != 0u);
-            }
-            cp_async_commit();
+            return it;
         };
-        issue(0);
-        if (n_chunks > 1) issue(1); else cp_async_commit();
-        for (int kc = 0; kc < n_chunks; ++kc) {
-            // with a ring of 3 the stage of chunk kc + 2 is the one chunk kc - 1 used: its MMAs were
-            // committed one step ago, issue() waits for them
-            if (kc + 2 < n_chunks) issue(kc + 2); else cp_async_commit();
-            cp_async_wait<2>();                                          // this thread's copies of chunk kc have landed
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> async-proxy reads
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t s = (it0 + kc) % stages;
-                const uint32_t a = tc.a_addr + s * TC_A_STAGE, b = tc.b_addr[RGN] + kc * ns * 128;
+        uint4 it_next = my_tiles ? load_item(rg) : make_uint4(0u, 0u, 0u, 0u);
+        // chunks this thread has issued in this call, and how many of them it has reported as landed
+        uint32_t issued = 0, arrived = 0;
+        // Waits until at most `limit` of this thread's chunks are still in flight and reports the others.
+        // (Writer side of the hand-over: own copies complete, proxy fence, arrive.)
+        auto report = [&](uint32_t limit) {
+            if (issued - arrived <= limit) return;
+            cp_async_wait_upto(limit);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async-proxy reads
+            while (issued - arrived > limit) {
+                mbar_arrive(full0 + 8 * ((tc.g + arrived) % STAGES));
+                ++arrived;
+            }
+        };
+        for (int i = 0; i < my_tiles && ok; ++i) {
+            const uint32_t T = tc.T + i, b = T & 1u;
+            // The epilogue of the tile before last must have finished with this record buffer.  It can
+            // only finish once all chunks of that tile are reported: at most one tile's worth may be open.
+            if (T >= 2) {
+                report(min((uint32_t)D, (uint32_t)n_chunks));
+                ok = mbar_wait(c, acc_empty0 + 8 * b, ((T >> 1) - 1) & 1u);
+            }
+            sh.items[b][p] = it_next;
+            mbar_arrive(items_full0 + 8 * b);
+            if (i + 1 < my_tiles) it_next = load_item(rg + (i + 1) * n_rg);      // in flight during this tile
+            ok = mbar_wait(c, items_full0 + 8 * b, (T >> 1) & 1u) && ok;
+            // the eight rows this thread copies: r8 + 16 q
+            uint32_t src0[8], src1[8], valid = 0;
 #pragma unroll
-                for (int ks = 0; ks < TC_KC / 16; ++ks)
-                    tc_mma(tc.tmem_base, tc_desc(a + ks * 32), tc_desc(b + ks * 32), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(tc.mbar_addr + 8 * s);
+            for (int q = 0; q < 8; ++q) {
+                const uint4 it = sh.items[b][r8 + 16 * q];
+                if (it.w) valid |= 1u << q;
+                if (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL) { src0[q] = it.y; src1[q] = it.z; }
+                else if (MODE == TC_LSTM_LEAF) { src0[q] = it.y; src1[q] = it.y; }
+                else { src0[q] = it.x; src1[q] = it.x; }
+            }
+            const size_t lda = (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? (size_t)5 * Hp : (size_t)Hp;
+            for (int kc = 0; kc < n_chunks && ok; ++kc) {
+                const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
+                // the MMAs that last read this stage must have completed
+                if (g >= (uint32_t)STAGES) ok = mbar_wait(c, empty0 + 8 * s, ((g / STAGES) - 1) & 1u);
+                const int koff = kc * TC_KC;
+                const bool second = (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL) && koff >= Hp;
+                const size_t col = (size_t)(second ? koff - Hp : koff) + c16 * 8;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r8 + 16 * q, c16),
+                               Arows + (size_t)(second ? src1[q] : src0[q]) * lda + col, (valid >> q) & 1u);
+                cp_async_commit();
+                ++issued;
+                report(D);                                     // D chunks stay in flight
             }
         }
-        tc.iter = it0 + n_chunks;
-        // accumulators are complete when the last commit has arrived
-        {
-            const uint32_t g = tc.iter - 1;
-            if (ok) ok = mbar_wait(c, tc.mbar_addr + 8 * (g % stages), (g / stages) & 1u);
+        report(0);                                             // drain
+    } else if (warp == TC_MMA_WARP) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = tc_idesc(ns);
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const uint32_t T = tc.T + i, b = T & 1u;
+                // the epilogue has read the previous contents of this accumulator buffer
+                if (T >= 2) ok = mbar_wait(c, acc_empty0 + 8 * b, ((T >> 1) - 1) & 1u);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int kc = 0; kc < n_chunks && ok; ++kc) {
+                    const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
+                    ok = mbar_wait(c, full0 + 8 * s, (g / STAGES) & 1u);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a = tc.a_addr + s * TC_A_STAGE, bw = tc.b_addr[RGN] + kc * ns * 128;
+#pragma unroll
+                    for (int ks = 0; ks < TC_KC / 16; ++ks)
+                        tc_mma(tc.tmem_base + b * TC_ACC_COLS, tc_desc(a + ks * 32), tc_desc(bw + ks * 32), idesc,
+                               (kc > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(empty0 + 8 * s);                 // the stage is free when these MMAs have read it
+                }
+                if (ok) tc_commit(acc_full0 + 8 * b);          // the accumulators are complete when all MMAs so far are
+            }
         }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue
+        for (int i = 0; i < my_tiles && ok; ++i) {
+            const uint32_t T = tc.T + i, b = T & 1u;
+            ok = mbar_wait(c, items_full0 + 8 * b, (T >> 1) & 1u);
+            ok = ok && mbar_wait(c, acc_full0 + 8 * b, (T >> 1) & 1u);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int row = (warp & 3) * 32 + lane;                       // warp w reads TMEM lanes 32 (w % 4) ..
-            const uint32_t lane_base = tc.tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-            const uint4 it = s_items[row];
+            const uint32_t lane_base = tc.tmem_base + (uint32_t)(b * TC_ACC_COLS) + ((uint32_t)((warp & 3) * 32) << 16);
+            const uint4 it = sh.items[b][row];
             const bool live = it.w != 0u;
             if (MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) {
                 // slice = 16 hidden units, columns gate * 16 + unit; warps 0-3 take units 0-7, warps 4-7 units 8-15
@@ -384,11 +463,15 @@ __device__ void tc_tiles(const DevCtx& c, TcState& tc, uint4* s_items, uint32_t 
                     }
                 }
             }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(acc_empty0 + 8 * b);                   // buffer and records may be reused
         }
-        // TMEM, the stages and s_items may be overwritten by the next tile only after everybody has read them
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
     }
+    tc.g += (uint32_t)(my_tiles * n_chunks);
+    tc.T += (uint32_t)my_tiles;
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
 // Leaves in bf16 mode: state(slot) = bf16(E[tok]), pad columns of the row zero.  Each warp takes four
@@ -469,14 +552,12 @@ static __global__ void __launch_bounds__(256) rdf_pack_lstm_kernel(const DevCtx 
 }
 
 // dE of the TreeLSTM on tensor cores: one launch after the gradient waves, blocks = (row group, 64-column slice of D)
-static __global__ void __launch_bounds__(256, 1) rdf_de_tc_kernel(const DevCtx c) {
+static __global__ void __launch_bounds__(TC_THREADS, 1) rdf_de_tc_kernel(const DevCtx c) {
     extern __shared__ unsigned char dyn_smem[];
-    __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t tc_mbars[TC_MAX_STAGES];
-    __shared__ uint4 tc_items[TC_M];
+    __shared__ TcShared sh;
     TcState tc;
-    tc_setup(tc, dyn_smem, &tmem_slot, tc_mbars, c.Hp / 64, 4, c.WxTp, 3 * c.Hp, 64);
-    tc_tiles<TC_LSTM_DE>(c, tc, tc_items, 0, c.ctl->all_leaves);
+    tc_setup(tc, sh, dyn_smem, c.Hp / 64, c.WxTp, 3 * c.Hp, 64);
+    tc_pipe<TC_LSTM_DE, 5>(c, tc, sh, 0, c.ctl->all_leaves);
     tc_teardown(tc);
 }
 
