@@ -595,6 +595,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     // every wave of a vector program holds at least one token of an invocation on its way down or up
     L.wave_cap = g->has_vector_ops ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
     L.wave_marks = P.take<uint4>(L.wave_cap);
+    L.list_seg = P.take<uint2>(want_grad ? (size_t)in->max_invocations / 2048 + 2 : 0);
     L.all_cells = P.take<uint32_t>(gf);
     L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
     L.leaf_ops = P.take<uint4>(tcl ? gf : 0);

@@ -229,144 +229,240 @@ __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int
 }
 
 // ----------------------------------------------------------- backward waves
-// The cells (and, for the TreeLSTM, the leaves) among the up to blockDim.x frames [base, end) of this block
-// are appended to the global lists with one atomic per list.  The cells of a wave, in list order, are
-// the rows of the wave's operand-gradient contraction.  Called by every thread of the block.
-struct FrameLists {
-    uint32_t wcnt[2][16], gbase[2];          // up to 16 warps per block
-};
+// Lists of the gradient pass, formed once before the waves.  Frame ids are handed out in wave order,
+// so listing the cells in frame order puts the cells of every gradient wave next to each other:
+// wave d owns all_cells[marks[d-1].w, marks[d].w), the rows of its operand-gradient contraction.
+// Three small kernels: per-segment counts, scan of the counts, fill (and the per-wave ends).
+static const int LIST_SEG = 2048;            // frames per segment (256 threads x 8)
 
-__device__ __forceinline__ void backward_list_frames(const DevCtx& c, FrameLists& fl, uint32_t base, uint32_t end) {
-    const uint32_t t = base + threadIdx.x;
-    const bool valid = t < end;
-    uint32_t l = LEAF_MARK, r = 0;
-    if (valid) {
-        l = __ldcg(&c.op_l[t]);
-        r = __ldcg(&c.op_r[t]);
-    }
-    const bool cell = valid && l != LEAF_MARK, leaf = valid && l == LEAF_MARK && c.lstm;
-    const uint32_t mc = __ballot_sync(0xffffffffu, cell), ml = __ballot_sync(0xffffffffu, leaf);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) {
-        fl.wcnt[0][warp] = __popc(mc);
-        fl.wcnt[1][warp] = __popc(ml);
-    }
-    __syncthreads();
-    if (threadIdx.x < 2) {
-        uint32_t tot = 0;
-        for (int w = 0; w < (int)(blockDim.x / 32); ++w) tot += fl.wcnt[threadIdx.x][w];
-        fl.gbase[threadIdx.x] = tot ? atomicAdd(threadIdx.x ? &c.ctl->all_leaves : &c.ctl->all_cells, tot) : 0u;
-    }
-    __syncthreads();
-    uint32_t pre_c = fl.gbase[0], pre_l = fl.gbase[1];
-    for (int w = 0; w < warp; ++w) {
-        pre_c += fl.wcnt[0][w];
-        pre_l += fl.wcnt[1][w];
-    }
-    const uint32_t below = (1u << lane) - 1u;
-    if (cell) {
-        const uint32_t idx = pre_c + __popc(mc & below);
-        c.all_cells[idx] = t;
-        if (c.cell_ops) c.cell_ops[idx] = make_uint4(t, l, r, 1u);
-    }
-    if (leaf) {
-        const uint32_t idx = pre_l + __popc(ml & below);
-        c.all_leaves[idx] = t;
-        if (c.leaf_ops) c.leaf_ops[idx] = make_uint4(t, r, 0u, 1u);       // r = token id of a leaf
-    }
-    __syncthreads();                                   // fl is reused by the next round
-}
-
-// A (bf16 TreeRNN), one invocation t per 8 lanes: dh = (gradient from the caller) + W_s^T dlog;
-//    cell: dz = dh * (1 - h^2) as the bf16 operand row of the contractions; leaf: dE[tok] += dh.
-// A lane owns 8 consecutive hidden units per 64 and loads all its pieces of the rows before it uses them.
-__device__ __forceinline__ void backward_frame_tc(const DevCtx& c, uint32_t t, int sl) {
-    const int H = c.H, Hp = c.Hp, C = c.n_classes;
-    const uint32_t parent = __ldcg(&c.frames[t].parent);
-    const uint32_t l = __ldcg(&c.op_l[t]);
-    const bool from_result = parent < (uint32_t)c.B, leaf = l == LEAF_MARK;
-    const uint32_t tok = leaf ? __ldcg(&c.op_r[t]) : 0u;
-    const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8);
-    const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8 + 4);
-    const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-    const float* g = c.dhp + (size_t)t * H;
-    constexpr int NQ = TC_HP_MAX / 64;
-    float4 gv[NQ][2];
-    uint4 hv[NQ];
+__device__ __forceinline__ void list_flags(const DevCtx& c, uint32_t f0, uint32_t F, uint32_t (&l)[8], uint32_t (&r)[8],
+                                           uint32_t& cells, uint32_t& leaves) {
+    cells = leaves = 0;
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        const int j = sl * 8 + 64 * q;
-        gv[q][0] = gv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        hv[q] = make_uint4(0u, 0u, 0u, 0u);
-        if (!from_result && j < H) gv[q][0] = ldcg4(g + j);
-        if (!from_result && j + 4 < H) gv[q][1] = ldcg4(g + j + 4);
-        if (!leaf && j < Hp) hv[q] = *reinterpret_cast<const uint4*>(c.arena_bf + (size_t)t * Hp + j);
-    }
-#pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        const int j = sl * 8 + 64 * q;
-        if (j >= Hp) continue;
-        float dh[8] = {gv[q][0].x, gv[q][0].y, gv[q][0].z, gv[q][0].w, gv[q][1].x, gv[q][1].y, gv[q][1].z, gv[q][1].w};
-#pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            if (k < C) {
-                if (j < H) {
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                    dh[0] = fmaf(w.x, dl[k], dh[0]); dh[1] = fmaf(w.y, dl[k], dh[1]);
-                    dh[2] = fmaf(w.z, dl[k], dh[2]); dh[3] = fmaf(w.w, dl[k], dh[3]);
-                }
-                if (j + 4 < H) {
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j + 4]));
-                    dh[4] = fmaf(w.x, dl[k], dh[4]); dh[5] = fmaf(w.y, dl[k], dh[5]);
-                    dh[6] = fmaf(w.z, dl[k], dh[6]); dh[7] = fmaf(w.w, dl[k], dh[7]);
-                }
-            }
-        if (leaf) {
-            float* de = c.dE + (size_t)tok * c.D + j;
-            if (j < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(dh[0], dh[1], dh[2], dh[3]));
-            if (j + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(dh[4], dh[5], dh[6], dh[7]));
-        } else {
-            float x[8];
-            unpack_bf8(hv[q], x);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dh[i] *= 1.f - x[i] * x[i];      // pad columns: dh = 0 and h = 0, so dz = 0
-            __align__(16) __nv_bfloat162 pk[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(dh[2 * i], dh[2 * i + 1]);
-            *reinterpret_cast<uint4*>(c.dz_bf + (size_t)t * Hp + j) = *reinterpret_cast<const uint4*>(pk);
+    for (int i = 0; i < 8; ++i) {                       // thread-contiguous: frames f0 + 8 tid + i
+        const uint32_t f = f0 + threadIdx.x * 8 + i;
+        l[i] = LEAF_MARK; r[i] = 0;
+        if (f < F) {
+            l[i] = c.op_l[f]; r[i] = c.op_r[f];
+            if (l[i] != LEAF_MARK) ++cells; else ++leaves;
         }
     }
 }
 
-// A (fp32 TreeRNN), one invocation t per 8 lanes; dz (cell) / dh (leaf) replaces the incoming gradient.
-__device__ __forceinline__ void backward_frame_f32(const DevCtx& c, uint32_t t, int sl) {
-    const int H = c.H, C = c.n_classes;
-    const uint32_t parent = __ldcg(&c.frames[t].parent);
-    const uint32_t l = __ldcg(&c.op_l[t]);
-    const bool from_result = parent < (uint32_t)c.B, leaf = l == LEAF_MARK;
-    const uint32_t tok = leaf ? __ldcg(&c.op_r[t]) : 0u;
-    const float4 d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8);
-    const float4 d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8 + 4);
-    const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-    float* g = c.dhp + (size_t)t * H;
-    const float* h = c.arena + (size_t)t * H;
-#pragma unroll 4
-    for (int j = sl * 4; j < H; j += 32) {
-        float4 dh = from_result ? make_float4(0.f, 0.f, 0.f, 0.f) : ldcg4(g + j);
+__global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uint2* seg_counts) {
+    __shared__ uint32_t wc[8], wl[8];
+    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
+    uint32_t l[8], r[8], cells, leaves;
+    list_flags(c, f0, F, l, r, cells, leaves);
+    for (int o = 16; o > 0; o >>= 1) {
+        cells += __shfl_xor_sync(0xffffffffu, cells, o);
+        leaves += __shfl_xor_sync(0xffffffffu, leaves, o);
+    }
+    if (threadIdx.x % 32 == 0) { wc[threadIdx.x / 32] = cells; wl[threadIdx.x / 32] = leaves; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t a = 0, b = 0;
+        for (int w = 0; w < 8; ++w) { a += wc[w]; b += wl[w]; }
+        seg_counts[blockIdx.x] = make_uint2(a, b);
+    }
+}
+
+// one block: exclusive scan of the segment counts in place; totals to the control block
+__global__ void __launch_bounds__(1024) rdf_list_scan_kernel(const DevCtx c, uint2* seg_counts, int n_seg) {
+    __shared__ uint32_t wa[32], wb[32];
+    const int per = (n_seg + 1023) / 1024, s0 = threadIdx.x * per, s1 = min(n_seg, s0 + per);
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    uint32_t a = 0, b = 0;
+    for (int i = s0; i < s1; ++i) { a += seg_counts[i].x; b += seg_counts[i].y; }
+    uint32_t pa = a, pb = b;                            // inclusive scan over the threads
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t x = __shfl_up_sync(0xffffffffu, pa, o), y = __shfl_up_sync(0xffffffffu, pb, o);
+        if (lane >= o) { pa += x; pb += y; }
+    }
+    if (lane == 31) { wa[warp] = pa; wb[warp] = pb; }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t x = wa[lane], y = wb[lane];
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xffffffffu, x, o), v = __shfl_up_sync(0xffffffffu, y, o);
+            if (lane >= o) { x += u; y += v; }
+        }
+        wa[lane] = x; wb[lane] = y;                     // inclusive over the warps
+        if (lane == 31) { c.ctl->all_cells = x; c.ctl->all_leaves = y; }
+    }
+    __syncthreads();
+    a = pa - a + (warp ? wa[warp - 1] : 0u);
+    b = pb - b + (warp ? wb[warp - 1] : 0u);
+    for (int i = s0; i < s1; ++i) {
+        const uint2 v = seg_counts[i];
+        seg_counts[i] = make_uint2(a, b);
+        a += v.x; b += v.y;
+    }
+}
+
+__global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, const uint2* seg_base) {
+    __shared__ uint32_t wc[8], wl[8];
+    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
+    uint32_t l[8], r[8], cells, leaves;
+    list_flags(c, f0, F, l, r, cells, leaves);
+    // exclusive prefix of (cells, leaves) over the threads of the block
+    uint32_t pc = cells, pl = leaves;
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t a = __shfl_up_sync(0xffffffffu, pc, o), b = __shfl_up_sync(0xffffffffu, pl, o);
+        if (lane >= o) { pc += a; pl += b; }
+    }
+    if (lane == 31) { wc[warp] = pc; wl[warp] = pl; }
+    __syncthreads();
+    const uint2 sb = seg_base[blockIdx.x];
+    uint32_t ic = sb.x + pc - cells, il = sb.y + pl - leaves;
+    for (int w = 0; w < warp; ++w) { ic += wc[w]; il += wl[w]; }
 #pragma unroll
-        for (int k = 0; k < MAX_CLASSES; ++k)
-            if (k < C) {
-                const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
-                dh.x = fmaf(w.x, dl[k], dh.x); dh.y = fmaf(w.y, dl[k], dh.y);
-                dh.z = fmaf(w.z, dl[k], dh.z); dh.w = fmaf(w.w, dl[k], dh.w);
-            }
-        if (leaf) {
-            atomicAdd(reinterpret_cast<float4*>(c.dE + (size_t)tok * c.D + j), dh);
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t f = f0 + threadIdx.x * 8 + i;
+        if (f >= F) break;
+        if (l[i] != LEAF_MARK) {
+            c.all_cells[ic] = f;
+            if (c.cell_ops) c.cell_ops[ic] = make_uint4(f, l[i], r[i], 1u);
+            ++ic;
         } else {
-            const float4 hv = *reinterpret_cast<const float4*>(h + j);
-            dh.x *= 1.f - hv.x * hv.x; dh.y *= 1.f - hv.y * hv.y;
-            dh.z *= 1.f - hv.z * hv.z; dh.w *= 1.f - hv.w * hv.w;
-            *reinterpret_cast<float4*>(g + j) = dh;
+            if (c.lstm) {
+                c.all_leaves[il] = f;
+                if (c.leaf_ops) c.leaf_ops[il] = make_uint4(f, r[i], 0u, 1u);      // r = token id of a leaf
+            }
+            ++il;
+        }
+    }
+}
+
+// marks[d].w = cells among the frames below marks[d].x: where wave d ends in all_cells.  One warp per wave.
+__global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, const uint2* seg_base) {
+    const uint32_t lane = threadIdx.x % 32, n_warps = gridDim.x * blockDim.x / 32;
+    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
+    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), B = (uint32_t)c.B;
+    for (uint32_t d = (blockIdx.x * blockDim.x + threadIdx.x) / 32; d < n_waves; d += n_warps) {
+        const uint32_t f = max(B, min(c.wave_marks[d].x, F));
+        const uint32_t seg = (f - B) / LIST_SEG, s0 = B + seg * LIST_SEG;      // (the segment array has one entry to spare)
+        uint32_t cnt = 0;
+        for (uint32_t g = s0 + lane; g < f; g += 32) cnt += c.op_l[g] != LEAF_MARK;
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (lane == 0) c.wave_marks[d].w = seg_base[seg].x + cnt;
+    }
+}
+
+// What a thread needs to know about an invocation before it touches its rows; all of it is left
+// behind by the forward pass and the loss head, so it can be fetched one step ahead.
+struct FrameMeta {
+    uint32_t l, r, parent;
+    float4 d0, d1;
+};
+__device__ __forceinline__ FrameMeta load_meta(const DevCtx& c, uint32_t t) {
+    FrameMeta m;
+    m.l = c.op_l[t]; m.r = c.op_r[t]; m.parent = c.frames[t].parent;
+    m.d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8);
+    m.d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)t * 8 + 4);
+    return m;
+}
+
+// A (bf16 TreeRNN), one invocation per 8 lanes and step: dh = (gradient from the caller) + W_s^T dlog;
+//    cell: dz = dh * (1 - h^2) as the bf16 operand row of the contractions; leaf: dE[tok] += dh.
+// A lane owns 8 consecutive hidden units per 64.  All loads of a step are independent of each other
+// (the record of the invocation was fetched during the previous step), so a step costs one round trip.
+__device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0, uint32_t end, uint32_t stride, int sl) {
+    const int H = c.H, Hp = c.Hp, C = c.n_classes;
+    constexpr int NQ = TC_HP_MAX / 64;
+    if (t0 >= end) return;
+    FrameMeta m = load_meta(c, t0);
+    for (uint32_t t = t0; t < end; t += stride) {
+        const bool from_result = m.parent < (uint32_t)c.B, leaf = m.l == LEAF_MARK;
+        const uint32_t tok = m.r;
+        const float dl[MAX_CLASSES] = {m.d0.x, m.d0.y, m.d0.z, m.d0.w, m.d1.x, m.d1.y, m.d1.z, m.d1.w};
+        const float* g = c.dhp + (size_t)t * H;
+        float4 gv[NQ][2];
+        uint4 hv[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int j = sl * 8 + 64 * q;
+            gv[q][0] = gv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            hv[q] = make_uint4(0u, 0u, 0u, 0u);
+            // (an invocation called from `result` has no incoming gradient: what is loaded is not used)
+            if (j < H) gv[q][0] = ldcg4(g + j);
+            if (j + 4 < H) gv[q][1] = ldcg4(g + j + 4);
+            if (!leaf && j < Hp) hv[q] = *reinterpret_cast<const uint4*>(c.arena_bf + (size_t)t * Hp + j);
+        }
+        if (t + stride < end) m = load_meta(c, t + stride);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int j = sl * 8 + 64 * q;
+            if (j >= Hp) continue;
+            float dh[8] = {gv[q][0].x, gv[q][0].y, gv[q][0].z, gv[q][0].w, gv[q][1].x, gv[q][1].y, gv[q][1].z, gv[q][1].w};
+            if (from_result) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) dh[i] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) {
+                    if (j < H) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                        dh[0] = fmaf(w.x, dl[k], dh[0]); dh[1] = fmaf(w.y, dl[k], dh[1]);
+                        dh[2] = fmaf(w.z, dl[k], dh[2]); dh[3] = fmaf(w.w, dl[k], dh[3]);
+                    }
+                    if (j + 4 < H) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j + 4]));
+                        dh[4] = fmaf(w.x, dl[k], dh[4]); dh[5] = fmaf(w.y, dl[k], dh[5]);
+                        dh[6] = fmaf(w.z, dl[k], dh[6]); dh[7] = fmaf(w.w, dl[k], dh[7]);
+                    }
+                }
+            if (leaf) {
+                float* de = c.dE + (size_t)tok * c.D + j;
+                if (j < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(dh[0], dh[1], dh[2], dh[3]));
+                if (j + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(dh[4], dh[5], dh[6], dh[7]));
+            } else {
+                float x[8];
+                unpack_bf8(hv[q], x);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) dh[i] *= 1.f - x[i] * x[i];      // pad columns: dh = 0 and h = 0, so dz = 0
+                __align__(16) __nv_bfloat162 pk[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(dh[2 * i], dh[2 * i + 1]);
+                *reinterpret_cast<uint4*>(c.dz_bf + (size_t)t * Hp + j) = *reinterpret_cast<const uint4*>(pk);
+            }
+        }
+    }
+}
+
+// A (fp32 TreeRNN), one invocation per 8 lanes and step; dz (cell) replaces the incoming gradient.
+__device__ __forceinline__ void backward_frames_f32(const DevCtx& c, uint32_t t0, uint32_t end, uint32_t stride, int sl) {
+    const int H = c.H, C = c.n_classes;
+    if (t0 >= end) return;
+    FrameMeta m = load_meta(c, t0);
+    for (uint32_t t = t0; t < end; t += stride) {
+        const bool from_result = m.parent < (uint32_t)c.B, leaf = m.l == LEAF_MARK;
+        const uint32_t tok = m.r;
+        const float dl[MAX_CLASSES] = {m.d0.x, m.d0.y, m.d0.z, m.d0.w, m.d1.x, m.d1.y, m.d1.z, m.d1.w};
+        if (t + stride < end) m = load_meta(c, t + stride);
+        float* g = c.dhp + (size_t)t * H;
+        const float* h = c.arena + (size_t)t * H;
+#pragma unroll 4
+        for (int j = sl * 4; j < H; j += 32) {
+            float4 dh = ldcg4(g + j);                    // (not used for an invocation called from `result`)
+            const float4 hv = leaf ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(h + j);
+            if (from_result) dh = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + j]));
+                    dh.x = fmaf(w.x, dl[k], dh.x); dh.y = fmaf(w.y, dl[k], dh.y);
+                    dh.z = fmaf(w.z, dl[k], dh.z); dh.w = fmaf(w.w, dl[k], dh.w);
+                }
+            if (leaf) {
+                atomicAdd(reinterpret_cast<float4*>(c.dE + (size_t)tok * c.D + j), dh);
+            } else {
+                dh.x *= 1.f - hv.x * hv.x; dh.y *= 1.f - hv.y * hv.y;
+                dh.z *= 1.f - hv.z * hv.z; dh.w *= 1.f - hv.w * hv.w;
+                *reinterpret_cast<float4*>(g + j) = dh;
+            }
         }
     }
 }
@@ -554,7 +650,6 @@ template <bool TC>
 __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
     __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // fp32: tiles use the first part; thin patches stage rows in it
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
-    __shared__ FrameLists lists;
     if (c.ctl->forward_status != 0) return;                          // the forward pass failed: nothing to differentiate
     TcState tc;
     if constexpr (TC) {
@@ -578,29 +673,24 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
         if (f1 == f0) continue;                                      // a wave without calls
         ++wave;
-        // ---- A: per-invocation work, a contiguous piece of the range per block, one frame per thread and round
+        // ---- A: per-invocation work, a contiguous piece of the range per block
         const uint32_t n = f1 - f0;
         const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
         const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
         const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
-        for (uint32_t base = c0; base < c1; base += blockDim.x) {
-            const uint32_t end = min(c1, base + blockDim.x);
-            if (c.lstm) {
-                for (uint32_t t = base + wib; t < end; t += n_warps) lstm_backward_frame(c, t, lane);
-            } else {
-                for (uint32_t t = base + wib * 4 + lane / 8; t < end; t += 4 * n_warps) {
-                    if constexpr (TC) backward_frame_tc(c, t, lane % 8);
-                    else backward_frame_f32(c, t, lane % 8);
-                }
-            }
-            backward_list_frames(c, lists, base, end);
+        if (c.lstm) {
+            for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
+        } else if constexpr (TC) {
+            backward_frames_tc(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+        } else {
+            backward_frames_f32(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
         }
         __syncthreads();
         lap(cyc_a);
         if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
         lap(cyc_b);
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
-        const uint32_t end = ld_volatile_u32(&c.ctl->all_cells);
+        const uint32_t end = max(first, min(c.wave_marks[d].w, c.frame_cap));     // the wave's cells: all_cells[first, end)
         if (end > first) {
             if constexpr (TC) {
                 if (c.lstm) tc_pipe<TC_LSTM_BWD, TC_STAGES_LSTM_BWD>(c, tc, smem, first, end - first);
@@ -827,6 +917,15 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks);
     }
     rdf_mark(S, 3, stream);
+    // lists of the gradient pass (cells in frame order, per-wave ends)
+    {
+        const int n_seg = (int)(in->max_invocations / LIST_SEG) + 1;
+        uint2* seg = reinterpret_cast<uint2*>(ws + L.list_seg);
+        rdf_list_count_kernel<<<n_seg, 256, 0, stream>>>(c, seg);
+        rdf_list_scan_kernel<<<1, 1024, 0, stream>>>(c, seg, n_seg);
+        rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg);
+        rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg);
+    }
     // gradient waves
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
