@@ -590,7 +590,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(32, 5 * L.Hp, 0, 0, TC_STAGES_LSTM_BWD) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, TC_STAGES_RNN_BWD);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
-    L.dhp = P.take<float>(gf * S);
+    L.dhp = P.take<float>(tcr ? 0 : gf * S);            // (the bf16 TreeRNN hands its gradients on as dz rows)
     L.dlog = P.take<float>(gf * 8);
     // every wave of a vector program holds at least one token of an invocation on its way down or up
     L.wave_cap = g->has_vector_ops ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
@@ -686,7 +686,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.y = out->y;
     }
     c.trace = out->trace; c.trace_cap = out->trace ? out->trace_capacity : 0;
-    c.dhp = reinterpret_cast<float*>(ws + L.dhp);
+    c.dhp = L.use_tc && !g->has_lstm ? nullptr : reinterpret_cast<float*>(ws + L.dhp);
     c.dlog = reinterpret_cast<float*>(ws + L.dlog);
     c.wave_marks = L.wave_cap ? reinterpret_cast<uint4*>(ws + L.wave_marks) : nullptr;
     c.wave_cap = L.wave_cap;

@@ -364,30 +364,24 @@ __device__ __forceinline__ FrameMeta load_meta(const DevCtx& c, uint32_t t) {
     return m;
 }
 
-// A (bf16 TreeRNN), one invocation per 8 lanes and step: dh = (gradient from the caller) + W_s^T dlog;
-//    cell: dz = dh * (1 - h^2) as the bf16 operand row of the contractions; leaf: dE[tok] += dh.
-// A lane owns 8 consecutive hidden units per 64.  All loads of a step are independent of each other
-// (the record of the invocation was fetched during the previous step), so a step costs one round trip.
+// A (bf16 TreeRNN), the invocations called from `result` (no gradient comes in from a caller), one per
+// 8 lanes and step: dh = W_s^T dlog; cell: dz = dh * (1 - h^2) as the bf16 operand row of the
+// contractions; leaf: dE[tok] += dh.  A lane owns 8 consecutive hidden units per 64.  Every other
+// invocation gets the same treatment from the epilogue of its caller's operand-gradient tile.
 __device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0, uint32_t end, uint32_t stride, int sl) {
     const int H = c.H, Hp = c.Hp, C = c.n_classes;
     constexpr int NQ = TC_HP_MAX / 64;
     if (t0 >= end) return;
     FrameMeta m = load_meta(c, t0);
     for (uint32_t t = t0; t < end; t += stride) {
-        const bool from_result = m.parent < (uint32_t)c.B, leaf = m.l == LEAF_MARK;
+        const bool leaf = m.l == LEAF_MARK;
         const uint32_t tok = m.r;
         const float dl[MAX_CLASSES] = {m.d0.x, m.d0.y, m.d0.z, m.d0.w, m.d1.x, m.d1.y, m.d1.z, m.d1.w};
-        const float* g = c.dhp + (size_t)t * H;
-        float4 gv[NQ][2];
         uint4 hv[NQ];
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
             const int j = sl * 8 + 64 * q;
-            gv[q][0] = gv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
             hv[q] = make_uint4(0u, 0u, 0u, 0u);
-            // (an invocation called from `result` has no incoming gradient: what is loaded is not used)
-            if (j < H) gv[q][0] = ldcg4(g + j);
-            if (j + 4 < H) gv[q][1] = ldcg4(g + j + 4);
             if (!leaf && j < Hp) hv[q] = *reinterpret_cast<const uint4*>(c.arena_bf + (size_t)t * Hp + j);
         }
         if (t + stride < end) m = load_meta(c, t + stride);
@@ -395,11 +389,7 @@ __device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0,
         for (int q = 0; q < NQ; ++q) {
             const int j = sl * 8 + 64 * q;
             if (j >= Hp) continue;
-            float dh[8] = {gv[q][0].x, gv[q][0].y, gv[q][0].z, gv[q][0].w, gv[q][1].x, gv[q][1].y, gv[q][1].z, gv[q][1].w};
-            if (from_result) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) dh[i] = 0.f;
-            }
+            float dh[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int k = 0; k < MAX_CLASSES; ++k)
                 if (k < C) {
@@ -673,22 +663,25 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
         if (f1 == f0) continue;                                      // a wave without calls
         ++wave;
-        // ---- A: per-invocation work, a contiguous piece of the range per block
-        const uint32_t n = f1 - f0;
-        const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
-        const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
-        const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
-        if (c.lstm) {
-            for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
-        } else if constexpr (TC) {
-            backward_frames_tc(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
-        } else {
-            backward_frames_f32(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+        // ---- A: per-invocation work, a contiguous piece of the range per block.  (bf16 TreeRNN: only the
+        //      invocations called from `result` -- further down the epilogue of B does this work for the callees.)
+        if (!(TC && !c.lstm && d > 0)) {
+            const uint32_t n = f1 - f0;
+            const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
+            const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
+            const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
+            if (c.lstm) {
+                for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
+            } else if constexpr (TC) {
+                backward_frames_tc(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+            } else {
+                backward_frames_f32(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+            }
+            __syncthreads();
+            lap(cyc_a);
+            if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+            lap(cyc_b);
         }
-        __syncthreads();
-        lap(cyc_a);
-        if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
-        lap(cyc_b);
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
         const uint32_t end = max(first, min(c.wave_marks[d].w, c.frame_cap));     // the wave's cells: all_cells[first, end)
         if (end > first) {

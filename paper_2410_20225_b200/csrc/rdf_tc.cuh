@@ -36,7 +36,7 @@ static const int TC_STAGES_RNN_FWD = 7, TC_STAGES_LSTM_FWD = 5, TC_STAGES_RNN_BW
 // tile loops (template parameter of tc_pipe)
 enum TcMode {
     TC_RNN_FWD = 0,     // A = [h_l ; h_r] (bf16 states), B = Wp slice;           epilogue: tanh, bf16 state
-    TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: operand gradients
+    TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: dz of the callee cells, dE of the callee leaves
     TC_LSTM_CELL = 2,   // A = [h_l ; h_r],                B = W5p slice (5 gates x 16 units); epilogue: gates, c, h
     TC_LSTM_LEAF = 3,   // A = E_bf[tok],                  B = Wxp slice (3 gates x 16 units); epilogue: gates, c, h
     TC_LSTM_BWD = 4,    // A = gate gradients (5 Hp),      B = WT5p slice;         epilogue: operand gradients (dh)
@@ -353,14 +353,84 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
         for (int i = 0; i < my_tiles && ok; ++i) {
             const uint32_t T = tc.T + i, b = T & 1u;
             ok = mbar_wait(c, items_full0 + 8 * b, (T >> 1) & 1u);
-            ok = ok && mbar_wait(c, acc_full0 + 8 * b, (T >> 1) & 1u);
             if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int row = (warp & 3) * 32 + lane;                       // warp w reads TMEM lanes 32 (w % 4) ..
             const uint32_t lane_base = tc.tmem_base + (uint32_t)(b * TC_ACC_COLS) + ((uint32_t)((warp & 3) * 32) << 16);
             const uint4 it = sh.items[b][row];
             const bool live = it.w != 0u;
-            if (MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) {
+            // TreeRNN gradient: what the epilogue needs about the callee frame is fetched while the MMAs run.
+            // All columns of a slice belong to one callee: [0, Hp) to the left one, [Hp, 2Hp) to the right one.
+            constexpr int BWD_MAXG = (TC_HP_MAX / 4 / 16 + 1) / 2;
+            const int e_groups = ns / 16, e_lo = (e_groups + 1) / 2;
+            const int e_begin = warp < 4 ? 0 : e_lo, e_end = warp < 4 ? e_lo : e_groups;
+            const int e_col0 = slice * ns;
+            const uint32_t child = e_col0 < Hp ? it.y : it.z;
+            const int e_cc0 = e_col0 < Hp ? e_col0 : e_col0 - Hp;
+            uint32_t child_l = LEAF_MARK, child_tok = 0;
+            float4 cd0 = make_float4(0.f, 0.f, 0.f, 0.f), cd1 = cd0;
+            uint4 chq[BWD_MAXG][2];
+            if (MODE == TC_RNN_BWD && live) {
+                child_l = c.op_l[child];
+                child_tok = c.op_r[child];
+                cd0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
+                cd1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
+#pragma unroll
+                for (int q = 0; q < BWD_MAXG; ++q)
+                    if (e_begin + q < e_end) {
+                        const uint4* hp = reinterpret_cast<const uint4*>(c.arena_bf + (size_t)child * Hp + e_cc0 + (e_begin + q) * 16);
+                        chq[q][0] = hp[0];
+                        chq[q][1] = hp[1];
+                    }
+            }
+            ok = mbar_wait(c, acc_full0 + 8 * b, (T >> 1) & 1u);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (MODE == TC_RNN_BWD) {
+                // dh of the callee = its slice of W^T dz (the accumulators) + W_s^T dlog of the callee;
+                // a cell callee gets dz = dh (1 - h^2) as its bf16 operand row for the next wave (and for dW),
+                // a leaf callee adds dh to row tok of dE.  No gradient ever goes to memory in fp32.
+                const float dl[8] = {cd0.x, cd0.y, cd0.z, cd0.w, cd1.x, cd1.y, cd1.z, cd1.w};
+#pragma unroll
+                for (int q = 0; q < BWD_MAXG; ++q) {
+                    if (e_begin + q >= e_end) continue;                   // (uniform over the warp)
+                    float v[16];
+                    tc_ld16(lane_base + (uint32_t)((e_begin + q) * 16), v);
+                    if (!live) continue;
+                    const int cc = e_cc0 + (e_begin + q) * 16;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (k < c.n_classes) {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 4)
+                                if (cc + i < H) {
+                                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + cc + i]));
+                                    v[i] = fmaf(w.x, dl[k], v[i]); v[i + 1] = fmaf(w.y, dl[k], v[i + 1]);
+                                    v[i + 2] = fmaf(w.z, dl[k], v[i + 2]); v[i + 3] = fmaf(w.w, dl[k], v[i + 3]);
+                                }
+                        }
+                    if (child_l == LEAF_MARK) {
+                        float* de = c.dE + (size_t)child_tok * c.D + cc;
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            if (cc + i < H) atomicAdd(reinterpret_cast<float4*>(de + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+                    } else {
+                        __align__(16) __nv_bfloat162 pk[8];
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&chq[q][half]);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 x = __bfloat1622float2(hb[i]);   // pad columns: v = 0 and h = 0, so dz = 0
+                                pk[half * 4 + i] = __floats2bfloat162_rn(v[half * 8 + 2 * i] * (1.f - x.x * x.x),
+                                                                         v[half * 8 + 2 * i + 1] * (1.f - x.y * x.y));
+                            }
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(c.dz_bf + (size_t)child * Hp + cc);
+                        dst[0] = *reinterpret_cast<const uint4*>(&pk[0]);
+                        dst[1] = *reinterpret_cast<const uint4*>(&pk[4]);
+                    }
+                }
+            } else if (MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) {
                 // slice = 16 hidden units, columns gate * 16 + unit; warps 0-3 take units 0-7, warps 4-7 units 8-15
                 constexpr int NG = MODE == TC_LSTM_CELL ? 5 : 3;
                 const int wg = warp >> 2, u0 = slice * 16 + wg * 8;
