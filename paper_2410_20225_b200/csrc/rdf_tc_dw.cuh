@@ -12,8 +12,10 @@
 static const int DW_KT = 64;                          // cells per stage
 static const int DW_HALF = DW_KT * 256;               // 16 KB: one operand of a stage
 static const int DW_STAGE = 2 * DW_HALF;
-static const int DW_STAGES = 4;
+static const int DW_STAGES = 6;
+static const int DW_INFLIGHT = 4;                     // stages a producer thread keeps in flight
 static const int DW_SMEM_BYTES = 1024 + DW_STAGES * DW_STAGE;
+static const int DW_PRODUCERS = 128;                  // warps 0-3 gather, warp 4 issues the MMAs, all 8 warps write out
 
 // MN-major operand descriptor: atoms of 64 elements (128 bytes) along M/N by 8 along K;
 // lbo = byte distance between atoms along M/N, sbo = between atoms along K.
@@ -46,88 +48,109 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
     const uint32_t lbo = 8192u, sbo = 1024u;       // next atom along M/N, next atom along K
     extern __shared__ unsigned char dyn_smem[];
     __shared__ uint32_t tmem_slot;
-    __shared__ __align__(8) uint64_t mbars[DW_STAGES];
-    __shared__ uint4 s_ops[DW_STAGES][DW_KT];
+    __shared__ __align__(8) uint64_t full[DW_STAGES], empty[DW_STAGES], done;
     const uint32_t n_cells = *a.count;
     const int tile = blockIdx.x % a.n_tiles, split = blockIdx.x / a.n_tiles;
     const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_cells, t_begin + a.chunk);
     if (t_begin >= t_end) return;                                  // the whole block leaves before any set-up
     const int H = c.H, Hp = c.Hp;
     const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
-    const int n_chunks = (int)((t_end - t_begin + DW_KT - 1) / DW_KT);
+    const uint32_t n_chunks = (t_end - t_begin + DW_KT - 1) / DW_KT;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const uint32_t raw = smem_u32(dyn_smem);
     const uint32_t stage0 = (raw + 1023u) & ~1023u;
-    const uint32_t mbar = smem_u32(mbars);
+    const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), done0 = smem_u32(&done);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < DW_STAGES; ++s) mbar_init(mbar + 8 * s, 1);
+        for (int s = 0; s < DW_STAGES; ++s) {
+            mbar_init(full0 + 8 * s, DW_PRODUCERS);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(done0, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < 32) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;" ::"r"(smem_u32(&tmem_slot)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    auto load_ops = [&](int kc) {
-        if (threadIdx.x < DW_KT) {
-            const uint32_t idx = t_begin + kc * DW_KT + threadIdx.x;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (idx < t_end) v = a.ops[idx];
-            s_ops[kc % DW_STAGES][threadIdx.x] = v;
-        }
-    };
-    for (int kc = 0; kc < 3 && kc < n_chunks; ++kc) load_ops(kc);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
-    const uint32_t idesc = tc_idesc(128) | (1u << 15) | (1u << 16);        // both operands MN-major
-
     bool ok = true;
-    auto issue = [&](int kc) {
-        const uint32_t s = kc % DW_STAGES;
-        if (kc >= DW_STAGES) ok = mbar_wait(c, mbar + 8 * s, ((kc / DW_STAGES) - 1) & 1u) && ok;
-        const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
-        for (int p = threadIdx.x; p < DW_KT * 16; p += blockDim.x) {
-            const int tr = p >> 4, q = p & 15, atom = q >> 3, c16 = q & 7;
-            const uint4 it = s_ops[s][tr];
-            const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
-            const int m = m0 + atom * 64 + c16 * 8;
-            const bool mv = it.w != 0u && m < a.Mp;
-            cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
-            const int n = n0 + atom * 64 + c16 * 8;
-            const bool nv = it.w != 0u && n < a.Np;
-            size_t src = 0;
-            if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
-            cp_async16(b_st + off, (a.mode == 0 ? c.arena_bf : c.E_bf) + src, nv);
-        }
-        cp_async_commit();
-    };
-    issue(0);
-    if (n_chunks > 1) issue(1); else cp_async_commit();
-    for (int kc = 0; kc < n_chunks; ++kc) {
-        if (kc + 3 < n_chunks) load_ops(kc + 3);
-        if (kc + 2 < n_chunks) issue(kc + 2); else cp_async_commit();
-        cp_async_wait<2>();
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp < 4) {
+        // ---- producers: a thread copies one 16-byte piece (q) of eight cells (tr0 + 8 i) of both operands per stage
+        const int q = threadIdx.x & 15, tr0 = threadIdx.x >> 4, atom = q >> 3, c16 = q & 7;
+        const int m = m0 + atom * 64 + c16 * 8, n = n0 + atom * 64 + c16 * 8;
+        const bool m_in = m < a.Mp, n_in = n < a.Np;
+        const __nv_bfloat16* Brows = a.mode == 0 ? c.arena_bf : c.E_bf;
+        auto load_ops = [&](uint32_t kc, uint4 (&ops)[8]) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t idx = t_begin + kc * DW_KT + tr0 + 8 * i;
+                ops[i] = idx < t_end ? a.ops[idx] : make_uint4(0u, 0u, 0u, 0u);
+            }
+        };
+        uint4 ops[8], ops_next[8];
+        load_ops(0, ops);
+        uint32_t issued = 0, arrived = 0;
+        auto report = [&](uint32_t limit) {                    // own copies complete -> proxy fence -> arrive
+            if (issued - arrived <= limit) return;
+            cp_async_wait_upto(limit);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            while (issued - arrived > limit) {
+                mbar_arrive(full0 + 8 * (arrived % DW_STAGES));
+                ++arrived;
+            }
+        };
+        for (uint32_t kc = 0; kc < n_chunks && ok; ++kc) {
             const uint32_t s = kc % DW_STAGES;
+            if (kc + 1 < n_chunks) load_ops(kc + 1, ops_next);                 // in flight during this stage
+            if (kc >= (uint32_t)DW_STAGES) ok = mbar_wait(c, empty0 + 8 * s, ((kc / DW_STAGES) - 1) & 1u);
             const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
 #pragma unroll
-            for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 invocations = two K atoms = 2048 bytes per step
-                tc_mma(tmem, tc_desc_mn(a_st + ks * 2048, lbo, sbo), tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc,
-                       (kc > 0 || ks > 0) ? 1u : 0u);
-            tc_commit(mbar + 8 * s);
+            for (int i = 0; i < 8; ++i) {
+                const int tr = tr0 + 8 * i;
+                const uint4 it = ops[i];
+                const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
+                const bool mv = it.w != 0u && m_in;
+                cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
+                const bool nv = it.w != 0u && n_in;
+                size_t src = 0;
+                if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
+                cp_async16(b_st + off, Brows + src, nv);
+            }
+            cp_async_commit();
+            ++issued;
+            report(DW_INFLIGHT);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ops[i] = ops_next[i];
         }
+        report(0);
+    } else if (warp == 4) {
+        // ---- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = tc_idesc(128) | (1u << 15) | (1u << 16);        // both operands MN-major
+            for (uint32_t kc = 0; kc < n_chunks && ok; ++kc) {
+                const uint32_t s = kc % DW_STAGES;
+                ok = mbar_wait(c, full0 + 8 * s, (kc / DW_STAGES) & 1u);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
+#pragma unroll
+                for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 invocations = two K atoms = 2048 bytes per step
+                    tc_mma(tmem, tc_desc_mn(a_st + ks * 2048, lbo, sbo), tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc,
+                           (kc > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(empty0 + 8 * s);
+            }
+            if (ok) tc_commit(done0);
+        }
+        __syncwarp();
     }
-    {
-        const uint32_t g = n_chunks - 1;
-        if (ok) ok = mbar_wait(c, mbar + 8 * (g % DW_STAGES), (g / DW_STAGES) & 1u);
-    }
+    // ---- everybody: the accumulators are complete when the last commit has arrived
+    ok = mbar_wait(c, done0, 0u);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
         const int m = m0 + (warp & 3) * 32 + lane;
         const int mj = m % Hp, row = (m / Hp) * H + mj;              // gate block, unit
         const int n_limit = a.mode == 0 ? H : c.D;
