@@ -34,7 +34,11 @@ WORKLOAD_NAMES = {
     4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 3, "grad": 11, "grad_lstm": 13, "grad_tc": 12, "grad_lstm_tc": 15}
+# kernels of the library launched per step (memsets and copies not counted):
+#   seed, scheduler | + operators, root gather | + loss head, loss sum, 4 list kernels, gradient waves, dW, db
+#   bf16: + weight packing (TreeLSTM: + table packing); TreeLSTM: + dW_x, db_x, dE
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 4, "eval_trees_tc": 5, "grad": 13, "grad_tc": 14, "grad_lstm": 16,
+                    "grad_lstm_tc": 18}
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
 
 
@@ -109,8 +113,7 @@ def peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
 # (profiles/rdf_forward_kernel_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {("rdf_forward_kernel", 3, None): 924.30e6,             # profiles/rdf_forward_kernel_config3.md
-                     ("rdf_forward_int_kernel", 1, 131072): 37.04e9}      # profiles/rdf_forward_int_kernel_fib_scaled.md
+NCU_TRAFFIC_BYTES = {}
 
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
@@ -294,7 +297,7 @@ def main():
                 return l.item()
             h2d, d2h = sum(v.numel() * 4 for v in host.values()), 4
         else:
-            kind = "eval_trees"
+            kind = "eval_trees_tc" if use_tc else "eval_trees"
 
             def step():
                 g.eval_trees(dt, dp, compute, check=False, h_root=h_root)
@@ -353,36 +356,49 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel
+    # ---- roofline of the dominant kernel (the phase with the largest share of the step)
     pk = peaks()
     mean_phase = {k: sum(v) / len(v) for k, v in phases.items()}
-    dominant = max(mean_phase, key=mean_phase.get) if mean_phase else "forward"
+    dominant = max(mean_phase, key=mean_phase.get) if mean_phase else "schedule"
     dom_ms = mean_phase.get(dominant, total_ms / args.steps)
-    if cfg["kind"] == "fib":
-        alg_bytes = 128.0 * N          # 6 token touches x 16 B + one 32 B store slot per invocation
-        achieved = alg_bytes / (dom_ms * 1e-3) / 1e9
-        roof = {"kernel": "rdf_forward_int_kernel", "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
+    hbm_roof = lambda kernel, alg_bytes, what: {  # noqa: E731
+        "kernel": kernel, "bound": "hbm", "achieved": alg_bytes / (dom_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+        "unit": "GB/s", "frac": alg_bytes / (dom_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None,
+        "peak_source": pk["source"], "algorithmic_bytes": alg_bytes, "bytes_are": what}
+    if dominant == "schedule" or cfg["kind"] == "fib":
+        # 6 token touches x 16 B + one 32 B store slot / frame record per invocation
+        roof = hbm_roof("rdf_scheduler_kernel", 128.0 * N, "128 B per invocation (token write+read, return/store slot write+read, frame record)")
+    elif dominant == "loss":
+        rowbytes = (64 * ((cfg["H"] + 63) // 64)) * 2 if use_tc else cfg["H"] * 4 * (2 if cell == "lstm" else 1)
+        roof = hbm_roof("rdf_loss_heads_kernel", float(N) * (rowbytes + 32), "one state row read + 32 B dlog written per invocation")
     else:
         H = cfg["H"]
         C = cfg["trees"].n_cells
         # algorithmic flops of the contraction in each phase: 2 * 2H * (rows of W) per cell
-        flops = {"forward": flops_fwd, "backward": flops_fwd, "dW": flops_fwd}.get(dominant, flops_fwd)
-        achieved = flops / (dom_ms * 1e-3) / 1e12
-        kernel = {"forward": "rdf_forward_kernel", "backward": "rdf_backward_kernel",
+        flops = flops_fwd
+        kernel = {"operators": "rdf_operator_kernel", "backward": "rdf_backward_kernel",
                   "dW": "rdf_dw_tc_kernel" if use_tc else "rdf_outer_kernel"}.get(dominant, dominant)
         if use_tc:
             peak = pk["bf16_tflops_sustained"]
+            achieved = flops / (dom_ms * 1e-3) / 1e12
             roof = {"kernel": kernel, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": achieved / peak, "traffic": None,
                     "peak_source": pk["source"] + " (bf16 dense, sustained)", "cells": C, "flops_phase": flops,
-                    "note": "the persistent kernel also runs token scheduling and grid barriers of every wave; "
-                            "see block0_ms_at_max_clock for the split"}
+                    "note": "a persistent kernel: every wave ends at a grid barrier; block0_ms_at_max_clock gives the split"}
+            if dominant == "operators" and cell == "rnn":
+                Hp = 64 * ((H + 63) // 64)
+                # per cell: two bf16 operand rows read, one bf16 state row written; per leaf: an fp32 table row read, a bf16 row written
+                alg = C * (3.0 * Hp * 2) + (tb.N - C) * (H * 4.0 + Hp * 2)
+                roof["hbm_view"] = {"algorithmic_bytes": alg, "achieved_gbs": alg / (dom_ms * 1e-3) / 1e9,
+                                    "frac_of_hbm_peak": alg / (dom_ms * 1e-3) / 1e9 / pk["hbm_gbs"]}
         else:
+            achieved = flops / (dom_ms * 1e-3) / 1e12
             roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
                     "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
                     "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
                     "cells": C, "flops_phase": flops}
+    roof["phase"] = dominant
+    roof["phase_ms"] = dom_ms
 
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((roof["kernel"], args.workload, args.fib_batch if args.workload == 1 else None))
     cpu = None

@@ -227,8 +227,9 @@ typedef struct {
     uint32_t max_depth;          /* deepest tag (PATH mode) */
     uint64_t cells;              /* batched cell firings */
     uint64_t leaves;             /* batched leaf firings */
-    /* SM clock cycles spent by thread block 0, forward kernel then gradient kernel:
-       token scheduling / per-frame work, batched operators, waiting at grid barriers */
+    /* SM clock cycles spent by thread block 0.  Forward: token scheduling (scheduler kernel), batched
+       operators (operator kernel), waiting at grid barriers (both).  Gradient kernel: per-invocation
+       work, batched operand gradients, waiting at grid barriers. */
     uint64_t cycles_schedule, cycles_batch, cycles_barrier;
     uint64_t cycles_bwd_frames, cycles_bwd_batch, cycles_bwd_barrier;
 } rdf_stats;
@@ -275,7 +276,8 @@ int rdf_eval_noalloc(rdf_graph* g, const rdf_batch* in, const rdf_params* params
  * invocation; the gradient pass re-enters every invocation under the tag its
  * forward Call_i created and accumulates parameter gradients over all
  * invocations.  Loss = sum over all invocations marked by NODE_LOSS of the
- * softmax cross-entropy of W_s h + b_s against label[node]. */
+ * softmax cross-entropy of W_s h + b_s against label[node].
+ * Limits: H <= 1024 and n_classes <= 8 (UNSUPPORTED / BAD_ARG otherwise). */
 int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
              rdf_param_grads* grads, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -290,11 +292,13 @@ const char* rdf_strerror(int status);
  * on their stream between the phases of a call.  rdf_last_phase_ms synchronises
  * those events and writes up to `capacity` durations in milliseconds to the
  * host array `ms`, in this order:
- *   0 set-up (clears, program upload, seed tokens)   1 forward waves
- *   2 loss head   3 gradient waves   4 dW   5 db   6 dW_s, db_s   7 dE
- * (rdf_eval fills 0..1).  *n receives the number written. */
-enum { RDF_PHASE_SETUP = 0, RDF_PHASE_FORWARD, RDF_PHASE_LOSS, RDF_PHASE_BACKWARD, RDF_PHASE_DW, RDF_PHASE_DB,
-       RDF_PHASE_DWS, RDF_PHASE_DE, RDF_PHASE__COUNT };
+ *   0 set-up (clears, program upload, seed tokens, weight packing)
+ *   1 scheduler waves (tokens: tag push / pop, matching, lists of ready operators)
+ *   2 operator waves (batched leaves and cells)   3 loss head with dW_s, db_s
+ *   4 gradient waves   5 dW   6 db   7 dE (TreeLSTM; the TreeRNN's dE is formed during the waves)
+ * (rdf_eval fills 0..2).  *n receives the number written. */
+enum { RDF_PHASE_SETUP = 0, RDF_PHASE_SCHEDULE, RDF_PHASE_OPERATORS, RDF_PHASE_LOSS, RDF_PHASE_BACKWARD, RDF_PHASE_DW,
+       RDF_PHASE_DB, RDF_PHASE_DE, RDF_PHASE__COUNT };
 int rdf_set_profiling(rdf_graph* g, int enable);
 int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n);
 

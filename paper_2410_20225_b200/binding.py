@@ -113,7 +113,7 @@ class rdf_stats(C.Structure):
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
            "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
-PHASES = ["setup", "forward", "loss", "backward", "dW", "db", "dW_s", "dE"]
+PHASES = ["setup", "schedule", "operators", "loss", "backward", "dW", "db", "dE"]
 
 _lib = None
 

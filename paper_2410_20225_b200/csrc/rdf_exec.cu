@@ -749,6 +749,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
     CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
+    rdf_mark(S, 2, stream);
     if (g->has_vector_ops) {
         if (c.use_tc)
             CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
@@ -760,7 +761,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     if (out->trace)
         CUDA_OK(cudaMemcpyAsync(out->trace_count, &c.ctl->trace_count, sizeof(uint64_t), cudaMemcpyDeviceToDevice, stream));
-    rdf_mark(S, 2, stream);
+    rdf_mark(S, 3, stream);
     S->last_ctl = c.ctl;
     S->last_stream = stream;
     S->ran = true;

@@ -909,7 +909,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
         rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks);
     }
-    rdf_mark(S, 3, stream);
+    rdf_mark(S, 4, stream);
     // lists of the gradient pass (cells in frame order, per-wave ends)
     {
         const int n_seg = (int)(in->max_invocations / LIST_SEG) + 1;
@@ -929,7 +929,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     } else {
         CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args, 0, stream));
     }
-    rdf_mark(S, 4, stream);
+    rdf_mark(S, 5, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
     const long long max_leaves = std::max<long long>(1, in->max_invocations);
@@ -966,12 +966,11 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
         }
     }
-    rdf_mark(S, 5, stream);
+    rdf_mark(S, 6, stream);
     if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, grads->db);
     else rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
     if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
-    rdf_mark(S, 6, stream);
-    rdf_mark(S, 7, stream);       // (dW_s and db_s come from the loss-head pass)
+    rdf_mark(S, 7, stream);       // (dW_s and db_s came from the loss-head pass)
     if (tc_lstm) {
         const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 5);
         CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));

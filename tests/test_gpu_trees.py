@@ -105,6 +105,25 @@ def test_tags_of_tree_invocations():
     assert got == want
 
 
+def test_frame_ids_are_handed_out_in_wave_order():
+    """The gradient pass walks frame-id ranges: every frame must have a larger id than any frame of a
+    shallower call depth (ids are interned wave by wave, a call fires one wave after its caller)."""
+    tb = workloads.config(3, B=64, V=300, H=32)["trees"]
+    p = workloads.treernn_params(2, 300, 32, 32)
+    g = graph()
+    _, tr = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), trace_capacity=2 * tb.N)
+    calls = tr[tr["kind"] == 0]
+    frames = calls["tag"].astype(np.int64)
+    parents = calls["parent"].astype(np.int64)
+    assert sorted(frames.tolist()) == list(range(tb.B, tb.B + tb.N))        # ids B .. B + N - 1, each once
+    depth = np.zeros(tb.B + tb.N, dtype=np.int64)
+    for f, q in sorted(zip(frames.tolist(), parents.tolist())):             # a parent's id is smaller: already done
+        assert q < f
+        depth[f] = depth[q] + 1
+    d = depth[tb.B:]
+    assert np.all(np.diff(d) >= 0)                                          # depth never decreases with the id
+
+
 def test_treernn_grad_small_fp32():
     cfg = workloads.config(3, B=96, V=500, H=64)
     cfg["params"] = workloads.treernn_params(5, 500, 64, 64)
