@@ -89,7 +89,10 @@ struct DevCtx {
     uint32_t* children;           // [frame_cap * K]: frame created by call site k of this frame's body
     uint32_t  frame_cap;
     int64_t*  frame_args;         // [frame_cap * 2]: parameters 1 and 2 of invocations of multi-parameter functions
-    // token store, dense form: one cell per (frame, port) and an arrival counter per (frame, match node)
+    // token store, dense form.  Two-input operators: one 16-byte slot per (frame, match node), operand
+    // and arrival exchanged in one atomic.  More inputs: one cell per (frame, port) and an arrival
+    // counter per (frame, match node).
+    Slot*     pair_slots;
     int64_t*  port_val;
     uint32_t* arrived;
     // token store, hash form: one open-addressing table per match node
@@ -367,10 +370,38 @@ __device__ __forceinline__ int hash_insert_or_consume(const DevCtx& c, int node,
     return -1;
 }
 
-// Dense form (frame tags): the operand goes to its (frame, port) cell; the
-// arrival that completes the set reads the others.  Returns 1 when complete.
+__device__ __forceinline__ void exch128(Slot* addr, uint64_t new_lo, uint64_t new_hi, uint64_t& old_lo, uint64_t& old_hi) {
+    asm volatile(
+        "{\n"
+        " .reg .b128 n, o;\n"
+        " mov.b128 n, {%2, %3};\n"
+        " atom.global.exch.b128 o, [%4], n;\n"
+        " mov.b128 {%0, %1}, o;\n"
+        "}\n"
+        : "=l"(old_lo), "=l"(old_hi)
+        : "l"(new_lo), "l"(new_hi), "l"(addr)
+        : "memory");
+}
+
+// Dense form (frame tags).  Two-input operator: the operand and the fact of its arrival go into the
+// (frame, node) slot with one 128-bit exchange -- {1 + port, value}; the slot starts as {0, 0}.  The
+// first operand finds the slot empty and stays there, the second gets the first one back.
+// More inputs: the operand goes to its (frame, port) cell; the arrival that completes the set reads
+// the others.  Returns 1 when complete.
 __device__ __forceinline__ int dense_deliver(const DevCtx& c, const MatchNode& M, int node, uint64_t frame, int port,
                                              int64_t val, int64_t* regs, StoreCounters& sc) {
+    if (M.n_ports == 2) {
+        uint64_t old_state, old_val;
+        exch128(&c.pair_slots[(size_t)frame * c.n_match + node], 1ull + (uint64_t)port, (uint64_t)val, old_state, old_val);
+        if (old_state == 0) {
+            ++sc.inserts;
+            return 0;
+        }
+        regs[port] = val;
+        regs[1 - port] = (int64_t)old_val;
+        ++sc.matches;
+        return 1;
+    }
     int64_t* cells = c.port_val + (size_t)frame * c.n_ports_total + M.port_base;
     cells[port] = val;
     __threadfence();

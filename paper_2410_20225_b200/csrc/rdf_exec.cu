@@ -560,6 +560,8 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.frames = P.take<Frame>(L.frame_cap);
     L.frame_args = P.take<int64_t>(g->max_params > 1 ? (size_t)L.frame_cap * 2 : 0);
     L.children = P.take<uint32_t>((size_t)L.frame_cap * g->max_calls_per_body);
+    L.pair_bytes = (size_t)L.frame_cap * g->match.size() * sizeof(Slot);
+    L.pair_slots = P.take<char>(L.pair_bytes);
     L.port_val = P.take<int64_t>((size_t)L.frame_cap * g->n_ports_total);
     L.arrived_bytes = (size_t)L.frame_cap * std::max<size_t>(1, g->match.size()) * sizeof(uint32_t);
     L.arrived = P.take<char>(L.arrived_bytes);
@@ -653,6 +655,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.children = reinterpret_cast<uint32_t*>(ws + L.children);
     c.frame_args = reinterpret_cast<int64_t*>(ws + L.frame_args);
     c.frame_cap = L.frame_cap;
+    c.pair_slots = reinterpret_cast<Slot*>(ws + L.pair_slots);
     c.port_val = reinterpret_cast<int64_t*>(ws + L.port_val);
     c.arrived = reinterpret_cast<uint32_t*>(ws + L.arrived);
     c.table = reinterpret_cast<Slot*>(ws + L.table);
@@ -726,7 +729,12 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
                        DevCtx& c, cudaStream_t stream) {
     rdf_mark(S, 0, stream);
     CUDA_OK(cudaMemsetAsync(ws + L.ctl, 0, 4096, stream));
-    if (L.arrived_bytes && g->tag_mode == RDF_TAGS_FRAME) CUDA_OK(cudaMemsetAsync(ws + L.arrived, 0, L.arrived_bytes, stream));
+    if (g->tag_mode == RDF_TAGS_FRAME) {
+        bool wide = false;                        // an operator with more than two tagged inputs
+        for (const MatchNode& m : g->match) wide = wide || m.n_ports > 2;
+        if (L.pair_bytes) CUDA_OK(cudaMemsetAsync(ws + L.pair_slots, 0, L.pair_bytes, stream));
+        if (wide && L.arrived_bytes) CUDA_OK(cudaMemsetAsync(ws + L.arrived, 0, L.arrived_bytes, stream));
+    }
     if (L.table_bytes) CUDA_OK(cudaMemsetAsync(ws + L.table, 0xFF, L.table_bytes, stream));
     CUDA_OK(cudaMemcpyAsync(ws + L.code, g->code.data(), g->code.size() * sizeof(VmInstr), cudaMemcpyHostToDevice, stream));
     if (!g->match.empty())
