@@ -156,6 +156,12 @@ __device__ __forceinline__ uint32_t swz(int r, int c16) {
     return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
 }
 
+// The executing thread arrives on the mbarrier once all cp.async copies it has issued so far have landed
+// (the barrier's count already includes this arrival).
+__device__ __forceinline__ void cp_async_arrive(uint32_t mbar_addr) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mbar_addr) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive(uint32_t addr) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(addr) : "memory");
 }
@@ -239,7 +245,6 @@ template <int MODE, int STAGES>
 __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t first, uint32_t n_items) {
     static_assert(STAGES >= 3 && STAGES <= TC_MAX_STAGES, "ring depth");
     constexpr int RGN = MODE == TC_LSTM_LEAF ? 1 : 0;
-    constexpr int D = STAGES - 2;                              // chunks a producer thread keeps in flight
     const int H = c.H, Hp = c.Hp, S = c.S, ns = tc.ns[RGN], n_chunks = tc.n_chunks[RGN];
     const int slice = blockIdx.x % tc.n_split, rg = blockIdx.x / tc.n_split, n_rg = gridDim.x / tc.n_split;
     const int tiles = (n_items + TC_M - 1) / TC_M;
@@ -270,27 +275,10 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             return it;
         };
         uint4 it_next = my_tiles ? load_item(rg) : make_uint4(0u, 0u, 0u, 0u);
-        // chunks this thread has issued in this call, and how many of them it has reported as landed
-        uint32_t issued = 0, arrived = 0;
-        // Waits until at most `limit` of this thread's chunks are still in flight and reports the others.
-        // (Writer side of the hand-over: own copies complete, proxy fence, arrive.)
-        auto report = [&](uint32_t limit) {
-            if (issued - arrived <= limit) return;
-            cp_async_wait_upto(limit);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async-proxy reads
-            while (issued - arrived > limit) {
-                mbar_arrive(full0 + 8 * ((tc.g + arrived) % STAGES));
-                ++arrived;
-            }
-        };
         for (int i = 0; i < my_tiles && ok; ++i) {
             const uint32_t T = tc.T + i, b = T & 1u;
-            // The epilogue of the tile before last must have finished with this record buffer.  It can
-            // only finish once all chunks of that tile are reported: at most one tile's worth may be open.
-            if (T >= 2) {
-                report(min((uint32_t)D, (uint32_t)n_chunks));
-                ok = mbar_wait(c, acc_empty0 + 8 * b, ((T >> 1) - 1) & 1u);
-            }
+            // the epilogue of the tile before last has finished with this record buffer
+            if (T >= 2) ok = mbar_wait(c, acc_empty0 + 8 * b, ((T >> 1) - 1) & 1u);
             sh.items[b][p] = it_next;
             mbar_arrive(items_full0 + 8 * b);
             if (i + 1 < my_tiles) it_next = load_item(rg + (i + 1) * n_rg);      // in flight during this tile
@@ -317,12 +305,9 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 for (int q = 0; q < 8; ++q)
                     cp_async16(tc.a_addr + s * TC_A_STAGE + swz(r8 + 16 * q, c16),
                                Arows + (size_t)(second ? src1[q] : src0[q]) * lda + col, (valid >> q) & 1u);
-                cp_async_commit();
-                ++issued;
-                report(D);                                     // D chunks stay in flight
+                cp_async_arrive(full0 + 8 * s);                // this thread's share of the stage: arrives when its copies have landed
             }
         }
-        report(0);                                             // drain
     } else if (warp == TC_MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
@@ -336,6 +321,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                     const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
                     ok = mbar_wait(c, full0 + 8 * s, (g / STAGES) & 1u);
                     if (!ok) break;
+                    // the stage was written by cp.async (generic proxy) and is read by the MMA (async proxy)
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a = tc.a_addr + s * TC_A_STAGE, bw = tc.b_addr[RGN] + kc * ns * 128;
 #pragma unroll

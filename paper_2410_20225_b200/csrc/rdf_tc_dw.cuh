@@ -13,7 +13,6 @@ static const int DW_KT = 64;                          // cells per stage
 static const int DW_HALF = DW_KT * 256;               // 16 KB: one operand of a stage
 static const int DW_STAGE = 2 * DW_HALF;
 static const int DW_STAGES = 6;
-static const int DW_INFLIGHT = 4;                     // stages a producer thread keeps in flight
 static const int DW_SMEM_BYTES = 1024 + DW_STAGES * DW_STAGE;
 static const int DW_PRODUCERS = 128;                  // warps 0-3 gather, warp 4 issues the MMAs, all 8 warps write out
 
@@ -93,16 +92,6 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
         };
         uint4 ops[8], ops_next[8];
         load_ops(0, ops);
-        uint32_t issued = 0, arrived = 0;
-        auto report = [&](uint32_t limit) {                    // own copies complete -> proxy fence -> arrive
-            if (issued - arrived <= limit) return;
-            cp_async_wait_upto(limit);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            while (issued - arrived > limit) {
-                mbar_arrive(full0 + 8 * (arrived % DW_STAGES));
-                ++arrived;
-            }
-        };
         for (uint32_t kc = 0; kc < n_chunks && ok; ++kc) {
             const uint32_t s = kc % DW_STAGES;
             if (kc + 1 < n_chunks) load_ops(kc + 1, ops_next);                 // in flight during this stage
@@ -120,13 +109,10 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
                 if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
                 cp_async16(b_st + off, Brows + src, nv);
             }
-            cp_async_commit();
-            ++issued;
-            report(DW_INFLIGHT);
+            cp_async_arrive(full0 + 8 * s);                    // arrives when this thread's copies of the stage have landed
 #pragma unroll
             for (int i = 0; i < 8; ++i) ops[i] = ops_next[i];
         }
-        report(0);
     } else if (warp == 4) {
         // ---- MMA issuer
         if (lane == 0) {
@@ -135,6 +121,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
                 const uint32_t s = kc % DW_STAGES;
                 ok = mbar_wait(c, full0 + 8 * s, (kc / DW_STAGES) & 1u);
                 if (!ok) break;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cp.async writes -> MMA reads
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
 #pragma unroll
