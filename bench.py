@@ -112,8 +112,9 @@ def peaks():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
-# (profiles/rdf_forward_kernel_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {}
+# (profiles/persistent_kernels_config3.md); None where no capture of the current kernel exists
+NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 399.2e6, ("rdf_operator_kernel", 3, None): 310.8e6,
+                     ("rdf_scheduler_kernel", 3, None): 9.7e6}
 
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
@@ -314,14 +315,14 @@ def main():
         torch.cuda.synchronize()
 
     g.set_profiling(True)
+    clocks = ClockSampler(local)
+    clocks.start()                                   # samples from the warm-up on: short runs still get samples under load
     for _ in range(args.warmup):
         step()
     st = g.stats()                                   # also checks the device status word
 
     # ---- device-timed region: K steps, L2 flushed between steps, one event pair per step
-    clocks = ClockSampler(local)
     barrier()
-    clocks.start()
     times, phases = [], {}
     for _ in range(args.steps):
         flush.fill_(1)
