@@ -210,6 +210,193 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_kernel(const DevCtx c, int
     }
 }
 
+// ---- the same pass for the bf16 TreeRNN, with the two small contractions on the tensor cores
+// (warp-level mma.sync m16n8k16: the shapes are [64 rows x Hp] x [Hp x 8 classes] and [Hp x 64 rows] x [64 x 8],
+// far too small for a tcgen05 tile).  States are bf16 already; W_s and dlog enter as a bf16 pair hi + lo
+// (two MMAs), so the products carry about 16 mantissa bits and the sums are fp32.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// x = hi + lo with hi, lo in bf16; packs (x0, x1) -> hi pair, lo pair
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+    const __nv_bfloat162 hp = __halves2bfloat162(h0, h1);
+    const __nv_bfloat162 lp = __floats2bfloat162_rn(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
+    hi = *reinterpret_cast<const uint32_t*>(&hp);
+    lo = *reinterpret_cast<const uint32_t*>(&lp);
+}
+
+static const int LM_ROWS = 64;                         // rows per slab
+static const int LM_KSTEPS_MAX = TC_HP_MAX / 16;       // k steps of the logits contraction
+static const int LM_MT_MAX = (TC_HP_MAX / 16 + 7) / 8; // 16-unit tiles of dW_s per warp
+
+__global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c) {
+    extern __shared__ __align__(128) unsigned char slab_smem[];        // 2 stages of LM_ROWS rows, stride Hp * 2 + 16 bytes
+    __shared__ __align__(8) uint64_t mbars[2];
+    __shared__ __align__(16) float s_z[2][LM_ROWS][8];                 // partial logits of the two k halves
+    __shared__ __align__(16) float s_dl[LM_ROWS][8];
+    __shared__ int s_lab[2][LM_ROWS];
+    __shared__ float warp_loss[8];
+    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
+    const uint32_t n = F > B ? F - B : 0u, per = (n + gridDim.x - 1) / gridDim.x;
+    const uint32_t f0 = min(F, B + blockIdx.x * per), f1 = min(F, f0 + per);
+    const int n_slabs = (int)((f1 - f0 + LM_ROWS - 1) / LM_ROWS);
+    const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32, g = lane >> 2, t = lane & 3;
+    const int H = c.H, Hp = c.Hp, C = c.n_classes;
+    const uint32_t rowbytes = (uint32_t)Hp * 2u, stride = rowbytes + 16u, stage_bytes = LM_ROWS * stride;
+    const uint32_t mbar = smem_u32(mbars), stage0 = smem_u32(slab_smem);
+    // stale rows of a short last slab must at least be finite: they meet dlog = 0 in the dW_s contraction
+    for (uint32_t q = tid; q < 2 * stage_bytes / 16; q += 256) reinterpret_cast<uint4*>(slab_smem)[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (tid == 0) {
+        mbar_init(mbar, 1);
+        mbar_init(mbar + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // the zeroes before the bulk copies that follow
+    __syncthreads();
+    auto issue = [&](int i) {
+        const uint32_t fs = f0 + (uint32_t)i * LM_ROWS, cnt = min((uint32_t)LM_ROWS, f1 - fs), mb = mbar + 8 * (i & 1);
+        if (tid == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mb), "r"(cnt * rowbytes) : "memory");
+        __syncthreads();                                               // the expectation is registered before any copy completes
+        if (tid < (int)cnt) {
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(stage0 + (i & 1) * stage_bytes + tid * stride), "l"(c.arena_bf + (size_t)(fs + tid) * Hp), "r"(rowbytes), "r"(mb) : "memory");
+            s_lab[i & 1][tid] = __ldg(&c.label[(int)c.frames[fs + tid].arg]);
+        }
+    };
+    // W_s fragments of this warp's k half: b0 = (k = 16 ks + 2t, +1; class g), b1 = (k + 8, + 9; class g), hi and lo
+    const int ksteps = Hp / 16, khalf = (ksteps + 1) / 2, ks0 = (warp >> 2) * khalf, ks1 = min(ksteps, ks0 + khalf);
+    uint32_t wb[(LM_KSTEPS_MAX + 1) / 2][4];
+#pragma unroll
+    for (int q = 0; q < (LM_KSTEPS_MAX + 1) / 2; ++q) {
+        const int k = (ks0 + q) * 16 + 2 * t;
+        float w[4] = {0.f, 0.f, 0.f, 0.f};
+        if (ks0 + q < ks1 && g < C) {
+            if (k < H) { w[0] = c.W_s[g * H + k]; w[1] = c.W_s[g * H + k + 1]; }         // H is a multiple of 4: k + 1 < H
+            if (k + 8 < H) { w[2] = c.W_s[g * H + k + 8]; w[3] = c.W_s[g * H + k + 9]; }
+        }
+        split_bf16x2(w[0], w[1], wb[q][0], wb[q][2]);
+        split_bf16x2(w[2], w[3], wb[q][1], wb[q][3]);
+    }
+    // dW_s accumulators: 16-unit tiles warp, warp + 8, warp + 16 of the Hp units; (unit g / g + 8, class 2t / 2t + 1)
+    const int mtiles = Hp / 16;
+    float acc[LM_MT_MAX][4];
+#pragma unroll
+    for (int m = 0; m < LM_MT_MAX; ++m)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[m][e] = 0.f;
+    float my_loss = 0.f, my_dbs = 0.f;
+    bool ok = true;
+    if (n_slabs > 0) issue(0);
+    for (int i = 0; i < n_slabs; ++i) {
+        if (i + 1 < n_slabs) issue(i + 1);             // its stage was released by the barrier that ended slab i - 1
+        const uint32_t fs = f0 + (uint32_t)i * LM_ROWS, cnt = min((uint32_t)LM_ROWS, f1 - fs);
+        ok = __syncthreads_and(mbar_wait(c, mbar + 8 * (i & 1), (uint32_t)(i >> 1) & 1u)) != 0;
+        if (!ok) break;                                // the whole block agrees
+        const uint32_t st = stage0 + (i & 1) * stage_bytes;
+        // ---- logits: warp = (16-row tile warp & 3, k half warp >> 2)
+        {
+            float z[4] = {0.f, 0.f, 0.f, 0.f};
+            const int mi = lane >> 3, ri = lane & 7;
+            const uint32_t a_row = st + (uint32_t)((warp & 3) * 16 + (mi & 1) * 8 + ri) * stride + (uint32_t)(mi >> 1) * 16u;
+#pragma unroll
+            for (int q = 0; q < (LM_KSTEPS_MAX + 1) / 2; ++q) {
+                if (ks0 + q >= ks1) break;
+                uint32_t a[4];
+                ldmatrix_x4(a, a_row + (uint32_t)(ks0 + q) * 32u);
+                mma_bf16_16816(z, a, wb[q][0], wb[q][1]);
+                mma_bf16_16816(z, a, wb[q][2], wb[q][3]);
+            }
+            float* zp = &s_z[warp >> 2][(warp & 3) * 16 + g][2 * t];
+            zp[0] = z[0]; zp[1] = z[1];
+            zp[8 * 8] = z[2]; zp[8 * 8 + 1] = z[3];    // row + 8
+        }
+        __syncthreads();
+        // ---- softmax, loss, dlog: one thread per row
+        if (tid < LM_ROWS) {
+            float d[MAX_CLASSES];
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k) d[k] = 0.f;
+            if (tid < (int)cnt) {
+                const int lab = s_lab[i & 1][tid];
+                float zr[MAX_CLASSES], m = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        zr[k] = s_z[0][tid][k] + s_z[1][tid][k] + __ldg(&c.b_s[k]);
+                        m = fmaxf(m, zr[k]);
+                    }
+                float sum = 0.f, zl = 0.f;
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) {
+                        sum += expf(zr[k] - m);
+                        if (k == lab) zl = zr[k];
+                    }
+                my_loss += logf(sum) + m - zl;
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k) d[k] = k < C ? expf(zr[k] - m) / sum - (k == lab ? 1.f : 0.f) : 0.f;
+                *reinterpret_cast<float4*>(c.dlog + (size_t)(fs + tid) * 8) = make_float4(d[0], d[1], d[2], d[3]);
+                *reinterpret_cast<float4*>(c.dlog + (size_t)(fs + tid) * 8 + 4) = make_float4(d[4], d[5], d[6], d[7]);
+            }
+            *reinterpret_cast<float4*>(&s_dl[tid][0]) = make_float4(d[0], d[1], d[2], d[3]);      // rows past the end: zero
+            *reinterpret_cast<float4*>(&s_dl[tid][4]) = make_float4(d[4], d[5], d[6], d[7]);
+        }
+        __syncthreads();
+        // ---- dW_s^T [units x classes] += h^T [units x rows] dlog [rows x classes]
+        {
+            const int mi = lane >> 3, ri = lane & 7;
+#pragma unroll
+            for (int kk = 0; kk < LM_ROWS / 16; ++kk) {
+                uint32_t bh0, bl0, bh1, bl1;
+                split_bf16x2(s_dl[kk * 16 + 2 * t][g], s_dl[kk * 16 + 2 * t + 1][g], bh0, bl0);
+                split_bf16x2(s_dl[kk * 16 + 2 * t + 8][g], s_dl[kk * 16 + 2 * t + 9][g], bh1, bl1);
+                const uint32_t a_row = st + (uint32_t)(kk * 16 + (mi >> 1) * 8 + ri) * stride + (uint32_t)(mi & 1) * 16u;
+#pragma unroll
+                for (int m = 0; m < LM_MT_MAX; ++m) {
+                    const int mt = warp + 8 * m;
+                    if (mt >= mtiles) break;
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, a_row + (uint32_t)mt * 32u);
+                    mma_bf16_16816(acc[m], a, bh0, bh1);
+                    mma_bf16_16816(acc[m], a, bl0, bl1);
+                }
+            }
+        }
+        if (tid < C)
+            for (uint32_t fi = 0; fi < cnt; ++fi) my_dbs += s_dl[fi][tid];
+        __syncthreads();                               // the stage, s_z and s_dl are free again
+    }
+    if (n_slabs > 0) {
+#pragma unroll
+        for (int m = 0; m < LM_MT_MAX; ++m) {
+            const int mt = warp + 8 * m;
+            if (mt >= mtiles) break;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int unit = mt * 16 + g + (e >> 1) * 8, cls = 2 * t + (e & 1);
+                if (unit < H && cls < C) atomicAdd(&c.dW_s[cls * H + unit], acc[m][e]);
+            }
+        }
+        if (tid < C) atomicAdd(&c.db_s[tid], my_dbs);
+    }
+    // threads 0 .. 63 hold row losses: fixed-order sums inside the two warps, then over the warps
+    for (int o = 16; o > 0; o >>= 1) my_loss += __shfl_down_sync(0xffffffffu, my_loss, o);
+    if (lane == 0) warp_loss[warp] = my_loss;
+    __syncthreads();
+    if (tid == 0) c.loss_partial[blockIdx.x] = warp_loss[0] + warp_loss[1];
+}
+
 // Sum of the per-block partial losses in a fixed order (the same partials always give the same sum).
 __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int n_partials) {
     __shared__ double part[256];
@@ -901,8 +1088,9 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         const int smem = 2 * fr * rowbytes + params->n_classes * H * (int)sizeof(float);
         const int loss_blocks = std::min(4096, 2 * S->grid);
         if (tc_rnn) {
-            CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            rdf_loss_heads_kernel<true><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes);
+            const int smem_mma = 2 * LM_ROWS * (rowbytes + 16);
+            CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mma));
+            rdf_loss_heads_mma_kernel<<<loss_blocks, 256, smem_mma, stream>>>(c);
         } else {
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             rdf_loss_heads_kernel<false><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes);
