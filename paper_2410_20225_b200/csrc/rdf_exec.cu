@@ -451,6 +451,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
     if constexpr (TC) {
         if (c.lstm) tc_setup(tc, smem, dyn_smem, c.Hp / 16, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
         else tc_setup(tc, smem, dyn_smem, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
+        tc_setup_epilogue(c, tc, smem, false);
     }
     uint32_t generation = 0;
     long long cyc_c = 0, cyc_b = 0, t_mark = clock64();

@@ -832,6 +832,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     if constexpr (TC) {
         if (c.lstm) tc_setup(tc, smem, dyn_smem, 2 * c.Hp / 32, c.WTp, 5 * c.Hp, 32);
         else tc_setup(tc, smem, dyn_smem, 8, c.WTp, c.Hp, c.Hp / 4);
+        tc_setup_epilogue(c, tc, smem, true);
     }
     const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, n_warps = blockDim.x / 32;
     uint32_t generation = 0, wave = 0, first = 0;

@@ -51,8 +51,11 @@ struct __align__(16) TcShared {
     uint64_t acc_full[2], acc_empty[2];      // accumulator buffer complete / read out by the epilogue
     uint64_t items_full[2];                  // tile records written
     uint32_t tmem_slot;
+    // what the epilogue adds to this block's slice of columns, copied once per kernel (the 30 KB of L1 left
+    // beside the operand stages do not keep it): TreeRNN forward: bias[col]; TreeLSTM: cell bias [gate][unit]
+    // at 0, leaf bias at TC_EP_LEAF; TreeRNN gradient: W_s[class][col of the callee] (zero beyond H and C)
+    __align__(16) float ep[8 * (TC_HP_MAX / 4)];       // read with 128-bit loads
 };
-
 struct TcState {
     uint32_t tmem_base;      // TMEM address returned by tcgen05.alloc
     uint32_t a_addr;         // shared-space address of A stage 0
@@ -63,6 +66,30 @@ struct TcState {
     uint32_t b_addr[2];
     int      ns[2], n_chunks[2];
 };
+
+static const int TC_EP_LD = TC_HP_MAX / 4, TC_EP_LEAF = 5 * 16;
+
+// Fills TcShared::ep for the kernel's mode (all threads call it, after tc_setup).
+__device__ __forceinline__ void tc_setup_epilogue(const DevCtx& c, const TcState& tc, TcShared& sh, bool gradient) {
+    const int H = c.H, Hp = c.Hp, slice = blockIdx.x % tc.n_split;
+    for (int q = threadIdx.x; q < 8 * TC_EP_LD; q += blockDim.x) {
+        float v = 0.f;
+        const int k = q / TC_EP_LD, j = q % TC_EP_LD;
+        if (gradient) {                                   // W_s[k][column of the callee]
+            const int col = slice * tc.ns[0] + j, cc = col < Hp ? col : col - Hp;
+            if (!c.lstm && j < tc.ns[0] && k < c.n_classes && cc < H) v = c.W_s[k * H + cc];
+        } else if (c.lstm) {                              // [gate][unit] of the slice's 16 units
+            const int g = q / 16, u = slice * 16 + q % 16;
+            if (q < TC_EP_LEAF) { if (u < H) v = c.b[g * H + u]; }
+            else if (q < TC_EP_LEAF + 48) { if (u < H) v = c.b_x[(g - 5) * H + u]; }
+        } else if (k == 0) {
+            const int col = slice * tc.ns[0] + j;
+            if (j < tc.ns[0] && col < H) v = c.b[col];
+        }
+        sh.ep[q] = v;
+    }
+    __syncthreads();
+}
 
 // dynamic shared memory a kernel needs for the given resident slices and ring depth
 inline int tc_smem_bytes(int ns0, int k0, int ns1, int k1, int stages) {
@@ -385,16 +412,15 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                     if (!live) continue;
                     const int cc = e_cc0 + (e_begin + q) * 16;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        if (k < c.n_classes) {
+                    for (int k = 0; k < 8; ++k) {                         // classes beyond the last: zero rows
+                        const float* wk = &sh.ep[k * TC_EP_LD + (e_begin + q) * 16];
 #pragma unroll
-                            for (int i = 0; i < 16; i += 4)
-                                if (cc + i < H) {
-                                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + cc + i]));
-                                    v[i] = fmaf(w.x, dl[k], v[i]); v[i + 1] = fmaf(w.y, dl[k], v[i + 1]);
-                                    v[i + 2] = fmaf(w.z, dl[k], v[i + 2]); v[i + 3] = fmaf(w.w, dl[k], v[i + 3]);
-                                }
+                        for (int i = 0; i < 16; i += 4) {
+                            const float4 w = *reinterpret_cast<const float4*>(wk + i);
+                            v[i] = fmaf(w.x, dl[k], v[i]); v[i + 1] = fmaf(w.y, dl[k], v[i + 1]);
+                            v[i + 2] = fmaf(w.z, dl[k], v[i + 2]); v[i + 3] = fmaf(w.w, dl[k], v[i + 3]);
                         }
+                    }
                     if (child_l == LEAF_MARK) {
                         float* de = c.dE + (size_t)child_tok * c.D + cc;
 #pragma unroll
@@ -425,7 +451,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
 #pragma unroll
                 for (int g = 0; g < NG; ++g) tc_ld8(lane_base + (uint32_t)(g * 16 + wg * 8), v[g]);
                 if (live) {
-                    const float* bias = MODE == TC_LSTM_CELL ? c.b : c.b_x;
+                    const float* bias = MODE == TC_LSTM_CELL ? sh.ep : sh.ep + TC_EP_LEAF;     // [gate][unit of the slice]
                     float cl[8], cr[8], hv[8], cv[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) cl[i] = cr[i] = 0.f;
@@ -446,18 +472,18 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                         float h = 0.f, cc = 0.f;
                         if (u < H) {
                             if (MODE == TC_LSTM_CELL) {
-                                const float gi = tc_sigmoid(v[0][i] + __ldg(&bias[u]));
-                                const float fl = tc_sigmoid(v[1][i] + __ldg(&bias[H + u]));
-                                const float fr = tc_sigmoid(v[2][i] + __ldg(&bias[2 * H + u]));
-                                const float go = tc_sigmoid(v[3 % NG][i] + __ldg(&bias[3 * H + u]));
-                                const float gu = tanhf(v[4 % NG][i] + __ldg(&bias[4 * H + u]));
+                                const float gi = tc_sigmoid(v[0][i] + bias[wg * 8 + i]);
+                                const float fl = tc_sigmoid(v[1][i] + bias[16 + wg * 8 + i]);
+                                const float fr = tc_sigmoid(v[2][i] + bias[32 + wg * 8 + i]);
+                                const float go = tc_sigmoid(v[3 % NG][i] + bias[48 + wg * 8 + i]);
+                                const float gu = tanhf(v[4 % NG][i] + bias[64 + wg * 8 + i]);
                                 cc = gi * gu + fl * cl[i] + fr * cr[i];
                                 h = go * tanhf(cc);
                                 v[0][i] = gi; v[1][i] = fl; v[2][i] = fr; v[3 % NG][i] = go; v[4 % NG][i] = gu;
                             } else {
-                                const float gi = tc_sigmoid(v[0][i] + __ldg(&bias[u]));
-                                const float go = tc_sigmoid(v[1][i] + __ldg(&bias[H + u]));
-                                const float gu = tanhf(v[2][i] + __ldg(&bias[2 * H + u]));
+                                const float gi = tc_sigmoid(v[0][i] + bias[wg * 8 + i]);
+                                const float go = tc_sigmoid(v[1][i] + bias[16 + wg * 8 + i]);
+                                const float gu = tanhf(v[2][i] + bias[32 + wg * 8 + i]);
                                 cc = gi * gu;
                                 h = go * tanhf(cc);
                                 v[0][i] = gi; v[1][i] = go; v[2][i] = gu;
@@ -498,7 +524,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float h = 0.f;
-                            if (col + i < H) h = tanhf(v[i] + __ldg(&c.b[col + i]));
+                            if (col + i < H) h = tanhf(v[i] + sh.ep[gi * 16 + i]);
                             hb[i] = __float2bfloat16_rn(h);
                         }
                         uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
