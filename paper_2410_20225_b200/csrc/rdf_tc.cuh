@@ -263,7 +263,14 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8]) {
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ float tc_sigmoid(float x) { return 1.f / (1.f + expf(-x)); }
+// Activations of the bf16 path: one MUFU instruction each (relative error about 2^-11, below the bf16
+// rounding of the operands they feed).
+__device__ __forceinline__ float tc_tanh(float x) {
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float tc_sigmoid(float x) { return fmaf(0.5f, tc_tanh(0.5f * x), 0.5f); }
 
 // The tile loop over n_items ready operators (see TcMode), 128 rows per tile.  Rows come from
 // cell_items / leaf_items (forward modes) or from cell_ops / leaf_ops at [first ..] (gradient modes).
@@ -476,16 +483,16 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                                 const float fl = tc_sigmoid(v[1][i] + bias[16 + wg * 8 + i]);
                                 const float fr = tc_sigmoid(v[2][i] + bias[32 + wg * 8 + i]);
                                 const float go = tc_sigmoid(v[3 % NG][i] + bias[48 + wg * 8 + i]);
-                                const float gu = tanhf(v[4 % NG][i] + bias[64 + wg * 8 + i]);
+                                const float gu = tc_tanh(v[4 % NG][i] + bias[64 + wg * 8 + i]);
                                 cc = gi * gu + fl * cl[i] + fr * cr[i];
-                                h = go * tanhf(cc);
+                                h = go * tc_tanh(cc);
                                 v[0][i] = gi; v[1][i] = fl; v[2][i] = fr; v[3 % NG][i] = go; v[4 % NG][i] = gu;
                             } else {
                                 const float gi = tc_sigmoid(v[0][i] + bias[wg * 8 + i]);
                                 const float go = tc_sigmoid(v[1][i] + bias[16 + wg * 8 + i]);
-                                const float gu = tanhf(v[2][i] + bias[32 + wg * 8 + i]);
+                                const float gu = tc_tanh(v[2][i] + bias[32 + wg * 8 + i]);
                                 cc = gi * gu;
-                                h = go * tanhf(cc);
+                                h = go * tc_tanh(cc);
                                 v[0][i] = gi; v[1][i] = go; v[2][i] = gu;
                             }
                         }
@@ -524,7 +531,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float h = 0.f;
-                            if (col + i < H) h = tanhf(v[i] + sh.ep[gi * 16 + i]);
+                            if (col + i < H) h = tc_tanh(v[i] + sh.ep[gi * 16 + i]);
                             hb[i] = __float2bfloat16_rn(h);
                         }
                         uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
