@@ -48,19 +48,26 @@ struct __align__(8) LeafItem {
     int32_t  tok;
 };
 
+// A counter that many warps hit with atomics in the same wave, alone on its 128-byte line: atomics on
+// different counters then do not queue up behind each other in one L2 slice, and the polling of a
+// barrier word does not compete with them.
+struct alignas(128) HotCounter {
+    uint32_t v;
+};
+
 // Counters and control words, one 4 KB block at the start of the workspace.
 struct Control {
+    HotCounter qcount[3];         // tokens in the queue of wave w at [w % 3]
+    HotCounter cell_count;        // ready cells queued so far, all waves (length of cell_items)
+    HotCounter leaf_count;        // ready leaves queued so far (length of leaf_items)
+    HotCounter frame_count;
+    HotCounter bar;               // grid barrier arrivals of the scheduler kernel (monotone)
+    HotCounter bar2;              // barrier counter of the backward kernel
+    HotCounter bar_ops;           // barrier counter of the operator kernel
     int32_t  status;
-    uint32_t bar;                 // grid barrier arrivals (monotone)
-    uint32_t qcount[3];           // tokens in the queue of wave w at [w % 3]
-    uint32_t cell_count;          // ready cells queued so far, all waves (length of cell_items)
-    uint32_t leaf_count;          // ready leaves queued so far (length of leaf_items)
-    uint32_t frame_count;
     uint32_t waves, waves_backward, max_wave_tokens, max_probe, max_depth;
     uint32_t all_cells;           // backward: cells seen so far (length of the all-cells list)
     uint32_t all_leaves;          // backward: leaves seen so far
-    uint32_t bar2;                // barrier counter of the backward kernel
-    uint32_t bar_ops;             // barrier counter of the operator kernel
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
@@ -68,6 +75,7 @@ struct Control {
     float    loss;
     int32_t  forward_status;      // status word at the end of the forward pass and the loss head
 };
+static_assert(sizeof(Control) <= 4096, "the control block is 4 KB");
 
 struct DevCtx {
     // lowered program (copied into the workspace at every call)
@@ -172,8 +180,8 @@ __device__ __forceinline__ uint32_t aggregated_inc(uint32_t* counter) {
 // every block has finished wave w and none has begun wave w + 1.
 __device__ __forceinline__ void mark_wave(const DevCtx& c, uint32_t wave) {
     if (c.wave_marks && wave < c.wave_cap)
-        c.wave_marks[wave] = make_uint4(ld_volatile_u32(&c.ctl->frame_count), ld_volatile_u32(&c.ctl->cell_count),
-                                        ld_volatile_u32(&c.ctl->leaf_count), 0u);
+        c.wave_marks[wave] = make_uint4(ld_volatile_u32(&c.ctl->frame_count.v), ld_volatile_u32(&c.ctl->cell_count.v),
+                                        ld_volatile_u32(&c.ctl->leaf_count.v), 0u);
 }
 static const uint32_t NO_MARK = 0xFFFFFFFFu;
 
@@ -220,7 +228,7 @@ __device__ __forceinline__ void store_token(Token* dst_tok, uint64_t tag, int64_
 }
 
 __device__ __forceinline__ void push_token(const DevCtx& c, uint32_t wave, uint64_t tag, int64_t datum, uint32_t pc) {
-    const uint32_t idx = aggregated_inc(&c.ctl->qcount[(wave + 1) % 3]);
+    const uint32_t idx = aggregated_inc(&c.ctl->qcount[(wave + 1) % 3].v);
     if (idx >= c.qcap) {
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
@@ -273,7 +281,7 @@ __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* label
         trace_rec(c, out, arg, 0, label, 0);
         return true;
     }
-    const uint32_t id = aggregated_inc(&c.ctl->frame_count);
+    const uint32_t id = aggregated_inc(&c.ctl->frame_count.v);
     if (id >= c.frame_cap) {
         set_status(c, RDF_ERR_FRAMES_FULL);
         return false;

@@ -43,7 +43,7 @@ __device__ __forceinline__ void load_program(const DevCtx& c, SharedProgram& sp)
 // that carries its state onwards in the next wave.
 __device__ __forceinline__ void fire_cell(const DevCtx& c, const MatchNode& M, uint32_t wave, uint64_t tag,
                                           const int64_t* regs, ThreadStats& st) {
-    const uint32_t i = aggregated_inc(&c.ctl->cell_count);
+    const uint32_t i = aggregated_inc(&c.ctl->cell_count.v);
     if (i >= c.work_cap) {
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
@@ -164,7 +164,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
             }
             case VM_EMBED:
             case VM_LEAF_LSTM: {
-                const uint32_t i = aggregated_inc(&c.ctl->leaf_count);
+                const uint32_t i = aggregated_inc(&c.ctl->leaf_count.v);
                 if (i >= c.work_cap) {
                     set_status(c, RDF_ERR_QUEUE_FULL);
                     return;
@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
         t_mark = now;
     };
     for (;; ++wave) {
-        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
+        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
         if (n == 0) break;
         if (wave >= c.wave_limit) {
             set_status(c, RDF_ERR_WAVE_LIMIT);
@@ -356,7 +356,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
             if (blockIdx.x == 0) {
                 uint32_t m = n, k = 0;
                 do {
-                    if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
+                    if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
                     if (threadIdx.x < m) run_token(c, sp, wave, load_token(&c.q[wave & 1][threadIdx.x]), st);
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
                     if (threadIdx.x == 0) mark_wave(c, wave);
@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                             const uint32_t target = generation * gridDim.x + gridDim.x - 1;
                             const long long t0 = clock64();
                             int good = 1;
-                            while (ld_volatile_u32(&c.ctl->bar) < target) {
+                            while (ld_volatile_u32(&c.ctl->bar.v) < target) {
                                 if (clock64() - t0 > c.spin_limit) {
                                     set_status(c, RDF_ERR_TIMEOUT);
                                     good = 0;
@@ -387,25 +387,25 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                     }
                     ++wave;
                     ++k;
-                    m = ld_volatile_u32(&c.ctl->qcount[wave % 3]);
+                    m = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
                     widest = max(widest, m);
                 } while (m != 0 && m <= blockDim.x && k < NARROW_STRETCH && wave < c.wave_limit &&
                          ld_volatile_i32(&c.ctl->status) == 0);
                 if (threadIdx.x == 0) c.ctl->resume_wave = wave;
             }
             lap(cyc_s);
-            if (!grid_barrier(c, &c.ctl->bar, generation)) break;
+            if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
             lap(cyc_b);
             wave = ld_volatile_u32(&c.ctl->resume_wave) - 1;      // the loop header adds the one back
             continue;
         }
-        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3] = 0;
+        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
         const Token* q = c.q[wave & 1];
         for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
             run_token(c, sp, wave, load_token(&q[i]), st);
         __syncthreads();
         lap(cyc_s);
-        if (!grid_barrier(c, &c.ctl->bar, generation, wave)) break;
+        if (!grid_barrier(c, &c.ctl->bar.v, generation, wave)) break;
         lap(cyc_b);
     }
     flush_stats(c, st);
@@ -434,8 +434,8 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     }
     store_token(&c.q[0][b], tag, datum, (uint32_t)c.result_entry_pc);
     if (b == 0) {
-        c.ctl->qcount[0] = (uint32_t)c.B;
-        c.ctl->frame_count = c.tag_mode == RDF_TAGS_FRAME ? (uint32_t)c.B : 0u;
+        c.ctl->qcount[0].v = (uint32_t)c.B;
+        c.ctl->frame_count.v = c.tag_mode == RDF_TAGS_FRAME ? (uint32_t)c.B : 0u;
     }
 }
 
@@ -461,7 +461,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         t_mark = now;
     };
     const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
-    const uint32_t n_leaf = min(c.ctl->leaf_count, c.work_cap);
+    const uint32_t n_leaf = min(c.ctl->leaf_count.v, c.work_cap);
     bool alive = true;
     if (n_leaf) {
         if constexpr (TC) {
@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         }
         __syncthreads();
         lap(cyc_c);
-        alive = grid_barrier(c, &c.ctl->bar_ops, generation);
+        alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
     uint32_t first = 0;
@@ -494,7 +494,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         first = end;
         __syncthreads();
         lap(cyc_c);
-        alive = grid_barrier(c, &c.ctl->bar_ops, generation);
+        alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
     if constexpr (TC) tc_teardown(tc);

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_kernel(const DevCtx c, int
     __shared__ __align__(16) float s_dl[LH_MAX_ROWS][8];
     __shared__ int s_lab[2][LH_MAX_ROWS];
     __shared__ float warp_loss[8];
-    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
+    const uint32_t F = c.ctl->frame_count.v, B = (uint32_t)c.B;
     const uint32_t n = F > B ? F - B : 0u, per = (n + gridDim.x - 1) / gridDim.x;
     const uint32_t f0 = min(F, B + blockIdx.x * per), f1 = min(F, f0 + per);
     const int n_slabs = (int)((f1 - f0 + fr - 1) / fr);
@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
     __shared__ __align__(16) float s_dl[LM_ROWS][8];
     __shared__ int s_lab[2][LM_ROWS];
     __shared__ float warp_loss[8];
-    const uint32_t F = c.ctl->frame_count, B = (uint32_t)c.B;
+    const uint32_t F = c.ctl->frame_count.v, B = (uint32_t)c.B;
     const uint32_t n = F > B ? F - B : 0u, per = (n + gridDim.x - 1) / gridDim.x;
     const uint32_t f0 = min(F, B + blockIdx.x * per), f1 = min(F, f0 + per);
     const int n_slabs = (int)((f1 - f0 + LM_ROWS - 1) / LM_ROWS);
@@ -438,7 +438,7 @@ __device__ __forceinline__ void list_flags(const DevCtx& c, uint32_t f0, uint32_
 
 __global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uint2* seg_counts) {
     __shared__ uint32_t wc[8], wl[8];
-    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
     uint32_t l[8], r[8], cells, leaves;
     list_flags(c, f0, F, l, r, cells, leaves);
     for (int o = 16; o > 0; o >>= 1) {
@@ -489,7 +489,7 @@ __global__ void __launch_bounds__(1024) rdf_list_scan_kernel(const DevCtx c, uin
 
 __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, const uint2* seg_base) {
     __shared__ uint32_t wc[8], wl[8];
-    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
     uint32_t l[8], r[8], cells, leaves;
     list_flags(c, f0, F, l, r, cells, leaves);
     // exclusive prefix of (cells, leaves) over the threads of the block
@@ -526,7 +526,7 @@ __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, cons
 __global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, const uint2* seg_base) {
     const uint32_t lane = threadIdx.x % 32, n_warps = gridDim.x * blockDim.x / 32;
     const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
-    const uint32_t F = min(c.ctl->frame_count, c.frame_cap), B = (uint32_t)c.B;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
     for (uint32_t d = (blockIdx.x * blockDim.x + threadIdx.x) / 32; d < n_waves; d += n_warps) {
         const uint32_t f = max(B, min(c.wave_marks[d].x, F));
         const uint32_t seg = (f - B) / LIST_SEG, s0 = B + seg * LIST_SEG;      // (the segment array has one entry to spare)
@@ -867,7 +867,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             }
             __syncthreads();
             lap(cyc_a);
-            if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+            if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
             lap(cyc_b);
         }
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
@@ -885,7 +885,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             first = end;
             __syncthreads();
             lap(cyc_c);
-            if (!grid_barrier(c, &c.ctl->bar2, generation)) break;
+            if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
             lap(cyc_b);
         }
     }
