@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_kernel(const DevCtx c, int
     }
 }
 
-// ---- the same pass for the bf16 TreeRNN, with the two small contractions on the tensor cores
+// ---- the same pass for the bf16 workloads (rows = the bf16 h of arena_bf), with the two small contractions on the tensor cores
 // (warp-level mma.sync m16n8k16: the shapes are [64 rows x Hp] x [Hp x 8 classes] and [Hp x 64 rows] x [64 x 8],
 // far too small for a tcgen05 tile).  States are bf16 already; W_s and dlog enter as a bf16 pair hi + lo
 // (two MMAs), so the products carry about 16 mantissa bits and the sums are fp32.
@@ -662,6 +662,7 @@ __device__ __forceinline__ void lstm_backward_frame(const DevCtx& c, uint32_t t,
         // 128-bit accesses: four hidden units per lane and step
         auto ld = [](const float* p) { const float4 v = ldcg4(p); return v; };
         auto st4 = [](float* p, const float (&v)[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); };
+        const bool keep_f32 = c.dg_bf == nullptr;       // bf16 path: the gate gradients live on as bf16 operand rows only
         auto stb = [&](int gate, int j, const float (&v)[4]) {
             if (!c.dg_bf) return;
             __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
@@ -694,7 +695,7 @@ __device__ __forceinline__ void lstm_backward_frame(const DevCtx& c, uint32_t t,
                     g1[e] = dh[e] * tc * go[e] * (1.f - go[e]);
                     g2[e] = dc * gi[e] * (1.f - gu[e] * gu[e]);
                 }
-                st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2);
+                if (keep_f32) { st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2); }
                 stb(0, j, g0); stb(1, j, g1); stb(2, j, g2);
             } else {
                 const float4 a4 = ld(gt + j), l4 = ld(gt + H + j), r4 = ld(gt + 2 * H + j), o4 = ld(gt + 3 * H + j), u4 = ld(gt + 4 * H + j);
@@ -715,7 +716,7 @@ __device__ __forceinline__ void lstm_backward_frame(const DevCtx& c, uint32_t t,
                     dl_[e] = dc * fl[e];
                     dr_[e] = dc * fr[e];
                 }
-                st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2); st4(gt + 3 * H + j, g3); st4(gt + 4 * H + j, g4);
+                if (keep_f32) { st4(gt + j, g0); st4(gt + H + j, g1); st4(gt + 2 * H + j, g2); st4(gt + 3 * H + j, g3); st4(gt + 4 * H + j, g4); }
                 stb(0, j, g0); stb(1, j, g1); stb(2, j, g2); stb(3, j, g3); stb(4, j, g4);
                 st4(c.dhp + (size_t)l * S + H + j, dl_);
                 st4(c.dhp + (size_t)r * S + H + j, dr_);
@@ -960,21 +961,23 @@ __global__ void __launch_bounds__(256) rdf_outer_kernel(const DevCtx c, const Ou
     }
 }
 
-// out[m] = sum over the listed invocations of A_t[m]   (bias gradients)
+// out[g * H + u] = sum over the listed invocations of A_t[g * Hb + u]   (bias gradients; Hb = H for
+// fp32 rows, the padded Hp for the bf16 operand rows)
 __device__ __forceinline__ float as_float(float v) { return v; }
 __device__ __forceinline__ float as_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
 template <typename T>
 __global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, const uint32_t* count, const T* A,
-                                                         int lda, int M, float* out) {
+                                                         int lda, int M, int H, int Hb, float* out) {
     const uint32_t n = *count;
     const uint32_t per = (n + gridDim.x - 1) / gridDim.x;
     const uint32_t t0 = blockIdx.x * per, t1 = min(n, t0 + per);
     if (t0 >= t1) return;
     for (int j = threadIdx.x; j < M; j += blockDim.x) {
+        const int col = (j / H) * Hb + j % H;
         float s = 0.f;
 #pragma unroll 8
-        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)list[i] * lda + j]);
+        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)list[i] * lda + col]);
         atomicAdd(&out[j], s);
     }
 }
@@ -1088,8 +1091,8 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         const int fr = std::max(1, std::min(LH_MAX_ROWS, LH_SLAB_BYTES / rowbytes));
         const int smem = 2 * fr * rowbytes + params->n_classes * H * (int)sizeof(float);
         const int loss_blocks = std::min(4096, 2 * S->grid);
-        if (tc_rnn) {
-            const int smem_mma = 2 * LM_ROWS * (rowbytes + 16);
+        if (c.use_tc) {                    // bf16 states (TreeRNN and TreeLSTM): the h rows of arena_bf
+            const int smem_mma = 2 * LM_ROWS * (c.Hp * 2 + 16);
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mma));
             rdf_loss_heads_mma_kernel<<<loss_blocks, 256, smem_mma, stream>>>(c);
         } else {
@@ -1156,9 +1159,14 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 6, stream);
-    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, grads->db);
-    else rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, grads->db);
-    if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, grads->db_x);
+    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);
+    else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
+        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
+        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);
+    } else {
+        rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, H, H, grads->db);
+        if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, H, H, grads->db_x);
+    }
     rdf_mark(S, 7, stream);       // (dW_s and db_s came from the loss-head pass)
     if (tc_lstm) {
         const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 5);
