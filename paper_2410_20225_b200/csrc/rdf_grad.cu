@@ -1128,11 +1128,11 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     const float* dgA = lstm ? c.gates : c.dhp;
     const int lda = lstm ? c.G : H;
     if (c.use_tc) {
-        // 128 x 128 tiles of the padded gradient, the invocations split over the remaining blocks
+        // 256 x 256 tiles of the padded gradient, the invocations split over the remaining blocks
         CUDA_OK(cudaFuncSetAttribute(rdf_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BYTES));
         auto launch_dw = [&](DwArgs a, long long max_items) {
-            a.tiles_n = (a.Np + 127) / 128;
-            a.n_tiles = ((a.Mp + 127) / 128) * a.tiles_n;
+            a.tiles_n = (a.Np + DW_TILE - 1) / DW_TILE;
+            a.n_tiles = ((a.Mp + DW_TILE - 1) / DW_TILE) * a.tiles_n;
             const int splits = std::max(1, S->grid / a.n_tiles);
             uint32_t chunk = (uint32_t)((max_items + splits - 1) / splits);
             a.chunk = (chunk + DW_KT - 1) / DW_KT * DW_KT;

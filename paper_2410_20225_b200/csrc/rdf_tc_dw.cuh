@@ -1,18 +1,22 @@
-// Weight gradient of the TreeRNN cell on tensor cores:
+// Weight gradient of the cells on tensor cores:
 //     dW[j][k] = sum over cells t of dz_t[j] * x_t[k],      x_t = [h(l_t) ; h(r_t)]
 // The contraction runs over the cells, and both operands are stored with the
 // contracted index outermost (dz_bf[t][j], arena_bf[.][k]): the "MN-major"
-// operand form.  A stage holds 64 cells: for A, two 64-wide groups of j, for B
-// two 64-wide groups of k, each as 8 atoms of (8 cells x 128 bytes) with the
-// 128-byte swizzle.  Each thread block owns one 128 x 128 tile of dW and a
-// range of the cells (split-K); partial tiles are added to dW with atomics.
+// operand form.  A stage holds 64 cells: for each operand four 64-wide groups
+// of j (of k), each as 8 atoms of (8 cells x 128 bytes) with the 128-byte
+// swizzle.  Each thread block owns one 256 x 256 tile of dW (two 128-row
+// accumulators: all 512 columns of tensor memory) and a range of the cells
+// (split-K); partial tiles are added to dW with atomics.  The large tile is
+// what keeps the gather small: an operand row is fetched once per tile that
+// needs it, and the gather (16-byte cp.async pieces) is what bounds the kernel.
 #pragma once
 #include "rdf_tc.cuh"
 
 static const int DW_KT = 64;                          // cells per stage
-static const int DW_HALF = DW_KT * 256;               // 16 KB: one operand of a stage
+static const int DW_TILE = 256;                       // rows and columns of dW per block
+static const int DW_HALF = DW_KT * DW_TILE * 2;       // 32 KB: one operand of a stage
 static const int DW_STAGE = 2 * DW_HALF;
-static const int DW_STAGES = 6;
+static const int DW_STAGES = 3;
 static const int DW_SMEM_BYTES = 1024 + DW_STAGES * DW_STAGE;
 static const int DW_PRODUCERS = 128;                  // warps 0-3 gather, warp 4 issues the MMAs, all 8 warps write out
 
@@ -48,12 +52,14 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
     extern __shared__ unsigned char dyn_smem[];
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(8) uint64_t full[DW_STAGES], empty[DW_STAGES], done;
+    __shared__ uint4 s_ops[2][DW_KT];                              // records of the stage being copied / the next one
+    __shared__ int s_abort;                                        // a producer's bounded wait expired: all producers leave together
     const uint32_t n_cells = *a.count;
     const int tile = blockIdx.x % a.n_tiles, split = blockIdx.x / a.n_tiles;
     const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_cells, t_begin + a.chunk);
     if (t_begin >= t_end) return;                                  // the whole block leaves before any set-up
     const int H = c.H, Hp = c.Hp;
-    const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
+    const int m0 = (tile / a.tiles_n) * DW_TILE, n0 = (tile % a.tiles_n) * DW_TILE;
     const uint32_t n_chunks = (t_end - t_begin + DW_KT - 1) / DW_KT;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -66,10 +72,11 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(done0, 1);
+        s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < 32) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;" ::"r"(smem_u32(&tmem_slot)) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_slot)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -78,29 +85,27 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
     bool ok = true;
     if (warp < 4) {
-        // ---- producers: a thread copies one 16-byte piece (q) of eight cells (tr0 + 8 i) of both operands per stage
-        const int q = threadIdx.x & 15, tr0 = threadIdx.x >> 4, atom = q >> 3, c16 = q & 7;
+        // ---- producers: a thread copies one 16-byte piece (q) of sixteen cells (tr0 + 4 i) of both operands per stage
+        const int q = threadIdx.x & 31, tr0 = threadIdx.x >> 5, atom = q >> 3, c16 = q & 7;
         const int m = m0 + atom * 64 + c16 * 8, n = n0 + atom * 64 + c16 * 8;
         const bool m_in = m < a.Mp, n_in = n < a.Np;
         const __nv_bfloat16* Brows = a.mode == 0 ? c.arena_bf : c.E_bf;
-        auto load_ops = [&](uint32_t kc, uint4 (&ops)[8]) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t idx = t_begin + kc * DW_KT + tr0 + 8 * i;
-                ops[i] = idx < t_end ? a.ops[idx] : make_uint4(0u, 0u, 0u, 0u);
-            }
+        auto load_op = [&](uint32_t kc) {                          // the record of cell threadIdx.x of stage kc
+            const uint32_t idx = t_begin + kc * DW_KT + threadIdx.x;
+            return threadIdx.x < DW_KT && kc < n_chunks && idx < t_end ? a.ops[idx] : make_uint4(0u, 0u, 0u, 0u);
         };
-        uint4 ops[8], ops_next[8];
-        load_ops(0, ops);
-        for (uint32_t kc = 0; kc < n_chunks && ok; ++kc) {
+        if (threadIdx.x < DW_KT) s_ops[0][threadIdx.x] = load_op(0);
+        uint4 op_next = load_op(1);
+        asm volatile("bar.sync 1, 128;" ::: "memory");             // the producer warps only
+        for (uint32_t kc = 0; kc < n_chunks; ++kc) {
             const uint32_t s = kc % DW_STAGES;
-            if (kc + 1 < n_chunks) load_ops(kc + 1, ops_next);                 // in flight during this stage
             if (kc >= (uint32_t)DW_STAGES) ok = mbar_wait(c, empty0 + 8 * s, ((kc / DW_STAGES) - 1) & 1u);
+            if (!ok) s_abort = 1;
             const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int tr = tr0 + 8 * i;
-                const uint4 it = ops[i];
+#pragma unroll 4
+            for (int i = 0; ok && i < DW_KT / 4; ++i) {
+                const int tr = tr0 + 4 * i;
+                const uint4 it = s_ops[kc & 1][tr];
                 const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
                 const bool mv = it.w != 0u && m_in;
                 cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
@@ -109,14 +114,16 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
                 if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
                 cp_async16(b_st + off, Brows + src, nv);
             }
-            cp_async_arrive(full0 + 8 * s);                    // arrives when this thread's copies of the stage have landed
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ops[i] = ops_next[i];
+            if (ok) cp_async_arrive(full0 + 8 * s);            // arrives when this thread's copies of the stage have landed
+            if (threadIdx.x < DW_KT) s_ops[(kc + 1) & 1][threadIdx.x] = op_next;
+            op_next = load_op(kc + 2);                         // in flight during the next stage
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*reinterpret_cast<volatile int*>(&s_abort)) break;   // the same answer for all producers
         }
     } else if (warp == 4) {
-        // ---- MMA issuer
+        // ---- MMA issuer: two 128-row accumulators of 256 columns
         if (lane == 0) {
-            const uint32_t idesc = tc_idesc(128) | (1u << 15) | (1u << 16);        // both operands MN-major
+            const uint32_t idesc = tc_idesc(DW_TILE) | (1u << 15) | (1u << 16);    // both operands MN-major
             for (uint32_t kc = 0; kc < n_chunks && ok; ++kc) {
                 const uint32_t s = kc % DW_STAGES;
                 ok = mbar_wait(c, full0 + 8 * s, (kc / DW_STAGES) & 1u);
@@ -126,8 +133,10 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
                 const uint32_t a_st = stage0 + s * DW_STAGE, b_st = a_st + DW_HALF;
 #pragma unroll
                 for (int ks = 0; ks < DW_KT / 16; ++ks)          // 16 invocations = two K atoms = 2048 bytes per step
-                    tc_mma(tmem, tc_desc_mn(a_st + ks * 2048, lbo, sbo), tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc,
-                           (kc > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tc_mma(tmem + h * DW_TILE, tc_desc_mn(a_st + h * 16384 + ks * 2048, lbo, sbo),
+                               tc_desc_mn(b_st + ks * 2048, lbo, sbo), idesc, (kc > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(empty0 + 8 * s);
             }
             if (ok) tc_commit(done0);
@@ -138,23 +147,25 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
     ok = mbar_wait(c, done0, 0u);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
-        const int m = m0 + (warp & 3) * 32 + lane;
-        const int mj = m % Hp, row = (m / Hp) * H + mj;              // gate block, unit
         const int n_limit = a.mode == 0 ? H : c.D;
-        for (int gi = 0; gi < 4; ++gi) {
-            float v[16];
-            const int cl = (warp >> 2) * 64 + gi * 16;
-            tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)cl, v);
-            if (m >= a.Mp || mj >= H) continue;
+        for (int h = 0; h < 2; ++h) {
+            const int m = m0 + h * 128 + (warp & 3) * 32 + lane;
+            const int mj = m % Hp, row = (m / Hp) * H + mj;          // gate block, unit
+            for (int gi = 0; gi < 8; ++gi) {
+                float v[16];
+                const int cl = (warp >> 2) * 128 + gi * 16;
+                tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(h * DW_TILE + cl), v);
+                if (m >= a.Mp || mj >= H || n0 + cl >= a.Np) continue;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int n = n0 + cl + i;
-                const int k = n < Hp ? n : n - Hp;
-                if (n < a.Np && k < n_limit) atomicAdd(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)], v[i]);
+                for (int i = 0; i < 16; ++i) {
+                    const int n = n0 + cl + i;
+                    const int k = n < Hp ? n : n - Hp;
+                    if (n < a.Np && k < n_limit) atomicAdd(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)], v[i]);
+                }
             }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;" ::"r"(tmem) : "memory");
+    if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
