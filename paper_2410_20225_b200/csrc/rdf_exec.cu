@@ -246,7 +246,10 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, ui
 // a handful of blocks busy with a long dependent k-loop.  Here one block step computes an 8 cell x 16
 // column patch with the whole contraction spread over its threads: thread = (cell, column, half of k),
 // streaming its operand row and weight row with independent 128-bit loads.
-__device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t first, uint32_t n_items) {
+// wres: this block's resident 16 columns of W in shared memory (or nullptr), as float4 [k / 4][column]:
+// the 16 columns of the column group blockIdx.x % units_n, which is the group of every patch the block
+// gets while a wave has no more patches than blocks.
+__device__ void rnn_cell_thin(const DevCtx& c, float* xs, const float4* wres, uint32_t first, uint32_t n_items) {
     // xs: shared staging for the 8 operand rows [h_l ; h_r] of the patch (8 x 2H floats) + 128 floats
     const int H = c.H, K2 = 2 * c.H;
     float* red = xs + 8 * K2;
@@ -270,13 +273,23 @@ __device__ void rnn_cell_thin(const DevCtx& c, float* xs, uint32_t first, uint32
         float acc = 0.f;
         if (live) {
             const float4* x = reinterpret_cast<const float4*>(xs + rr * K2 + kh * H);
-            const float4* w = reinterpret_cast<const float4*>(c.W + (size_t)col * K2 + kh * H);   // L1-resident across waves
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            if (wres && unit % units_n == (int)(blockIdx.x % units_n)) {
+                const float4* w = wres + (size_t)(kh * (H / 4)) * 16 + cc;          // lanes: consecutive columns, no bank conflicts
 #pragma unroll 8
-            for (int k4 = 0; k4 < H / 4; ++k4) {
-                const float4 xv = x[k4], wv = __ldg(w + k4);
-                a0 = fmaf(xv.x, wv.x, a0); a1 = fmaf(xv.y, wv.y, a1);
-                a2 = fmaf(xv.z, wv.z, a2); a3 = fmaf(xv.w, wv.w, a3);
+                for (int k4 = 0; k4 < H / 4; ++k4) {
+                    const float4 xv = x[k4], wv = w[k4 * 16];
+                    a0 = fmaf(xv.x, wv.x, a0); a1 = fmaf(xv.y, wv.y, a1);
+                    a2 = fmaf(xv.z, wv.z, a2); a3 = fmaf(xv.w, wv.w, a3);
+                }
+            } else {
+                const float4* w = reinterpret_cast<const float4*>(c.W + (size_t)col * K2 + kh * H);
+#pragma unroll 8
+                for (int k4 = 0; k4 < H / 4; ++k4) {
+                    const float4 xv = x[k4], wv = __ldg(w + k4);
+                    a0 = fmaf(xv.x, wv.x, a0); a1 = fmaf(xv.y, wv.y, a1);
+                    a2 = fmaf(xv.z, wv.z, a2); a3 = fmaf(xv.w, wv.w, a3);
+                }
             }
             acc = (a0 + a1) + (a2 + a3);
         }
@@ -453,6 +466,20 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         else tc_setup(tc, smem, dyn_smem, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
         tc_setup_epilogue(c, tc, smem, false);
     }
+    // fp32 TreeRNN, narrow waves: this block's 16 columns of W stay in shared memory for all waves
+    const float4* wres = nullptr;
+    if constexpr (!TC) {
+        if (!c.lstm && c.H <= THIN_RESIDENT_MAX_H) {
+            float4* wr = reinterpret_cast<float4*>(dyn_smem);
+            const int K2 = 2 * c.H, units_n = (c.H + 15) / 16, cg0 = blockIdx.x % units_n;
+            for (int q = threadIdx.x; q < (K2 / 4) * 16; q += blockDim.x) {
+                const int k4 = q / 16, col = cg0 * 16 + q % 16;
+                wr[q] = col < c.H ? __ldg(reinterpret_cast<const float4*>(c.W + (size_t)col * K2) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            __syncthreads();
+            wres = wr;
+        }
+    }
     uint32_t generation = 0;
     long long cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
@@ -488,7 +515,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
             if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
             // thin patches while they fit in two rounds over the grid, tiles for wide waves
             else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
-                rnn_cell_thin(c, reinterpret_cast<float*>(&smem), first, nc);      // 8 x 2H + 128 floats <= 26 KB
+                rnn_cell_thin(c, reinterpret_cast<float*>(&smem), wres, first, nc);      // 8 x 2H + 128 floats <= 26 KB
             else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
         }
         first = end;
@@ -628,7 +655,8 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<true>, TC_THREADS, max_dyn));
     if (per_sm < 1) return RDF_ERR_CUDA;
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 0));
+    CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 128 * THIN_RESIDENT_MAX_H));
     if (per_sm < 1) return RDF_ERR_CUDA;
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 0));
     if (per_sm < 1) return RDF_ERR_CUDA;
@@ -764,7 +792,8 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
             CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
                                                 (size_t)L.tc_smem_fwd, stream));
         else
-            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), args, 0, stream));
+            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), args,
+                                                thin_resident_bytes(c.lstm, c.H), stream));
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());
     }

@@ -34,6 +34,11 @@ __device__ __forceinline__ void gemm_tile_step(const GemmSmem& sm, int tx, int t
     }
 }
 
+// fp32 TreeRNN, narrow waves: a block keeps its 16 (forward) / 32 (gradient) columns of W in shared memory,
+// 128 * H bytes, while that fits beside the tiles
+static const int THIN_RESIDENT_MAX_H = 384;
+inline size_t thin_resident_bytes(int lstm, int H) { return !lstm && H <= THIN_RESIDENT_MAX_H ? (size_t)128 * H : 0; }
+
 // ---- host state
 struct ExecState {
     int device = -1;

@@ -778,7 +778,9 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
 
 // Narrow waves: an 8 cell x 32 column patch of [dh_l ; dh_r] = W^T dz per block step;
 // thread = (cell, 4 columns, quarter of the contraction over j).
-__device__ void backward_operand_thin(const DevCtx& c, float* zs, uint32_t first, uint32_t n_items) {
+// wres: this block's resident 32 columns of W in shared memory (or nullptr) as float4 [j][4-column group],
+// the columns of the column group blockIdx.x % units_n.
+__device__ void backward_operand_thin(const DevCtx& c, float* zs, const float4* wres, uint32_t first, uint32_t n_items) {
     // zs: shared staging for the 8 dz rows of the patch (8 x H floats) followed by 768 floats of partial sums
     const int H = c.H, K2 = 2 * c.H;
     float* red = zs + 8 * H;
@@ -800,12 +802,22 @@ __device__ void backward_operand_thin(const DevCtx& c, float* zs, uint32_t first
         if (live) {
             const float* dz = zs + rr * H;
             const int j0 = jq * jlen, j1 = min(H, j0 + jlen);
+            if (wres && unit % units_n == (int)(blockIdx.x % units_n)) {
 #pragma unroll 8
-            for (int j = j0; j < j1; ++j) {
-                const float d = dz[j];
-                const float4 w = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col));   // L1-resident across waves
-                acc.x = fmaf(d, w.x, acc.x); acc.y = fmaf(d, w.y, acc.y);
-                acc.z = fmaf(d, w.z, acc.z); acc.w = fmaf(d, w.w, acc.w);
+                for (int j = j0; j < j1; ++j) {
+                    const float d = dz[j];
+                    const float4 w = wres[j * 8 + c4];
+                    acc.x = fmaf(d, w.x, acc.x); acc.y = fmaf(d, w.y, acc.y);
+                    acc.z = fmaf(d, w.z, acc.z); acc.w = fmaf(d, w.w, acc.w);
+                }
+            } else {
+#pragma unroll 8
+                for (int j = j0; j < j1; ++j) {
+                    const float d = dz[j];
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col));
+                    acc.x = fmaf(d, w.x, acc.x); acc.y = fmaf(d, w.y, acc.y);
+                    acc.z = fmaf(d, w.z, acc.z); acc.w = fmaf(d, w.w, acc.w);
+                }
             }
         }
         if (jq > 0) *reinterpret_cast<float4*>(red + ((jq - 1) * 64 + o) * 4) = acc;
@@ -834,6 +846,20 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         if (c.lstm) tc_setup(tc, smem, dyn_smem, 2 * c.Hp / 32, c.WTp, 5 * c.Hp, 32);
         else tc_setup(tc, smem, dyn_smem, 8, c.WTp, c.Hp, c.Hp / 4);
         tc_setup_epilogue(c, tc, smem, true);
+    }
+    // fp32 TreeRNN, narrow waves: this block's 32 columns of W stay in shared memory for all waves
+    const float4* wres = nullptr;
+    if constexpr (!TC) {
+        if (!c.lstm && c.H <= THIN_RESIDENT_MAX_H) {
+            float4* wr = reinterpret_cast<float4*>(dyn_smem);
+            const int K2 = 2 * c.H, units_n = (K2 + 31) / 32, cg0 = blockIdx.x % units_n;
+            for (int q = threadIdx.x; q < c.H * 8; q += blockDim.x) {
+                const int j = q / 8, col = cg0 * 32 + (q % 8) * 4;
+                wr[q] = col < K2 ? __ldg(reinterpret_cast<const float4*>(c.W + (size_t)j * K2 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            __syncthreads();
+            wres = wr;
+        }
     }
     const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, n_warps = blockDim.x / 32;
     uint32_t generation = 0, wave = 0, first = 0;
@@ -880,7 +906,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             } else {
                 if (c.lstm) backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.gates, c.G, 5 * c.H);
                 else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
-                    backward_operand_thin(c, reinterpret_cast<float*>(&smem), first, end - first);   // 8 x H + 768 floats <= 26 KB
+                    backward_operand_thin(c, reinterpret_cast<float*>(&smem), wres, first, end - first);   // 8 x H + 768 floats <= 26 KB
                 else backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.dhp, c.H, c.H);
             }
             first = end;
@@ -1119,7 +1145,9 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
                                             (size_t)L.tc_smem_bwd, stream));
     } else {
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args, 0, stream));
+        CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
+        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
+                                            thin_resident_bytes(c.lstm, c.H), stream));
     }
     rdf_mark(S, 5, stream);
     // parameter gradients
