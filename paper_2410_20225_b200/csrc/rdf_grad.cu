@@ -777,18 +777,30 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
 }
 
 // Narrow waves: an 8 cell x 32 column patch of [dh_l ; dh_r] = W^T dz per block step;
-// thread = (cell, 4 columns, quarter of the contraction over j).
+// thread = (cell, 4 columns, quarter of the contraction over j).  The thread that ends up with the four
+// sums finishes the callee they belong to right away (what the per-invocation pass would do one wave
+// later): dh += W_s^T dlog; a cell callee gets dz = dh (1 - h^2) in place of its incoming gradient, a leaf
+// callee adds dh to dE[tok].  What it needs of the callee is fetched before the contraction starts.
 // wres: this block's resident 32 columns of W in shared memory (or nullptr) as float4 [j][4-column group],
 // the columns of the column group blockIdx.x % units_n.
 __device__ void backward_operand_thin(const DevCtx& c, float* zs, const float4* wres, uint32_t first, uint32_t n_items) {
-    // zs: shared staging for the 8 dz rows of the patch (8 x H floats) followed by 768 floats of partial sums
-    const int H = c.H, K2 = 2 * c.H;
+    // zs: shared staging for the 8 dz rows of the patch (8 x H floats), 768 floats of partial sums, 8 records
+    const int H = c.H, K2 = 2 * c.H, C = c.n_classes;
     float* red = zs + 8 * H;
+    uint4* s_rec = reinterpret_cast<uint4*>(red + 768);                    // {cell, left callee, right callee, valid}
     const int units_n = (K2 + 31) / 32, units = ((n_items + 7) / 8) * units_n;
     const int o = threadIdx.x & 63, jq = threadIdx.x >> 6, rr = o >> 3, c4 = o & 7;
     const int jlen = (H + 3) / 4;
     for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
         const int row0 = (unit / units_n) * 8;
+        if (threadIdx.x < 8) {
+            uint4 rec = make_uint4(0u, 0u, 0u, 0u);
+            if (row0 + (int)threadIdx.x < (int)n_items) {
+                rec.x = __ldcg(&c.all_cells[first + row0 + threadIdx.x]);
+                rec.y = c.op_l[rec.x]; rec.z = c.op_r[rec.x]; rec.w = 1u;
+            }
+            s_rec[threadIdx.x] = rec;
+        }
         for (int p = threadIdx.x; p < 8 * (H / 4); p += blockDim.x) {
             const int r = p / (H / 4), k = (p % (H / 4)) * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -798,6 +810,18 @@ __device__ void backward_operand_thin(const DevCtx& c, float* zs, const float4* 
         __syncthreads();
         const int row = row0 + rr, col = (unit % units_n) * 32 + c4 * 4;
         const bool live = row < (int)n_items && col < K2;
+        // the callee this thread will finish, fetched while the contraction runs
+        const int cc = col < H ? col : col - H;
+        uint32_t child = 0, child_l = LEAF_MARK, child_tok = 0;
+        float4 d0 = make_float4(0.f, 0.f, 0.f, 0.f), d1 = d0, hv = d0;
+        if (jq == 0 && live) {
+            const uint4 rec = s_rec[rr];
+            child = col < H ? rec.y : rec.z;
+            child_l = c.op_l[child]; child_tok = c.op_r[child];
+            d0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
+            d1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
+            hv = *reinterpret_cast<const float4*>(c.arena + (size_t)child * H + cc);
+        }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live) {
             const float* dz = zs + rr * H;
@@ -828,9 +852,21 @@ __device__ void backward_operand_thin(const DevCtx& c, float* zs, const float4* 
                 const float4 p = *reinterpret_cast<const float4*>(red + (q * 64 + o) * 4);
                 acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
             }
-            const uint32_t t = __ldcg(&c.all_cells[first + row]);
-            const uint32_t child = col < H ? __ldcg(&c.op_l[t]) : __ldcg(&c.op_r[t]);
-            *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + (col < H ? col : col - H)) = acc;
+            const float dl[MAX_CLASSES] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+            for (int k = 0; k < MAX_CLASSES; ++k)
+                if (k < C) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(&c.W_s[k * H + cc]));
+                    acc.x = fmaf(w.x, dl[k], acc.x); acc.y = fmaf(w.y, dl[k], acc.y);
+                    acc.z = fmaf(w.z, dl[k], acc.z); acc.w = fmaf(w.w, dl[k], acc.w);
+                }
+            if (child_l == LEAF_MARK) {
+                atomicAdd(reinterpret_cast<float4*>(c.dE + (size_t)child_tok * c.D + cc), acc);
+            } else {
+                acc.x *= 1.f - hv.x * hv.x; acc.y *= 1.f - hv.y * hv.y;
+                acc.z *= 1.f - hv.z * hv.z; acc.w *= 1.f - hv.w * hv.w;
+                *reinterpret_cast<float4*>(c.dhp + (size_t)child * H + cc) = acc;
+            }
         }
         __syncthreads();
     }
@@ -873,14 +909,16 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     // handed out in wave order, so they are the range [f0, f1) and their rows are consecutive in memory.
     const uint32_t n_fwd = min(c.ctl->waves, c.wave_cap);
     uint32_t f1 = (uint32_t)c.B;
+    bool callees_done = false;        // the previous wave's contraction has already finished this wave's invocations
     for (uint32_t d = 0; d < n_fwd; ++d) {
         const uint32_t f0 = f1;
         f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
         if (f1 == f0) continue;                                      // a wave without calls
         ++wave;
         // ---- A: per-invocation work, a contiguous piece of the range per block.  (bf16 TreeRNN: only the
-        //      invocations called from `result` -- further down the epilogue of B does this work for the callees.)
-        if (!(TC && !c.lstm && d > 0)) {
+        //      invocations called from `result` -- further down the epilogue of B does this work for the callees;
+        //      fp32 TreeRNN: not after a wave of narrow patches, which do the same.)
+        if (!(TC && !c.lstm && d > 0) && !callees_done) {
             const uint32_t n = f1 - f0;
             const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
             const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
@@ -899,15 +937,17 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         }
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
         const uint32_t end = max(first, min(c.wave_marks[d].w, c.frame_cap));     // the wave's cells: all_cells[first, end)
+        bool thin = false;
         if (end > first) {
             if constexpr (TC) {
                 if (c.lstm) tc_pipe<TC_LSTM_BWD, TC_STAGES_LSTM_BWD>(c, tc, smem, first, end - first);
                 else tc_pipe<TC_RNN_BWD, TC_STAGES_RNN_BWD>(c, tc, smem, first, end - first);
             } else {
                 if (c.lstm) backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.gates, c.G, 5 * c.H);
-                else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x)
-                    backward_operand_thin(c, reinterpret_cast<float*>(&smem), wres, first, end - first);   // 8 x H + 768 floats <= 26 KB
-                else backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.dhp, c.H, c.H);
+                else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x) {
+                    backward_operand_thin(c, reinterpret_cast<float*>(&smem), wres, first, end - first);   // 8 x H + 800 floats <= 26 KB
+                    thin = true;
+                } else backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.dhp, c.H, c.H);
             }
             first = end;
             __syncthreads();
@@ -915,6 +955,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
             lap(cyc_b);
         }
+        callees_done = thin;
     }
     if constexpr (TC) tc_teardown(tc);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
