@@ -227,13 +227,42 @@ __device__ __forceinline__ void store_token(Token* dst_tok, uint64_t tag, int64_
     dst[1] = make_uint4(pc, 0u, 0u, 0u);
 }
 
-__device__ __forceinline__ void push_token(const DevCtx& c, uint32_t wave, uint64_t tag, int64_t datum, uint32_t pc) {
+// The queue of a stretch of narrow waves that one block runs alone: the next wave's tokens stay in that
+// block's shared memory (same slot numbering as the global queue; a token beyond the local capacity goes
+// to its slot of the global queue, and the stretch ends there).
+static const uint32_t LQ_CAP = 1024;
+struct LocalQ {
+    Token*    buf[2];        // shared memory, by wave parity
+    uint32_t* count;         // shared memory, [3], by wave % 3
+};
+
+__device__ __forceinline__ void push_token(const DevCtx& c, const LocalQ* lq, uint32_t wave, uint64_t tag, int64_t datum,
+                                           uint32_t pc) {
+    if (lq) {
+        const uint32_t idx = aggregated_inc(&lq->count[(wave + 1) % 3]);
+        if (idx < LQ_CAP) store_token(&lq->buf[(wave + 1) & 1][idx], tag, datum, pc);
+        else if (idx < c.qcap) store_token(&c.q[(wave + 1) & 1][idx], tag, datum, pc);
+        else set_status(c, RDF_ERR_QUEUE_FULL);
+        return;
+    }
     const uint32_t idx = aggregated_inc(&c.ctl->qcount[(wave + 1) % 3].v);
     if (idx >= c.qcap) {
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
     }
     store_token(&c.q[(wave + 1) & 1][idx], tag, datum, pc);
+}
+
+__device__ __forceinline__ Token load_local_token(const Token* p) {       // from shared memory
+    const uint4* src = reinterpret_cast<const uint4*>(p);
+    const uint4 a = src[0], b = src[1];
+    Token t;
+    t.tag = (uint64_t)a.x | ((uint64_t)a.y << 32);
+    t.datum = (int64_t)((uint64_t)a.z | ((uint64_t)a.w << 32));
+    t.pc = b.x;
+    t.aux = 0;
+    t.pad = 0;
+    return t;
 }
 
 // two coalesced 128-bit loads per token, through L2

@@ -41,7 +41,7 @@ __device__ __forceinline__ void load_program(const DevCtx& c, SharedProgram& sp)
 
 // A completed match of a batched (cell) operator: queue the cell and the token
 // that carries its state onwards in the next wave.
-__device__ __forceinline__ void fire_cell(const DevCtx& c, const MatchNode& M, uint32_t wave, uint64_t tag,
+__device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, const MatchNode& M, uint32_t wave, uint64_t tag,
                                           const int64_t* regs, ThreadStats& st) {
     const uint32_t i = aggregated_inc(&c.ctl->cell_count.v);
     if (i >= c.work_cap) {
@@ -54,13 +54,13 @@ __device__ __forceinline__ void fire_cell(const DevCtx& c, const MatchNode& M, u
     c.op_l[tag] = it.l;
     c.op_r[tag] = it.r;
     ++st.cells;
-    push_token(c, wave, tag, (int64_t)tag, (uint32_t)M.cont_pc);
+    push_token(c, lq, wave, tag, (int64_t)tag, (uint32_t)M.cont_pc);
 }
 
 // Runs one token through its segment and on through every continuation it
 // completes (a returning value that finds its partner in the store carries on
 // in the caller's context in the same thread).
-__device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wave, Token t, ThreadStats& st) {
+__device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ* lq, uint32_t wave, Token t, ThreadStats& st) {
     int64_t r[RDF_MAX_REGS];
     uint64_t tag = t.tag;
     int pc = (int)t.pc;
@@ -98,7 +98,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
                     c.frame_args[(size_t)nt * 2] = r[in.b];
                     c.frame_args[(size_t)nt * 2 + 1] = r[in.dst];
                 }
-                push_token(c, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
+                push_token(c, lq, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
                 break;
             }
             case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)tag * 2 + in.imm - 1])); break;
@@ -154,7 +154,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
                     pc = M.cont_pc;                                 // r[0..n) hold the operands
                     break;
                 }
-                fire_cell(c, M, wave, tag, r, st);
+                fire_cell(c, lq, M, wave, tag, r, st);
                 return;
             }
             case VM_OUT: {
@@ -176,7 +176,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, uint32_t wav
                 c.op_l[tag] = LEAF_MARK;
                 c.op_r[tag] = (uint32_t)it.tok;
                 ++st.leaves;
-                push_token(c, wave, tag, (int64_t)tag, (uint32_t)in.imm);
+                push_token(c, lq, wave, tag, (int64_t)tag, (uint32_t)in.imm);
                 break;
             }
             default:   // VM_HALT
@@ -343,6 +343,12 @@ static const uint32_t NARROW_STRETCH = 4096;   // waves block 0 runs alone befor
 // frame table, store) are hidden by the number of tokens in flight.
 __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_constant__ DevCtx c) {
     __shared__ SharedProgram sp;
+    __shared__ uint32_t lq_count[3];
+    extern __shared__ __align__(16) unsigned char lq_smem[];         // local queue of narrow stretches: 2 x LQ_CAP tokens
+    LocalQ lq;
+    lq.buf[0] = reinterpret_cast<Token*>(lq_smem);
+    lq.buf[1] = lq.buf[0] + LQ_CAP;
+    lq.count = lq_count;
     load_program(c, sp);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
@@ -367,15 +373,24 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
             // block, when the queue is empty, or after NARROW_STRETCH waves (so that the bounded
             // wait of the other blocks never expires on a long stretch).
             if (blockIdx.x == 0) {
+                // The tokens of the stretch stay in this block's shared memory: the first wave is read from
+                // the global queue, the following ones from the local queue, and what is left at the end
+                // goes back to the global queue.
                 uint32_t m = n, k = 0;
+                bool local = false;
+                if (threadIdx.x < 3) lq_count[threadIdx.x] = 0;
+                __syncthreads();
                 do {
-                    if (threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
-                    if (threadIdx.x < m) run_token(c, sp, wave, load_token(&c.q[wave & 1][threadIdx.x]), st);
+                    if (threadIdx.x == 0) lq_count[(wave + 2) % 3] = 0;
+                    if (threadIdx.x < m) {
+                        const Token t = local ? load_local_token(&lq.buf[wave & 1][threadIdx.x]) : load_token(&c.q[wave & 1][threadIdx.x]);
+                        run_token(c, sp, &lq, wave, t, st);
+                    }
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
                     if (threadIdx.x == 0) mark_wave(c, wave);
                     if (k == 0) {
-                        // The next wave clears the counter that the other blocks read to take this branch:
-                        // carry on only when all of them have arrived at the grid barrier below (they
+                        // The end of the stretch rewrites the counters that the other blocks read to take this
+                        // branch: carry on only when all of them have arrived at the grid barrier below (they
                         // read the counter before they arrive).  Bounded like every other wait.
                         __shared__ int others_in;
                         if (threadIdx.x == 0) {
@@ -395,16 +410,27 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                         __syncthreads();
                         if (!others_in) {
                             ++wave;
+                            m = 0;
                             break;
                         }
                     }
                     ++wave;
                     ++k;
-                    m = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
+                    local = true;
+                    m = lq_count[wave % 3];
                     widest = max(widest, m);
                 } while (m != 0 && m <= blockDim.x && k < NARROW_STRETCH && wave < c.wave_limit &&
                          ld_volatile_i32(&c.ctl->status) == 0);
-                if (threadIdx.x == 0) c.ctl->resume_wave = wave;
+                // hand the next wave back to the global queue (tokens beyond the local capacity are there already)
+                for (uint32_t i = threadIdx.x; i < min(m, LQ_CAP); i += blockDim.x) {
+                    const Token t = load_local_token(&lq.buf[wave & 1][i]);
+                    store_token(&c.q[wave & 1][i], t.tag, t.datum, t.pc);
+                }
+                if (threadIdx.x == 0) {
+                    c.ctl->qcount[wave % 3].v = m;
+                    c.ctl->qcount[(wave + 1) % 3].v = 0;
+                    c.ctl->resume_wave = wave;
+                }
             }
             lap(cyc_s);
             if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
@@ -415,7 +441,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
         if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
         const Token* q = c.q[wave & 1];
         for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-            run_token(c, sp, wave, load_token(&q[i]), st);
+            run_token(c, sp, nullptr, wave, load_token(&q[i]), st);
         __syncthreads();
         lap(cyc_s);
         if (!grid_barrier(c, &c.ctl->bar.v, generation, wave)) break;
@@ -658,7 +684,8 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 128 * THIN_RESIDENT_MAX_H));
     if (per_sm < 1) return RDF_ERR_CUDA;
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 0));
+    CUDA_OK(cudaFuncSetAttribute(rdf_scheduler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * LQ_CAP * sizeof(Token))));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 2 * LQ_CAP * sizeof(Token)));
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
     S->device = dev;
@@ -785,7 +812,8 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args, 0, stream));
+    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
+                                        2 * LQ_CAP * sizeof(Token), stream));
     rdf_mark(S, 2, stream);
     if (g->has_vector_ops) {
         if (c.use_tc)
