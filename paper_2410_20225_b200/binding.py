@@ -446,11 +446,13 @@ class Graph:
                           n_classes=dp["W_s"].shape[0] if "W_s" in dp else 0, E=g("E"), W=g("W"), b=g("b"),
                           W_x=g("W_x"), b_x=g("b_x"), W_s=g("W_s"), b_s=g("b_s"))
 
-    def eval_trees(self, dt, dp, compute=F32, trace_capacity=0, check=True, h_root=None):
+    def eval_trees(self, dt, dp, compute=F32, trace_capacity=0, check=True, h_root=None, max_invocations=None):
         """Forward pass over a batch of trees.  dt/dp: device_trees()/device_params().
         For integer tree programs (no parameters) pass dp=None: returns (y, trace)."""
         torch = _torch()
         batch = self._batch(dt)
+        if max_invocations is not None:
+            batch.max_invocations = int(max_invocations)
         B = batch.B
         if dp is None:
             y = torch.empty(B, dtype=torch.int64, device="cuda")
@@ -469,10 +471,12 @@ class Graph:
             self.stats()
         return y, self._read_trace(tr)
 
-    def grad_trees(self, dt, dp, compute=F32, check=True, grads=None, loss=None, h_root=None):
+    def grad_trees(self, dt, dp, compute=F32, check=True, grads=None, loss=None, h_root=None, max_invocations=None):
         """Forward + reverse pass.  Returns (loss tensor [1], h_root, {name: gradient tensor})."""
         torch = _torch()
         batch = self._batch(dt)
+        if max_invocations is not None:
+            batch.max_invocations = int(max_invocations)
         params = self._params(dp, compute)
         if h_root is None:
             h_root = torch.empty(batch.B, params.H, dtype=torch.float32, device="cuda")

@@ -41,6 +41,7 @@ static const int GRAD_MAX_H = 1024;         // widest hidden size of the gradien
 
 template <bool BF>
 __global__ void __launch_bounds__(256) rdf_loss_heads_kernel(const DevCtx c, int fr, int rowbytes) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     extern __shared__ __align__(128) unsigned char slab_smem[];
     __shared__ __align__(8) uint64_t mbars[2];
     __shared__ __align__(16) float s_dl[LH_MAX_ROWS][8];
@@ -241,6 +242,7 @@ static const int LM_KSTEPS_MAX = TC_HP_MAX / 16;       // k steps of the logits 
 static const int LM_MT_MAX = (TC_HP_MAX / 16 + 7) / 8; // 16-unit tiles of dW_s per warp
 
 __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     extern __shared__ __align__(128) unsigned char slab_smem[];        // 2 stages of LM_ROWS rows, stride Hp * 2 + 16 bytes
     __shared__ __align__(8) uint64_t mbars[2];
     __shared__ __align__(16) float s_z[2][LM_ROWS][8];                 // partial logits of the two k halves
@@ -437,6 +439,7 @@ __device__ __forceinline__ void list_flags(const DevCtx& c, uint32_t f0, uint32_
 }
 
 __global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uint2* seg_counts) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     __shared__ uint32_t wc[8], wl[8];
     const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
     uint32_t l[8], r[8], cells, leaves;
@@ -456,6 +459,7 @@ __global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uin
 
 // one block: exclusive scan of the segment counts in place; totals to the control block
 __global__ void __launch_bounds__(1024) rdf_list_scan_kernel(const DevCtx c, uint2* seg_counts, int n_seg) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     __shared__ uint32_t wa[32], wb[32];
     const int per = (n_seg + 1023) / 1024, s0 = threadIdx.x * per, s1 = min(n_seg, s0 + per);
     const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
@@ -488,6 +492,7 @@ __global__ void __launch_bounds__(1024) rdf_list_scan_kernel(const DevCtx c, uin
 }
 
 __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, const uint2* seg_base) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     __shared__ uint32_t wc[8], wl[8];
     const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
     uint32_t l[8], r[8], cells, leaves;
@@ -524,6 +529,7 @@ __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, cons
 
 // marks[d].w = cells among the frames below marks[d].x: where wave d ends in all_cells.  One warp per wave.
 __global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, const uint2* seg_base) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     const uint32_t lane = threadIdx.x % 32, n_warps = gridDim.x * blockDim.x / 32;
     const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
     const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
@@ -980,6 +986,7 @@ struct OuterArgs {
 };
 
 __global__ void __launch_bounds__(256) rdf_outer_kernel(const DevCtx c, const OuterArgs a) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     __shared__ GemmSmem sm;
     const uint32_t n_items = *a.count;
     const int tile = blockIdx.x % (a.tiles_m * a.tiles_n), split = blockIdx.x / (a.tiles_m * a.tiles_n);
@@ -1034,8 +1041,9 @@ __device__ __forceinline__ float as_float(float v) { return v; }
 __device__ __forceinline__ float as_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
 template <typename T>
-__global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, const uint32_t* count, const T* A,
-                                                         int lda, int M, int H, int Hb, float* out) {
+__global__ void __launch_bounds__(256) rdf_colsum_kernel(const int32_t* status, const uint32_t* list, const uint32_t* count,
+                                                         const T* A, int lda, int M, int H, int Hb, float* out) {
+    if (*status != 0) return;                          // an earlier kernel of this call failed
     const uint32_t n = *count;
     const uint32_t per = (n + gridDim.x - 1) / gridDim.x;
     const uint32_t t0 = blockIdx.x * per, t1 = min(n, t0 + per);
@@ -1051,6 +1059,7 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const uint32_t* list, c
 
 // TreeLSTM: dE[tok_t] += W_x^T dg_t for every leaf t (dg_t = the 3H gate gradients)
 __global__ void __launch_bounds__(256) rdf_de_lstm_kernel(const DevCtx c, int tiles_n) {
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
     __shared__ GemmSmem sm;
     const uint32_t n_items = c.ctl->all_leaves;
     const int D = c.D, Kdim = 3 * c.H;
@@ -1228,13 +1237,13 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 6, stream);
-    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);
+    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
-        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
-        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);
+        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
+        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);
     } else {
-        rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, H, H, grads->db);
-        if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, H, H, grads->db_x);
+        rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, dgA, lda, MW, H, H, grads->db);
+        if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, H, H, grads->db_x);
     }
     rdf_mark(S, 7, stream);       // (dW_s and db_s came from the loss-head pass)
     if (tc_lstm) {

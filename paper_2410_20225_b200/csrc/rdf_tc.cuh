@@ -645,6 +645,7 @@ static __global__ void __launch_bounds__(256) rdf_pack_lstm_kernel(const DevCtx 
 static __global__ void __launch_bounds__(TC_THREADS, 1) rdf_de_tc_kernel(const DevCtx c) {
     extern __shared__ unsigned char dyn_smem[];
     __shared__ TcShared sh;
+    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed
     TcState tc;
     tc_setup(tc, sh, dyn_smem, c.Hp / 64, c.WxTp, 3 * c.Hp, 64);
     tc_pipe<TC_LSTM_DE, 5>(c, tc, sh, 0, c.ctl->all_leaves);

@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
     __shared__ __align__(8) uint64_t full[DW_STAGES], empty[DW_STAGES], done;
     __shared__ uint4 s_ops[2][DW_KT];                              // records of the stage being copied / the next one
     __shared__ int s_abort;                                        // a producer's bounded wait expired: all producers leave together
+    if (c.ctl->status != 0) return;                                // an earlier kernel of this call failed: nothing to contract
     const uint32_t n_cells = *a.count;
     const int tile = blockIdx.x % a.n_tiles, split = blockIdx.x / a.n_tiles;
     const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_cells, t_begin + a.chunk);

@@ -172,6 +172,28 @@ def test_frame_tags_required_for_depth():
     assert y.item() == 300
 
 
+@pytest.mark.parametrize("compute", [rdf.F32, rdf.BF16])
+def test_undersized_capacity_is_a_status_code_for_tree_networks(compute):
+    """A frame table too small for the batch: the scheduler reports RDF_ERR_FRAMES_FULL, every later kernel
+    of the call does nothing, and the same graph runs a correctly sized call afterwards."""
+    cfg = workloads.config(3, B=40, V=300, H=64)
+    tb, p = cfg["trees"], cfg["params"]
+    dt, dp = rdf.Graph.device_trees(tb), rdf.Graph.device_params(p)
+    g = graph("rnn", with_loss=True)
+    with pytest.raises(rdf.RdfError) as e:
+        g.grad_trees(dt, dp, compute, max_invocations=tb.N // 3)
+    assert e.value.code == -6                     # RDF_ERR_FRAMES_FULL
+    ge = graph("rnn")
+    with pytest.raises(rdf.RdfError) as e:
+        ge.eval_trees(dt, dp, compute, max_invocations=tb.N // 3)
+    assert e.value.code == -6
+    loss, h, grads = g.grad_trees(dt, dp, compute)
+    want_loss, G, roots = direct.loss_and_grad(tb, p, "rnn")
+    assert relerr(h.cpu().numpy(), roots) <= TOL[compute]
+    assert abs(loss.item() - want_loss) <= TOL[compute] * abs(want_loss)
+    assert all(relerr(grads[k].cpu().numpy(), G[k]) <= TOL[compute] for k in G)
+
+
 def test_treernn_config3_full_size():
     """8192 trees, H = 300, fwd + bwd at full size; the oracle runs over a pool of processes."""
     cfg = workloads.config(3)
