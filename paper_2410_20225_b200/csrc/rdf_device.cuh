@@ -77,6 +77,9 @@ struct Control {
 };
 static_assert(sizeof(Control) <= 4096, "the control block is 4 KB");
 
+// A tensor map as the driver encodes it (128 opaque bytes; the host fills it with cuTensorMapEncodeTiled).
+struct alignas(64) TensorMap { unsigned long long opaque[16]; };
+
 struct DevCtx {
     // lowered program (copied into the workspace at every call)
     const VmInstr*   code;
@@ -119,7 +122,10 @@ struct DevCtx {
     __nv_bfloat16* arena_bf;
     __nv_bfloat16* Wp;            // [Hp, 2Hp]   forward operand
     __nv_bfloat16* WTp;           // [2Hp, Hp]   gradient operand
-    __nv_bfloat16* dz_bf;         // [frame_cap, Hp] bf16 copy of dz (rdf_grad)
+    __nv_bfloat16* dz_bf;         // [frame_cap, Hp] bf16 dz rows of the cells (rdf_grad), row = position of the cell in
+                                  // all_cells: the cells of a gradient wave are consecutive rows, read as plain 2D tiles
+    uint32_t* cell_pos;           // per frame: position of a cell in all_cells (written with the lists; leaves: undefined)
+    TensorMap tmap_dz128, tmap_dz64;   // dz_bf as [rows, Hp], 128-byte swizzle, boxes of 128 / 64 rows by 64 columns
     // TreeLSTM on tensor cores: Wp / WTp hold the slice-major W5p [5Hp, 2Hp] and WT5p [2Hp, 5Hp]
     __nv_bfloat16* Wxp;           // [3Hp, Hp] leaf projection, slice-major
     __nv_bfloat16* WxTp;          // [Hp, 3Hp] its transpose (operand of the embedding gradient)

@@ -638,6 +638,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.wp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
     L.wtp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
     L.dz_bf = P.take<__nv_bfloat16>(tcr && want_grad ? vf * L.Hp : 0);
+    L.cell_pos = P.take<uint32_t>(tcr && want_grad ? vf : 0);
     L.wxp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.wxtp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
@@ -736,6 +737,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.Wp = reinterpret_cast<__nv_bfloat16*>(ws + L.wp);
         c.WTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wtp);
         c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
+        c.cell_pos = L.use_tc && !g->has_lstm ? reinterpret_cast<uint32_t*>(ws + L.cell_pos) : nullptr;
         c.Wxp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxp);
         c.WxTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxtp);
         c.E_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.e_bf);

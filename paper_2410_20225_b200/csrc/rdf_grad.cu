@@ -11,6 +11,8 @@
 #include <cstring>
 #include <type_traits>
 
+#include <cuda.h>              // CUtensorMap and the prototype of its encoder (the entry point is looked up at run time)
+
 #include "rdf_exec.h"
 #include "rdf_tc.cuh"
 #include "rdf_tc_dw.cuh"
@@ -516,6 +518,7 @@ __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, cons
         if (l[i] != LEAF_MARK) {
             c.all_cells[ic] = f;
             if (c.cell_ops) c.cell_ops[ic] = make_uint4(f, l[i], r[i], 1u);
+            if (c.cell_pos) c.cell_pos[f] = ic;
             ++ic;
         } else {
             if (c.lstm) {
@@ -540,6 +543,13 @@ __global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, cons
         for (uint32_t g = s0 + lane; g < f; g += 32) cnt += c.op_l[g] != LEAF_MARK;
         for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
         if (lane == 0) c.wave_marks[d].w = seg_base[seg].x + cnt;
+    }
+    // bf16 TreeRNN: the weight gradient reads dz in whole stages of 64 rows; the rows after the last cell are zero
+    if (c.cell_pos && blockIdx.x == 0) {
+        const uint32_t n = min(c.ctl->all_cells, c.frame_cap), n_end = min((n + 63u) & ~63u, c.frame_cap);
+        const uint32_t per_row = (uint32_t)c.Hp / 8;
+        for (uint32_t q = threadIdx.x; q < (n_end - n) * per_row; q += blockDim.x)
+            *reinterpret_cast<uint4*>(c.dz_bf + (size_t)(n + q / per_row) * c.Hp + (q % per_row) * 8) = make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
@@ -569,6 +579,7 @@ __device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0,
     for (uint32_t t = t0; t < end; t += stride) {
         const bool leaf = m.l == LEAF_MARK;
         const uint32_t tok = m.r;
+        const uint32_t pos = leaf ? 0u : c.cell_pos[t];               // the cell's dz row
         const float dl[MAX_CLASSES] = {m.d0.x, m.d0.y, m.d0.z, m.d0.w, m.d1.x, m.d1.y, m.d1.z, m.d1.w};
         uint4 hv[NQ];
 #pragma unroll
@@ -609,7 +620,7 @@ __device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0,
                 __align__(16) __nv_bfloat162 pk[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(dh[2 * i], dh[2 * i + 1]);
-                *reinterpret_cast<uint4*>(c.dz_bf + (size_t)t * Hp + j) = *reinterpret_cast<const uint4*>(pk);
+                *reinterpret_cast<uint4*>(c.dz_bf + (size_t)pos * Hp + j) = *reinterpret_cast<const uint4*>(pk);
             }
         }
     }
@@ -970,6 +981,30 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     }
 }
 
+// dz_bf as a 2D tensor [rows, Hp] of bf16 for tile copies: boxes of box_rows x 64 columns in the 128-byte swizzle.
+typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                           const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                           CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static int encode_row_tiles(TensorMap* out, void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "tensor map size");
+    static TensorMapEncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
+            return RDF_ERR_CUDA;
+        encode = reinterpret_cast<TensorMapEncodeTiledFn>(fn);
+    }
+    const cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows}, estr[2] = {1, 1};
+    CUtensorMap m;
+    if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return RDF_ERR_CUDA;
+    memcpy(out, &m, sizeof(m));
+    return RDF_OK;
+}
+
 // ------------------------------------------- parameter gradients (post pass)
 // out[m][n] = sum over the listed invocations t of A_t[m] * B_t[n]   (split over the list)
 //   A_t = A + t * lda (M values: dz, or gate gradients)
@@ -1052,7 +1087,7 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const int32_t* status, 
         const int col = (j / H) * Hb + j % H;
         float s = 0.f;
 #pragma unroll 8
-        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)list[i] * lda + col]);
+        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)(list ? list[i] : i) * lda + col]);
         atomicAdd(&out[j], s);
     }
 }
@@ -1162,6 +1197,11 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     if (rc != RDF_OK) return rc;
     // loss head over every retained invocation
     const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
+    if (tc_rnn) {                          // dz rows are read as 2D tiles by the gradient waves and by the weight gradient
+        rc = encode_row_tiles(&c.tmap_dz128, c.dz_bf, c.frame_cap, (uint64_t)c.Hp, 128);
+        if (rc == RDF_OK) rc = encode_row_tiles(&c.tmap_dz64, c.dz_bf, c.frame_cap, (uint64_t)c.Hp, 64);
+        if (rc != RDF_OK) return rc;
+    }
     {
         const int rowbytes = tc_rnn ? c.Hp * 2 : c.S * 4;
         const int fr = std::max(1, std::min(LH_MAX_ROWS, LH_SLAB_BYTES / rowbytes));
@@ -1221,6 +1261,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         a.ops = c.cell_ops; a.count = &c.ctl->all_cells;
         a.A = tc_lstm ? c.dg_bf : c.dz_bf; a.lda = tc_lstm ? 5 * c.Hp : c.Hp; a.Mp = tc_lstm ? 5 * c.Hp : c.Hp;
         a.Np = 2 * c.Hp; a.mode = 0; a.out = grads->dW; a.ldo = 2 * H;
+        a.a_tiles = tc_rnn ? 1 : 0;
         launch_dw(a, max_cells);
         if (tc_lstm) {
             DwArgs x{};
@@ -1237,7 +1278,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 6, stream);
-    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);
+    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);   // dz rows are in all_cells order
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
         rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
         rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);

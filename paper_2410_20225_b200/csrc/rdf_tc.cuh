@@ -189,6 +189,18 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t mbar_addr) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mbar_addr) : "memory");
 }
 
+// One box of a 2D tensor map (tile mode) into shared memory; completion is counted in bytes on the mbarrier.
+// x (innermost coordinate) times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const TensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t addr, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(addr), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t addr) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(addr) : "memory");
 }
@@ -292,7 +304,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
     if (warp >= TC_PROD_WARP0) {
         // ------------------------------------------------------------ producers
         const int p = threadIdx.x - TC_PROD_WARP0 * 32, r8 = p >> 3, c16 = p & 7;
-        const __nv_bfloat16* Arows = MODE == TC_RNN_BWD ? c.dz_bf : (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? c.dg_bf
+        const __nv_bfloat16* Arows = (MODE == TC_LSTM_BWD || MODE == TC_LSTM_DE) ? c.dg_bf
                                      : MODE == TC_LSTM_LEAF ? c.E_bf : c.arena_bf;
         auto load_item = [&](int tile) {                     // the record of row p of the tile
             uint4 it = make_uint4(0u, 0u, 0u, 0u);
@@ -332,6 +344,17 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
                 // the MMAs that last read this stage must have completed
                 if (g >= (uint32_t)STAGES) ok = mbar_wait(c, empty0 + 8 * s, ((g / STAGES) - 1) & 1u);
+                if (MODE == TC_RNN_BWD) {
+                    // the dz rows of the wave's cells are consecutive: one 2D tile (128 rows x 64 columns, written in the
+                    // 128-byte swizzle by the copy engine) per stage.  Rows after the wave's last cell hold other cells'
+                    // rows or old data: their accumulator rows are never read.
+                    if (!ok) break;
+                    if (p == 0) {
+                        mbar_arrive_expect_tx(full0 + 8 * s, TC_A_STAGE);
+                        tma_load_2d(tc.a_addr + s * TC_A_STAGE, &c.tmap_dz128, kc * TC_KC, (int)(first + (uint32_t)(rg + i * n_rg) * TC_M), full0 + 8 * s);
+                    } else mbar_arrive(full0 + 8 * s);
+                    continue;
+                }
                 const int koff = kc * TC_KC;
                 const bool second = (MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL) && koff >= Hp;
                 const size_t col = (size_t)(second ? koff - Hp : koff) + c16 * 8;
@@ -387,12 +410,13 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             const int e_col0 = slice * ns;
             const uint32_t child = e_col0 < Hp ? it.y : it.z;
             const int e_cc0 = e_col0 < Hp ? e_col0 : e_col0 - Hp;
-            uint32_t child_l = LEAF_MARK, child_tok = 0;
+            uint32_t child_l = LEAF_MARK, child_tok = 0, child_pos = 0;
             float4 cd0 = make_float4(0.f, 0.f, 0.f, 0.f), cd1 = cd0;
             uint4 chq[BWD_MAXG][2];
             if (MODE == TC_RNN_BWD && live) {
                 child_l = c.op_l[child];
                 child_tok = c.op_r[child];
+                child_pos = c.cell_pos[child];                            // (a cell's dz row; meaningless for a leaf)
                 cd0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
                 cd1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
 #pragma unroll
@@ -445,7 +469,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                                                                          v[half * 8 + 2 * i + 1] * (1.f - x.y * x.y));
                             }
                         }
-                        uint4* dst = reinterpret_cast<uint4*>(c.dz_bf + (size_t)child * Hp + cc);
+                        uint4* dst = reinterpret_cast<uint4*>(c.dz_bf + (size_t)child_pos * Hp + cc);
                         dst[0] = *reinterpret_cast<const uint4*>(&pk[0]);
                         dst[1] = *reinterpret_cast<const uint4*>(&pk[4]);
                     }

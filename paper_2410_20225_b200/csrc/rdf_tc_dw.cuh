@@ -45,9 +45,11 @@ struct DwArgs {
     int ldo;
     int tiles_n, n_tiles;
     uint32_t chunk;
+    int a_tiles;                 // 1: the rows of A are in list order (row = position in the list) and are read as 2D tiles
+                                 //    through DevCtx::tmap_dz64; the rows after the last listed one are zero up to a multiple of 64
 };
 
-__global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const DwArgs a) {
+__global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant__ DevCtx c, const DwArgs a) {
     const uint32_t lbo = 8192u, sbo = 1024u;       // next atom along M/N, next atom along K
     extern __shared__ unsigned char dyn_smem[];
     __shared__ uint32_t tmem_slot;
@@ -108,12 +110,23 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const DevCtx c, const
                 const int tr = tr0 + 4 * i;
                 const uint4 it = s_ops[kc & 1][tr];
                 const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
-                const bool mv = it.w != 0u && m_in;
-                cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
+                if (!a.a_tiles) {
+                    const bool mv = it.w != 0u && m_in;
+                    cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
+                }
                 const bool nv = it.w != 0u && n_in;
                 size_t src = 0;
                 if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
                 cp_async16(b_st + off, Brows + src, nv);
+            }
+            if (ok && a.a_tiles && threadIdx.x == 0) {
+                // A: four boxes of 64 rows x 64 columns, each written as the eight swizzled atoms of its column group
+                int boxes = 0;
+                for (int g = 0; g < 4; ++g) boxes += m0 + g * 64 < a.Mp;
+                mbar_expect_tx(full0 + 8 * s, (uint32_t)boxes * 8192u);
+                for (int g = 0; g < 4; ++g)
+                    if (m0 + g * 64 < a.Mp)
+                        tma_load_2d(a_st + g * 8192, &c.tmap_dz64, m0 + g * 64, (int)(t_begin + kc * DW_KT), full0 + 8 * s);
             }
             if (ok) cp_async_arrive(full0 + 8 * s);            // arrives when this thread's copies of the stage have landed
             if (threadIdx.x < DW_KT) s_ops[(kc + 1) & 1][threadIdx.x] = op_next;
