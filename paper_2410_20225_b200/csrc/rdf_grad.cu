@@ -1251,17 +1251,16 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         auto launch_dw = [&](DwArgs a, long long max_items) {
             a.tiles_n = (a.Np + DW_TILE - 1) / DW_TILE;
             a.n_tiles = ((a.Mp + DW_TILE - 1) / DW_TILE) * a.tiles_n;
-            const int splits = std::max(1, S->grid / a.n_tiles);
-            uint32_t chunk = (uint32_t)((max_items + splits - 1) / splits);
-            a.chunk = (chunk + DW_KT - 1) / DW_KT * DW_KT;
-            const int blocks = a.n_tiles * (int)((max_items + a.chunk - 1) / a.chunk);
-            rdf_dw_tc_kernel<<<blocks, 256, DW_SMEM_BYTES, stream>>>(c, a);
+            const long long stages = (max_items + DW_KT - 1) / DW_KT;
+            a.splits = (int)std::max<long long>(1, std::min<long long>(S->grid / a.n_tiles, stages));
+            rdf_dw_tc_kernel<<<a.n_tiles * a.splits, 256, DW_SMEM_BYTES, stream>>>(c, a);
         };
         DwArgs a{};
         a.ops = c.cell_ops; a.count = &c.ctl->all_cells;
         a.A = tc_lstm ? c.dg_bf : c.dz_bf; a.lda = tc_lstm ? 5 * c.Hp : c.Hp; a.Mp = tc_lstm ? 5 * c.Hp : c.Hp;
         a.Np = 2 * c.Hp; a.mode = 0; a.out = grads->dW; a.ldo = 2 * H;
         a.a_tiles = tc_rnn ? 1 : 0;
+        a.bias_out = tc_rnn && H < c.Hp ? grads->db : nullptr;      // db comes out of the same contraction
         launch_dw(a, max_cells);
         if (tc_lstm) {
             DwArgs x{};
@@ -1278,7 +1277,8 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 6, stream);
-    if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);   // dz rows are in all_cells order
+    if (tc_rnn && H < c.Hp) {}          // (column H of the dW contraction)
+    else if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);   // dz rows are in all_cells order
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
         rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
         rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);

@@ -443,7 +443,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                     if (!live) continue;
                     const int cc = e_cc0 + (e_begin + q) * 16;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {                         // classes beyond the last: zero rows
+                    for (int k = 0; k < 8; ++k) {
+                        if (k >= c.n_classes) break;                      // (uniform)
                         const float* wk = &sh.ep[k * TC_EP_LD + (e_begin + q) * 16];
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {
@@ -558,6 +559,9 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                             if (col + i < H) h = tc_tanh(v[i] + sh.ep[gi * 16 + i]);
                             hb[i] = __float2bfloat16_rn(h);
                         }
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)                         // first pad column: the constant 1 (H is a multiple of 4)
+                            if (col + i == H) hb[i] = __float2bfloat16_rn(1.f);
                         uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
                         dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
                         dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
@@ -590,6 +594,9 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
 
 // Leaves in bf16 mode: state(slot) = bf16(E[tok]), pad columns of the row zero.  Each warp takes four
 // leaves at a time, so that four rows are in flight per warp.
+// TreeRNN state rows carry the constant 1 in their first pad column (column H, when H < Hp): the packed weights
+// have zero rows there, so no contraction of the forward or the gradient pass sees it, and the weight-gradient
+// contraction dz (x) [h_l ; h_r] yields the bias gradient sum_t dz_t as its column H.
 static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
     const int H = c.H, Hp = c.Hp;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
@@ -615,6 +622,8 @@ static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
                 __align__(16) __nv_bfloat162 hb[4];
                 hb[0] = __floats2bfloat162_rn(v[q][0].x, v[q][0].y); hb[1] = __floats2bfloat162_rn(v[q][0].z, v[q][0].w);
                 hb[2] = __floats2bfloat162_rn(v[q][1].x, v[q][1].y); hb[3] = __floats2bfloat162_rn(v[q][1].z, v[q][1].w);
+                if (k == H) hb[0].x = __float2bfloat16_rn(1.f);            // the constant input (H is a multiple of 4;
+                else if (k + 4 == H) hb[2].x = __float2bfloat16_rn(1.f);   //  k < Hp, so this is a pad column)
                 *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it[q].x * Hp + k) = *reinterpret_cast<const uint4*>(hb);
             }
         }

@@ -44,7 +44,9 @@ struct DwArgs {
     float* out;
     int ldo;
     int tiles_n, n_tiles;
-    uint32_t chunk;
+    int splits;                  // blocks per tile: block `split` takes the stages split, split + splits, ... of the list
+    float* bias_out;             // mode 0 with H < Hp: column H of the left half of B is the constant 1 of the state rows,
+                                 // so that column of the product is sum_t A_t = the bias gradient (null: not wanted)
     int a_tiles;                 // 1: the rows of A are in list order (row = position in the list) and are read as 2D tiles
                                  //    through DevCtx::tmap_dz64; the rows after the last listed one are zero up to a multiple of 64
 };
@@ -59,11 +61,14 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
     if (c.ctl->status != 0) return;                                // an earlier kernel of this call failed: nothing to contract
     const uint32_t n_cells = *a.count;
     const int tile = blockIdx.x % a.n_tiles, split = blockIdx.x / a.n_tiles;
-    const uint32_t t_begin = (uint32_t)split * a.chunk, t_end = min(n_cells, t_begin + a.chunk);
-    if (t_begin >= t_end) return;                                  // the whole block leaves before any set-up
+    // Stages of 64 listed invocations are dealt out round robin, so that at any time the blocks together read one
+    // window of consecutive rows (a contiguous range per block reads its rows measurably slower).
+    const uint32_t n_stages = (n_cells + DW_KT - 1) / DW_KT;
+    if ((uint32_t)split >= n_stages) return;                       // the whole block leaves before any set-up
+    const uint32_t n_chunks = (n_stages - (uint32_t)split + (uint32_t)a.splits - 1) / (uint32_t)a.splits;
+    const uint32_t t_end = n_cells;
     const int H = c.H, Hp = c.Hp;
     const int m0 = (tile / a.tiles_n) * DW_TILE, n0 = (tile % a.tiles_n) * DW_TILE;
-    const uint32_t n_chunks = (t_end - t_begin + DW_KT - 1) / DW_KT;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const uint32_t raw = smem_u32(dyn_smem);
@@ -94,7 +99,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
         const bool m_in = m < a.Mp, n_in = n < a.Np;
         const __nv_bfloat16* Brows = a.mode == 0 ? c.arena_bf : c.E_bf;
         auto load_op = [&](uint32_t kc) {                          // the record of cell threadIdx.x of stage kc
-            const uint32_t idx = t_begin + kc * DW_KT + threadIdx.x;
+            const uint32_t idx = ((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT + threadIdx.x;
             return threadIdx.x < DW_KT && kc < n_chunks && idx < t_end ? a.ops[idx] : make_uint4(0u, 0u, 0u, 0u);
         };
         if (threadIdx.x < DW_KT) s_ops[0][threadIdx.x] = load_op(0);
@@ -110,23 +115,24 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
                 const int tr = tr0 + 4 * i;
                 const uint4 it = s_ops[kc & 1][tr];
                 const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
-                if (!a.a_tiles) {
+                if (a.a_tiles != 1) {
                     const bool mv = it.w != 0u && m_in;
-                    cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
+                    const size_t arow = a.a_tiles == 2 ? (size_t)(((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT + tr) : (size_t)it.x;
+                    cp_async16(a_st + off, a.A + arow * a.lda + (mv ? m : 0), mv);
                 }
                 const bool nv = it.w != 0u && n_in;
                 size_t src = 0;
                 if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
                 cp_async16(b_st + off, Brows + src, nv);
             }
-            if (ok && a.a_tiles && threadIdx.x == 0) {
+            if (ok && a.a_tiles == 1 && threadIdx.x == 0) {
                 // A: four boxes of 64 rows x 64 columns, each written as the eight swizzled atoms of its column group
                 int boxes = 0;
                 for (int g = 0; g < 4; ++g) boxes += m0 + g * 64 < a.Mp;
                 mbar_expect_tx(full0 + 8 * s, (uint32_t)boxes * 8192u);
                 for (int g = 0; g < 4; ++g)
                     if (m0 + g * 64 < a.Mp)
-                        tma_load_2d(a_st + g * 8192, &c.tmap_dz64, m0 + g * 64, (int)(t_begin + kc * DW_KT), full0 + 8 * s);
+                        tma_load_2d(a_st + g * 8192, &c.tmap_dz64, m0 + g * 64, (int)(((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT), full0 + 8 * s);
             }
             if (ok) cp_async_arrive(full0 + 8 * s);            // arrives when this thread's copies of the stage have landed
             if (threadIdx.x < DW_KT) s_ops[(kc + 1) & 1][threadIdx.x] = op_next;
@@ -175,6 +181,7 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
                     const int n = n0 + cl + i;
                     const int k = n < Hp ? n : n - Hp;
                     if (n < a.Np && k < n_limit) atomicAdd(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)], v[i]);
+                    else if (a.bias_out && n == H) atomicAdd(&a.bias_out[row], v[i]);
                 }
             }
         }
