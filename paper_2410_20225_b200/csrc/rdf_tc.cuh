@@ -404,15 +404,16 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             const bool live = it.w != 0u;
             // TreeRNN gradient: what the epilogue needs about the callee frame is fetched while the MMAs run.
             // All columns of a slice belong to one callee: [0, Hp) to the left one, [Hp, 2Hp) to the right one.
-            constexpr int BWD_MAXG = (TC_HP_MAX / 4 / 16 + 1) / 2;
-            const int e_groups = ns / 16, e_lo = (e_groups + 1) / 2;
-            const int e_begin = warp < 4 ? 0 : e_lo, e_end = warp < 4 ? e_lo : e_groups;
+            // Units of 8 columns, warps 0-3 take the first half of them and warps 4-7 the rest.
+            constexpr int BWD_MAXU = (TC_HP_MAX / 4 / 8 + 1) / 2;
+            const int e_units = ns / 8, e_lo = (e_units + 1) / 2;
+            const int e_begin = warp < 4 ? 0 : e_lo, e_end = warp < 4 ? e_lo : e_units;
             const int e_col0 = slice * ns;
             const uint32_t child = e_col0 < Hp ? it.y : it.z;
             const int e_cc0 = e_col0 < Hp ? e_col0 : e_col0 - Hp;
             uint32_t child_l = LEAF_MARK, child_tok = 0, child_pos = 0;
             float4 cd0 = make_float4(0.f, 0.f, 0.f, 0.f), cd1 = cd0;
-            uint4 chq[BWD_MAXG][2];
+            uint4 chq[BWD_MAXU];
             if (MODE == TC_RNN_BWD && live) {
                 child_l = c.op_l[child];
                 child_tok = c.op_r[child];
@@ -420,12 +421,9 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 cd0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
                 cd1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
 #pragma unroll
-                for (int q = 0; q < BWD_MAXG; ++q)
-                    if (e_begin + q < e_end) {
-                        const uint4* hp = reinterpret_cast<const uint4*>(c.arena_bf + (size_t)child * Hp + e_cc0 + (e_begin + q) * 16);
-                        chq[q][0] = hp[0];
-                        chq[q][1] = hp[1];
-                    }
+                for (int q = 0; q < BWD_MAXU; ++q)
+                    if (e_begin + q < e_end)
+                        chq[q] = *reinterpret_cast<const uint4*>(c.arena_bf + (size_t)child * Hp + e_cc0 + (e_begin + q) * 8);
             }
             ok = mbar_wait(c, acc_full0 + 8 * b, (T >> 1) & 1u);
             if (!ok) break;
@@ -436,43 +434,35 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 // a leaf callee adds dh to row tok of dE.  No gradient ever goes to memory in fp32.
                 const float dl[8] = {cd0.x, cd0.y, cd0.z, cd0.w, cd1.x, cd1.y, cd1.z, cd1.w};
 #pragma unroll
-                for (int q = 0; q < BWD_MAXG; ++q) {
+                for (int q = 0; q < BWD_MAXU; ++q) {
                     if (e_begin + q >= e_end) continue;                   // (uniform over the warp)
-                    float v[16];
-                    tc_ld16(lane_base + (uint32_t)((e_begin + q) * 16), v);
+                    float v[8];
+                    tc_ld8(lane_base + (uint32_t)((e_begin + q) * 8), v);
                     if (!live) continue;
-                    const int cc = e_cc0 + (e_begin + q) * 16;
+                    const int cc = e_cc0 + (e_begin + q) * 8;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         if (k >= c.n_classes) break;                      // (uniform)
-                        const float* wk = &sh.ep[k * TC_EP_LD + (e_begin + q) * 16];
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4) {
-                            const float4 w = *reinterpret_cast<const float4*>(wk + i);
-                            v[i] = fmaf(w.x, dl[k], v[i]); v[i + 1] = fmaf(w.y, dl[k], v[i + 1]);
-                            v[i + 2] = fmaf(w.z, dl[k], v[i + 2]); v[i + 3] = fmaf(w.w, dl[k], v[i + 3]);
-                        }
+                        const float* wk = &sh.ep[k * TC_EP_LD + (e_begin + q) * 8];
+                        const float4 w0 = *reinterpret_cast<const float4*>(wk), w1 = *reinterpret_cast<const float4*>(wk + 4);
+                        v[0] = fmaf(w0.x, dl[k], v[0]); v[1] = fmaf(w0.y, dl[k], v[1]);
+                        v[2] = fmaf(w0.z, dl[k], v[2]); v[3] = fmaf(w0.w, dl[k], v[3]);
+                        v[4] = fmaf(w1.x, dl[k], v[4]); v[5] = fmaf(w1.y, dl[k], v[5]);
+                        v[6] = fmaf(w1.z, dl[k], v[6]); v[7] = fmaf(w1.w, dl[k], v[7]);
                     }
                     if (child_l == LEAF_MARK) {
                         float* de = c.dE + (size_t)child_tok * c.D + cc;
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4)
-                            if (cc + i < H) atomicAdd(reinterpret_cast<float4*>(de + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+                        if (cc < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(v[0], v[1], v[2], v[3]));
+                        if (cc + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(v[4], v[5], v[6], v[7]));
                     } else {
-                        __align__(16) __nv_bfloat162 pk[8];
+                        __align__(16) __nv_bfloat162 pk[4];
+                        const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&chq[q]);
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&chq[q][half]);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float2 x = __bfloat1622float2(hb[i]);   // pad columns: v = 0 and h = 0, so dz = 0
-                                pk[half * 4 + i] = __floats2bfloat162_rn(v[half * 8 + 2 * i] * (1.f - x.x * x.x),
-                                                                         v[half * 8 + 2 * i + 1] * (1.f - x.y * x.y));
-                            }
+                        for (int i = 0; i < 4; ++i) {
+                            const float2 x = __bfloat1622float2(hb[i]);       // pad columns: v = 0, so dz = 0
+                            pk[i] = __floats2bfloat162_rn(v[2 * i] * (1.f - x.x * x.x), v[2 * i + 1] * (1.f - x.y * x.y));
                         }
-                        uint4* dst = reinterpret_cast<uint4*>(c.dz_bf + (size_t)child_pos * Hp + cc);
-                        dst[0] = *reinterpret_cast<const uint4*>(&pk[0]);
-                        dst[1] = *reinterpret_cast<const uint4*>(&pk[4]);
+                        *reinterpret_cast<uint4*>(c.dz_bf + (size_t)child_pos * Hp + cc) = *reinterpret_cast<const uint4*>(pk);
                     }
                 }
             } else if (MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) {

@@ -153,6 +153,19 @@ def test_treernn_bf16_tensor_core_path(H):
     assert st["cells"] > 3 * 128
 
 
+@pytest.mark.parametrize("H", [100, 256])
+def test_treernn_bf16_padding_and_biases(H):
+    """H = 100 leaves 28 pad columns in the bf16 state rows (the first of them holds the constant input from
+    which the bias gradient is contracted); H = 256 leaves none (the bias gradient is a column sum then).
+    Nonzero biases; several tiles per wave."""
+    cfg = workloads.config(3, B=300, V=500, H=H)
+    rng = np.random.default_rng(11)
+    cfg["params"]["b"] = workloads.bf16_round((0.2 * rng.standard_normal(H)).astype(np.float32))
+    cfg["params"]["b_s"] = workloads.bf16_round((0.2 * rng.standard_normal(5)).astype(np.float32))
+    check_forward(cfg, rdf.BF16)
+    check_grad(cfg, rdf.BF16)
+
+
 def test_depth_stress_reduced():
     cfg = workloads.config(5, chains=3, chain_depth=300, perfect=2, perfect_height=7, V=400, H=32)
     st, _ = check_grad(cfg)
