@@ -176,11 +176,14 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
                 const int cl = (warp >> 2) * 128 + gi * 16;
                 tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(h * DW_TILE + cl), v);
                 if (m >= a.Mp || mj >= H || n0 + cl >= a.Np) continue;
+                // four columns per atomic: H, D and the row stride of the output are multiples of 4
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < 16; i += 4) {
                     const int n = n0 + cl + i;
                     const int k = n < Hp ? n : n - Hp;
-                    if (n < a.Np && k < n_limit) atomicAdd(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)], v[i]);
+                    if (n < a.Np && k < n_limit)
+                        atomicAdd(reinterpret_cast<float4*>(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)]),
+                                  make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
                     else if (a.bias_out && n == H) atomicAdd(&a.bias_out[row], v[i]);
                 }
             }
