@@ -944,6 +944,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
                 for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
             } else if constexpr (TC) {
                 backward_frames_tc(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+                asm volatile("fence.proxy.async;" ::: "memory");       // its dz rows are read by tile copies after the barrier
             } else {
                 backward_frames_f32(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
             }

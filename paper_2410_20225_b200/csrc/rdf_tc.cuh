@@ -320,6 +320,9 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             }
             return it;
         };
+        // dz rows were written with plain stores by other blocks before the last grid barrier: order this call's
+        // tile copies (async proxy) after what that barrier acquired
+        if (MODE == TC_RNN_BWD) asm volatile("fence.proxy.async;" ::: "memory");
         uint4 it_next = my_tiles ? load_item(rg) : make_uint4(0u, 0u, 0u, 0u);
         for (int i = 0; i < my_tiles && ok; ++i) {
             const uint32_t T = tc.T + i, b = T & 1u;
@@ -575,6 +578,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             mbar_arrive(acc_empty0 + 8 * b);                   // buffer and records may be reused
         }
     }
+    // (writer side of the same ordering: the dz rows stored above are read by tile copies after the next grid barrier)
+    if (MODE == TC_RNN_BWD) asm volatile("fence.proxy.async;" ::: "memory");
     tc.g += (uint32_t)(my_tiles * n_chunks);
     tc.T += (uint32_t)my_tiles;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
