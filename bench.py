@@ -61,7 +61,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "25"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -147,7 +147,9 @@ def oracle_sample_size(cfg):
     return 256 if cfg["grad"] else 512
 
 
-def time_oracle(cfg, steps, warmup, scale=1):
+def time_oracle(cfg, steps, warmup, scale=1, budget_s=None):
+    """Times the oracle as it stands on a bounded sample per step.  With budget_s the sample shrinks (never grows) so
+    that warm-up and timed steps together stay near that many seconds (a short calibration step decides)."""
     try:
         from threadpoolctl import threadpool_limits
         ctx = threadpool_limits(limits=1)
@@ -156,6 +158,12 @@ def time_oracle(cfg, steps, warmup, scale=1):
         ctx = contextlib.nullcontext()
     sample = oracle_sample_size(cfg) * scale
     with ctx:
+        if budget_s is not None and sample > 8:
+            probe = max(1, sample // 16)
+            t0 = time.perf_counter()
+            oracle_step(cfg, probe)
+            per_item = (time.perf_counter() - t0) / probe
+            sample = max(min(sample, 8), min(sample, int(budget_s / ((steps + warmup) * per_item))))
         for _ in range(warmup):
             oracle_step(cfg, sample)
         t0 = time.perf_counter()
@@ -197,7 +205,7 @@ def sum_gradients(dist, grads):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", type=int, default=3, choices=sorted(WORKLOAD_NAMES))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -216,7 +224,7 @@ def main():
         if rank != 0:
             return
         cfg = load(args.workload, args.seed, args.fib_batch)
-        value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup))
+        value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup), budget_s=90.0)
         print(json.dumps({
             "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * s_per_step, "higher_is_better": True,
