@@ -5,10 +5,13 @@
 // operand form.  A stage holds 64 cells: for each operand four 64-wide groups
 // of j (of k), each as 8 atoms of (8 cells x 128 bytes) with the 128-byte
 // swizzle.  Each thread block owns one 256 x 256 tile of dW (two 128-row
-// accumulators: all 512 columns of tensor memory) and a range of the cells
-// (split-K); partial tiles are added to dW with atomics.  The large tile is
-// what keeps the gather small: an operand row is fetched once per tile that
-// needs it, and the gather (16-byte cp.async pieces) is what bounds the kernel.
+// accumulators: all 512 columns of tensor memory) and every splits-th stage
+// of the cell list (split-K); partial tiles are added to dW with vector
+// atomics.  The large tile is what keeps the gather small: an operand row is
+// fetched once per tile that needs it, and the gather (16-byte cp.async
+// pieces) is what bounds the kernel.  bf16 TreeRNN: the dz rows are stored in
+// list order, so that operand arrives as 2D tile copies instead, and column H
+// of the product (the constant 1 of the state rows) is the bias gradient.
 #pragma once
 #include "rdf_tc.cuh"
 
@@ -115,17 +118,16 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
                 const int tr = tr0 + 4 * i;
                 const uint4 it = s_ops[kc & 1][tr];
                 const uint32_t off = atom * 8192 + (tr >> 3) * 1024 + (tr & 7) * 128 + ((c16 ^ (tr & 7)) << 4);
-                if (a.a_tiles != 1) {
+                if (!a.a_tiles) {
                     const bool mv = it.w != 0u && m_in;
-                    const size_t arow = a.a_tiles == 2 ? (size_t)(((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT + tr) : (size_t)it.x;
-                    cp_async16(a_st + off, a.A + arow * a.lda + (mv ? m : 0), mv);
+                    cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
                 }
                 const bool nv = it.w != 0u && n_in;
                 size_t src = 0;
                 if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
                 cp_async16(b_st + off, Brows + src, nv);
             }
-            if (ok && a.a_tiles == 1 && threadIdx.x == 0) {
+            if (ok && a.a_tiles && threadIdx.x == 0) {
                 // A: four boxes of 64 rows x 64 columns, each written as the eight swizzled atoms of its column group
                 int boxes = 0;
                 for (int g = 0; g < 4; ++g) boxes += m0 + g * 64 < a.Mp;
