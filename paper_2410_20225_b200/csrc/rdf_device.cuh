@@ -41,7 +41,8 @@ struct __align__(16) Slot {
 static const uint64_t SLOT_EMPTY = ~0ull;     // depth field 63: never a tag
 
 struct __align__(16) CellItem {               // one ready cell: state of `out` from states of l, r
-    uint32_t out, l, r, pad;
+    uint32_t out, l, r;
+    uint32_t height;                          // 1 + the larger height of its operands (leaves: 0)
 };
 struct __align__(8) LeafItem {
     uint32_t slot;
@@ -69,6 +70,7 @@ struct Control {
     uint32_t all_cells;           // backward: cells seen so far (length of the all-cells list)
     uint32_t all_leaves;          // backward: leaves seen so far
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
+    uint32_t max_height;          // largest height of a cell of this call (operator waves run height by height)
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
     unsigned long long cyc[6];    // block 0: forward schedule / batch / barrier, backward frames / batch / barrier
@@ -110,7 +112,11 @@ struct DevCtx {
     Slot*     table;
     uint64_t  table_cap;          // slots per match node, power of two
     // batched operators
-    CellItem* cell_items;         // every cell in the order it became ready (wave after wave)
+    CellItem* cell_items;         // every cell in the order it became ready (wave after wave); the operator kernel
+                                  // gets the copy sorted by height here
+    CellItem* cell_sorted;        // the cells grouped by height: the operands of a cell of height k have heights < k, so
+                                  // all cells of one height fire together whatever wave the scheduler found them in
+    uint32_t* height_ends;        // [wave_cap + 2]: cells per height, then (after the scatter) the end of each group
     LeafItem* leaf_items;         // every leaf in the order it was reached
     uint32_t  work_cap;
     uint32_t* op_l;               // per frame: operand frames of the operator that made its state

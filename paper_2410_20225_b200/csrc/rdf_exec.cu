@@ -48,13 +48,16 @@ __device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, con
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
     }
+    // A vector value travels as the frame that holds it (low half of the datum) and the height of the
+    // operator tree below it (high half): leaves 0, a cell one more than the higher of its operands.
     CellItem it;
-    it.out = (uint32_t)tag; it.l = (uint32_t)regs[0]; it.r = (uint32_t)regs[1]; it.pad = 0;
+    it.out = (uint32_t)tag; it.l = (uint32_t)regs[0]; it.r = (uint32_t)regs[1];
+    it.height = max((uint32_t)((uint64_t)regs[0] >> 32), (uint32_t)((uint64_t)regs[1] >> 32)) + 1u;
     c.cell_items[i] = it;
     c.op_l[tag] = it.l;
     c.op_r[tag] = it.r;
     ++st.cells;
-    push_token(c, lq, wave, tag, (int64_t)tag, (uint32_t)M.cont_pc);
+    push_token(c, lq, wave, tag, (int64_t)(((uint64_t)it.height << 32) | (uint32_t)tag), (uint32_t)M.cont_pc);
 }
 
 // Runs one token through its segment and on through every continuation it
@@ -115,7 +118,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                         uint32_t label;
                         uint64_t parent;
                         tag_pop(c, tag, label, parent);
-                        trace_rec(c, tag, val, 1, label, (uint32_t)parent);
+                        trace_rec(c, tag, c.H > 0 ? (int64_t)(uint32_t)val : val, 1, label, (uint32_t)parent);   // (vector value: its frame)
                         tag = parent;
                         const LabelInfo& L = sp.labels[label];
                         if (L.k_kind == K_RET) continue;           // the call was the caller's own output
@@ -159,7 +162,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             }
             case VM_OUT: {
                 const long long inst = c.tag_mode == RDF_TAGS_PATH ? (long long)(tag >> RDF_INST_SHIFT) : (long long)tag;
-                if (inst >= 0 && inst < c.B) c.y[inst] = r[in.a];
+                if (inst >= 0 && inst < c.B) c.y[inst] = c.H > 0 ? (int64_t)(uint32_t)r[in.a] : r[in.a];   // (vector value: its frame)
                 return;
             }
             case VM_EMBED:
@@ -529,10 +532,12 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
+    // (cell_items is the height-sorted list here: the launch passes cell_sorted in its place)
     uint32_t first = 0;
-    for (uint32_t w = 0; w < n_waves && alive; ++w) {
-        const uint32_t end = min(c.wave_marks[w].y, c.work_cap);
-        if (end <= first) continue;                                  // no cell became ready in this wave
+    const uint32_t top = min(c.ctl->max_height, c.wave_cap);
+    for (uint32_t w = 1; w <= top && alive; ++w) {
+        const uint32_t end = min(c.height_ends[w], c.work_cap);
+        if (end <= first) continue;                                  // (no cell of this height)
         const uint32_t nc = end - first;
         if constexpr (TC) {
             if (c.lstm) tc_pipe<TC_LSTM_CELL, TC_STAGES_LSTM_FWD>(c, tc, smem, first, nc);
@@ -554,6 +559,77 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         c.ctl->cyc[1] = cyc_c;
         c.ctl->cyc[2] += cyc_b;
+    }
+}
+
+// ---- cells grouped by height (between the scheduler and the operator kernel)
+// The scheduler finds a cell ready in the wave in which its second operand returns, which depends on how deep the
+// whole tree below it reaches; what the arithmetic needs is only that operands come first.  Grouping the cells by
+// height gives the smallest number of dependent operator waves (the largest height instead of about twice the depth).
+__global__ void __launch_bounds__(256) rdf_height_count_kernel(const DevCtx c) {
+    if (c.ctl->status != 0) return;
+    const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
+    uint32_t top = 0;
+    for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
+        const uint32_t i = i0 + lane;
+        const uint32_t h = i < n ? min(c.cell_items[i].height, c.wave_cap) : 0u;      // (0: not a cell)
+        const unsigned peers = __match_any_sync(0xffffffffu, h);                      // one atomic per height and warp
+        if (h && (uint32_t)(__ffs(peers) - 1) == lane) atomicAdd(&c.height_ends[h], (uint32_t)__popc(peers));
+        top = max(top, h);
+    }
+    for (int o = 16; o > 0; o >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
+    if (lane == 0 && top) atomicMax(&c.ctl->max_height, top);
+}
+
+// counts -> first position of each height (one block; heights 1 .. max_height)
+__global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c) {
+    __shared__ uint32_t warp_sum[32];
+    __shared__ uint32_t carry;
+    if (c.ctl->status != 0) return;
+    const uint32_t top = c.ctl->max_height, lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (uint32_t h0 = 1; h0 <= top; h0 += 1024) {
+        const uint32_t h = h0 + threadIdx.x;
+        const uint32_t v = h <= top ? c.height_ends[h] : 0u;
+        uint32_t x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+            if ((int)lane >= o) x += y;
+        }
+        if (lane == 31) warp_sum[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t w = warp_sum[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, w, o);
+                if ((int)lane >= o) w += y;
+            }
+            warp_sum[lane] = w;
+        }
+        __syncthreads();
+        const uint32_t before = carry + (warp ? warp_sum[warp - 1] : 0u) + x - v;
+        if (h <= top) c.height_ends[h] = before;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = before + v;
+        __syncthreads();
+    }
+}
+
+// every cell to its group; afterwards height_ends[h] is where group h ends (group h starts where group h - 1 ends)
+__global__ void __launch_bounds__(256) rdf_height_scatter_kernel(const DevCtx c) {
+    if (c.ctl->status != 0) return;
+    const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
+    for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
+        const uint32_t i = i0 + lane;
+        CellItem it = i < n ? c.cell_items[i] : CellItem{0u, 0u, 0u, 0u};
+        const uint32_t h = min(it.height, c.wave_cap);
+        const unsigned peers = __match_any_sync(0xffffffffu, h);
+        const int leader = __ffs(peers) - 1;
+        uint32_t base = 0;
+        if (h && (uint32_t)leader == lane) base = atomicAdd(&c.height_ends[h], (uint32_t)__popc(peers));
+        base = __shfl_sync(0xffffffffu, base, leader);
+        if (h) c.cell_sorted[min(base + (uint32_t)__popc(peers & ((1u << lane) - 1u)), c.work_cap - 1u)] = it;
     }
 }
 
@@ -624,6 +700,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.table = P.take<char>(L.table_bytes);
     L.cell_items = P.take<CellItem>(L.work_cap);
     L.leaf_items = P.take<LeafItem>(L.work_cap);
+    L.cell_sorted = P.take<CellItem>(g->has_vector_ops ? L.work_cap : 0);
     const size_t vf = g->has_vector_ops ? L.frame_cap : 0;
     L.op_l = P.take<uint32_t>(vf);
     L.op_r = P.take<uint32_t>(vf);
@@ -652,6 +729,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     // every wave of a vector program holds at least one token of an invocation on its way down or up
     L.wave_cap = g->has_vector_ops ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
     L.wave_marks = P.take<uint4>(L.wave_cap);
+    L.height_ends = P.take<uint32_t>(L.wave_cap ? (size_t)L.wave_cap + 2 : 0);
     L.list_seg = P.take<uint2>(want_grad ? (size_t)in->max_invocations / 2048 + 2 : 0);
     L.all_cells = P.take<uint32_t>(gf);
     L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
@@ -718,6 +796,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.table = reinterpret_cast<Slot*>(ws + L.table);
     c.table_cap = L.table_cap;
     c.cell_items = reinterpret_cast<CellItem*>(ws + L.cell_items);
+    c.cell_sorted = reinterpret_cast<CellItem*>(ws + L.cell_sorted);
+    c.height_ends = reinterpret_cast<uint32_t*>(ws + L.height_ends);
     c.leaf_items = reinterpret_cast<LeafItem*>(ws + L.leaf_items);
     c.work_cap = L.work_cap;
     c.op_l = reinterpret_cast<uint32_t*>(ws + L.op_l);
@@ -787,6 +867,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
                        DevCtx& c, cudaStream_t stream) {
     rdf_mark(S, 0, stream);
     CUDA_OK(cudaMemsetAsync(ws + L.ctl, 0, 4096, stream));
+    if (L.wave_cap) CUDA_OK(cudaMemsetAsync(ws + L.height_ends, 0, ((size_t)L.wave_cap + 2) * sizeof(uint32_t), stream));
     if (g->tag_mode == RDF_TAGS_FRAME) {
         bool wide = false;                        // an operator with more than two tagged inputs
         for (const MatchNode& m : g->match) wide = wide || m.n_ports > 2;
@@ -818,11 +899,19 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
                                         2 * LQ_CAP * sizeof(Token), stream));
     rdf_mark(S, 2, stream);
     if (g->has_vector_ops) {
+        // the cells grouped by height; the operator kernel reads the grouped list in place of the scheduler's
+        rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+        rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c);
+        rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+        CUDA_OK(cudaGetLastError());
+        DevCtx co = c;
+        co.cell_items = c.cell_sorted;
+        void* oargs[] = {(void*)&co};
         if (c.use_tc)
-            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
+            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), oargs,
                                                 (size_t)L.tc_smem_fwd, stream));
         else
-            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), args,
+            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
                                                 thin_resident_bytes(c.lstm, c.H), stream));
         rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
         CUDA_OK(cudaGetLastError());

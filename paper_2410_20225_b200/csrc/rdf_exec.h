@@ -64,7 +64,7 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, children, pair_slots, port_val, arrived, table, cell_items,
-        leaf_items, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, total;
+        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, total;
     uint32_t qcap, frame_cap, work_cap, wave_cap;
     int use_tc, Hp, tc_smem_fwd, tc_smem_bwd;
     uint64_t table_cap;
