@@ -35,10 +35,10 @@ WORKLOAD_NAMES = {
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
 # kernels of the library launched per step (memsets and copies not counted):
-#   seed, scheduler | + operators, root gather | + loss head, loss sum, 4 list kernels, gradient waves, dW, db
+#   seed, scheduler | + 3 kernels that group the cells by height, operators, root gather | + loss head, loss sum, 4 list kernels, gradient waves, dW, db
 #   bf16: + weight packing (TreeLSTM: + table packing); TreeLSTM: + dW_x, db_x, dE
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 4, "eval_trees_tc": 5, "grad": 13, "grad_tc": 14, "grad_lstm": 16,
-                    "grad_lstm_tc": 18}
+KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 7, "eval_trees_tc": 8, "grad": 16, "grad_tc": 17, "grad_lstm": 19,
+                    "grad_lstm_tc": 21}
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
 
 
@@ -113,8 +113,8 @@ def peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
 # (profiles/persistent_kernels_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 394.6e6, ("rdf_operator_kernel", 3, None): 312.8e6,
-                     ("rdf_scheduler_kernel", 3, None): 10.1e6}
+NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 394.2e6, ("rdf_operator_kernel", 3, None): 298.5e6,
+                     ("rdf_scheduler_kernel", 3, None): 10.5e6}
 
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
