@@ -721,7 +721,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
     L.dg_bf = P.take<__nv_bfloat16>(tcl && want_grad ? vf * 5 * L.Hp : 0);
     L.tc_smem_fwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(80, 2 * L.Hp, 48, L.Hp, TC_STAGES_LSTM_FWD) : tc_smem_bytes(L.Hp / 4, 2 * L.Hp, 0, 0, TC_STAGES_RNN_FWD);
-    L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(32, 5 * L.Hp, 0, 0, TC_STAGES_LSTM_BWD) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, TC_STAGES_RNN_BWD);
+    L.tc_smem_bwd = !L.use_tc ? 0 : tcl ? tc_smem_bytes(TC_LSTM_BWD_NS, 5 * L.Hp, 0, 0, TC_STAGES_LSTM_BWD) : tc_smem_bytes(L.Hp / 4, L.Hp, 0, 0, TC_STAGES_RNN_BWD);
     L.ybuf = P.take<int64_t>(g->has_vector_ops ? in->B : 0);
     const size_t gf = want_grad ? L.frame_cap : 0;
     L.dhp = P.take<float>(tcr ? 0 : gf * S);            // (the bf16 TreeRNN hands its gradients on as dz rows)

@@ -896,7 +896,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     if (c.ctl->forward_status != 0) return;                          // the forward pass failed: nothing to differentiate
     TcState tc;
     if constexpr (TC) {
-        if (c.lstm) tc_setup(tc, smem, dyn_smem, 2 * c.Hp / 32, c.WTp, 5 * c.Hp, 32);
+        if (c.lstm) tc_setup(tc, smem, dyn_smem, (2 * c.Hp + TC_LSTM_BWD_NS - 1) / TC_LSTM_BWD_NS, c.WTp, 5 * c.Hp, TC_LSTM_BWD_NS, nullptr, 0, 0, 2 * c.Hp);
         else tc_setup(tc, smem, dyn_smem, 8, c.WTp, c.Hp, c.Hp / 4);
         tc_setup_epilogue(c, tc, smem, true);
     }

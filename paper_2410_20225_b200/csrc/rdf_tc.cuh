@@ -31,7 +31,10 @@ static const int TC_TMEM_COLS = 2 * TC_ACC_COLS;
 static const int TC_THREADS = 416;           // warps 0-7 epilogue, warp 8 MMA issuer, warps 9-12 producers
 static const int TC_EPI_THREADS = 256, TC_MMA_WARP = 8, TC_PROD_WARP0 = 9, TC_PRODUCERS = 128;
 // ring depth per kernel: what is left of the shared memory beside the resident weight slices
-static const int TC_STAGES_RNN_FWD = 7, TC_STAGES_LSTM_FWD = 5, TC_STAGES_RNN_BWD = 8, TC_STAGES_LSTM_BWD = 7;
+static const int TC_STAGES_RNN_FWD = 7, TC_STAGES_LSTM_FWD = 5, TC_STAGES_RNN_BWD = 8, TC_STAGES_LSTM_BWD = 4;
+// TreeLSTM operand gradient: columns of WT5p per block.  Every block of a row group gathers the same operand rows, so
+// the wider the slice the fewer copies of them cross L2; 48 columns x 5 Hp is what fits beside a ring of 4 stages.
+static const int TC_LSTM_BWD_NS = 48;
 
 // tile loops (template parameter of tc_pipe)
 enum TcMode {
@@ -209,7 +212,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t addr) {
 // block's resident slices of the packed weights: rows [slice * ns, +ns) of B[. x K], chunk by chunk.
 __device__ __forceinline__ void tc_setup(TcState& tc, TcShared& sh, unsigned char* dyn_smem, int n_split,
                                          const __nv_bfloat16* B0, int K0, int ns0,
-                                         const __nv_bfloat16* B1 = nullptr, int K1 = 0, int ns1 = 0) {
+                                         const __nv_bfloat16* B1 = nullptr, int K1 = 0, int ns1 = 0, int rows0 = 1 << 30) {
+    // (rows0: rows of B0 that exist; the last slice may reach beyond them and holds zeros there)
     const uint32_t raw = smem_u32(dyn_smem);
     const uint32_t aligned = (raw + 1023u) & ~1023u;
     unsigned char* base = dyn_smem + (aligned - raw);
@@ -246,7 +250,8 @@ __device__ __forceinline__ void tc_setup(TcState& tc, TcShared& sh, unsigned cha
         unsigned char* bp = base + (which ? bytes0 : 0);
         for (int p = threadIdx.x; p < (Kp / TC_KC) * ns * 8; p += blockDim.x) {
             const int kc = p / (ns * 8), q = p % (ns * 8), r = q >> 3, c16 = q & 7;
-            const uint4 v = *reinterpret_cast<const uint4*>(Bp + (size_t)(slice * ns + r) * Kp + kc * TC_KC + c16 * 8);
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (which || slice * ns + r < rows0) v = *reinterpret_cast<const uint4*>(Bp + (size_t)(slice * ns + r) * Kp + kc * TC_KC + c16 * 8);
             *reinterpret_cast<uint4*>(bp + kc * ns * 128 + swz(r, c16)) = v;
         }
     }
