@@ -425,8 +425,8 @@ def main():
                    "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
         "clocks": clk,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        # (bf16 TreeRNN with padded state rows: db comes out of the dW contraction, one kernel fewer)
-        "gpu_launches": (KERNELS_PER_STEP[kind] - (1 if kind == "grad_tc" and cfg["H"] % 64 else 0)) * args.steps,
+        # (bf16 with padded state rows: db / db_x come out of the dW / dW_x contractions, one / two kernels fewer)
+        "gpu_launches": (KERNELS_PER_STEP[kind] - ({"grad_tc": 1, "grad_lstm_tc": 2}.get(kind, 0) if cfg.get("H", 64) % 64 else 0)) * args.steps,
         "roofline": roof,
         "cpu_baseline": cpu,
         "phase_ms": mean_phase,

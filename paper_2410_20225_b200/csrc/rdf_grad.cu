@@ -1261,12 +1261,13 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         a.A = tc_lstm ? c.dg_bf : c.dz_bf; a.lda = tc_lstm ? 5 * c.Hp : c.Hp; a.Mp = tc_lstm ? 5 * c.Hp : c.Hp;
         a.Np = 2 * c.Hp; a.mode = 0; a.out = grads->dW; a.ldo = 2 * H;
         a.a_tiles = tc_rnn ? 1 : 0;
-        a.bias_out = tc_rnn && H < c.Hp ? grads->db : nullptr;      // db comes out of the same contraction
+        a.bias_out = H < c.Hp ? grads->db : nullptr;                // db comes out of the same contraction
         launch_dw(a, max_cells);
         if (tc_lstm) {
             DwArgs x{};
             x.ops = c.leaf_ops; x.count = &c.ctl->all_leaves;
             x.A = c.dg_bf; x.lda = 5 * c.Hp; x.Mp = 3 * c.Hp; x.Np = c.Hp; x.mode = 1; x.out = grads->dW_x; x.ldo = D;
+            x.bias_out = H < c.Hp ? grads->db_x : nullptr;
             launch_dw(x, max_leaves);
         }
     } else {
@@ -1278,7 +1279,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     }
     rdf_mark(S, 6, stream);
-    if (tc_rnn && H < c.Hp) {}          // (column H of the dW contraction)
+    if (c.use_tc && H < c.Hp) {}        // (column H of the dW / dW_x contractions)
     else if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);   // dz rows are in all_cells order
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
         rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);

@@ -523,6 +523,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                         hv[i] = __bfloat162float(hb[i]);        // the h every consumer sees is the bf16 value
                         cv[i] = cc;
                     }
+                    if (u0 == H) hb[0] = __float2bfloat16_rn(1.f);            // first pad column of the bf16 row: the constant
+                    else if (u0 + 4 == H) hb[4] = __float2bfloat16_rn(1.f);   // input (see tc_leaf_rows); H is a multiple of 4
                     *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + u0) = *reinterpret_cast<const uint4*>(hb);
                     float* st = c.arena + (size_t)it.x * S;
 #pragma unroll
@@ -594,9 +596,10 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
 
 // Leaves in bf16 mode: state(slot) = bf16(E[tok]), pad columns of the row zero.  Each warp takes four
 // leaves at a time, so that four rows are in flight per warp.
-// TreeRNN state rows carry the constant 1 in their first pad column (column H, when H < Hp): the packed weights
-// have zero rows there, so no contraction of the forward or the gradient pass sees it, and the weight-gradient
-// contraction dz (x) [h_l ; h_r] yields the bias gradient sum_t dz_t as its column H.
+// bf16 state rows (and, for the TreeLSTM, the bf16 embedding rows) carry the constant 1 in their first pad column
+// (column H, when H < Hp): the packed weights have zero rows there, so no contraction of the forward or the gradient
+// pass sees it, and the weight-gradient contraction dz (x) [h_l ; h_r] yields the bias gradient sum_t dz_t as its
+// column H.
 static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
     const int H = c.H, Hp = c.Hp;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
@@ -691,6 +694,7 @@ static __global__ void __launch_bounds__(256) rdf_pack_e_kernel(const DevCtx c) 
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
         const size_t v = idx / c.Hp;
         const int k = (int)(idx % c.Hp);
-        c.E_bf[idx] = __float2bfloat16_rn(k < c.D ? c.E[v * c.D + k] : 0.f);
+        // (first pad column: the constant 1, so that the leaf weight-gradient contraction also yields the leaf bias gradient)
+        c.E_bf[idx] = __float2bfloat16_rn(k < c.D ? c.E[v * c.D + k] : k == c.D ? 1.f : 0.f);
     }
 }
