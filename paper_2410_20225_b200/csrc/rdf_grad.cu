@@ -259,6 +259,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
     const int H = c.H, Hp = c.Hp, C = c.n_classes;
     const uint32_t rowbytes = (uint32_t)Hp * 2u, stride = rowbytes + 16u, stage_bytes = LM_ROWS * stride;
     const uint32_t mbar = smem_u32(mbars), stage0 = smem_u32(slab_smem);
+    int lab_next = 0;                                  // this thread's label of the slab that was issued last
     // stale rows of a short last slab must at least be finite: they meet dlog = 0 in the dW_s contraction
     for (uint32_t q = tid; q < 2 * stage_bytes / 16; q += 256) reinterpret_cast<uint4*>(slab_smem)[q] = make_uint4(0u, 0u, 0u, 0u);
     if (tid == 0) {
@@ -275,7 +276,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
         if (tid < (int)cnt) {
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(stage0 + (i & 1) * stage_bytes + tid * stride), "l"(c.arena_bf + (size_t)(fs + tid) * Hp), "r"(rowbytes), "r"(mb) : "memory");
-            s_lab[i & 1][tid] = __ldg(&c.label[(int)c.frames[fs + tid].arg]);
+            lab_next = __ldg(&c.label[(int)c.frames[fs + tid].arg]);       // two dependent loads: used one slab later
         }
     };
     // W_s fragments of this warp's k half: b0 = (k = 16 ks + 2t, +1; class g), b1 = (k + 8, + 9; class g), hi and lo
@@ -301,7 +302,10 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
         for (int e = 0; e < 4; ++e) acc[m][e] = 0.f;
     float my_loss = 0.f, my_dbs = 0.f;
     bool ok = true;
-    if (n_slabs > 0) issue(0);
+    if (n_slabs > 0) {
+        issue(0);
+        if (tid < LM_ROWS) s_lab[0][tid] = lab_next;
+    }
     for (int i = 0; i < n_slabs; ++i) {
         if (i + 1 < n_slabs) issue(i + 1);             // its stage was released by the barrier that ended slab i - 1
         const uint32_t fs = f0 + (uint32_t)i * LM_ROWS, cnt = min((uint32_t)LM_ROWS, f1 - fs);
@@ -379,6 +383,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
         }
         if (tid < C)
             for (uint32_t fi = 0; fi < cnt; ++fi) my_dbs += s_dl[fi][tid];
+        if (tid < LM_ROWS) s_lab[(i + 1) & 1][tid] = lab_next;      // labels of slab i + 1 (loaded while this slab was worked on)
         __syncthreads();                               // the stage, s_z and s_dl are free again
     }
     if (n_slabs > 0) {
