@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         }
         __syncthreads();
         lap(cyc_c);
-        alive = grid_barrier<true>(c, &c.ctl->bar_ops.v, generation);
+        alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
     // (cell_items is the height-sorted list here: the launch passes cell_sorted in its place)
@@ -552,7 +552,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         first = end;
         __syncthreads();
         lap(cyc_c);
-        alive = grid_barrier<true>(c, &c.ctl->bar_ops.v, generation);
+        alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
     if constexpr (TC) tc_teardown(tc);

@@ -955,7 +955,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             }
             __syncthreads();
             lap(cyc_a);
-            if (!grid_barrier<true>(c, &c.ctl->bar2.v, generation)) break;
+            if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
             lap(cyc_b);
         }
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
@@ -975,7 +975,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             first = end;
             __syncthreads();
             lap(cyc_c);
-            if (!grid_barrier<true>(c, &c.ctl->bar2.v, generation)) break;
+            if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
             lap(cyc_b);
         }
         callees_done = thin;
