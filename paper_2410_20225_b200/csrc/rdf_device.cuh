@@ -187,6 +187,19 @@ __device__ __forceinline__ uint32_t aggregated_inc(uint32_t* counter) {
     return g.shfl(base, 0) + g.thread_rank();
 }
 
+// Two counters bumped by the same converged group: both atomics are in flight together (one L2 round trip
+// instead of two on the token's critical path).
+__device__ __forceinline__ void aggregated_inc2(uint32_t* ca, uint32_t* cb, uint32_t& a, uint32_t& b) {
+    cg::coalesced_group g = cg::coalesced_threads();
+    uint32_t ba = 0, bb = 0;
+    if (g.thread_rank() == 0) {
+        ba = atomicAdd(ca, g.size());
+        bb = atomicAdd(cb, g.size());
+    }
+    a = g.shfl(ba, 0) + g.thread_rank();
+    b = g.shfl(bb, 0) + g.thread_rank();
+}
+
 // What the operator kernel and the gradient pass need to know about scheduler wave w: how many
 // frames, ready cells and ready leaves existed at its end.  Written by one thread at a moment when
 // every block has finished wave w and none has begun wave w + 1.
@@ -313,6 +326,16 @@ __device__ __forceinline__ void trace_rec(const DevCtx& c, uint64_t tag, int64_t
     }
 }
 
+// The record of a new frame (frame-form tags): its caller's frame, the label of the call site, the argument.
+__device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label, int64_t arg,
+                                           uint32_t id) {
+    Frame f;
+    f.parent = (uint32_t)tag; f.label = label; f.arg = arg;
+    c.frames[id] = f;
+    c.children[(size_t)tag * c.K + labels[label].child_index] = id;
+    trace_rec(c, id, arg, 0, label, (uint32_t)tag);
+}
+
 // Call_i: <t, d> -> <i:t, d>.  Returns false (status set) when the tag cannot be formed.
 __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label,
                                          int64_t arg, uint64_t& out) {
@@ -333,12 +356,8 @@ __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* label
         set_status(c, RDF_ERR_FRAMES_FULL);
         return false;
     }
-    Frame f;
-    f.parent = (uint32_t)tag; f.label = label; f.arg = arg;
-    c.frames[id] = f;
-    c.children[(size_t)tag * c.K + labels[label].child_index] = id;
+    frame_init(c, labels, tag, label, arg, id);
     out = id;
-    trace_rec(c, out, arg, 0, label, (uint32_t)tag);
     return true;
 }
 

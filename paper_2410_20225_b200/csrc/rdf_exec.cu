@@ -43,8 +43,11 @@ __device__ __forceinline__ void load_program(const DevCtx& c, SharedProgram& sp)
 // that carries its state onwards in the next wave.
 __device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, const MatchNode& M, uint32_t wave, uint64_t tag,
                                           const int64_t* regs, ThreadStats& st) {
-    const uint32_t i = aggregated_inc(&c.ctl->cell_count.v);
-    if (i >= c.work_cap) {
+    // (global queue: the place in the list and the queue slot of the token that carries the state on are reserved together)
+    uint32_t i, slot = 0;
+    if (lq) i = aggregated_inc(&c.ctl->cell_count.v);
+    else aggregated_inc2(&c.ctl->cell_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
+    if (i >= c.work_cap || (!lq && slot >= c.qcap)) {
         set_status(c, RDF_ERR_QUEUE_FULL);
         return;
     }
@@ -57,7 +60,9 @@ __device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, con
     c.op_l[tag] = it.l;
     c.op_r[tag] = it.r;
     ++st.cells;
-    push_token(c, lq, wave, tag, (int64_t)(((uint64_t)it.height << 32) | (uint32_t)tag), (uint32_t)M.cont_pc);
+    const int64_t datum = (int64_t)(((uint64_t)it.height << 32) | (uint32_t)tag);
+    if (lq) push_token(c, lq, wave, tag, datum, (uint32_t)M.cont_pc);
+    else store_token(&c.q[(wave + 1) & 1][slot], tag, datum, (uint32_t)M.cont_pc);
 }
 
 // Runs one token through its segment and on through every continuation it
@@ -91,7 +96,19 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             case VM_JMP: pc = in.imm; break;
             case VM_CALL: {                                         // Call_i
                 uint64_t nt;
-                if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt)) return;
+                // frame-form tags, global queue: the new frame's id and the token's queue slot are reserved together
+                const bool fused = c.tag_mode != RDF_TAGS_PATH && lq == nullptr;
+                uint32_t slot = 0;
+                if (fused) {
+                    uint32_t id;
+                    aggregated_inc2(&c.ctl->frame_count.v, &c.ctl->qcount[(wave + 1) % 3].v, id, slot);
+                    if (id >= c.frame_cap) {
+                        set_status(c, RDF_ERR_FRAMES_FULL);
+                        return;
+                    }
+                    frame_init(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], id);
+                    nt = id;
+                } else if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt)) return;
                 ++st.invocations;
                 if (c.tag_mode == RDF_TAGS_PATH) {
                     const uint32_t d = (uint32_t)(nt >> RDF_DEPTH_SHIFT) & 63u;
@@ -101,7 +118,13 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                     c.frame_args[(size_t)nt * 2] = r[in.b];
                     c.frame_args[(size_t)nt * 2 + 1] = r[in.dst];
                 }
-                push_token(c, lq, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
+                if (fused) {
+                    if (slot >= c.qcap) {
+                        set_status(c, RDF_ERR_QUEUE_FULL);
+                        return;
+                    }
+                    store_token(&c.q[(wave + 1) & 1][slot], nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
+                } else push_token(c, lq, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
                 break;
             }
             case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)tag * 2 + in.imm - 1])); break;
@@ -167,8 +190,10 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             }
             case VM_EMBED:
             case VM_LEAF_LSTM: {
-                const uint32_t i = aggregated_inc(&c.ctl->leaf_count.v);
-                if (i >= c.work_cap) {
+                uint32_t i, slot = 0;
+                if (lq) i = aggregated_inc(&c.ctl->leaf_count.v);
+                else aggregated_inc2(&c.ctl->leaf_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
+                if (i >= c.work_cap || (!lq && slot >= c.qcap)) {
                     set_status(c, RDF_ERR_QUEUE_FULL);
                     return;
                 }
@@ -179,7 +204,8 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                 c.op_l[tag] = LEAF_MARK;
                 c.op_r[tag] = (uint32_t)it.tok;
                 ++st.leaves;
-                push_token(c, lq, wave, tag, (int64_t)tag, (uint32_t)in.imm);
+                if (lq) push_token(c, lq, wave, tag, (int64_t)tag, (uint32_t)in.imm);
+                else store_token(&c.q[(wave + 1) & 1][slot], tag, (int64_t)tag, (uint32_t)in.imm);
                 break;
             }
             default:   // VM_HALT
