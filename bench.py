@@ -113,8 +113,8 @@ def peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
 # (profiles/persistent_kernels_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 394.3e6, ("rdf_operator_kernel", 3, None): 297.3e6,
-                     ("rdf_scheduler_kernel", 3, None): 11.3e6}
+NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 396.0e6, ("rdf_operator_kernel", 3, None): 297.0e6,
+                     ("rdf_scheduler_kernel", 3, None): 10.8e6}
 
 # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
