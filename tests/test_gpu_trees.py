@@ -166,6 +166,19 @@ def test_treernn_bf16_padding_and_biases(H):
     check_grad(cfg, rdf.BF16)
 
 
+def test_treernn_bf16_tiny_and_all_leaf_batches():
+    """The tensor-core path on degenerate batches: a single leaf, only leaves (no cell at all: every contraction of
+    the gradient pass is empty), one cell, a handful of small trees."""
+    rng = np.random.default_rng(3)
+    p = workloads.treernn_params(9, 60, 64, 64, bf16=True)
+    p["b"] = workloads.bf16_round((0.2 * rng.standard_normal(64)).astype(np.float32))
+    for Ls in ([1], [1, 1, 1, 1], [2], [1, 3, 1, 2, 5]):
+        tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, L) for L in Ls], 7, vocab=60)
+        cfg = {"trees": tb, "params": p}
+        check_forward(cfg, rdf.BF16)
+        check_grad(cfg, rdf.BF16)
+
+
 def test_depth_stress_reduced():
     cfg = workloads.config(5, chains=3, chain_depth=300, perfect=2, perfect_height=7, V=400, H=32)
     st, _ = check_grad(cfg)
