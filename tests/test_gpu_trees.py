@@ -249,6 +249,21 @@ def test_treelstm_small_and_tiny():
     check_grad(_lstm_cfg(96, 500, 64), cell="lstm")
 
 
+def test_treelstm_bf16_tiny_and_all_leaf_batches():
+    """The tensor-core TreeLSTM on degenerate batches (a single leaf, only leaves, one cell, a few small trees), with
+    H = 64 (no pad column: bias gradients by column sums) and H = 40 (pad columns: bias gradients from the contractions)."""
+    rng = np.random.default_rng(4)
+    for H in (64, 40):
+        p = workloads.treelstm_params(9, 60, H, H, bf16=True)
+        for k in ("b", "b_x", "b_s"):
+            p[k] = workloads.bf16_round((0.1 * rng.standard_normal(p[k].shape)).astype(np.float32))
+        for Ls in ([1], [1, 1, 1, 1], [2], [1, 3, 1, 2, 5]):
+            tb = workloads.tree_batch_from_shapes([workloads.random_split_shape(rng, L) for L in Ls], 7, vocab=60)
+            cfg = {"trees": tb, "params": p}
+            check_forward(cfg, rdf.BF16, cell="lstm")
+            check_grad(cfg, rdf.BF16, cell="lstm")
+
+
 def test_treelstm_ragged_hidden_size():
     check_grad(_lstm_cfg(48, 700, 300), cell="lstm")
 
