@@ -4,9 +4,11 @@
 //      push / pop, Switch, token-store insert or match) and emits the next
 //      wave's tokens.  A vector value travels by reference (the frame that
 //      holds it), so a ready leaf / cell operator is queued, not computed: the
-//      kernel leaves behind, wave by wave, the lists of ready operators.
-//   Operator kernel: fires the ready operators of each wave as one batch, the
-//      waves in the order in which the scheduler formed them.
+//      kernel leaves behind the lists of ready operators, each cell with the
+//      height of the operator tree below it.
+//   Operator kernel: fires the ready operators as batches, the leaves first and
+//      then the cells height by height (grouped by three small kernels between
+//      the two): operands before results, in as few dependent waves as possible.
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
@@ -507,8 +509,8 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     }
 }
 
-// The operator kernel: the leaves first (they wait for nothing), then, wave by wave, the cells that
-// became ready in that wave; a grid barrier separates the waves (a cell reads states of earlier waves).
+// The operator kernel: the leaves first (they wait for nothing), then, height by height, the cells of that
+// height; a grid barrier separates the waves (a cell reads states of smaller heights).
 // TC: bf16 operands on the tensor cores (the tile pipeline of rdf_tc.cuh); otherwise fp32 FMA tiles.
 template <bool TC>
 __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
