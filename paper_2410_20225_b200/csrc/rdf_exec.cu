@@ -903,13 +903,18 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
         if (wide && L.arrived_bytes) CUDA_OK(cudaMemsetAsync(ws + L.arrived, 0, L.arrived_bytes, stream));
     }
     if (L.table_bytes) CUDA_OK(cudaMemsetAsync(ws + L.table, 0xFF, L.table_bytes, stream));
-    CUDA_OK(cudaMemcpyAsync(ws + L.code, g->code.data(), g->code.size() * sizeof(VmInstr), cudaMemcpyHostToDevice, stream));
-    if (!g->match.empty())
-        CUDA_OK(cudaMemcpyAsync(ws + L.match, g->match.data(), g->match.size() * sizeof(MatchNode), cudaMemcpyHostToDevice, stream));
-    if (!g->labels.empty())
-        CUDA_OK(cudaMemcpyAsync(ws + L.labels, g->labels.data(), g->labels.size() * sizeof(LabelInfo), cudaMemcpyHostToDevice, stream));
-    if (!g->consts.empty())
-        CUDA_OK(cudaMemcpyAsync(ws + L.consts, g->consts.data(), g->consts.size() * sizeof(int64_t), cudaMemcpyHostToDevice, stream));
+    {
+        // the four program tables sit next to each other in the workspace (code first, constants last): one copy
+        const size_t bytes = L.consts + g->consts.size() * sizeof(int64_t) - L.code;
+        if (S->tables.size() != bytes) {
+            S->tables.assign(bytes, 0);
+            memcpy(S->tables.data(), g->code.data(), g->code.size() * sizeof(VmInstr));
+            if (!g->match.empty()) memcpy(S->tables.data() + (L.match - L.code), g->match.data(), g->match.size() * sizeof(MatchNode));
+            if (!g->labels.empty()) memcpy(S->tables.data() + (L.labels - L.code), g->labels.data(), g->labels.size() * sizeof(LabelInfo));
+            if (!g->consts.empty()) memcpy(S->tables.data() + (L.consts - L.code), g->consts.data(), g->consts.size() * sizeof(int64_t));
+        }
+        CUDA_OK(cudaMemcpyAsync(ws + L.code, S->tables.data(), bytes, cudaMemcpyHostToDevice, stream));
+    }
     rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
     CUDA_OK(cudaGetLastError());
     if (c.use_tc) {

@@ -1,6 +1,7 @@
 // Shared between the forward executor (rdf_exec.cu) and the gradient pass
 // (rdf_grad.cu): workspace layout, per-graph host state, the fp32 tile step.
 #pragma once
+#include <vector>
 #include "rdf_device.cuh"
 
 // ---- fp32 tiled contraction: 64 x 64 output tile, 16-deep steps, 256 threads, 4 x 4 per thread
@@ -52,6 +53,9 @@ struct ExecState {
     cudaEvent_t ev[RDF_PHASE__COUNT + 1] = {};
     bool have_events = false;
     int n_phases = 0;
+    // the lowered program (code, match nodes, labels, constants) as one block with the workspace's own spacing, so that
+    // every call copies it to the device in one piece
+    std::vector<char> tables;
 };
 
 // records the boundary after phase `k - 1` (k = 0: start of the call)
