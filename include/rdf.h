@@ -51,10 +51,10 @@ enum {
 
 /* ----------------------------------------------------------------- program
  * A program is a set of function definitions, one of which is `result`
- * (Section 3, "Assume we are given a set S of dataflow graphs ...").  Each
- * definition is an expression DAG over its formal parameters.  A CALL node is
- * a node "labeled with the name of f" (Section 2.4, Figure 2); IF is the
- * Switch/Merge conditional of Figure 2.
+ * (Section 3, the statement of the transformation's input).  Each definition
+ * is an expression DAG over its formal parameters.  A CALL node is one of the
+ * function-call nodes of Section 2.4, Figure 2; IF is the Switch/Merge
+ * conditional of the same figure.
  */
 typedef enum {
     RDF_OP_PARAM = 0,    /* imm = parameter index                                   */
@@ -267,7 +267,10 @@ int rdf_eval(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_ou
  * start from zero on `stream` before its kernels run, but two calls that overlap
  * on the GPU (different streams, or different graphs used concurrently) race on
  * it -- keep calls to this entry point ordered on one stream per device.
- * Everything else (arguments, outputs, status reporting) is as for rdf_eval. */
+ * The status word and the counters that rdf_last_status reports live in the same
+ * array: read them before the next call to this entry point on that device (with
+ * any graph), or they describe that later call.
+ * Everything else (arguments, outputs) is as for rdf_eval. */
 #define RDF_NOALLOC_SCRATCH_BYTES (16u << 20)
 int rdf_eval_noalloc(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out,
                      void* stream);
@@ -286,6 +289,17 @@ int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_ou
 int rdf_last_status(rdf_graph* g, rdf_stats* s);
 
 const char* rdf_strerror(int status);
+
+/* Limits of the device executor for the following calls on this graph (the paper's
+ * executor simply runs until both queues are empty, Section 5.1; these guards have
+ * no counterpart there).
+ *   wait_cycles : SM clock cycles a device-side wait (grid barrier, mbarrier) may last before the
+ *                 kernel gives up with RDF_ERR_TIMEOUT; 0 restores the default (about two seconds).
+ *   wave_limit  : scheduler waves a call may run before it stops with RDF_ERR_WAVE_LIMIT (the
+ *                 guard against recursion that never reaches a base case); 0 restores the
+ *                 default (2^24 for integer programs, twice the frame capacity for tree programs).
+ * A call that ends with either status leaves the graph usable: the next call starts clean. */
+int rdf_set_limits(rdf_graph* g, long long wait_cycles, long long wave_limit);
 
 /* Measurement aid (the paper reports only wall-clock times, Section 6; there is
  * no counterpart to cite): when enabled, rdf_eval / rdf_grad record CUDA events

@@ -23,7 +23,7 @@ class Node:
     value: object = None  # constant value / parameter index / label i
     func: str = ""       # the function graph this node came from
     n_in: int = 0        # number of data input ports
-    param: int = 0       # for 'Call'/'merge' made from parameter k: k
+    param: int = 0       # for 'Call'/'merge' made from parameter k: k; for 'Return'/'out' of output j: j
 
 
 @dataclass
@@ -69,7 +69,14 @@ class FunctionGraph:
         self.n_params = n_params
         self.g = Graph()
         self.inputs = [self.g.add("in", value=k, func=name) for k in range(n_params)]
-        self.out = None
+        self.out = None          # the output node (the first one of a function with several outputs)
+        self.outs = []           # all output nodes, in order
+        # For a function that pairs a forward computation with its gradient computation (Section 4): which
+        # parameters and which outputs belong to the gradient half.  The control edge Call_i -> Return_i is
+        # drawn between nodes of the same half only (the forward Return_i must not wait for the gradient
+        # Call_i, which fires in the backward phase).
+        self.grad_params = set()
+        self.grad_outputs = set()
 
     def param(self, k=0):
         return (self.inputs[k], 0)
@@ -102,7 +109,19 @@ class FunctionGraph:
             self.g.connect(s, nid, p, src_port=sp)
         return (nid, 0)
 
+    def call_open(self, fname, n_args):
+        """A call node whose arguments are connected afterwards with `set_arg` (needed where an argument
+        depends on one of the call's own outputs, as the gradient input of a paired call does).
+        Output j of the callee is the value (node, j)."""
+        return self.g.add("fcall", name=fname, func=self.name, n_in=n_args)
+
+    def set_arg(self, call_node, port, v):
+        self.g.connect(v[0], call_node, port, src_port=v[1])
+
     def output(self, v):
-        self.out = self.g.add("out", func=self.name, n_in=1)
-        self.g.connect(v[0], self.out, 0, src_port=v[1])
-        return self.out
+        nid = self.g.add("out", func=self.name, n_in=1, param=len(self.outs))
+        self.g.connect(v[0], nid, 0, src_port=v[1])
+        self.outs.append(nid)
+        if self.out is None:
+            self.out = nid
+        return nid

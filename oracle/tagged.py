@@ -50,7 +50,8 @@ class RunResult:
     def __init__(self):
         self.outputs = {}        # tag -> datum, tokens that reached the output node
         self.calls = {}          # tag after the push (tuple) -> argument datum(s) by parameter
-        self.returns = {}        # tag before the pop (tuple) -> returned datum
+        self.returns = {}        # tag before the pop (tuple) -> returned datum (output 0 of the function)
+        self.returns_by_output = {}   # (tag, output index) -> returned datum, for functions with several outputs
         self.firings = 0
         self.max_depth = 0
         self.leftover = 0        # tokens still waiting when the queue ran empty
@@ -157,7 +158,9 @@ def run(graph, feeds, ops, dead_tokens=True, max_firings=None) -> RunResult:
                     emit(nid, 0, tag[1:], DEAD)
                 elif key in held:
                     d = held.pop(key)
-                    res.returns[tag] = d
+                    res.returns_by_output[(tag, n.param)] = d
+                    if n.param == 0:
+                        res.returns[tag] = d
                     emit(nid, 0, tag[1:], d)
                 else:
                     ctrl[key] = True
@@ -167,7 +170,9 @@ def run(graph, feeds, ops, dead_tokens=True, max_firings=None) -> RunResult:
                 if not tag or tag[0] != n.value:
                     continue                      # label mismatch: no output
                 if ctrl.pop(key, False):
-                    res.returns[tag] = datum
+                    res.returns_by_output[(tag, n.param)] = datum
+                    if n.param == 0:
+                        res.returns[tag] = datum
                     emit(nid, 0, tag[1:], datum)
                 else:
                     held[key] = datum

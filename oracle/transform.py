@@ -17,14 +17,20 @@ One more kind of edge comes from Figure 3 rather than from the list: inside a
 called function every constant gets a control edge from the entry Merge, so
 that it emits once per activation (the figure draws Merge -> 1 twice).
 
+Functions with several outputs (the paired function of Section 4 has m + n of
+them: the outputs of f and the gradient outputs of f^grad) get one Return_i per
+output and call site; output j of call node i feeds the consumers of that
+output.  The control edge of step 5 connects the Call_i and Return_i nodes of
+the same half (forward or gradient) of such a function.
+
 Readings taken where the text is silent:
-  * the numbering order is free ("not important which node receives which
-    number"); here call nodes are numbered in the order result-first, then the
+  * the numbering order is free (Section 3 says any assignment of the numbers
+    works); here call nodes are numbered in the order result-first, then the
     other graphs in the order given, nodes in creation order.  For the
     factorial example this gives Call_0 in `result` and Call_1 in `fact`, as
     in Figure 3.
-  * numbering restarts at 0 for every callee f, as the text numbers "the nodes
-    labeled with the name of f".
+  * numbering restarts at 0 for every callee f: step 1 numbers the call nodes
+    of one f at a time.
 """
 from __future__ import annotations
 
@@ -46,7 +52,7 @@ def transform(functions, result_name: str = "result") -> Graph:
         for e in f.g.edges:
             g.connect(e.src + off, e.dst + off, e.dst_port, e.src_port, e.control)
         in_of[f.name] = [i + off for i in f.inputs]
-        out_of[f.name] = f.out + off
+        out_of[f.name] = [o + off for o in f.outs]
     removed = set()
 
     for f in fs:
@@ -66,9 +72,12 @@ def transform(functions, result_name: str = "result") -> Graph:
             node = g.nodes[nid]
             node.kind, node.name, node.param, node.n_in = "merge", "entry", k, n_calls
             entry.append(nid)
-        # the single edge that feeds f's output node
-        (out_edge,) = g.in_edges(out_of[f.name])
-        removed.add(out_of[f.name])
+        # the single edge that feeds each output node of f
+        out_edges = []
+        for o in out_of[f.name]:
+            (oe,) = g.in_edges(o)
+            out_edges.append(oe)
+            removed.add(o)
         for i, c in enumerate(calls):
             # step 2: m nodes Call_i, each with the one input of its parameter
             call_nodes = []
@@ -80,14 +89,18 @@ def transform(functions, result_name: str = "result") -> Graph:
                 # step 3 (edge part)
                 g.connect(cid, entry[k], i)
                 call_nodes.append(cid)
-            # step 4: Return_i takes f's output and feeds the old consumers
-            rid = g.add("Return", name=f.name, value=i, func=g.nodes[c].func, n_in=1)
-            g.connect(out_edge.src, rid, 0, src_port=out_edge.src_port)
-            for e in g.out_edges(c):
-                g.connect(rid, e.dst, e.dst_port, 0, e.control)
-            # step 5: control edge(s) Call_i -> Return_i
-            for cid in call_nodes:
-                g.connect(cid, rid, -1, control=True)
+            # step 4: Return_i takes f's output and feeds the old consumers (one Return_i per output)
+            consumers = g.out_edges(c)
+            for j, out_edge in enumerate(out_edges):
+                rid = g.add("Return", name=f.name, value=i, func=g.nodes[c].func, n_in=1, param=j)
+                g.connect(out_edge.src, rid, 0, src_port=out_edge.src_port)
+                for e in consumers:
+                    if e.src_port == j:
+                        g.connect(rid, e.dst, e.dst_port, 0, e.control)
+                # step 5: control edge(s) Call_i -> Return_i
+                for k, cid in enumerate(call_nodes):
+                    if (k in f.grad_params) == (j in f.grad_outputs):
+                        g.connect(cid, rid, -1, control=True)
             removed.add(c)
         # Figure 3: constants of a called function are triggered by its entry Merge
         for n in g.nodes:

@@ -111,7 +111,8 @@ class rdf_stats(C.Structure):
 
 
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
-           "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc"]
+           "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc",
+           "rdf_set_limits"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 PHASES = ["setup", "schedule", "operators", "loss", "backward", "dW", "db", "dE"]
 
@@ -138,6 +139,7 @@ def lib() -> C.CDLL:
                                        C.POINTER(rdf_outputs), C.c_void_p]
         L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
         L.rdf_set_profiling.argtypes = [C.c_void_p, C.c_int]
+        L.rdf_set_limits.argtypes = [C.c_void_p, C.c_longlong, C.c_longlong]
         L.rdf_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
         L.rdf_strerror.argtypes = [C.c_int]
         L.rdf_strerror.restype = C.c_char_p
@@ -343,6 +345,12 @@ class Graph:
         if rc != RDF_OK:
             raise RdfError(rc, "rdf_set_profiling")
 
+    def set_limits(self, wait_cycles=0, wave_limit=0):
+        """Bound of the device-side waits (SM cycles) and of the number of scheduler waves; 0 = default."""
+        rc = lib().rdf_set_limits(self.handle, int(wait_cycles), int(wave_limit))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_set_limits")
+
     def phase_ms(self):
         """{phase name: milliseconds} of the last call (needs set_profiling(True) before it)."""
         ms = (C.c_float * len(PHASES))()
@@ -417,6 +425,22 @@ class Graph:
         if check:
             self.stats()
         return y
+
+    def eval_trees_noalloc(self, dt, dp, h_root, compute=F32, check=True):
+        """rdf_eval_noalloc for a tree network: inputs dt/dp and the output h_root ([B, H] float32 CUDA
+        tensor) are the caller's; scratch is the library's built-in array."""
+        torch = _torch()
+        batch = self._batch(dt)
+        params = self._params(dp, compute)
+        out = rdf_outputs()
+        out.h_root = h_root.data_ptr()
+        rc = lib().rdf_eval_noalloc(self.handle, C.byref(batch), C.byref(params), C.byref(out),
+                                    torch.cuda.current_stream().cuda_stream)
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_eval_noalloc")
+        if check:
+            self.stats()
+        return h_root
 
     # ---- tree programs
     @staticmethod

@@ -29,9 +29,11 @@ static_assert(sizeof(Token) == 32, "two 128-bit words");
 // the reference to the previous scope (Section 5.1).
 struct __align__(16) Frame {
     uint32_t parent;
-    uint32_t label;
+    uint32_t label;               // [7:0] label i of the Call_i that made the frame, [31:8] the scheduler wave it fired in
     int64_t  arg;
 };
+static const uint32_t FRAME_LABEL_MASK = 0xFFu;
+static const int FRAME_WAVE_SHIFT = 8;
 
 // Hash-store slot: a parked operand keyed by the packed tag.
 struct __align__(16) Slot {
@@ -149,10 +151,10 @@ struct DevCtx {
     float*    dhp;                // [frame_cap, S]: gradient arriving from the caller (dh, and dc for the TreeLSTM);
                                   //                 TreeRNN: overwritten by dz (cell) / dh (leaf)
     float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
-    uint4*    wave_marks;         // [wave_cap]: {frames, cells, leaves} counted up to the end of scheduler wave w.
+    uint4*    wave_marks;         // [wave_cap], filled by the list kernels of the gradient pass: .x = frames created up to
+                                  // the end of scheduler wave w (0: none in that wave), .w = cells among them.
                                   // Frame ids are handed out in wave order, so the invocations that Call_i created
-                                  // in wave w are the id range [marks[w-1].x, marks[w].x) -- one wave of the gradient
-                                  // pass; the cells that became ready in wave w are cell_items[marks[w-1].y, marks[w].y)
+                                  // in wave w are one id range -- one wave of the gradient pass
     uint32_t  wave_cap;
     uint32_t* all_cells;          // every cell frame, in backward wave order
     uint4*    cell_ops;           // {cell frame, left operand frame, right operand frame, 1} in all_cells order
@@ -200,40 +202,26 @@ __device__ __forceinline__ void aggregated_inc2(uint32_t* ca, uint32_t* cb, uint
     b = g.shfl(bb, 0) + g.thread_rank();
 }
 
-// What the operator kernel and the gradient pass need to know about scheduler wave w: how many
-// frames, ready cells and ready leaves existed at its end.  Written by one thread at a moment when
-// every block has finished wave w and none has begun wave w + 1.
-__device__ __forceinline__ void mark_wave(const DevCtx& c, uint32_t wave) {
-    if (c.wave_marks && wave < c.wave_cap)
-        c.wave_marks[wave] = make_uint4(ld_volatile_u32(&c.ctl->frame_count.v), ld_volatile_u32(&c.ctl->cell_count.v),
-                                        ld_volatile_u32(&c.ctl->leaf_count.v), 0u);
-}
-static const uint32_t NO_MARK = 0xFFFFFFFFu;
-
 // Grid-wide barrier with a bounded wait.  All blocks of the (cooperatively
 // launched, hence co-resident) grid call it the same number of times.  The
 // counter only grows; generation k is complete when it reaches k * gridDim.x.
 // Returns false when the wait expired or any block reported an error; the
-// caller then leaves the kernel.  With mark != NO_MARK the last block to arrive
-// (all others have finished their work, none has left the barrier) records the
-// counts of scheduler wave `mark`.
-// The arrival is a release atomic and the wait polls with acquire loads (GPU scope): what a block wrote before
-// the barrier is visible to every block that sees the full count, and no separate fence has to wait for the
-// stores and atomics still in flight (fences around a relaxed atomic cost the gradient kernel 0.05 ms of its
-// 0.47 ms on the headline workload).
-__device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter, uint32_t& generation,
-                                             uint32_t mark = NO_MARK) {
+// caller then leaves the kernel.
+// The arrival is a release reduction (no value comes back, so the thread goes straight on to poll) and the
+// wait polls with acquire loads (GPU scope): what a block wrote before the barrier is visible to every block
+// that sees the full count, and no separate fence has to wait for the stores and atomics still in flight.
+// The status word is looked at every few polls, so that a block that is still waiting when another block has
+// reported an error leaves at once instead of waiting for its own limit.
+__device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter, uint32_t& generation) {
     __shared__ int ok;
     __syncthreads();
     if (threadIdx.x == 0) {
         ++generation;
         const uint32_t target = generation * gridDim.x;
-        uint32_t before;
-        asm volatile("atom.add.release.gpu.global.u32 %0, [%1], 1;" : "=r"(before) : "l"(counter) : "memory");
-        if (mark != NO_MARK && before + 1 == target) mark_wave(c, mark);
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
         const long long t0 = clock64();
         int good = 1;
-        for (;;) {
+        for (uint32_t polls = 0;; ++polls) {
             uint32_t seen;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if (seen >= target) break;
@@ -242,7 +230,10 @@ __device__ __forceinline__ bool grid_barrier(const DevCtx& c, uint32_t* counter,
                 good = 0;
                 break;
             }
-            __nanosleep(32);
+            if ((polls & 15u) == 15u && ld_volatile_i32(&c.ctl->status) != 0) {
+                good = 0;
+                break;
+            }
         }
         if (ld_volatile_i32(&c.ctl->status) != 0) good = 0;
         ok = good;
@@ -327,10 +318,12 @@ __device__ __forceinline__ void trace_rec(const DevCtx& c, uint64_t tag, int64_t
 }
 
 // The record of a new frame (frame-form tags): its caller's frame, the label of the call site, the argument.
+// The record also keeps the scheduler wave in which the call fired: ids are handed out wave after wave, so
+// the frames of one wave are one id range, and the gradient pass finds the ranges from these fields.
 __device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label, int64_t arg,
-                                           uint32_t id) {
+                                           uint32_t id, uint32_t wave) {
     Frame f;
-    f.parent = (uint32_t)tag; f.label = label; f.arg = arg;
+    f.parent = (uint32_t)tag; f.label = label | (wave << FRAME_WAVE_SHIFT); f.arg = arg;
     c.frames[id] = f;
     c.children[(size_t)tag * c.K + labels[label].child_index] = id;
     trace_rec(c, id, arg, 0, label, (uint32_t)tag);
@@ -338,7 +331,7 @@ __device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* lab
 
 // Call_i: <t, d> -> <i:t, d>.  Returns false (status set) when the tag cannot be formed.
 __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label,
-                                         int64_t arg, uint64_t& out) {
+                                         int64_t arg, uint64_t& out, uint32_t wave) {
     if (c.tag_mode == RDF_TAGS_PATH) {
         const uint32_t depth = (uint32_t)(tag >> RDF_DEPTH_SHIFT) & 63u;
         if ((depth + 1) * (uint32_t)c.label_bits > (uint32_t)RDF_PATH_BITS) {
@@ -356,7 +349,7 @@ __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* label
         set_status(c, RDF_ERR_FRAMES_FULL);
         return false;
     }
-    frame_init(c, labels, tag, label, arg, id);
+    frame_init(c, labels, tag, label, arg, id, wave);
     out = id;
     return true;
 }
@@ -371,7 +364,7 @@ __device__ __forceinline__ void tag_pop(const DevCtx& c, uint64_t tag, uint32_t&
                  (path >> c.label_bits);
     } else {
         const uint4 f = __ldcg(reinterpret_cast<const uint4*>(&c.frames[tag]));   // {parent, label, arg}
-        label = f.y;
+        label = f.y & FRAME_LABEL_MASK;
         parent = f.x;
     }
 }

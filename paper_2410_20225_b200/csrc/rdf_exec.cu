@@ -12,6 +12,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <type_traits>
 
 #include "rdf_exec.h"
@@ -90,10 +91,19 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             case VM_REM: r[in.dst] = r[in.b] == 0 ? 0 : r[in.a] % r[in.b]; break;
             case VM_LT: r[in.dst] = r[in.a] < r[in.b]; break;
             case VM_EQ: r[in.dst] = r[in.a] == r[in.b]; break;
-            case VM_ISLEAF: r[in.dst] = __ldg(&c.left[r[in.a]]) < 0; break;
-            case VM_LEFT: r[in.dst] = __ldg(&c.left[r[in.a]]); break;
-            case VM_RIGHT: r[in.dst] = __ldg(&c.right[r[in.a]]); break;
-            case VM_TOK: r[in.dst] = __ldg(&c.tok[r[in.a]]); break;
+            case VM_ISLEAF: case VM_LEFT: case VM_RIGHT: case VM_TOK: {
+                // accessors of the caller's flat tree arrays: an index outside [0, N) is the caller's mistake and
+                // ends the token with a status code, never with an access
+                const int64_t v = r[in.a];
+                if (v < 0 || v >= c.N) {
+                    set_status(c, RDF_ERR_BAD_ARG);
+                    return;
+                }
+                const int32_t* arr = in.op == VM_RIGHT ? c.right : in.op == VM_TOK ? c.tok : c.left;
+                const int32_t x = __ldg(&arr[v]);
+                r[in.dst] = in.op == VM_ISLEAF ? (int64_t)(x < 0) : (int64_t)x;
+                break;
+            }
             case VM_BRZ: if (r[in.a] == 0) pc = in.imm; break;     // Switch: the false side
             case VM_JMP: pc = in.imm; break;
             case VM_CALL: {                                         // Call_i
@@ -108,9 +118,9 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                         set_status(c, RDF_ERR_FRAMES_FULL);
                         return;
                     }
-                    frame_init(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], id);
+                    frame_init(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], id, wave);
                     nt = id;
-                } else if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt)) return;
+                } else if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt, wave)) return;
                 ++st.invocations;
                 if (c.tag_mode == RDF_TAGS_PATH) {
                     const uint32_t d = (uint32_t)(nt >> RDF_DEPTH_SHIFT) & 63u;
@@ -192,6 +202,10 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             }
             case VM_EMBED:
             case VM_LEAF_LSTM: {
+                if (r[in.a] < 0 || r[in.a] >= c.V) {             // a token id that is no row of the embedding table
+                    set_status(c, RDF_ERR_BAD_ARG);
+                    return;
+                }
                 uint32_t i, slot = 0;
                 if (lq) i = aggregated_inc(&c.ctl->leaf_count.v);
                 else aggregated_inc2(&c.ctl->leaf_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
@@ -418,7 +432,6 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                         run_token(c, sp, &lq, wave, t, st);
                     }
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
-                    if (threadIdx.x == 0) mark_wave(c, wave);
                     if (k == 0) {
                         // The end of the stretch rewrites the counters that the other blocks read to take this
                         // branch: carry on only when all of them have arrived at the grid barrier below (they
@@ -434,7 +447,10 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                                     good = 0;
                                     break;
                                 }
-                                __nanosleep(32);
+                                if (ld_volatile_i32(&c.ctl->status) != 0) {       // another block gave up: so does this one
+                                    good = 0;
+                                    break;
+                                }
                             }
                             others_in = good;
                         }
@@ -475,7 +491,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
             run_token(c, sp, nullptr, wave, load_token(&q[i]), st);
         __syncthreads();
         lap(cyc_s);
-        if (!grid_barrier(c, &c.ctl->bar.v, generation, wave)) break;
+        if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
         lap(cyc_b);
     }
     flush_stats(c, st);
@@ -499,7 +515,7 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     } else {
         tag = (uint64_t)b;            // frames 0..B-1 are the contexts of `result`
         Frame f;
-        f.parent = LEAF_MARK; f.label = 0; f.arg = datum;
+        f.parent = LEAF_MARK; f.label = 0; f.arg = datum;          // (wave field 0: before the first wave)
         c.frames[b] = f;
     }
     store_token(&c.q[0][b], tag, datum, (uint32_t)c.result_entry_pc);
@@ -867,7 +883,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.loss_out = out->loss;
     c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
     c.wave_limit = L.wave_cap ? L.wave_cap : 1u << 24;
-    c.spin_limit = (long long)S->clock_khz * 2000ll;       // about two seconds of SM clock
+    if (S->wave_limit > 0) c.wave_limit = (uint32_t)std::min<long long>(S->wave_limit, c.wave_limit);
+    c.spin_limit = S->wait_cycles > 0 ? S->wait_cycles : (long long)S->clock_khz * 2000ll;       // default: about two seconds of SM clock
 }
 
 int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, void* ws) {
@@ -1010,6 +1027,14 @@ extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
     return h.status;
 }
 
+extern "C" int rdf_set_limits(rdf_graph* g, long long wait_cycles, long long wave_limit) {
+    if (!g || wait_cycles < 0 || wave_limit < 0) return RDF_ERR_BAD_ARG;
+    ExecState* S = rdf_state_of(g);
+    S->wait_cycles = wait_cycles;
+    S->wave_limit = wave_limit;
+    return RDF_OK;
+}
+
 extern "C" int rdf_set_profiling(rdf_graph* g, int enable) {
     if (!g) return RDF_ERR_BAD_ARG;
     ExecState* S = rdf_state_of(g);
@@ -1048,11 +1073,13 @@ namespace {
 // that cudaGetSymbolAddress returns for the device that is current.
 const int kMaxDevices = 64;
 void* g_builtin_scratch[kMaxDevices] = {};
+std::mutex g_builtin_scratch_lock;      // first calls may come from several host threads
 
 int builtin_scratch(void** out) {
     int dev = 0;
     CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return RDF_ERR_BAD_ARG;
+    std::lock_guard<std::mutex> hold(g_builtin_scratch_lock);
     if (!g_builtin_scratch[dev]) {
         void* p = nullptr;
         CUDA_OK(cudaGetSymbolAddress(&p, rdf_builtin_scratch));

@@ -48,6 +48,8 @@ struct ExecState {
     void* last_ctl = nullptr;
     cudaStream_t last_stream = nullptr;
     bool ran = false;
+    long long wait_cycles = 0;   // rdf_set_limits: 0 = default
+    long long wave_limit = 0;
     // optional phase timing
     bool profiling = false;
     cudaEvent_t ev[RDF_PHASE__COUNT + 1] = {};

@@ -429,6 +429,8 @@ __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int
 // so listing the cells in frame order puts the cells of every gradient wave next to each other:
 // wave d owns all_cells[marks[d-1].w, marks[d].w), the rows of its operand-gradient contraction.
 // Three small kernels: per-segment counts, scan of the counts, fill (and the per-wave ends).
+// Where a wave ends in the id space is read off the frames themselves (every frame records the scheduler
+// wave its Call_i fired in): marks[w].x = one past the last frame of wave w, 0 for a wave without calls.
 static const int LIST_SEG = 2048;            // frames per segment (256 threads x 8)
 
 __device__ __forceinline__ void list_flags(const DevCtx& c, uint32_t f0, uint32_t F, uint32_t (&l)[8], uint32_t (&r)[8],
@@ -462,6 +464,10 @@ __global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uin
         for (int w = 0; w < 8; ++w) { a += wc[w]; b += wl[w]; }
         seg_counts[blockIdx.x] = make_uint2(a, b);
     }
+    // the marks of this call's waves start empty (the fill kernel writes the ends of the waves that made calls)
+    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
+    for (uint32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_waves; w += gridDim.x * blockDim.x)
+        c.wave_marks[w] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // one block: exclusive scan of the segment counts in place; totals to the control block
@@ -516,6 +522,19 @@ __global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, cons
     const uint2 sb = seg_base[blockIdx.x];
     uint32_t ic = sb.x + pc - cells, il = sb.y + pl - leaves;
     for (int w = 0; w < warp; ++w) { ic += wc[w]; il += wl[w]; }
+    // ends of the waves in the id space: frame f is the last of its wave when the next frame belongs to a later one
+    {
+        const uint32_t fa = f0 + threadIdx.x * 8;
+        uint32_t wv = fa < F ? c.frames[fa].label >> FRAME_WAVE_SHIFT : 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t f = fa + i;
+            if (f >= F) break;
+            const uint32_t wn = f + 1 < F ? c.frames[f + 1].label >> FRAME_WAVE_SHIFT : 0xFFFFFFFFu;
+            if (wn != wv && wv < c.wave_cap) c.wave_marks[wv].x = f + 1;
+            wv = wn;
+        }
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const uint32_t f = f0 + threadIdx.x * 8 + i;

@@ -87,8 +87,65 @@ void validate(const Prog& P) {
     }
 }
 
+// --------------------------------------------------------------- value kinds
+// An expression is integer-valued or vector-valued (a state of the tree networks).  What the device
+// executor supports: integer operators, conditions, accessors and call arguments take integers; a cell
+// takes the results of two calls (it reads the states that the two callee invocations left in their
+// frames), so an invocation fires at most one vector operator and a cell invocation makes exactly two
+// calls -- which is what the per-invocation state slot and the sizing of the cell lists rely on.
+// Anything else is a valid program that this executor does not lower: RDF_ERR_UNSUPPORTED.
+void check_kinds(const Prog& P) {
+    const int nf = P.p->n_functions;
+    std::vector<int> fvec(nf, 0);                  // function returns a vector (fixpoint from "integer")
+    std::function<int(int, int)> kind = [&](int f, int e) -> int {
+        const rdf_expr& x = P.ex(f, e);
+        switch (x.op) {
+            case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
+            case RDF_OP_NODE_LOSS: return 1;
+            case RDF_OP_CALL: return fvec[x.imm];
+            case RDF_OP_IF: return kind(f, x.b) | kind(f, x.c);
+            default: return 0;
+        }
+    };
+    for (bool changed = true; changed;) {
+        changed = false;
+        for (int f = 0; f < nf; ++f) {
+            const int k = kind(f, P.fn(f).root);
+            if (k != fvec[f]) { fvec[f] = k; changed = true; }
+        }
+    }
+    for (int f = 0; f < nf; ++f) {
+        const rdf_function& F = P.fn(f);
+        std::vector<char> seen(F.n_exprs, 0);
+        std::function<void(int)> walk = [&](int e) {
+            if (seen[e]) return;
+            seen[e] = 1;
+            const rdf_expr& x = F.exprs[e];
+            const int ops[3] = {x.a, x.b, x.c};
+            const int n = P.n_ops(x);
+            for (int k = 0; k < n; ++k) walk(ops[k]);
+            switch (x.op) {
+                case RDF_OP_IF:
+                    require(kind(f, x.a) == 0, RDF_ERR_UNSUPPORTED);                 // a Switch driven by a vector value
+                    require(kind(f, x.b) == kind(f, x.c), RDF_ERR_UNSUPPORTED);
+                    break;
+                case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
+                    for (int k = 0; k < 2; ++k)                                          // operands: states of two callees
+                        require(F.exprs[ops[k]].op == RDF_OP_CALL && kind(f, ops[k]) == 1, RDF_ERR_UNSUPPORTED);
+                    break;
+                case RDF_OP_NODE_LOSS:
+                    require(kind(f, x.a) == 1 && kind(f, x.b) == 0, RDF_ERR_UNSUPPORTED);
+                    break;
+                default:                                                                 // integer operands only
+                    for (int k = 0; k < n; ++k) require(kind(f, ops[k]) == 0, RDF_ERR_UNSUPPORTED);
+            }
+        };
+        walk(F.root);
+    }
+}
+
 // ------------------------------------------------- literal graph (Section 3)
-const int NODE_FCALL = 100;   // placeholder: "a node labeled with the name of f"
+const int NODE_FCALL = 100;   // placeholder: a function-call node of Section 2.4 (replaced by Call_i / Return_i)
 
 struct Literal {
     const Prog& P;
@@ -670,6 +727,7 @@ extern "C" int rdf_graph_build(const rdf_program* prog, rdf_graph** out_graph) {
     try {
         Prog P{prog};
         validate(P);
+        check_kinds(P);
         g->tag_mode = prog->tag_mode;
         for (int f = 0; f < prog->n_functions; ++f) g->func_names.push_back(prog->functions[f].name);
         build_literal(P, g);

@@ -108,7 +108,7 @@ __device__ __forceinline__ void mbar_init(uint32_t addr, uint32_t count) {
 // Bounded wait for the phase with the given parity.  Returns false on expiry.
 __device__ __forceinline__ bool mbar_wait(const DevCtx& c, uint32_t addr, uint32_t parity) {
     const long long t0 = clock64();
-    for (;;) {
+    for (uint32_t polls = 0;; ++polls) {
         uint32_t done;
         asm volatile(
             "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
@@ -118,6 +118,8 @@ __device__ __forceinline__ bool mbar_wait(const DevCtx& c, uint32_t addr, uint32
             set_status(c, RDF_ERR_TIMEOUT);
             return false;
         }
+        // a role that gave up elsewhere (any block) will not complete this phase: leave with it
+        if ((polls & 255u) == 255u && ld_volatile_i32(&c.ctl->status) != 0) return false;
     }
 }
 

@@ -165,6 +165,69 @@ def test_capacity_errors_are_status_codes():
     assert y.tolist() == [610] * 8
 
 
+def test_token_store_full_and_wave_limit_are_status_codes():
+    """Path tags park operands in a hash table sized from max_invocations (entries are never removed): a table
+    that is too small for the run reports RDF_ERR_STORE_FULL.  A wave limit below what the recursion needs
+    reports RDF_ERR_WAVE_LIMIT (the guard against recursion without a base case).  Neither faults, and the
+    graph runs a correct call afterwards."""
+    fs, r = rdf.fib_program()
+    x = torch.tensor([15] * 64, dtype=torch.int64, device="cuda")
+    g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(x, max_invocations=1000, max_wave_tokens=64 * 4096)     # 64 x 986 operands into 1024 slots
+    assert e.value.code == -5                     # RDF_ERR_STORE_FULL
+    y, _ = g.eval_int(x, max_invocations=64 * 1973)
+    assert y.tolist() == [610] * 64
+    for mode in (rdf.TAGS_PATH, rdf.TAGS_FRAME):
+        g = rdf.Graph(fs, r, mode)
+        g.set_limits(wave_limit=6)
+        with pytest.raises(rdf.RdfError) as e:
+            g.eval_int(x, max_invocations=64 * 1973)
+        assert e.value.code == -8                 # RDF_ERR_WAVE_LIMIT
+        g.set_limits(wave_limit=0)
+        y, _ = g.eval_int(x, max_invocations=64 * 1973)
+        assert y.tolist() == [610] * 64
+
+
+@pytest.mark.parametrize("mode", [rdf.TAGS_PATH, rdf.TAGS_FRAME])
+def test_expired_device_wait_is_a_status_code(mode):
+    """Every device-side wait is bounded.  With the bound set to a single clock cycle the first block to
+    reach a grid barrier gives up at once: the call ends with RDF_ERR_TIMEOUT as a status (every other
+    block sees the status word and leaves too), nothing hangs, and the same graph runs a normal call
+    afterwards.  Integer program: only the scheduler kernel runs."""
+    import time
+    fs, r = rdf.fib_program()
+    ns = [12] * 4096                               # waves far wider than one block: the grid barrier is in use
+    x = torch.tensor(ns, dtype=torch.int64, device="cuda")
+    n_inv = 4096 * 465
+    g = rdf.Graph(fs, r, mode)
+    g.set_limits(wait_cycles=1)
+    t0 = time.perf_counter()
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(x, max_invocations=n_inv)
+    assert e.value.code == -9                     # RDF_ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0         # gave up, did not sit out a long wait
+    g.set_limits(wait_cycles=0)
+    y, _ = g.eval_int(x, max_invocations=n_inv)
+    assert y.tolist() == [144] * 4096 and g.stats()["invocations"] == n_inv
+
+
+def test_capacity_error_returns_promptly():
+    """A block that is still waiting at a barrier when another block reports an error leaves as soon as it sees
+    the status word, not when its own wait limit runs out."""
+    import time
+    fs, r = rdf.fib_program()
+    x = torch.tensor([15] * 2048, dtype=torch.int64, device="cuda")
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    g.eval_int(torch.tensor([3], dtype=torch.int64, device="cuda"), max_invocations=16)      # (library start-up not timed)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(x, max_invocations=50000)
+    assert e.value.code == -6
+    assert time.perf_counter() - t0 < 0.5
+
+
 def test_bad_arguments():
     fs, r = rdf.fib_program()
     g = rdf.Graph(fs, r)

@@ -42,13 +42,42 @@ def check_forward(cfg, compute=rdf.F32, trees=None, cell="rnn"):
     return st
 
 
-def check_grad(cfg, compute=rdf.F32, workers=1, cell="rnn"):
+def check_embedding_rows(tb, dE, want, tol):
+    """The embedding gradient row by row (one maximum over the whole table would hide a wrong row): the rows of
+    tokens that no leaf carries are exactly zero, and every other row is within the tolerance of the larger of
+    its own largest entry and a floor of 5 % of the table's largest entry (a row whose contributions cancel
+    is small against the values that were rounded on the way to it)."""
+    dE = np.asarray(dE, dtype=np.float64)
+    touched = np.zeros(dE.shape[0], dtype=bool)
+    touched[tb.tok[tb.left < 0]] = True
+    assert not dE[~touched].any()
+    scale = np.maximum(np.abs(want[touched]).max(axis=1), 0.05 * np.abs(want).max())
+    row_err = np.abs(dE[touched] - want[touched]).max(axis=1) / scale
+    assert row_err.max() <= tol, float(row_err.max())
+    return float(row_err.max())
+
+
+_ORACLE_CACHE = {}
+
+
+def oracle_grad(name, cfg, cell, workers):
+    """loss, gradients and root states of the fp64 oracle for a named full-size workload (computed once)."""
+    if name not in _ORACLE_CACHE:
+        tb, p = cfg["trees"], cfg["params"]
+        _ORACLE_CACHE[name] = (direct.loss_and_grad_pool(tb, p, cell, workers=workers) if workers > 1
+                               else direct.loss_and_grad(tb, p, cell))
+    return _ORACLE_CACHE[name]
+
+
+def check_grad(cfg, compute=rdf.F32, workers=1, cell="rnn", name=None):
     tb, p = cfg["trees"], cfg["params"]
     g = graph(cell, with_loss=True)
     loss, h, grads = g.grad_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), compute)
     st = g.stats()
     assert st["status"] == 0 and st["invocations"] == tb.N
-    if workers > 1:
+    if name is not None:
+        want_loss, G, roots = oracle_grad(name, cfg, cell, workers)
+    elif workers > 1:
         want_loss, G, roots = direct.loss_and_grad_pool(tb, p, cell, workers=workers)
     else:
         want_loss, G, roots = direct.loss_and_grad(tb, p, cell)
@@ -57,6 +86,7 @@ def check_grad(cfg, compute=rdf.F32, workers=1, cell="rnn"):
     assert abs(loss.item() - want_loss) <= tol * abs(want_loss)
     errs = {k: relerr(grads[k].cpu().numpy(), G[k]) for k in G}
     assert all(e <= tol for e in errs.values()), errs
+    errs["E rows"] = check_embedding_rows(tb, grads["E"].cpu().numpy(), G["E"], tol)
     return st, errs
 
 
@@ -224,8 +254,51 @@ def test_treernn_config3_full_size():
     """8192 trees, H = 300, fwd + bwd at full size; the oracle runs over a pool of processes."""
     cfg = workloads.config(3)
     compute = rdf.BF16
-    st, errs = check_grad(cfg, compute, workers=WORKERS)
+    st, errs = check_grad(cfg, compute, workers=WORKERS, name="config3")
     print("config 3 errors:", errs, st)
+
+
+@pytest.mark.parametrize("k,cell", [(3, "rnn"), (4, "lstm")])
+def test_forward_only_full_size_bf16(k, cell):
+    """rdf_eval (forward only: no retained gates, no gradient buffers) on the 8192-tree workloads with bf16
+    operands: the root state of every tree against the fp64 oracle."""
+    cfg = workloads.config(k)
+    tb, p = cfg["trees"], cfg["params"]
+    g = graph(cell)
+    h, _ = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(p), rdf.BF16)
+    st = g.stats()
+    assert st["invocations"] == tb.N and st["cells"] == tb.n_cells and st["leaves"] == tb.N - tb.n_cells
+    _, _, roots = oracle_grad("config%d" % k, cfg, cell, WORKERS)
+    assert roots.shape == (tb.B, cfg["H"])
+    assert relerr(h.cpu().numpy(), roots) <= TOL[rdf.BF16]
+
+
+def test_bad_indices_in_the_batch_are_a_status_code():
+    """A token id outside the embedding table, or a child index outside the node arrays, is reported as
+    RDF_ERR_BAD_ARG by the device (the access is skipped, nothing faults), for rdf_eval and rdf_grad, fp32 and
+    bf16; the graph runs the intact batch afterwards."""
+    cfg = workloads.config(3, B=40, V=300, H=64)
+    tb, p = cfg["trees"], cfg["params"]
+    dp = rdf.Graph.device_params(p)
+    leaf = int(np.flatnonzero(tb.left < 0)[7])
+    cell = int(np.flatnonzero(tb.left >= 0)[5])
+    g = graph("rnn", with_loss=True)
+    ge = graph("rnn")
+    for compute in (rdf.F32, rdf.BF16):
+        for field, at, value in (("tok", leaf, 300), ("tok", leaf, -5), ("right", cell, tb.N + 3), ("left", cell, 2 ** 30),
+                                 ("tree_root", 3, tb.N)):
+            dt = rdf.Graph.device_trees(tb)
+            dt[field][at] = value
+            with pytest.raises(rdf.RdfError) as e:
+                g.grad_trees(dt, dp, compute)
+            assert e.value.code == -2
+            with pytest.raises(rdf.RdfError) as e:
+                ge.eval_trees(dt, dp, compute)
+            assert e.value.code == -2
+        loss, h, grads = g.grad_trees(rdf.Graph.device_trees(tb), dp, compute)
+        want_loss, G, roots = direct.loss_and_grad(tb, p, "rnn")
+        assert relerr(h.cpu().numpy(), roots) <= TOL[compute]
+        assert all(relerr(grads[k].cpu().numpy(), G[k]) <= TOL[compute] for k in G)
 
 
 def _lstm_cfg(B, V, H, seed=5):
@@ -280,21 +353,19 @@ def test_treelstm_bf16_tensor_core_path(H):
 
 
 def test_treelstm_config4_full_size():
-    """Binary TreeLSTM, 8192 trees, H = 300, fwd + bwd in the benchmark's launch configuration.
-    The fp64 oracle needs ~3 ms per node for this gradient, so at full size it checks what it can
-    compute piecewise: root states of sampled trees and the gradients of a 512-tree sub-batch;
-    the full-size gradients are then checked through additivity over the two halves of the batch
-    (the gradient of a sum of per-tree losses is the sum of the per-half gradients)."""
+    """Binary TreeLSTM, 8192 trees, H = 300, fwd + bwd in the benchmark's launch configuration: loss, the root
+    state of every tree and all seven gradients of the full batch against the fp64 oracle (run over a pool of
+    processes), element by element.  As an extra, additivity: the gradient of a sum of per-tree losses is the
+    sum of the gradients of the two halves of the batch."""
     cfg = workloads.config(4)
     tb, p = cfg["trees"], cfg["params"]
-    compute, tol = rdf.BF16, TOL[rdf.BF16]
+    compute = rdf.BF16
+    st, errs = check_grad(cfg, compute, workers=WORKERS, cell="lstm", name="config4")
+    print("config 4 errors:", errs)
+    assert st["cells"] == tb.n_cells
     g = graph("lstm", with_loss=True)
     dp = rdf.Graph.device_params(p)
     loss, h, grads = g.grad_trees(rdf.Graph.device_trees(tb), dp, compute)
-    st = g.stats()
-    assert st["invocations"] == tb.N and st["cells"] == tb.n_cells
-    sample = list(range(0, tb.B, 257))
-    assert relerr(h.cpu().numpy()[sample], direct.forward(tb, p, "lstm", trees=sample)) <= tol
     full = {k: v.cpu().numpy().astype(np.float64) for k, v in grads.items()}
     halves, loss_sum = None, 0.0
     for part in (range(0, tb.B // 2), range(tb.B // 2, tb.B)):
@@ -305,9 +376,6 @@ def test_treelstm_config4_full_size():
         halves = cur if halves is None else {k: halves[k] + cur[k] for k in cur}
     assert abs(loss.item() - loss_sum) <= 1e-4 * abs(loss_sum)
     assert all(relerr(full[k], halves[k]) <= 1e-4 for k in full)
-    # oracle parity of every gradient on a sub-batch of the same workload
-    sub = workloads.subset_trees(tb, list(range(512)))
-    check_grad({"trees": sub, "params": p}, compute, workers=WORKERS, cell="lstm")
 
 
 def test_depth_stress_config5_forward_sampled():

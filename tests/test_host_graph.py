@@ -79,6 +79,44 @@ def test_bad_programs_are_rejected():
         _build([a2, b], 0, rdf.TAGS_FRAME)
 
 
+def test_vector_programs_outside_the_executor_are_rejected():
+    """An invocation owns one state slot, so its body may fire one vector operator, a cell reads the states
+    of two callees, and integer operators, conditions and call arguments take integers.  Programs outside
+    that are valid but not lowered: RDF_ERR_UNSUPPORTED at build time, not wrong states at run time."""
+    def prog(body):
+        r = rdf.Function("result", 1)
+        r.ret(r.call(1, r.param()))
+        f = rdf.Function("h", 1)
+        v = f.param()
+        f.ret(body(f, v))
+        return [r, f]
+
+    bad = [
+        # a cell whose operand is another cell of the same invocation
+        lambda f, v: f.if_(f.is_leaf(v), f.embed(f.tok(v)),
+                           f.cell_rnn(f.cell_rnn(f.call(1, f.left(v)), f.call(1, f.right(v))), f.call(1, f.left(v)))),
+        # a cell that reads an embedding computed in the same invocation
+        lambda f, v: f.if_(f.is_leaf(v), f.embed(f.tok(v)), f.cell_rnn(f.embed(f.tok(v)), f.call(1, f.left(v)))),
+        # an integer operator applied to a vector value
+        lambda f, v: f.if_(f.is_leaf(v), f.embed(f.tok(v)), f.add(f.call(1, f.left(v)), f.const(1))),
+        # a condition that is a vector value
+        lambda f, v: f.if_(f.call(1, f.left(v)), f.embed(f.tok(v)), f.embed(f.tok(v))),
+        # a vector value as a call argument
+        lambda f, v: f.if_(f.is_leaf(v), f.embed(f.tok(v)), f.call(1, f.embed(f.tok(v)))),
+        # the two sides of a conditional of different kinds
+        lambda f, v: f.if_(f.is_leaf(v), f.embed(f.tok(v)), f.tok(v)),
+    ]
+    for body in bad:
+        with pytest.raises(rdf.RdfError) as e:
+            _build(prog(body), 0, rdf.TAGS_FRAME)
+        assert e.value.code == -11
+    # the supported shapes still build
+    for cell in ("rnn", "lstm"):
+        for with_loss in (False, True):
+            fs, r = rdf.tree_net_program(cell, with_loss)
+            _build(fs, r, rdf.TAGS_FRAME)
+
+
 # ---------------------------------------- literal graph through the oracle
 OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.OP_REM: "%", bd.OP_LT: "<", bd.OP_EQ: "==",
           bd.OP_IS_LEAF: "is_leaf", bd.OP_LEFT: "left", bd.OP_RIGHT: "right", bd.OP_TOK: "tok",

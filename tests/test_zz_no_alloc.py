@@ -4,9 +4,10 @@ fully handed out, a latency-critical path).  The entry point takes its scratch
 from a 16 MiB array built into the library instead of a caller workspace.
 
 Checked here, through the C boundary: its results equal those of rdf_eval
-exactly (integer results: bit for bit) on two calls in a row with different
-inputs -- the second call must not see anything the first one left in the shared
-array -- and a batch that needs more than the built-in array is refused.
+exactly (integer results: bit for bit) and those of the CPU oracle, on two calls
+in a row with different inputs -- the second call must not see anything the first
+one left in the shared array -- for an integer program and for a small TreeRNN,
+and a batch that needs more than the built-in array is refused.
 Collected last on purpose (file name), and self-contained so that it also passes
 when run alone in a fresh process."""
 import numpy as np
@@ -14,6 +15,7 @@ import pytest
 
 import workloads
 import paper_2410_20225_b200 as rdf
+from oracle import direct
 from paper_2410_20225_b200 import binding as bd
 
 torch = pytest.importorskip("torch")
@@ -42,7 +44,30 @@ def test_noalloc_matches_rdf_eval_twice_in_a_row(mode):
         g.eval_int_noalloc(x, y, max_invocations=n_inv)
         assert torch.cuda.memory_allocated() == before   # nothing was taken from torch's allocator either
         assert torch.equal(y, want)
+        assert y.tolist() == [direct.fib(int(n)) for n in x_host]        # and the recursive definition itself
         assert g.stats()["invocations"] == n_inv
+
+
+def test_noalloc_tree_network_twice_in_a_row():
+    """A small TreeRNN forward pass out of the built-in scratch: equal to rdf_eval bit for bit (the same kernels
+    on the same inputs) and within the fp32 tolerance of the oracle, on two different batches in a row."""
+    fs, r = rdf.tree_net_program("rnn")
+    g_ref = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    for seed in (21, 22):
+        cfg = workloads.config(3, seed=seed, B=32, V=200, H=32)
+        tb = cfg["trees"]
+        p = workloads.treernn_params(seed, 200, 32, 32)
+        dt, dp = rdf.Graph.device_trees(tb), rdf.Graph.device_params(p)
+        want, _ = g_ref.eval_trees(dt, dp)
+        h = torch.full((tb.B, 32), float("nan"), dtype=torch.float32, device="cuda")
+        before = torch.cuda.memory_allocated()
+        g.eval_trees_noalloc(dt, dp, h)
+        assert torch.cuda.memory_allocated() == before
+        assert torch.equal(h, want)
+        roots = direct.forward(tb, p, "rnn")
+        assert float(np.abs(h.cpu().numpy() - roots).max() / np.abs(roots).max()) <= 1e-4
+        assert g.stats()["invocations"] == tb.N
 
 
 def test_noalloc_refuses_batches_beyond_the_builtin_scratch():
