@@ -6,11 +6,18 @@
 A step is one pass of the whole hot path over one batch of synthetic input:
 lowered graph -> seed tokens -> all forward waves (tag push/pop, matching, batched
 cells) -> loss head -> gradient waves -> parameter gradients (workloads 3-5), or
-the forward pass alone (workloads 1-2).  Prints one JSON line.
+the forward pass alone (workloads 1-2).  Prints one JSON line: the headline workload
+(default 3) with its roofline, and -- on one GPU -- a table of all five workloads
+(forward and forward+backward), a table of every kernel of the headline step with
+its algorithmic work against the measured peak, and the CPU oracle's rate.
+
+With --gpus N > 1 and no RANK in the environment the script starts the N ranks
+itself (one process per GPU, NCCL); under torchrun it joins the ranks it is given.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -34,12 +41,9 @@ WORKLOAD_NAMES = {
     4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
-# kernels of the library launched per step (memsets and copies not counted):
-#   seed, scheduler | + 3 kernels that group the cells by height, operators, root gather | + loss head, loss sum, 4 list kernels, gradient waves, dW, db
-#   bf16: + weight packing (TreeLSTM: + table packing); TreeLSTM: + dW_x, db_x, dE
-KERNELS_PER_STEP = {"eval_int": 2, "eval_trees": 7, "eval_trees_tc": 8, "grad": 16, "grad_tc": 17, "grad_lstm": 19,
-                    "grad_lstm_tc": 21}
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
+KERNEL_SOURCES = ["rdf_device.cuh", "rdf_exec.cu", "rdf_exec.h", "rdf_grad.cu", "rdf_internal.h", "rdf_lstm.cuh", "rdf_tc.cuh",
+                  "rdf_tc_dw.cuh"]
 
 
 def fib_iter(n):
@@ -111,17 +115,52 @@ def peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the same kernel
-# (profiles/persistent_kernels_config3.md); None where no capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {("rdf_backward_kernel", 3, None): 396.0e6, ("rdf_operator_kernel", 3, None): 297.0e6,
-                     ("rdf_scheduler_kernel", 3, None): 10.8e6}
+def kernel_source_hash():
+    """Fingerprint of the CUDA sources: DRAM traffic taken from a profiler capture is reported only while the
+    kernels are the ones that were captured."""
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2410_20225_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
-# fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
-FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+def dram_traffic_table():
+    """{(kernel, workload): bytes per launch} from the tracked table of profiler captures; only the rows whose
+    source fingerprint is the current one count (a changed kernel has no traffic figure until it is captured again)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    table, cur = {}, kernel_source_hash()
+    if not os.path.exists(path):
+        return table
+    for line in open(path):
+        line = line.split("#")[0].split()
+        if len(line) >= 4 and line[3] == cur:
+            table[(line[0], int(line[1]))] = float(line[2])
+    return table
+
+
+# nominal fp32 FMA peak (148 SMs x 128 lanes x 2 flop x 1.965 GHz); the run measures the achieved rate itself
+FP32_ALU_NOMINAL_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def oracle_step(cfg, sample):
+def cpu_info():
+    model = "unknown"
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                model = line.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except AttributeError:
+        usable = os.cpu_count() or 1
+    return model, usable
+
+
+def oracle_step(cfg, sample, grad=None):
     """One bounded sample of the workload on the CPU oracle; returns invocations processed."""
     from oracle import direct
     if cfg["kind"] == "fib":
@@ -132,7 +171,7 @@ def oracle_step(cfg, sample):
         return n
     tb = cfg["trees"]
     trees = list(range(min(sample, tb.B)))
-    if cfg["grad"]:
+    if cfg["grad"] if grad is None else grad:
         direct.loss_and_grad(tb, cfg["params"], CELL[cfg["kind"]], trees=trees)
     else:
         direct.forward(tb, cfg["params"], CELL[cfg["kind"]], trees=trees)
@@ -176,6 +215,31 @@ def time_oracle(cfg, steps, warmup, scale=1, budget_s=None):
     return n / dt, dt / steps, what
 
 
+def time_oracle_all_cores(cfg, cores, budget_s=20.0):
+    """The oracle over a pool of processes (trees are independent), one per usable core, on a sample sized from the
+    one-thread rate for about budget_s of wall time; the wall time includes the start of the worker processes."""
+    if cfg["kind"] == "fib" or not cfg["grad"] or cores < 2:
+        return None
+    from oracle import direct
+    tb = cfg["trees"]
+    workers = max(1, cores)
+    t0 = time.perf_counter()
+    probe = list(range(min(8, tb.B)))
+    direct.loss_and_grad(tb, cfg["params"], CELL[cfg["kind"]], trees=probe)
+    per_node = (time.perf_counter() - t0) / max(1, int(tb.tree_sizes()[probe].sum()))
+    want_nodes = budget_s * workers / per_node
+    sizes = np.cumsum(tb.tree_sizes())
+    n_trees = int(min(tb.B, max(workers, np.searchsorted(sizes, want_nodes) + 1)))
+    trees = list(range(n_trees))
+    t0 = time.perf_counter()
+    direct.loss_and_grad_pool(tb, cfg["params"], CELL[cfg["kind"]], workers=workers, trees=trees)
+    dt = time.perf_counter() - t0
+    n = int(tb.tree_sizes()[trees].sum())
+    return {"value": n / dt, "unit": UNIT, "cores": workers, "kind": "oracle",
+            "sample": f"first {n_trees} trees of the workload, one pass, fp64 Python+numpy oracle over {workers} spawned processes "
+                      f"(wall time {dt:.1f} s including their start-up)"}
+
+
 # --------------------------------------------------------------------------- multi-rank host logic
 def rank_seed(seed, rank):
     """Every rank draws a batch of its own: instances never exchange tokens (weak scaling)."""
@@ -194,14 +258,368 @@ def reduce_job(dist, device, elapsed, units):
     return float(t.item()), float(n.item())
 
 
+def flat_gradients(shapes, device):
+    """One buffer for all parameter gradients; returns (flat, {name: view}).  Views start on 256-byte boundaries."""
+    import torch
+    offs, total = {}, 0
+    for k, shp in shapes.items():
+        offs[k] = total
+        total += (int(np.prod(shp)) + 63) // 64 * 64
+    flat = torch.zeros(total, dtype=torch.float32, device=device)
+    views = {k: flat[offs[k]: offs[k] + int(np.prod(shp))].view(*shp) for k, shp in shapes.items()}
+    return flat, views
+
+
 def sum_gradients(dist, grads):
-    """The one exchange step of data-parallel rdf_grad: parameter gradients are summed over ranks."""
-    if dist is not None:
-        for t in grads.values():
-            dist.all_reduce(t)
+    """The one exchange step of data-parallel rdf_grad: parameter gradients are summed over ranks -- one
+    all-reduce when the gradients are views of one flat buffer (pass that buffer), else one per tensor."""
+    if dist is None:
+        return
+    import torch
+    if isinstance(grads, torch.Tensor):
+        dist.all_reduce(grads)
+        return
+    for t in grads.values():
+        dist.all_reduce(t)
+
+
+def _free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_entry(rank, world, port, target, payload):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    target(payload)
+
+
+def spawn_ranks(world, target, payload):
+    """Starts `world` processes on this node (rank r = local rank r) that each run target(payload) with the
+    rendezvous variables set; raises if one of them fails."""
+    import torch.multiprocessing as mp
+    mp.spawn(_rank_entry, args=(world, _free_port(), target, payload), nprocs=world, join=True)
+
+
+# --------------------------------------------------------------------------- one workload on the device
+class Case:
+    """One workload set up on the current device: resident inputs, host copies for the end-to-end path, step functions."""
+
+    def __init__(self, rdf, torch, cfg, grad, dist=None):
+        self.rdf, self.torch, self.cfg, self.dist = rdf, torch, cfg, dist
+        self.N = cfg["N"]
+        self.grad = bool(grad)
+        if cfg["kind"] == "fib":
+            fs, r = rdf.fib_program()
+            self.g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+            self.x_host = torch.from_numpy(cfg["x"]).pin_memory()
+            self.x_dev = self.x_host.cuda()
+            self.y = torch.empty_like(self.x_dev)
+            self.y_host = torch.empty_like(self.x_host).pin_memory()
+            self.dtype, self.use_tc, self.cell = "int64", False, None
+            # the widest wave of fib(18) holds 2048 calls + their continuations per instance: 4096 tokens bound it
+            self.wave_cap = min(self.N + len(cfg["x"]), 4096 * len(cfg["x"]))
+            self.h2d, self.d2h = self.x_host.numel() * 8, self.x_host.numel() * 8
+            self.d2h_full = self.d2h
+            return
+        tb, p = cfg["trees"], cfg["params"]
+        self.tb = tb
+        self.cell = CELL[cfg["kind"]]
+        fs, r = rdf.tree_net_program(self.cell, with_loss=self.grad)
+        self.g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+        self.compute = rdf.BF16 if cfg["bf16"] else rdf.F32
+        # arithmetic type of the contractions: bf16 operands on the tensor cores (fp32 accumulate) for the
+        # bf16 workloads, fp32 FMA otherwise
+        self.use_tc = bool(cfg["bf16"])
+        self.dtype = "bf16" if self.use_tc else "f32"
+        self.host = {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).pin_memory()
+                     for k in ("tree_root", "left", "right", "tok", "label")}
+        self.dt = {k: v.cuda() for k, v in self.host.items()}
+        self.dp = rdf.Graph.device_params(p)
+        self.H = cfg["H"]
+        self.h_root = torch.empty(tb.B, self.H, dtype=torch.float32, device="cuda")
+        self.h_root_host = torch.empty(tb.B, self.H, dtype=torch.float32).pin_memory()
+        self.h2d = sum(v.numel() * 4 for v in self.host.values())
+        if self.grad:
+            self.flat, self.grads = flat_gradients({k: tuple(v.shape) for k, v in self.dp.items()}, "cuda")
+            self.flat_host = torch.empty_like(self.flat, device="cpu").pin_memory()
+            self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+            self.d2h = 4
+            self.d2h_full = 4 + self.flat.numel() * 4 + tb.B * self.H * 4
+        else:
+            self.d2h = self.d2h_full = tb.B * self.H * 4
+
+    # the timed step: inputs and parameters resident
+    def step(self):
+        if self.cfg["kind"] == "fib":
+            self.g.eval_int(self.x_dev, self.N, check=False, y=self.y, max_wave_tokens=self.wave_cap)
+        elif self.grad:
+            self.g.grad_trees(self.dt, self.dp, self.compute, check=False, grads=self.grads, loss=self.loss, h_root=self.h_root)
+            sum_gradients(self.dist, self.flat)      # data-parallel exchange: one sum of the parameter gradients
+        else:
+            self.g.eval_trees(self.dt, self.dp, self.compute, check=False, h_root=self.h_root)
+
+    # end to end: host buffers in, result out; full = every output of the call comes back
+    def step_e2e(self, full=False):
+        if self.cfg["kind"] == "fib":
+            xd = self.x_host.cuda(non_blocking=True)
+            self.g.eval_int(xd, self.N, check=False, y=self.y, max_wave_tokens=self.wave_cap)
+            self.y_host.copy_(self.y, non_blocking=True)
+            self.torch.cuda.current_stream().synchronize()
+            return self.y_host
+        d = {k: v.cuda(non_blocking=True) for k, v in self.host.items()}
+        if self.grad:
+            self.g.grad_trees(d, self.dp, self.compute, check=False, grads=self.grads, loss=self.loss, h_root=self.h_root)
+            sum_gradients(self.dist, self.flat)
+            if full:
+                self.flat_host.copy_(self.flat, non_blocking=True)
+                self.h_root_host.copy_(self.h_root, non_blocking=True)
+            return self.loss.item()
+        self.g.eval_trees(d, self.dp, self.compute, check=False, h_root=self.h_root)
+        self.h_root_host.copy_(self.h_root, non_blocking=True)
+        self.torch.cuda.current_stream().synchronize()
+        return self.h_root_host
+
+    def flops_fwd(self):
+        if self.cfg["kind"] == "fib":
+            return 0.0
+        H, tb = self.H, self.tb
+        if self.cell == "lstm":
+            return tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
+        return tb.n_cells * 2.0 * (2 * H) * H
+
+
+def time_case(case, steps, warmup, flush, dist=None, e2e_steps=None, full_e2e=False):
+    """W warm-up steps, K device-timed steps (one CUDA event pair per step on the launching stream, L2 flushed
+    between steps), then the end-to-end loop.  Returns whole-job figures (max over ranks / sum of units)."""
+    torch = case.torch
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    case.g.set_profiling(True)
+    for _ in range(warmup):
+        case.step()
+    case.g.stats()                                   # also checks the device status word
+    barrier()
+    times, phases = [], {}
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        case.step()
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+        for k, v in case.g.phase_ms().items():
+            phases.setdefault(k, []).append(v)
+    barrier()
+    st = case.g.stats()
+    total_ms, N_all = reduce_job(dist, "cuda", sum(times), case.N)
+    out = {"ms_per_step": total_ms / steps, "value": N_all * steps / (total_ms * 1e-3), "N_all": N_all,
+           "phase_ms": {k: sum(v) / len(v) for k, v in phases.items()}, "stats": st, "min_ms": min(times)}
+    # ---- end to end through the public call, host buffers, copies inside the timed region
+    ke = e2e_steps or steps
+    variants = [("e2e", False)] + ([("e2e_all_outputs", True)] if full_e2e and case.grad else [])
+    for name, full in variants:
+        for _ in range(2):
+            case.step_e2e(full)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(ke):
+            case.step_e2e(full)
+        barrier()
+        e2e_s, _ = reduce_job(dist, "cuda", time.perf_counter() - t0, case.N)
+        out[name] = {"value": N_all * ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": case.h2d,
+                     "d2h_bytes_per_step": case.d2h_full if full else case.d2h}
+        if full:
+            out[name]["what_comes_back"] = "loss, every parameter gradient and the root states, to pinned host buffers"
+    return out
+
+
+# --------------------------------------------------------------------------- kernels against their rooflines
+def kernel_table(case, phase_ms, pk, fp32_peak, traffic, workload):
+    """One row per kernel (group) of the step: CUDA-event time of its phase, algorithmic bytes or flops, the
+    measured peak that bounds it and the fraction reached.  Tensor peak: the burst figure for a kernel of under a
+    millisecond (it runs alone between two events on an otherwise idle device), the sustained one above that."""
+    N = case.N
+    rows = []
+
+    def add(kernel, phase, bound, work, what):
+        ms = phase_ms.get(phase)
+        if ms is None or ms <= 0:
+            return
+        if bound == "hbm":
+            peak, unit, ach, src = pk["hbm_gbs"], "GB/s", work / (ms * 1e-3) / 1e9, pk["source"] + " copy bandwidth"
+        elif bound == "tensor":
+            burst = ms < 1.0
+            peak = pk["bf16_tflops"] if burst else pk["bf16_tflops_sustained"]
+            unit, ach = "TFLOP/s", work / (ms * 1e-3) / 1e12
+            src = pk["source"] + (" bf16 dense, burst" if burst else " bf16 dense, sustained")
+        else:
+            peak, unit, ach, src = fp32_peak, "TFLOP/s", work / (ms * 1e-3) / 1e12, "fp32 FMA loop measured in this run"
+        rows.append({"kernel": kernel, "phase": phase, "ms": ms, "bound": bound, "algorithmic": work, "work_is": what,
+                     "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak if peak else None, "peak_source": src,
+                     "traffic": traffic.get((kernel, workload))})
+
+    add("rdf_scheduler_kernel", "schedule", "hbm", 128.0 * N,
+        "128 B per invocation: call token write+read, return token / store slot write+read, frame record")
+    if case.cfg["kind"] == "fib":
+        return rows
+    tb, H = case.tb, case.H
+    C, Lf = tb.n_cells, tb.N - tb.n_cells
+    Hp = 64 * ((H + 63) // 64)
+    lstm = case.cell == "lstm"
+    mm = "tensor" if case.use_tc else "alu"
+    add("rdf_height_count/scan/scatter_kernel", "group", "hbm", 48.0 * C, "16 B cell record read twice and written once")
+    add("rdf_operator_kernel", "operators", mm, case.flops_fwd(),
+        "cell contraction 2*2H*H per cell" + (" (x5 gates) + leaf projection 2*D*3H per leaf" if lstm else ""))
+    add("rdf_gather_roots_kernel", "roots", "hbm", tb.B * H * (4.0 + (2 if case.use_tc and not lstm else 4)), "root rows read and written")
+    if case.grad:
+        rowbytes = Hp * 2 if case.use_tc else H * 4 * (2 if lstm else 1)
+        add("rdf_loss_heads_kernel", "loss", "hbm", float(N) * (rowbytes + 32), "one state row read + 32 B of dlog written per invocation")
+        add("rdf_list_count/scan/fill/ends_kernel", "lists", "hbm", N * 28.0 + C * 24.0,
+            "operand ids and frame records read (two passes), cell lists written")
+        bwd = C * 2.0 * H * (2 * H) * (5 if lstm else 1)
+        add("rdf_backward_kernel", "backward", mm, bwd, "operand-gradient contraction W^T dz: 2*H*2H per cell" + (" (x5 gates)" if lstm else ""))
+        dw = bwd + (Lf * 2.0 * H * 3 * H if lstm else 0.0)
+        add("rdf_dw_tc_kernel" if case.use_tc else "rdf_outer_kernel", "dW", mm, dw,
+            "weight-gradient contraction dz (x) [h_l;h_r]: 2*H*2H per cell" + (" (x5 gates) + leaf 2*3H*D" if lstm else ""))
+        if not (case.use_tc and H % 64):       # (bf16 with padded rows: db is a column of the dW contraction, no kernel of its own)
+            add("rdf_colsum_kernel", "db", "hbm", C * (5 if lstm else 1) * H * (2.0 if case.use_tc else 4.0), "one gradient row read per cell")
+        if lstm:
+            add("rdf_de_tc_kernel" if case.use_tc else "rdf_de_lstm_kernel", "dE", mm, Lf * 2.0 * H * 3 * H, "W_x^T dg: 2*3H*D per leaf")
+    return rows
 
 
 # --------------------------------------------------------------------------- main
+def run(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import torch
+    import paper_2410_20225_b200 as rdf
+    from paper_2410_20225_b200.binding import probe_fp32_fma_tflops
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the recursive-dataflow path has no CPU route")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} wants GPU {local} but this node has {torch.cuda.device_count()}")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank processes a batch of its own (instances never exchange tokens): weak scaling
+    cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
+    case = Case(rdf, torch, cfg, cfg.get("grad", False), dist)
+
+    clocks = ClockSampler(local)
+    clocks.start()                                   # samples from the warm-up on: short runs still get samples under load
+    head = time_case(case, args.steps, args.warmup, flush, dist, full_e2e=True)
+    clk = clocks.stop()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    fp32_peak = probe_fp32_fma_tflops()
+    traffic = dram_traffic_table()
+    kernels = kernel_table(case, head["phase_ms"], pk, fp32_peak, traffic, args.workload)
+    # ---- roofline of the dominant kernel (the phase with the largest share of the step)
+    dom = max(kernels, key=lambda r: r["ms"])
+    roof = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
+            "frac": dom["frac"], "traffic": dom["traffic"], "peak_source": dom["peak_source"], "phase": dom["phase"],
+            "phase_ms": dom["ms"], "algorithmic": dom["algorithmic"], "work_is": dom["work_is"],
+            "note": "a persistent kernel: every wave ends at a grid barrier; block0_ms_at_max_clock gives the split"}
+    st = head["stats"]
+
+    # ---- the other workloads, forward and forward+backward (one GPU only: the table is not part of the scaling run)
+    table = None
+    if world == 1 and not args.no_table:
+        table = []
+        for k in sorted(WORKLOAD_NAMES):
+            c_k = cfg if k == args.workload and not args.fib_batch else load(k, args.seed)
+            passes = [False, True] if c_k.get("grad") else [False]
+            for grad in passes:
+                if k == args.workload and grad == bool(cfg.get("grad", False)) and not args.fib_batch:
+                    res, cs = head, case
+                else:
+                    cs = Case(rdf, torch, c_k, grad)
+                    n = 5 if c_k["N"] > 2_000_000 else min(args.steps, 20)
+                    res = time_case(cs, n, 3, flush, e2e_steps=min(n, 5))
+                kt = kernel_table(cs, res["phase_ms"], pk, fp32_peak, traffic, k)
+                top = max(kt, key=lambda r: r["ms"])
+                table.append({"workload": k, "pass": "forward+backward" if grad else "forward", "dtype": cs.dtype,
+                              "invocations_per_step": c_k["N"], "ms_per_step": res["ms_per_step"], "value": res["value"],
+                              "e2e": res["e2e"]["value"], "unit": UNIT, "waves": res["stats"]["waves"],
+                              "waves_backward": res["stats"]["waves_backward"],
+                              "kernels": [{"kernel": r["kernel"], "ms": round(r["ms"], 4), "bound": r["bound"],
+                                           "achieved": r["achieved"], "unit": r["unit"], "frac": r["frac"]} for r in kt],
+                              "dominant": {"kernel": top["kernel"], "bound": top["bound"], "frac": top["frac"]}})
+                del cs
+                torch.cuda.empty_cache()
+
+    cpu, cpu_all = None, None
+    if not args.no_cpu_baseline:
+        model, usable = cpu_info()
+        v, _, what = time_oracle(cfg, 1, 0, scale=1 if cfg["kind"] != "fib" and cfg["trees"].N > 2_000_000 else 4)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what, "cpu_model": model, "usable_cores": usable}
+        cpu_all = time_oracle_all_cores(cfg, usable)
+        if cpu_all is not None:
+            cpu["all_cores"] = cpu_all
+
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": case.dtype, "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else ""),
+                   "invocations_per_step": case.N, "instances": cfg.get("B") or cfg["trees"].B,
+                   "pass": "forward+backward" if cfg.get("grad") else "forward",
+                   "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
+        "clocks": clk,
+        "e2e": head["e2e"],
+        "e2e_all_outputs": head.get("e2e_all_outputs"),
+        "gpu_launches": st["kernel_launches"] * args.steps,          # counted by the library at every launch of the call
+        "roofline": roof,
+        "kernels": kernels,
+        "workloads": table,
+        "cpu_baseline": cpu,
+        "phase_ms": head["phase_ms"],
+        "min_ms_per_step": head["min_ms"],
+        "fp32_fma_tflops": {"measured": fp32_peak, "nominal": FP32_ALU_NOMINAL_TFLOPS},
+        "waves": {"forward": st["waves"], "backward": st["waves_backward"], "widest": st["max_wave_tokens"]},
+        "block0_ms_at_max_clock": {k[7:]: round(st[k] / 1.965e6, 4) for k in st if k.startswith("cycles_")},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def reference(args):
+    cfg = load(args.workload, args.seed, args.fib_batch)
+    value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup), budget_s=90.0)
+    model, usable = cpu_info()
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * s_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.workload]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what, "cpu_model": model,
+                         "usable_cores": usable},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -211,231 +629,28 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=workloads.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="skip the table of the other workloads")
     ap.add_argument("--fib-batch", type=int, default=None,
                     help="workload 1 only: number of independent fib calls (default 1024, the named configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-
     if args.impl == "reference":
-        if rank != 0:
-            return
-        cfg = load(args.workload, args.seed, args.fib_batch)
-        value, s_per_step, what = time_oracle(cfg, max(1, args.steps), max(0, args.warmup), budget_s=90.0)
-        print(json.dumps({
-            "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * s_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD_NAMES[args.workload]},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        }))
+        if int(os.environ.get("RANK", "0")) == 0:
+            reference(args)
         return
-
-    import torch
-    import paper_2410_20225_b200 as rdf
-
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the recursive-dataflow path has no CPU route")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    # every rank processes a batch of its own (instances never exchange tokens): weak scaling
-    cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch)
-    N = cfg["N"]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
-
-    if cfg["kind"] == "fib":
-        fs, r = rdf.fib_program()
-        g = rdf.Graph(fs, r, rdf.TAGS_PATH)
-        x_host = torch.from_numpy(cfg["x"]).pin_memory()
-        x_dev = x_host.cuda()
-        y = torch.empty_like(x_dev)
-        kind, compute, dtype = "eval_int", None, "int64"
-
-        # the widest wave of fib(18) holds 2048 calls + their continuations per instance: 4096 tokens bound it
-        wave_cap = min(N + len(cfg["x"]), 4096 * len(cfg["x"]))
-
-        def step():
-            g.eval_int(x_dev, N, check=False, y=y, max_wave_tokens=wave_cap)
-
-        def step_e2e():
-            xd = x_host.cuda(non_blocking=True)
-            out, _ = g.eval_int(xd, N, check=False, max_wave_tokens=wave_cap)
-            return out.cpu()
-        h2d, d2h = x_host.numel() * 8, x_host.numel() * 8
-        flops_fwd = 0.0
-    else:
-        tb, p = cfg["trees"], cfg["params"]
-        cell = CELL[cfg["kind"]]
-        fs, r = rdf.tree_net_program(cell, with_loss=cfg["grad"])
-        g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
-        compute = rdf.BF16 if cfg["bf16"] else rdf.F32
-        # arithmetic type of the contractions: bf16 operands on the tensor cores (fp32 accumulate) for the
-        # bf16 workloads, fp32 FMA otherwise
-        use_tc = bool(cfg["bf16"])
-        dtype = "bf16" if use_tc else "f32"
-        host = {k: torch.from_numpy(np.ascontiguousarray(getattr(tb, k), dtype=np.int32)).pin_memory()
-                for k in ("tree_root", "left", "right", "tok", "label")}
-        dt = {k: v.cuda() for k, v in host.items()}
-        dp = rdf.Graph.device_params(p)
-        H = cfg["H"]
-        h_root = torch.empty(tb.B, H, dtype=torch.float32, device="cuda")
-        flops_fwd = tb.n_cells * 2.0 * (2 * H) * H
-        if cell == "lstm":
-            flops_fwd = tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
-        if cfg["grad"]:
-            kind = ("grad_lstm_tc" if use_tc else "grad_lstm") if cell == "lstm" else ("grad_tc" if use_tc else "grad")
-            grads = {k: torch.empty_like(v) for k, v in dp.items()}
-            loss = torch.zeros(1, dtype=torch.float32, device="cuda")
-
-            def step():
-                g.grad_trees(dt, dp, compute, check=False, grads=grads, loss=loss, h_root=h_root)
-                sum_gradients(dist, grads)      # data-parallel exchange: one sum of the parameter gradients
-
-            def step_e2e():
-                d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
-                l, _, _ = g.grad_trees(d, dp, compute, check=False, grads=grads, h_root=h_root)
-                sum_gradients(dist, grads)
-                return l.item()
-            h2d, d2h = sum(v.numel() * 4 for v in host.values()), 4
-        else:
-            kind = "eval_trees_tc" if use_tc else "eval_trees"
-
-            def step():
-                g.eval_trees(dt, dp, compute, check=False, h_root=h_root)
-
-            def step_e2e():
-                d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
-                out, _ = g.eval_trees(d, dp, compute, check=False)
-                return out.cpu()
-            h2d, d2h = sum(v.numel() * 4 for v in host.values()), tb.B * H * 4
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    g.set_profiling(True)
-    clocks = ClockSampler(local)
-    clocks.start()                                   # samples from the warm-up on: short runs still get samples under load
-    for _ in range(args.warmup):
-        step()
-    st = g.stats()                                   # also checks the device status word
-
-    # ---- device-timed region: K steps, L2 flushed between steps, one event pair per step
-    barrier()
-    times, phases = [], {}
-    for _ in range(args.steps):
-        flush.fill_(1)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        step()
-        e1.record()
-        e1.synchronize()
-        times.append(e0.elapsed_time(e1))
-        for k, v in g.phase_ms().items():
-            phases.setdefault(k, []).append(v)
-    barrier()
-    clk = clocks.stop()
-    st = g.stats()
-    total_ms, N_all = reduce_job(dist, "cuda", sum(times), N)
-    value = N_all * args.steps / (total_ms * 1e-3)
-
-    # ---- end to end through the public call, host buffers, copies inside the timed region
-    for _ in range(2):
-        step_e2e()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        step_e2e()
-    barrier()
-    e2e_s = time.perf_counter() - t0
-    e2e_s, _ = reduce_job(dist, "cuda", e2e_s, N)
-    e2e_value = N_all * args.steps / e2e_s
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+    in_ranks = "RANK" in os.environ and "WORLD_SIZE" in os.environ
+    if args.gpus > 1 and not in_ranks:
+        # no launcher gave us ranks: start them here, one process per GPU
+        import torch
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            raise SystemExit(f"bench.py --gpus {args.gpus}: this node has {have} CUDA device(s); refusing to report fewer GPUs than asked")
+        spawn_ranks(args.gpus, run, args)
         return
-
-    # ---- roofline of the dominant kernel (the phase with the largest share of the step)
-    pk = peaks()
-    mean_phase = {k: sum(v) / len(v) for k, v in phases.items()}
-    dominant = max(mean_phase, key=mean_phase.get) if mean_phase else "schedule"
-    dom_ms = mean_phase.get(dominant, total_ms / args.steps)
-    hbm_roof = lambda kernel, alg_bytes, what: {  # noqa: E731
-        "kernel": kernel, "bound": "hbm", "achieved": alg_bytes / (dom_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
-        "unit": "GB/s", "frac": alg_bytes / (dom_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None,
-        "peak_source": pk["source"], "algorithmic_bytes": alg_bytes, "bytes_are": what}
-    if dominant == "schedule" or cfg["kind"] == "fib":
-        # 6 token touches x 16 B + one 32 B store slot / frame record per invocation
-        roof = hbm_roof("rdf_scheduler_kernel", 128.0 * N, "128 B per invocation (token write+read, return/store slot write+read, frame record)")
-    elif dominant == "loss":
-        rowbytes = (64 * ((cfg["H"] + 63) // 64)) * 2 if use_tc else cfg["H"] * 4 * (2 if cell == "lstm" else 1)
-        roof = hbm_roof("rdf_loss_heads_kernel", float(N) * (rowbytes + 32), "one state row read + 32 B dlog written per invocation")
-    else:
-        H = cfg["H"]
-        C = cfg["trees"].n_cells
-        # algorithmic flops of the contraction in each phase: 2 * 2H * (rows of W) per cell
-        flops = flops_fwd
-        kernel = {"operators": "rdf_operator_kernel", "backward": "rdf_backward_kernel",
-                  "dW": "rdf_dw_tc_kernel" if use_tc else "rdf_outer_kernel"}.get(dominant, dominant)
-        if use_tc:
-            peak = pk["bf16_tflops_sustained"]
-            achieved = flops / (dom_ms * 1e-3) / 1e12
-            roof = {"kernel": kernel, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": None,
-                    "peak_source": pk["source"] + " (bf16 dense, sustained)", "cells": C, "flops_phase": flops,
-                    "note": "a persistent kernel: every wave ends at a grid barrier; block0_ms_at_max_clock gives the split"}
-            if dominant == "operators" and cell == "rnn":
-                Hp = 64 * ((H + 63) // 64)
-                # per cell: two bf16 operand rows read, one bf16 state row written; per leaf: an fp32 table row read, a bf16 row written
-                alg = C * (3.0 * Hp * 2) + (tb.N - C) * (H * 4.0 + Hp * 2)
-                roof["hbm_view"] = {"algorithmic_bytes": alg, "achieved_gbs": alg / (dom_ms * 1e-3) / 1e9,
-                                    "frac_of_hbm_peak": alg / (dom_ms * 1e-3) / 1e9 / pk["hbm_gbs"]}
-        else:
-            achieved = flops / (dom_ms * 1e-3) / 1e12
-            roof = {"kernel": kernel, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS,
-                    "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
-                    "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
-                    "cells": C, "flops_phase": flops}
-    roof["phase"] = dominant
-    roof["phase_ms"] = dom_ms
-
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((roof["kernel"], args.workload, args.fib_batch if args.workload == 1 else None))
-    cpu = None
-    if not args.no_cpu_baseline:
-        v, _, what = time_oracle(cfg, 1, 0, scale=1 if cfg["trees"].N > 2_000_000 else 4) if cfg["kind"] != "fib" else time_oracle(cfg, 1, 0, scale=4)
-        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
-
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": dtype, "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else ""),
-                   "invocations_per_step": N, "instances": cfg.get("B") or cfg["trees"].B,
-                   "pass": "forward+backward" if cfg.get("grad") else "forward",
-                   "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
-        "clocks": clk,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        # (bf16 with padded state rows: db / db_x come out of the dW / dW_x contractions, one / two kernels fewer)
-        "gpu_launches": (KERNELS_PER_STEP[kind] - ({"grad_tc": 1, "grad_lstm_tc": 2}.get(kind, 0) if cfg.get("H", 64) % 64 else 0)) * args.steps,
-        "roofline": roof,
-        "cpu_baseline": cpu,
-        "phase_ms": mean_phase,
-        "waves": {"forward": st["waves"], "backward": st["waves_backward"], "widest": st["max_wave_tokens"]},
-        "block0_ms_at_max_clock": {k[7:]: round(st[k] / 1.965e6, 4) for k in st if k.startswith("cycles_")},
-    }
-    print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    if in_ranks and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"bench.py --gpus {args.gpus} but the launcher started {os.environ['WORLD_SIZE']} rank(s)")
+    run(args)
 
 
 if __name__ == "__main__":

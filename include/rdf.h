@@ -232,6 +232,8 @@ typedef struct {
        work, batched operand gradients, waiting at grid barriers. */
     uint64_t cycles_schedule, cycles_batch, cycles_barrier;
     uint64_t cycles_bwd_frames, cycles_bwd_batch, cycles_bwd_barrier;
+    uint32_t kernel_launches;    /* kernels of the library that the last call launched (host count; memsets and copies excluded) */
+    uint32_t reserved;
 } rdf_stats;
 
 /* Bytes of device scratch rdf_eval (want_grad = 0) or rdf_grad (1) needs for
@@ -308,13 +310,20 @@ int rdf_set_limits(rdf_graph* g, long long wait_cycles, long long wave_limit);
  * host array `ms`, in this order:
  *   0 set-up (clears, program upload, seed tokens, weight packing)
  *   1 scheduler waves (tokens: tag push / pop, matching, lists of ready operators)
- *   2 operator waves (batched leaves and cells)   3 loss head with dW_s, db_s
- *   4 gradient waves   5 dW   6 db   7 dE (TreeLSTM; the TreeRNN's dE is formed during the waves)
- * (rdf_eval fills 0..2).  *n receives the number written. */
-enum { RDF_PHASE_SETUP = 0, RDF_PHASE_SCHEDULE, RDF_PHASE_OPERATORS, RDF_PHASE_LOSS, RDF_PHASE_BACKWARD, RDF_PHASE_DW,
-       RDF_PHASE_DB, RDF_PHASE_DE, RDF_PHASE__COUNT };
+ *   2 grouping of the ready cells by height     3 operator waves (batched leaves and cells)
+ *   4 root states to the caller's buffer        5 loss head with dW_s, db_s
+ *   6 lists of the gradient pass                7 gradient waves
+ *   8 dW (and dW_x)   9 db   10 dE (TreeLSTM; the TreeRNN's dE is formed during the waves)
+ * (rdf_eval fills 0..4).  *n receives the number written. */
+enum { RDF_PHASE_SETUP = 0, RDF_PHASE_SCHEDULE, RDF_PHASE_GROUP, RDF_PHASE_OPERATORS, RDF_PHASE_ROOTS, RDF_PHASE_LOSS,
+       RDF_PHASE_LISTS, RDF_PHASE_BACKWARD, RDF_PHASE_DW, RDF_PHASE_DB, RDF_PHASE_DE, RDF_PHASE__COUNT };
 int rdf_set_profiling(rdf_graph* g, int enable);
 int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n);
+
+/* Measurement aid (no counterpart in the paper): the fp32 fused-multiply-add rate the current device reaches
+ * on a register-resident loop, in TFLOP/s (host double) -- the peak the fp32 cell kernels are put against.
+ * Runs a few short kernels on `stream` and synchronises them. */
+int rdf_probe_fp32_fma(double* tflops, void* stream);
 
 #ifdef __cplusplus
 }

@@ -104,7 +104,8 @@ class rdf_stats(C.Structure):
                 ("store_inserts", C.c_uint64), ("store_matches", C.c_uint64), ("store_probes", C.c_uint64),
                 ("max_probe", C.c_uint32), ("max_depth", C.c_uint32), ("cells", C.c_uint64), ("leaves", C.c_uint64),
                 ("cycles_schedule", C.c_uint64), ("cycles_batch", C.c_uint64), ("cycles_barrier", C.c_uint64),
-                ("cycles_bwd_frames", C.c_uint64), ("cycles_bwd_batch", C.c_uint64), ("cycles_bwd_barrier", C.c_uint64)]
+                ("cycles_bwd_frames", C.c_uint64), ("cycles_bwd_batch", C.c_uint64), ("cycles_bwd_barrier", C.c_uint64),
+                ("kernel_launches", C.c_uint32), ("reserved", C.c_uint32)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -112,9 +113,9 @@ class rdf_stats(C.Structure):
 
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
            "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc",
-           "rdf_set_limits"]
+           "rdf_set_limits", "rdf_probe_fp32_fma"]
 NOALLOC_SCRATCH_BYTES = 16 << 20
-PHASES = ["setup", "schedule", "operators", "loss", "backward", "dW", "db", "dE"]
+PHASES = ["setup", "schedule", "group", "operators", "roots", "loss", "lists", "backward", "dW", "db", "dE"]
 
 _lib = None
 
@@ -140,11 +141,22 @@ def lib() -> C.CDLL:
         L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
         L.rdf_set_profiling.argtypes = [C.c_void_p, C.c_int]
         L.rdf_set_limits.argtypes = [C.c_void_p, C.c_longlong, C.c_longlong]
+        L.rdf_probe_fp32_fma.argtypes = [C.POINTER(C.c_double), C.c_void_p]
         L.rdf_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
         L.rdf_strerror.argtypes = [C.c_int]
         L.rdf_strerror.restype = C.c_char_p
         _lib = L
     return _lib
+
+
+def probe_fp32_fma_tflops() -> float:
+    """fp32 FMA rate of the current CUDA device on a register-resident loop (TFLOP/s)."""
+    torch = _torch()
+    v = C.c_double()
+    rc = lib().rdf_probe_fp32_fma(C.byref(v), torch.cuda.current_stream().cuda_stream)
+    if rc != RDF_OK:
+        raise RdfError(rc, "rdf_probe_fp32_fma")
+    return float(v.value)
 
 
 # ------------------------------------------------------- program description

@@ -911,6 +911,7 @@ int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params
 int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
                        DevCtx& c, cudaStream_t stream) {
     rdf_mark(S, 0, stream);
+    S->launches = 0;
     CUDA_OK(cudaMemsetAsync(ws + L.ctl, 0, 4096, stream));
     if (L.wave_cap) CUDA_OK(cudaMemsetAsync(ws + L.height_ends, 0, ((size_t)L.wave_cap + 2) * sizeof(uint32_t), stream));
     if (g->tag_mode == RDF_TAGS_FRAME) {
@@ -932,43 +933,48 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
         }
         CUDA_OK(cudaMemcpyAsync(ws + L.code, S->tables.data(), bytes, cudaMemcpyHostToDevice, stream));
     }
-    rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c);
+    RDF_KERNEL(S, rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c));
     CUDA_OK(cudaGetLastError());
     if (c.use_tc) {
         if (c.lstm) {
-            rdf_pack_lstm_kernel<<<256, 256, 0, stream>>>(c);
-            rdf_pack_e_kernel<<<1024, 256, 0, stream>>>(c);
+            RDF_KERNEL(S, rdf_pack_lstm_kernel<<<256, 256, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_pack_e_kernel<<<1024, 256, 0, stream>>>(c));
         } else {
-            rdf_pack_w_kernel<<<64, 256, 0, stream>>>(c);
+            RDF_KERNEL(S, rdf_pack_w_kernel<<<64, 256, 0, stream>>>(c));
         }
         CUDA_OK(cudaGetLastError());
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
-                                        2 * LQ_CAP * sizeof(Token), stream));
+    RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
+                                        2 * LQ_CAP * sizeof(Token), stream)));
     rdf_mark(S, 2, stream);
     if (g->has_vector_ops) {
         // the cells grouped by height; the operator kernel reads the grouped list in place of the scheduler's
-        rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
-        rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c);
-        rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c);
+        RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
+        RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c));
+        RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
         CUDA_OK(cudaGetLastError());
+        rdf_mark(S, 3, stream);
         DevCtx co = c;
         co.cell_items = c.cell_sorted;
         void* oargs[] = {(void*)&co};
         if (c.use_tc)
-            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), oargs,
-                                                (size_t)L.tc_smem_fwd, stream));
+            RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), oargs,
+                                                (size_t)L.tc_smem_fwd, stream)));
         else
-            CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
-                                                thin_resident_bytes(c.lstm, c.H), stream));
-        rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root);
+            RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
+                                                thin_resident_bytes(c.lstm, c.H), stream)));
+        rdf_mark(S, 4, stream);
+        RDF_KERNEL(S, rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root));
         CUDA_OK(cudaGetLastError());
+    } else {
+        rdf_mark(S, 3, stream);
+        rdf_mark(S, 4, stream);
     }
     if (out->trace)
         CUDA_OK(cudaMemcpyAsync(out->trace_count, &c.ctl->trace_count, sizeof(uint64_t), cudaMemcpyDeviceToDevice, stream));
-    rdf_mark(S, 3, stream);
+    rdf_mark(S, 5, stream);
     S->last_ctl = c.ctl;
     S->last_stream = stream;
     S->ran = true;
@@ -1024,6 +1030,7 @@ extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
     s->max_probe = h.max_probe; s->max_depth = h.max_depth; s->cells = h.cells; s->leaves = h.leaves;
     s->cycles_schedule = h.cyc[0]; s->cycles_batch = h.cyc[1]; s->cycles_barrier = h.cyc[2];
     s->cycles_bwd_frames = h.cyc[3]; s->cycles_bwd_batch = h.cyc[4]; s->cycles_bwd_barrier = h.cyc[5];
+    s->kernel_launches = S->launches;
     return h.status;
 }
 
@@ -1058,6 +1065,51 @@ extern "C" int rdf_last_phase_ms(rdf_graph* g, float* ms, int capacity, int* n) 
         *n = k + 1;
     }
     return RDF_OK;
+}
+
+// ===========================================================================
+// fp32 FMA rate of the device (the denominator for the fp32 cell kernels)
+// ===========================================================================
+static __device__ float rdf_probe_sink;
+
+__global__ void __launch_bounds__(256) rdf_probe_fma_kernel(int iters, float seed) {
+    // eight independent chains per thread, operands in registers: nothing but the FMA pipe is busy
+    float a0 = seed + threadIdx.x, a1 = a0 + 1.f, a2 = a0 + 2.f, a3 = a0 + 3.f, a4 = a0 + 4.f, a5 = a0 + 5.f, a6 = a0 + 6.f,
+          a7 = a0 + 7.f;
+    const float m = 0.999f, b = 1e-3f;
+#pragma unroll 4
+    for (int i = 0; i < iters; ++i) {
+        a0 = fmaf(a0, m, b); a1 = fmaf(a1, m, b); a2 = fmaf(a2, m, b); a3 = fmaf(a3, m, b);
+        a4 = fmaf(a4, m, b); a5 = fmaf(a5, m, b); a6 = fmaf(a6, m, b); a7 = fmaf(a7, m, b);
+    }
+    const float t = ((a0 + a1) + (a2 + a3)) + ((a4 + a5) + (a6 + a7));
+    if (t == -1.2345e30f) rdf_probe_sink = t;          // never true: keeps the chains alive
+}
+
+extern "C" int rdf_probe_fp32_fma(double* tflops, void* stream_v) {
+    if (!tflops) return RDF_ERR_BAD_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int dev = 0, sms = 0;
+    CUDA_OK(cudaGetDevice(&dev));
+    CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    cudaEvent_t e0, e1;
+    CUDA_OK(cudaEventCreate(&e0));
+    CUDA_OK(cudaEventCreate(&e1));
+    const int iters = 1 << 15, blocks = sms * 8;
+    double best = 0.0;
+    int rc = RDF_OK;
+    for (int rep = 0; rep < 4 && rc == RDF_OK; ++rep) {                    // the first repetition warms up
+        cudaEventRecord(e0, stream);
+        rdf_probe_fma_kernel<<<blocks, 256, 0, stream>>>(iters, 1.f);
+        cudaEventRecord(e1, stream);
+        float ms = 0.f;
+        if (cudaEventSynchronize(e1) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) rc = RDF_ERR_CUDA;
+        else if (rep > 0) best = std::max(best, 2.0 * 8.0 * iters * 256.0 * blocks / (ms * 1e-3) / 1e12);
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *tflops = best;
+    return rc;
 }
 
 // ===========================================================================

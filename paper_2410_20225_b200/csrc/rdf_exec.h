@@ -48,6 +48,7 @@ struct ExecState {
     void* last_ctl = nullptr;
     cudaStream_t last_stream = nullptr;
     bool ran = false;
+    unsigned launches = 0;       // kernels launched by the last call
     long long wait_cycles = 0;   // rdf_set_limits: 0 = default
     long long wave_limit = 0;
     // optional phase timing
@@ -76,6 +77,13 @@ struct Layout {
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes, pair_bytes;
 };
+
+// a kernel launch of the library, counted per call (rdf_stats.kernel_launches)
+#define RDF_KERNEL(S, ...)  \
+    do {                    \
+        __VA_ARGS__;        \
+        ++(S)->launches;    \
+    } while (0)
 
 #define CUDA_OK(expr)                                  \
     do {                                               \

@@ -1235,36 +1235,37 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         if (c.use_tc) {                    // bf16 states (TreeRNN and TreeLSTM): the h rows of arena_bf
             const int smem_mma = 2 * LM_ROWS * (c.Hp * 2 + 16);
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mma));
-            rdf_loss_heads_mma_kernel<<<loss_blocks, 256, smem_mma, stream>>>(c);
+            RDF_KERNEL(S, rdf_loss_heads_mma_kernel<<<loss_blocks, 256, smem_mma, stream>>>(c));
         } else {
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            rdf_loss_heads_kernel<false><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes);
+            RDF_KERNEL(S, rdf_loss_heads_kernel<false><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes));
         }
-        rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks);
+        RDF_KERNEL(S, rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks));
     }
-    rdf_mark(S, 4, stream);
+    rdf_mark(S, 6, stream);
     // lists of the gradient pass (cells in frame order, per-wave ends)
     {
         const int n_seg = (int)(in->max_invocations / LIST_SEG) + 1;
         uint2* seg = reinterpret_cast<uint2*>(ws + L.list_seg);
-        rdf_list_count_kernel<<<n_seg, 256, 0, stream>>>(c, seg);
-        rdf_list_scan_kernel<<<1, 1024, 0, stream>>>(c, seg, n_seg);
-        rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg);
-        rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg);
+        RDF_KERNEL(S, rdf_list_count_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
+        RDF_KERNEL(S, rdf_list_scan_kernel<<<1, 1024, 0, stream>>>(c, seg, n_seg));
+        RDF_KERNEL(S, rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
+        RDF_KERNEL(S, rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg));
     }
+    rdf_mark(S, 7, stream);
     // gradient waves
     CUDA_OK(cudaGetLastError());
     void* args[] = {(void*)&c};
     if (c.use_tc) {
         CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.tc_smem_bwd));
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
-                                            (size_t)L.tc_smem_bwd, stream));
+        RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
+                                            (size_t)L.tc_smem_bwd, stream)));
     } else {
         CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
-        CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
-                                            thin_resident_bytes(c.lstm, c.H), stream));
+        RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
+                                            thin_resident_bytes(c.lstm, c.H), stream)));
     }
-    rdf_mark(S, 5, stream);
+    rdf_mark(S, 8, stream);
     // parameter gradients
     const long long max_cells = std::max<long long>(1, in->max_invocations / 2 + 1);
     const long long max_leaves = std::max<long long>(1, in->max_invocations);
@@ -1278,7 +1279,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             a.n_tiles = ((a.Mp + DW_TILE - 1) / DW_TILE) * a.tiles_n;
             const long long stages = (max_items + DW_KT - 1) / DW_KT;
             a.splits = (int)std::max<long long>(1, std::min<long long>(S->grid / a.n_tiles, stages));
-            rdf_dw_tc_kernel<<<a.n_tiles * a.splits, 256, DW_SMEM_BYTES, stream>>>(c, a);
+            RDF_KERNEL(S, rdf_dw_tc_kernel<<<a.n_tiles * a.splits, 256, DW_SMEM_BYTES, stream>>>(c, a));
         };
         DwArgs a{};
         a.ops = c.cell_ops; a.count = &c.ctl->all_cells;
@@ -1296,30 +1297,30 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         }
     } else {
         OuterArgs aw = outer_args(c.all_cells, &c.ctl->all_cells, dgA, lda, MW, 2 * H, 0, grads->dW, max_cells, S->grid);
-        rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw);
+        RDF_KERNEL(S, rdf_outer_kernel<<<outer_blocks(aw, max_cells), 256, 0, stream>>>(c, aw));
         if (lstm) {
             OuterArgs ax = outer_args(c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, D, 1, grads->dW_x, max_leaves, S->grid);
-            rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax);
+            RDF_KERNEL(S, rdf_outer_kernel<<<outer_blocks(ax, max_leaves), 256, 0, stream>>>(c, ax));
         }
     }
-    rdf_mark(S, 6, stream);
+    rdf_mark(S, 9, stream);
     if (c.use_tc && H < c.Hp) {}        // (column H of the dW / dW_x contractions)
-    else if (tc_rnn) rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db);   // dz rows are in all_cells order
+    else if (tc_rnn) RDF_KERNEL(S, rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db));   // dz rows are in all_cells order
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
-        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db);
-        rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x);
+        RDF_KERNEL(S, rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db));
+        RDF_KERNEL(S, rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, H, c.Hp, grads->db_x));
     } else {
-        rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, dgA, lda, MW, H, H, grads->db);
-        if (lstm) rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, H, H, grads->db_x);
+        RDF_KERNEL(S, rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, dgA, lda, MW, H, H, grads->db));
+        if (lstm) RDF_KERNEL(S, rdf_colsum_kernel<float><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_leaves, &c.ctl->all_leaves, c.gates, c.G, 3 * H, H, H, grads->db_x));
     }
-    rdf_mark(S, 7, stream);       // (dW_s and db_s came from the loss-head pass)
+    rdf_mark(S, 10, stream);      // (dW_s and db_s came from the loss-head pass)
     if (tc_lstm) {
         const int n_split = c.Hp / 64, de_smem = tc_smem_bytes(64, 3 * c.Hp, 0, 0, 5);
         CUDA_OK(cudaFuncSetAttribute(rdf_de_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, de_smem));
-        rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, TC_THREADS, de_smem, stream>>>(c);
-    } else if (lstm) rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN);
+        RDF_KERNEL(S, rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, TC_THREADS, de_smem, stream>>>(c));
+    } else if (lstm) RDF_KERNEL(S, rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN));
     // (TreeRNN: the leaves added their dh to dE during the gradient waves)
-    rdf_mark(S, 8, stream);
+    rdf_mark(S, 11, stream);
     CUDA_OK(cudaGetLastError());
     return RDF_OK;
 }
