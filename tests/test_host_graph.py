@@ -21,7 +21,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def test_library_exports_every_declared_symbol():
     lib = rdf.lib()
     header = open(os.path.join(ROOT, "include", "rdf.h")).read()
-    declared = set(re.findall(r"^(?:int|void|const char\*)\s+(rdf_[a-z_]+)\s*\(", header, flags=re.M))
+    declared = set(re.findall(r"^(?:int|void|const char\*)\s+(rdf_[a-z0-9_]+)\s*\(", header, flags=re.M))
     assert {"rdf_graph_build", "rdf_eval", "rdf_grad", "rdf_graph_free", "rdf_strerror"} <= declared
     for name in declared:
         assert hasattr(lib, name), name
