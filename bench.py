@@ -42,8 +42,8 @@ WORKLOAD_NAMES = {
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
 }
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
-KERNEL_SOURCES = ["rdf_device.cuh", "rdf_exec.cu", "rdf_exec.h", "rdf_grad.cu", "rdf_internal.h", "rdf_lstm.cuh", "rdf_tc.cuh",
-                  "rdf_tc_dw.cuh"]
+KERNEL_SOURCES = ["rdf_device.cuh", "rdf_exec.cu", "rdf_exec.h", "rdf_grad.cu", "rdf_internal.h", "rdf_lists.cuh", "rdf_lstm.cuh",
+                  "rdf_tc.cuh", "rdf_tc_dw.cuh"]
 
 
 def fib_iter(n):

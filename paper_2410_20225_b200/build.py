@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "librdf.so")
 SOURCES = ["rdf_graph.cpp", "rdf_exec.cu", "rdf_grad.cu"]
-HEADERS = ["rdf_internal.h", "rdf_device.cuh", "rdf_exec.h", "rdf_lstm.cuh", "rdf_tc.cuh", "rdf_tc_dw.cuh"]
+HEADERS = ["rdf_internal.h", "rdf_device.cuh", "rdf_exec.h", "rdf_lstm.cuh", "rdf_tc.cuh", "rdf_tc_dw.cuh", "rdf_lists.cuh"]
 
 
 def _stale() -> bool:

@@ -73,6 +73,7 @@ struct Control {
     uint32_t all_leaves;          // backward: leaves seen so far
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     uint32_t max_height;          // largest height of a cell of this call (operator waves run height by height)
+    uint32_t n_depth_waves;       // scheduler waves that made calls = call depths of the run (length of the compacted wave_marks)
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
     unsigned long long cyc[6];    // block 0: forward schedule / batch / barrier, backward frames / batch / barrier
@@ -134,6 +135,12 @@ struct DevCtx {
                                   // all_cells: the cells of a gradient wave are consecutive rows, read as plain 2D tiles
     uint32_t* cell_pos;           // per frame: position of a cell in all_cells (written with the lists; leaves: undefined)
     TensorMap tmap_dz128, tmap_dz64;   // dz_bf as [rows, Hp], 128-byte swizzle, boxes of 128 / 64 rows by 64 columns
+    __nv_bfloat16* z_bf;          // [cells_cap, 2Hp] operand rows [h_l ; h_r] of the cells, row = position of the cell in
+                                  // all_cells: every invocation writes its state into the half of its caller's row
+                                  // that it feeds, so a tile of consecutive cells reads its operands as plain 2D tiles
+    uint32_t* zdst;               // per frame: 2 * (position of the calling cell) + operand port, or NO_ZDST
+    uint32_t  cells_cap;          // rows of z_bf / dz_bf that exist
+    TensorMap tmap_z128, tmap_z64;     // z_bf as [rows, 2Hp]
     // TreeLSTM on tensor cores: Wp / WTp hold the slice-major W5p [5Hp, 2Hp] and WT5p [2Hp, 5Hp]
     __nv_bfloat16* Wxp;           // [3Hp, Hp] leaf projection, slice-major
     __nv_bfloat16* WxTp;          // [Hp, 3Hp] its transpose (operand of the embedding gradient)
@@ -151,10 +158,11 @@ struct DevCtx {
     float*    dhp;                // [frame_cap, S]: gradient arriving from the caller (dh, and dc for the TreeLSTM);
                                   //                 TreeRNN: overwritten by dz (cell) / dh (leaf)
     float*    dlog;               // [frame_cap, 8]: softmax - onehot per invocation
-    uint4*    wave_marks;         // [wave_cap], filled by the list kernels of the gradient pass: .x = frames created up to
-                                  // the end of scheduler wave w (0: none in that wave), .w = cells among them.
-                                  // Frame ids are handed out in wave order, so the invocations that Call_i created
-                                  // in wave w are one id range -- one wave of the gradient pass
+    uint4*    wave_marks;         // [wave_cap], filled by the list kernels: entry k = {first frame, one past the last frame,
+                                  // first cell, one past the last cell (positions in all_cells)} of the k-th scheduler
+                                  // wave that made calls.  Frame ids are handed out in wave order, so the invocations
+                                  // of one call depth are one id range -- one wave of the gradient pass, and (from
+                                  // the deepest one up) one wave of the tensor-core operator kernel
     uint32_t  wave_cap;
     uint32_t* all_cells;          // every cell frame, in backward wave order
     uint4*    cell_ops;           // {cell frame, left operand frame, right operand frame, 1} in all_cells order
@@ -170,6 +178,7 @@ struct DevCtx {
 };
 
 static const uint32_t LEAF_MARK = 0xFFFFFFFFu;
+static const uint32_t NO_ZDST = 0xFFFFFFFFu;
 
 // ---------------------------------------------------------------- utilities
 __device__ __forceinline__ void set_status(const DevCtx& c, int code) { atomicCAS(&c.ctl->status, 0, code); }

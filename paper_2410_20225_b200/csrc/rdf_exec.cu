@@ -16,6 +16,7 @@
 #include <type_traits>
 
 #include "rdf_exec.h"
+#include "rdf_lists.cuh"
 #include "rdf_lstm.cuh"
 #include "rdf_tc.cuh"
 
@@ -525,9 +526,9 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     }
 }
 
-// The operator kernel: the leaves first (they wait for nothing), then, height by height, the cells of that
-// height; a grid barrier separates the waves (a cell reads states of smaller heights).
-// TC: bf16 operands on the tensor cores (the tile pipeline of rdf_tc.cuh); otherwise fp32 FMA tiles.
+// The operator kernel: the leaves first (they wait for nothing), then the cells in waves whose operands are complete;
+// a grid barrier separates the waves.  fp32 FMA tiles: height by height (a cell reads states of smaller heights).
+// TC: bf16 operands on the tensor cores (the tile pipeline of rdf_tc.cuh), depth by depth from the deepest cells up.
 template <bool TC>
 __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
     __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // (the TreeRNN tiles use the first part of LstmSmem)
@@ -560,13 +561,15 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         acc += now - t_mark;
         t_mark = now;
     };
-    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
     const uint32_t n_leaf = min(c.ctl->leaf_count.v, c.work_cap);
     bool alive = true;
     if (n_leaf) {
         if constexpr (TC) {
             if (c.lstm) tc_pipe<TC_LSTM_LEAF, TC_STAGES_LSTM_FWD>(c, tc, smem, 0, n_leaf);
-            else tc_leaf_rows(c, n_leaf);
+            else {
+                tc_leaf_rows(c, n_leaf);
+                asm volatile("fence.proxy.async;" ::: "memory");      // the operand rows it wrote are read by tile copies after the barrier
+            }
         } else {
             if (c.lstm) lstm_forward_tiles<3>(c, smem, 0, n_leaf);
             else rnn_leaf_rows(c, n_leaf);
@@ -576,28 +579,43 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
         alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
         lap(cyc_b);
     }
-    // (cell_items is the height-sorted list here: the launch passes cell_sorted in its place)
-    uint32_t first = 0;
-    const uint32_t top = min(c.ctl->max_height, c.wave_cap);
-    for (uint32_t w = 1; w <= top && alive; ++w) {
-        const uint32_t end = min(c.height_ends[w], c.work_cap);
-        if (end <= first) continue;                                  // (no cell of this height)
-        const uint32_t nc = end - first;
-        if constexpr (TC) {
+    if constexpr (TC) {
+        // Tensor-core path: the cells depth by depth, deepest first (the states a cell of depth k reads belong to
+        // depth k + 1).  The cells of one depth are consecutive in the cell list, and so are their operand rows,
+        // which their callees wrote: the tiles read plain 2D boxes.
+        const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap);
+        uint4 wv = nw ? c.wave_marks[nw - 1] : make_uint4(0u, 0u, 0u, 0u);      // {first frame, end frame, first cell, end cell}
+        for (uint32_t k = nw; k-- > 0 && alive;) {
+            const uint4 cur = wv;
+            if (k > 0) wv = c.wave_marks[k - 1];                         // in flight during this wave
+            if (cur.w <= cur.z) continue;                                // (a depth of leaves only)
+            const uint32_t first = min(cur.z, c.cells_cap), nc = min(cur.w, c.cells_cap) - first;
             if (c.lstm) tc_pipe<TC_LSTM_CELL, TC_STAGES_LSTM_FWD>(c, tc, smem, first, nc);
             else tc_pipe<TC_RNN_FWD, TC_STAGES_RNN_FWD>(c, tc, smem, first, nc);
-        } else {
+            __syncthreads();
+            lap(cyc_c);
+            alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
+            lap(cyc_b);
+        }
+    } else {
+        // fp32 path: height by height (cell_items is the height-sorted list here: the launch passes cell_sorted in its place)
+        uint32_t first = 0;
+        const uint32_t top = min(c.ctl->max_height, c.wave_cap);
+        for (uint32_t w = 1; w <= top && alive; ++w) {
+            const uint32_t end = min(c.height_ends[w], c.work_cap);
+            if (end <= first) continue;                                  // (no cell of this height)
+            const uint32_t nc = end - first;
             if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
             // thin patches while they fit in two rounds over the grid, tiles for wide waves
             else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
                 rnn_cell_thin(c, reinterpret_cast<float*>(&smem), wres, first, nc);      // 8 x 2H + 128 floats <= 26 KB
             else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
+            first = end;
+            __syncthreads();
+            lap(cyc_c);
+            alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
+            lap(cyc_b);
         }
-        first = end;
-        __syncthreads();
-        lap(cyc_c);
-        alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
-        lap(cyc_b);
     }
     if constexpr (TC) tc_teardown(tc);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -758,8 +776,13 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.arena_bf = P.take<__nv_bfloat16>(L.use_tc ? vf * L.Hp : 0);
     L.wp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
     L.wtp = P.take<__nv_bfloat16>(L.use_tc ? wcount : 0);
-    L.dz_bf = P.take<__nv_bfloat16>(tcr && want_grad ? vf * L.Hp : 0);
-    L.cell_pos = P.take<uint32_t>(tcr && want_grad ? vf : 0);
+    // a cell makes two calls, so a run has at most half as many cells as invocations; rows in whole tiles, one tile to spare
+    L.cells_cap = L.use_tc ? ((uint32_t)(vf / 2 + 1) + 127u) / 128u * 128u + 128u : 0;
+    L.want_grad = want_grad;
+    L.dz_bf = P.take<__nv_bfloat16>(tcr && want_grad ? (size_t)L.cells_cap * L.Hp : 0);
+    L.z_bf = P.take<__nv_bfloat16>(L.use_tc ? (size_t)L.cells_cap * 2 * L.Hp : 0);
+    L.zdst = P.take<uint32_t>(L.use_tc ? vf : 0);
+    L.cell_pos = P.take<uint32_t>(L.use_tc ? vf : 0);
     L.wxp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.wxtp = P.take<__nv_bfloat16>(tcl ? (size_t)3 * L.Hp * L.Hp : 0);
     L.e_bf = P.take<__nv_bfloat16>(tcl ? (size_t)params->V * L.Hp : 0);
@@ -774,11 +797,13 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.wave_cap = g->has_vector_ops ? (uint32_t)std::min<long long>(2 * (long long)L.frame_cap + 64, 1ll << 24) : 0;
     L.wave_marks = P.take<uint4>(L.wave_cap);
     L.height_ends = P.take<uint32_t>(L.wave_cap ? (size_t)L.wave_cap + 2 : 0);
-    L.list_seg = P.take<uint2>(want_grad ? (size_t)in->max_invocations / 2048 + 2 : 0);
-    L.all_cells = P.take<uint32_t>(gf);
-    L.cell_ops = P.take<uint4>(L.use_tc ? gf : 0);
+    // the lists over the frames: the gradient pass needs them, and so do the tensor-core operator waves
+    const size_t lf = want_grad || L.use_tc ? L.frame_cap : 0;
+    L.list_seg = P.take<uint2>(lf ? (size_t)in->max_invocations / LIST_SEG + 2 : 0);
+    L.all_cells = P.take<uint32_t>(lf);
+    L.cell_ops = P.take<uint4>(L.use_tc ? lf : 0);
     L.leaf_ops = P.take<uint4>(tcl ? gf : 0);
-    L.all_leaves = P.take<uint32_t>(gf);
+    L.all_leaves = P.take<uint32_t>(g->has_lstm ? lf : gf);
     L.loss_partial = P.take<float>(want_grad ? 4096 : 0);
     L.total = (P.off + 255) & ~(size_t)255;
     return RDF_OK;
@@ -860,8 +885,11 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
         c.arena_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.arena_bf);
         c.Wp = reinterpret_cast<__nv_bfloat16*>(ws + L.wp);
         c.WTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wtp);
-        c.dz_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf);
-        c.cell_pos = L.use_tc && !g->has_lstm ? reinterpret_cast<uint32_t*>(ws + L.cell_pos) : nullptr;
+        c.dz_bf = L.use_tc && !g->has_lstm && L.want_grad ? reinterpret_cast<__nv_bfloat16*>(ws + L.dz_bf) : nullptr;
+        c.z_bf = L.use_tc ? reinterpret_cast<__nv_bfloat16*>(ws + L.z_bf) : nullptr;
+        c.zdst = L.use_tc ? reinterpret_cast<uint32_t*>(ws + L.zdst) : nullptr;
+        c.cells_cap = L.cells_cap;
+        c.cell_pos = L.use_tc ? reinterpret_cast<uint32_t*>(ws + L.cell_pos) : nullptr;
         c.Wxp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxp);
         c.WxTp = reinterpret_cast<__nv_bfloat16*>(ws + L.wxtp);
         c.E_bf = reinterpret_cast<__nv_bfloat16*>(ws + L.e_bf);
@@ -877,7 +905,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.wave_cap = L.wave_cap;
     c.all_cells = reinterpret_cast<uint32_t*>(ws + L.all_cells);
     c.cell_ops = L.use_tc ? reinterpret_cast<uint4*>(ws + L.cell_ops) : nullptr;
-    c.leaf_ops = L.use_tc && g->has_lstm ? reinterpret_cast<uint4*>(ws + L.leaf_ops) : nullptr;
+    c.leaf_ops = L.use_tc && g->has_lstm && L.want_grad ? reinterpret_cast<uint4*>(ws + L.leaf_ops) : nullptr;
     c.all_leaves = reinterpret_cast<uint32_t*>(ws + L.all_leaves);
     c.loss_partial = reinterpret_cast<float*>(ws + L.loss_partial);
     c.loss_out = out->loss;
@@ -950,21 +978,29 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
                                         2 * LQ_CAP * sizeof(Token), stream)));
     rdf_mark(S, 2, stream);
     if (g->has_vector_ops) {
-        // the cells grouped by height; the operator kernel reads the grouped list in place of the scheduler's
-        RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
-        RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c));
-        RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
-        CUDA_OK(cudaGetLastError());
-        rdf_mark(S, 3, stream);
+        void* oargs[] = {(void*)&c};
         DevCtx co = c;
-        co.cell_items = c.cell_sorted;
-        void* oargs[] = {(void*)&co};
-        if (c.use_tc)
+        if (c.use_tc) {
+            // the cells listed by call depth, with the operand row that every invocation's state goes to
+            int rc = encode_row_tiles(&c.tmap_z128, c.z_bf, c.cells_cap, (uint64_t)2 * c.Hp, 128);
+            if (rc == RDF_OK) rc = encode_row_tiles(&c.tmap_z64, c.z_bf, c.cells_cap, (uint64_t)2 * c.Hp, 64);
+            if (rc == RDF_OK) rc = rdf_launch_lists(in, ws, L, S, c, stream);
+            if (rc != RDF_OK) return rc;
+            rdf_mark(S, 3, stream);
             RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<true>, dim3(S->grid), dim3(TC_THREADS), oargs,
                                                 (size_t)L.tc_smem_fwd, stream)));
-        else
+        } else {
+            // the cells grouped by height; the operator kernel reads the grouped list in place of the scheduler's
+            RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
+            CUDA_OK(cudaGetLastError());
+            rdf_mark(S, 3, stream);
+            co.cell_items = c.cell_sorted;
+            oargs[0] = (void*)&co;
             RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
                                                 thin_resident_bytes(c.lstm, c.H), stream)));
+        }
         rdf_mark(S, 4, stream);
         RDF_KERNEL(S, rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root));
         CUDA_OK(cudaGetLastError());
@@ -978,6 +1014,18 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     S->last_ctl = c.ctl;
     S->last_stream = stream;
     S->ran = true;
+    return RDF_OK;
+}
+
+int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* S, DevCtx& c, cudaStream_t stream) {
+    const int n_seg = (int)(in->max_invocations / LIST_SEG) + 1;
+    uint2* seg = reinterpret_cast<uint2*>(ws + L.list_seg);
+    RDF_KERNEL(S, rdf_list_count_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
+    RDF_KERNEL(S, rdf_list_scan_kernel<<<1, 1024, 0, stream>>>(c, seg, n_seg));
+    RDF_KERNEL(S, rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
+    RDF_KERNEL(S, rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg));
+    RDF_KERNEL(S, rdf_wave_compact_kernel<<<1, 1024, 0, stream>>>(c));
+    CUDA_OK(cudaGetLastError());
     return RDF_OK;
 }
 

@@ -40,6 +40,8 @@ __device__ __forceinline__ void gemm_tile_step(const GemmSmem& sm, int tx, int t
 static const int THIN_RESIDENT_MAX_H = 384;
 inline size_t thin_resident_bytes(int lstm, int H) { return !lstm && H <= THIN_RESIDENT_MAX_H ? (size_t)128 * H : 0; }
 
+static const int LIST_SEG = 2048;            // frames per segment of the list kernels (256 threads x 8)
+
 // ---- host state
 struct ExecState {
     int device = -1;
@@ -71,9 +73,9 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, children, pair_slots, port_val, arrived, table, cell_items,
-        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, total;
-    uint32_t qcap, frame_cap, work_cap, wave_cap;
-    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd;
+        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, total;
+    uint32_t qcap, frame_cap, work_cap, wave_cap, cells_cap;
+    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad;
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes, pair_bytes;
 };
@@ -97,5 +99,9 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S);
 void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, char* ws,
                   const Layout& L, ExecState* S, DevCtx& c);
 int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params, rdf_outputs* out, void* ws);
+// a row-major bf16 matrix [rows, cols] as a 2D tensor map for tile copies: boxes of box_rows x 64 columns, 128-byte swizzle
+int encode_row_tiles(TensorMap* out, void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// the lists over the frames (cells in depth order, waves, operand-row destinations); TC path: part of the forward pass
+int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* S, DevCtx& c, cudaStream_t stream);
 int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
                        DevCtx& c, cudaStream_t stream);

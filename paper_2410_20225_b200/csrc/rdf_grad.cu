@@ -11,8 +11,6 @@
 #include <cstring>
 #include <type_traits>
 
-#include <cuda.h>              // CUtensorMap and the prototype of its encoder (the entry point is looked up at run time)
-
 #include "rdf_exec.h"
 #include "rdf_tc.cuh"
 #include "rdf_tc_dw.cuh"
@@ -425,158 +423,6 @@ __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int
 }
 
 // ----------------------------------------------------------- backward waves
-// Lists of the gradient pass, formed once before the waves.  Frame ids are handed out in wave order,
-// so listing the cells in frame order puts the cells of every gradient wave next to each other:
-// wave d owns all_cells[marks[d-1].w, marks[d].w), the rows of its operand-gradient contraction.
-// Three small kernels: per-segment counts, scan of the counts, fill (and the per-wave ends).
-// Where a wave ends in the id space is read off the frames themselves (every frame records the scheduler
-// wave its Call_i fired in): marks[w].x = one past the last frame of wave w, 0 for a wave without calls.
-static const int LIST_SEG = 2048;            // frames per segment (256 threads x 8)
-
-__device__ __forceinline__ void list_flags(const DevCtx& c, uint32_t f0, uint32_t F, uint32_t (&l)[8], uint32_t (&r)[8],
-                                           uint32_t& cells, uint32_t& leaves) {
-    cells = leaves = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {                       // thread-contiguous: frames f0 + 8 tid + i
-        const uint32_t f = f0 + threadIdx.x * 8 + i;
-        l[i] = LEAF_MARK; r[i] = 0;
-        if (f < F) {
-            l[i] = c.op_l[f]; r[i] = c.op_r[f];
-            if (l[i] != LEAF_MARK) ++cells; else ++leaves;
-        }
-    }
-}
-
-__global__ void __launch_bounds__(256) rdf_list_count_kernel(const DevCtx c, uint2* seg_counts) {
-    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
-    __shared__ uint32_t wc[8], wl[8];
-    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
-    uint32_t l[8], r[8], cells, leaves;
-    list_flags(c, f0, F, l, r, cells, leaves);
-    for (int o = 16; o > 0; o >>= 1) {
-        cells += __shfl_xor_sync(0xffffffffu, cells, o);
-        leaves += __shfl_xor_sync(0xffffffffu, leaves, o);
-    }
-    if (threadIdx.x % 32 == 0) { wc[threadIdx.x / 32] = cells; wl[threadIdx.x / 32] = leaves; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t a = 0, b = 0;
-        for (int w = 0; w < 8; ++w) { a += wc[w]; b += wl[w]; }
-        seg_counts[blockIdx.x] = make_uint2(a, b);
-    }
-    // the marks of this call's waves start empty (the fill kernel writes the ends of the waves that made calls)
-    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
-    for (uint32_t w = blockIdx.x * blockDim.x + threadIdx.x; w < n_waves; w += gridDim.x * blockDim.x)
-        c.wave_marks[w] = make_uint4(0u, 0u, 0u, 0u);
-}
-
-// one block: exclusive scan of the segment counts in place; totals to the control block
-__global__ void __launch_bounds__(1024) rdf_list_scan_kernel(const DevCtx c, uint2* seg_counts, int n_seg) {
-    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
-    __shared__ uint32_t wa[32], wb[32];
-    const int per = (n_seg + 1023) / 1024, s0 = threadIdx.x * per, s1 = min(n_seg, s0 + per);
-    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    uint32_t a = 0, b = 0;
-    for (int i = s0; i < s1; ++i) { a += seg_counts[i].x; b += seg_counts[i].y; }
-    uint32_t pa = a, pb = b;                            // inclusive scan over the threads
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t x = __shfl_up_sync(0xffffffffu, pa, o), y = __shfl_up_sync(0xffffffffu, pb, o);
-        if (lane >= o) { pa += x; pb += y; }
-    }
-    if (lane == 31) { wa[warp] = pa; wb[warp] = pb; }
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t x = wa[lane], y = wb[lane];
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t u = __shfl_up_sync(0xffffffffu, x, o), v = __shfl_up_sync(0xffffffffu, y, o);
-            if (lane >= o) { x += u; y += v; }
-        }
-        wa[lane] = x; wb[lane] = y;                     // inclusive over the warps
-        if (lane == 31) { c.ctl->all_cells = x; c.ctl->all_leaves = y; }
-    }
-    __syncthreads();
-    a = pa - a + (warp ? wa[warp - 1] : 0u);
-    b = pb - b + (warp ? wb[warp - 1] : 0u);
-    for (int i = s0; i < s1; ++i) {
-        const uint2 v = seg_counts[i];
-        seg_counts[i] = make_uint2(a, b);
-        a += v.x; b += v.y;
-    }
-}
-
-__global__ void __launch_bounds__(256) rdf_list_fill_kernel(const DevCtx c, const uint2* seg_base) {
-    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
-    __shared__ uint32_t wc[8], wl[8];
-    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), f0 = (uint32_t)c.B + blockIdx.x * LIST_SEG;
-    uint32_t l[8], r[8], cells, leaves;
-    list_flags(c, f0, F, l, r, cells, leaves);
-    // exclusive prefix of (cells, leaves) over the threads of the block
-    uint32_t pc = cells, pl = leaves;
-    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t a = __shfl_up_sync(0xffffffffu, pc, o), b = __shfl_up_sync(0xffffffffu, pl, o);
-        if (lane >= o) { pc += a; pl += b; }
-    }
-    if (lane == 31) { wc[warp] = pc; wl[warp] = pl; }
-    __syncthreads();
-    const uint2 sb = seg_base[blockIdx.x];
-    uint32_t ic = sb.x + pc - cells, il = sb.y + pl - leaves;
-    for (int w = 0; w < warp; ++w) { ic += wc[w]; il += wl[w]; }
-    // ends of the waves in the id space: frame f is the last of its wave when the next frame belongs to a later one
-    {
-        const uint32_t fa = f0 + threadIdx.x * 8;
-        uint32_t wv = fa < F ? c.frames[fa].label >> FRAME_WAVE_SHIFT : 0u;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t f = fa + i;
-            if (f >= F) break;
-            const uint32_t wn = f + 1 < F ? c.frames[f + 1].label >> FRAME_WAVE_SHIFT : 0xFFFFFFFFu;
-            if (wn != wv && wv < c.wave_cap) c.wave_marks[wv].x = f + 1;
-            wv = wn;
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t f = f0 + threadIdx.x * 8 + i;
-        if (f >= F) break;
-        if (l[i] != LEAF_MARK) {
-            c.all_cells[ic] = f;
-            if (c.cell_ops) c.cell_ops[ic] = make_uint4(f, l[i], r[i], 1u);
-            if (c.cell_pos) c.cell_pos[f] = ic;
-            ++ic;
-        } else {
-            if (c.lstm) {
-                c.all_leaves[il] = f;
-                if (c.leaf_ops) c.leaf_ops[il] = make_uint4(f, r[i], 0u, 1u);      // r = token id of a leaf
-            }
-            ++il;
-        }
-    }
-}
-
-// marks[d].w = cells among the frames below marks[d].x: where wave d ends in all_cells.  One warp per wave.
-__global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, const uint2* seg_base) {
-    if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
-    const uint32_t lane = threadIdx.x % 32, n_warps = gridDim.x * blockDim.x / 32;
-    const uint32_t n_waves = min(c.ctl->waves, c.wave_cap);
-    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
-    for (uint32_t d = (blockIdx.x * blockDim.x + threadIdx.x) / 32; d < n_waves; d += n_warps) {
-        const uint32_t f = max(B, min(c.wave_marks[d].x, F));
-        const uint32_t seg = (f - B) / LIST_SEG, s0 = B + seg * LIST_SEG;      // (the segment array has one entry to spare)
-        uint32_t cnt = 0;
-        for (uint32_t g = s0 + lane; g < f; g += 32) cnt += c.op_l[g] != LEAF_MARK;
-        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        if (lane == 0) c.wave_marks[d].w = seg_base[seg].x + cnt;
-    }
-    // bf16 TreeRNN: the weight gradient reads dz in whole stages of 64 rows; the rows after the last cell are zero
-    if (c.cell_pos && blockIdx.x == 0) {
-        const uint32_t n = min(c.ctl->all_cells, c.frame_cap), n_end = min((n + 63u) & ~63u, c.frame_cap);
-        const uint32_t per_row = (uint32_t)c.Hp / 8;
-        for (uint32_t q = threadIdx.x; q < (n_end - n) * per_row; q += blockDim.x)
-            *reinterpret_cast<uint4*>(c.dz_bf + (size_t)(n + q / per_row) * c.Hp + (q % per_row) * 8) = make_uint4(0u, 0u, 0u, 0u);
-    }
-}
-
 // What a thread needs to know about an invocation before it touches its rows; all of it is left
 // behind by the forward pass and the loss head, so it can be fetched one step ahead.
 struct FrameMeta {
@@ -939,27 +785,29 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         }
     }
     const int lane = threadIdx.x % 32, wib = threadIdx.x / 32, n_warps = blockDim.x / 32;
-    uint32_t generation = 0, wave = 0, first = 0;
+    uint32_t generation = 0, wave = 0;
     long long cyc_a = 0, cyc_c = 0, cyc_b = 0, t_mark = clock64();
     auto lap = [&](long long& acc) {
         const long long now = clock64();
         acc += now - t_mark;
         t_mark = now;
     };
-    // Gradient wave d re-enters the invocations that Call_i created in forward wave d: frame ids are
-    // handed out in wave order, so they are the range [f0, f1) and their rows are consecutive in memory.
-    const uint32_t n_fwd = min(c.ctl->waves, c.wave_cap);
-    uint32_t f1 = (uint32_t)c.B;
+    // Gradient wave k re-enters the invocations of call depth k (the k-th scheduler wave that made calls): frame ids
+    // are handed out in wave order, so they are one id range [f0, f1) and their rows are consecutive in memory; the
+    // cells among them are all_cells[first, end).
+    const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap);
     bool callees_done = false;        // the previous wave's contraction has already finished this wave's invocations
-    for (uint32_t d = 0; d < n_fwd; ++d) {
-        const uint32_t f0 = f1;
-        f1 = max(f0, min(c.wave_marks[d].x, c.frame_cap));
-        if (f1 == f0) continue;                                      // a wave without calls
+    uint4 wv = nw ? c.wave_marks[0] : make_uint4(0u, 0u, 0u, 0u);
+    for (uint32_t k = 0; k < nw; ++k) {
+        const uint4 cur = wv;
+        if (k + 1 < nw) wv = c.wave_marks[k + 1];                    // in flight during this wave
+        const uint32_t f0 = min(cur.x, c.frame_cap), f1 = min(cur.y, c.frame_cap);
+        if (f1 <= f0) continue;
         ++wave;
         // ---- A: per-invocation work, a contiguous piece of the range per block.  (bf16 TreeRNN: only the
         //      invocations called from `result` -- further down the epilogue of B does this work for the callees;
         //      fp32 TreeRNN: not after a wave of narrow patches, which do the same.)
-        if (!(TC && !c.lstm && d > 0) && !callees_done) {
+        if (!(TC && !c.lstm && k > 0) && !callees_done) {
             const uint32_t n = f1 - f0;
             const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
             const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
@@ -978,7 +826,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
             lap(cyc_b);
         }
         // ---- B: operand gradients of the wave's cells, handed to the frames of the calls they made
-        const uint32_t end = max(first, min(c.wave_marks[d].w, c.frame_cap));     // the wave's cells: all_cells[first, end)
+        const uint32_t first = min(cur.z, c.frame_cap), end = min(cur.w, c.frame_cap);
         bool thin = false;
         if (end > first) {
             if constexpr (TC) {
@@ -991,7 +839,6 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
                     thin = true;
                 } else backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.dhp, c.H, c.H);
             }
-            first = end;
             __syncthreads();
             lap(cyc_c);
             if (!grid_barrier(c, &c.ctl->bar2.v, generation)) break;
@@ -1004,30 +851,6 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         c.ctl->waves_backward = wave;
         c.ctl->cyc[3] = cyc_a; c.ctl->cyc[4] = cyc_c; c.ctl->cyc[5] = cyc_b;
     }
-}
-
-// dz_bf as a 2D tensor [rows, Hp] of bf16 for tile copies: boxes of box_rows x 64 columns in the 128-byte swizzle.
-typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                           const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                           CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static int encode_row_tiles(TensorMap* out, void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "tensor map size");
-    static TensorMapEncodeTiledFn encode = nullptr;
-    if (!encode) {
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
-            return RDF_ERR_CUDA;
-        encode = reinterpret_cast<TensorMapEncodeTiledFn>(fn);
-    }
-    const cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {64, box_rows}, estr[2] = {1, 1};
-    CUtensorMap m;
-    if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return RDF_ERR_CUDA;
-    memcpy(out, &m, sizeof(m));
-    return RDF_OK;
 }
 
 // ------------------------------------------- parameter gradients (post pass)
@@ -1223,8 +1046,8 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     // loss head over every retained invocation
     const bool tc_rnn = c.use_tc && !lstm, tc_lstm = c.use_tc && lstm;
     if (tc_rnn) {                          // dz rows are read as 2D tiles by the gradient waves and by the weight gradient
-        rc = encode_row_tiles(&c.tmap_dz128, c.dz_bf, c.frame_cap, (uint64_t)c.Hp, 128);
-        if (rc == RDF_OK) rc = encode_row_tiles(&c.tmap_dz64, c.dz_bf, c.frame_cap, (uint64_t)c.Hp, 64);
+        rc = encode_row_tiles(&c.tmap_dz128, c.dz_bf, c.cells_cap, (uint64_t)c.Hp, 128);
+        if (rc == RDF_OK) rc = encode_row_tiles(&c.tmap_dz64, c.dz_bf, c.cells_cap, (uint64_t)c.Hp, 64);
         if (rc != RDF_OK) return rc;
     }
     {
@@ -1243,14 +1066,10 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         RDF_KERNEL(S, rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks));
     }
     rdf_mark(S, 6, stream);
-    // lists of the gradient pass (cells in frame order, per-wave ends)
-    {
-        const int n_seg = (int)(in->max_invocations / LIST_SEG) + 1;
-        uint2* seg = reinterpret_cast<uint2*>(ws + L.list_seg);
-        RDF_KERNEL(S, rdf_list_count_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
-        RDF_KERNEL(S, rdf_list_scan_kernel<<<1, 1024, 0, stream>>>(c, seg, n_seg));
-        RDF_KERNEL(S, rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
-        RDF_KERNEL(S, rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg));
+    // lists of the gradient pass (cells in frame order, the waves that made calls); the tensor-core forward pass made them already
+    if (!c.use_tc) {
+        rc = rdf_launch_lists(in, ws, L, S, c, stream);
+        if (rc != RDF_OK) return rc;
     }
     rdf_mark(S, 7, stream);
     // gradient waves
@@ -1286,6 +1105,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         a.A = tc_lstm ? c.dg_bf : c.dz_bf; a.lda = tc_lstm ? 5 * c.Hp : c.Hp; a.Mp = tc_lstm ? 5 * c.Hp : c.Hp;
         a.Np = 2 * c.Hp; a.mode = 0; a.out = grads->dW; a.ldo = 2 * H;
         a.a_tiles = tc_rnn ? 1 : 0;
+        a.b_tiles = 1;                                              // [h_l ; h_r] of the listed cells: the operand rows
         a.bias_out = H < c.Hp ? grads->db : nullptr;                // db comes out of the same contraction
         launch_dw(a, max_cells);
         if (tc_lstm) {

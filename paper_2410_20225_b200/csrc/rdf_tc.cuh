@@ -38,7 +38,7 @@ static const int TC_LSTM_BWD_NS = 48;
 
 // tile loops (template parameter of tc_pipe)
 enum TcMode {
-    TC_RNN_FWD = 0,     // A = [h_l ; h_r] (bf16 states), B = Wp slice;           epilogue: tanh, bf16 state
+    TC_RNN_FWD = 0,     // A = [h_l ; h_r] (operand rows), B = Wp slice;           epilogue: tanh, bf16 state
     TC_RNN_BWD = 1,     // A = dz,                         B = WTp slice;          epilogue: dz of the callee cells, dE of the callee leaves
     TC_LSTM_CELL = 2,   // A = [h_l ; h_r],                B = W5p slice (5 gates x 16 units); epilogue: gates, c, h
     TC_LSTM_LEAF = 3,   // A = E_bf[tok],                  B = Wxp slice (3 gates x 16 units); epilogue: gates, c, h
@@ -298,6 +298,11 @@ template <int MODE, int STAGES>
 __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t first, uint32_t n_items) {
     static_assert(STAGES >= 3 && STAGES <= TC_MAX_STAGES, "ring depth");
     constexpr int RGN = MODE == TC_LSTM_LEAF ? 1 : 0;
+    // The rows of the A operand are consecutive rows of a matrix (the operand rows z_bf of the listed cells, or their
+    // dz rows): one 2D tile copy per stage instead of a gather.
+    constexpr bool TMA_A = MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL || MODE == TC_RNN_BWD;
+    // These modes write rows that later tile copies read (states into operand rows, dz rows).
+    constexpr bool WRITES_TILE_ROWS = MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF || MODE == TC_RNN_BWD;
     const int H = c.H, Hp = c.Hp, S = c.S, ns = tc.ns[RGN], n_chunks = tc.n_chunks[RGN];
     const int slice = blockIdx.x % tc.n_split, rg = blockIdx.x / tc.n_split, n_rg = gridDim.x / tc.n_split;
     const int tiles = (n_items + TC_M - 1) / TC_M;
@@ -318,18 +323,17 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             const uint32_t row = (uint32_t)tile * TC_M + p;
             if (row < n_items) {
                 if (MODE == TC_LSTM_DE) it = __ldcg(&c.leaf_ops[first + row]);                   // {leaf frame, token id, -, 1}
-                else if (MODE == TC_RNN_BWD || MODE == TC_LSTM_BWD) it = __ldcg(&c.cell_ops[first + row]);   // {cell, left, right, 1}
                 else if (MODE == TC_LSTM_LEAF) {
                     const uint2 lf = __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[first + row]));     // {slot, tok}
                     it.x = lf.x; it.y = lf.y;
-                } else it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + row]));  // {out, l, r, -}
+                } else it = __ldcg(&c.cell_ops[first + row]);                                    // {cell, left, right, 1}
                 it.w = 1u;
             }
             return it;
         };
-        // dz rows were written with plain stores by other blocks before the last grid barrier: order this call's
-        // tile copies (async proxy) after what that barrier acquired
-        if (MODE == TC_RNN_BWD) asm volatile("fence.proxy.async;" ::: "memory");
+        // the rows the tiles read were written with plain stores by other blocks before the last grid barrier: order
+        // this call's tile copies (async proxy) after what that barrier acquired
+        if (TMA_A) asm volatile("fence.proxy.async;" ::: "memory");
         uint4 it_next = my_tiles ? load_item(rg) : make_uint4(0u, 0u, 0u, 0u);
         for (int i = 0; i < my_tiles && ok; ++i) {
             const uint32_t T = tc.T + i, b = T & 1u;
@@ -354,14 +358,15 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
                 // the MMAs that last read this stage must have completed
                 if (g >= (uint32_t)STAGES) ok = mbar_wait(c, empty0 + 8 * s, ((g / STAGES) - 1) & 1u);
-                if (MODE == TC_RNN_BWD) {
-                    // the dz rows of the wave's cells are consecutive: one 2D tile (128 rows x 64 columns, written in the
+                if (TMA_A) {
+                    // the rows of the wave's cells are consecutive: one 2D tile (128 rows x 64 columns, written in the
                     // 128-byte swizzle by the copy engine) per stage.  Rows after the wave's last cell hold other cells'
                     // rows or old data: their accumulator rows are never read.
                     if (!ok) break;
                     if (p == 0) {
                         mbar_arrive_expect_tx(full0 + 8 * s, TC_A_STAGE);
-                        tma_load_2d(tc.a_addr + s * TC_A_STAGE, &c.tmap_dz128, kc * TC_KC, (int)(first + (uint32_t)(rg + i * n_rg) * TC_M), full0 + 8 * s);
+                        tma_load_2d(tc.a_addr + s * TC_A_STAGE, MODE == TC_RNN_BWD ? &c.tmap_dz128 : &c.tmap_z128, kc * TC_KC,
+                                    (int)(first + (uint32_t)(rg + i * n_rg) * TC_M), full0 + 8 * s);
                     } else mbar_arrive(full0 + 8 * s);
                     continue;
                 }
@@ -421,6 +426,10 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             const int e_col0 = slice * ns;
             const uint32_t child = e_col0 < Hp ? it.y : it.z;
             const int e_cc0 = e_col0 < Hp ? e_col0 : e_col0 - Hp;
+            // forward modes: where this invocation's state goes besides its own row (the operand row of its caller)
+            uint32_t zd = NO_ZDST;
+            if ((MODE == TC_RNN_FWD || MODE == TC_LSTM_CELL || MODE == TC_LSTM_LEAF) && live) zd = __ldg(&c.zdst[it.x]);
+            __nv_bfloat16* zrow = zd != NO_ZDST ? c.z_bf + (size_t)(zd >> 1) * 2 * Hp + (size_t)(zd & 1u) * Hp : nullptr;
             uint32_t child_l = LEAF_MARK, child_tok = 0, child_pos = 0;
             float4 cd0 = make_float4(0.f, 0.f, 0.f, 0.f), cd1 = cd0;
             uint4 chq[BWD_MAXU];
@@ -528,6 +537,7 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                     if (u0 == H) hb[0] = __float2bfloat16_rn(1.f);            // first pad column of the bf16 row: the constant
                     else if (u0 + 4 == H) hb[4] = __float2bfloat16_rn(1.f);   // input (see tc_leaf_rows); H is a multiple of 4
                     *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + u0) = *reinterpret_cast<const uint4*>(hb);
+                    if (zrow) *reinterpret_cast<uint4*>(zrow + u0) = *reinterpret_cast<const uint4*>(hb);
                     float* st = c.arena + (size_t)it.x * S;
 #pragma unroll
                     for (int i = 0; i < 8; i += 4)
@@ -567,6 +577,11 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                         uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
                         dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
                         dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
+                        if (zrow) {
+                            uint4* dstz = reinterpret_cast<uint4*>(zrow + col);
+                            dstz[0] = *reinterpret_cast<const uint4*>(&hb[0]);
+                            dstz[1] = *reinterpret_cast<const uint4*>(&hb[8]);
+                        }
                     } else if (MODE == TC_LSTM_DE) {
                         // embedding gradient: row tok of dE gathers the contribution of this leaf
 #pragma unroll
@@ -587,8 +602,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
             mbar_arrive(acc_empty0 + 8 * b);                   // buffer and records may be reused
         }
     }
-    // (writer side of the same ordering: the dz rows stored above are read by tile copies after the next grid barrier)
-    if (MODE == TC_RNN_BWD) asm volatile("fence.proxy.async;" ::: "memory");
+    // (writer side of the same ordering: the rows stored above are read by tile copies after the next grid barrier)
+    if (WRITES_TILE_ROWS) asm volatile("fence.proxy.async;" ::: "memory");
     tc.g += (uint32_t)(my_tiles * n_chunks);
     tc.T += (uint32_t)my_tiles;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -608,9 +623,13 @@ static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
     const int n_warps = gridDim.x * blockDim.x / 32;
     for (uint32_t i0 = warp * 4; i0 < n_items; i0 += n_warps * 4) {
         uint2 it[4];
+        __nv_bfloat16* zrow[4];                               // the half of the caller's operand row that this leaf feeds
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
+        for (int q = 0; q < 4; ++q) {
             it[q] = i0 + q < n_items ? __ldcg(reinterpret_cast<const uint2*>(&c.leaf_items[i0 + q])) : make_uint2(0u, 0u);   // {slot, tok}
+            const uint32_t zd = i0 + q < n_items ? __ldg(&c.zdst[it[q].x]) : NO_ZDST;
+            zrow[q] = zd != NO_ZDST ? c.z_bf + (size_t)(zd >> 1) * 2 * Hp + (size_t)(zd & 1u) * Hp : nullptr;
+        }
         for (int k = lane * 8; k < Hp; k += 256) {             // 8 elements per lane: 32 bytes in, 16 bytes out
             float4 v[4][2];
 #pragma unroll
@@ -630,6 +649,7 @@ static __device__ void tc_leaf_rows(const DevCtx& c, uint32_t n_items) {
                 if (k == H) hb[0].x = __float2bfloat16_rn(1.f);            // the constant input (H is a multiple of 4;
                 else if (k + 4 == H) hb[2].x = __float2bfloat16_rn(1.f);   //  k < Hp, so this is a pad column)
                 *reinterpret_cast<uint4*>(c.arena_bf + (size_t)it[q].x * Hp + k) = *reinterpret_cast<const uint4*>(hb);
+                if (zrow[q]) *reinterpret_cast<uint4*>(zrow[q] + k) = *reinterpret_cast<const uint4*>(hb);
             }
         }
     }

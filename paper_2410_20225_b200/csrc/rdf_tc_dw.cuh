@@ -52,6 +52,7 @@ struct DwArgs {
                                  // so that column of the product is sum_t A_t = the bias gradient (null: not wanted)
     int a_tiles;                 // 1: the rows of A are in list order (row = position in the list) and are read as 2D tiles
                                  //    through DevCtx::tmap_dz64; the rows after the last listed one are zero up to a multiple of 64
+    int b_tiles;                 // 1 (mode 0): B_t is row t of the operand rows z_bf (list order too), read through DevCtx::tmap_z64
 };
 
 __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant__ DevCtx c, const DwArgs a) {
@@ -122,19 +123,23 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
                     const bool mv = it.w != 0u && m_in;
                     cp_async16(a_st + off, a.A + (size_t)it.x * a.lda + (mv ? m : 0), mv);
                 }
-                const bool nv = it.w != 0u && n_in;
-                size_t src = 0;
-                if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
-                cp_async16(b_st + off, Brows + src, nv);
+                if (!a.b_tiles) {
+                    const bool nv = it.w != 0u && n_in;
+                    size_t src = 0;
+                    if (nv) src = a.mode == 0 ? (n < Hp ? (size_t)it.y * Hp + n : (size_t)it.z * Hp + (n - Hp)) : (size_t)it.y * Hp + n;
+                    cp_async16(b_st + off, Brows + src, nv);
+                }
             }
-            if (ok && a.a_tiles && threadIdx.x == 0) {
-                // A: four boxes of 64 rows x 64 columns, each written as the eight swizzled atoms of its column group
+            if (ok && (a.a_tiles || a.b_tiles) && threadIdx.x == 0) {
+                // four boxes of 64 rows x 64 columns per operand, each written as the eight swizzled atoms of its column group
                 int boxes = 0;
-                for (int g = 0; g < 4; ++g) boxes += m0 + g * 64 < a.Mp;
+                for (int g = 0; g < 4; ++g) boxes += (a.a_tiles && m0 + g * 64 < a.Mp) + (a.b_tiles && n0 + g * 64 < a.Np);
                 mbar_expect_tx(full0 + 8 * s, (uint32_t)boxes * 8192u);
-                for (int g = 0; g < 4; ++g)
-                    if (m0 + g * 64 < a.Mp)
-                        tma_load_2d(a_st + g * 8192, &c.tmap_dz64, m0 + g * 64, (int)(((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT), full0 + 8 * s);
+                const int row0 = (int)(((uint32_t)split + kc * (uint32_t)a.splits) * DW_KT);
+                for (int g = 0; g < 4; ++g) {
+                    if (a.a_tiles && m0 + g * 64 < a.Mp) tma_load_2d(a_st + g * 8192, &c.tmap_dz64, m0 + g * 64, row0, full0 + 8 * s);
+                    if (a.b_tiles && n0 + g * 64 < a.Np) tma_load_2d(b_st + g * 8192, &c.tmap_z64, n0 + g * 64, row0, full0 + 8 * s);
+                }
             }
             if (ok) cp_async_arrive(full0 + 8 * s);            // arrives when this thread's copies of the stage have landed
             if (threadIdx.x < DW_KT) s_ops[(kc + 1) & 1][threadIdx.x] = op_next;
