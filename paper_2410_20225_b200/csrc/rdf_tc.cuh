@@ -162,6 +162,23 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// the same without the wait: several loads in flight, then one tc_wait_ld()
+__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// 32 contiguous bytes in one store (a whole sector per lane: half the requests of two 16-byte stores);
+// the address is 32-byte aligned
+__device__ __forceinline__ void st_global_32(void* p, const uint4& a, const uint4& b) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w),
+                 "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
+
 // 16-byte asynchronous copy global -> shared through L2; `valid == false` writes zeros
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
     const int n = valid ? 16 : 0;
@@ -393,8 +410,8 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                     const uint32_t g = tc.g + (uint32_t)(i * n_chunks + kc), s = g % STAGES;
                     ok = mbar_wait(c, full0 + 8 * s, (g / STAGES) & 1u);
                     if (!ok) break;
-                    // the stage was written by cp.async (generic proxy) and is read by the MMA (async proxy)
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    // a stage written by cp.async (generic proxy) is read by the MMA (async proxy); tile copies are async-proxy writes
+                    if (!TMA_A) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a = tc.a_addr + s * TC_A_STAGE, bw = tc.b_addr[RGN] + kc * ns * 128;
 #pragma unroll
@@ -557,32 +574,41 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                 // warps 0-3 take the first 16-column groups, warps 4-7 the rest
                 const int groups = ns / 16, g_lo = (groups + 1) / 2;
                 const int g_begin = warp < 4 ? 0 : g_lo, g_end = warp < 4 ? g_lo : groups;
-                for (int gi = g_begin; gi < g_end; ++gi) {
-                    float v[16];
-                    tc_ld16(lane_base + (uint32_t)(gi * 16), v);
-                    if (!live) continue;
-                    const int col = slice * ns + gi * 16;                       // column of the padded N range
-                    if (MODE == TC_RNN_FWD) {
+                if (MODE == TC_RNN_FWD) {
+                    // all of this thread's accumulator groups in flight, one wait; 32-byte stores
+                    constexpr int MAXG = (TC_HP_MAX / 4 / 16 + 1) / 2;
+                    uint32_t raw[MAXG][16];
+                    // (groups past the slice read unused columns of the 128-column accumulator buffer: never looked at)
+#pragma unroll
+                    for (int q = 0; q < MAXG; ++q) tc_ld16_issue(lane_base + (uint32_t)((g_begin + q) * 16), raw[q]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < MAXG; ++q) {
+                        const int gi = g_begin + q;
+                        if (gi >= g_end || !live) continue;
+                        const int col = slice * ns + gi * 16;                   // column of the padded N range
                         // the state lives in bf16 only: every consumer reads the rounded value
                         __align__(16) __nv_bfloat16 hb[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float h = 0.f;
-                            if (col + i < H) h = tc_tanh(v[i] + sh.ep[gi * 16 + i]);
+                            if (col + i < H) h = tc_tanh(__uint_as_float(raw[q][i]) + sh.ep[gi * 16 + i]);
                             hb[i] = __float2bfloat16_rn(h);
                         }
 #pragma unroll
                         for (int i = 0; i < 16; i += 4)                         // first pad column: the constant 1 (H is a multiple of 4)
                             if (col + i == H) hb[i] = __float2bfloat16_rn(1.f);
-                        uint4* dstb = reinterpret_cast<uint4*>(c.arena_bf + (size_t)it.x * Hp + col);
-                        dstb[0] = *reinterpret_cast<const uint4*>(&hb[0]);
-                        dstb[1] = *reinterpret_cast<const uint4*>(&hb[8]);
-                        if (zrow) {
-                            uint4* dstz = reinterpret_cast<uint4*>(zrow + col);
-                            dstz[0] = *reinterpret_cast<const uint4*>(&hb[0]);
-                            dstz[1] = *reinterpret_cast<const uint4*>(&hb[8]);
-                        }
-                    } else if (MODE == TC_LSTM_DE) {
+                        const uint4 lo = *reinterpret_cast<const uint4*>(&hb[0]), hi = *reinterpret_cast<const uint4*>(&hb[8]);
+                        st_global_32(c.arena_bf + (size_t)it.x * Hp + col, lo, hi);
+                        if (zrow) st_global_32(zrow + col, lo, hi);
+                    }
+                }
+                for (int gi = g_begin; gi < g_end && MODE != TC_RNN_FWD; ++gi) {
+                    float v[16];
+                    tc_ld16(lane_base + (uint32_t)(gi * 16), v);
+                    if (!live) continue;
+                    const int col = slice * ns + gi * 16;                       // column of the padded N range
+                    if (MODE == TC_LSTM_DE) {
                         // embedding gradient: row tok of dE gathers the contribution of this leaf
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
