@@ -180,6 +180,13 @@ typedef enum { RDF_F32 = 0, RDF_BF16 = 1 } rdf_compute;
 typedef struct {
     int32_t      compute;        /* rdf_compute */
     int32_t      H, D, V, n_classes;
+    int32_t      reproducible;   /* rdf_grad with RDF_BF16 on the tensor-core path: 1 = the parameter gradients and the loss
+                                    come out bit for bit the same on every call with the same inputs (the cells are put in
+                                    an order that depends on the input alone -- by call depth, then by the argument of the
+                                    invocation -- every floating-point sum has a fixed order, and the sums that many thread
+                                    blocks contribute to are exact integer sums in fixed point).  Slower; 0 = sums by
+                                    atomics in arrival order (equal up to rounding).  Invocations of one depth that share
+                                    an argument (a node reached twice) keep their arrival order.  UNSUPPORTED elsewhere. */
     const float* E;              /* [V, D]                                          */
     const float* W;              /* TreeRNN [H, 2H]; TreeLSTM [5H, 2H] (i, f_l, f_r, o, u) */
     const float* b;              /* [H] or [5H]                                     */

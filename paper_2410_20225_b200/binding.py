@@ -75,7 +75,7 @@ class rdf_batch(C.Structure):
 
 class rdf_params(C.Structure):
     _fields_ = [("compute", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("V", C.c_int32),
-                ("n_classes", C.c_int32), ("E", C.c_void_p), ("W", C.c_void_p), ("b", C.c_void_p),
+                ("n_classes", C.c_int32), ("reproducible", C.c_int32), ("E", C.c_void_p), ("W", C.c_void_p), ("b", C.c_void_p),
                 ("W_x", C.c_void_p), ("b_x", C.c_void_p), ("W_s", C.c_void_p), ("b_s", C.c_void_p)]
 
 
@@ -475,10 +475,10 @@ class Graph:
                          max_wave_tokens=0)
 
     @staticmethod
-    def _params(dp, compute):
+    def _params(dp, compute, reproducible=False):
         g = lambda k: dp[k].data_ptr() if k in dp else None  # noqa: E731
         H = dp["W"].shape[1] // 2
-        return rdf_params(compute=compute, H=H, D=dp["E"].shape[1], V=dp["E"].shape[0],
+        return rdf_params(compute=compute, H=H, D=dp["E"].shape[1], V=dp["E"].shape[0], reproducible=int(reproducible),
                           n_classes=dp["W_s"].shape[0] if "W_s" in dp else 0, E=g("E"), W=g("W"), b=g("b"),
                           W_x=g("W_x"), b_x=g("b_x"), W_s=g("W_s"), b_s=g("b_s"))
 
@@ -507,13 +507,15 @@ class Graph:
             self.stats()
         return y, self._read_trace(tr)
 
-    def grad_trees(self, dt, dp, compute=F32, check=True, grads=None, loss=None, h_root=None, max_invocations=None):
-        """Forward + reverse pass.  Returns (loss tensor [1], h_root, {name: gradient tensor})."""
+    def grad_trees(self, dt, dp, compute=F32, check=True, grads=None, loss=None, h_root=None, max_invocations=None,
+                   reproducible=False):
+        """Forward + reverse pass.  Returns (loss tensor [1], h_root, {name: gradient tensor}).
+        reproducible (BF16 only): bit-identical results on every call with the same inputs."""
         torch = _torch()
         batch = self._batch(dt)
         if max_invocations is not None:
             batch.max_invocations = int(max_invocations)
-        params = self._params(dp, compute)
+        params = self._params(dp, compute, reproducible)
         if h_root is None:
             h_root = torch.empty(batch.B, params.H, dtype=torch.float32, device="cuda")
         if loss is None:

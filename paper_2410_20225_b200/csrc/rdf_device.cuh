@@ -169,6 +169,13 @@ struct DevCtx {
     uint4*    leaf_ops;           // {leaf frame, token id, 0, 1} in all_leaves order
     uint32_t* all_leaves;         // every leaf frame
     float*    loss_partial;       // per-block partial sums of the loss
+    // reproducible mode (tensor-core path): sums that do not depend on the order in which thread blocks get to them
+    int       repro;
+    float*    dw_partial;         // split-K partial tiles of the weight gradient [block, 256, 256] (also the per-block rows
+                                  // of the column sums), added up in block order
+    long long* dE_fix;            // [V, D] the embedding gradient in 64-bit fixed point (integer sums are exact)
+    long long* head_fix;          // [n_classes * (H + 1) + 1] dW_s, db_s and the loss in fixed point
+    uint32_t* rank_tmp;           // [frame_cap] scratch of the pass that puts the cells of a depth in argument order
     float    *dE, *dW, *db, *dW_x, *db_x, *dW_s, *db_s;
     float*    loss_out;
     // control
@@ -179,6 +186,14 @@ struct DevCtx {
 
 static const uint32_t LEAF_MARK = 0xFFFFFFFFu;
 static const uint32_t NO_ZDST = 0xFFFFFFFFu;
+
+// 64-bit fixed point, 2^-36 per unit (|sum| < 1.3e8, resolution 1.5e-11): integer additions commute exactly
+#define RDF_FIX_SCALE 68719476736.0f
+__device__ __forceinline__ long long to_fix(float v) { return __float2ll_rn(v * RDF_FIX_SCALE); }
+__device__ __forceinline__ void fix_add(long long* p, long long v) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
+}
+__device__ __forceinline__ float from_fix(long long v) { return (float)((double)v * (1.0 / (double)RDF_FIX_SCALE)); }
 
 // ---------------------------------------------------------------- utilities
 __device__ __forceinline__ void set_status(const DevCtx& c, int code) { atomicCAS(&c.ctl->status, 0, code); }

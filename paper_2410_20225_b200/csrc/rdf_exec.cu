@@ -805,6 +805,11 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.leaf_ops = P.take<uint4>(tcl ? gf : 0);
     L.all_leaves = P.take<uint32_t>(g->has_lstm ? lf : gf);
     L.loss_partial = P.take<float>(want_grad ? 4096 : 0);
+    L.repro = want_grad && L.use_tc && params->reproducible ? 1 : 0;
+    L.dw_partial = P.take<float>(L.repro ? (size_t)DW_BLOCKS_MAX * 65536 : 0);
+    L.de_fix = P.take<long long>(L.repro ? (size_t)params->V * params->D : 0);
+    L.head_fix = P.take<long long>(L.repro ? (size_t)params->n_classes * (H + 1) + 1 : 0);
+    L.rank_tmp = P.take<uint32_t>(L.repro ? (size_t)2 * L.frame_cap : 0);      // 64-bit keys of the cells or of the leaves
     L.total = (P.off + 255) & ~(size_t)255;
     return RDF_OK;
 }
@@ -908,6 +913,11 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.leaf_ops = L.use_tc && g->has_lstm && L.want_grad ? reinterpret_cast<uint4*>(ws + L.leaf_ops) : nullptr;
     c.all_leaves = reinterpret_cast<uint32_t*>(ws + L.all_leaves);
     c.loss_partial = reinterpret_cast<float*>(ws + L.loss_partial);
+    c.repro = L.repro;
+    c.dw_partial = L.repro ? reinterpret_cast<float*>(ws + L.dw_partial) : nullptr;
+    c.dE_fix = L.repro ? reinterpret_cast<long long*>(ws + L.de_fix) : nullptr;
+    c.head_fix = L.repro ? reinterpret_cast<long long*>(ws + L.head_fix) : nullptr;
+    c.rank_tmp = L.repro ? reinterpret_cast<uint32_t*>(ws + L.rank_tmp) : nullptr;
     c.loss_out = out->loss;
     c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
     c.wave_limit = L.wave_cap ? L.wave_cap : 1u << 24;
@@ -1025,6 +1035,14 @@ int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* 
     RDF_KERNEL(S, rdf_list_fill_kernel<<<n_seg, 256, 0, stream>>>(c, seg));
     RDF_KERNEL(S, rdf_list_ends_kernel<<<2 * S->grid, 256, 0, stream>>>(c, seg));
     RDF_KERNEL(S, rdf_wave_compact_kernel<<<1, 1024, 0, stream>>>(c));
+    if (c.repro) {                                  // the cells of every depth in argument order
+        for (int leaves = c.lstm ? 1 : 0; leaves >= 0; --leaves) {     // (the leaves first: the cells' positions are used afterwards)
+            RDF_KERNEL(S, rdf_canon_keys_kernel<<<2 * S->grid, 256, 0, stream>>>(c, leaves));
+            RDF_KERNEL(S, rdf_canon_rank_kernel<<<4 * S->grid, 256, 0, stream>>>(c, leaves));
+            RDF_KERNEL(S, rdf_canon_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c, leaves));
+        }
+    }
+    if (c.zdst) RDF_KERNEL(S, rdf_list_zdst_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
     CUDA_OK(cudaGetLastError());
     return RDF_OK;
 }

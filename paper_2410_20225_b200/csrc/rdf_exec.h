@@ -40,6 +40,7 @@ __device__ __forceinline__ void gemm_tile_step(const GemmSmem& sm, int tx, int t
 static const int THIN_RESIDENT_MAX_H = 384;
 inline size_t thin_resident_bytes(int lstm, int H) { return !lstm && H <= THIN_RESIDENT_MAX_H ? (size_t)128 * H : 0; }
 
+static const int DW_BLOCKS_MAX = 256;        // blocks of the tensor-core weight-gradient pass (reproducible mode: one partial tile each)
 static const int LIST_SEG = 2048;            // frames per segment of the list kernels (256 threads x 8)
 
 // ---- host state
@@ -73,9 +74,9 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, children, pair_slots, port_val, arrived, table, cell_items,
-        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, total;
+        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, dw_partial, de_fix, head_fix, rank_tmp, total;
     uint32_t qcap, frame_cap, work_cap, wave_cap, cells_cap;
-    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad;
+    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad, repro;
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes, pair_bytes;
 };

@@ -422,6 +422,114 @@ __global__ void __launch_bounds__(256) rdf_loss_final_kernel(const DevCtx c, int
     }
 }
 
+// ---- reproducible mode: the loss head with sums that do not depend on how the invocations are spread over the blocks
+// One warp per invocation.  Its logits are dot products in a fixed lane order (the value of an invocation is the same
+// whichever warp computes it); the loss, dW_s and db_s are sums over all invocations and are accumulated as 64-bit
+// fixed-point integers, per thread and then with integer atomics: exact, hence independent of the order.
+// States: the bf16 h rows of arena_bf (tensor-core path).
+__global__ void __launch_bounds__(256) rdf_loss_heads_exact_kernel(const DevCtx c) {
+    if (c.ctl->status != 0) return;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
+    const int lane = threadIdx.x % 32, H = c.H, Hp = c.Hp, C = c.n_classes;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, n_warps = gridDim.x * blockDim.x / 32;
+    constexpr int MAXJ = TC_HP_MAX / 32;                               // hidden units per lane: j = lane + 32 q
+    long long acc[MAX_CLASSES][MAXJ];
+#pragma unroll
+    for (int k = 0; k < MAX_CLASSES; ++k)
+#pragma unroll
+        for (int q = 0; q < MAXJ; ++q) acc[k][q] = 0;
+    long long loss_acc = 0, dbs_acc = 0;                               // lane 0: the loss; lane k < C: db_s[k]
+    for (uint32_t f = B + warp; f < F; f += n_warps) {
+        float x[MAXJ], z[MAX_CLASSES];
+#pragma unroll
+        for (int q = 0; q < MAXJ; ++q) {
+            const int j = lane + 32 * q;
+            x[q] = j < H ? __bfloat162float(c.arena_bf[(size_t)f * Hp + j]) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) {
+            float t = 0.f;
+            if (k < C) {
+#pragma unroll
+                for (int q = 0; q < MAXJ; ++q) {
+                    const int j = lane + 32 * q;
+                    if (j < H) t = fmaf(__ldg(&c.W_s[k * H + j]), x[q], t);
+                }
+                for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+                t += __ldg(&c.b_s[k]);
+            }
+            z[k] = t;
+        }
+        const int lab = __ldg(&c.label[(int)c.frames[f].arg]);
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) m = fmaxf(m, z[k]);
+        float sum = 0.f, zl = 0.f;
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k)
+            if (k < C) {
+                sum += expf(z[k] - m);
+                if (k == lab) zl = z[k];
+            }
+        float d[MAX_CLASSES];
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) d[k] = k < C ? expf(z[k] - m) / sum - (k == lab ? 1.f : 0.f) : 0.f;
+        if (lane == 0) {
+            loss_acc += to_fix(logf(sum) + m - zl);
+            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8) = make_float4(d[0], d[1], d[2], d[3]);
+            *reinterpret_cast<float4*>(c.dlog + (size_t)f * 8 + 4) = make_float4(d[4], d[5], d[6], d[7]);
+        }
+#pragma unroll
+        for (int k = 0; k < MAX_CLASSES; ++k) {
+            if (k >= C) continue;
+            if (lane == k) dbs_acc += to_fix(d[k]);
+#pragma unroll
+            for (int q = 0; q < MAXJ; ++q) acc[k][q] += to_fix(d[k] * x[q]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < MAX_CLASSES; ++k) {
+        if (k >= C) continue;
+#pragma unroll
+        for (int q = 0; q < MAXJ; ++q) {
+            const int j = lane + 32 * q;
+            if (j < H && acc[k][q] != 0) fix_add(&c.head_fix[k * H + j], acc[k][q]);
+        }
+    }
+    if (lane < C && dbs_acc != 0) fix_add(&c.head_fix[C * H + lane], dbs_acc);
+    if (lane == 0 && loss_acc != 0) fix_add(&c.head_fix[C * (H + 1)], loss_acc);
+}
+
+// the fixed-point sums as fp32: dW_s, db_s, the loss
+__global__ void __launch_bounds__(256) rdf_head_convert_kernel(const DevCtx c) {
+    const int C = c.n_classes, H = c.H, n = C * (H + 1) + 1;
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n) return;
+    if (q == n - 1) {
+        // (this thread also closes the forward pass: what the gradient kernel checks before it starts)
+        const float loss = from_fix(c.head_fix[q]);
+        c.ctl->loss = loss;
+        if (c.loss_out) *c.loss_out = loss;
+        c.ctl->forward_status = c.ctl->status;
+        return;
+    }
+    if (c.ctl->status != 0) return;
+    const float v = from_fix(c.head_fix[q]);
+    if (q < C * H) c.dW_s[q] = v;
+    else c.db_s[q - C * H] = v;
+}
+
+// the embedding gradient from its fixed-point sums
+__global__ void __launch_bounds__(256) rdf_de_convert_kernel(const DevCtx c) {
+    if (c.ctl->status != 0) return;
+    const size_t total = (size_t)c.V * c.D / 2;                        // two elements per thread step (D is a multiple of 4)
+    for (size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (size_t)gridDim.x * blockDim.x) {
+        const longlong2 v = *reinterpret_cast<const longlong2*>(c.dE_fix + 2 * q);
+        *reinterpret_cast<float2*>(c.dE + 2 * q) = make_float2(from_fix(v.x), from_fix(v.y));
+    }
+}
+
 // ----------------------------------------------------------- backward waves
 // What a thread needs to know about an invocation before it touches its rows; all of it is left
 // behind by the forward pass and the loss head, so it can be fetched one step ahead.
@@ -478,7 +586,12 @@ __device__ __forceinline__ void backward_frames_tc(const DevCtx& c, uint32_t t0,
                         dh[6] = fmaf(w.z, dl[k], dh[6]); dh[7] = fmaf(w.w, dl[k], dh[7]);
                     }
                 }
-            if (leaf) {
+            if (leaf && c.dE_fix) {                              // reproducible mode: exact integer sums
+                long long* de = c.dE_fix + (size_t)tok * c.D + j;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (j + i < H) fix_add(de + i, to_fix(dh[i]));
+            } else if (leaf) {
                 float* de = c.dE + (size_t)tok * c.D + j;
                 if (j < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(dh[0], dh[1], dh[2], dh[3]));
                 if (j + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(dh[4], dh[5], dh[6], dh[7]));
@@ -940,6 +1053,31 @@ __global__ void __launch_bounds__(256) rdf_colsum_kernel(const int32_t* status, 
     }
 }
 
+// reproducible mode: one row of partial sums per block, the rows added up in block order
+template <typename T>
+__global__ void __launch_bounds__(256) rdf_colsum_partial_kernel(const int32_t* status, const uint32_t* list, const uint32_t* count,
+                                                                 const T* A, int lda, int M, int H, int Hb, float* partial) {
+    if (*status != 0) return;
+    const uint32_t n = *count;
+    const uint32_t per = (n + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = min(n, blockIdx.x * per), t1 = min(n, t0 + per);
+    for (int j = threadIdx.x; j < M; j += blockDim.x) {
+        const int col = (j / H) * Hb + j % H;
+        float s = 0.f;
+#pragma unroll 8
+        for (uint32_t i = t0; i < t1; ++i) s += as_float(A[(size_t)(list ? list[i] : i) * lda + col]);
+        partial[(size_t)blockIdx.x * M + j] = s;
+    }
+}
+__global__ void __launch_bounds__(256) rdf_rows_reduce_kernel(const int32_t* status, const float* partial, int n_rows, int n, float* out) {
+    if (*status != 0) return;
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n) return;
+    float t = 0.f;
+    for (int r = 0; r < n_rows; ++r) t += partial[(size_t)r * n + q];
+    out[q] = t;
+}
+
 // TreeLSTM: dE[tok_t] += W_x^T dg_t for every leaf t (dg_t = the 3H gate gradients)
 __global__ void __launch_bounds__(256) rdf_de_lstm_kernel(const DevCtx c, int tiles_n) {
     if (c.ctl->status != 0) return;                    // an earlier kernel of this call failed: its lists and rows are not to be trusted
@@ -1017,6 +1155,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     Layout L;
     rc = rdf_make_layout(g, in, params, 1, L);
     if (rc != RDF_OK) return rc;
+    if (params->reproducible && !L.repro) return RDF_ERR_UNSUPPORTED;     // (only the tensor-core path has the ordered sums)
     if (workspace_bytes < L.total) return RDF_ERR_WORKSPACE_TOO_SMALL;
     ExecState* S = rdf_state_of(g);
     rc = rdf_prepare_device(g, S);
@@ -1032,7 +1171,10 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     const int H = params->H, D = params->D;
     const int MW = lstm ? 5 * H : H;          // rows of W
     // gradients are sums: start from zero
-    CUDA_OK(cudaMemsetAsync(grads->dE, 0, (size_t)params->V * D * sizeof(float), stream));
+    if (c.repro) {                         // the fixed-point sums start from zero; dE itself is written whole at the end
+        CUDA_OK(cudaMemsetAsync(c.dE_fix, 0, (size_t)params->V * D * sizeof(long long), stream));
+        CUDA_OK(cudaMemsetAsync(c.head_fix, 0, ((size_t)params->n_classes * (H + 1) + 1) * sizeof(long long), stream));
+    } else CUDA_OK(cudaMemsetAsync(grads->dE, 0, (size_t)params->V * D * sizeof(float), stream));
     CUDA_OK(cudaMemsetAsync(grads->dW, 0, (size_t)MW * 2 * H * sizeof(float), stream));
     CUDA_OK(cudaMemsetAsync(grads->db, 0, (size_t)MW * sizeof(float), stream));
     CUDA_OK(cudaMemsetAsync(grads->dW_s, 0, (size_t)params->n_classes * H * sizeof(float), stream));
@@ -1055,7 +1197,10 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         const int fr = std::max(1, std::min(LH_MAX_ROWS, LH_SLAB_BYTES / rowbytes));
         const int smem = 2 * fr * rowbytes + params->n_classes * H * (int)sizeof(float);
         const int loss_blocks = std::min(4096, 2 * S->grid);
-        if (c.use_tc) {                    // bf16 states (TreeRNN and TreeLSTM): the h rows of arena_bf
+        if (c.repro) {
+            RDF_KERNEL(S, rdf_loss_heads_exact_kernel<<<8 * S->grid, 256, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_head_convert_kernel<<<(params->n_classes * (H + 1) + 1 + 255) / 256, 256, 0, stream>>>(c));
+        } else if (c.use_tc) {             // bf16 states (TreeRNN and TreeLSTM): the h rows of arena_bf
             const int smem_mma = 2 * LM_ROWS * (c.Hp * 2 + 16);
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mma));
             RDF_KERNEL(S, rdf_loss_heads_mma_kernel<<<loss_blocks, 256, smem_mma, stream>>>(c));
@@ -1063,7 +1208,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             CUDA_OK(cudaFuncSetAttribute(rdf_loss_heads_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             RDF_KERNEL(S, rdf_loss_heads_kernel<false><<<loss_blocks, 256, smem, stream>>>(c, fr, rowbytes));
         }
-        RDF_KERNEL(S, rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks));
+        if (!c.repro) RDF_KERNEL(S, rdf_loss_final_kernel<<<1, 256, 0, stream>>>(c, loss_blocks));
     }
     rdf_mark(S, 6, stream);
     // lists of the gradient pass (cells in frame order, the waves that made calls); the tensor-core forward pass made them already
@@ -1097,8 +1242,10 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             a.tiles_n = (a.Np + DW_TILE - 1) / DW_TILE;
             a.n_tiles = ((a.Mp + DW_TILE - 1) / DW_TILE) * a.tiles_n;
             const long long stages = (max_items + DW_KT - 1) / DW_KT;
-            a.splits = (int)std::max<long long>(1, std::min<long long>(S->grid / a.n_tiles, stages));
+            a.splits = (int)std::max<long long>(1, std::min<long long>(std::min(S->grid, DW_BLOCKS_MAX) / a.n_tiles, stages));
+            a.partial = c.repro ? c.dw_partial : nullptr;
             RDF_KERNEL(S, rdf_dw_tc_kernel<<<a.n_tiles * a.splits, 256, DW_SMEM_BYTES, stream>>>(c, a));
+            if (c.repro) RDF_KERNEL(S, rdf_dw_reduce_kernel<<<2 * S->grid, 256, 0, stream>>>(c, a));   // the partial tiles, added up in split order
         };
         DwArgs a{};
         a.ops = c.cell_ops; a.count = &c.ctl->all_cells;
@@ -1125,6 +1272,20 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
     }
     rdf_mark(S, 9, stream);
     if (c.use_tc && H < c.Hp) {}        // (column H of the dW / dW_x contractions)
+    else if (c.repro) {
+        // column sums in two steps: a row of partial sums per block (in the buffer the weight gradient is done with), then
+        // the rows added up in block order.  TreeRNN: dz rows are in all_cells order; TreeLSTM: bf16 gate-gradient rows.
+        const int cs_blocks = std::min(8 * S->grid, (int)((size_t)DW_BLOCKS_MAX * 65536 / (5 * (size_t)H)));
+        auto colsum = [&](const uint32_t* list, const uint32_t* count, const __nv_bfloat16* A, int lda_, int M, float* out_) {
+            RDF_KERNEL(S, rdf_colsum_partial_kernel<__nv_bfloat16><<<cs_blocks, 256, 0, stream>>>(&c.ctl->status, list, count, A, lda_, M, H, c.Hp, c.dw_partial));
+            RDF_KERNEL(S, rdf_rows_reduce_kernel<<<(M + 255) / 256, 256, 0, stream>>>(&c.ctl->status, c.dw_partial, cs_blocks, M, out_));
+        };
+        if (tc_rnn) colsum(nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, grads->db);
+        else {
+            colsum(c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, grads->db);
+            colsum(c.all_leaves, &c.ctl->all_leaves, c.dg_bf, 5 * c.Hp, 3 * H, grads->db_x);
+        }
+    }
     else if (tc_rnn) RDF_KERNEL(S, rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, nullptr, &c.ctl->all_cells, c.dz_bf, c.Hp, H, H, c.Hp, grads->db));   // dz rows are in all_cells order
     else if (tc_lstm) {                 // the gate gradients exist as bf16 operand rows only
         RDF_KERNEL(S, rdf_colsum_kernel<__nv_bfloat16><<<8 * S->grid, 256, 0, stream>>>(&c.ctl->status, c.all_cells, &c.ctl->all_cells, c.dg_bf, 5 * c.Hp, 5 * H, H, c.Hp, grads->db));
@@ -1140,6 +1301,7 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         RDF_KERNEL(S, rdf_de_tc_kernel<<<(S->grid / n_split) * n_split, TC_THREADS, de_smem, stream>>>(c));
     } else if (lstm) RDF_KERNEL(S, rdf_de_lstm_kernel<<<4 * S->grid, 256, 0, stream>>>(c, (D + TN - 1) / TN));
     // (TreeRNN: the leaves added their dh to dE during the gradient waves)
+    if (c.repro) RDF_KERNEL(S, rdf_de_convert_kernel<<<8 * S->grid, 256, 0, stream>>>(c));
     rdf_mark(S, 11, stream);
     CUDA_OK(cudaGetLastError());
     return RDF_OK;

@@ -167,17 +167,84 @@ __global__ void __launch_bounds__(256) rdf_list_ends_kernel(const DevCtx c, cons
                 *reinterpret_cast<uint4*>(c.z_bf + (size_t)(n + q / per_row) * 2 * c.Hp + (q % per_row) * 8) = make_uint4(0u, 0u, 0u, 0u);
         }
     }
-    // Where an invocation's state goes besides its own row: the operand row of the cell that called it
-    // (row = position of the caller in the cell list, half = the operand port that the call's Return_i feeds).
-    if (c.zdst) {
-        for (uint32_t f = B + blockIdx.x * blockDim.x + threadIdx.x; f < F; f += gridDim.x * blockDim.x) {
-            const Frame fr = c.frames[f];
-            const LabelInfo& L = c.labels[fr.label & FRAME_LABEL_MASK];
-            uint32_t z = NO_ZDST;
-            if (fr.parent >= B && fr.parent < F && L.k_kind == K_PORT && c.match[L.k_node].kind != MATCH_INT &&
-                c.op_l[fr.parent] != LEAF_MARK)
-                z = c.cell_pos[fr.parent] * 2u + (uint32_t)L.k_port;
-            c.zdst[f] = z;
+}
+
+// Where an invocation's state goes besides its own row: the operand row of the cell that called it
+// (row = position of the caller in the cell list, half = the operand port that the call's Return_i feeds).
+__global__ void __launch_bounds__(256) rdf_list_zdst_kernel(const DevCtx c) {
+    if (c.ctl->status != 0 || !c.zdst) return;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
+    for (uint32_t f = B + blockIdx.x * blockDim.x + threadIdx.x; f < F; f += gridDim.x * blockDim.x) {
+        const Frame fr = c.frames[f];
+        const LabelInfo& L = c.labels[fr.label & FRAME_LABEL_MASK];
+        uint32_t z = NO_ZDST;
+        if (fr.parent >= B && fr.parent < F && L.k_kind == K_PORT && c.match[L.k_node].kind != MATCH_INT &&
+            c.op_l[fr.parent] != LEAF_MARK)
+            z = c.cell_pos[fr.parent] * 2u + (uint32_t)L.k_port;
+        c.zdst[f] = z;
+    }
+}
+
+// ---- reproducible mode: the cells of every depth in an order that depends on the input alone
+// Frame ids are handed out in the order the scheduler's warps reach the frame counter, so the position of a cell
+// among the cells of its depth differs from run to run, and with it the order of every sum over the cells.  Here the
+// cells of a depth are re-ordered by the argument of their invocation (for the tree networks: the node index, which is
+// unique), ties by their previous position.  A cell's rank is counted directly (every cell against the cells of its
+// depth: about the square of the widest depth in comparisons, which is what this mode pays for).
+// (leaves != 0: the same for the list of leaves -- the TreeLSTM's leaf projection sums over it; the leaves of a
+// depth are the frames of the depth that are not cells, so their range in the leaf list follows from the two others)
+__global__ void __launch_bounds__(256) rdf_canon_keys_kernel(const DevCtx c, int leaves) {
+    if (c.ctl->status != 0) return;
+    long long* key = reinterpret_cast<long long*>(c.rank_tmp);
+    const uint32_t* list = leaves ? c.all_leaves : c.all_cells;
+    const uint32_t n = leaves ? min(c.ctl->all_leaves, c.frame_cap) : min(c.ctl->all_cells, c.cells_cap);
+    for (uint32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n; p += gridDim.x * blockDim.x)
+        key[p] = c.frames[list[p]].arg;
+}
+
+__global__ void __launch_bounds__(256) rdf_canon_rank_kernel(const DevCtx c, int leaves) {
+    if (c.ctl->status != 0) return;
+    const long long* key = reinterpret_cast<const long long*>(c.rank_tmp);
+    const uint32_t* list = leaves ? c.all_leaves : c.all_cells;
+    const uint32_t n = leaves ? min(c.ctl->all_leaves, c.frame_cap) : min(c.ctl->all_cells, c.cells_cap);
+    const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap), B = (uint32_t)c.B;
+    // first position of depth k in the list
+    auto start_of = [&](uint32_t k) { const uint4 m = c.wave_marks[k]; return leaves ? m.x - B - m.z : m.z; };
+    auto end_of = [&](uint32_t k) { const uint4 m = c.wave_marks[k]; return leaves ? m.y - B - m.w : m.w; };
+    for (uint32_t p0 = blockIdx.x * blockDim.x; p0 < n; p0 += gridDim.x * blockDim.x) {
+        const uint32_t p = p0 + threadIdx.x;
+        if (p >= n) continue;
+        // the depth that holds position p: the last one that starts at or before p
+        uint32_t lo = 0, hi = nw;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) / 2;
+            if (start_of(mid) <= p) lo = mid; else hi = mid;
+        }
+        const uint32_t c0 = start_of(lo), c1 = min(end_of(lo), n);
+        const long long mine = key[p];
+        uint32_t below = 0;
+        for (uint32_t q = c0; q < c1; ++q) {
+            const long long k = key[q];
+            below += (k < mine) || (k == mine && q < p);
+        }
+        c.cell_pos[list[p]] = c0 + below;
+    }
+}
+
+// the lists rewritten in the new order (by frame: a cell or leaf knows its new position)
+__global__ void __launch_bounds__(256) rdf_canon_scatter_kernel(const DevCtx c, int leaves) {
+    if (c.ctl->status != 0) return;
+    const uint32_t F = min(c.ctl->frame_count.v, c.frame_cap), B = (uint32_t)c.B;
+    for (uint32_t f = B + blockIdx.x * blockDim.x + threadIdx.x; f < F; f += gridDim.x * blockDim.x) {
+        const uint32_t l = c.op_l[f];
+        if ((l == LEAF_MARK) != (leaves != 0)) continue;
+        const uint32_t np = c.cell_pos[f];
+        if (leaves) {
+            c.all_leaves[np] = f;
+            if (c.leaf_ops) c.leaf_ops[np] = make_uint4(f, c.op_r[f], 0u, 1u);
+        } else {
+            c.all_cells[np] = f;
+            if (c.cell_ops) c.cell_ops[np] = make_uint4(f, l, c.op_r[f], 1u);
         }
     }
 }

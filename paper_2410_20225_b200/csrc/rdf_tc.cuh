@@ -487,9 +487,16 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                         v[6] = fmaf(w1.z, dl[k], v[6]); v[7] = fmaf(w1.w, dl[k], v[7]);
                     }
                     if (child_l == LEAF_MARK) {
-                        float* de = c.dE + (size_t)child_tok * c.D + cc;
-                        if (cc < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(v[0], v[1], v[2], v[3]));
-                        if (cc + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(v[4], v[5], v[6], v[7]));
+                        if (c.dE_fix) {                               // reproducible mode: exact integer sums
+                            long long* de = c.dE_fix + (size_t)child_tok * c.D + cc;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (cc + i < H) fix_add(de + i, to_fix(v[i]));
+                        } else {
+                            float* de = c.dE + (size_t)child_tok * c.D + cc;
+                            if (cc < H) atomicAdd(reinterpret_cast<float4*>(de), make_float4(v[0], v[1], v[2], v[3]));
+                            if (cc + 4 < H) atomicAdd(reinterpret_cast<float4*>(de + 4), make_float4(v[4], v[5], v[6], v[7]));
+                        }
                     } else {
                         __align__(16) __nv_bfloat162 pk[4];
                         const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&chq[q]);
@@ -612,7 +619,10 @@ __device__ void tc_pipe(const DevCtx& c, TcState& tc, TcShared& sh, uint32_t fir
                         // embedding gradient: row tok of dE gathers the contribution of this leaf
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
-                            if (col + i < c.D) atomicAdd(&c.dE[(size_t)it.y * c.D + col + i], v[i]);
+                            if (col + i < c.D) {
+                                if (c.dE_fix) fix_add(&c.dE_fix[(size_t)it.y * c.D + col + i], to_fix(v[i]));
+                                else atomicAdd(&c.dE[(size_t)it.y * c.D + col + i], v[i]);
+                            }
                     } else {
                         // operand gradients: columns [0, Hp) belong to the left callee frame, [Hp, 2Hp) to the right
                         const uint32_t child = col < Hp ? it.y : it.z;

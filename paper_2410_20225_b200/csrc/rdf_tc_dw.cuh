@@ -7,7 +7,8 @@
 // swizzle.  Each thread block owns one 256 x 256 tile of dW (two 128-row
 // accumulators: all 512 columns of tensor memory) and every splits-th stage
 // of the cell list (split-K); partial tiles are added to dW with vector
-// atomics.  The large tile is what keeps the gather small: an operand row is
+// atomics, or (reproducible mode) left in a buffer per block and added up in
+// split order by a second kernel.  The large tile is what keeps the gather small: an operand row is
 // fetched once per tile that needs it, and the gather (16-byte cp.async
 // pieces) is what bounds the kernel.  bf16 TreeRNN: the dz rows are stored in
 // list order, so that operand arrives as 2D tile copies instead, and column H
@@ -53,6 +54,8 @@ struct DwArgs {
     int a_tiles;                 // 1: the rows of A are in list order (row = position in the list) and are read as 2D tiles
                                  //    through DevCtx::tmap_dz64; the rows after the last listed one are zero up to a multiple of 64
     int b_tiles;                 // 1 (mode 0): B_t is row t of the operand rows z_bf (list order too), read through DevCtx::tmap_z64
+    float* partial;              // reproducible mode: [n_tiles * splits][256][256], the block's partial tile (block = split *
+                                 // n_tiles + tile) instead of atomics on `out`; null otherwise
 };
 
 __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant__ DevCtx c, const DwArgs a) {
@@ -173,7 +176,20 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
     // ---- everybody: the accumulators are complete when the last commit has arrived
     ok = mbar_wait(c, done0, 0u);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
+    if (ok && a.partial) {
+        float* mine = a.partial + (size_t)blockIdx.x * (DW_TILE * DW_TILE);
+        for (int h = 0; h < 2; ++h) {
+            const int r = h * 128 + (warp & 3) * 32 + lane;                // row of the tile
+            for (int gi = 0; gi < 8; ++gi) {
+                float v[16];
+                const int cl = (warp >> 2) * 128 + gi * 16;
+                tc_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(h * DW_TILE + cl), v);
+                float4* dst = reinterpret_cast<float4*>(mine + (size_t)r * DW_TILE + cl);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+        }
+    } else if (ok) {
         const int n_limit = a.mode == 0 ? H : c.D;
         for (int h = 0; h < 2; ++h) {
             const int m = m0 + h * 128 + (warp & 3) * 32 + lane;
@@ -199,4 +215,31 @@ __global__ void __launch_bounds__(256, 1) rdf_dw_tc_kernel(const __grid_constant
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+// Reproducible mode: out = the partial tiles of every split added up in split order (the blocks that had no stage wrote
+// nothing and are not read); rows and columns of the padded tile go to their places in the gradient, column H of the
+// left half to the bias gradient.  One thread per four columns of a tile row.
+__global__ void __launch_bounds__(256) rdf_dw_reduce_kernel(const __grid_constant__ DevCtx c, const DwArgs a) {
+    if (c.ctl->status != 0) return;
+    const uint32_t n_stages = (*a.count + DW_KT - 1) / DW_KT;
+    const int splits = (int)min((uint32_t)a.splits, n_stages);
+    const int H = c.H, Hp = c.Hp, n_limit = a.mode == 0 ? H : c.D;
+    const int per_tile = DW_TILE * DW_TILE / 4;
+    for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < a.n_tiles * per_tile; q += gridDim.x * blockDim.x) {
+        const int tile = q / per_tile, e = q % per_tile, r = e / (DW_TILE / 4), c4 = (e % (DW_TILE / 4)) * 4;
+        const int m = (tile / a.tiles_n) * DW_TILE + r, n = (tile % a.tiles_n) * DW_TILE + c4;
+        const int mj = m % Hp, row = (m / Hp) * H + mj;              // gate block, unit
+        if (m >= a.Mp || mj >= H || n >= a.Np) continue;
+        const int k = n < Hp ? n : n - Hp;
+        const bool bias = a.bias_out && n == H;
+        if (k >= n_limit && !bias) continue;
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp = 0; sp < splits; ++sp) {
+            const float4 v = *reinterpret_cast<const float4*>(a.partial + ((size_t)sp * a.n_tiles + tile) * (DW_TILE * DW_TILE) + (size_t)r * DW_TILE + c4);
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        if (k < n_limit) *reinterpret_cast<float4*>(&a.out[(size_t)row * a.ldo + (n < Hp ? k : H + k)]) = t;
+        else a.bias_out[row] = t.x;
+    }
 }

@@ -378,6 +378,58 @@ def test_treelstm_config4_full_size():
     assert all(relerr(full[k], halves[k]) <= 1e-4 for k in full)
 
 
+@pytest.mark.parametrize("cell,H", [("rnn", 300), ("rnn", 64), ("lstm", 300), ("lstm", 64)])
+def test_bf16_gradient_sums_run_to_run(cell, H):
+    """Parameter gradients are sums over every invocation.  By default they are added up with floating-point atomics
+    in arrival order: two runs on the same input agree up to the rounding of those sums (bounded here: 1e-5 of the
+    largest entry; the tolerance against the oracle is 2e-2), and the root states -- one fixed expression per
+    invocation -- agree bit for bit.
+    With `reproducible` the cells are put in an order that depends on the input alone (call depth, then node
+    index), the floating-point sums run in a fixed order over that order (split-K partial tiles and per-block
+    partials added up in sequence) and the sums that many blocks contribute to are exact integer sums in fixed point:
+    loss and all gradients are bit-identical from call to call, also from a fresh graph and workspace, and still
+    within the tolerance of the oracle.  H = 300 takes the bias gradients out of the weight-gradient contraction,
+    H = 64 from column sums."""
+    cfg = workloads.config(3 if cell == "rnn" else 4, B=700, V=900, H=H)
+    tb, p = cfg["trees"], cfg["params"]
+    dt, dp = rdf.Graph.device_trees(tb), rdf.Graph.device_params(p)
+    for reproducible in (False, True):
+        runs = []
+        g = graph(cell, with_loss=True)
+        for k in range(3):
+            if k == 2:
+                g = graph(cell, with_loss=True)
+            loss, h, grads = g.grad_trees(dt, dp, rdf.BF16, reproducible=reproducible)
+            runs.append((loss.clone(), h.clone(), {n: v.clone() for n, v in grads.items()}))
+        spread = {}
+        for loss, h, grads in runs[1:]:
+            assert torch.equal(h, runs[0][1])
+            if reproducible:
+                assert torch.equal(loss, runs[0][0])
+                for n in grads:
+                    assert torch.equal(grads[n], runs[0][2][n]), n
+            else:
+                assert abs(loss.item() - runs[0][0].item()) <= 1e-6 * abs(runs[0][0].item())
+                for n in grads:
+                    ref = runs[0][2][n]
+                    spread[n] = max(spread.get(n, 0.0), float((grads[n] - ref).abs().max() / ref.abs().max().clamp_min(1e-30)))
+        if not reproducible:
+            print("run-to-run spread:", spread)
+            assert all(v <= 1e-5 for v in spread.values()), spread
+    # the reproducible results against the oracle
+    want_loss, G, roots = direct.loss_and_grad_pool(tb, p, cell, workers=WORKERS)
+    loss, h, grads = runs[0]
+    tol = TOL[rdf.BF16]
+    assert relerr(h.cpu().numpy(), roots) <= tol and abs(loss.item() - want_loss) <= tol * abs(want_loss)
+    errs = {k: relerr(grads[k].cpu().numpy(), G[k]) for k in G}
+    assert all(e <= tol for e in errs.values()), errs
+    check_embedding_rows(tb, grads["E"].cpu().numpy(), G["E"], tol)
+    # reproducible sums exist on the tensor-core path only
+    with pytest.raises(rdf.RdfError) as e:
+        graph(cell, with_loss=True).grad_trees(dt, dp, rdf.F32, reproducible=True)
+    assert e.value.code == -11
+
+
 def test_depth_stress_config5_forward_sampled():
     """Full config 5 forward (chains of depth 4096, perfect trees of 2^16 leaves); the oracle
     evaluates one chain and one perfect tree."""

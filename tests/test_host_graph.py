@@ -32,6 +32,7 @@ def test_library_exports_every_declared_symbol():
 def test_struct_layouts_match_the_header():
     assert C.sizeof(bd.rdf_expr) == 24 and C.sizeof(bd.rdf_trace_rec) == 32 and bd.TRACE_DTYPE.itemsize == 32
     assert C.sizeof(bd.rdf_batch) == 10 * 8 and C.sizeof(bd.rdf_node) == 32 and C.sizeof(bd.rdf_edge) == 20
+    assert C.sizeof(bd.rdf_params) == 6 * 4 + 7 * 8 and bd.rdf_params.E.offset == 24
 
 
 # ----------------------------------------------------------------- errors
