@@ -307,13 +307,16 @@ def spawn_ranks(world, target, payload):
 class Case:
     """One workload set up on the current device: resident inputs, host copies for the end-to-end path, step functions."""
 
-    def __init__(self, rdf, torch, cfg, grad, dist=None):
+    def __init__(self, rdf, torch, cfg, grad, dist=None, store="thread", hash_load=None):
         self.rdf, self.torch, self.cfg, self.dist = rdf, torch, cfg, dist
         self.N = cfg["N"]
         self.grad = bool(grad)
         if cfg["kind"] == "fib":
             fs, r = rdf.fib_program()
             self.g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+            # token store: probing strategy, and (hash_load) the table sized for that load factor instead of the default
+            parked = int(sum(fib_iter(int(n) + 1) - 1 for n in cfg["x"]))
+            self.g.set_store(1 if store == "warp" else 0, int(parked / hash_load) if hash_load else 0)
             self.x_host = torch.from_numpy(cfg["x"]).pin_memory()
             self.x_dev = self.x_host.cuda()
             self.y = torch.empty_like(self.x_dev)
@@ -519,7 +522,7 @@ def run(args):
     # every rank processes a batch of its own (instances never exchange tokens): weak scaling
     cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
-    case = Case(rdf, torch, cfg, cfg.get("grad", False), dist)
+    case = Case(rdf, torch, cfg, cfg.get("grad", False), dist, args.store, args.hash_load)
 
     clocks = ClockSampler(local)
     clocks.start()                                   # samples from the warm-up on: short runs still get samples under load
@@ -582,7 +585,8 @@ def run(args):
         "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": case.dtype, "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else ""),
+        "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else "")
+                   + (f" [store: {args.store} probes" + (f", load {args.hash_load}" if args.hash_load else "") + "]" if args.workload == 1 else ""),
                    "invocations_per_step": case.N, "instances": cfg.get("B") or cfg["trees"].B,
                    "pass": "forward+backward" if cfg.get("grad") else "forward",
                    "timing": "CUDA events per step; 256 MB L2 flush between steps; inputs and parameters resident"},
@@ -630,6 +634,10 @@ def main():
     ap.add_argument("--seed", type=int, default=workloads.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="skip the table of the other workloads")
+    ap.add_argument("--store", default="thread", choices=["thread", "warp"],
+                    help="workload 1: probing of the hash token store (per thread / warp-cooperative)")
+    ap.add_argument("--hash-load", type=float, default=None,
+                    help="workload 1: size the hash table for this load factor (parked operands / slots, rounded to a power of two)")
     ap.add_argument("--fib-batch", type=int, default=None,
                     help="workload 1 only: number of independent fib calls (default 1024, the named configuration)")
     args = ap.parse_args()

@@ -299,6 +299,18 @@ int rdf_last_status(rdf_graph* g, rdf_stats* s);
 
 const char* rdf_strerror(int status);
 
+/* The hash form of the token store (RDF_TAGS_PATH; Section 2.2: an operator fires when its inputs hold tokens with
+ * the same tag -- the store is where the first operand waits for the second), for the following calls on this graph.
+ *   probe_mode : RDF_PROBE_THREAD -- every thread probes linearly for its own key (default);
+ *                RDF_PROBE_WARP   -- the threads of a warp that reach the store together probe for one key at a time,
+ *                                    each looking at one of 32 consecutive slots (a coalesced 512-byte load and a ballot).
+ *   hash_slots : slots per matching operator (rounded up to a power of two, at least 1024); 0 = the default,
+ *                the power of two at or above rdf_batch.max_invocations.  Entries are never removed, so a run
+ *                needs one slot per parked operand; a table that is too small reports RDF_ERR_STORE_FULL.
+ * Results do not depend on either setting.  rdf_workspace_bytes reflects hash_slots. */
+enum { RDF_PROBE_THREAD = 0, RDF_PROBE_WARP = 1 };
+int rdf_set_store(rdf_graph* g, int probe_mode, long long hash_slots);
+
 /* Limits of the device executor for the following calls on this graph (the paper's
  * executor simply runs until both queues are empty, Section 5.1; these guards have
  * no counterpart there).

@@ -100,6 +100,30 @@ def primes(n, count=None):
     return found
 
 
+def sum_to(n):
+    """0 + 1 + .. + (n - 1), by the loop itself."""
+    s, i = 0, 0
+    while i < n:
+        s, i = s + i, i + 1
+    return s
+
+
+def pairs(n):
+    """Number of pairs (j, i) with 0 <= j < i < n, by the two nested loops."""
+    acc, i = 0, 0
+    while i < n:
+        j = 0
+        while j < i:
+            acc, j = acc + 1, j + 1
+        i += 1
+    return acc
+
+
+def tri(n):
+    """tri(n) = 0 if n < 1 else sum_to(n) + tri(n - 1)."""
+    return 0 if n < 1 else sum_to(n) + tri(n - 1)
+
+
 def fib_invocations(n, tag=(0,), out=None):
     """Every invocation of fib below the call `result = fib(n)` as
     (tag, argument, result); the call in `result` is call site 0, the two

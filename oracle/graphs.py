@@ -18,7 +18,7 @@ from dataclasses import dataclass, field
 @dataclass
 class Node:
     id: int
-    kind: str            # 'in' 'out' 'const' 'op' 'switch' 'merge' 'fcall' 'Call' 'Return'
+    kind: str            # 'in' 'out' 'const' 'op' 'switch' 'merge' 'fcall' 'Call' 'Return' 'Enter' 'Exit' 'Next'
     name: str = ""       # op symbol, or callee name for 'fcall', or owner function
     value: object = None  # constant value / parameter index / label i
     func: str = ""       # the function graph this node came from
@@ -102,6 +102,49 @@ class FunctionGraph:
         self.g.connect(a[0], nid, 0, src_port=a[1])
         self.g.connect(b[0], nid, 1, src_port=b[1])
         return (nid, 0)
+
+    # ---- tagged iteration (Section 2.3, the while-loop of Figure 1)
+    def enter(self, v):
+        nid = self.g.add("Enter", func=self.name, n_in=1)
+        self.g.connect(v[0], nid, 0, src_port=v[1])
+        return (nid, 0)
+
+    def exit_(self, v):
+        nid = self.g.add("Exit", func=self.name, n_in=1)
+        self.g.connect(v[0], nid, 0, src_port=v[1])
+        return (nid, 0)
+
+    def next_(self, v):
+        nid = self.g.add("Next", func=self.name, n_in=1)
+        self.g.connect(v[0], nid, 0, src_port=v[1])
+        return (nid, 0)
+
+    def loop_merge(self, entered):
+        """The Merge at the head of a loop: input 0 from Enter now, input 1 from Next through `close_loop`."""
+        nid = self.g.add("merge", name="loop", func=self.name, n_in=2)
+        self.g.connect(entered[0], nid, 0, src_port=entered[1])
+        return (nid, 0)
+
+    def close_loop(self, merge, nxt):
+        self.g.connect(nxt[0], merge[0], 1, src_port=nxt[1])
+
+    def while_loop(self, inits, cond, body, result):
+        """The graph of Figure 1 for loop-carried variables v_1..v_m, one Enter / Merge / Switch / Next per variable
+        and an Exit for the variable that is the loop's value:
+            inits  : initial values (outside the loop);
+            cond   : f(builder, merged values) -> predicate value;
+            body   : f(builder, values on the true side) -> next values;
+            result : index of the variable whose final value leaves through Exit.
+        Inside `cond` and `body` constants must be derived from a loop value with a unary operator (a constant node
+        would carry the tag of the enclosing activation, not of the iteration)."""
+        merged = [self.loop_merge(self.enter(v)) for v in inits]
+        p = cond(self, merged)
+        sides = [self.switch(p, m) for m in merged]
+        nxt = body(self, [t for t, _ in sides])
+        assert len(nxt) == len(inits)
+        for m, n in zip(merged, nxt):
+            self.close_loop(m, self.next_(n))
+        return self.exit_(sides[result][1])
 
     def call(self, fname, *args):
         nid = self.g.add("fcall", name=fname, func=self.name, n_in=len(args))

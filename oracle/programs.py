@@ -29,6 +29,13 @@ from .graphs import FunctionGraph
 # integer programs
 # --------------------------------------------------------------------------
 INT_OPS = {
+    # unary operators with a built-in constant (inside a loop a constant is derived from a loop value, see
+    # FunctionGraph.while_loop)
+    "add1": lambda a: a + 1,
+    "sub1": lambda a: a - 1,
+    "zero": lambda a: 0,
+    "two": lambda a: 2,
+    "not": lambda a: not a,
     "+": lambda a, b: a + b,
     "-": lambda a, b: a - b,
     "*": lambda a, b: a * b,
@@ -141,6 +148,69 @@ def tak_program(y_const=12, z_const=6):
     b = f.call("tak", f.op("-", y_t, one), z_t, x_t)
     c = f.call("tak", f.op("-", z_t, one), x_t, y_t)
     f.output(f.merge(f.call("tak", a, b, c), f.op("id", z_e)))
+    return [r, f]
+
+
+# --------------------------------------------------------------------------
+# tagged iteration (Section 2.3) alone, nested, with calls inside, and inside a recursive function
+# --------------------------------------------------------------------------
+def sum_loop_program():
+    """result(n) = { s = 0; i = 0; while (i < n) { s = s + i; i = i + 1 }; s }  -- the while-loop of Figure 1 with the
+    loop-carried variables (s, i, n)."""
+    r = FunctionGraph("result", 1)
+    n = r.param(0)
+    out = r.while_loop([r.const(0), r.const(0), n],
+                       lambda f, v: f.op("<", v[1], v[2]),
+                       lambda f, v: [f.op("+", v[0], v[1]), f.op("add1", v[1]), f.op("id", v[2])], 0)
+    r.output(out)
+    return [r]
+
+
+def pairs_loop_program():
+    """result(n) = number of pairs (j, i) with 0 <= j < i < n, by two nested loops: the inner loop runs under tags
+    [j, i] (inner counter first), as in the two-loop example of Section 2.3."""
+    r = FunctionGraph("result", 1)
+    n = r.param(0)
+
+    def outer_body(f, v):                     # v = (acc, i, n)
+        inner = f.while_loop([v[0], f.op("zero", v[1]), v[1]],          # (acc, j = 0, i)
+                             lambda g, w: g.op("<", w[1], w[2]),
+                             lambda g, w: [g.op("add1", w[0]), g.op("add1", w[1]), g.op("id", w[2])], 0)
+        return [inner, f.op("add1", v[1]), f.op("id", v[2])]
+    out = r.while_loop([r.const(0), r.const(0), n], lambda f, v: f.op("<", v[1], v[2]), outer_body, 0)
+    r.output(out)
+    return [r]
+
+
+def primes_loop_program():
+    """result(x) = { c = 0; i = 2; while (not x < i) { c = c + isprime(i, 2); i = i + 1 }; c } with the recursive
+    isprime of `primes_program`: a function called from inside a loop body (the call's label goes on top of the
+    iteration counter)."""
+    r = FunctionGraph("result", 1)
+    x = r.param(0)
+    out = r.while_loop([r.const(0), r.const(2), x],
+                       lambda f, v: f.op("not", f.op("<", v[2], v[1])),
+                       lambda f, v: [f.op("+", v[0], f.call("isprime", v[1], f.op("two", v[1]))), f.op("add1", v[1]),
+                                     f.op("id", v[2])], 0)
+    r.output(out)
+    q = [f for f in primes_program() if f.name == "isprime"][0]
+    return [r, q]
+
+
+def tri_program():
+    """result(x) = tri(x);  tri(n) = if n < 1 then 0 else sumto(n) + tri(n - 1), where sumto(n) = 0 + 1 + .. + (n - 1)
+    is a while-loop inside the body of the recursive function: loop frames on top of call frames."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("tri", r.param(0)))
+    f = FunctionGraph("tri", 1)
+    n = f.param(0)
+    t, e = f.switch(f.op("<", n, f.const(1)), n)
+    zero = f.op("zero", e)
+    s = f.while_loop([zero, f.op("zero", e), e],
+                     lambda g, v: g.op("<", v[1], v[2]),
+                     lambda g, v: [g.op("+", v[0], v[1]), g.op("add1", v[1]), g.op("id", v[2])], 0)
+    rec = f.call("tri", f.op("sub1", e))
+    f.output(f.merge(f.op("zero", t), f.op("+", s, rec)))
     return [r, f]
 
 

@@ -17,7 +17,10 @@ time, following the paper's semantic equations:
     along the control edge Call_i -> Return_i, and Return_i hands it on to its
     successors (Section 5.2.1);
   * nodes wait in a pending table keyed by (node, tag) and tokens are taken
-    from a FIFO queue until it is empty (Section 5.1).
+    from a FIFO queue until it is empty (Section 5.1);
+  * Enter <t, d> = <0:t, d>;  Exit <n:t, d> = <t, d>;  Next <n:t, d> = <(n+1):t, d>
+    (Section 2.3).  Iteration counters and call labels live in the one tag list
+    (Section 5.1: loops and functions share the stack).
 
 Readings where the text is silent:
   * the entry Merge of a function has one input per call site; tokens from
@@ -26,6 +29,9 @@ Readings where the text is silent:
   * a constant inside a called function fires when the control token from the
     entry Merge arrives (Figure 3); a constant of `result` fires once, with
     the empty tag;
+  * a hiaton that reaches Exit or Next is dropped: every iteration but the last sends one to Exit (the Switch's
+    other side) and the last one sends one round the body to Next; letting them through would put several tokens
+    with one tag on the loop's consumers, or keep a dead loop turning (the paper does not treat this case);
   * `dead_tokens=False` elides hiatons altogether (Switch emits only the live
     side).  Results are the same; operands left waiting for a partner on the
     branch not taken are dropped when the queue runs empty.
@@ -54,6 +60,9 @@ class RunResult:
         self.returns_by_output = {}   # (tag, output index) -> returned datum, for functions with several outputs
         self.firings = 0
         self.max_depth = 0
+        self.enters = []         # tags produced by Enter nodes, in firing order
+        self.nexts = []          # tags produced by Next nodes
+        self.exits = []          # tags consumed by Exit nodes
         self.leftover = 0        # tokens still waiting when the queue ran empty
         self.max_pending = 0
 
@@ -176,6 +185,20 @@ def run(graph, feeds, ops, dead_tokens=True, max_firings=None) -> RunResult:
                     emit(nid, 0, tag[1:], datum)
                 else:
                     held[key] = datum
+        elif kind == "Enter":
+            if datum is not DEAD:
+                res.enters.append((0,) + tag)
+                if len(tag) + 1 > res.max_depth:
+                    res.max_depth = len(tag) + 1
+            emit(nid, 0, (0,) + tag, datum)
+        elif kind == "Exit":
+            if datum is not DEAD:
+                res.exits.append(tag)
+                emit(nid, 0, tag[1:], datum)
+        elif kind == "Next":
+            if datum is not DEAD:
+                res.nexts.append((tag[0] + 1,) + tag[1:])
+                emit(nid, 0, (tag[0] + 1,) + tag[1:], datum)
         elif kind == "out":
             if datum is not DEAD:
                 assert tag not in res.outputs

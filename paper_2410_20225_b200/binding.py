@@ -113,7 +113,8 @@ class rdf_stats(C.Structure):
 
 EXPORTS = ["rdf_graph_build", "rdf_graph_free", "rdf_graph_describe", "rdf_workspace_bytes", "rdf_eval", "rdf_grad",
            "rdf_last_status", "rdf_strerror", "rdf_set_profiling", "rdf_last_phase_ms", "rdf_eval_noalloc",
-           "rdf_set_limits", "rdf_probe_fp32_fma"]
+           "rdf_set_limits", "rdf_probe_fp32_fma", "rdf_set_store"]
+PROBE_THREAD, PROBE_WARP = 0, 1
 NOALLOC_SCRATCH_BYTES = 16 << 20
 PHASES = ["setup", "schedule", "group", "operators", "roots", "loss", "lists", "backward", "dW", "db", "dE"]
 
@@ -141,6 +142,7 @@ def lib() -> C.CDLL:
         L.rdf_last_status.argtypes = [C.c_void_p, C.POINTER(rdf_stats)]
         L.rdf_set_profiling.argtypes = [C.c_void_p, C.c_int]
         L.rdf_set_limits.argtypes = [C.c_void_p, C.c_longlong, C.c_longlong]
+        L.rdf_set_store.argtypes = [C.c_void_p, C.c_int, C.c_longlong]
         L.rdf_probe_fp32_fma.argtypes = [C.POINTER(C.c_double), C.c_void_p]
         L.rdf_last_phase_ms.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
         L.rdf_strerror.argtypes = [C.c_int]
@@ -362,6 +364,12 @@ class Graph:
         rc = lib().rdf_set_limits(self.handle, int(wait_cycles), int(wave_limit))
         if rc != RDF_OK:
             raise RdfError(rc, "rdf_set_limits")
+
+    def set_store(self, probe_mode=PROBE_THREAD, hash_slots=0):
+        """Hash token store (path tags): probing strategy and slots per matching operator (0 = default)."""
+        rc = lib().rdf_set_store(self.handle, int(probe_mode), int(hash_slots))
+        if rc != RDF_OK:
+            raise RdfError(rc, "rdf_set_store")
 
     def phase_ms(self):
         """{phase name: milliseconds} of the last call (needs set_profiling(True) before it)."""

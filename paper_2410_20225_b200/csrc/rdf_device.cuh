@@ -181,6 +181,7 @@ struct DevCtx {
     // control
     Control*  ctl;
     uint32_t  wave_limit;
+    int       probe_mode;         // hash store: 0 = every thread probes for itself, 1 = the threads of a warp probe together
     long long spin_limit;         // clock64 ticks a barrier wait may last
 };
 
@@ -426,11 +427,10 @@ struct StoreCounters {
 // in place; capacity is sized for all insertions of the run.
 // Returns 1 and the partner's value when the match completed, 0 when parked,
 // -1 when the table is full.
-__device__ __forceinline__ int hash_insert_or_consume(const DevCtx& c, int node, uint64_t key, int64_t val,
-                                                      int64_t& partner, StoreCounters& sc) {
+__device__ __forceinline__ int hash_insert_or_consume_from(const DevCtx& c, int node, uint64_t key, int64_t val,
+                                                           int64_t& partner, StoreCounters& sc, uint64_t h) {
     Slot* tab = c.table + (size_t)node * c.table_cap;
     const uint64_t mask = c.table_cap - 1;
-    uint64_t h = mix64(key) & mask;
     for (uint64_t probe = 0; probe < c.table_cap; ++probe) {
         ++sc.probes;
         const uint4 raw = __ldcv(reinterpret_cast<const uint4*>(&tab[h]));
@@ -459,6 +459,43 @@ __device__ __forceinline__ int hash_insert_or_consume(const DevCtx& c, int node,
         h = (h + 1) & mask;
     }
     return -1;
+}
+__device__ __forceinline__ int hash_insert_or_consume(const DevCtx& c, int node, uint64_t key, int64_t val,
+                                                      int64_t& partner, StoreCounters& sc) {
+    return hash_insert_or_consume_from(c, node, key, val, partner, sc, mix64(key) & (c.table_cap - 1));
+}
+
+// The same with cooperative probing: the threads of a warp that reach the store together look for one key at a
+// time -- each inspects one of as many consecutive slots as there are threads (one coalesced load of 16 bytes per
+// thread, 512 bytes for a full warp) and a ballot picks the first slot that holds the key or is empty.  When every
+// key of the group has its slot, each thread finishes its own access there (128-bit CAS; should the slot have
+// changed meanwhile it carries on alone from that slot).  Long probe sequences (a table filled close to capacity)
+// cost one step per 32 slots instead of one per slot; at low load factors the per-thread form above needs about one
+// load anyway and the rounds only add latency.
+__device__ __forceinline__ int hash_insert_or_consume_group(const DevCtx& c, int node, uint64_t key, int64_t val,
+                                                            int64_t& partner, StoreCounters& sc) {
+    cg::coalesced_group g = cg::coalesced_threads();
+    const uint32_t n = g.size(), me = g.thread_rank();
+    const uint64_t mask = c.table_cap - 1;
+    const uint64_t h = mix64(key) & mask;
+    long long found = -1;
+    for (uint32_t r = 0; r < n; ++r) {
+        const uint64_t key_r = g.shfl(key, r), h_r = g.shfl(h, r);
+        const Slot* tab_r = c.table + (size_t)g.shfl(node, r) * c.table_cap;
+        for (uint64_t step = 0; step < c.table_cap; step += n) {
+            const uint64_t idx = (h_r + step + me) & mask;
+            const uint4 raw = __ldcv(reinterpret_cast<const uint4*>(&tab_r[idx]));
+            const uint64_t k = (uint64_t)raw.x | ((uint64_t)raw.y << 32);
+            const unsigned hits = g.ballot(k == key_r || k == SLOT_EMPTY);
+            if (me == r) ++sc.probes;
+            if (hits) {
+                if (me == r) found = (long long)((h_r + step + (uint64_t)(__ffs(hits) - 1)) & mask);
+                break;
+            }
+        }
+    }
+    if (found < 0) return -1;
+    return hash_insert_or_consume_from(c, node, key, val, partner, sc, (uint64_t)found);
 }
 
 __device__ __forceinline__ void exch128(Slot* addr, uint64_t new_lo, uint64_t new_hi, uint64_t& old_lo, uint64_t& old_hi) {

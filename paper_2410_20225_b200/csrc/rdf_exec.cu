@@ -173,7 +173,8 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                 int done;
                 if (c.tag_mode == RDF_TAGS_PATH) {
                     int64_t partner = 0;
-                    done = hash_insert_or_consume(c, node, tag, val, partner, st.sc);
+                    done = c.probe_mode ? hash_insert_or_consume_group(c, node, tag, val, partner, st.sc)
+                                        : hash_insert_or_consume(c, node, tag, val, partner, st.sc);
                     if (done < 0) {
                         set_status(c, RDF_ERR_STORE_FULL);
                         return;
@@ -488,8 +489,18 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
         const Token* q = c.q[wave & 1];
-        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-            run_token(c, sp, nullptr, wave, load_token(&q[i]), st);
+        {
+            // a wave wider than the grid: the thread's next token is on its way while it runs the current one
+            const uint32_t stride = gridDim.x * blockDim.x;
+            uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+            Token next = i < n ? load_token(&q[i]) : Token{};
+            while (i < n) {
+                const Token cur = next;
+                i += stride;
+                if (i < n) next = load_token(&q[i]);
+                run_token(c, sp, nullptr, wave, cur, st);
+            }
+        }
         __syncthreads();
         lap(cyc_s);
         if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
@@ -758,6 +769,10 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.arrived_bytes = (size_t)L.frame_cap * std::max<size_t>(1, g->match.size()) * sizeof(uint32_t);
     L.arrived = P.take<char>(L.arrived_bytes);
     L.table_cap = g->tag_mode == RDF_TAGS_PATH && !g->match.empty() ? pow2_at_least((uint64_t)in->max_invocations) : 0;
+    {
+        const ExecState* S = static_cast<const ExecState*>(g->dev);
+        if (S && S->hash_slots > 0 && L.table_cap) L.table_cap = pow2_at_least((uint64_t)S->hash_slots);
+    }
     L.table_bytes = (size_t)L.table_cap * g->match.size() * sizeof(Slot);
     L.table = P.take<char>(L.table_bytes);
     L.cell_items = P.take<CellItem>(L.work_cap);
@@ -922,6 +937,7 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
     c.wave_limit = L.wave_cap ? L.wave_cap : 1u << 24;
     if (S->wave_limit > 0) c.wave_limit = (uint32_t)std::min<long long>(S->wave_limit, c.wave_limit);
+    c.probe_mode = S->probe_mode;
     c.spin_limit = S->wait_cycles > 0 ? S->wait_cycles : (long long)S->clock_khz * 2000ll;       // default: about two seconds of SM clock
 }
 
@@ -1105,6 +1121,14 @@ extern "C" int rdf_set_limits(rdf_graph* g, long long wait_cycles, long long wav
     ExecState* S = rdf_state_of(g);
     S->wait_cycles = wait_cycles;
     S->wave_limit = wave_limit;
+    return RDF_OK;
+}
+
+extern "C" int rdf_set_store(rdf_graph* g, int probe_mode, long long hash_slots) {
+    if (!g || (probe_mode != RDF_PROBE_THREAD && probe_mode != RDF_PROBE_WARP) || hash_slots < 0) return RDF_ERR_BAD_ARG;
+    ExecState* S = rdf_state_of(g);
+    S->probe_mode = probe_mode;
+    S->hash_slots = hash_slots;
     return RDF_OK;
 }
 

@@ -52,6 +52,8 @@ struct ExecState {
     cudaStream_t last_stream = nullptr;
     bool ran = false;
     unsigned launches = 0;       // kernels launched by the last call
+    int probe_mode = 0;          // rdf_set_store
+    long long hash_slots = 0;
     long long wait_cycles = 0;   // rdf_set_limits: 0 = default
     long long wave_limit = 0;
     // optional phase timing

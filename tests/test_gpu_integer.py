@@ -7,6 +7,7 @@ import pytest
 
 import workloads
 import paper_2410_20225_b200 as rdf
+from paper_2410_20225_b200 import binding as bd
 from oracle import direct, programs, tagged, transform
 
 torch = pytest.importorskip("torch")
@@ -226,6 +227,35 @@ def test_capacity_error_returns_promptly():
         g.eval_int(x, max_invocations=50000)
     assert e.value.code == -6
     assert time.perf_counter() - t0 < 0.5
+
+
+@pytest.mark.parametrize("probe", [bd.PROBE_THREAD, bd.PROBE_WARP])
+@pytest.mark.parametrize("tight", [False, True])
+def test_hash_store_probing_variants(probe, tight):
+    """The hash token store with per-thread and with warp-cooperative probing, at the default size and with just
+    enough slots for the operands of the run (long probe sequences): the same values, the same multiset of
+    Call / Return records with their packed tags, every parked operand matched exactly once."""
+    x_host = workloads.fib_batch(seed=5, B=512, n_hi=16)
+    x = torch.from_numpy(x_host).cuda()
+    n_inv = int(sum(2 * _fib_iter(int(n) + 1) - 1 for n in x_host))
+    parked = int(sum(_fib_iter(int(n) + 1) - 1 for n in x_host))
+    fs, r = rdf.fib_program()
+    ref = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    y0, t0 = ref.eval_int(x, n_inv, trace_capacity=2 * n_inv)
+    g = rdf.Graph(fs, r, rdf.TAGS_PATH)
+    g.set_store(probe, parked if tight else 0)
+    y, t = g.eval_int(x, n_inv, trace_capacity=2 * n_inv)
+    st = g.stats()
+    assert y.tolist() == [_fib_iter(int(n)) for n in x_host] and torch.equal(y, y0)
+    assert st["store_inserts"] == st["store_matches"] == parked and st["invocations"] == n_inv
+    assert np.array_equal(np.sort(t, order=["tag", "kind", "value"]), np.sort(t0, order=["tag", "kind", "value"]))
+    if tight:
+        assert st["max_probe"] > ref.stats()["max_probe"] or probe == bd.PROBE_WARP
+    # a table smaller than the operands of the run is reported, whatever the probing
+    g.set_store(probe, 1024)
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(x, n_inv)
+    assert e.value.code == -5
 
 
 def test_bad_arguments():
