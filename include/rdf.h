@@ -84,6 +84,8 @@ typedef struct {
     int64_t imm;
 } rdf_expr;
 
+typedef enum { RDF_FN_FUNCTION = 0, RDF_FN_LOOP = 1 } rdf_function_kind;
+
 typedef struct {
     const char*     name;        /* host, NUL-terminated, copied by rdf_graph_build */
     int32_t         n_params;    /* m formal parameters: 1 for `result`, 1..3 for the others; m > 1 needs
@@ -91,6 +93,16 @@ typedef struct {
     int32_t         n_exprs;
     const rdf_expr* exprs;       /* host, [n_exprs]; a DAG (no cycles) */
     int32_t         root;        /* index of the expression that is the function's output */
+    /* A definition of kind RDF_FN_LOOP is a while-loop (Section 2.3, Figure 1) over m loop-carried variables, its
+     * parameters: while `cond` holds, variable k takes the value of `next[k]`; when it fails the loop's value is `root`,
+     * evaluated on the final values.  A CALL of it with the initial values stands for the loop at that place: in
+     * the static graph one Enter / Merge / Switch / Next per variable and an Exit, tags <0:t> on entry and
+     * <(n+1):t> per iteration; loops and calls share the tag stack (Section 5.1).  `cond` and `root` must not
+     * contain calls; `next[k]` may (functions, recursive ones, other loops).  Integer values, RDF_TAGS_FRAME.
+     * (RDF_FN_FUNCTION: cond and next are ignored.) */
+    int32_t         kind;        /* rdf_function_kind */
+    int32_t         cond;
+    int32_t         next[3];
 } rdf_function;
 
 typedef enum { RDF_TAGS_PATH = 0, RDF_TAGS_FRAME = 1 } rdf_tag_mode;
@@ -123,7 +135,8 @@ void rdf_graph_free(rdf_graph* g);
  * Figure 3).  Arrays are host memory owned by the graph. */
 typedef enum {
     RDF_NODE_IN = 0, RDF_NODE_OUT, RDF_NODE_CONST, RDF_NODE_OP, RDF_NODE_SWITCH,
-    RDF_NODE_MERGE, RDF_NODE_ENTRY_MERGE, RDF_NODE_CALL, RDF_NODE_RETURN
+    RDF_NODE_MERGE, RDF_NODE_ENTRY_MERGE, RDF_NODE_CALL, RDF_NODE_RETURN,
+    RDF_NODE_ENTER, RDF_NODE_EXIT, RDF_NODE_NEXT      /* tagged iteration, Section 2.3 */
 } rdf_node_kind;
 
 typedef struct {
@@ -199,12 +212,16 @@ typedef struct {
 /* One record per Call firing and one per Return firing, in no particular
  * order (optional; for parity checks of tags). */
 typedef struct {
-    uint64_t tag;        /* PATH: packed tag of the invocation; FRAME: its frame id */
-    int64_t  value;      /* kind 0: the argument; kind 1: the returned integer (vector programs: frame id of the state) */
-    uint32_t kind;       /* 0 = Call fired (tag after the push), 1 = Return fired (tag before the pop) */
-    uint32_t label;      /* i of Call_i / Return_i (global label id) */
-    uint32_t parent;     /* FRAME: frame id of the caller's context; PATH: 0 */
-    uint32_t instance;   /* FRAME: unused (0); PATH: bits [63:44] of the tag */
+    uint64_t tag;        /* PATH: packed tag of the invocation; FRAME: its frame id in the low half; inside a loop the
+                            high half holds the iteration counter of the loop frame (the tag <n:t> of Section 2.3) */
+    int64_t  value;      /* kind 0: the argument; kind 1: the returned integer (vector programs: frame id of the state);
+                            kinds 2-4: the first loop variable */
+    uint32_t kind;       /* 0 = Call fired (tag after the push), 1 = Return fired (tag before the pop),
+                            2 = Enter fired (tag after), 3 = Next fired (tag after), 4 = Exit fired (tag before) */
+    uint32_t label;      /* i of Call_i / Return_i (global label id); loops: 255 */
+    uint32_t parent;     /* FRAME: frame id of the enclosing context (the tag below this one); PATH: 0 */
+    uint32_t instance;   /* FRAME: iteration counter of the enclosing context when that is a loop frame, else 0;
+                            PATH: bits [63:44] of the tag */
 } rdf_trace_rec;
 
 typedef struct {

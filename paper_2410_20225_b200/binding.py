@@ -24,7 +24,10 @@ ERRORS = {
  OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS, OP_REM) = range(20)
 TAGS_PATH, TAGS_FRAME = 0, 1
 F32, BF16 = 0, 1
-(NODE_IN, NODE_OUT, NODE_CONST, NODE_OP, NODE_SWITCH, NODE_MERGE, NODE_ENTRY_MERGE, NODE_CALL, NODE_RETURN) = range(9)
+(NODE_IN, NODE_OUT, NODE_CONST, NODE_OP, NODE_SWITCH, NODE_MERGE, NODE_ENTRY_MERGE, NODE_CALL, NODE_RETURN, NODE_ENTER,
+ NODE_EXIT, NODE_NEXT) = range(12)
+FN_FUNCTION, FN_LOOP = 0, 1
+LOOP_LABEL = 255
 
 PATH_BITS, DEPTH_SHIFT, INST_SHIFT = 38, 38, 44
 
@@ -42,7 +45,8 @@ class rdf_expr(C.Structure):
 
 class rdf_function(C.Structure):
     _fields_ = [("name", C.c_char_p), ("n_params", C.c_int32), ("n_exprs", C.c_int32),
-                ("exprs", C.POINTER(rdf_expr)), ("root", C.c_int32)]
+                ("exprs", C.POINTER(rdf_expr)), ("root", C.c_int32), ("kind", C.c_int32), ("cond", C.c_int32),
+                ("next", C.c_int32 * 3)]
 
 
 class rdf_program(C.Structure):
@@ -167,6 +171,14 @@ class Function:
 
     def __init__(self, name: str, n_params: int):
         self.name, self.n_params, self.exprs, self.root = name, n_params, [], -1
+        self.kind, self.cond, self.next = FN_FUNCTION, -1, [-1, -1, -1]
+
+    def loop(self, cond, nexts, value):
+        """Makes this definition a while-loop over its parameters (the loop-carried variables): while `cond`, variable k
+        becomes nexts[k]; at exit the loop's value is `value`.  A call of it with the initial values is the loop."""
+        assert len(nexts) == self.n_params
+        self.kind, self.cond, self.next, self.root = FN_LOOP, cond, list(nexts) + [-1] * (3 - len(nexts)), value
+        return self
 
     def _add(self, op, a=-1, b=-1, c=-1, imm=0):
         self.exprs.append((op, a, b, c, imm))
@@ -261,6 +273,58 @@ def tak_program(y_const=12, z_const=6):
     return [r, f], 0
 
 
+def sum_loop_program():
+    """result(n) = { s = 0; i = 0; while (i < n) { s = s + i; i = i + 1 }; s }: the while-loop of Figure 1."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.const(0), r.const(0), r.param()))
+    lp = Function("sum_while", 3)
+    s_, i, n = lp.param(0), lp.param(1), lp.param(2)
+    lp.loop(lp.lt(i, n), [lp.add(s_, i), lp.add(i, lp.const(1)), n], s_)
+    return [r, lp], 0
+
+
+def pairs_loop_program():
+    """result(n) = number of pairs (j, i), 0 <= j < i < n, by two nested loops (tags [j, i] in the inner one)."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.const(0), r.const(0), r.param()))
+    outer = Function("outer", 3)
+    acc, i, n = outer.param(0), outer.param(1), outer.param(2)
+    outer.loop(outer.lt(i, n), [outer.call(2, acc, outer.const(0), i), outer.add(i, outer.const(1)), n], acc)
+    inner = Function("inner", 3)
+    a, j, lim = inner.param(0), inner.param(1), inner.param(2)
+    inner.loop(inner.lt(j, lim), [inner.add(a, inner.const(1)), inner.add(j, inner.const(1)), lim], a)
+    return [r, outer, inner], 0
+
+
+def primes_loop_program():
+    """result(x) = { c = 0; i = 2; while (not x < i) { c = c + isprime(i, 2); i = i + 1 }; c }: a recursive function
+    called from a loop body."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.const(0), r.const(2), r.param()))
+    lp = Function("count_while", 3)
+    c, i, x = lp.param(0), lp.param(1), lp.param(2)
+    lp.loop(lp.eq(lp.lt(x, i), lp.const(0)), [lp.add(c, lp.call(2, i, lp.const(2))), lp.add(i, lp.const(1)), x], c)
+    q = Function("isprime", 2)
+    i, d = q.param(0), q.param(1)
+    q.ret(q.if_(q.lt(i, q.mul(d, d)), q.const(1),
+                q.if_(q.eq(q.rem(i, d), q.const(0)), q.const(0), q.call(2, i, q.add(d, q.const(1))))))
+    return [r, lp, q], 0
+
+
+def tri_program():
+    """result(x) = tri(x); tri(n) = 0 if n < 1 else sumto(n) + tri(n - 1), sumto a while-loop inside the recursive body."""
+    r = Function("result", 1)
+    r.ret(r.call(1, r.param()))
+    f = Function("tri", 1)
+    n = f.param()
+    loop = f.call(2, f.const(0), f.const(0), n)
+    f.ret(f.if_(f.lt(n, f.const(1)), f.const(0), f.add(loop, f.call(1, f.sub(n, f.const(1))))))
+    lp = Function("sum_while", 3)
+    s_, i, m = lp.param(0), lp.param(1), lp.param(2)
+    lp.loop(lp.lt(i, m), [lp.add(s_, i), lp.add(i, lp.const(1)), m], s_)
+    return [r, f, lp], 0
+
+
 def tree_fold_program(kind: str):
     """Integer folds over the input trees: 'sum' of leaf tokens, leaf 'count', 'height'."""
     r = Function("result", 1)
@@ -309,7 +373,8 @@ class Graph:
         for i, f in enumerate(functions):
             ex = (rdf_expr * max(1, len(f.exprs)))(*[rdf_expr(*e) for e in f.exprs])
             self._keep.append(ex)
-            fs[i] = rdf_function(f.name.encode(), f.n_params, len(f.exprs), ex, f.root)
+            fs[i] = rdf_function(f.name.encode(), f.n_params, len(f.exprs), ex, f.root, f.kind, f.cond,
+                                 (C.c_int32 * 3)(*f.next))
         prog = rdf_program(len(functions), fs, result, tag_mode)
         self.handle = C.c_void_p()
         self.tag_mode = tag_mode

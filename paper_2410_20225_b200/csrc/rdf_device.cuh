@@ -33,6 +33,10 @@ struct __align__(16) Frame {
     int64_t  arg;
 };
 static const uint32_t FRAME_LABEL_MASK = 0xFFu;
+static const uint32_t LOOP_LABEL = 0xFFu;     // label field of a loop frame (Enter), which no call site has
+// A tag in frame form: the frame id in the low half; for a loop frame the iteration counter in the high half
+// (Section 5.1: a tag is a pair of an iteration number and a pointer into the frame stack).
+__device__ __forceinline__ uint32_t frame_of(uint64_t tag) { return (uint32_t)tag; }
 static const int FRAME_WAVE_SHIFT = 8;
 
 // Hash-store slot: a parked operand keyed by the packed tag.
@@ -102,7 +106,9 @@ struct DevCtx {
     uint32_t qcap;
     // frames (frame-form tags)
     Frame*    frames;
-    uint32_t* children;           // [frame_cap * K]: frame created by call site k of this frame's body
+    uint64_t* frame_ptag;         // [frame_cap] programs with loops: the full tag below a frame (its frame id and, when
+                                  // that frame is a loop's, the iteration counter in the high half)
+    int       has_loops;
     uint32_t  frame_cap;
     int64_t*  frame_args;         // [frame_cap * 2]: parameters 1 and 2 of invocations of multi-parameter functions
     // token store, dense form.  Two-input operators: one 16-byte slot per (frame, match node), operand
@@ -329,15 +335,16 @@ __device__ __forceinline__ Token load_token(const Token* p) {
 // Packed path form: [63:44] instance | [43:38] depth | [37:0] labels, innermost lowest.
 __device__ __forceinline__ uint64_t path_root(long long instance) { return (uint64_t)instance << RDF_INST_SHIFT; }
 
+// (parent: the tag below -- frame form: frame id and, in the high half, the iteration counter of a loop frame)
 __device__ __forceinline__ void trace_rec(const DevCtx& c, uint64_t tag, int64_t value, uint32_t kind, uint32_t label,
-                                          uint32_t parent) {
+                                          uint64_t parent) {
     if (!c.trace) return;
     const unsigned long long i = atomicAdd(&c.ctl->trace_count, 1ull);
     if ((long long)i < c.trace_cap) {
         rdf_trace_rec r;
         r.tag = tag; r.value = value; r.kind = kind; r.label = label;
-        r.parent = c.tag_mode == RDF_TAGS_PATH ? 0u : parent;
-        r.instance = c.tag_mode == RDF_TAGS_PATH ? (uint32_t)(tag >> RDF_INST_SHIFT) : 0u;
+        r.parent = c.tag_mode == RDF_TAGS_PATH ? 0u : (uint32_t)parent;
+        r.instance = c.tag_mode == RDF_TAGS_PATH ? (uint32_t)(tag >> RDF_INST_SHIFT) : (uint32_t)(parent >> 32);
         c.trace[i] = r;
     }
 }
@@ -348,10 +355,10 @@ __device__ __forceinline__ void trace_rec(const DevCtx& c, uint64_t tag, int64_t
 __device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label, int64_t arg,
                                            uint32_t id, uint32_t wave) {
     Frame f;
-    f.parent = (uint32_t)tag; f.label = label | (wave << FRAME_WAVE_SHIFT); f.arg = arg;
+    f.parent = frame_of(tag); f.label = label | (wave << FRAME_WAVE_SHIFT); f.arg = arg;
     c.frames[id] = f;
-    c.children[(size_t)tag * c.K + labels[label].child_index] = id;
-    trace_rec(c, id, arg, 0, label, (uint32_t)tag);
+    if (c.frame_ptag) c.frame_ptag[id] = tag;
+    trace_rec(c, id, arg, 0, label, tag);
 }
 
 // Call_i: <t, d> -> <i:t, d>.  Returns false (status set) when the tag cannot be formed.
@@ -388,9 +395,9 @@ __device__ __forceinline__ void tag_pop(const DevCtx& c, uint64_t tag, uint32_t&
         parent = (tag & ~((1ull << RDF_INST_SHIFT) - 1)) | ((uint64_t)(depth - 1) << RDF_DEPTH_SHIFT) |
                  (path >> c.label_bits);
     } else {
-        const uint4 f = __ldcg(reinterpret_cast<const uint4*>(&c.frames[tag]));   // {parent, label, arg}
+        const uint4 f = __ldcg(reinterpret_cast<const uint4*>(&c.frames[frame_of(tag)]));   // {parent, label, arg}
         label = f.y & FRAME_LABEL_MASK;
-        parent = f.x;
+        parent = c.frame_ptag ? __ldcg(reinterpret_cast<const unsigned long long*>(&c.frame_ptag[frame_of(tag)])) : (uint64_t)f.x;
     }
 }
 
@@ -516,17 +523,22 @@ __device__ __forceinline__ void exch128(Slot* addr, uint64_t new_lo, uint64_t ne
 // first operand finds the slot empty and stays there, the second gets the first one back.
 // More inputs: the operand goes to its (frame, port) cell; the arrival that completes the set reads
 // the others.  Returns 1 when complete.
-__device__ __forceinline__ int dense_deliver(const DevCtx& c, const MatchNode& M, int node, uint64_t frame, int port,
+// In a program with loops a slot serves every iteration of its loop frame (the iterations of one loop follow one
+// another: Next fires when the whole body is done), so a completed match leaves the slot empty again.
+__device__ __forceinline__ int dense_deliver(const DevCtx& c, const MatchNode& M, int node, uint64_t tag, int port,
                                              int64_t val, int64_t* regs, StoreCounters& sc) {
+    const uint32_t frame = frame_of(tag);
     if (M.n_ports == 2) {
         uint64_t old_state, old_val;
-        exch128(&c.pair_slots[(size_t)frame * c.n_match + node], 1ull + (uint64_t)port, (uint64_t)val, old_state, old_val);
+        Slot* slot = &c.pair_slots[(size_t)frame * c.n_match + node];
+        exch128(slot, 1ull + (uint64_t)port, (uint64_t)val, old_state, old_val);
         if (old_state == 0) {
             ++sc.inserts;
             return 0;
         }
         regs[port] = val;
         regs[1 - port] = (int64_t)old_val;
+        if (c.has_loops) *reinterpret_cast<uint4*>(slot) = make_uint4(0u, 0u, 0u, 0u);
         ++sc.matches;
         return 1;
     }
@@ -540,6 +552,7 @@ __device__ __forceinline__ int dense_deliver(const DevCtx& c, const MatchNode& M
     }
     __threadfence();
     for (int p = 0; p < M.n_ports; ++p) regs[p] = __ldcv(reinterpret_cast<const long long*>(&cells[p]));
+    if (c.has_loops) c.arrived[(size_t)frame * c.n_match + node] = 0u;
     ++sc.matches;
     return 1;
 }

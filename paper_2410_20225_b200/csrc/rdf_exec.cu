@@ -128,8 +128,8 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                     if (d > st.max_depth) st.max_depth = d;
                 }
                 if (sp.labels[in.imm].n_args > 1) {             // the other Call_i nodes of this call site
-                    c.frame_args[(size_t)nt * 2] = r[in.b];
-                    c.frame_args[(size_t)nt * 2 + 1] = r[in.dst];
+                    c.frame_args[(size_t)frame_of(nt) * 2] = r[in.b];
+                    c.frame_args[(size_t)frame_of(nt) * 2 + 1] = r[in.dst];
                 }
                 if (fused) {
                     if (slot >= c.qcap) {
@@ -140,7 +140,38 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                 } else push_token(c, lq, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
                 break;
             }
-            case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)tag * 2 + in.imm - 1])); break;
+            case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)frame_of(tag) * 2 + in.imm - 1])); break;
+            case VM_ENTER: {                                        // Enter: <t, d> -> <0:t, d>
+                // a loop frame under the current tag: counter 0 in the high half of the new tag, the tag below kept whole
+                const uint32_t id = aggregated_inc(&c.ctl->frame_count.v);
+                if (id >= c.frame_cap) {
+                    set_status(c, RDF_ERR_FRAMES_FULL);
+                    return;
+                }
+                Frame f;
+                f.parent = frame_of(tag); f.label = LOOP_LABEL | (wave << FRAME_WAVE_SHIFT); f.arg = r[in.a];
+                c.frames[id] = f;
+                c.frame_ptag[id] = tag;
+                c.frame_args[(size_t)id * 2] = r[in.b];             // variables 1 and 2 live in the loop frame
+                c.frame_args[(size_t)id * 2 + 1] = r[in.dst];
+                trace_rec(c, id, r[in.a], 2, LOOP_LABEL, tag);
+                push_token(c, lq, wave, (uint64_t)id, r[in.a], (uint32_t)in.imm);
+                break;
+            }
+            case VM_NEXT: {                                         // Next: <n:t, d> -> <(n+1):t, d>
+                const int64_t v0 = r[in.a], v1 = r[in.b], v2 = r[in.dst];
+                c.frame_args[(size_t)frame_of(tag) * 2] = v1;
+                c.frame_args[(size_t)frame_of(tag) * 2 + 1] = v2;
+                const uint64_t nt = tag + (1ull << 32);
+                trace_rec(c, nt, v0, 3, LOOP_LABEL, 0);
+                push_token(c, lq, wave, nt, v0, (uint32_t)in.imm);
+                return;                                             // this iteration's token ends here
+            }
+            case VM_EXIT: {                                         // Exit: <n:t, d> -> <t, d>
+                trace_rec(c, tag, r[in.a], 4, LOOP_LABEL, 0);
+                tag = __ldcg(reinterpret_cast<const unsigned long long*>(&c.frame_ptag[frame_of(tag)]));
+                break;
+            }
             case VM_RET:
             case VM_PORT: {
                 const int64_t val = r[in.a];
@@ -154,7 +185,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                         uint32_t label;
                         uint64_t parent;
                         tag_pop(c, tag, label, parent);
-                        trace_rec(c, tag, c.H > 0 ? (int64_t)(uint32_t)val : val, 1, label, (uint32_t)parent);   // (vector value: its frame)
+                        trace_rec(c, tag, c.H > 0 ? (int64_t)(uint32_t)val : val, 1, label, parent);   // (vector value: its frame)
                         tag = parent;
                         const LabelInfo& L = sp.labels[label];
                         if (L.k_kind == K_RET) continue;           // the call was the caller's own output
@@ -761,8 +792,8 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.q0 = P.take<Token>(L.qcap);
     L.q1 = P.take<Token>(L.qcap);
     L.frames = P.take<Frame>(L.frame_cap);
-    L.frame_args = P.take<int64_t>(g->max_params > 1 ? (size_t)L.frame_cap * 2 : 0);
-    L.children = P.take<uint32_t>((size_t)L.frame_cap * g->max_calls_per_body);
+    L.frame_args = P.take<int64_t>(g->max_params > 1 || g->has_loops ? (size_t)L.frame_cap * 2 : 0);
+    L.frame_ptag = P.take<uint64_t>(g->has_loops ? (size_t)L.frame_cap : 0);
     L.pair_bytes = (size_t)L.frame_cap * g->match.size() * sizeof(Slot);
     L.pair_slots = P.take<char>(L.pair_bytes);
     L.port_val = P.take<int64_t>((size_t)L.frame_cap * g->n_ports_total);
@@ -871,12 +902,13 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.n_labels = (int)g->labels.size(); c.n_consts = (int)g->consts.size();
     c.label_bits = g->label_bits; c.tag_mode = g->tag_mode; c.result_entry_pc = g->result_entry_pc;
     c.n_ports_total = g->n_ports_total; c.K = g->max_calls_per_body;
+    c.has_loops = g->has_loops ? 1 : 0;
+    c.frame_ptag = g->has_loops ? reinterpret_cast<uint64_t*>(ws + L.frame_ptag) : nullptr;
     c.B = in->B; c.N = in->N; c.x = in->x;
     c.tree_root = in->tree_root; c.left = in->left; c.right = in->right; c.tok = in->tok; c.label = in->label;
     c.q[0] = reinterpret_cast<Token*>(ws + L.q0); c.q[1] = reinterpret_cast<Token*>(ws + L.q1);
     c.qcap = L.qcap;
     c.frames = reinterpret_cast<Frame*>(ws + L.frames);
-    c.children = reinterpret_cast<uint32_t*>(ws + L.children);
     c.frame_args = reinterpret_cast<int64_t*>(ws + L.frame_args);
     c.frame_cap = L.frame_cap;
     c.pair_slots = reinterpret_cast<Slot*>(ws + L.pair_slots);

@@ -37,6 +37,7 @@ struct Prog {
     const rdf_program* p;
     const rdf_function& fn(int i) const { return p->functions[i]; }
     const rdf_expr& ex(int f, int e) const { return p->functions[f].exprs[e]; }
+    bool is_loop(int f) const { return p->functions[f].kind == RDF_FN_LOOP; }
     // number of operand expressions: a call has one per formal parameter of its callee
     int n_ops(const rdf_expr& x) const {
         if (x.op == RDF_OP_CALL) return (x.imm >= 0 && x.imm < p->n_functions) ? p->functions[x.imm].n_params : 0;
@@ -55,6 +56,13 @@ void validate(const Prog& P) {
         const rdf_function& F = p->functions[f];
         require(F.exprs && F.n_exprs > 0 && F.n_params >= 0 && F.name, RDF_ERR_BAD_PROGRAM);
         require(F.root >= 0 && F.root < F.n_exprs, RDF_ERR_BAD_PROGRAM);
+        require(F.kind == RDF_FN_FUNCTION || F.kind == RDF_FN_LOOP, RDF_ERR_BAD_PROGRAM);
+        if (F.kind == RDF_FN_LOOP) {
+            require(f != p->result && F.n_params >= 1 && F.n_params <= 3, RDF_ERR_BAD_PROGRAM);
+            require(F.cond >= 0 && F.cond < F.n_exprs, RDF_ERR_BAD_PROGRAM);
+            for (int k = 0; k < F.n_params; ++k) require(F.next[k] >= 0 && F.next[k] < F.n_exprs, RDF_ERR_BAD_PROGRAM);
+            require(p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);     // the counter lives beside a frame id
+        }
         for (int e = 0; e < F.n_exprs; ++e) {
             const rdf_expr& x = F.exprs[e];
             require(arity_of(x.op) >= 0, RDF_ERR_BAD_PROGRAM);
@@ -84,7 +92,24 @@ void validate(const Prog& P) {
             state[e] = 2;
         };
         dfs(F.root);
+        if (F.kind == RDF_FN_LOOP) {
+            dfs(F.cond);
+            for (int k = 0; k < F.n_params; ++k) dfs(F.next[k]);
+        }
     }
+    // a loop stands in the graph of its caller: loops that contain themselves have no finite graph
+    std::vector<int> lstate(p->n_functions, 0);
+    std::function<void(int)> lwalk = [&](int f) {
+        require(lstate[f] != 1, RDF_ERR_BAD_PROGRAM);
+        if (lstate[f] == 2) return;
+        lstate[f] = 1;
+        const rdf_function& F = p->functions[f];
+        for (int e = 0; e < F.n_exprs; ++e)
+            if (F.exprs[e].op == RDF_OP_CALL && p->functions[F.exprs[e].imm].kind == RDF_FN_LOOP) lwalk((int)F.exprs[e].imm);
+        lstate[f] = 2;
+    };
+    for (int f = 0; f < p->n_functions; ++f)
+        if (p->functions[f].kind == RDF_FN_LOOP) lwalk(f);
 }
 
 // --------------------------------------------------------------- value kinds
@@ -141,6 +166,22 @@ void check_kinds(const Prog& P) {
             }
         };
         walk(F.root);
+        if (F.kind == RDF_FN_LOOP) {
+            walk(F.cond);
+            for (int k = 0; k < F.n_params; ++k) walk(F.next[k]);
+            require(kind(f, F.root) == 0 && kind(f, F.cond) == 0, RDF_ERR_UNSUPPORTED);      // integer loops
+            for (int k = 0; k < F.n_params; ++k) require(kind(f, F.next[k]) == 0, RDF_ERR_UNSUPPORTED);
+            // the condition and the value at exit are evaluated where the variables are at hand: no calls in them
+            std::function<bool(int)> has_call = [&](int e) {
+                const rdf_expr& x = F.exprs[e];
+                if (x.op == RDF_OP_CALL) return true;
+                const int ops[3] = {x.a, x.b, x.c};
+                for (int k = 0; k < P.n_ops(x); ++k)
+                    if (has_call(ops[k])) return true;
+                return false;
+            };
+            require(!has_call(F.cond) && !has_call(F.root), RDF_ERR_UNSUPPORTED);
+        }
     }
 }
 
@@ -195,14 +236,16 @@ struct Literal {
         Ctx root{0, {}, {}};
         in_node[f] = (int)nodes.size();
         for (int k = 0; k < F.n_params; ++k) root.param.push_back(Val(add(RDF_NODE_IN, -1, f, 0, 0, k), 0));
-        std::map<std::pair<int, int>, Val> memo;
-        std::map<int, uint32_t> used;
+        std::map<std::pair<int, int>, Val> memo;             // (expression, context): a context belongs to one definition
+        std::map<int, std::map<int, uint32_t>> used;         // per definition
         int next_ctx = 1;
-        std::function<Val(int, const Ctx&)> build = [&](int e, const Ctx& c) -> Val {
+        // fn: the definition whose expression e is built (f itself, or a loop that stands inside f's graph)
+        std::function<Val(int, int, const Ctx&)> build = [&](int fn, int e, const Ctx& c) -> Val {
             auto key = std::make_pair(e, c.id);
             auto it = memo.find(key);
             if (it != memo.end()) return it->second;
-            const rdf_expr& x = F.exprs[e];
+            const rdf_function& G = P.fn(fn);
+            const rdf_expr& x = G.exprs[e];
             Val v;
             if (x.op == RDF_OP_PARAM) {
                 v = c.param[x.imm];
@@ -210,13 +253,13 @@ struct Literal {
                 v = Val(add(RDF_NODE_CONST, -1, f, 0, x.imm), 0);
             } else if (x.op == RDF_OP_IF) {
                 // Figure 2: the predicate drives a Switch that routes the parameter to one side
-                Val pred = build(x.a, c);
-                uint32_t m = params_used(f, x.b, used) | params_used(f, x.c, used);
+                Val pred = build(fn, x.a, c);
+                uint32_t m = params_used(fn, x.b, used[fn]) | params_used(fn, x.c, used[fn]);
                 Ctx ct{next_ctx++, c.param, c.gates}, cf{next_ctx++, c.param, c.gates};
-                const bool conditional = params_used(f, x.a, used) != 0;
+                const bool conditional = params_used(fn, x.a, used[fn]) != 0;
                 ct.gates.push_back(Gate{pred, 0, conditional});
                 cf.gates.push_back(Gate{pred, 1, conditional});
-                for (int k = 0; k < F.n_params; ++k) {
+                for (int k = 0; k < G.n_params; ++k) {
                     if (!(m >> k & 1)) continue;
                     int sw = add(RDF_NODE_SWITCH, -1, f, 2);
                     connect(pred.first, pred.second, sw, 0);
@@ -224,16 +267,16 @@ struct Literal {
                     ct.param[k] = Val(sw, 0);
                     cf.param[k] = Val(sw, 1);
                 }
-                Val a = build(x.b, ct), b = build(x.c, cf);
+                Val a = build(fn, x.b, ct), b = build(fn, x.c, cf);
                 // a side that reads no parameter (a bare constant) would fire under every
                 // tag; route its value through a Switch so that only the chosen side is live
-                if (params_used(f, x.b, used) == 0) {
+                if (params_used(fn, x.b, used[fn]) == 0) {
                     int sw = add(RDF_NODE_SWITCH, -1, f, 2);
                     connect(pred.first, pred.second, sw, 0);
                     connect(a.first, a.second, sw, 1);
                     a = Val(sw, 0);
                 }
-                if (params_used(f, x.c, used) == 0) {
+                if (params_used(fn, x.c, used[fn]) == 0) {
                     int sw = add(RDF_NODE_SWITCH, -1, f, 2);
                     connect(pred.first, pred.second, sw, 0);
                     connect(b.first, b.second, sw, 1);
@@ -248,10 +291,10 @@ struct Literal {
                 const int ops[3] = {x.a, x.b, x.c};
                 Val in[3];
                 for (int k = 0; k < m; ++k) {
-                    in[k] = build(ops[k], c);
+                    in[k] = build(fn, ops[k], c);
                     // an argument that reads no parameter would feed its Call_i under every tag of
                     // this function: let the enclosing conditionals' Switches pass it on instead
-                    if (params_used(f, ops[k], used) != 0) continue;
+                    if (params_used(fn, ops[k], used[fn]) != 0) continue;
                     for (int gi = (int)c.gates.size() - 1; gi >= 0; --gi) {
                         const Gate& gt = c.gates[gi];
                         int sw = add(RDF_NODE_SWITCH, -1, f, 2);
@@ -261,15 +304,60 @@ struct Literal {
                         if (gt.conditional) break;
                     }
                 }
-                int n = add(NODE_FCALL, -1, f, m);
-                callee[n] = x.imm;
-                for (int k = 0; k < m; ++k) connect(in[k].first, in[k].second, n, k);
-                v = Val(n, 0);
+                if (P.is_loop((int)x.imm)) {
+                    // The while-loop of Figure 1 in place of the call: per loop-carried variable an Enter, a Merge fed by
+                    // Enter and Next, a Switch on the condition; the body on the true side ends in Next, the value on
+                    // the false side leaves through Exit.
+                    const int lp = (int)x.imm;
+                    const rdf_function& Lf = P.fn(lp);
+                    const int first_new = (int)nodes.size();
+                    Ctx cm{next_ctx++, {}, {}};
+                    std::vector<int> merges;
+                    for (int k = 0; k < m; ++k) {
+                        int en = add(RDF_NODE_ENTER, -1, f, 1, 0, k);
+                        connect(in[k].first, in[k].second, en, 0);
+                        int mg = add(RDF_NODE_MERGE, -1, f, 2, 0, k);
+                        connect(en, 0, mg, 0);
+                        merges.push_back(mg);
+                        cm.param.push_back(Val(mg, 0));
+                    }
+                    Val pred = build(lp, Lf.cond, cm);
+                    Ctx ct{next_ctx++, {}, {Gate{pred, 0, true}}}, cf{next_ctx++, {}, {Gate{pred, 1, true}}};
+                    for (int k = 0; k < m; ++k) {
+                        int sw = add(RDF_NODE_SWITCH, -1, f, 2);
+                        connect(pred.first, pred.second, sw, 0);
+                        connect(merges[k], 0, sw, 1);
+                        ct.param.push_back(Val(sw, 0));
+                        cf.param.push_back(Val(sw, 1));
+                    }
+                    for (int k = 0; k < m; ++k) {
+                        Val nv = build(lp, Lf.next[k], ct);
+                        int nx = add(RDF_NODE_NEXT, -1, f, 1, 0, k);
+                        connect(nv.first, nv.second, nx, 0);
+                        connect(nx, 0, merges[k], 1);
+                    }
+                    Val rv = build(lp, Lf.root, cf);
+                    int ex = add(RDF_NODE_EXIT, -1, f, 1);
+                    connect(rv.first, rv.second, ex, 0);
+                    // a constant inside the loop emits once per iteration, under the iteration's tag: fired by the Merge
+                    // (param = 1 marks it as fired by a loop, not by the entry Merge of the enclosing function)
+                    for (int n = first_new; n < (int)nodes.size(); ++n)
+                        if (nodes[n].kind == RDF_NODE_CONST && nodes[n].param == 0) {
+                            nodes[n].param = 1;
+                            connect(merges[0], 0, n, -1, 1);
+                        }
+                    v = Val(ex, 0);
+                } else {
+                    int n = add(NODE_FCALL, -1, f, m);
+                    callee[n] = x.imm;
+                    for (int k = 0; k < m; ++k) connect(in[k].first, in[k].second, n, k);
+                    v = Val(n, 0);
+                }
             } else {
                 int ar = arity_of(x.op);
                 int ops[3] = {x.a, x.b, x.c};
                 Val in[3];
-                for (int k = 0; k < ar; ++k) in[k] = build(ops[k], c);
+                for (int k = 0; k < ar; ++k) in[k] = build(fn, ops[k], c);
                 int n = add(RDF_NODE_OP, x.op, f, ar);
                 for (int k = 0; k < ar; ++k) connect(in[k].first, in[k].second, n, k);
                 v = Val(n, 0);
@@ -277,7 +365,7 @@ struct Literal {
             memo[key] = v;
             return v;
         };
-        Val r = build(F.root, root);
+        Val r = build(f, F.root, root);
         out_node[f] = add(RDF_NODE_OUT, -1, f, 1);
         connect(r.first, r.second, out_node[f], 0);
     }
@@ -287,7 +375,7 @@ struct Literal {
         const int nf = P.p->n_functions;
         std::set<int> removed;
         for (int f = 0; f < nf; ++f) {
-            if (f == P.p->result) continue;
+            if (f == P.p->result || P.is_loop(f)) continue;
             const int m = P.fn(f).n_params;
             // 1. number the nodes that call f: 0 .. n-1 (callers in `result` first)
             std::vector<int> calls;
@@ -338,7 +426,7 @@ struct Literal {
             }
             // Figure 3: constants of a called function fire on its entry Merge
             for (int n = 0; n < (int)nodes.size(); ++n)
-                if (nodes[n].kind == RDF_NODE_CONST && nodes[n].func == f) connect(in_node[f], 0, n, -1, 1);
+                if (nodes[n].kind == RDF_NODE_CONST && nodes[n].func == f && nodes[n].param == 0) connect(in_node[f], 0, n, -1, 1);
         }
         // drop replaced nodes, renumber
         std::vector<int> new_id(nodes.size(), -1);
@@ -364,7 +452,7 @@ void build_literal(const Prog& P, rdf_graph* g) {
     L.out_node.assign(nf, -1);
     L.build_function(P.p->result);          // `result` first, as the paper draws it
     for (int f = 0; f < nf; ++f)
-        if (f != P.p->result) L.build_function(f);
+        if (f != P.p->result && !P.is_loop(f)) L.build_function(f);      // (a loop stands inside the graphs that use it)
     L.transform();
 }
 
@@ -539,6 +627,61 @@ struct Lower {
         return (int)g->match.size() - 1;
     }
 
+    // The while-loop `lp` at this place of segment s, entered with the variables in registers r[0 .. m): Enter makes the
+    // loop frame and sends the first iteration to the loop head (a segment of its own, run once per iteration, with the
+    // variables in r0 .. r(m-1) like the parameters of a function entry).  There: the condition; while it holds, the next
+    // values (from this segment, or gathered in the token store when some of them wait for calls) and Next; when it
+    // fails, the value, Exit and what the enclosing code does with it (K).
+    void emit_loop(int s, int lp, const int r[3], const Cont& K) {
+        const rdf_function& Lf = P.fn(lp);
+        const int m = Lf.n_params;
+        g->has_loops = true;
+        const int head = new_seg();
+        segs[head].entry = true;
+        segs[head].nregs = std::max(1, m);
+        emit(s, VM_ENTER, r[2], r[0], r[1], -(head + 1));                  // (target fixed up at layout)
+        const int outer = cur_func;
+        cur_func = lp;
+        for (int k = 1; k < m; ++k) emit(head, VM_LDARG, k, 0, 0, k);        // variables 1, 2 live in the loop frame
+        const int c = value(head, Lf.cond);
+        const std::map<int, int> saved = segs[head].memo;                   // values of the body are not live after the exit
+        const size_t brz = segs[head].code.size();
+        emit(head, VM_BRZ, 0, c);
+        bool all_free = true;
+        for (int k = 0; k < m; ++k) all_free = all_free && call_free(lp, Lf.next[k]);
+        if (all_free) {
+            int nr[3] = {0, 0, 0};
+            for (int k = 0; k < m; ++k) nr[k] = value(head, Lf.next[k]);
+            emit(head, VM_NEXT, nr[2], nr[0], nr[1], -(head + 1));
+        } else if (m == 1) {
+            // the one next value waits for a call: Next fires where that value arrives
+            Cont K1{3};
+            K1.fn = [this, head](int s2, int rv) { emit(s2, VM_NEXT, 0, rv, 0, -(head + 1)); };
+            cps(head, Lf.next[0], K1);
+            emit(head, VM_HALT);
+        } else {
+            // some next value waits for a call: the m values meet in the token store under the iteration's tag
+            const int ks = new_seg();
+            int rr[3] = {0, 0, 0};
+            for (int k = 0; k < m; ++k) rr[k] = reg(ks);
+            emit(ks, VM_NEXT, rr[2], rr[0], rr[1], -(head + 1));
+            emit(ks, VM_HALT);
+            const int M = new_match(m, MATCH_INT, ks);
+            for (int k = 0; k < m; ++k) {
+                Cont Kk{2, M, k};
+                cps(head, Lf.next[k], Kk);
+            }
+            emit(head, VM_HALT);
+        }
+        segs[head].memo = saved;
+        segs[head].code[brz].imm = (int32_t)segs[head].code.size();
+        const int rv = value(head, Lf.root);
+        emit(head, VM_EXIT);
+        cur_func = outer;
+        apply(K, head, rv);
+        emit(head, VM_HALT);
+    }
+
     // start the evaluation of expression e in segment s; its value goes to K
     void cps(int s, int e, const Cont& K) {
         const int f = cur_func;
@@ -554,19 +697,41 @@ struct Lower {
                 const int ops[3] = {x.a, x.b, x.c};
                 bool all_free = true;
                 for (int k = 0; k < m; ++k) all_free = all_free && call_free(f, ops[k]);
+                const bool loop = P.is_loop(callee);
                 if (all_free) {
                     // the m Call_i nodes of this call site fire together: all arguments are at hand
                     int r[3] = {0, 0, 0};
                     for (int k = 0; k < m; ++k) r[k] = value(s, ops[k]);
+                    if (loop) {
+                        emit_loop(s, callee, r, K);
+                        break;
+                    }
                     int label = new_label(callee, K);
                     emit(s, VM_CALL, r[2], r[0], r[1], label);
                 } else if (m == 1) {
                     Cont K2{3};
-                    K2.fn = [this, callee, K](int s2, int r) {
+                    K2.fn = [this, callee, K, loop](int s2, int r) {
+                        if (loop) {
+                            const int rr[3] = {r, 0, 0};
+                            emit_loop(s2, callee, rr, K);
+                            return;
+                        }
                         int label = new_label(callee, K);
                         emit(s2, VM_CALL, 0, r, 0, label);
                     };
                     cps(s, x.a, K2);
+                } else if (loop) {
+                    // initial values that wait for calls meet in the token store; the loop is entered when the last has arrived
+                    int ks = new_seg();
+                    int r[3] = {0, 0, 0};
+                    for (int k = 0; k < m; ++k) r[k] = reg(ks);
+                    int M = new_match(m, MATCH_INT, ks);
+                    for (int k = 0; k < m; ++k) {
+                        Cont Kk{2, M, k};
+                        cps(s, ops[k], Kk);
+                    }
+                    emit_loop(ks, callee, r, K);
+                    emit(ks, VM_HALT);
                 } else {
                     // some argument is itself the result of a call: the arguments meet in the token store
                     // under the caller's tag, and the call fires when the last one has arrived
@@ -676,7 +841,7 @@ struct Lower {
         }
         std::vector<int> order{P.p->result};
         for (int f = 0; f < nf; ++f)
-            if (f != P.p->result) order.push_back(f);
+            if (f != P.p->result && !P.is_loop(f)) order.push_back(f);          // (loops are lowered where they stand)
         for (int f : order) {
             cur_func = f;
             calls_in_body = 0;
@@ -697,7 +862,7 @@ struct Lower {
         for (Seg& S : segs)
             for (VmInstr in : S.code) {
                 if (in.op == VM_BRZ || in.op == VM_JMP) in.imm += S.base;
-                if (in.op == VM_EMBED || in.op == VM_LEAF_LSTM) in.imm = segs[-in.imm - 1].base;
+                if (in.op == VM_EMBED || in.op == VM_LEAF_LSTM || in.op == VM_ENTER || in.op == VM_NEXT) in.imm = segs[-in.imm - 1].base;
                 g->code.push_back(in);
             }
         for (size_t i = 0; i < g->labels.size(); ++i) {
@@ -714,6 +879,7 @@ struct Lower {
             g->label_local.push_back(L.local_label);
         }
         if (g->has_vector_ops) require(P.p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);
+        require(!(g->has_vector_ops && g->has_loops), RDF_ERR_UNSUPPORTED);      // loops are integer programs here
         require(!(g->has_rnn && g->has_lstm), RDF_ERR_UNSUPPORTED);
     }
 };

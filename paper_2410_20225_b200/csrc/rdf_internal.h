@@ -31,6 +31,9 @@ enum VmOp : uint8_t {
     VM_OUT,        // r[a] is the program's output for this instance
     VM_EMBED,      // leaf state: queue E[r[a]] -> state of this frame; continue at segment imm next wave
     VM_LEAF_LSTM,  // same for the TreeLSTM leaf
+    VM_ENTER,      // Enter: new loop frame under the current tag, counter 0; variables r[a], r[b], r[dst]; loop head at imm
+    VM_NEXT,       // Next: counter + 1, variables r[a], r[b], r[dst], back to the loop head at imm (next wave)
+    VM_EXIT,       // Exit: the tag below the loop frame again; carries on in the same segment
     VM_HALT
 };
 
@@ -90,6 +93,7 @@ struct rdf_graph {
     bool has_vector_ops = false;
     bool has_rnn = false, has_lstm = false, has_loss = false;
     bool uses_tree = false;
+    bool has_loops = false;
     std::vector<std::string> func_names;
     // per-run state owned by the executor (rdf_exec.cu)
     void* dev = nullptr;

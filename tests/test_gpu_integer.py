@@ -258,6 +258,87 @@ def test_hash_store_probing_variants(probe, tight):
     assert e.value.code == -5
 
 
+def _decode_loop_trace(tr, B, label_local):
+    """Tags as lists (innermost first) from a frame-form trace of a program with loops: a frame is a call frame
+    (Call record: label, the tag below it) or a loop frame (Enter record); a tag = (iteration counter, frame)."""
+    below, kind_of, label = {}, {}, {}
+    for rec in tr[(tr["kind"] == 0) | (tr["kind"] == 2)]:
+        f = int(rec["tag"]) & 0xFFFFFFFF
+        below[f] = (int(rec["instance"]), int(rec["parent"]))           # (iteration counter of the tag below, its frame)
+        kind_of[f] = int(rec["kind"])
+        label[f] = label_local[int(rec["label"])] if rec["kind"] == 0 else None
+
+    def decode(it, f):
+        out = []
+        while f >= B:
+            out.append(label[f] if kind_of[f] == 0 else it)
+            it, f = below[f]
+        return f, tuple(out)
+    return decode
+
+
+LOOP_CASES = {"sum": (rdf.sum_loop_program, programs.sum_loop_program, direct.sum_to, [0, 1, 2, 5, 17, 40, 300]),
+              "pairs": (rdf.pairs_loop_program, programs.pairs_loop_program, direct.pairs, [0, 1, 2, 5, 9, 14]),
+              "primes": (rdf.primes_loop_program, programs.primes_loop_program, direct.primes, [0, 1, 2, 3, 10, 30, 97]),
+              "tri": (rdf.tri_program, programs.tri_program, direct.tri, [0, 1, 2, 6, 12])}
+
+
+@pytest.mark.parametrize("name", sorted(LOOP_CASES))
+def test_loops_values_and_tags(name):
+    """Tagged iteration on the device (Enter / Next / Exit share the frame table with Call / Return): values against
+    the plain definitions, and every Enter, Next, Exit and Call with its tag against the literal interpreter --
+    iteration counters on top of the enclosing tag, inner counter first for nested loops, a call's label on top of the
+    counter of the iteration that made it."""
+    make, oracle_prog, plain, xs = LOOP_CASES[name]
+    fs, r = make()
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    x = torch.tensor(xs, dtype=torch.int64, device="cuda")
+    y, tr = g.eval_int(x, max_invocations=20000, trace_capacity=400000)
+    assert y.tolist() == [plain(v) for v in xs]
+    st = g.stats()
+    assert st["status"] == 0
+    B = len(xs)
+    decode = _decode_loop_trace(tr, B, g.describe()["label_local"])
+    got = {k: set() for k in ("enter", "next", "exit", "call")}
+    for rec in tr:
+        it, f = int(rec["tag"]) >> 32, int(rec["tag"]) & 0xFFFFFFFF
+        inst, tag = decode(it, f)
+        if rec["kind"] == 2:
+            got["enter"].add((inst, tag))
+        elif rec["kind"] == 3:
+            got["next"].add((inst, tag))
+        elif rec["kind"] == 4:
+            got["exit"].add((inst, tag))
+        elif rec["kind"] == 0:
+            got["call"].add((inst, tag, int(rec["value"])))
+    og = transform.transform(oracle_prog())
+    want = {k: set() for k in got}
+    for b, v in enumerate(xs):
+        res = tagged.run(og, {0: v}, programs.INT_OPS, dead_tokens=False, max_firings=2_000_000)
+        assert res.value == y[b].item()
+        want["enter"] |= {(b, t) for t in res.enters}
+        want["next"] |= {(b, t) for t in res.nexts}
+        want["exit"] |= {(b, t) for t in res.exits}
+        want["call"] |= {(b, t, a[0]) for t, a in res.calls.items()}
+    assert got == want
+    # one wave per iteration (and per call level): a loop of n iterations needs at least n waves
+    assert st["waves"] >= max(xs)
+
+
+def test_loop_iteration_guard():
+    """A loop whose condition never fails is stopped by the wave limit, as a status code."""
+    r = rdf.Function("result", 1)
+    r.ret(r.call(1, r.param()))
+    lp = rdf.Function("forever", 1)
+    v = lp.param()
+    lp.loop(lp.lt(lp.const(0), lp.const(1)), [lp.add(v, lp.const(1))], v)
+    g = rdf.Graph([r, lp], 0, rdf.TAGS_FRAME)
+    g.set_limits(wave_limit=500)
+    with pytest.raises(rdf.RdfError) as e:
+        g.eval_int(torch.tensor([3, 4], dtype=torch.int64, device="cuda"), max_invocations=64)
+    assert e.value.code == -8
+
+
 def test_bad_arguments():
     fs, r = rdf.fib_program()
     g = rdf.Graph(fs, r)

@@ -33,6 +33,7 @@ def test_struct_layouts_match_the_header():
     assert C.sizeof(bd.rdf_expr) == 24 and C.sizeof(bd.rdf_trace_rec) == 32 and bd.TRACE_DTYPE.itemsize == 32
     assert C.sizeof(bd.rdf_batch) == 10 * 8 and C.sizeof(bd.rdf_node) == 32 and C.sizeof(bd.rdf_edge) == 20
     assert C.sizeof(bd.rdf_params) == 6 * 4 + 7 * 8 and bd.rdf_params.E.offset == 24
+    assert C.sizeof(bd.rdf_function) == 48 and bd.rdf_function.kind.offset == 28 and bd.rdf_function.next.offset == 36
 
 
 # ----------------------------------------------------------------- errors
@@ -124,7 +125,8 @@ OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.O
           bd.OP_EMBED: "leaf_rnn", bd.OP_CELL_RNN: "cell_rnn", bd.OP_LEAF_LSTM: "leaf_lstm",
           bd.OP_CELL_LSTM: "cell_lstm", bd.OP_NODE_LOSS: "pass_state"}
 KIND = {bd.NODE_IN: "in", bd.NODE_OUT: "out", bd.NODE_CONST: "const", bd.NODE_OP: "op", bd.NODE_SWITCH: "switch",
-        bd.NODE_MERGE: "merge", bd.NODE_ENTRY_MERGE: "merge", bd.NODE_CALL: "Call", bd.NODE_RETURN: "Return"}
+        bd.NODE_MERGE: "merge", bd.NODE_ENTRY_MERGE: "merge", bd.NODE_CALL: "Call", bd.NODE_RETURN: "Return",
+        bd.NODE_ENTER: "Enter", bd.NODE_EXIT: "Exit", bd.NODE_NEXT: "Next"}
 
 
 def _as_oracle_graph(desc):
@@ -237,6 +239,63 @@ def test_tree_net_literal_graph_runs_in_the_oracle(cell):
         got = res.value if cell == "rnn" else res.value[0]
         np.testing.assert_allclose(got, want[t], atol=1e-13)
         assert len(res.calls) == tb.tree_sizes()[t]
+
+
+LOOPS = {"sum": (rdf.sum_loop_program, programs.sum_loop_program, direct.sum_to, [0, 1, 5, 17]),
+         "pairs": (rdf.pairs_loop_program, programs.pairs_loop_program, direct.pairs, [0, 1, 4, 7]),
+         "primes": (rdf.primes_loop_program, programs.primes_loop_program, direct.primes, [0, 2, 3, 20]),
+         "tri": (rdf.tri_program, programs.tri_program, direct.tri, [0, 1, 3, 6])}
+
+
+@pytest.mark.parametrize("name", sorted(LOOPS))
+def test_loop_literal_graphs_run_in_the_oracle(name):
+    """The literal graph the library builds for a loop (Figure 1 in place of the call of the loop definition) is run
+    by the oracle's interpreter: the values of the plain definitions, and the same iteration and call tags as the
+    oracle's own graph of the program."""
+    make, oracle_prog, plain, xs = LOOPS[name]
+    fs, r = make()
+    d = _build(fs, r, rdf.TAGS_FRAME).describe()
+    kinds = [n["kind"] for n in d["nodes"]]
+    assert kinds.count(bd.NODE_ENTER) == kinds.count(bd.NODE_NEXT) and kinds.count(bd.NODE_ENTER) % 3 == 0
+    assert kinds.count(bd.NODE_EXIT) == kinds.count(bd.NODE_ENTER) // 3                 # three variables per loop, one value
+    g = _as_oracle_graph(d)
+    og = transform.transform(oracle_prog())
+    assert g.count("Enter") == og.count("Enter") and g.count("Next") == og.count("Next") and g.count("Exit") == og.count("Exit")
+    assert g.count("Call") == og.count("Call") and g.count("Return") == og.count("Return")
+    for x in xs:
+        res = tagged.run(g, {0: x}, programs.INT_OPS, dead_tokens=False, max_firings=500000)
+        want = tagged.run(og, {0: x}, programs.INT_OPS, dead_tokens=False, max_firings=500000)
+        assert res.value == want.value == plain(x)
+        assert sorted(res.nexts) == sorted(want.nexts) and sorted(res.enters) == sorted(want.enters)
+        assert sorted(res.exits) == sorted(want.exits)
+        assert {t: tuple(a[k] for k in sorted(a)) for t, a in res.calls.items()} == \
+            {t: tuple(a[k] for k in sorted(a)) for t, a in want.calls.items()}
+
+
+def test_bad_loops_are_rejected():
+    fs, r = rdf.sum_loop_program()
+    with pytest.raises(rdf.RdfError) as e:
+        _build(fs, r, rdf.TAGS_PATH)                       # the iteration counter lives beside a frame id
+    assert e.value.code == -11
+    fs, r = rdf.sum_loop_program()
+    fs[1].cond = 99
+    with pytest.raises(rdf.RdfError):
+        _build(fs, r, rdf.TAGS_FRAME)
+    # a call in the condition is not lowered
+    fs, r = rdf.primes_loop_program()
+    lp = fs[1]
+    lp.cond = lp.call(2, lp.param(1), lp.const(2))
+    with pytest.raises(rdf.RdfError) as e:
+        _build(fs, r, rdf.TAGS_FRAME)
+    assert e.value.code == -11
+    # a loop that contains itself has no finite graph
+    a = rdf.Function("result", 1)
+    a.ret(a.call(1, a.param()))
+    lp = rdf.Function("self", 1)
+    v = lp.param()
+    lp.loop(lp.lt(v, lp.const(3)), [lp.call(1, v)], v)
+    with pytest.raises(rdf.RdfError):
+        _build([a, lp], 0, rdf.TAGS_FRAME)
 
 
 def test_product_path_has_no_cpu_route():
