@@ -257,7 +257,8 @@ typedef struct {
     uint64_t cycles_schedule, cycles_batch, cycles_barrier;
     uint64_t cycles_bwd_frames, cycles_bwd_batch, cycles_bwd_barrier;
     uint32_t kernel_launches;    /* kernels of the library that the last call launched (host count; memsets and copies excluded) */
-    uint32_t reserved;
+    uint32_t clusters;           /* thread-block clusters that fired the cells of the last call (fp32 TreeRNN without a grid
+                                    barrier); 0 = the grid-wide operator kernel did */
 } rdf_stats;
 
 /* Bytes of device scratch rdf_eval (want_grad = 0) or rdf_grad (1) needs for

@@ -109,7 +109,7 @@ class rdf_stats(C.Structure):
                 ("max_probe", C.c_uint32), ("max_depth", C.c_uint32), ("cells", C.c_uint64), ("leaves", C.c_uint64),
                 ("cycles_schedule", C.c_uint64), ("cycles_batch", C.c_uint64), ("cycles_barrier", C.c_uint64),
                 ("cycles_bwd_frames", C.c_uint64), ("cycles_bwd_batch", C.c_uint64), ("cycles_bwd_barrier", C.c_uint64),
-                ("kernel_launches", C.c_uint32), ("reserved", C.c_uint32)]
+                ("kernel_launches", C.c_uint32), ("clusters", C.c_uint32)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

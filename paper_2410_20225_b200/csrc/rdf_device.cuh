@@ -77,6 +77,7 @@ struct Control {
     uint32_t all_leaves;          // backward: leaves seen so far
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     uint32_t max_height;          // largest height of a cell of this call (operator waves run height by height)
+    uint32_t h_split;             // clustered fp32 path: heights up to here are wide and fired by the whole grid, the rest cluster by cluster
     uint32_t n_depth_waves;       // scheduler waves that made calls = call depths of the run (length of the compacted wave_marks)
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
@@ -106,6 +107,10 @@ struct DevCtx {
     uint32_t qcap;
     // frames (frame-form tags)
     Frame*    frames;
+    uint32_t* finst;              // [frame_cap] fp32 tree networks: the instance (tree) an invocation belongs to, handed down
+                                  // from caller to callee; instances never exchange tokens, so the cells of different
+                                  // instances can be fired by different groups of thread blocks without a grid barrier
+    int       n_groups;           // thread-block clusters of the clustered operator kernel (0: not used)
     uint64_t* frame_ptag;         // [frame_cap] programs with loops: the full tag below a frame (its frame id and, when
                                   // that frame is a loop's, the iteration counter in the high half)
     int       has_loops;
@@ -192,6 +197,17 @@ struct DevCtx {
 };
 
 static const uint32_t LEAF_MARK = 0xFFFFFFFFu;
+
+// How many groups the ready cells are sorted into (by instance, then by height): the clusters of the clustered
+// operator kernel when the (group, height) table fits the space of the height table, else one group (all cells
+// by height, fired by the whole grid).  Every kernel of a call computes the same answer from the same words.
+// Shallow batches stay with the grid-wide kernel: a few dozen waves are too few for the second kernel to pay.
+static const uint32_t CLUSTER_MIN_HEIGHT = 64;
+__device__ __forceinline__ uint32_t cell_groups(const DevCtx& c) {
+    const uint64_t stride = (uint64_t)min(c.ctl->max_height, c.wave_cap) + 1u;
+    return c.n_groups > 1 && stride > CLUSTER_MIN_HEIGHT && (uint64_t)c.n_groups * stride <= (uint64_t)c.wave_cap + 2u
+               ? (uint32_t)c.n_groups : 1u;
+}
 static const uint32_t NO_ZDST = 0xFFFFFFFFu;
 
 // 64-bit fixed point, 2^-36 per unit (|sum| < 1.3e8, resolution 1.5e-11): integer additions commute exactly
@@ -358,6 +374,7 @@ __device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* lab
     f.parent = frame_of(tag); f.label = label | (wave << FRAME_WAVE_SHIFT); f.arg = arg;
     c.frames[id] = f;
     if (c.frame_ptag) c.frame_ptag[id] = tag;
+    if (c.finst) c.finst[id] = __ldcg(&c.finst[frame_of(tag)]);
     trace_rec(c, id, arg, 0, label, tag);
 }
 

@@ -31,7 +31,7 @@ struct SharedProgram {
 };
 
 struct ThreadStats {
-    uint32_t invocations = 0, tokens = 0, cells = 0, leaves = 0, max_depth = 0;
+    uint32_t invocations = 0, tokens = 0, cells = 0, leaves = 0, max_depth = 0, max_height = 0;
     StoreCounters sc;
 };
 
@@ -61,6 +61,7 @@ __device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, con
     it.out = (uint32_t)tag; it.l = (uint32_t)regs[0]; it.r = (uint32_t)regs[1];
     it.height = max((uint32_t)((uint64_t)regs[0] >> 32), (uint32_t)((uint64_t)regs[1] >> 32)) + 1u;
     c.cell_items[i] = it;
+    st.max_height = max(st.max_height, it.height);
     c.op_l[tag] = it.l;
     c.op_r[tag] = it.r;
     ++st.cells;
@@ -398,12 +399,13 @@ __device__ void rnn_leaf_rows(const DevCtx& c, uint32_t n_items) {
 // per-thread counters -> one set of atomics per warp
 __device__ __forceinline__ void flush_stats(const DevCtx& c, const ThreadStats& st) {
     unsigned long long v[7] = {st.invocations, st.tokens, st.cells, st.leaves, st.sc.inserts, st.sc.matches, st.sc.probes};
-    uint32_t mp = st.sc.max_probe, md = st.max_depth;
+    uint32_t mp = st.sc.max_probe, md = st.max_depth, mh = st.max_height;
     for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
         for (int k = 0; k < 7; ++k) v[k] += __shfl_xor_sync(0xffffffffu, v[k], o);
         mp = max(mp, __shfl_xor_sync(0xffffffffu, mp, o));
         md = max(md, __shfl_xor_sync(0xffffffffu, md, o));
+        mh = max(mh, __shfl_xor_sync(0xffffffffu, mh, o));
     }
     if ((threadIdx.x & 31) == 0) {
         atomicAdd(&c.ctl->invocations, v[0]); atomicAdd(&c.ctl->tokens, v[1]); atomicAdd(&c.ctl->cells, v[2]);
@@ -411,6 +413,7 @@ __device__ __forceinline__ void flush_stats(const DevCtx& c, const ThreadStats& 
         atomicAdd(&c.ctl->store_probes, v[6]);
         atomicMax(&c.ctl->max_probe, mp);
         atomicMax(&c.ctl->max_depth, md);
+        if (mh) atomicMax(&c.ctl->max_height, mh);        // (the operator waves run height by height)
     }
 }
 
@@ -560,6 +563,7 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
         Frame f;
         f.parent = LEAF_MARK; f.label = 0; f.arg = datum;          // (wave field 0: before the first wave)
         c.frames[b] = f;
+        if (c.finst) c.finst[b] = (uint32_t)b;
     }
     store_token(&c.q[0][b], tag, datum, (uint32_t)c.result_entry_pc);
     if (b == 0) {
@@ -640,20 +644,27 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
             lap(cyc_b);
         }
     } else {
-        // fp32 path: height by height (cell_items is the height-sorted list here: the launch passes cell_sorted in its place)
-        uint32_t first = 0;
-        const uint32_t top = min(c.ctl->max_height, c.wave_cap);
+        // fp32 path: height by height (cell_items is the sorted list here: the launch passes cell_sorted in its place).
+        // With the clustered path the list is sorted by (group of instances, height): this kernel fires the wide heights
+        // (1 .. h_split: every group's cells of the height, then one barrier) and leaves the rest to the clusters.
+        const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
+        const uint32_t top = groups > 1u ? min(c.ctl->h_split, stride - 1u) : stride - 1u;
         for (uint32_t w = 1; w <= top && alive; ++w) {
-            const uint32_t end = min(c.height_ends[w], c.work_cap);
-            if (end <= first) continue;                                  // (no cell of this height)
-            const uint32_t nc = end - first;
-            if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
-            // thin patches while they fit in two rounds over the grid, tiles for wide waves
-            else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
-                rnn_cell_thin(c, reinterpret_cast<float*>(&smem), wres, first, nc);      // 8 x 2H + 128 floats <= 26 KB
-            else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
-            first = end;
-            __syncthreads();
+            bool any = false;
+            for (uint32_t gq = 0; gq < groups; ++gq) {
+                const uint32_t first = min(c.height_ends[(size_t)gq * stride + w - 1], c.work_cap);
+                const uint32_t end = min(c.height_ends[(size_t)gq * stride + w], c.work_cap);
+                if (end <= first) continue;                              // (no cell of this height in the group)
+                const uint32_t nc = end - first;
+                any = true;
+                if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
+                // thin patches while they fit in two rounds over the grid, tiles for wide waves
+                else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
+                    rnn_cell_thin(c, reinterpret_cast<float*>(&smem), wres, first, nc);      // 8 x 2H + 128 floats <= 26 KB
+                else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
+                __syncthreads();
+            }
+            if (!any) continue;
             lap(cyc_c);
             alive = grid_barrier(c, &c.ctl->bar_ops.v, generation);
             lap(cyc_b);
@@ -666,31 +677,157 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
     }
 }
 
+// ===========================================================================
+// fp32 TreeRNN cells without a grid barrier: one thread-block cluster per group of instances
+// ===========================================================================
+// Tokens of different instances never meet (matching needs equal tags, and a tag belongs to one instance), so the cells
+// of different instances do not depend on one another.  The ready cells are sorted by (group of their instance,
+// height); a cluster of CLUSTER_CTAS blocks fires the cells of its group height by height and synchronises with the
+// hardware cluster barrier only -- a deep, thin recursion (a wave of a few dozen cells, thousands of waves) pays about
+// a microsecond per wave instead of a barrier over the whole grid.  The blocks of a cluster split the columns of W
+// (kept in shared memory for the whole kernel); a block step computes `cells_per_step` cells x its columns, thread =
+// (cell, column), operand rows staged in shared memory.  States travel between the blocks through global memory
+// (L2): the cluster barrier's release / acquire orders them.
+static const int CLUSTER_CTAS = 8;
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// CPC: columns of W per block (8 blocks x CPC >= H).  A block step fires CS = 256 / CPC cells: thread = (column, slice
+// of the contraction index), CS accumulators per thread -- a weight is read from shared memory once per step and an
+// operand word once per warp; the slices are added up through shared memory by thread = (cell, column).
+template <int CPC>
+__global__ void __launch_bounds__(256, 1) rdf_operator_cluster_kernel(const __grid_constant__ DevCtx c) {
+    constexpr int CS = 256 / CPC;              // cells per step = slices of k
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    // every block of the grid takes the same decision from the same words: no block of a cluster is left waiting
+    if (c.ctl->forward_status != 0 || cell_groups(c) <= 1u) return;
+    const int H = c.H, K2 = 2 * c.H;
+    const int rank = blockIdx.x % CLUSTER_CTAS, group = blockIdx.x / CLUSTER_CTAS;
+    const int j0 = rank * CPC;
+    float* wres = reinterpret_cast<float*>(dyn_smem);                  // [K2][CPC]: this block's columns of W
+    float* xs = wres + (size_t)K2 * CPC;                               // [2][CS][K2]: operand rows, double buffered
+    float* part = xs + (size_t)2 * CS * K2;                            // [CS slices][CS cells][CPC]: partial sums
+    uint32_t* s_out = reinterpret_cast<uint32_t*>(part + (size_t)CS * CS * CPC);   // [2][CS]: frames of the results
+    for (int q = threadIdx.x; q < K2 * CPC; q += blockDim.x) {
+        const int k = q / CPC, jj = q % CPC;
+        wres[q] = j0 + jj < H ? __ldg(&c.W[(size_t)(j0 + jj) * K2 + k]) : 0.f;
+    }
+    __syncthreads();
+    const uint32_t stride = min(c.ctl->max_height, c.wave_cap) + 1u, top = stride - 1u;
+    const uint32_t* ends = c.height_ends + (size_t)group * stride;      // ends[h]: end of (group, h); ends[0]: start of the group
+    const int jj = threadIdx.x % CPC, ks = threadIdx.x / CPC;           // column; slice of k (contraction) / cell (reduction)
+    const bool active = ks < CS;
+    const int klen = ((K2 + CS - 1) / CS + 3) & ~3, k_begin = ks * klen, k_end = min(K2, k_begin + klen);
+    const float bias = active && j0 + jj < H ? __ldg(&c.b[j0 + jj]) : 0.f;
+    // rows of a step: CS cells x K2 floats, fetched by all threads as 128-bit pieces
+    const int pieces = CS * (K2 / 4);
+    // (pre: the records of the step's cells when they were fetched ahead -- thread p holds the record of row p / (K2 / 4)
+    //  of its first piece -- else null)
+    auto stage = [&](int buf, uint32_t first, uint32_t n, const uint4* pre) {
+        float* dst = xs + (size_t)buf * CS * K2;
+        for (int p = threadIdx.x; p < pieces; p += blockDim.x) {
+            const int r = p / (K2 / 4), k = (p % (K2 / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if ((uint32_t)r < n) {
+                const uint4 it = pre && p == (int)threadIdx.x ? *pre : __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[first + r]));   // {out, l, r, height}
+                v = k < H ? ldcg4(c.arena + (size_t)it.y * H + k) : ldcg4(c.arena + (size_t)it.z * H + (k - H));
+                if (k == 0) s_out[buf * CS + r] = it.x;
+            }
+            *reinterpret_cast<float4*>(dst + (size_t)r * K2 + k) = v;
+        }
+    };
+    const uint32_t h0 = min(c.ctl->h_split, top);                     // (the grid-wide kernel fired heights 1 .. h0)
+    uint32_t begin = min(ends[h0], c.work_cap);
+    uint32_t end_next = top > h0 ? min(ends[h0 + 1], c.work_cap) : begin;
+    // the list is complete before the kernel starts: the record this thread needs first in the next wave is fetched a wave ahead
+    const int my_row = threadIdx.x / (K2 / 4);
+    uint4 rec_next = make_uint4(0u, 0u, 0u, 0u);
+    if (threadIdx.x < pieces && begin + my_row < end_next) rec_next = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[begin + my_row]));
+    for (uint32_t h = h0 + 1; h <= top; ++h) {
+        const uint32_t end = end_next;
+        if (h < top) end_next = min(ends[h + 1], c.work_cap);           // in flight during this wave
+        // the cells of (group, h), CS at a time; the next step's rows are fetched while this one computes
+        int buf = 0;
+        const uint4 rec = rec_next;
+        if (end > begin) stage(0, begin, min((uint32_t)CS, end - begin), &rec);
+        if (threadIdx.x < pieces && end + my_row < end_next) rec_next = __ldcg(reinterpret_cast<const uint4*>(&c.cell_items[end + my_row]));
+        for (uint32_t first = begin; first < end; first += CS) {
+            const uint32_t n = min((uint32_t)CS, end - first);
+            __syncthreads();                                            // rows of this step are in place, `part` is free
+            if (first + CS < end) stage(buf ^ 1, first + CS, min((uint32_t)CS, end - first - CS), nullptr);
+            if (active) {
+                float acc[CS];
+#pragma unroll
+                for (int q = 0; q < CS; ++q) acc[q] = 0.f;
+                const float* x = xs + (size_t)buf * CS * K2;
+                for (int k = k_begin; k < k_end; k += 4) {
+                    const float w0 = wres[(size_t)k * CPC + jj], w1 = wres[(size_t)(k + 1) * CPC + jj];
+                    const float w2 = wres[(size_t)(k + 2) * CPC + jj], w3 = wres[(size_t)(k + 3) * CPC + jj];
+#pragma unroll
+                    for (int q = 0; q < CS; ++q) {
+                        const float4 xv = *reinterpret_cast<const float4*>(x + (size_t)q * K2 + k);   // (one word for the whole warp)
+                        acc[q] = fmaf(xv.x, w0, fmaf(xv.y, w1, fmaf(xv.z, w2, fmaf(xv.w, w3, acc[q]))));
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < CS; ++q) part[((size_t)ks * CS + q) * CPC + jj] = acc[q];
+            }
+            __syncthreads();
+            if (active && (uint32_t)ks < n && j0 + jj < H) {            // thread = (cell ks, column jj): the slices added in order
+                float t = bias;
+#pragma unroll
+                for (int q = 0; q < CS; ++q) t += part[((size_t)q * CS + ks) * CPC + jj];
+                c.arena[(size_t)s_out[buf * CS + ks] * H + j0 + jj] = tanhf(t);
+            }
+            buf ^= 1;
+        }
+        begin = end;
+        __syncthreads();
+        cluster_sync_all();                                             // the states of height h are complete for the whole cluster
+    }
+}
+
+inline int cluster_cols_per_block(int H) { return H <= 64 ? 8 : H <= 128 ? 16 : H <= 256 ? 32 : 48; }
+inline size_t cluster_smem_bytes(int H) {
+    const int CPC = cluster_cols_per_block(H), CS = 256 / CPC, K2 = 2 * H;
+    return ((size_t)K2 * CPC + (size_t)2 * CS * K2 + (size_t)CS * CS * CPC) * sizeof(float) + 2 * CS * sizeof(uint32_t);
+}
+static const int CLUSTER_MAX_H = 384;
+
 // ---- cells grouped by height (between the scheduler and the operator kernel)
 // The scheduler finds a cell ready in the wave in which its second operand returns, which depends on how deep the
 // whole tree below it reaches; what the arithmetic needs is only that operands come first.  Grouping the cells by
 // height gives the smallest number of dependent operator waves (the largest height instead of about twice the depth).
+// (With the clustered operator kernel the cells are grouped by (cluster of their instance, height): bucket index
+// group * (max height + 1) + height; one group otherwise.  The largest height is known from the scheduler.)
+__device__ __forceinline__ uint32_t cell_bucket(const DevCtx& c, const CellItem& it, uint32_t groups, uint32_t stride) {
+    const uint32_t h = min(it.height, stride - 1u);
+    if (h == 0u) return 0u;                                                          // (0: not a cell)
+    return (groups > 1u ? __ldcg(&c.finst[it.out]) % groups : 0u) * stride + h;
+}
+
 __global__ void __launch_bounds__(256) rdf_height_count_kernel(const DevCtx c) {
     if (c.ctl->status != 0) return;
     const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
-    uint32_t top = 0;
+    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
     for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
         const uint32_t i = i0 + lane;
-        const uint32_t h = i < n ? min(c.cell_items[i].height, c.wave_cap) : 0u;      // (0: not a cell)
-        const unsigned peers = __match_any_sync(0xffffffffu, h);                      // one atomic per height and warp
-        if (h && (uint32_t)(__ffs(peers) - 1) == lane) atomicAdd(&c.height_ends[h], (uint32_t)__popc(peers));
-        top = max(top, h);
+        const uint32_t k = i < n ? cell_bucket(c, c.cell_items[i], groups, stride) : 0u;
+        const unsigned peers = __match_any_sync(0xffffffffu, k);                      // one atomic per bucket and warp
+        if (k && (uint32_t)(__ffs(peers) - 1) == lane) atomicAdd(&c.height_ends[k], (uint32_t)__popc(peers));
     }
-    for (int o = 16; o > 0; o >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
-    if (lane == 0 && top) atomicMax(&c.ctl->max_height, top);
 }
 
-// counts -> first position of each height (one block; heights 1 .. max_height)
+// counts -> first position of each bucket (one block; buckets 1 .. groups * (max height + 1) - 1)
 __global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c) {
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry;
     if (c.ctl->status != 0) return;
-    const uint32_t top = c.ctl->max_height, lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    const uint32_t top = cell_groups(c) * (min(c.ctl->max_height, c.wave_cap) + 1u) - 1u;
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
     if (threadIdx.x == 0) carry = 0;
     __syncthreads();
     for (uint32_t h0 = 1; h0 <= top; h0 += 1024) {
@@ -720,20 +857,35 @@ __global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c) {
     }
 }
 
-// every cell to its group; afterwards height_ends[h] is where group h ends (group h starts where group h - 1 ends)
+// every cell to its bucket; afterwards height_ends[k] is where bucket k ends (it starts where bucket k - 1 ends;
+// bucket group * stride + 0 is empty, so it ends where the previous group ends)
 __global__ void __launch_bounds__(256) rdf_height_scatter_kernel(const DevCtx c) {
     if (c.ctl->status != 0) return;
     const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
+    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
     for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
         const uint32_t i = i0 + lane;
         CellItem it = i < n ? c.cell_items[i] : CellItem{0u, 0u, 0u, 0u};
-        const uint32_t h = min(it.height, c.wave_cap);
-        const unsigned peers = __match_any_sync(0xffffffffu, h);
+        const uint32_t k = cell_bucket(c, it, groups, stride);
+        const unsigned peers = __match_any_sync(0xffffffffu, k);
         const int leader = __ffs(peers) - 1;
         uint32_t base = 0;
-        if (h && (uint32_t)leader == lane) base = atomicAdd(&c.height_ends[h], (uint32_t)__popc(peers));
+        if (k && (uint32_t)leader == lane) base = atomicAdd(&c.height_ends[k], (uint32_t)__popc(peers));
         base = __shfl_sync(0xffffffffu, base, leader);
-        if (h) c.cell_sorted[min(base + (uint32_t)__popc(peers & ((1u << lane) - 1u)), c.work_cap - 1u)] = it;
+        if (k) c.cell_sorted[min(base + (uint32_t)__popc(peers & ((1u << lane) - 1u)), c.work_cap - 1u)] = it;
+    }
+}
+
+// Which heights are wide enough for the whole grid (clustered path): the last height that has more than `threshold` cells
+// over all groups; the heights above it are left to the clusters.
+__global__ void __launch_bounds__(256) rdf_height_split_kernel(const DevCtx c, uint32_t threshold) {
+    if (c.ctl->status != 0) return;
+    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
+    if (groups <= 1u) return;
+    for (uint32_t h = 1 + blockIdx.x * blockDim.x + threadIdx.x; h < stride; h += gridDim.x * blockDim.x) {
+        uint32_t total = 0;
+        for (uint32_t gq = 0; gq < groups; ++gq) total += c.height_ends[(size_t)gq * stride + h] - c.height_ends[(size_t)gq * stride + h - 1];
+        if (total > threshold) atomicMax(&c.ctl->h_split, h);
     }
 }
 
@@ -794,6 +946,11 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.frames = P.take<Frame>(L.frame_cap);
     L.frame_args = P.take<int64_t>(g->max_params > 1 || g->has_loops ? (size_t)L.frame_cap * 2 : 0);
     L.frame_ptag = P.take<uint64_t>(g->has_loops ? (size_t)L.frame_cap : 0);
+    // fp32 TreeRNN: the cells are fired cluster by cluster of instances (no grid barrier); needs the instance of every frame
+    // (eligibility only: whether the device takes clusters is known at launch, and the workspace must not depend on it)
+    L.clustered = g->has_vector_ops && g->has_rnn && !g->has_lstm && H <= CLUSTER_MAX_H &&
+                  !(params->compute == RDF_BF16 && (H + 63) / 64 * 64 <= TC_HP_MAX && params->D == params->H);   // (not the tensor-core path)
+    L.finst = P.take<uint32_t>(L.clustered ? (size_t)L.frame_cap : 0);
     L.pair_bytes = (size_t)L.frame_cap * g->match.size() * sizeof(Slot);
     L.pair_slots = P.take<char>(L.pair_bytes);
     L.port_val = P.take<int64_t>((size_t)L.frame_cap * g->n_ports_total);
@@ -888,6 +1045,26 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
     S->device = dev;
+    // the clustered fp32 operator kernel: how many clusters of CLUSTER_CTAS blocks the device holds at once
+    S->n_clusters = 0;
+    {
+        const size_t smem = cluster_smem_bytes(CLUSTER_MAX_H);
+        bool ok = cudaFuncSetAttribute(rdf_operator_cluster_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster_smem_bytes(64)) == cudaSuccess &&
+                  cudaFuncSetAttribute(rdf_operator_cluster_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster_smem_bytes(128)) == cudaSuccess &&
+                  cudaFuncSetAttribute(rdf_operator_cluster_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cluster_smem_bytes(256)) == cudaSuccess &&
+                  cudaFuncSetAttribute(rdf_operator_cluster_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = CLUSTER_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((sms / CLUSTER_CTAS) * CLUSTER_CTAS); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int n = 0;
+        if (ok && cudaOccupancyMaxActiveClusters(&n, rdf_operator_cluster_kernel<48>, &cfg) == cudaSuccess)
+            S->n_clusters = std::min(n, sms / CLUSTER_CTAS);
+        else
+            cudaGetLastError();            // (no clusters: the grid-wide kernel is used)
+    }
     return RDF_OK;
 }
 
@@ -902,6 +1079,8 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.n_labels = (int)g->labels.size(); c.n_consts = (int)g->consts.size();
     c.label_bits = g->label_bits; c.tag_mode = g->tag_mode; c.result_entry_pc = g->result_entry_pc;
     c.n_ports_total = g->n_ports_total; c.K = g->max_calls_per_body;
+    c.finst = L.clustered ? reinterpret_cast<uint32_t*>(ws + L.finst) : nullptr;
+    c.n_groups = L.clustered && S->n_clusters > 1 ? S->n_clusters : 0;
     c.has_loops = g->has_loops ? 1 : 0;
     c.frame_ptag = g->has_loops ? reinterpret_cast<uint64_t*>(ws + L.frame_ptag) : nullptr;
     c.B = in->B; c.N = in->N; c.x = in->x;
@@ -1056,8 +1235,28 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
             rdf_mark(S, 3, stream);
             co.cell_items = c.cell_sorted;
             oargs[0] = (void*)&co;
+            S->last_clusters = c.n_groups > 1 ? c.n_groups : 0;
+            if (c.n_groups > 1) RDF_KERNEL(S, rdf_height_split_kernel<<<S->grid, 256, 0, stream>>>(c, 40u * (uint32_t)c.n_groups));
+            // the leaves and the wide heights with the whole grid ...
             RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
                                                 thin_resident_bytes(c.lstm, c.H), stream)));
+            if (c.n_groups > 1) {
+                // ... the narrow ones cluster by cluster of instances (the kernel leaves at once when the grouped table
+                // did not fit and the grid-wide kernel did all the work)
+                cudaLaunchConfig_t cfg = {};
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = CLUSTER_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                cfg.gridDim = dim3(c.n_groups * CLUSTER_CTAS); cfg.blockDim = dim3(256);
+                cfg.dynamicSmemBytes = cluster_smem_bytes(c.H); cfg.stream = stream;
+                cfg.attrs = at; cfg.numAttrs = 1;
+                switch (cluster_cols_per_block(c.H)) {
+                    case 8: RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_operator_cluster_kernel<8>, co))); break;
+                    case 16: RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_operator_cluster_kernel<16>, co))); break;
+                    case 32: RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_operator_cluster_kernel<32>, co))); break;
+                    default: RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_operator_cluster_kernel<48>, co))); break;
+                }
+            }
         }
         rdf_mark(S, 4, stream);
         RDF_KERNEL(S, rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root));
@@ -1145,6 +1344,7 @@ extern "C" int rdf_last_status(rdf_graph* g, rdf_stats* s) {
     s->cycles_schedule = h.cyc[0]; s->cycles_batch = h.cyc[1]; s->cycles_barrier = h.cyc[2];
     s->cycles_bwd_frames = h.cyc[3]; s->cycles_bwd_batch = h.cyc[4]; s->cycles_bwd_barrier = h.cyc[5];
     s->kernel_launches = S->launches;
+    s->clusters = (uint32_t)S->last_clusters;
     return h.status;
 }
 

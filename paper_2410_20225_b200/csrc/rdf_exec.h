@@ -47,6 +47,8 @@ static const int LIST_SEG = 2048;            // frames per segment of the list k
 struct ExecState {
     int device = -1;
     int grid = 0;
+    int last_clusters = 0;       // clusters the last call used
+    int n_clusters = 0;          // clusters of the clustered fp32 operator kernel that fit the device at once (0: none)
     int clock_khz = 0;
     void* last_ctl = nullptr;
     cudaStream_t last_stream = nullptr;
@@ -75,10 +77,10 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 }
 
 struct Layout {
-    size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, frame_ptag, pair_slots, port_val, arrived, table, cell_items,
+    size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, frame_ptag, finst, pair_slots, port_val, arrived, table, cell_items,
         leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, dw_partial, de_fix, head_fix, rank_tmp, total;
     uint32_t qcap, frame_cap, work_cap, wave_cap, cells_cap;
-    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad, repro;
+    int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad, repro, clustered;
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes, pair_bytes;
 };
