@@ -97,8 +97,12 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- workloads
-def load(k, seed, fib_batch=None):
-    cfg = workloads.config(k, seed=seed, B=fib_batch) if (k == 1 and fib_batch) else workloads.config(k, seed=seed)
+def load(k, seed, fib_batch=None, over=None):
+    """Workload k; `over`: generator arguments that replace the named configuration's (reduced cases for profiling)."""
+    over = dict(over or {})
+    if k == 1 and fib_batch:
+        over["B"] = fib_batch
+    cfg = workloads.config(k, seed=seed, **over)
     if cfg["kind"] == "fib":
         cfg["N"] = int(sum(2 * fib_iter(int(n) + 1) - 1 for n in cfg["x"]))
     else:
@@ -478,15 +482,20 @@ def kernel_table(case, phase_ms, pk, fp32_peak, traffic, workload):
     Hp = 64 * ((H + 63) // 64)
     lstm = case.cell == "lstm"
     mm = "tensor" if case.use_tc else "alu"
-    add("rdf_height_count/scan/scatter_kernel", "group", "hbm", 48.0 * C, "16 B cell record read twice and written once")
+    if case.use_tc:       # tensor-core path: the cells listed by call depth (the same lists serve the gradient pass)
+        add("rdf_list_count/scan/fill/ends/compact/zdst_kernel", "group", "hbm", N * 32.0 + C * 24.0,
+            "operand ids and frame records read (two passes), cell lists and operand-row destinations written")
+    else:
+        add("rdf_height_count/scan/scatter_kernel", "group", "hbm", 48.0 * C, "16 B cell record read twice and written once")
     add("rdf_operator_kernel", "operators", mm, case.flops_fwd(),
         "cell contraction 2*2H*H per cell" + (" (x5 gates) + leaf projection 2*D*3H per leaf" if lstm else ""))
     add("rdf_gather_roots_kernel", "roots", "hbm", tb.B * H * (4.0 + (2 if case.use_tc and not lstm else 4)), "root rows read and written")
     if case.grad:
         rowbytes = Hp * 2 if case.use_tc else H * 4 * (2 if lstm else 1)
         add("rdf_loss_heads_kernel", "loss", "hbm", float(N) * (rowbytes + 32), "one state row read + 32 B of dlog written per invocation")
-        add("rdf_list_count/scan/fill/ends_kernel", "lists", "hbm", N * 28.0 + C * 24.0,
-            "operand ids and frame records read (two passes), cell lists written")
+        if not case.use_tc:
+            add("rdf_list_count/scan/fill/ends/compact_kernel", "lists", "hbm", N * 28.0 + C * 24.0,
+                "operand ids and frame records read (two passes), cell lists written")
         bwd = C * 2.0 * H * (2 * H) * (5 if lstm else 1)
         add("rdf_backward_kernel", "backward", mm, bwd, "operand-gradient contraction W^T dz: 2*H*2H per cell" + (" (x5 gates)" if lstm else ""))
         dw = bwd + (Lf * 2.0 * H * 3 * H if lstm else 0.0)
@@ -520,7 +529,7 @@ def run(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # every rank processes a batch of its own (instances never exchange tokens): weak scaling
-    cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch)
+    cfg = load(args.workload, rank_seed(args.seed, rank), args.fib_batch, args.override)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
     case = Case(rdf, torch, cfg, cfg.get("grad", False), dist, args.store, args.hash_load)
 
@@ -551,10 +560,10 @@ def run(args):
     if world == 1 and not args.no_table:
         table = []
         for k in sorted(WORKLOAD_NAMES):
-            c_k = cfg if k == args.workload and not args.fib_batch else load(k, args.seed)
+            c_k = cfg if k == args.workload and not args.fib_batch and not args.override else load(k, args.seed)
             passes = [False, True] if c_k.get("grad") else [False]
             for grad in passes:
-                if k == args.workload and grad == bool(cfg.get("grad", False)) and not args.fib_batch:
+                if k == args.workload and grad == bool(cfg.get("grad", False)) and not args.fib_batch and not args.override:
                     res, cs = head, case
                 else:
                     cs = Case(rdf, torch, c_k, grad)
@@ -571,6 +580,38 @@ def run(args):
                               "dominant": {"kernel": top["kernel"], "bound": top["bound"], "frac": top["frac"]}})
                 del cs
                 torch.cuda.empty_cache()
+        # the hash token store with warp-cooperative probes, and the scaled run (131072 calls) that takes the store out of L2
+        for label, fb, store in (("1 (warp-cooperative probes)", None, "warp"), ("1 scaled: 131072 calls", 131072, "thread"),
+                                 ("1 scaled: 131072 calls (warp-cooperative probes)", 131072, "warp")):
+            c_k = load(1, args.seed, fb)
+            cs = Case(rdf, torch, c_k, False, store=store)
+            res = time_case(cs, 5, 3, flush, e2e_steps=3)
+            kt = kernel_table(cs, res["phase_ms"], pk, fp32_peak, traffic, 1)
+            table.append({"workload": label, "pass": "forward", "dtype": cs.dtype, "invocations_per_step": c_k["N"],
+                          "ms_per_step": res["ms_per_step"], "value": res["value"], "e2e": res["e2e"]["value"], "unit": UNIT,
+                          "waves": res["stats"]["waves"], "waves_backward": 0,
+                          "kernels": [{"kernel": r["kernel"], "ms": round(r["ms"], 4), "bound": r["bound"], "achieved": r["achieved"],
+                                       "unit": r["unit"], "frac": r["frac"]} for r in kt],
+                          "dominant": {"kernel": kt[0]["kernel"], "bound": kt[0]["bound"], "frac": kt[0]["frac"]}})
+            del cs
+            torch.cuda.empty_cache()
+
+    # ---- the same step with reproducible sums (tensor-core path only)
+    repro = None
+    if world == 1 and case.grad and case.use_tc and not args.no_table:
+        rep_times = []
+        for k in range(3 + min(args.steps, 10)):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            case.g.grad_trees(case.dt, case.dp, case.compute, check=False, grads=case.grads, loss=case.loss, h_root=case.h_root,
+                              reproducible=True)
+            e1.record()
+            e1.synchronize()
+            if k >= 3:
+                rep_times.append(e0.elapsed_time(e1))
+        case.g.stats()
+        repro = {"ms_per_step": sum(rep_times) / len(rep_times), "what": "rdf_grad with rdf_params.reproducible = 1: bit-identical gradients and loss on every call"}
 
     cpu, cpu_all = None, None
     if not args.no_cpu_baseline:
@@ -586,6 +627,7 @@ def run(args):
         "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": case.dtype, "data": "synthetic",
         "config": {"workload": WORKLOAD_NAMES[args.workload] + (f" [scaled: {args.fib_batch} calls]" if args.fib_batch and args.workload == 1 else "")
+                   + (f" [reduced: {args.override}]" if args.override else "")
                    + (f" [store: {args.store} probes" + (f", load {args.hash_load}" if args.hash_load else "") + "]" if args.workload == 1 else ""),
                    "invocations_per_step": case.N, "instances": cfg.get("B") or cfg["trees"].B,
                    "pass": "forward+backward" if cfg.get("grad") else "forward",
@@ -593,6 +635,7 @@ def run(args):
         "clocks": clk,
         "e2e": head["e2e"],
         "e2e_all_outputs": head.get("e2e_all_outputs"),
+        "reproducible_mode": repro,
         "gpu_launches": st["kernel_launches"] * args.steps,          # counted by the library at every launch of the call
         "roofline": roof,
         "kernels": kernels,
@@ -638,9 +681,13 @@ def main():
                     help="workload 1: probing of the hash token store (per thread / warp-cooperative)")
     ap.add_argument("--hash-load", type=float, default=None,
                     help="workload 1: size the hash table for this load factor (parked operands / slots, rounded to a power of two)")
+    ap.add_argument("--override", action="append", default=[], metavar="KEY=INT",
+                    help="replace an argument of the workload generator (B, V, H, chains, chain_depth, perfect, perfect_height): "
+                         "reduced cases for profiler captures; the line says so in config.workload")
     ap.add_argument("--fib-batch", type=int, default=None,
                     help="workload 1 only: number of independent fib calls (default 1024, the named configuration)")
     args = ap.parse_args()
+    args.override = {kv.split("=")[0]: int(kv.split("=")[1]) for kv in args.override}
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
