@@ -218,6 +218,46 @@ def treelstm_hc(tb, P, v, store=None):
     return h, c
 
 
+def topdown(params, tok, depth_limit, log=None):
+    """Recursion whose *shape* depends on the values it computes -- the kind of definition Section 6.2 closes
+    with (a tree generated top-down by the model cannot be written as an iteration over a given structure):
+
+        result(tok)  = expand(E[tok], 0)
+        expand(h, d) = h                                                 if d >= D or gate(h)
+                     = cell(expand(left(h), d+1), expand(right(h), d+1))   otherwise
+        left(h)  = tanh(W[:, :H] h + b)      right(h) = tanh(W[:, H:] h + b)
+        gate(h)  = W_s[0] . h + b_s[0] > 0
+
+    (the cell and the halves of W are those of the TreeRNN; the paper gives no equations for such a model, these
+    are the smallest ones that make the Switch of `expand` read a vector value).  Returns the state of the
+    generated tree's root.  `log`, if a dict, receives "expand" / "child" invocation counts and "margin": the
+    smallest |W_s[0].h + b_s[0]| over the invocations whose gate decided (d < D) -- how far the nearest decision
+    was from flipping."""
+    P = _f64(params)
+    H = P["W"].shape[0]
+    WL, WR = P["W"][:, :H], P["W"][:, H:]
+    if log is not None:
+        log.setdefault("expand", 0)
+        log.setdefault("child", 0)
+        log.setdefault("margin", np.inf)
+
+    def expand(h, d):
+        g = float(P["W_s"][0] @ h + P["b_s"][0])
+        if log is not None:
+            log["expand"] += 1
+            if d < depth_limit:
+                log["margin"] = min(log["margin"], abs(g))
+        if d >= depth_limit or g > 0:
+            return h
+        if log is not None:
+            log["child"] += 2
+        hl = np.tanh(WL @ h + P["b"])
+        hr = np.tanh(WR @ h + P["b"])
+        return rnn_cell(P, expand(hl, d + 1), expand(hr, d + 1))
+
+    return deep(expand, P["E"][tok], 0)
+
+
 def node_loss(h, P, label):
     """-log softmax(W_s h + b_s)[label]"""
     z = P["W_s"] @ h + P["b_s"]

@@ -13,7 +13,9 @@ Programs:
     tanh(W [h(l); h(r)] + b) otherwise; the binary TreeLSTM; both optionally
     returning the pair (state, summed per-node loss).  The paper's Section 6.2
     names the TreeRNN sentiment model without giving its equations; the cell
-    forms are the ones fixed by the workload list.
+    forms are the ones fixed by the workload list;
+  * a top-down recursion whose Switch reads a vector value (`topdown_program`):
+    the data-dependent recursion that Section 6.2's last paragraph points to.
 
 Only tests, the smoke check and the CPU-baseline leg of the benchmark may
 import anything under `oracle/`.
@@ -274,6 +276,49 @@ def tree_net_program(cell: str, with_loss: bool):
     pair = f.op("pack", x, f.op("+", f.op("node_loss", x, e), below))
     f.output(f.merge(leaf_pair, pair))
     return [r, f]
+
+
+def topdown_program():
+    """The top-down recursion of `direct.topdown` as a set of function graphs:
+
+        result(v)    = expand(seed(v), 0)          seed(v) = leaf_rnn(tok v)
+        expand(h, d) = Merge( h,  cell_rnn(expand(left(h), d+1), expand(right(h), d+1)) )
+                       with the Switches of h and d driven by  stop(h, d) = at_limit(d) or gate(h)
+        left(h) = child_l(h)        right(h) = child_r(h)
+
+    The predicate of the Switch reads the vector h: which Call nodes fire is decided by values computed during
+    the run."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("expand", r.call("seed", r.param(0)), r.op("zero", r.param(0))))
+    s = FunctionGraph("seed", 1)
+    s.output(s.op("leaf_rnn", s.op("tok", s.param(0))))
+    f = FunctionGraph("expand", 2)
+    h, d = f.param(0), f.param(1)
+    p = f.op("or", f.op("at_limit", d), f.op("gate", h))
+    h_t, h_e = f.switch(p, h)
+    _, d_e = f.switch(p, d)
+    d1 = f.op("add1", d_e)
+    a = f.call("expand", f.call("left", h_e), d1)
+    b = f.call("expand", f.call("right", h_e), d1)
+    f.output(f.merge(h_t, f.op("cell_rnn", a, b)))
+    fl = FunctionGraph("left", 1)
+    fl.output(fl.op("child_l", fl.param(0)))
+    fr = FunctionGraph("right", 1)
+    fr.output(fr.op("child_r", fr.param(0)))
+    return [r, s, f, fl, fr]
+
+
+def topdown_ops(tb, params, depth_limit):
+    """Operator table for `topdown_program` (fp64)."""
+    ops = tree_net_ops(tb, params, "rnn")
+    P = {k: np.asarray(v, dtype=np.float64) for k, v in params.items()}
+    H = P["W"].shape[0]
+    ops["child_l"] = lambda h: np.tanh(P["W"][:, :H] @ h + P["b"])
+    ops["child_r"] = lambda h: np.tanh(P["W"][:, H:] @ h + P["b"])
+    ops["gate"] = lambda h: bool(P["W_s"][0] @ h + P["b_s"][0] > 0)
+    ops["at_limit"] = lambda d: d >= depth_limit
+    ops["or"] = lambda a, b: bool(a or b)
+    return ops
 
 
 def sigmoid(x):

@@ -15,6 +15,8 @@ from .gen import (  # noqa: F401
     perfect_tree_shape,
     random_split_shape,
     subset_trees,
+    topdown_batch,
+    topdown_params,
     tree_batch_from_shapes,
     treelstm_params,
     treernn_params,

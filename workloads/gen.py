@@ -208,6 +208,27 @@ def treelstm_params(seed: int, V: int, D: int, H: int, n_classes: int = 5, bf16:
     return p
 
 
+def topdown_params(seed: int, V: int, H: int, stop_bias: float = -0.3):
+    """Parameters for the top-down recursion (a tree grown from a seed vector; a gate on the state decides at
+    every node whether it is expanded): the TreeRNN parameter set with a seed table E ~ N(0, 1), W scaled by 2 so
+    that the child states keep their spread from level to level, and b_s[0] = stop_bias so that a node is expanded
+    a little more often than not (the generated trees neither die out at once nor fill every level)."""
+    r = _rng(seed, 7)
+    return {
+        "E": r.standard_normal((V, H)).astype(np.float32),
+        "W": (2.0 * _xavier(r, H, 2 * H)).astype(np.float32),
+        "b": np.zeros(H, dtype=np.float32),
+        "W_s": _xavier(r, 5, H),
+        "b_s": np.array([stop_bias, 0, 0, 0, 0], dtype=np.float32),
+    }
+
+
+def topdown_batch(seed: int, B: int, V: int) -> TreeBatch:
+    """B seeds: single-node trees whose token selects the seed row."""
+    one = (np.full(1, -1, dtype=np.int32), np.full(1, -1, dtype=np.int32))
+    return tree_batch_from_shapes([one] * B, seed, vocab=V)
+
+
 # --------------------------------------------------------------------------
 # the five named workloads
 # --------------------------------------------------------------------------
