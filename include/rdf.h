@@ -75,6 +75,13 @@ typedef enum {
                             marks the invocation as a term of the summed per-node
                             softmax cross-entropy loss that rdf_grad differentiates */
     RDF_OP_REM,          /* a, b -> remainder of the truncating division a / b (sign of a); 0 when b == 0 */
+    /* Recursion driven by vector values (Section 6.2, last paragraph: a structure generated top-down by the model).
+     * A program that uses one of the three operators below is executed with token scheduling and vector operators
+     * interleaved wave by wave, because its Switches read states: fp32, RDF_TAGS_FRAME, rdf_eval only, H <= 256.
+     * In such programs a formal parameter may be vector-valued (a call passes the state on by reference). */
+    RDF_OP_CHILD_L,      /* a = state -> tanh(W[:, 0:H] a + b): the state of a node's left child, from its own */
+    RDF_OP_CHILD_R,      /* a = state -> tanh(W[:, H:2H] a + b): the right child                              */
+    RDF_OP_GATE,         /* a = state -> integer 1 if W_s[0] . a + b_s[0] > 0 else 0 (fp32 arithmetic)        */
     RDF_OP__COUNT
 } rdf_opcode;
 

@@ -21,7 +21,8 @@ ERRORS = {
     -9: "RDF_ERR_TIMEOUT", -10: "RDF_ERR_CUDA", -11: "RDF_ERR_UNSUPPORTED",
 }
 (OP_PARAM, OP_CONST, OP_ADD, OP_SUB, OP_MUL, OP_MAX, OP_LT, OP_EQ, OP_IF, OP_CALL, OP_IS_LEAF, OP_LEFT, OP_RIGHT,
- OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS, OP_REM) = range(20)
+ OP_TOK, OP_EMBED, OP_CELL_RNN, OP_LEAF_LSTM, OP_CELL_LSTM, OP_NODE_LOSS, OP_REM, OP_CHILD_L, OP_CHILD_R,
+ OP_GATE) = range(23)
 TAGS_PATH, TAGS_FRAME = 0, 1
 F32, BF16 = 0, 1
 (NODE_IN, NODE_OUT, NODE_CONST, NODE_OP, NODE_SWITCH, NODE_MERGE, NODE_ENTRY_MERGE, NODE_CALL, NODE_RETURN, NODE_ENTER,
@@ -204,6 +205,9 @@ class Function:
     def leaf_lstm(self, t): return self._add(OP_LEAF_LSTM, t)
     def cell_lstm(self, a, b): return self._add(OP_CELL_LSTM, a, b)
     def node_loss(self, s, v): return self._add(OP_NODE_LOSS, s, v)
+    def child_l(self, h): return self._add(OP_CHILD_L, h)
+    def child_r(self, h): return self._add(OP_CHILD_R, h)
+    def gate(self, h): return self._add(OP_GATE, h)
 
     def ret(self, e):
         self.root = e
@@ -271,6 +275,28 @@ def tak_program(y_const=12, z_const=6):
     c = f.call(1, f.sub(z, one), x, y)
     f.ret(f.if_(f.lt(y, x), f.call(1, a, b, c), z))
     return [r, f], 0
+
+
+def topdown_program(depth_limit):
+    """Recursion shaped by the values it computes (Section 6.2, last paragraph):
+    result(v) = expand(seed(v), 0); seed(v) = EMBED(TOK(v));
+    expand(h, d) = h if d >= D or GATE(h) else CELL_RNN(expand(left(h), d+1), expand(right(h), d+1));
+    left(h) = CHILD_L(h); right(h) = CHILD_R(h)."""
+    RESULT, SEED, EXPAND, LEFT, RIGHT = range(5)
+    r = Function("result", 1)
+    r.ret(r.call(EXPAND, r.call(SEED, r.param()), r.const(0)))
+    s = Function("seed", 1)
+    s.ret(s.embed(s.tok(s.param())))
+    f = Function("expand", 2)
+    h, d = f.param(0), f.param(1)
+    d1 = f.add(d, f.const(1))
+    stop = f.max(f.lt(f.const(depth_limit - 1), d), f.gate(h))
+    f.ret(f.if_(stop, h, f.cell_rnn(f.call(EXPAND, f.call(LEFT, h), d1), f.call(EXPAND, f.call(RIGHT, h), d1))))
+    fl = Function("left", 1)
+    fl.ret(fl.child_l(fl.param()))
+    fr = Function("right", 1)
+    fr.ret(fr.child_r(fr.param()))
+    return [r, s, f, fl, fr], RESULT
 
 
 def sum_loop_program():

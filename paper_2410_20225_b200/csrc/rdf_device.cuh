@@ -33,6 +33,8 @@ struct __align__(16) Frame {
     int64_t  arg;
 };
 static const uint32_t FRAME_LABEL_MASK = 0xFFu;
+static const uint32_t CHILD_L_MARK = 0xFFFFFFFDu, CHILD_R_MARK = 0xFFFFFFFEu;   // CellItem.r of a unary vector operator (no frame has these ids)
+static const int INTERLEAVED_MAX_H = 256;          // interleaved execution stages 2 H floats per warp in shared memory
 static const uint32_t LOOP_LABEL = 0xFFu;     // label field of a loop frame (Enter), which no call site has
 // A tag in frame form: the frame id in the low half; for a loop frame the iteration counter in the high half
 // (Section 5.1: a tag is a pair of an iteration number and a pointer into the frame stack).

@@ -258,6 +258,39 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                 else store_token(&c.q[(wave + 1) & 1][slot], tag, (int64_t)tag, (uint32_t)in.imm);
                 break;
             }
+            case VM_VGATE: {
+                // An integer read off a vector value: W_s[0] . h + b_s[0] > 0 in fp32, terms added in index order.  The
+                // state was written by the operator phase of an earlier wave (any block): read through L2.
+                const uint32_t ref = (uint32_t)r[in.a];
+                if (ref >= c.frame_cap) {
+                    set_status(c, RDF_ERR_BAD_ARG);
+                    return;
+                }
+                const float* h = c.arena + (size_t)ref * c.S;
+                float acc = c.b_s[0];
+                for (int k = 0; k < c.H; ++k) acc = fmaf(__ldg(&c.W_s[k]), __ldcg(&h[k]), acc);
+                r[in.dst] = acc > 0.f;
+                break;
+            }
+            case VM_VCHILD: {
+                // a unary vector operator: queued like a cell whose second operand is the marker of the operator
+                uint32_t i, slot = 0;
+                aggregated_inc2(&c.ctl->cell_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
+                if (i >= c.work_cap || slot >= c.qcap) {
+                    set_status(c, RDF_ERR_QUEUE_FULL);
+                    return;
+                }
+                CellItem it;
+                it.out = (uint32_t)tag; it.l = (uint32_t)r[in.a]; it.r = in.dst ? CHILD_R_MARK : CHILD_L_MARK;
+                it.height = (uint32_t)((uint64_t)r[in.a] >> 32) + 1u;
+                c.cell_items[i] = it;
+                st.max_height = max(st.max_height, it.height);
+                c.op_l[tag] = it.l;
+                c.op_r[tag] = it.r;
+                ++st.cells;
+                store_token(&c.q[(wave + 1) & 1][slot], tag, (int64_t)(((uint64_t)it.height << 32) | (uint32_t)tag), (uint32_t)in.imm);
+                break;
+            }
             default:   // VM_HALT
                 return;
         }
@@ -549,6 +582,92 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
     }
 }
 
+
+// Token scheduling and vector operators interleaved wave by wave, for programs in which a Switch reads a vector
+// value (RDF_OP_GATE): the tokens of wave w may read any state whose operator was queued before wave w, so every
+// wave ends with the operators it queued -- leaves E[tok], unary operators tanh(W_half x + b), cells
+// tanh(W [x_l ; x_r] + b) -- one warp per operator, its operand rows staged in the warp's shared memory, the lanes
+// striding over the contracted index with coalesced loads of the weight row and a butterfly sum per output.
+// Two grid barriers per wave (tokens | operators).  fp32, H <= INTERLEAVED_MAX_H.
+__global__ void __launch_bounds__(1024, 1) rdf_interleaved_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ SharedProgram sp;
+    extern __shared__ __align__(16) unsigned char il_smem[];          // per warp: 2 H floats of operands
+    load_program(c, sp);
+    ThreadStats st;
+    uint32_t generation = 0, wave = 0, widest = 0, done_cells = 0, done_leaves = 0;
+    long long cyc_s = 0, cyc_o = 0, cyc_b = 0, t_mark = clock64();
+    auto lap = [&](long long& acc) {
+        const long long now = clock64();
+        acc += now - t_mark;
+        t_mark = now;
+    };
+    const int H = c.H, lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    float* xs = reinterpret_cast<float*>(il_smem) + (size_t)warp * 2 * H;
+    const uint32_t gwarp = blockIdx.x * (blockDim.x / 32) + warp, n_warps = gridDim.x * (blockDim.x / 32);
+    for (;; ++wave) {
+        const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
+        if (n == 0) break;
+        if (wave >= c.wave_limit) {
+            set_status(c, RDF_ERR_WAVE_LIMIT);
+            break;
+        }
+        widest = max(widest, n);
+        if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->qcount[(wave + 2) % 3].v = 0;
+        const Token* q = c.q[wave & 1];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+            run_token(c, sp, nullptr, wave, load_token(&q[i]), st);
+        __syncthreads();
+        lap(cyc_s);
+        if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
+        lap(cyc_b);
+        // ---- the operators this wave queued
+        const uint32_t n_leaf = min(ld_volatile_u32(&c.ctl->leaf_count.v), c.work_cap);
+        const uint32_t n_cell = min(ld_volatile_u32(&c.ctl->cell_count.v), c.work_cap);
+        for (uint32_t i = done_leaves + gwarp; i < n_leaf; i += n_warps) {
+            const LeafItem it = c.leaf_items[i];
+            const float* e = c.E + (size_t)it.tok * c.D;
+            float* out = c.arena + (size_t)it.slot * c.S;
+            for (int k = lane; k < H; k += 32) out[k] = __ldg(&e[k]);
+        }
+        for (uint32_t i = done_cells + gwarp; i < n_cell; i += n_warps) {
+            const CellItem it = c.cell_items[i];
+            const bool unary = it.r == CHILD_L_MARK || it.r == CHILD_R_MARK;
+            const int K = unary ? H : 2 * H;
+            const int off = it.r == CHILD_R_MARK ? H : 0;             // the half of W a unary operator applies
+            if (it.l >= c.frame_cap || (!unary && it.r >= c.frame_cap)) {
+                set_status(c, RDF_ERR_BAD_ARG);
+                continue;
+            }
+            __syncwarp();
+            for (int k = lane; k < H; k += 32) {
+                xs[k] = __ldcg(&c.arena[(size_t)it.l * c.S + k]);
+                if (!unary) xs[H + k] = __ldcg(&c.arena[(size_t)it.r * c.S + k]);
+            }
+            __syncwarp();
+            float* out = c.arena + (size_t)it.out * c.S;
+            for (int j = 0; j < H; ++j) {
+                const float* w = c.W + (size_t)j * 2 * H + off;
+                float acc = 0.f;
+                for (int k = lane; k < K; k += 32) acc = fmaf(__ldg(&w[k]), xs[k], acc);
+                for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                if (lane == 0) out[j] = tanhf(acc + c.b[j]);
+            }
+        }
+        done_leaves = n_leaf;
+        done_cells = n_cell;
+        __syncthreads();
+        lap(cyc_o);
+        if (!grid_barrier(c, &c.ctl->bar.v, generation)) break;
+        lap(cyc_b);
+    }
+    flush_stats(c, st);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        c.ctl->waves = wave;
+        c.ctl->max_wave_tokens = widest;
+        c.ctl->cyc[0] = cyc_s; c.ctl->cyc[1] = cyc_o; c.ctl->cyc[2] = cyc_b;
+        c.ctl->forward_status = c.ctl->status;
+    }
+}
 
 __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -929,6 +1048,11 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     if (in->B + in->max_invocations >= 0xFFFFFFF0ll) return RDF_ERR_BAD_ARG;
     if (g->tag_mode == RDF_TAGS_PATH && in->B > (1ll << 20)) return RDF_ERR_BAD_ARG;
     if (want_grad && !g->has_vector_ops) return RDF_ERR_UNSUPPORTED;
+    if (g->interleaved) {
+        // a Switch reads a vector value: token waves and operators interleaved, fp32, forward only
+        if (want_grad || params->compute == RDF_BF16 || params->H > INTERLEAVED_MAX_H || params->D != params->H) return RDF_ERR_UNSUPPORTED;
+        if (!params->W_s || !params->b_s || !params->W || !params->b || !params->E) return RDF_ERR_BAD_ARG;
+    }
     const int H = g->has_vector_ops ? params->H : 0;
     Plan P;
     L.qcap = (uint32_t)std::min<long long>(in->max_wave_tokens > 0 ? in->max_wave_tokens : in->max_invocations + in->B,
@@ -948,7 +1072,7 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.frame_ptag = P.take<uint64_t>(g->has_loops ? (size_t)L.frame_cap : 0);
     // fp32 TreeRNN: the cells are fired cluster by cluster of instances (no grid barrier); needs the instance of every frame
     // (eligibility only: whether the device takes clusters is known at launch, and the workspace must not depend on it)
-    L.clustered = g->has_vector_ops && g->has_rnn && !g->has_lstm && H <= CLUSTER_MAX_H &&
+    L.clustered = g->has_vector_ops && g->has_rnn && !g->has_lstm && !g->interleaved && H <= CLUSTER_MAX_H &&
                   !(params->compute == RDF_BF16 && (H + 63) / 64 * 64 <= TC_HP_MAX && params->D == params->H);   // (not the tensor-core path)
     L.finst = P.take<uint32_t>(L.clustered ? (size_t)L.frame_cap : 0);
     L.pair_bytes = (size_t)L.frame_cap * g->match.size() * sizeof(Slot);
@@ -1039,6 +1163,9 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     if (per_sm < 1) return RDF_ERR_CUDA;
     CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 128 * THIN_RESIDENT_MAX_H));
+    if (per_sm < 1) return RDF_ERR_CUDA;
+    CUDA_OK(cudaFuncSetAttribute(rdf_interleaved_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * 2 * INTERLEAVED_MAX_H * (int)sizeof(float)));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_interleaved_kernel, 1024, 32 * 2 * INTERLEAVED_MAX_H * sizeof(float)));
     if (per_sm < 1) return RDF_ERR_CUDA;
     CUDA_OK(cudaFuncSetAttribute(rdf_scheduler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * LQ_CAP * sizeof(Token))));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 2 * LQ_CAP * sizeof(Token)));
@@ -1211,10 +1338,20 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     }
     rdf_mark(S, 1, stream);
     void* args[] = {(void*)&c};
-    RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
-                                        2 * LQ_CAP * sizeof(Token), stream)));
+    if (g->interleaved)
+        RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_interleaved_kernel, dim3(S->grid), dim3(1024), args,
+                                            32 * 2 * (size_t)c.H * sizeof(float), stream)));
+    else
+        RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
+                                            2 * LQ_CAP * sizeof(Token), stream)));
     rdf_mark(S, 2, stream);
-    if (g->has_vector_ops) {
+    if (g->interleaved) {
+        // the states were computed between the token waves: only the root rows are left to copy out
+        rdf_mark(S, 3, stream);
+        rdf_mark(S, 4, stream);
+        RDF_KERNEL(S, rdf_gather_roots_kernel<<<(unsigned)in->B, 128, 0, stream>>>(c, out->h_root));
+        CUDA_OK(cudaGetLastError());
+    } else if (g->has_vector_ops) {
         void* oargs[] = {(void*)&c};
         DevCtx co = c;
         if (c.use_tc) {

@@ -28,7 +28,7 @@ int arity_of(int op) {
         case RDF_OP_NODE_LOSS: return 2;
         case RDF_OP_IF: return 3;
         case RDF_OP_CALL: case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK:
-        case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: return 1;
+        case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: case RDF_OP_GATE: return 1;
         default: return -1;
     }
 }
@@ -122,11 +122,13 @@ void validate(const Prog& P) {
 void check_kinds(const Prog& P) {
     const int nf = P.p->n_functions;
     std::vector<int> fvec(nf, 0);                  // function returns a vector (fixpoint from "integer")
+    std::vector<int> pvec(nf * 3, 0);              // formal parameter k of f is vector-valued: some call passes a state
     std::function<int(int, int)> kind = [&](int f, int e) -> int {
         const rdf_expr& x = P.ex(f, e);
         switch (x.op) {
             case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
-            case RDF_OP_NODE_LOSS: return 1;
+            case RDF_OP_NODE_LOSS: case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: return 1;
+            case RDF_OP_PARAM: return pvec[f * 3 + (int)x.imm];
             case RDF_OP_CALL: return fvec[x.imm];
             case RDF_OP_IF: return kind(f, x.b) | kind(f, x.c);
             default: return 0;
@@ -137,10 +139,35 @@ void check_kinds(const Prog& P) {
         for (int f = 0; f < nf; ++f) {
             const int k = kind(f, P.fn(f).root);
             if (k != fvec[f]) { fvec[f] = k; changed = true; }
+            for (int e = 0; e < P.fn(f).n_exprs; ++e) {
+                const rdf_expr& x = P.ex(f, e);
+                if (x.op != RDF_OP_CALL) continue;
+                const int ops[3] = {x.a, x.b, x.c};
+                for (int k2 = 0; k2 < P.n_ops(x); ++k2)
+                    if (kind(f, ops[k2]) && !pvec[(int)x.imm * 3 + k2]) { pvec[(int)x.imm * 3 + k2] = 1; changed = true; }
+            }
         }
     }
+    require(!pvec[P.p->result * 3], RDF_ERR_UNSUPPORTED);
     for (int f = 0; f < nf; ++f) {
         const rdf_function& F = P.fn(f);
+        // at most one vector operator along any path through the body: the invocation's frame holds one state
+        std::function<int(int)> vcount = [&](int e) -> int {
+            const rdf_expr& x = F.exprs[e];
+            if (x.op == RDF_OP_IF) return vcount(x.a) + std::max(vcount(x.b), vcount(x.c));
+            int n = 0;
+            switch (x.op) {
+                case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
+                case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: n = 1; break;
+                default: break;
+            }
+            if (x.op == RDF_OP_CALL) return 0;             // the operators of an argument that is a call run in the callee's frame;
+                                                           // other arguments are checked below (integers, or plain parameters)
+            const int ops[3] = {x.a, x.b, x.c};
+            for (int k = 0; k < P.n_ops(x); ++k) n += vcount(ops[k]);
+            return n;
+        };
+        require(vcount(F.root) <= 1, RDF_ERR_UNSUPPORTED);
         std::vector<char> seen(F.n_exprs, 0);
         std::function<void(int)> walk = [&](int e) {
             if (seen[e]) return;
@@ -151,7 +178,7 @@ void check_kinds(const Prog& P) {
             for (int k = 0; k < n; ++k) walk(ops[k]);
             switch (x.op) {
                 case RDF_OP_IF:
-                    require(kind(f, x.a) == 0, RDF_ERR_UNSUPPORTED);                 // a Switch driven by a vector value
+                    require(kind(f, x.a) == 0, RDF_ERR_UNSUPPORTED);                 // a Switch takes an integer (RDF_OP_GATE makes one)
                     require(kind(f, x.b) == kind(f, x.c), RDF_ERR_UNSUPPORTED);
                     break;
                 case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM:
@@ -160,6 +187,22 @@ void check_kinds(const Prog& P) {
                     break;
                 case RDF_OP_NODE_LOSS:
                     require(kind(f, x.a) == 1 && kind(f, x.b) == 0, RDF_ERR_UNSUPPORTED);
+                    break;
+                case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: case RDF_OP_GATE:
+                    // reads a state that exists when the invocation starts: a vector-valued parameter
+                    require(F.exprs[x.a].op == RDF_OP_PARAM && kind(f, x.a) == 1, RDF_ERR_UNSUPPORTED);
+                    require(P.p->tag_mode == RDF_TAGS_FRAME, RDF_ERR_UNSUPPORTED);
+                    break;
+                case RDF_OP_CALL:
+                    // an argument is of the kind the callee's parameter has at every call site; a state is passed on as a
+                    // parameter or as the result of a call (by reference), never computed in the argument itself
+                    for (int k = 0; k < n; ++k) {
+                        require(kind(f, ops[k]) == pvec[(int)x.imm * 3 + k], RDF_ERR_UNSUPPORTED);
+                        if (kind(f, ops[k]))
+                            require(F.exprs[ops[k]].op == RDF_OP_PARAM || F.exprs[ops[k]].op == RDF_OP_CALL, RDF_ERR_UNSUPPORTED);
+                    }
+                    require(!(P.is_loop((int)x.imm) && (pvec[(int)x.imm * 3] | pvec[(int)x.imm * 3 + 1] | pvec[(int)x.imm * 3 + 2])),
+                            RDF_ERR_UNSUPPORTED);
                     break;
                 default:                                                                 // integer operands only
                     for (int k = 0; k < n; ++k) require(kind(f, ops[k]) == 0, RDF_ERR_UNSUPPORTED);
@@ -499,7 +542,7 @@ struct Lower {
         const rdf_expr& x = P.ex(f, e);
         switch (x.op) {
             case RDF_OP_CALL: case RDF_OP_EMBED: case RDF_OP_LEAF_LSTM: case RDF_OP_CELL_RNN:
-            case RDF_OP_CELL_LSTM: case RDF_OP_NODE_LOSS: return false;
+            case RDF_OP_CELL_LSTM: case RDF_OP_NODE_LOSS: case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: return false;
             default: break;
         }
         int ops[3] = {x.a, x.b, x.c};
@@ -547,6 +590,13 @@ struct Lower {
                 g->uses_tree = true;
                 emit(s, x.op == RDF_OP_IS_LEAF ? VM_ISLEAF : x.op == RDF_OP_LEFT ? VM_LEFT
                         : x.op == RDF_OP_RIGHT ? VM_RIGHT : VM_TOK, r, a);
+                break;
+            }
+            case RDF_OP_GATE: {
+                int a = value(s, x.a);
+                r = reg(s);
+                g->interleaved = true;
+                emit(s, VM_VGATE, r, a);
                 break;
             }
             case RDF_OP_IF: {
@@ -782,6 +832,15 @@ struct Lower {
                 emit(s, x.op == RDF_OP_EMBED ? VM_EMBED : VM_LEAF_LSTM, 0, r, 0, -(ks + 1));   // fixed up at layout
                 break;
             }
+            case RDF_OP_CHILD_L: case RDF_OP_CHILD_R: {
+                g->has_vector_ops = true;
+                g->has_rnn = true;
+                g->interleaved = true;
+                int r = value(s, x.a);
+                int ks = cont_segment(K);
+                emit(s, VM_VCHILD, x.op == RDF_OP_CHILD_L ? 0 : 1, r, 0, -(ks + 1));            // fixed up at layout
+                break;
+            }
             case RDF_OP_CELL_RNN: case RDF_OP_CELL_LSTM: {
                 g->has_vector_ops = true;
                 (x.op == RDF_OP_CELL_RNN ? g->has_rnn : g->has_lstm) = true;
@@ -862,7 +921,7 @@ struct Lower {
         for (Seg& S : segs)
             for (VmInstr in : S.code) {
                 if (in.op == VM_BRZ || in.op == VM_JMP) in.imm += S.base;
-                if (in.op == VM_EMBED || in.op == VM_LEAF_LSTM || in.op == VM_ENTER || in.op == VM_NEXT) in.imm = segs[-in.imm - 1].base;
+                if (in.op == VM_EMBED || in.op == VM_LEAF_LSTM || in.op == VM_VCHILD || in.op == VM_ENTER || in.op == VM_NEXT) in.imm = segs[-in.imm - 1].base;
                 g->code.push_back(in);
             }
         for (size_t i = 0; i < g->labels.size(); ++i) {

@@ -34,6 +34,8 @@ enum VmOp : uint8_t {
     VM_ENTER,      // Enter: new loop frame under the current tag, counter 0; variables r[a], r[b], r[dst]; loop head at imm
     VM_NEXT,       // Next: counter + 1, variables r[a], r[b], r[dst], back to the loop head at imm (next wave)
     VM_EXIT,       // Exit: the tag below the loop frame again; carries on in the same segment
+    VM_VCHILD,     // unary vector operator dst (0 left, 1 right half of W) on the state r[a] -> state of this frame; continue at imm next wave
+    VM_VGATE,      // r[dst] = W_s[0] . state(r[a]) + b_s[0] > 0: an integer read off a vector value
     VM_HALT
 };
 
@@ -94,6 +96,7 @@ struct rdf_graph {
     bool has_rnn = false, has_lstm = false, has_loss = false;
     bool uses_tree = false;
     bool has_loops = false;
+    bool interleaved = false;     // some Switch reads a vector value: operators run between the token waves
     std::vector<std::string> func_names;
     // per-run state owned by the executor (rdf_exec.cu)
     void* dev = nullptr;

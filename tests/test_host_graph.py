@@ -123,7 +123,8 @@ def test_vector_programs_outside_the_executor_are_rejected():
 OPNAME = {bd.OP_ADD: "+", bd.OP_SUB: "-", bd.OP_MUL: "*", bd.OP_MAX: "max", bd.OP_REM: "%", bd.OP_LT: "<", bd.OP_EQ: "==",
           bd.OP_IS_LEAF: "is_leaf", bd.OP_LEFT: "left", bd.OP_RIGHT: "right", bd.OP_TOK: "tok",
           bd.OP_EMBED: "leaf_rnn", bd.OP_CELL_RNN: "cell_rnn", bd.OP_LEAF_LSTM: "leaf_lstm",
-          bd.OP_CELL_LSTM: "cell_lstm", bd.OP_NODE_LOSS: "pass_state"}
+          bd.OP_CELL_LSTM: "cell_lstm", bd.OP_NODE_LOSS: "pass_state", bd.OP_CHILD_L: "child_l", bd.OP_CHILD_R: "child_r",
+          bd.OP_GATE: "gate"}
 KIND = {bd.NODE_IN: "in", bd.NODE_OUT: "out", bd.NODE_CONST: "const", bd.NODE_OP: "op", bd.NODE_SWITCH: "switch",
         bd.NODE_MERGE: "merge", bd.NODE_ENTRY_MERGE: "merge", bd.NODE_CALL: "Call", bd.NODE_RETURN: "Return",
         bd.NODE_ENTER: "Enter", bd.NODE_EXIT: "Exit", bd.NODE_NEXT: "Next"}
@@ -239,6 +240,62 @@ def test_tree_net_literal_graph_runs_in_the_oracle(cell):
         got = res.value if cell == "rnn" else res.value[0]
         np.testing.assert_allclose(got, want[t], atol=1e-13)
         assert len(res.calls) == tb.tree_sizes()[t]
+
+
+def test_topdown_literal_graph_runs_in_the_oracle():
+    """Recursion shaped by vector values (Section 6.2, last paragraph): the graph rdf_graph_build makes of the
+    top-down program -- a Switch whose predicate comes from RDF_OP_GATE on a state -- run by the oracle's interpreter
+    against the direct recursion."""
+    V, H, D = 40, 6, 5
+    P = workloads.topdown_params(5, V, H)
+    tb = workloads.topdown_batch(5, 10, V)
+    ops = programs.topdown_ops(tb, P, D)
+    fs, r = rdf.topdown_program(D)
+    desc = _build(fs, r, rdf.TAGS_FRAME).describe()
+    g = _as_oracle_graph(desc)
+    kinds = [n["kind"] for n in desc["nodes"]]
+    # call sites: seed 1, expand 3 (one in result, two in expand), left 1, right 1; one Call_i per parameter
+    assert kinds.count(bd.NODE_CALL) == 1 + 3 * 2 + 1 + 1 and kinds.count(bd.NODE_RETURN) == 6
+    sizes = set()
+    for b in range(tb.B):
+        log = {}
+        want = direct.topdown(P, int(tb.tok[b]), D, log)
+        res = tagged.run(g, {0: int(tb.tree_root[b])}, ops)
+        np.testing.assert_allclose(res.value, want, atol=1e-13)
+        assert res.leftover == 0
+        sizes.add(log["expand"])
+    assert len(sizes) >= 3
+
+
+def test_topdown_programs_outside_the_executor_are_rejected():
+    def prog(expand_body, left_body=None, mode=rdf.TAGS_FRAME):
+        r = rdf.Function("result", 1)
+        r.ret(r.call(2, r.call(1, r.param()), r.const(0)))
+        s = rdf.Function("seed", 1)
+        s.ret(s.embed(s.tok(s.param())))
+        f = rdf.Function("expand", 2)
+        f.ret(expand_body(f, f.param(0), f.param(1)))
+        fl = rdf.Function("left", 1)
+        fl.ret((left_body or (lambda g, h: g.child_l(h)))(fl, fl.param()))
+        return [r, s, f, fl], mode
+
+    ok = lambda f, h, d: f.if_(f.max(f.lt(f.const(3), d), f.gate(h)), h,                      # noqa: E731
+                               f.cell_rnn(f.call(2, f.call(3, h), f.add(d, f.const(1))), f.call(2, f.call(3, h), f.add(d, f.const(1)))))
+    fs, mode = prog(ok)
+    _build(fs, 0, mode)
+    bad = [
+        prog(ok, mode=rdf.TAGS_PATH),                                                          # states live in frames
+        prog(lambda f, h, d: f.if_(f.gate(d), h, h)),                                          # a gate on an integer
+        prog(lambda f, h, d: f.if_(f.gate(h), h, f.child_l(f.call(3, h)))),                    # a child operator on a call's result
+        # two vector operators in one invocation (the child states computed where the cell is)
+        prog(lambda f, h, d: f.if_(f.gate(h), h, f.cell_rnn(f.call(2, f.child_l(h), d), f.call(2, f.child_r(h), d)))),
+        prog(ok, left_body=lambda g, h: g.child_l(g.child_r(h))),                              # a child operator on a computed state
+        prog(lambda f, h, d: f.if_(f.gate(h), h, f.call(2, d, d))),                            # an integer where the callee takes a state
+    ]
+    for fs, mode in bad:
+        with pytest.raises(rdf.RdfError) as e:
+            _build(fs, 0, mode)
+        assert e.value.code == -11
 
 
 LOOPS = {"sum": (rdf.sum_loop_program, programs.sum_loop_program, direct.sum_to, [0, 1, 5, 17]),
