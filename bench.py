@@ -40,6 +40,8 @@ WORKLOAD_NAMES = {
     3: "config3: TreeRNN forward+backward, 8192 trees (lognormal leaves, median 18), H=300, vocab 21000, 5-class loss at every node",
     4: "config4: binary TreeLSTM forward+backward, 8192 trees (same size mix), H=300, vocab 21000, 5-class loss at every node",
     5: "config5: depth stress, TreeRNN H=256 fp32 forward+backward, 64 chains of depth 4096 + 16 perfect trees of 2^16 leaves",
+    6: "extra: top-down recursion shaped by the values (a gate on each node's state decides its expansion), 8192 seeds, H=128, "
+       "depth limit 10, fp32, forward",
 }
 CELL = {"treernn": "rnn", "treelstm": "lstm"}
 KERNEL_SOURCES = ["rdf_device.cuh", "rdf_exec.cu", "rdf_exec.h", "rdf_grad.cu", "rdf_internal.h", "rdf_lists.cuh", "rdf_lstm.cuh",
@@ -105,6 +107,8 @@ def load(k, seed, fib_batch=None, over=None):
     cfg = workloads.config(k, seed=seed, **over)
     if cfg["kind"] == "fib":
         cfg["N"] = int(sum(2 * fib_iter(int(n) + 1) - 1 for n in cfg["x"]))
+    elif cfg["kind"] == "topdown":
+        cfg["N"] = 0                   # how many invocations the seeds generate is known after the first run
     else:
         cfg["N"] = cfg["trees"].N
     return cfg
@@ -175,6 +179,13 @@ def oracle_step(cfg, sample, grad=None):
         return n
     tb = cfg["trees"]
     trees = list(range(min(sample, tb.B)))
+    if cfg["kind"] == "topdown":
+        n = 0
+        for t in trees:
+            log = {}
+            direct.topdown(cfg["params"], int(tb.tok[t]), cfg["D"], log)
+            n += 1 + log["expand"] + log["child"]
+        return n
     if cfg["grad"] if grad is None else grad:
         direct.loss_and_grad(tb, cfg["params"], CELL[cfg["kind"]], trees=trees)
     else:
@@ -333,9 +344,11 @@ class Case:
             return
         tb, p = cfg["trees"], cfg["params"]
         self.tb = tb
-        self.cell = CELL[cfg["kind"]]
-        fs, r = rdf.tree_net_program(self.cell, with_loss=self.grad)
+        self.topdown = cfg["kind"] == "topdown"
+        self.cell = "rnn" if self.topdown else CELL[cfg["kind"]]
+        fs, r = rdf.topdown_program(cfg["D"]) if self.topdown else rdf.tree_net_program(self.cell, with_loss=self.grad)
         self.g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+        self.max_inv = cfg.get("max_invocations")
         self.compute = rdf.BF16 if cfg["bf16"] else rdf.F32
         # arithmetic type of the contractions: bf16 operands on the tensor cores (fp32 accumulate) for the
         # bf16 workloads, fp32 FMA otherwise
@@ -357,6 +370,9 @@ class Case:
             self.d2h_full = 4 + self.flat.numel() * 4 + tb.B * self.H * 4
         else:
             self.d2h = self.d2h_full = tb.B * self.H * 4
+        if self.topdown:               # one run tells how many invocations the seeds generate (the unit of the metric)
+            self.step()
+            self.N = cfg["N"] = int(self.g.stats()["invocations"])
 
     # the timed step: inputs and parameters resident
     def step(self):
@@ -366,7 +382,7 @@ class Case:
             self.g.grad_trees(self.dt, self.dp, self.compute, check=False, grads=self.grads, loss=self.loss, h_root=self.h_root)
             sum_gradients(self.dist, self.flat)      # data-parallel exchange: one sum of the parameter gradients
         else:
-            self.g.eval_trees(self.dt, self.dp, self.compute, check=False, h_root=self.h_root)
+            self.g.eval_trees(self.dt, self.dp, self.compute, check=False, h_root=self.h_root, max_invocations=self.max_inv)
 
     # end to end: host buffers in, result out; full = every output of the call comes back
     def step_e2e(self, full=False):
@@ -384,7 +400,7 @@ class Case:
                 self.flat_host.copy_(self.flat, non_blocking=True)
                 self.h_root_host.copy_(self.h_root, non_blocking=True)
             return self.loss.item()
-        self.g.eval_trees(d, self.dp, self.compute, check=False, h_root=self.h_root)
+        self.g.eval_trees(d, self.dp, self.compute, check=False, h_root=self.h_root, max_invocations=self.max_inv)
         self.h_root_host.copy_(self.h_root, non_blocking=True)
         self.torch.cuda.current_stream().synchronize()
         return self.h_root_host
@@ -393,6 +409,9 @@ class Case:
         if self.cfg["kind"] == "fib":
             return 0.0
         H, tb = self.H, self.tb
+        if self.topdown:               # N = B seeds + E expands + (E - B) children, (E - B) / 2 of the expands end in a cell
+            E = self.N // 2
+            return (E - tb.B) * 2.0 * H * H + (E - tb.B) / 2 * 2.0 * (2 * H) * H
         if self.cell == "lstm":
             return tb.n_cells * 2.0 * (2 * H) * (5 * H) + (tb.N - tb.n_cells) * 2.0 * H * (3 * H)
         return tb.n_cells * 2.0 * (2 * H) * H
@@ -476,6 +495,11 @@ def kernel_table(case, phase_ms, pk, fp32_peak, traffic, workload):
     add("rdf_scheduler_kernel", "schedule", "hbm", 128.0 * N,
         "128 B per invocation: call token write+read, return token / store slot write+read, frame record")
     if case.cfg["kind"] == "fib":
+        return rows
+    if case.cfg["kind"] == "topdown":
+        rows.clear()
+        add("rdf_interleaved_kernel", "schedule", "alu", case.flops_fwd(),
+            "child operators 2*H*H and cells 2*2H*H per expanded node (token waves and operators share the kernel)")
         return rows
     tb, H = case.tb, case.H
     C, Lf = tb.n_cells, tb.N - tb.n_cells

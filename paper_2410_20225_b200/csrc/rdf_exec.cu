@@ -583,15 +583,16 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
 }
 
 
+static inline int interleaved_smem_bytes(int H) { return 2 * H * 33 * (int)sizeof(float); }
+
 // Token scheduling and vector operators interleaved wave by wave, for programs in which a Switch reads a vector
 // value (RDF_OP_GATE): the tokens of wave w may read any state whose operator was queued before wave w, so every
 // wave ends with the operators it queued -- leaves E[tok], unary operators tanh(W_half x + b), cells
-// tanh(W [x_l ; x_r] + b) -- one warp per operator, its operand rows staged in the warp's shared memory, the lanes
-// striding over the contracted index with coalesced loads of the weight row and a butterfly sum per output.
+// tanh(W [x_l ; x_r] + b) -- in groups of 32 operators per block.
 // Two grid barriers per wave (tokens | operators).  fp32, H <= INTERLEAVED_MAX_H.
 __global__ void __launch_bounds__(1024, 1) rdf_interleaved_kernel(const __grid_constant__ DevCtx c) {
     __shared__ SharedProgram sp;
-    extern __shared__ __align__(16) unsigned char il_smem[];          // per warp: 2 H floats of operands
+    extern __shared__ __align__(16) unsigned char il_smem[];
     load_program(c, sp);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0, done_cells = 0, done_leaves = 0;
@@ -602,7 +603,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_interleaved_kernel(const __grid_c
         t_mark = now;
     };
     const int H = c.H, lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    float* xs = reinterpret_cast<float*>(il_smem) + (size_t)warp * 2 * H;
+    float* xs = reinterpret_cast<float*>(il_smem);                  // [2H][33]: operand rows of a group of 32 operators, transposed
     const uint32_t gwarp = blockIdx.x * (blockDim.x / 32) + warp, n_warps = gridDim.x * (blockDim.x / 32);
     for (;; ++wave) {
         const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
@@ -629,28 +630,53 @@ __global__ void __launch_bounds__(1024, 1) rdf_interleaved_kernel(const __grid_c
             float* out = c.arena + (size_t)it.slot * c.S;
             for (int k = lane; k < H; k += 32) out[k] = __ldg(&e[k]);
         }
-        for (uint32_t i = done_cells + gwarp; i < n_cell; i += n_warps) {
-            const CellItem it = c.cell_items[i];
-            const bool unary = it.r == CHILD_L_MARK || it.r == CHILD_R_MARK;
-            const int K = unary ? H : 2 * H;
-            const int off = it.r == CHILD_R_MARK ? H : 0;             // the half of W a unary operator applies
-            if (it.l >= c.frame_cap || (!unary && it.r >= c.frame_cap)) {
-                set_status(c, RDF_ERR_BAD_ARG);
-                continue;
+        // Unary operators and cells, 32 at a time per block: a unary operator on x is the cell on [x ; 0] (left half of
+        // W) or [0 ; x] (right half), so one loop serves all three.  The operand rows of the group are staged
+        // transposed (xs[k][item], rows padded to 33 floats: conflict-free both ways); warp w then computes outputs
+        // 4w .. 4w+3 (+128, ...) of all 32 items, lane = item, the weight rows read as uniform vector loads.
+        for (uint32_t g0 = done_cells + blockIdx.x * 32u; g0 < n_cell; g0 += gridDim.x * 32u) {
+            const uint32_t cnt = min(32u, n_cell - g0);
+            __syncthreads();                                        // (the previous group's operands are no longer read)
+            CellItem it = CellItem{0u, 0u, 0u, 0u};
+            bool ok = false;
+            if ((uint32_t)warp < cnt) {
+                it = c.cell_items[g0 + warp];
+                const bool unary = it.r == CHILD_L_MARK || it.r == CHILD_R_MARK;
+                ok = it.l < c.frame_cap && (unary || it.r < c.frame_cap) && it.out < c.frame_cap;
+                if (!ok && lane == 0) set_status(c, RDF_ERR_BAD_ARG);
+                for (int k = lane; k < H; k += 32) {
+                    float a = 0.f, b2 = 0.f;
+                    if (ok) {
+                        const float x = __ldcg(&c.arena[(size_t)it.l * c.S + k]);
+                        if (it.r == CHILD_R_MARK) b2 = x; else a = x;
+                        if (!unary) b2 = __ldcg(&c.arena[(size_t)it.r * c.S + k]);
+                    }
+                    xs[(size_t)k * 33 + warp] = a;
+                    xs[(size_t)(H + k) * 33 + warp] = b2;
+                }
             }
-            __syncwarp();
-            for (int k = lane; k < H; k += 32) {
-                xs[k] = __ldcg(&c.arena[(size_t)it.l * c.S + k]);
-                if (!unary) xs[H + k] = __ldcg(&c.arena[(size_t)it.r * c.S + k]);
-            }
-            __syncwarp();
-            float* out = c.arena + (size_t)it.out * c.S;
-            for (int j = 0; j < H; ++j) {
-                const float* w = c.W + (size_t)j * 2 * H + off;
-                float acc = 0.f;
-                for (int k = lane; k < K; k += 32) acc = fmaf(__ldg(&w[k]), xs[k], acc);
-                for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                if (lane == 0) out[j] = tanhf(acc + c.b[j]);
+            __syncthreads();
+            // lane = item of the group; its output row
+            const uint32_t out_row = (uint32_t)lane < cnt ? c.cell_items[g0 + lane].out : 0xFFFFFFFFu;
+            for (int j0 = warp * 4; j0 < H; j0 += 128) {
+                float acc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] = c.b[j0 + q];
+                const float4* w0 = reinterpret_cast<const float4*>(c.W + (size_t)j0 * 2 * H);
+                const int K4 = 2 * H / 4;
+                for (int k4 = 0; k4 < K4; ++k4) {
+                    float4 w[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) w[q] = __ldg(w0 + (size_t)q * K4 + k4);
+                    const float x0 = xs[(size_t)(4 * k4 + 0) * 33 + lane], x1 = xs[(size_t)(4 * k4 + 1) * 33 + lane];
+                    const float x2 = xs[(size_t)(4 * k4 + 2) * 33 + lane], x3 = xs[(size_t)(4 * k4 + 3) * 33 + lane];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        acc[q] = fmaf(w[q].w, x3, fmaf(w[q].z, x2, fmaf(w[q].y, x1, fmaf(w[q].x, x0, acc[q]))));
+                }
+                if (out_row < c.frame_cap)
+                    *reinterpret_cast<float4*>(c.arena + (size_t)out_row * c.S + j0) =
+                        make_float4(tanhf(acc[0]), tanhf(acc[1]), tanhf(acc[2]), tanhf(acc[3]));
             }
         }
         done_leaves = n_leaf;
@@ -1164,8 +1190,8 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_operator_kernel<false>, 256, 128 * THIN_RESIDENT_MAX_H));
     if (per_sm < 1) return RDF_ERR_CUDA;
-    CUDA_OK(cudaFuncSetAttribute(rdf_interleaved_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * 2 * INTERLEAVED_MAX_H * (int)sizeof(float)));
-    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_interleaved_kernel, 1024, 32 * 2 * INTERLEAVED_MAX_H * sizeof(float)));
+    CUDA_OK(cudaFuncSetAttribute(rdf_interleaved_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, interleaved_smem_bytes(INTERLEAVED_MAX_H)));
+    CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_interleaved_kernel, 1024, interleaved_smem_bytes(INTERLEAVED_MAX_H)));
     if (per_sm < 1) return RDF_ERR_CUDA;
     CUDA_OK(cudaFuncSetAttribute(rdf_scheduler_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * LQ_CAP * sizeof(Token))));
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 2 * LQ_CAP * sizeof(Token)));
@@ -1340,7 +1366,7 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     void* args[] = {(void*)&c};
     if (g->interleaved)
         RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_interleaved_kernel, dim3(S->grid), dim3(1024), args,
-                                            32 * 2 * (size_t)c.H * sizeof(float), stream)));
+                                            (size_t)interleaved_smem_bytes(c.H), stream)));
     else
         RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_scheduler_kernel, dim3(S->grid), dim3(1024), args,
                                             2 * LQ_CAP * sizeof(Token), stream)));

@@ -238,7 +238,7 @@ def _lognormal_leaves(rng, B, median=18.0, sigma=0.5, lo=1, hi=56):
 
 
 def config(k: int, seed: int = DEFAULT_SEED, B: int | None = None, **over):
-    """Workload k (1..5) as a dict.  `B` overrides the batch size (for small
+    """Workload k (1..5, and 6: the top-down recursion) as a dict.  `B` overrides the batch size (for small
     parity cases); for k == 5 `chains`, `chain_depth`, `perfect`,
     `perfect_height` may be overridden through keyword arguments."""
     if k == 1:
@@ -274,4 +274,11 @@ def config(k: int, seed: int = DEFAULT_SEED, B: int | None = None, **over):
         tb = tree_batch_from_shapes(shapes, seed, vocab=V)
         return {"kind": "treernn", "trees": tb, "H": H, "V": V, "bf16": False, "grad": True,
                 "params": treernn_params(seed, V, H, H)}
+    if k == 6:
+        # beyond the five named configurations: recursion whose shape follows the values (a tree grown top-down from
+        # a seed state, a gate on every node's state deciding whether it is expanded; depth limit D)
+        B = 8192 if B is None else B
+        V, H, D = over.get("V", 21000), over.get("H", 128), over.get("D", 10)
+        return {"kind": "topdown", "trees": topdown_batch(seed, B, V), "H": H, "V": V, "D": D, "bf16": False, "grad": False,
+                "params": topdown_params(seed, V, H), "max_invocations": 256 * B}
     raise ValueError(f"unknown workload {k}")
