@@ -80,6 +80,7 @@ struct Control {
     uint32_t resume_wave;         // wave index at which the grid carries on after a stretch of narrow waves
     uint32_t max_height;          // largest height of a cell of this call (operator waves run height by height)
     uint32_t h_split;             // clustered fp32 path: heights up to here are wide and fired by the whole grid, the rest cluster by cluster
+    uint32_t d_split;             // clustered gradient pass: call depths (scheduler wave + 1) up to here are wide and run by the whole grid
     uint32_t n_depth_waves;       // scheduler waves that made calls = call depths of the run (length of the compacted wave_marks)
     unsigned long long invocations, tokens, store_inserts, store_matches, store_probes, cells, leaves;
     unsigned long long trace_count;
@@ -210,7 +211,24 @@ __device__ __forceinline__ uint32_t cell_groups(const DevCtx& c) {
     return c.n_groups > 1 && stride > CLUSTER_MIN_HEIGHT && (uint64_t)c.n_groups * stride <= (uint64_t)c.wave_cap + 2u
                ? (uint32_t)c.n_groups : 1u;
 }
+// The same for the gradient pass, whose waves go by call depth (the scheduler wave that created the frame): cells grouped
+// by (cluster of their instance, scheduler wave + 1).
+__device__ __forceinline__ uint32_t depth_groups(const DevCtx& c) {
+    const uint64_t stride = (uint64_t)min(c.ctl->waves, c.wave_cap) + 1u;
+    return cell_groups(c) > 1u && (uint64_t)c.n_groups * stride <= (uint64_t)c.wave_cap + 2u ? (uint32_t)c.n_groups : 1u;
+}
+__device__ __forceinline__ uint32_t bucket_groups(const DevCtx& c, int by_depth) { return by_depth ? depth_groups(c) : cell_groups(c); }
+__device__ __forceinline__ uint32_t bucket_stride(const DevCtx& c, int by_depth) {
+    return min(by_depth ? c.ctl->waves : c.ctl->max_height, c.wave_cap) + 1u;
+}
 static const uint32_t NO_ZDST = 0xFFFFFFFFu;
+
+// thread-block clusters of the clustered fp32 kernels (forward cells, gradient waves)
+static const int CLUSTER_CTAS = 8;
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 // 64-bit fixed point, 2^-36 per unit (|sum| < 1.3e8, resolution 1.5e-11): integer additions commute exactly
 #define RDF_FIX_SCALE 68719476736.0f

@@ -833,12 +833,6 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
 // (kept in shared memory for the whole kernel); a block step computes `cells_per_step` cells x its columns, thread =
 // (cell, column), operand rows staged in shared memory.  States travel between the blocks through global memory
 // (L2): the cluster barrier's release / acquire orders them.
-static const int CLUSTER_CTAS = 8;
-
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 
 // CPC: columns of W per block (8 blocks x CPC >= H).  A block step fires CS = 256 / CPC cells: thread = (column, slice
 // of the contraction index), CS accumulators per thread -- a weight is read from shared memory once per step and an
@@ -948,30 +942,31 @@ static const int CLUSTER_MAX_H = 384;
 // height gives the smallest number of dependent operator waves (the largest height instead of about twice the depth).
 // (With the clustered operator kernel the cells are grouped by (cluster of their instance, height): bucket index
 // group * (max height + 1) + height; one group otherwise.  The largest height is known from the scheduler.)
-__device__ __forceinline__ uint32_t cell_bucket(const DevCtx& c, const CellItem& it, uint32_t groups, uint32_t stride) {
-    const uint32_t h = min(it.height, stride - 1u);
-    if (h == 0u) return 0u;                                                          // (0: not a cell)
+__device__ __forceinline__ uint32_t cell_bucket(const DevCtx& c, const CellItem& it, uint32_t groups, uint32_t stride, int by_depth) {
+    if (it.height == 0u) return 0u;                                                  // (0: not a cell)
+    // by_depth (gradient pass): the scheduler wave that created the cell's frame, + 1
+    const uint32_t h = min(by_depth ? (__ldcg(&c.frames[it.out].label) >> FRAME_WAVE_SHIFT) + 1u : it.height, stride - 1u);
     return (groups > 1u ? __ldcg(&c.finst[it.out]) % groups : 0u) * stride + h;
 }
 
-__global__ void __launch_bounds__(256) rdf_height_count_kernel(const DevCtx c) {
+__global__ void __launch_bounds__(256) rdf_height_count_kernel(const DevCtx c, int by_depth) {
     if (c.ctl->status != 0) return;
     const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
-    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
+    const uint32_t groups = bucket_groups(c, by_depth), stride = bucket_stride(c, by_depth);
     for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
         const uint32_t i = i0 + lane;
-        const uint32_t k = i < n ? cell_bucket(c, c.cell_items[i], groups, stride) : 0u;
+        const uint32_t k = i < n ? cell_bucket(c, c.cell_items[i], groups, stride, by_depth) : 0u;
         const unsigned peers = __match_any_sync(0xffffffffu, k);                      // one atomic per bucket and warp
         if (k && (uint32_t)(__ffs(peers) - 1) == lane) atomicAdd(&c.height_ends[k], (uint32_t)__popc(peers));
     }
 }
 
 // counts -> first position of each bucket (one block; buckets 1 .. groups * (max height + 1) - 1)
-__global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c) {
+__global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c, int by_depth) {
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry;
     if (c.ctl->status != 0) return;
-    const uint32_t top = cell_groups(c) * (min(c.ctl->max_height, c.wave_cap) + 1u) - 1u;
+    const uint32_t top = bucket_groups(c, by_depth) * bucket_stride(c, by_depth) - 1u;
     const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
     if (threadIdx.x == 0) carry = 0;
     __syncthreads();
@@ -1004,14 +999,14 @@ __global__ void __launch_bounds__(1024) rdf_height_scan_kernel(const DevCtx c) {
 
 // every cell to its bucket; afterwards height_ends[k] is where bucket k ends (it starts where bucket k - 1 ends;
 // bucket group * stride + 0 is empty, so it ends where the previous group ends)
-__global__ void __launch_bounds__(256) rdf_height_scatter_kernel(const DevCtx c) {
+__global__ void __launch_bounds__(256) rdf_height_scatter_kernel(const DevCtx c, int by_depth) {
     if (c.ctl->status != 0) return;
     const uint32_t n = min(c.ctl->cell_count.v, c.work_cap), lane = threadIdx.x % 32;
-    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
+    const uint32_t groups = bucket_groups(c, by_depth), stride = bucket_stride(c, by_depth);
     for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < n; i0 += gridDim.x * blockDim.x) {
         const uint32_t i = i0 + lane;
         CellItem it = i < n ? c.cell_items[i] : CellItem{0u, 0u, 0u, 0u};
-        const uint32_t k = cell_bucket(c, it, groups, stride);
+        const uint32_t k = cell_bucket(c, it, groups, stride, by_depth);
         const unsigned peers = __match_any_sync(0xffffffffu, k);
         const int leader = __ffs(peers) - 1;
         uint32_t base = 0;
@@ -1023,14 +1018,14 @@ __global__ void __launch_bounds__(256) rdf_height_scatter_kernel(const DevCtx c)
 
 // Which heights are wide enough for the whole grid (clustered path): the last height that has more than `threshold` cells
 // over all groups; the heights above it are left to the clusters.
-__global__ void __launch_bounds__(256) rdf_height_split_kernel(const DevCtx c, uint32_t threshold) {
+__global__ void __launch_bounds__(256) rdf_height_split_kernel(const DevCtx c, uint32_t threshold, int by_depth) {
     if (c.ctl->status != 0) return;
-    const uint32_t groups = cell_groups(c), stride = min(c.ctl->max_height, c.wave_cap) + 1u;
+    const uint32_t groups = bucket_groups(c, by_depth), stride = bucket_stride(c, by_depth);
     if (groups <= 1u) return;
     for (uint32_t h = 1 + blockIdx.x * blockDim.x + threadIdx.x; h < stride; h += gridDim.x * blockDim.x) {
         uint32_t total = 0;
         for (uint32_t gq = 0; gq < groups; ++gq) total += c.height_ends[(size_t)gq * stride + h] - c.height_ends[(size_t)gq * stride + h - 1];
-        if (total > threshold) atomicMax(&c.ctl->h_split, h);
+        if (total > threshold) atomicMax(by_depth ? &c.ctl->d_split : &c.ctl->h_split, h);
     }
 }
 
@@ -1391,15 +1386,15 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
                                                 (size_t)L.tc_smem_fwd, stream)));
         } else {
             // the cells grouped by height; the operator kernel reads the grouped list in place of the scheduler's
-            RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
-            RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c));
-            RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c, 0));
+            RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c, 0));
+            RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c, 0));
             CUDA_OK(cudaGetLastError());
             rdf_mark(S, 3, stream);
             co.cell_items = c.cell_sorted;
             oargs[0] = (void*)&co;
             S->last_clusters = c.n_groups > 1 ? c.n_groups : 0;
-            if (c.n_groups > 1) RDF_KERNEL(S, rdf_height_split_kernel<<<S->grid, 256, 0, stream>>>(c, 40u * (uint32_t)c.n_groups));
+            if (c.n_groups > 1) RDF_KERNEL(S, rdf_height_split_kernel<<<S->grid, 256, 0, stream>>>(c, 40u * (uint32_t)c.n_groups, 0));
             // the leaves and the wide heights with the whole grid ...
             RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
                                                 thin_resident_bytes(c.lstm, c.H), stream)));
@@ -1453,6 +1448,19 @@ int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* 
         }
     }
     if (c.zdst) RDF_KERNEL(S, rdf_list_zdst_kernel<<<2 * S->grid, 256, 0, stream>>>(c));
+    CUDA_OK(cudaGetLastError());
+    return RDF_OK;
+}
+
+// The cells grouped again for the clustered gradient pass: by (cluster of their instance, call depth).  Reuses the
+// grouped list and the bucket table of the forward pass, which is over.
+int rdf_launch_depth_groups(char* ws, const Layout& L, ExecState* S, DevCtx& c, cudaStream_t stream) {
+    if (c.n_groups <= 1) return RDF_OK;
+    CUDA_OK(cudaMemsetAsync(ws + L.height_ends, 0, ((size_t)L.wave_cap + 2) * sizeof(uint32_t), stream));
+    RDF_KERNEL(S, rdf_height_count_kernel<<<2 * S->grid, 256, 0, stream>>>(c, 1));
+    RDF_KERNEL(S, rdf_height_scan_kernel<<<1, 1024, 0, stream>>>(c, 1));
+    RDF_KERNEL(S, rdf_height_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c, 1));
+    RDF_KERNEL(S, rdf_height_split_kernel<<<S->grid, 256, 0, stream>>>(c, 40u * (uint32_t)c.n_groups, 1));
     CUDA_OK(cudaGetLastError());
     return RDF_OK;
 }

@@ -107,6 +107,7 @@ int rdf_check_common(rdf_graph* g, const rdf_batch* in, const rdf_params* params
 // a row-major bf16 matrix [rows, cols] as a 2D tensor map for tile copies: boxes of box_rows x 64 columns, 128-byte swizzle
 int encode_row_tiles(TensorMap* out, void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // the lists over the frames (cells in depth order, waves, operand-row destinations); TC path: part of the forward pass
+int rdf_launch_depth_groups(char* ws, const Layout& L, ExecState* S, DevCtx& c, cudaStream_t stream);
 int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* S, DevCtx& c, cudaStream_t stream);
 int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char* ws, const Layout& L, ExecState* S,
                        DevCtx& c, cudaStream_t stream);

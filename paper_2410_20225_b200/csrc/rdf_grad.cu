@@ -911,11 +911,26 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap);
     bool callees_done = false;        // the previous wave's contraction has already finished this wave's invocations
     uint4 wv = nw ? c.wave_marks[0] : make_uint4(0u, 0u, 0u, 0u);
+    // clustered gradient pass (fp32 TreeRNN, deep recursions): this kernel runs the wide call depths only, up to d_split
+    const bool clustered = !TC && !c.lstm && depth_groups(c) > 1u;
+    const uint32_t d_split = clustered ? c.ctl->d_split : 0u;
     for (uint32_t k = 0; k < nw; ++k) {
         const uint4 cur = wv;
         if (k + 1 < nw) wv = c.wave_marks[k + 1];                    // in flight during this wave
         const uint32_t f0 = min(cur.x, c.frame_cap), f1 = min(cur.y, c.frame_cap);
         if (f1 <= f0) continue;
+        if (clustered && (__ldcg(&c.frames[f0].label) >> FRAME_WAVE_SHIFT) + 1u > d_split) {
+            // The first depth of the clusters: they expect the invocations of a depth finished (gradient of the loss head
+            // added, dz in place of dh), as the contraction of the depth above leaves them; do that here where it has not.
+            if (!callees_done) {
+                const uint32_t n = f1 - f0;
+                const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
+                const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
+                const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
+                backward_frames_f32(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
+            }
+            break;
+        }
         ++wave;
         // ---- A: per-invocation work, a contiguous piece of the range per block.  (bf16 TreeRNN: only the
         //      invocations called from `result` -- further down the epilogue of B does this work for the callees;
@@ -964,6 +979,127 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         c.ctl->waves_backward = wave;
         c.ctl->cyc[3] = cyc_a; c.ctl->cyc[4] = cyc_c; c.ctl->cyc[5] = cyc_b;
     }
+}
+
+// ===========================================================================
+// fp32 TreeRNN gradient waves without a grid barrier: one thread-block cluster per group of instances
+// ===========================================================================
+// The counterpart of rdf_operator_cluster_kernel for the reverse pass.  The cells are grouped by (cluster of their
+// instance, call depth); a cluster runs the depths below the split one after the other for its own instances and
+// meets at the hardware cluster barrier only.  Per cell: [dh_l ; dh_r] = W^T dz; the blocks of a cluster split the 2H
+// output columns (their part of W stays in shared memory), a block step takes CS cells, thread = (column, slice of the
+// contraction index); the thread that adds the slices up finishes the callee of its column (adds W_s^T dlog; a cell
+// callee gets dz = dh (1 - h^2) as its row, a leaf callee adds dh to dE[tok]) -- what it needs of the callee is
+// fetched before the contraction starts.  Rows travel between the blocks through L2, ordered by the barrier.
+template <int CPC>
+__global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __grid_constant__ DevCtx c) {
+    constexpr int CS = 256 / CPC;              // cells per step = slices of the contraction index
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    // every block takes the same decision from the same words (the kernels before this one are complete)
+    if (c.ctl->forward_status != 0 || c.ctl->status != 0 || depth_groups(c) <= 1u) return;
+    const int H = c.H, K2 = 2 * c.H, C = c.n_classes;
+    const int rank = blockIdx.x % CLUSTER_CTAS, group = blockIdx.x / CLUSTER_CTAS;
+    const int j0 = rank * CPC;                                         // first of this block's output columns (of 2H)
+    float* wres = reinterpret_cast<float*>(dyn_smem);                  // [H][CPC]: W[j][j0 + jj]
+    float* zs = wres + (size_t)H * CPC;                                // [2][CS][H]: dz rows, double buffered
+    float* part = zs + (size_t)2 * CS * H;                             // [CS slices][CS cells][CPC]
+    uint4* s_rec = reinterpret_cast<uint4*>(part + (size_t)CS * CS * CPC);   // [2][CS]: {cell, left callee, right callee, -}
+    for (int q = threadIdx.x; q < H * CPC; q += blockDim.x) {
+        const int j = q / CPC, jj = q % CPC;
+        wres[q] = j0 + jj < K2 ? __ldg(&c.W[(size_t)j * K2 + j0 + jj]) : 0.f;
+    }
+    __syncthreads();
+    const uint32_t stride = bucket_stride(c, 1), top = stride - 1u;
+    const uint32_t* ends = c.height_ends + (size_t)group * stride;     // ends[d]: end of (group, depth d); ends[0]: start of the group
+    const int jj = threadIdx.x % CPC, ks = threadIdx.x / CPC;          // column; slice of the contraction (then: cell)
+    const int col = j0 + jj, cc = col < H ? col : col - H;
+    const int klen = ((H + CS - 1) / CS + 3) & ~3, k_begin = ks * klen, k_end = min(H, k_begin + klen);
+    const int pieces = CS * (H / 4);
+    auto stage = [&](int buf, uint32_t first, uint32_t n) {
+        float* dst = zs + (size_t)buf * CS * H;
+        for (int p = threadIdx.x; p < pieces; p += blockDim.x) {
+            const int r = p / (H / 4), k = (p % (H / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if ((uint32_t)r < n) {
+                const uint4 it = __ldcg(reinterpret_cast<const uint4*>(&c.cell_sorted[first + r]));   // {out, l, r, height}
+                if (it.x < c.frame_cap) v = ldcg4(c.dhp + (size_t)it.x * H + k);
+                if (k == 0) s_rec[buf * CS + r] = it;
+            }
+            *reinterpret_cast<float4*>(dst + (size_t)r * H + k) = v;
+        }
+    };
+    const uint32_t d0 = min(c.ctl->d_split, top);                     // (the grid-wide kernel ran depths 1 .. d0)
+    uint32_t begin = min(ends[d0], c.work_cap);
+    uint32_t end_next = top > d0 ? min(ends[d0 + 1], c.work_cap) : begin;
+    for (uint32_t d = d0 + 1; d <= top; ++d) {
+        const uint32_t end = end_next;
+        if (d < top) end_next = min(ends[d + 1], c.work_cap);           // in flight during this depth
+        int buf = 0;
+        if (end > begin) stage(0, begin, min((uint32_t)CS, end - begin));
+        for (uint32_t first = begin; first < end; first += CS) {
+            const uint32_t n = min((uint32_t)CS, end - first);
+            __syncthreads();                                            // rows and records of this step are in place, `part` is free
+            if (first + CS < end) stage(buf ^ 1, first + CS, min((uint32_t)CS, end - first - CS));
+            // the callee that thread (cell ks, column jj) finishes after the contraction
+            const bool fin = (uint32_t)ks < n && col < K2;
+            uint32_t child = 0, child_l = LEAF_MARK, child_tok = 0;
+            float4 dl0 = make_float4(0.f, 0.f, 0.f, 0.f), dl1 = dl0;
+            float hv = 0.f;
+            if (fin) {
+                const uint4 rec = s_rec[buf * CS + ks];
+                child = col < H ? rec.y : rec.z;
+                if (child < c.frame_cap) {
+                    child_l = c.op_l[child]; child_tok = c.op_r[child];
+                    dl0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
+                    dl1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
+                    hv = c.arena[(size_t)child * H + cc];
+                }
+            }
+            {
+                float acc[CS];
+#pragma unroll
+                for (int q = 0; q < CS; ++q) acc[q] = 0.f;
+                const float* z = zs + (size_t)buf * CS * H;
+                for (int k = k_begin; k < k_end; k += 4) {
+                    const float w0 = wres[(size_t)k * CPC + jj], w1 = wres[(size_t)(k + 1) * CPC + jj];
+                    const float w2 = wres[(size_t)(k + 2) * CPC + jj], w3 = wres[(size_t)(k + 3) * CPC + jj];
+#pragma unroll
+                    for (int q = 0; q < CS; ++q) {
+                        const float4 zv = *reinterpret_cast<const float4*>(z + (size_t)q * H + k);    // (one word for the whole warp)
+                        acc[q] = fmaf(zv.x, w0, fmaf(zv.y, w1, fmaf(zv.z, w2, fmaf(zv.w, w3, acc[q]))));
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < CS; ++q) part[((size_t)ks * CS + q) * CPC + jj] = acc[q];
+            }
+            __syncthreads();
+            if (fin && child < c.frame_cap) {
+                float t = 0.f;
+#pragma unroll
+                for (int q = 0; q < CS; ++q) t += part[((size_t)q * CS + ks) * CPC + jj];
+                const float dl[MAX_CLASSES] = {dl0.x, dl0.y, dl0.z, dl0.w, dl1.x, dl1.y, dl1.z, dl1.w};
+#pragma unroll
+                for (int k = 0; k < MAX_CLASSES; ++k)
+                    if (k < C) t = fmaf(__ldg(&c.W_s[k * H + cc]), dl[k], t);
+                if (child_l == LEAF_MARK) {
+                    if (child_tok < (uint32_t)c.V) atomicAdd(c.dE + (size_t)child_tok * c.D + cc, t);
+                } else {
+                    c.dhp[(size_t)child * H + cc] = t * (1.f - hv * hv);
+                }
+            }
+            buf ^= 1;
+        }
+        begin = end;
+        __syncthreads();
+        cluster_sync_all();                                             // the rows of depth d + 1 are complete for the whole cluster
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) c.ctl->waves_backward += top - d0;      // (after the grid-wide kernel's count)
+}
+
+inline int bwd_cluster_cols_per_block(int H) { return H <= 64 ? 16 : H <= 128 ? 32 : H <= 256 ? 64 : 128; }
+inline size_t bwd_cluster_smem_bytes(int H) {
+    const int CPC = bwd_cluster_cols_per_block(H), CS = 256 / CPC;
+    return ((size_t)H * CPC + (size_t)2 * CS * H + (size_t)CS * CS * CPC) * sizeof(float) + 2 * CS * sizeof(uint4);
 }
 
 // ------------------------------------------- parameter gradients (post pass)
@@ -1225,9 +1361,40 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
         RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<true>, dim3(S->grid), dim3(TC_THREADS), args,
                                             (size_t)L.tc_smem_bwd, stream)));
     } else {
+        // deep recursions: the cells grouped by (cluster of instances, call depth); the grid-wide kernel runs the wide depths,
+        // the clusters the narrow ones after them (both leave at once when there is nothing for them to do)
+        const bool clusters = c.n_groups > 1 && !c.lstm && H <= 512;
+        if (clusters) {
+            rc = rdf_launch_depth_groups(ws, L, S, c, stream);
+            if (rc != RDF_OK) return rc;
+        }
         CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
         RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
                                             thin_resident_bytes(c.lstm, c.H), stream)));
+        if (clusters) {
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = CLUSTER_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.gridDim = dim3(c.n_groups * CLUSTER_CTAS); cfg.blockDim = dim3(256);
+            cfg.dynamicSmemBytes = bwd_cluster_smem_bytes(H); cfg.stream = stream;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            const int smem = (int)cfg.dynamicSmemBytes;
+            switch (bwd_cluster_cols_per_block(H)) {
+                case 16:
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<16>, c))); break;
+                case 32:
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<32>, c))); break;
+                case 64:
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<64>, c))); break;
+                default:
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<128>, c))); break;
+            }
+        }
     }
     rdf_mark(S, 8, stream);
     // parameter gradients
