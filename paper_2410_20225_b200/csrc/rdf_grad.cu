@@ -991,9 +991,9 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
 // contraction index); the thread that adds the slices up finishes the callee of its column (adds W_s^T dlog; a cell
 // callee gets dz = dh (1 - h^2) as its row, a leaf callee adds dh to dE[tok]) -- what it needs of the callee is
 // fetched before the contraction starts.  Rows travel between the blocks through L2, ordered by the barrier.
-template <int CPC>
-__global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __grid_constant__ DevCtx c) {
-    constexpr int CS = 256 / CPC;              // cells per step = slices of the contraction index
+static const int BWD_CLUSTER_THREADS = 512;
+template <int CPC, int CS>                     // columns per block; cells per step = slices of the contraction index (CPC x CS threads work)
+__global__ void __launch_bounds__(BWD_CLUSTER_THREADS, 1) rdf_backward_cluster_kernel(const __grid_constant__ DevCtx c) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     // every block takes the same decision from the same words (the kernels before this one are complete)
     if (c.ctl->forward_status != 0 || c.ctl->status != 0 || depth_groups(c) <= 1u) return;
@@ -1003,7 +1003,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __gr
     float* wres = reinterpret_cast<float*>(dyn_smem);                  // [H][CPC]: W[j][j0 + jj]
     float* zs = wres + (size_t)H * CPC;                                // [2][CS][H]: dz rows, double buffered
     float* part = zs + (size_t)2 * CS * H;                             // [CS slices][CS cells][CPC]
-    uint4* s_rec = reinterpret_cast<uint4*>(part + (size_t)CS * CS * CPC);   // [2][CS]: {cell, left callee, right callee, -}
+    uint4* s_rec = reinterpret_cast<uint4*>(part + (size_t)CS * CS * CPC);   // [2][CS]: {cell, left callee, right callee, -}; then the ring
     for (int q = threadIdx.x; q < H * CPC; q += blockDim.x) {
         const int j = q / CPC, jj = q % CPC;
         wres[q] = j0 + jj < K2 ? __ldg(&c.W[(size_t)j * K2 + j0 + jj]) : 0.f;
@@ -1012,6 +1012,7 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __gr
     const uint32_t stride = bucket_stride(c, 1), top = stride - 1u;
     const uint32_t* ends = c.height_ends + (size_t)group * stride;     // ends[d]: end of (group, depth d); ends[0]: start of the group
     const int jj = threadIdx.x % CPC, ks = threadIdx.x / CPC;          // column; slice of the contraction (then: cell)
+    const bool active = ks < CS;
     const int col = j0 + jj, cc = col < H ? col : col - H;
     const int klen = ((H + CS - 1) / CS + 3) & ~3, k_begin = ks * klen, k_end = min(H, k_begin + klen);
     const int pieces = CS * (H / 4);
@@ -1029,67 +1030,101 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __gr
         }
     };
     const uint32_t d0 = min(c.ctl->d_split, top);                     // (the grid-wide kernel ran depths 1 .. d0)
+    // Only the dz rows of a depth depend on the depth above.  Everything else is known before the kernel starts and is
+    // fetched ahead, off the chain of dependent waves: the records of a depth's first CS cells two depths ahead (ring in
+    // shared memory), and what thread (cell ks, column jj) needs of its callee one depth ahead (registers).
+    uint4* s_ring = s_rec + 2 * CS;                                    // [3][CS]; .x == 0xFFFFFFFF: no cell
+    struct Callee { uint32_t child, child_l, child_tok; float4 dl0, dl1; float hv; };
+    auto callee_of = [&](const uint4& rec, bool valid) {
+        Callee q;
+        q.child = 0xFFFFFFFFu; q.child_l = LEAF_MARK; q.child_tok = 0u;
+        q.dl0 = make_float4(0.f, 0.f, 0.f, 0.f); q.dl1 = q.dl0; q.hv = 0.f;
+        const uint32_t ch = col < H ? rec.y : rec.z;
+        if (valid && col < K2 && rec.x < c.frame_cap && ch < c.frame_cap) {
+            q.child = ch;
+            q.child_l = c.op_l[ch]; q.child_tok = c.op_r[ch];
+            q.dl0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)ch * 8);
+            q.dl1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)ch * 8 + 4);
+            q.hv = c.arena[(size_t)ch * H + cc];
+        }
+        return q;
+    };
+    auto first_record = [&](uint32_t d, uint32_t t) {                 // record t of depth d, or the empty record
+        uint4 rec = make_uint4(0xFFFFFFFFu, 0u, 0u, 0u);
+        if (d <= top) {
+            const uint32_t b = min(ends[d - 1], c.work_cap), e = min(ends[d], c.work_cap);
+            if (b + t < e) rec = __ldcg(reinterpret_cast<const uint4*>(&c.cell_sorted[b + t]));
+        }
+        return rec;
+    };
+    if (threadIdx.x < CS) {
+        s_ring[((d0 + 1) % 3) * CS + threadIdx.x] = first_record(d0 + 1, threadIdx.x);
+        s_ring[((d0 + 2) % 3) * CS + threadIdx.x] = first_record(d0 + 2, threadIdx.x);
+    }
+    __syncthreads();
+    Callee ahead = callee_of(s_ring[((d0 + 1) % 3) * CS + (active ? ks : 0)], active);
     uint32_t begin = min(ends[d0], c.work_cap);
-    uint32_t end_next = top > d0 ? min(ends[d0 + 1], c.work_cap) : begin;
     for (uint32_t d = d0 + 1; d <= top; ++d) {
-        const uint32_t end = end_next;
-        if (d < top) end_next = min(ends[d + 1], c.work_cap);           // in flight during this depth
+        const uint32_t end = min(ends[d], c.work_cap);
+        uint4 rec_ahead = make_uint4(0xFFFFFFFFu, 0u, 0u, 0u);
+        if (threadIdx.x < CS) rec_ahead = first_record(d + 2, threadIdx.x);             // lands while this depth runs
         int buf = 0;
-        if (end > begin) stage(0, begin, min((uint32_t)CS, end - begin));
+        {   // first step: records from the ring, rows from the depth above
+            const uint32_t n = min((uint32_t)CS, end - begin);
+            for (int p = threadIdx.x; p < pieces; p += blockDim.x) {
+                const int r = p / (H / 4), k = (p % (H / 4)) * 4;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                const uint4 it = s_ring[(d % 3) * CS + r];
+                if ((uint32_t)r < n && it.x < c.frame_cap) v = ldcg4(c.dhp + (size_t)it.x * H + k);
+                if (k == 0) s_rec[r] = it;
+                *reinterpret_cast<float4*>(zs + (size_t)r * H + k) = v;
+            }
+        }
+        const Callee mine = ahead;
+        ahead = callee_of(s_ring[((d + 1) % 3) * CS + (active ? ks : 0)], active && d + 1 <= top);   // used one depth on
         for (uint32_t first = begin; first < end; first += CS) {
             const uint32_t n = min((uint32_t)CS, end - first);
             __syncthreads();                                            // rows and records of this step are in place, `part` is free
             if (first + CS < end) stage(buf ^ 1, first + CS, min((uint32_t)CS, end - first - CS));
             // the callee that thread (cell ks, column jj) finishes after the contraction
-            const bool fin = (uint32_t)ks < n && col < K2;
-            uint32_t child = 0, child_l = LEAF_MARK, child_tok = 0;
-            float4 dl0 = make_float4(0.f, 0.f, 0.f, 0.f), dl1 = dl0;
-            float hv = 0.f;
-            if (fin) {
-                const uint4 rec = s_rec[buf * CS + ks];
-                child = col < H ? rec.y : rec.z;
-                if (child < c.frame_cap) {
-                    child_l = c.op_l[child]; child_tok = c.op_r[child];
-                    dl0 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8);
-                    dl1 = *reinterpret_cast<const float4*>(c.dlog + (size_t)child * 8 + 4);
-                    hv = c.arena[(size_t)child * H + cc];
-                }
-            }
-            {
+            const Callee q = first == begin ? mine : callee_of(s_rec[buf * CS + (active ? ks : 0)], active && (uint32_t)ks < n);
+            const bool fin = active && (uint32_t)ks < n && q.child < c.frame_cap;
+            if (active) {
                 float acc[CS];
 #pragma unroll
-                for (int q = 0; q < CS; ++q) acc[q] = 0.f;
+                for (int qq = 0; qq < CS; ++qq) acc[qq] = 0.f;
                 const float* z = zs + (size_t)buf * CS * H;
                 for (int k = k_begin; k < k_end; k += 4) {
                     const float w0 = wres[(size_t)k * CPC + jj], w1 = wres[(size_t)(k + 1) * CPC + jj];
                     const float w2 = wres[(size_t)(k + 2) * CPC + jj], w3 = wres[(size_t)(k + 3) * CPC + jj];
 #pragma unroll
-                    for (int q = 0; q < CS; ++q) {
-                        const float4 zv = *reinterpret_cast<const float4*>(z + (size_t)q * H + k);    // (one word for the whole warp)
-                        acc[q] = fmaf(zv.x, w0, fmaf(zv.y, w1, fmaf(zv.z, w2, fmaf(zv.w, w3, acc[q]))));
+                    for (int qq = 0; qq < CS; ++qq) {
+                        const float4 zv = *reinterpret_cast<const float4*>(z + (size_t)qq * H + k);    // (one word for the whole warp)
+                        acc[qq] = fmaf(zv.x, w0, fmaf(zv.y, w1, fmaf(zv.z, w2, fmaf(zv.w, w3, acc[qq]))));
                     }
                 }
 #pragma unroll
-                for (int q = 0; q < CS; ++q) part[((size_t)ks * CS + q) * CPC + jj] = acc[q];
+                for (int qq = 0; qq < CS; ++qq) part[((size_t)ks * CS + qq) * CPC + jj] = acc[qq];
             }
             __syncthreads();
-            if (fin && child < c.frame_cap) {
+            if (fin) {
                 float t = 0.f;
 #pragma unroll
-                for (int q = 0; q < CS; ++q) t += part[((size_t)q * CS + ks) * CPC + jj];
-                const float dl[MAX_CLASSES] = {dl0.x, dl0.y, dl0.z, dl0.w, dl1.x, dl1.y, dl1.z, dl1.w};
+                for (int qq = 0; qq < CS; ++qq) t += part[((size_t)qq * CS + ks) * CPC + jj];
+                const float dl[MAX_CLASSES] = {q.dl0.x, q.dl0.y, q.dl0.z, q.dl0.w, q.dl1.x, q.dl1.y, q.dl1.z, q.dl1.w};
 #pragma unroll
                 for (int k = 0; k < MAX_CLASSES; ++k)
                     if (k < C) t = fmaf(__ldg(&c.W_s[k * H + cc]), dl[k], t);
-                if (child_l == LEAF_MARK) {
-                    if (child_tok < (uint32_t)c.V) atomicAdd(c.dE + (size_t)child_tok * c.D + cc, t);
+                if (q.child_l == LEAF_MARK) {
+                    if (q.child_tok < (uint32_t)c.V) atomicAdd(c.dE + (size_t)q.child_tok * c.D + cc, t);
                 } else {
-                    c.dhp[(size_t)child * H + cc] = t * (1.f - hv * hv);
+                    c.dhp[(size_t)q.child * H + cc] = t * (1.f - q.hv * q.hv);
                 }
             }
             buf ^= 1;
         }
         begin = end;
+        if (threadIdx.x < CS) s_ring[((d + 2) % 3) * CS + threadIdx.x] = rec_ahead;      // (slot of depth d - 1: no longer read)
         __syncthreads();
         cluster_sync_all();                                             // the rows of depth d + 1 are complete for the whole cluster
     }
@@ -1098,8 +1133,8 @@ __global__ void __launch_bounds__(256, 1) rdf_backward_cluster_kernel(const __gr
 
 inline int bwd_cluster_cols_per_block(int H) { return H <= 64 ? 16 : H <= 128 ? 32 : H <= 256 ? 64 : 128; }
 inline size_t bwd_cluster_smem_bytes(int H) {
-    const int CPC = bwd_cluster_cols_per_block(H), CS = 256 / CPC;
-    return ((size_t)H * CPC + (size_t)2 * CS * H + (size_t)CS * CS * CPC) * sizeof(float) + 2 * CS * sizeof(uint4);
+    const int CPC = bwd_cluster_cols_per_block(H), CS = CPC <= 64 ? 8 : 4;
+    return ((size_t)H * CPC + (size_t)2 * CS * H + (size_t)CS * CS * CPC) * sizeof(float) + 5 * CS * sizeof(uint4);
 }
 
 // ------------------------------------------- parameter gradients (post pass)
@@ -1376,23 +1411,23 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = CLUSTER_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-            cfg.gridDim = dim3(c.n_groups * CLUSTER_CTAS); cfg.blockDim = dim3(256);
+            cfg.gridDim = dim3(c.n_groups * CLUSTER_CTAS); cfg.blockDim = dim3(BWD_CLUSTER_THREADS);
             cfg.dynamicSmemBytes = bwd_cluster_smem_bytes(H); cfg.stream = stream;
             cfg.attrs = at; cfg.numAttrs = 1;
             const int smem = (int)cfg.dynamicSmemBytes;
             switch (bwd_cluster_cols_per_block(H)) {
                 case 16:
-                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<16>, c))); break;
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<16, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<16, 8>, c))); break;
                 case 32:
-                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<32>, c))); break;
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<32, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<32, 8>, c))); break;
                 case 64:
-                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<64>, c))); break;
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<64, 8>, c))); break;
                 default:
-                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<128>, c))); break;
+                    CUDA_OK(cudaFuncSetAttribute(rdf_backward_cluster_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                    RDF_KERNEL(S, CUDA_OK(cudaLaunchKernelEx(&cfg, rdf_backward_cluster_kernel<128, 4>, c))); break;
             }
         }
     }
