@@ -325,15 +325,21 @@ __device__ void rnn_cell_tiles(const DevCtx& c, GemmSmem& sm, uint32_t first, ui
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        for (int k0 = 0; k0 < K2; k0 += TK) {
+        // the operands of step k0 + TK are on their way (registers) while step k0 is multiplied
+        auto fetch = [&](int k0, float4& a, float4& b) {
             const int k = k0 + lk;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            a = make_float4(0.f, 0.f, 0.f, 0.f); b = a;
             if (xl && k < K2) a = k < H ? ldcg4(xl + k) : ldcg4(xr + (k - H));
             if (wrow && k < K2) b = __ldg(reinterpret_cast<const float4*>(wrow + k));
+        };
+        float4 a, b;
+        fetch(0, a, b);
+        for (int k0 = 0; k0 < K2; k0 += TK) {
             __syncthreads();
             sm.As[lk + 0][lrow] = a.x; sm.As[lk + 1][lrow] = a.y; sm.As[lk + 2][lrow] = a.z; sm.As[lk + 3][lrow] = a.w;
             sm.Bs[lk + 0][lrow] = b.x; sm.Bs[lk + 1][lrow] = b.y; sm.Bs[lk + 2][lrow] = b.z; sm.Bs[lk + 3][lrow] = b.w;
             __syncthreads();
+            if (k0 + TK < K2) fetch(k0 + TK, a, b);
             gemm_tile_step(sm, tx, ty, acc);
         }
         const int col = col0 + tx * 4;

@@ -748,15 +748,21 @@ __device__ void backward_operand_tiles(const DevCtx& c, GemmSmem& sm, uint32_t f
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        for (int k0 = 0; k0 < Kdim; k0 += TK) {
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        // the operands of step k0 + TK are on their way (registers) while step k0 is multiplied
+        auto fetch = [&](int k0, float4& a, float4& b) {
+            a = make_float4(0.f, 0.f, 0.f, 0.f); b = a;
             if (dz && k0 + ak < Kdim) a = ldcg4(dz + k0 + ak);
             if (k0 + bk < Kdim && col0 + bn < K2)
                 b = __ldg(reinterpret_cast<const float4*>(c.W + (size_t)(k0 + bk) * K2 + col0 + bn));
+        };
+        float4 a, b;
+        fetch(0, a, b);
+        for (int k0 = 0; k0 < Kdim; k0 += TK) {
             __syncthreads();
             sm.As[ak + 0][arow_l] = a.x; sm.As[ak + 1][arow_l] = a.y; sm.As[ak + 2][arow_l] = a.z; sm.As[ak + 3][arow_l] = a.w;
             *reinterpret_cast<float4*>(&sm.Bs[bk][bn]) = b;
             __syncthreads();
+            if (k0 + TK < Kdim) fetch(k0 + TK, a, b);
             gemm_tile_step(sm, tx, ty, acc);
         }
         const int col = col0 + tx * 4;
