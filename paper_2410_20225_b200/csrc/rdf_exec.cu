@@ -726,21 +726,24 @@ __global__ void __launch_bounds__(256) rdf_seed_kernel(const DevCtx c) {
 // The operator kernel: the leaves first (they wait for nothing), then the cells in waves whose operands are complete;
 // a grid barrier separates the waves.  fp32 FMA tiles: height by height (a cell reads states of smaller heights).
 // TC: bf16 operands on the tensor cores (the tile pipeline of rdf_tc.cuh), depth by depth from the deepest cells up.
-template <bool TC>
-__global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
-    __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // (the TreeRNN tiles use the first part of LstmSmem)
+// RNN32: the fp32 TreeRNN alone (no TreeLSTM code in the kernel): few enough registers for two blocks per SM, which is what
+// the FFMA tiles need to hide their shared-memory and barrier latencies.
+template <bool TC, bool RNN32 = false>
+__global__ void __launch_bounds__(TC ? TC_THREADS : 256, RNN32 ? 2 : 1) rdf_operator_kernel(const __grid_constant__ DevCtx c) {
+    __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // (the TreeRNN tiles and patches use the first part of LstmSmem)
+    const bool lstm = RNN32 ? false : c.lstm != 0;
     extern __shared__ unsigned char dyn_smem[];                      // TC: resident weight slices + operand stages
     if (c.ctl->forward_status != 0) return;                          // the scheduler failed: the lists are not to be trusted
     TcState tc;
     if constexpr (TC) {
-        if (c.lstm) tc_setup(tc, smem, dyn_smem, c.Hp / 16, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
+        if (lstm) tc_setup(tc, smem, dyn_smem, c.Hp / 16, c.Wp, 2 * c.Hp, 80, c.Wxp, c.Hp, 48);
         else tc_setup(tc, smem, dyn_smem, 4, c.Wp, 2 * c.Hp, c.Hp / 4);
         tc_setup_epilogue(c, tc, smem, false);
     }
     // fp32 TreeRNN, narrow waves: this block's 16 columns of W stay in shared memory for all waves
     const float4* wres = nullptr;
     if constexpr (!TC) {
-        if (!c.lstm && c.H <= THIN_RESIDENT_MAX_H) {
+        if (!lstm && c.H <= THIN_RESIDENT_MAX_H) {
             float4* wr = reinterpret_cast<float4*>(dyn_smem);
             const int K2 = 2 * c.H, units_n = (c.H + 15) / 16, cg0 = blockIdx.x % units_n;
             for (int q = threadIdx.x; q < (K2 / 4) * 16; q += blockDim.x) {
@@ -762,14 +765,17 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
     bool alive = true;
     if (n_leaf) {
         if constexpr (TC) {
-            if (c.lstm) tc_pipe<TC_LSTM_LEAF, TC_STAGES_LSTM_FWD>(c, tc, smem, 0, n_leaf);
+            if (lstm) tc_pipe<TC_LSTM_LEAF, TC_STAGES_LSTM_FWD>(c, tc, smem, 0, n_leaf);
             else {
                 tc_leaf_rows(c, n_leaf);
                 asm volatile("fence.proxy.async;" ::: "memory");      // the operand rows it wrote are read by tile copies after the barrier
             }
         } else {
-            if (c.lstm) lstm_forward_tiles<3>(c, smem, 0, n_leaf);
-            else rnn_leaf_rows(c, n_leaf);
+            if constexpr (RNN32) rnn_leaf_rows(c, n_leaf);
+            else {
+                if (lstm) lstm_forward_tiles<3>(c, smem, 0, n_leaf);
+                else rnn_leaf_rows(c, n_leaf);
+            }
         }
         __syncthreads();
         lap(cyc_c);
@@ -787,7 +793,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
             if (k > 0) wv = c.wave_marks[k - 1];                         // in flight during this wave
             if (cur.w <= cur.z) continue;                                // (a depth of leaves only)
             const uint32_t first = min(cur.z, c.cells_cap), nc = min(cur.w, c.cells_cap) - first;
-            if (c.lstm) tc_pipe<TC_LSTM_CELL, TC_STAGES_LSTM_FWD>(c, tc, smem, first, nc);
+            if (lstm) tc_pipe<TC_LSTM_CELL, TC_STAGES_LSTM_FWD>(c, tc, smem, first, nc);
             else tc_pipe<TC_RNN_FWD, TC_STAGES_RNN_FWD>(c, tc, smem, first, nc);
             __syncthreads();
             lap(cyc_c);
@@ -808,9 +814,16 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_operator_kernel(
                 if (end <= first) continue;                              // (no cell of this height in the group)
                 const uint32_t nc = end - first;
                 any = true;
-                if (c.lstm) lstm_forward_tiles<5>(c, smem, first, nc);
+                bool done = false;
+                if constexpr (!RNN32) {
+                    if (lstm) {
+                        lstm_forward_tiles<5>(c, smem, first, nc);
+                        done = true;
+                    }
+                }
                 // thin patches while they fit in two rounds over the grid, tiles for wide waves
-                else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
+                if (done) {
+                } else if (c.H <= 384 && ((nc + 7) / 8) * ((c.H + 15) / 16) <= 2 * gridDim.x)
                     rnn_cell_thin(c, reinterpret_cast<float*>(&smem), wres, first, nc);      // 8 x 2H + 128 floats <= 26 KB
                 else rnn_cell_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, nc);
                 __syncthreads();
@@ -1198,6 +1211,12 @@ int rdf_prepare_device(rdf_graph* g, ExecState* S) {
     CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_scheduler_kernel, 1024, 2 * LQ_CAP * sizeof(Token)));
     if (per_sm < 1) return RDF_ERR_CUDA;
     S->grid = sms;                 // one persistent block per SM
+    {   // the fp32 TreeRNN kernels: two blocks per SM where they fit
+        int a = 0;
+        CUDA_OK(cudaFuncSetAttribute(rdf_operator_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
+        CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, rdf_operator_kernel<false, true>, 256, 128 * THIN_RESIDENT_MAX_H));
+        S->rnn32_per_sm = std::max(1, std::min(2, a));
+    }
     S->device = dev;
     // the clustered fp32 operator kernel: how many clusters of CLUSTER_CTAS blocks the device holds at once
     S->n_clusters = 0;
@@ -1402,8 +1421,12 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
             S->last_clusters = c.n_groups > 1 ? c.n_groups : 0;
             if (c.n_groups > 1) RDF_KERNEL(S, rdf_height_split_kernel<<<S->grid, 256, 0, stream>>>(c, 40u * (uint32_t)c.n_groups, 0));
             // the leaves and the wide heights with the whole grid ...
-            RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
-                                                thin_resident_bytes(c.lstm, c.H), stream)));
+            if (c.lstm)
+                RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false>, dim3(S->grid), dim3(256), oargs,
+                                                    thin_resident_bytes(c.lstm, c.H), stream)));
+            else
+                RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_operator_kernel<false, true>, dim3(S->grid * S->rnn32_per_sm),
+                                                    dim3(256), oargs, thin_resident_bytes(0, c.H), stream)));
             if (c.n_groups > 1) {
                 // ... the narrow ones cluster by cluster of instances (the kernel leaves at once when the grouped table
                 // did not fit and the grid-wide kernel did all the work)

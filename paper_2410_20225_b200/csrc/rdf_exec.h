@@ -48,6 +48,7 @@ struct ExecState {
     int device = -1;
     int grid = 0;
     int last_clusters = 0;       // clusters the last call used
+    int rnn32_per_sm = 1;        // blocks per SM of the fp32 TreeRNN operator / gradient kernels
     int n_clusters = 0;          // clusters of the clustered fp32 operator kernel that fit the device at once (0: none)
     int clock_khz = 0;
     void* last_ctl = nullptr;

@@ -878,21 +878,22 @@ __device__ void backward_operand_thin(const DevCtx& c, float* zs, const float4* 
     }
 }
 
-template <bool TC>
-__global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
+template <bool TC, bool RNN32 = false>         // RNN32: the fp32 TreeRNN alone, two blocks per SM (see rdf_operator_kernel)
+__global__ void __launch_bounds__(TC ? TC_THREADS : 256, RNN32 ? 2 : 1) rdf_backward_kernel(const __grid_constant__ DevCtx c) {
+    const bool lstm = RNN32 ? false : c.lstm != 0;
     __shared__ typename std::conditional<TC, TcShared, LstmSmem>::type smem;   // fp32: tiles use the first part; thin patches stage rows in it
     extern __shared__ unsigned char dyn_smem[];                      // tensor-core path: resident W^T slice + A stages
     if (c.ctl->forward_status != 0) return;                          // the forward pass failed: nothing to differentiate
     TcState tc;
     if constexpr (TC) {
-        if (c.lstm) tc_setup(tc, smem, dyn_smem, (2 * c.Hp + TC_LSTM_BWD_NS - 1) / TC_LSTM_BWD_NS, c.WTp, 5 * c.Hp, TC_LSTM_BWD_NS, nullptr, 0, 0, 2 * c.Hp);
+        if (lstm) tc_setup(tc, smem, dyn_smem, (2 * c.Hp + TC_LSTM_BWD_NS - 1) / TC_LSTM_BWD_NS, c.WTp, 5 * c.Hp, TC_LSTM_BWD_NS, nullptr, 0, 0, 2 * c.Hp);
         else tc_setup(tc, smem, dyn_smem, 8, c.WTp, c.Hp, c.Hp / 4);
         tc_setup_epilogue(c, tc, smem, true);
     }
     // fp32 TreeRNN, narrow waves: this block's 32 columns of W stay in shared memory for all waves
     const float4* wres = nullptr;
     if constexpr (!TC) {
-        if (!c.lstm && c.H <= THIN_RESIDENT_MAX_H) {
+        if (!lstm && c.H <= THIN_RESIDENT_MAX_H) {
             float4* wr = reinterpret_cast<float4*>(dyn_smem);
             const int K2 = 2 * c.H, units_n = (K2 + 31) / 32, cg0 = blockIdx.x % units_n;
             for (int q = threadIdx.x; q < c.H * 8; q += blockDim.x) {
@@ -918,7 +919,7 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
     bool callees_done = false;        // the previous wave's contraction has already finished this wave's invocations
     uint4 wv = nw ? c.wave_marks[0] : make_uint4(0u, 0u, 0u, 0u);
     // clustered gradient pass (fp32 TreeRNN, deep recursions): this kernel runs the wide call depths only, up to d_split
-    const bool clustered = !TC && !c.lstm && depth_groups(c) > 1u;
+    const bool clustered = !TC && !lstm && depth_groups(c) > 1u;
     const uint32_t d_split = clustered ? c.ctl->d_split : 0u;
     for (uint32_t k = 0; k < nw; ++k) {
         const uint4 cur = wv;
@@ -941,13 +942,19 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         // ---- A: per-invocation work, a contiguous piece of the range per block.  (bf16 TreeRNN: only the
         //      invocations called from `result` -- further down the epilogue of B does this work for the callees;
         //      fp32 TreeRNN: not after a wave of narrow patches, which do the same.)
-        if (!(TC && !c.lstm && k > 0) && !callees_done) {
+        if (!(TC && !lstm && k > 0) && !callees_done) {
             const uint32_t n = f1 - f0;
             const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 31u) & ~31u;
             const unsigned long long c0l = (unsigned long long)f0 + (unsigned long long)blockIdx.x * per;
             const uint32_t c0 = (uint32_t)min(c0l, (unsigned long long)f1), c1 = (uint32_t)min(c0l + per, (unsigned long long)f1);
-            if (c.lstm) {
-                for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
+            bool done_a = false;
+            if constexpr (!RNN32) {
+                if (lstm) {
+                    for (uint32_t t = c0 + wib; t < c1; t += n_warps) lstm_backward_frame(c, t, lane);
+                    done_a = true;
+                }
+            }
+            if (done_a) {
             } else if constexpr (TC) {
                 backward_frames_tc(c, c0 + wib * 4 + lane / 8, c1, 4 * n_warps, lane % 8);
                 asm volatile("fence.proxy.async;" ::: "memory");       // its dz rows are read by tile copies after the barrier
@@ -964,10 +971,10 @@ __global__ void __launch_bounds__(TC ? TC_THREADS : 256, 1) rdf_backward_kernel(
         bool thin = false;
         if (end > first) {
             if constexpr (TC) {
-                if (c.lstm) tc_pipe<TC_LSTM_BWD, TC_STAGES_LSTM_BWD>(c, tc, smem, first, end - first);
+                if (lstm) tc_pipe<TC_LSTM_BWD, TC_STAGES_LSTM_BWD>(c, tc, smem, first, end - first);
                 else tc_pipe<TC_RNN_BWD, TC_STAGES_RNN_BWD>(c, tc, smem, first, end - first);
             } else {
-                if (c.lstm) backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.gates, c.G, 5 * c.H);
+                if (lstm) backward_operand_tiles(c, *reinterpret_cast<GemmSmem*>(&smem), first, end - first, c.gates, c.G, 5 * c.H);
                 else if (c.H <= 512 && ((end - first + 7) / 8) * ((2 * c.H + 31) / 32) <= 2 * gridDim.x) {
                     backward_operand_thin(c, reinterpret_cast<float*>(&smem), wres, first, end - first);   // 8 x H + 800 floats <= 26 KB
                     thin = true;
@@ -1409,9 +1416,19 @@ extern "C" int rdf_grad(rdf_graph* g, const rdf_batch* in, const rdf_params* par
             rc = rdf_launch_depth_groups(ws, L, S, c, stream);
             if (rc != RDF_OK) return rc;
         }
-        CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
-        RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
-                                            thin_resident_bytes(c.lstm, c.H), stream)));
+        if (c.lstm) {
+            CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
+            RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false>, dim3(S->grid), dim3(256), args,
+                                                thin_resident_bytes(c.lstm, c.H), stream)));
+        } else {
+            // fp32 TreeRNN: as many blocks per SM as both of its persistent kernels take
+            int per_sm = 0;
+            CUDA_OK(cudaFuncSetAttribute(rdf_backward_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * THIN_RESIDENT_MAX_H));
+            CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rdf_backward_kernel<false, true>, 256, 128 * THIN_RESIDENT_MAX_H));
+            per_sm = std::max(1, std::min(per_sm, S->rnn32_per_sm));
+            RDF_KERNEL(S, CUDA_OK(cudaLaunchCooperativeKernel((void*)rdf_backward_kernel<false, true>, dim3(S->grid * per_sm), dim3(256), args,
+                                                thin_resident_bytes(0, c.H), stream)));
+        }
         if (clusters) {
             cudaLaunchConfig_t cfg = {};
             cudaLaunchAttribute at[1];
