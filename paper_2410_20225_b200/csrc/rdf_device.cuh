@@ -323,7 +323,11 @@ static const uint32_t LQ_CAP = 1024;
 struct LocalQ {
     Token*    buf[2];        // shared memory, by wave parity
     uint32_t* count;         // shared memory, [3], by wave % 3
+    uint32_t* ctr;           // shared memory, [3]: the frame, cell and leaf counters while one block runs a stretch of narrow
+                             // waves alone (copied from the control block at its start, written back at its end): the
+                             // reservations of a token cost a shared-memory atomic instead of an L2 round trip
 };
+enum { LQ_FRAMES = 0, LQ_CELLS = 1, LQ_LEAVES = 2 };
 
 __device__ __forceinline__ void push_token(const DevCtx& c, const LocalQ* lq, uint32_t wave, uint64_t tag, int64_t datum,
                                            uint32_t pc) {
@@ -400,7 +404,7 @@ __device__ __forceinline__ void frame_init(const DevCtx& c, const LabelInfo* lab
 
 // Call_i: <t, d> -> <i:t, d>.  Returns false (status set) when the tag cannot be formed.
 __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* labels, uint64_t tag, uint32_t label,
-                                         int64_t arg, uint64_t& out, uint32_t wave) {
+                                         int64_t arg, uint64_t& out, uint32_t wave, const LocalQ* lq = nullptr) {
     if (c.tag_mode == RDF_TAGS_PATH) {
         const uint32_t depth = (uint32_t)(tag >> RDF_DEPTH_SHIFT) & 63u;
         if ((depth + 1) * (uint32_t)c.label_bits > (uint32_t)RDF_PATH_BITS) {
@@ -413,7 +417,7 @@ __device__ __forceinline__ bool tag_push(const DevCtx& c, const LabelInfo* label
         trace_rec(c, out, arg, 0, label, 0);
         return true;
     }
-    const uint32_t id = aggregated_inc(&c.ctl->frame_count.v);
+    const uint32_t id = aggregated_inc(lq ? &lq->ctr[LQ_FRAMES] : &c.ctl->frame_count.v);
     if (id >= c.frame_cap) {
         set_status(c, RDF_ERR_FRAMES_FULL);
         return false;

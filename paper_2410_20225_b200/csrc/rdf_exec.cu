@@ -49,7 +49,7 @@ __device__ __forceinline__ void fire_cell(const DevCtx& c, const LocalQ* lq, con
                                           const int64_t* regs, ThreadStats& st) {
     // (global queue: the place in the list and the queue slot of the token that carries the state on are reserved together)
     uint32_t i, slot = 0;
-    if (lq) i = aggregated_inc(&c.ctl->cell_count.v);
+    if (lq) i = aggregated_inc(&lq->ctr[LQ_CELLS]);
     else aggregated_inc2(&c.ctl->cell_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
     if (i >= c.work_cap || (!lq && slot >= c.qcap)) {
         set_status(c, RDF_ERR_QUEUE_FULL);
@@ -122,7 +122,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                     }
                     frame_init(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], id, wave);
                     nt = id;
-                } else if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt, wave)) return;
+                } else if (!tag_push(c, sp.labels, tag, (uint32_t)in.imm, r[in.a], nt, wave, lq)) return;
                 ++st.invocations;
                 if (c.tag_mode == RDF_TAGS_PATH) {
                     const uint32_t d = (uint32_t)(nt >> RDF_DEPTH_SHIFT) & 63u;
@@ -144,7 +144,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
             case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)frame_of(tag) * 2 + in.imm - 1])); break;
             case VM_ENTER: {                                        // Enter: <t, d> -> <0:t, d>
                 // a loop frame under the current tag: counter 0 in the high half of the new tag, the tag below kept whole
-                const uint32_t id = aggregated_inc(&c.ctl->frame_count.v);
+                const uint32_t id = aggregated_inc(lq ? &lq->ctr[LQ_FRAMES] : &c.ctl->frame_count.v);
                 if (id >= c.frame_cap) {
                     set_status(c, RDF_ERR_FRAMES_FULL);
                     return;
@@ -241,7 +241,7 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                     return;
                 }
                 uint32_t i, slot = 0;
-                if (lq) i = aggregated_inc(&c.ctl->leaf_count.v);
+                if (lq) i = aggregated_inc(&lq->ctr[LQ_LEAVES]);
                 else aggregated_inc2(&c.ctl->leaf_count.v, &c.ctl->qcount[(wave + 1) % 3].v, i, slot);
                 if (i >= c.work_cap || (!lq && slot >= c.qcap)) {
                     set_status(c, RDF_ERR_QUEUE_FULL);
@@ -463,12 +463,13 @@ static const uint32_t NARROW_STRETCH = 4096;   // waves block 0 runs alone befor
 // frame table, store) are hidden by the number of tokens in flight.
 __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_constant__ DevCtx c) {
     __shared__ SharedProgram sp;
-    __shared__ uint32_t lq_count[3];
+    __shared__ uint32_t lq_count[3], lq_ctr[3];
     extern __shared__ __align__(16) unsigned char lq_smem[];         // local queue of narrow stretches: 2 x LQ_CAP tokens
     LocalQ lq;
     lq.buf[0] = reinterpret_cast<Token*>(lq_smem);
     lq.buf[1] = lq.buf[0] + LQ_CAP;
     lq.count = lq_count;
+    lq.ctr = lq_ctr;
     load_program(c, sp);
     ThreadStats st;
     uint32_t generation = 0, wave = 0, widest = 0;
@@ -499,6 +500,12 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                 uint32_t m = n, k = 0;
                 bool local = false;
                 if (threadIdx.x < 3) lq_count[threadIdx.x] = 0;
+                // the other blocks are on their way to the grid barrier and reserve nothing: this block owns the counters
+                if (threadIdx.x == 0) {
+                    lq_ctr[LQ_FRAMES] = ld_volatile_u32(&c.ctl->frame_count.v);
+                    lq_ctr[LQ_CELLS] = ld_volatile_u32(&c.ctl->cell_count.v);
+                    lq_ctr[LQ_LEAVES] = ld_volatile_u32(&c.ctl->leaf_count.v);
+                }
                 __syncthreads();
                 do {
                     if (threadIdx.x == 0) lq_count[(wave + 2) % 3] = 0;
@@ -552,6 +559,9 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                     c.ctl->qcount[wave % 3].v = m;
                     c.ctl->qcount[(wave + 1) % 3].v = 0;
                     c.ctl->resume_wave = wave;
+                    c.ctl->frame_count.v = lq_ctr[LQ_FRAMES];
+                    c.ctl->cell_count.v = lq_ctr[LQ_CELLS];
+                    c.ctl->leaf_count.v = lq_ctr[LQ_LEAVES];
                 }
             }
             lap(cyc_s);
