@@ -269,6 +269,18 @@ __device__ __forceinline__ void aggregated_inc2(uint32_t* ca, uint32_t* cb, uint
     b = g.shfl(bb, 0) + g.thread_rank();
 }
 
+// The same for n consecutive places on each counter per thread (a pair of calls): the thread's places are a .. a + n - 1.
+__device__ __forceinline__ void aggregated_inc2n(uint32_t* ca, uint32_t* cb, uint32_t n, uint32_t& a, uint32_t& b) {
+    cg::coalesced_group g = cg::coalesced_threads();
+    uint32_t ba = 0, bb = 0;
+    if (g.thread_rank() == 0) {
+        ba = ca ? atomicAdd(ca, n * g.size()) : 0u;
+        bb = atomicAdd(cb, n * g.size());
+    }
+    a = g.shfl(ba, 0) + n * g.thread_rank();
+    b = g.shfl(bb, 0) + n * g.thread_rank();
+}
+
 // Grid-wide barrier with a bounded wait.  All blocks of the (cooperatively
 // launched, hence co-resident) grid call it the same number of times.  The
 // counter only grows; generation k is complete when it reaches k * gridDim.x.

@@ -79,6 +79,10 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
     int pc = (int)t.pc;
     r[0] = t.datum;
     ++st.tokens;
+    int64_t node_v = -1;                          // tree accessors: the node whose words are in node_l / node_r / node_t
+    int32_t node_l = 0, node_r = 0, node_t = 0;
+    bool have_pair = false;                       // VM_CALL_A reserved a frame and a queue slot for the VM_CALL_B that follows
+    uint32_t pair_id = 0, pair_slot = 0;
     // One instruction per iteration; the bound only guards against a corrupted program.
     for (uint32_t step = 0; step < (1u << 22); ++step) {
         const VmInstr in = sp.code[pc++];
@@ -101,21 +105,42 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                     set_status(c, RDF_ERR_BAD_ARG);
                     return;
                 }
-                const int32_t* arr = in.op == VM_RIGHT ? c.right : in.op == VM_TOK ? c.tok : c.left;
-                const int32_t x = __ldg(&arr[v]);
+                // the three words of a node are fetched together the first time one of them is asked for: a body reads
+                // is_leaf, then the token or the two children of the same node, and the later reads find their word on its way
+                if (v != node_v) {
+                    node_v = v;
+                    node_l = __ldg(&c.left[v]);
+                    if (c.right) node_r = __ldg(&c.right[v]);
+                    if (c.tok) node_t = __ldg(&c.tok[v]);
+                }
+                const int32_t x = in.op == VM_RIGHT ? node_r : in.op == VM_TOK ? node_t : node_l;
                 r[in.dst] = in.op == VM_ISLEAF ? (int64_t)(x < 0) : (int64_t)x;
                 break;
             }
             case VM_BRZ: if (r[in.a] == 0) pc = in.imm; break;     // Switch: the false side
             case VM_JMP: pc = in.imm; break;
-            case VM_CALL: {                                         // Call_i
+            case VM_CALL: case VM_CALL_A: case VM_CALL_B: {         // Call_i
                 uint64_t nt;
-                // frame-form tags, global queue: the new frame's id and the token's queue slot are reserved together
-                const bool fused = c.tag_mode != RDF_TAGS_PATH && lq == nullptr;
-                uint32_t slot = 0;
+                // global queue: the new frame's id (frame-form tags) and the token's queue slot are reserved together, and
+                // for a pair of calls (VM_CALL_A .. VM_CALL_B) both calls' places at once
+                const bool frames = c.tag_mode != RDF_TAGS_PATH;
+                const bool fused = lq == nullptr && (frames || in.op != VM_CALL);
+                uint32_t slot = 0, id = 0;
                 if (fused) {
-                    uint32_t id;
-                    aggregated_inc2(&c.ctl->frame_count.v, &c.ctl->qcount[(wave + 1) % 3].v, id, slot);
+                    if (in.op == VM_CALL_B && have_pair) {
+                        id = pair_id; slot = pair_slot;
+                        have_pair = false;
+                    } else if (in.op == VM_CALL_A) {
+                        aggregated_inc2n(frames ? &c.ctl->frame_count.v : nullptr, &c.ctl->qcount[(wave + 1) % 3].v, 2u, id, slot);
+                        pair_id = id + 1u; pair_slot = slot + 1u;
+                        have_pair = true;
+                        if (frames && pair_id >= c.frame_cap) {
+                            set_status(c, RDF_ERR_FRAMES_FULL);
+                            return;
+                        }
+                    } else aggregated_inc2n(frames ? &c.ctl->frame_count.v : nullptr, &c.ctl->qcount[(wave + 1) % 3].v, 1u, id, slot);
+                }
+                if (fused && frames) {
                     if (id >= c.frame_cap) {
                         set_status(c, RDF_ERR_FRAMES_FULL);
                         return;
@@ -1372,14 +1397,26 @@ int rdf_launch_forward(rdf_graph* g, const rdf_batch* in, rdf_outputs* out, char
     {
         // the four program tables sit next to each other in the workspace (code first, constants last): one copy
         const size_t bytes = L.consts + g->consts.size() * sizeof(int64_t) - L.code;
-        if (S->tables.size() != bytes) {
-            S->tables.assign(bytes, 0);
-            memcpy(S->tables.data(), g->code.data(), g->code.size() * sizeof(VmInstr));
-            if (!g->match.empty()) memcpy(S->tables.data() + (L.match - L.code), g->match.data(), g->match.size() * sizeof(MatchNode));
-            if (!g->labels.empty()) memcpy(S->tables.data() + (L.labels - L.code), g->labels.data(), g->labels.size() * sizeof(LabelInfo));
-            if (!g->consts.empty()) memcpy(S->tables.data() + (L.consts - L.code), g->consts.data(), g->consts.size() * sizeof(int64_t));
+        if (S->tables_bytes != bytes) {
+            // page-locked, so that the copy below is asynchronous to the host (made once per graph)
+            if (S->tables) { if (S->tables_pinned) cudaFreeHost(S->tables); else free(S->tables); }
+            S->tables = nullptr; S->tables_bytes = 0;
+            if (S->may_allocate) {
+                CUDA_OK(cudaHostAlloc(reinterpret_cast<void**>(&S->tables), bytes, cudaHostAllocDefault));
+                S->tables_pinned = true;
+            } else {
+                S->tables = static_cast<char*>(malloc(bytes));
+                if (!S->tables) return RDF_ERR_CUDA;
+                S->tables_pinned = false;
+            }
+            S->tables_bytes = bytes;
+            memset(S->tables, 0, bytes);
+            memcpy(S->tables, g->code.data(), g->code.size() * sizeof(VmInstr));
+            if (!g->match.empty()) memcpy(S->tables + (L.match - L.code), g->match.data(), g->match.size() * sizeof(MatchNode));
+            if (!g->labels.empty()) memcpy(S->tables + (L.labels - L.code), g->labels.data(), g->labels.size() * sizeof(LabelInfo));
+            if (!g->consts.empty()) memcpy(S->tables + (L.consts - L.code), g->consts.data(), g->consts.size() * sizeof(int64_t));
         }
-        CUDA_OK(cudaMemcpyAsync(ws + L.code, S->tables.data(), bytes, cudaMemcpyHostToDevice, stream));
+        CUDA_OK(cudaMemcpyAsync(ws + L.code, S->tables, bytes, cudaMemcpyHostToDevice, stream));
     }
     RDF_KERNEL(S, rdf_seed_kernel<<<(unsigned)((in->B + 255) / 256), 256, 0, stream>>>(c));
     CUDA_OK(cudaGetLastError());
@@ -1508,6 +1545,7 @@ void rdf_exec_release(rdf_graph* g) {
     ExecState* S = static_cast<ExecState*>(g->dev);
     if (S && S->have_events)
         for (cudaEvent_t e : S->ev) cudaEventDestroy(e);
+    if (S && S->tables) { if (S->tables_pinned) cudaFreeHost(S->tables); else free(S->tables); }
     delete S;
     g->dev = nullptr;
 }
@@ -1694,5 +1732,8 @@ extern "C" int rdf_eval_noalloc(rdf_graph* g, const rdf_batch* in, const rdf_par
     rdf_fill_ctx(g, in, params, out, static_cast<char*>(ws), L, S, c);
     // rdf_launch_forward clears the control block, the arrival counters and the hash tables
     // on the stream before the first kernel, so nothing of the previous call is read.
-    return rdf_launch_forward(g, in, out, static_cast<char*>(ws), L, S, c, static_cast<cudaStream_t>(stream));
+    S->may_allocate = false;                       // (no allocating CUDA call on this path: the program tables stay pageable)
+    rc = rdf_launch_forward(g, in, out, static_cast<char*>(ws), L, S, c, static_cast<cudaStream_t>(stream));
+    S->may_allocate = true;
+    return rc;
 }

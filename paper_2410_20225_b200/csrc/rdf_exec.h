@@ -66,7 +66,10 @@ struct ExecState {
     int n_phases = 0;
     // the lowered program (code, match nodes, labels, constants) as one block with the workspace's own spacing, so that
     // every call copies it to the device in one piece
-    std::vector<char> tables;
+    char*  tables = nullptr;     // the program tables as they lie in the workspace, in page-locked host memory (one async copy per call)
+    size_t tables_bytes = 0;
+    bool   tables_pinned = false;
+    bool   may_allocate = true;  // false while rdf_eval_noalloc runs: the tables then stay in ordinary host memory
 };
 
 // records the boundary after phase `k - 1` (k = 0: start of the call)

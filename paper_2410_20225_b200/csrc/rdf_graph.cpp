@@ -911,6 +911,24 @@ struct Lower {
             emit(entry_seg[f], VM_HALT);
             g->max_calls_per_body = std::max(g->max_calls_per_body, calls_in_body);
         }
+        // pairs of calls: a Call_i followed in straight-line code (register moves, arithmetic, tree accessors, parameter
+        // loads) by another one -- the two calls of a binary recursion -- reserve their frames and queue slots together
+        for (Seg& S : segs)
+            for (size_t i = 0; i < S.code.size(); ++i) {
+                if (S.code[i].op != VM_CALL) continue;
+                for (size_t j = i + 1; j < S.code.size(); ++j) {
+                    const uint8_t op = S.code[j].op;
+                    if (op == VM_CALL) {
+                        S.code[i].op = VM_CALL_A;
+                        S.code[j].op = VM_CALL_B;
+                        i = j;
+                        break;
+                    }
+                    const bool pure = op == VM_MOVI || op == VM_MOVC || op == VM_MOV || (op >= VM_ADD && op <= VM_REM) ||
+                                      op == VM_ISLEAF || op == VM_LEFT || op == VM_RIGHT || op == VM_TOK || op == VM_LDARG;
+                    if (!pure) break;
+                }
+            }
         // layout: concatenate segments, make jump targets absolute
         int pc = 0;
         for (Seg& S : segs) {

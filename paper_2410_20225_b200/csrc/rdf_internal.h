@@ -25,6 +25,8 @@ enum VmOp : uint8_t {
     VM_BRZ,        // Switch: if r[a] == 0 jump to imm (segment-relative before layout, absolute after)
     VM_JMP,        // jump to imm
     VM_CALL,       // Call_i: push label imm on the tag, send <i:t, r[a]> (further parameters r[b], r[dst]) to the callee
+    VM_CALL_A,     // a Call_i that is followed in straight-line code by another one (VM_CALL_B): reserves frames and queue
+    VM_CALL_B,     //   slots for both at once (one round of atomics on the token's critical path instead of two)
     VM_LDARG,      // r[dst] = parameter imm (> 0) of this invocation, kept in its frame
     VM_PORT,       // deliver r[a] to input port b of match node imm under the current tag
     VM_RET,        // the function's output r[a]: Return_i pops the tag and continues in the caller
