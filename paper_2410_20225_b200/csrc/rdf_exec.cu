@@ -505,6 +505,10 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
         t_mark = now;
     };
     for (;; ++wave) {
+        // the thread's first token of the wave is fetched together with the wave's token count (a slot past the count
+        // holds an old token, which is dropped)
+        const uint32_t gi = blockIdx.x * blockDim.x + threadIdx.x;
+        const Token first_tok = gi < c.qcap ? load_token(&c.q[wave & 1][gi]) : Token{};
         const uint32_t n = ld_volatile_u32(&c.ctl->qcount[wave % 3].v);
         if (n == 0) break;
         if (wave >= c.wave_limit) {
@@ -535,7 +539,7 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
                 do {
                     if (threadIdx.x == 0) lq_count[(wave + 2) % 3] = 0;
                     if (threadIdx.x < m) {
-                        const Token t = local ? load_local_token(&lq.buf[wave & 1][threadIdx.x]) : load_token(&c.q[wave & 1][threadIdx.x]);
+                        const Token t = local ? load_local_token(&lq.buf[wave & 1][threadIdx.x]) : first_tok;   // (block 0: gi == threadIdx.x)
                         run_token(c, sp, &lq, wave, t, st);
                     }
                     __syncthreads();          // orders this wave's queue writes before the next wave's reads (same block)
@@ -600,8 +604,8 @@ __global__ void __launch_bounds__(1024, 1) rdf_scheduler_kernel(const __grid_con
         {
             // a wave wider than the grid: the thread's next token is on its way while it runs the current one
             const uint32_t stride = gridDim.x * blockDim.x;
-            uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-            Token next = i < n ? load_token(&q[i]) : Token{};
+            uint32_t i = gi;
+            Token next = first_tok;
             while (i < n) {
                 const Token cur = next;
                 i += stride;
