@@ -255,6 +255,7 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
     const int n_slabs = (int)((f1 - f0 + LM_ROWS - 1) / LM_ROWS);
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32, g = lane >> 2, t = lane & 3;
     const int H = c.H, Hp = c.Hp, C = c.n_classes;
+    const bool dbs_from_pad = H < Hp;
     const uint32_t rowbytes = (uint32_t)Hp * 2u, stride = rowbytes + 16u, stage_bytes = LM_ROWS * stride;
     const uint32_t mbar = smem_u32(mbars), stage0 = smem_u32(slab_smem);
     int lab_next = 0;                                  // this thread's label of the slab that was issued last
@@ -379,7 +380,9 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
                 }
             }
         }
-        if (tid < C)
+        // db_s = sum of dlog over the rows: with a pad column (H < Hp) the state rows carry the constant 1 in column H, so
+        // row H of the contraction above is that sum; otherwise it is added up here
+        if (!dbs_from_pad && tid < C)
             for (uint32_t fi = 0; fi < cnt; ++fi) my_dbs += s_dl[fi][tid];
         if (tid < LM_ROWS) s_lab[(i + 1) & 1][tid] = lab_next;      // labels of slab i + 1 (loaded while this slab was worked on)
         __syncthreads();                               // the stage, s_z and s_dl are free again
@@ -393,9 +396,10 @@ __global__ void __launch_bounds__(256) rdf_loss_heads_mma_kernel(const DevCtx c)
             for (int e = 0; e < 4; ++e) {
                 const int unit = mt * 16 + g + (e >> 1) * 8, cls = 2 * t + (e & 1);
                 if (unit < H && cls < C) atomicAdd(&c.dW_s[cls * H + unit], acc[m][e]);
+                else if (dbs_from_pad && unit == H && cls < C) atomicAdd(&c.db_s[cls], acc[m][e]);
             }
         }
-        if (tid < C) atomicAdd(&c.db_s[tid], my_dbs);
+        if (!dbs_from_pad && tid < C) atomicAdd(&c.db_s[tid], my_dbs);
     }
     // threads 0 .. 63 hold row losses: fixed-order sums inside the two warps, then over the warps
     for (int o = 16; o > 0; o >>= 1) my_loss += __shfl_down_sync(0xffffffffu, my_loss, o);
