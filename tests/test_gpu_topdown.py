@@ -111,3 +111,25 @@ def test_topdown_is_forward_fp32_only():
     want, _ = oracle_run(P, tb, D)
     h, _ = g.eval_trees(dt, dp, rdf.F32, max_invocations=4096)
     assert np.abs(h.cpu().numpy() - want).max() / np.abs(want).max() <= TOL
+
+
+def test_topdown_full_size_as_benchmarked():
+    """The workload `bench.py --workload 6` times (8192 seeds, H = 128, depth limit 10, frame table of 256 frames per
+    seed): every instance against the oracle -- the root state of each decisive instance, the number of invocations
+    of the whole batch when every instance is decisive, else of the decisive ones through the Call records."""
+    cfg = workloads.config(6)
+    tb, P, D = cfg["trees"], cfg["params"], cfg["D"]
+    want, logs = oracle_run(P, tb, D)
+    total = sum(1 + l["expand"] + l["child"] for l in logs)
+    fs, r = rdf.topdown_program(D)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    h, _ = g.eval_trees(rdf.Graph.device_trees(tb), rdf.Graph.device_params(P), rdf.F32, max_invocations=cfg["max_invocations"])
+    h = h.cpu().numpy()
+    st = g.stats()
+    decisive = np.array([l["margin"] > MARGIN for l in logs])
+    assert decisive.mean() >= 0.99, decisive.mean()
+    err = np.abs(h[decisive] - want[decisive]).max() / np.abs(want[decisive]).max()
+    assert err <= TOL, err
+    # an instance that is not decisive may have grown another tree: the totals then differ by at most its size
+    slack = sum(2 * (2 ** (D + 1)) for d in decisive if not d)
+    assert abs(st["invocations"] - total) <= slack, (st["invocations"], total, slack)
