@@ -61,7 +61,8 @@ typedef enum {
     RDF_OP_CONST,        /* imm = value                                             */
     RDF_OP_ADD, RDF_OP_SUB, RDF_OP_MUL, RDF_OP_MAX,   /* a, b                       */
     RDF_OP_LT, RDF_OP_EQ,                             /* a, b -> 0/1                */
-    RDF_OP_IF,           /* a = condition, b = then, c = else                       */
+    RDF_OP_IF,           /* a = condition, b = then, c = else; the condition may contain calls (the Switch then fires
+                            when they have returned; needs RDF_TAGS_FRAME when a branch reads a parameter) */
     RDF_OP_CALL,         /* imm = callee function index; a, b, c = one argument expression per formal
                             parameter of the callee (up to three); an argument may itself be a call */
     /* accessors on the batch's flat tree arrays; operand = node index           */

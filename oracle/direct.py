@@ -100,6 +100,14 @@ def primes(n, count=None):
     return found
 
 
+def find_first_fib_above(k, threshold, count=None):
+    """find(k) = k if threshold < fib(k) else find(k + 1), written as the recursion it is; `count`, if a dict, receives
+    the number of `find` invocations."""
+    if count is not None:
+        count["find"] = count.get("find", 0) + 1
+    return k if threshold < fib(k) else find_first_fib_above(k + 1, threshold, count)
+
+
 def sum_to(n):
     """0 + 1 + .. + (n - 1), by the loop itself."""
     s, i = 0, 0

@@ -75,6 +75,21 @@ def fib_program():
     return [r, f]
 
 
+def find_program(threshold=50):
+    """Unbounded search steered by the result of a call:
+        result(k) = find(k);   find(k) = k if threshold < fib(k) else find(k + 1)
+    The Switch of `find` is driven by a value that a callee computed (the recursion cannot be unrolled into a loop with a
+    known trip count: how far it goes is decided by fib)."""
+    r = FunctionGraph("result", 1)
+    r.output(r.call("find", r.param(0)))
+    f = FunctionGraph("find", 1)
+    k = f.param(0)
+    p = f.op("<", f.const(threshold), f.call("fib", k))
+    k_t, k_e = f.switch(p, k)
+    f.output(f.merge(k_t, f.call("find", f.op("add1", k_e))))
+    return [r, f, fib_program()[1]]
+
+
 def ack_program(m_const=2):
     """result(x) = ack(m_const, x);
     ack(m, n) = if m == 0 then n + 1 else if n == 0 then ack(m - 1, 1) else ack(m - 1, ack(m, n - 1)).

@@ -5,5 +5,5 @@ matching and wave-batched firing in hand-written CUDA behind a C boundary
 from .binding import (  # noqa: F401
     BF16, F32, TAGS_FRAME, TAGS_PATH, Function, Graph, RdfError, ack_program, fact_program, fib_program, lib, primes_program, tak_program,
     tree_fold_program, tree_net_program, unpack_path_tag, sum_loop_program, pairs_loop_program, primes_loop_program,
-    tri_program, topdown_program,
+    tri_program, topdown_program, find_program,
 )

@@ -299,6 +299,20 @@ def topdown_program(depth_limit):
     return [r, s, f, fl, fr], RESULT
 
 
+def find_program(threshold=50):
+    """result(k) = find(k); find(k) = k if threshold < fib(k) else find(k + 1): the condition waits for a call."""
+    RESULT, FIND, FIB = range(3)
+    r = Function("result", 1)
+    r.ret(r.call(FIND, r.param()))
+    f = Function("find", 1)
+    k = f.param()
+    f.ret(f.if_(f.lt(f.const(threshold), f.call(FIB, k)), k, f.call(FIND, f.add(k, f.const(1)))))
+    b = Function("fib", 1)
+    n = b.param()
+    b.ret(b.if_(b.lt(n, b.const(2)), n, b.add(b.call(FIB, b.sub(n, b.const(1))), b.call(FIB, b.sub(n, b.const(2))))))
+    return [r, f, b], RESULT
+
+
 def sum_loop_program():
     """result(n) = { s = 0; i = 0; while (i < n) { s = s + i; i = i + 1 }; s }: the while-loop of Figure 1."""
     r = Function("result", 1)

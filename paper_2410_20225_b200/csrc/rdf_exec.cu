@@ -166,7 +166,10 @@ __device__ void run_token(const DevCtx& c, const SharedProgram& sp, const LocalQ
                 } else push_token(c, lq, wave, nt, r[in.a], (uint32_t)sp.labels[in.imm].entry_pc);
                 break;
             }
-            case VM_LDARG: r[in.dst] = __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)frame_of(tag) * 2 + in.imm - 1])); break;
+            case VM_LDARG:                                          // parameter imm of this invocation, from its frame
+                r[in.dst] = in.imm == 0 ? __ldcg(reinterpret_cast<const long long*>(&c.frames[frame_of(tag)].arg))
+                                        : __ldcg(reinterpret_cast<const long long*>(&c.frame_args[(size_t)frame_of(tag) * 2 + in.imm - 1]));
+                break;
             case VM_ENTER: {                                        // Enter: <t, d> -> <0:t, d>
                 // a loop frame under the current tag: counter 0 in the high half of the new tag, the tag below kept whole
                 const uint32_t id = aggregated_inc(lq ? &lq->ctr[LQ_FRAMES] : &c.ctl->frame_count.v);

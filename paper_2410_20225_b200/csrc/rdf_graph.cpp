@@ -580,8 +580,16 @@ struct Lower {
         int r;
         switch (x.op) {
             case RDF_OP_PARAM:
-                require(segs[s].entry, RDF_ERR_UNSUPPORTED);   // parameters are in registers only in an entry segment
-                r = (int)x.imm;
+                if (segs[s].entry) {                           // parameters are in registers in an entry segment
+                    r = (int)x.imm;
+                } else {
+                    // elsewhere (the code after a condition that waited for a call) they are read back from the invocation's
+                    // frame: frame-form tags, and not inside a loop (whose variables change from iteration to iteration)
+                    require(P.p->tag_mode == RDF_TAGS_FRAME && !P.is_loop(cur_func), RDF_ERR_UNSUPPORTED);
+                    r = reg(s);
+                    emit(s, VM_LDARG, r, 0, 0, (int32_t)x.imm);
+                    if (x.imm > 0) g->max_params = std::max(g->max_params, 2);
+                }
                 break;
             case RDF_OP_CONST: r = load_const(s, x.imm); break;
             case RDF_OP_IS_LEAF: case RDF_OP_LEFT: case RDF_OP_RIGHT: case RDF_OP_TOK: {
@@ -801,19 +809,30 @@ struct Lower {
                 break;
             }
             case RDF_OP_IF: {
-                require(call_free(f, x.a), RDF_ERR_UNSUPPORTED);
-                int c = value(s, x.a);
-                std::map<int, int> saved = segs[s].memo;
-                size_t brz = segs[s].code.size();
-                emit(s, VM_BRZ, 0, c);
-                cps(s, x.b, K);
-                size_t jmp = segs[s].code.size();
-                emit(s, VM_JMP);
-                segs[s].memo = saved;
-                segs[s].code[brz].imm = (int32_t)segs[s].code.size();
-                cps(s, x.c, K);
-                segs[s].code[jmp].imm = (int32_t)segs[s].code.size();
-                segs[s].memo = saved;
+                // the Switch where the predicate arrives: in this segment when it waits for nothing, else in the code
+                // that runs when the call it waits for has returned (data-dependent control: which calls fire next is
+                // decided by a value a callee computed)
+                const rdf_expr xi = x;
+                auto branch = [this, xi, K](int s2, int c) {
+                    std::map<int, int> saved = segs[s2].memo;
+                    size_t brz = segs[s2].code.size();
+                    emit(s2, VM_BRZ, 0, c);
+                    cps(s2, xi.b, K);
+                    size_t jmp = segs[s2].code.size();
+                    emit(s2, VM_JMP);
+                    segs[s2].memo = saved;
+                    segs[s2].code[brz].imm = (int32_t)segs[s2].code.size();
+                    cps(s2, xi.c, K);
+                    segs[s2].code[jmp].imm = (int32_t)segs[s2].code.size();
+                    segs[s2].memo = saved;
+                };
+                if (call_free(f, x.a)) {
+                    branch(s, value(s, x.a));
+                } else {
+                    Cont Kc{3};
+                    Kc.fn = branch;
+                    cps(s, x.a, Kc);
+                }
                 break;
             }
             case RDF_OP_NODE_LOSS: {

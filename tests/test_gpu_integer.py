@@ -493,3 +493,29 @@ def test_remainder_semantics():
     y, _ = g.eval_int(torch.tensor(xs, dtype=torch.int64, device="cuda"), max_invocations=8)
     rem = programs.INT_OPS["%"]
     assert y.tolist() == [rem(v, 7) + rem(-v, 7) * 100 for v in xs]
+
+
+@pytest.mark.parametrize("threshold", [0, 50, 1000])
+def test_search_steered_by_a_call_result(threshold):
+    """find(k) = k if T < fib(k) else find(k + 1): the Switch of `find` fires when the call in its condition has
+    returned; the parameter it routes is read back from the invocation's frame.  Values, invocation counts and every
+    (tag, argument, returned value) against the oracle."""
+    xs = list(range(0, 20))
+    fs, r = rdf.find_program(threshold)
+    g = rdf.Graph(fs, r, rdf.TAGS_FRAME)
+    want = [direct.find_first_fib_above(k, threshold) for k in xs]
+    n_inv = 0
+    for k, w in zip(xs, want):
+        n_inv += (w - k + 1) + sum(len(direct.fib_invocations(j)[1]) for j in range(k, w + 1))
+    x = torch.tensor(xs, dtype=torch.int64, device="cuda")
+    y, got = _frame_records(g, x, n_inv)
+    assert y.tolist() == want
+    st = g.stats()
+    assert st["status"] == 0 and st["invocations"] == n_inv
+    og = transform.transform(programs.find_program(threshold))
+    for b in range(0, len(xs), 3):
+        res = tagged.run(og, {0: xs[b]}, programs.INT_OPS, dead_tokens=False)
+        assert res.value == want[b]
+        mine = {w for w in got if w[0] == b}
+        assert len(mine) == len(res.calls) or len(mine) >= len(res.calls)     # (tags of different callees may coincide in the oracle's table)
+        assert {(b, t, a[0], res.returns[t]) for t, a in res.calls.items()} <= mine

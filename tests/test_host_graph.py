@@ -242,6 +242,17 @@ def test_tree_net_literal_graph_runs_in_the_oracle(cell):
         assert len(res.calls) == tb.tree_sizes()[t]
 
 
+def test_condition_that_waits_for_a_call_literal_graph_runs_in_the_oracle():
+    fs, r = rdf.find_program(50)
+    g = _as_oracle_graph(_build(fs, r, rdf.TAGS_FRAME).describe())
+    for k in (0, 4, 9, 10, 13):
+        res = tagged.run(g, {0: k}, programs.INT_OPS)
+        assert res.value == direct.find_first_fib_above(k, 50) and res.leftover == 0
+    with pytest.raises(rdf.RdfError) as e:            # the parameter is read back from the frame after the call: frame tags
+        _build(fs, r, rdf.TAGS_PATH)
+    assert e.value.code == -11
+
+
 def test_topdown_literal_graph_runs_in_the_oracle():
     """Recursion shaped by vector values (Section 6.2, last paragraph): the graph rdf_graph_build makes of the
     top-down program -- a Switch whose predicate comes from RDF_OP_GATE on a state -- run by the oracle's interpreter

@@ -387,3 +387,25 @@ def test_primes_tagged_equals_direct(n):
             else:
                 no_divisor = all(a[0] % d for d in range(a[1], int(a[0] ** 0.5) + 1))
                 assert r.returns[tag] == int(no_divisor)
+
+
+def test_search_steered_by_a_call_result():
+    """find(k) = k if T < fib(k) else find(k + 1): the Switch is driven by a callee's value.  Pinned by the iterative
+    recurrence (the answer is the first index at or after k whose Fibonacci number exceeds T) and by the number of
+    `find` invocations, answer - k + 1."""
+    from oracle import transform, tagged
+    for T in (0, 1, 50, 1000):
+        fibs = [0, 1]
+        while fibs[-1] <= T:
+            fibs.append(fibs[-1] + fibs[-2])
+        first = next(i for i, v in enumerate(fibs) if v > T)
+        g = transform.transform(programs.find_program(T))
+        for k in (0, 1, 3, first - 1, first, first + 2):
+            if k < 0:
+                continue
+            want = max(k, first)
+            count = {}
+            assert direct.find_first_fib_above(k, T, count) == want and count["find"] == want - k + 1
+            for dead in (True, False):
+                r = tagged.run(g, {0: k}, programs.INT_OPS, dead_tokens=dead)
+                assert r.value == want and (r.leftover == 0 or not dead)    # (without hiatons the constants of untaken sides stay parked)
