@@ -189,6 +189,9 @@ struct DevCtx {
                                   // of the column sums), added up in block order
     long long* dE_fix;            // [V, D] the embedding gradient in 64-bit fixed point (integer sums are exact)
     long long* head_fix;          // [n_classes * (H + 1) + 1] dW_s, db_s and the loss in fixed point
+    uint2*    node_info;          // [N] reproducible mode: per tree node {list position + 1, depth + 1} of the cell (leaf) it carries
+    uint32_t* canon_hist;         // [canon_cap + 1] entries per (segment of nodes, depth); the last word flags the fallback
+    uint32_t  canon_cap;
     uint32_t* rank_tmp;           // [frame_cap] scratch of the pass that puts the cells of a depth in argument order
     float    *dE, *dW, *db, *dW_x, *db_x, *dW_s, *db_s;
     float*    loss_out;

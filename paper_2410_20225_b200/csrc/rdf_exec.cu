@@ -1219,6 +1219,9 @@ int rdf_make_layout(const rdf_graph* g, const rdf_batch* in, const rdf_params* p
     L.de_fix = P.take<long long>(L.repro ? (size_t)params->V * params->D : 0);
     L.head_fix = P.take<long long>(L.repro ? (size_t)params->n_classes * (H + 1) + 1 : 0);
     L.rank_tmp = P.take<uint32_t>(L.repro ? (size_t)2 * L.frame_cap : 0);      // 64-bit keys of the cells or of the leaves
+    L.canon_cap = L.repro ? (uint32_t)std::min<unsigned long long>(std::max<unsigned long long>(1ull << 20, 8ull * L.frame_cap), 1ull << 28) : 0;
+    L.node_info = P.take<uint2>(L.repro ? (size_t)std::max<long long>(in->N, 1) : 0);
+    L.canon_hist = P.take<uint32_t>(L.repro ? (size_t)L.canon_cap + 1 : 0);
     L.total = (P.off + 255) & ~(size_t)255;
     return RDF_OK;
 }
@@ -1359,6 +1362,9 @@ void rdf_fill_ctx(rdf_graph* g, const rdf_batch* in, const rdf_params* params, r
     c.dE_fix = L.repro ? reinterpret_cast<long long*>(ws + L.de_fix) : nullptr;
     c.head_fix = L.repro ? reinterpret_cast<long long*>(ws + L.head_fix) : nullptr;
     c.rank_tmp = L.repro ? reinterpret_cast<uint32_t*>(ws + L.rank_tmp) : nullptr;
+    c.node_info = L.repro ? reinterpret_cast<uint2*>(ws + L.node_info) : nullptr;
+    c.canon_hist = L.repro ? reinterpret_cast<uint32_t*>(ws + L.canon_hist) : nullptr;
+    c.canon_cap = L.canon_cap;
     c.loss_out = out->loss;
     c.ctl = reinterpret_cast<Control*>(ws + L.ctl);
     c.wave_limit = L.wave_cap ? L.wave_cap : 1u << 24;
@@ -1525,6 +1531,14 @@ int rdf_launch_lists(const rdf_batch* in, char* ws, const Layout& L, ExecState* 
     RDF_KERNEL(S, rdf_wave_compact_kernel<<<1, 1024, 0, stream>>>(c));
     if (c.repro) {                                  // the cells of every depth in argument order
         for (int leaves = c.lstm ? 1 : 0; leaves >= 0; --leaves) {     // (the leaves first: the cells' positions are used afterwards)
+            // linear-time ranks over the node indices; the quadratic kernel takes over when they do not apply
+            CUDA_OK(cudaMemsetAsync(c.node_info, 0, (size_t)std::max<long long>(in->N, 1) * sizeof(uint2), stream));
+            CUDA_OK(cudaMemsetAsync(c.canon_hist, 0, ((size_t)c.canon_cap + 1) * sizeof(uint32_t), stream));
+            const int seg_blocks = (int)std::min<long long>((in->N / CANON_SEG + 1 + 7) / 8, 8 * S->grid);
+            RDF_KERNEL(S, rdf_canon_node_kernel<<<2 * S->grid, 256, 0, stream>>>(c, leaves));
+            RDF_KERNEL(S, rdf_canon_sweep_kernel<<<seg_blocks, 256, 0, stream>>>(c, leaves, 0));
+            RDF_KERNEL(S, rdf_canon_colscan_kernel<<<16, 256, 0, stream>>>(c));
+            RDF_KERNEL(S, rdf_canon_sweep_kernel<<<seg_blocks, 256, 0, stream>>>(c, leaves, 1));
             RDF_KERNEL(S, rdf_canon_keys_kernel<<<2 * S->grid, 256, 0, stream>>>(c, leaves));
             RDF_KERNEL(S, rdf_canon_rank_kernel<<<4 * S->grid, 256, 0, stream>>>(c, leaves));
             RDF_KERNEL(S, rdf_canon_scatter_kernel<<<2 * S->grid, 256, 0, stream>>>(c, leaves));

@@ -82,8 +82,8 @@ inline void rdf_mark(ExecState* S, int k, cudaStream_t stream) {
 
 struct Layout {
     size_t ctl, code, match, labels, consts, q0, q1, frames, frame_args, frame_ptag, finst, pair_slots, port_val, arrived, table, cell_items,
-        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, dw_partial, de_fix, head_fix, rank_tmp, total;
-    uint32_t qcap, frame_cap, work_cap, wave_cap, cells_cap;
+        leaf_items, cell_sorted, height_ends, op_l, op_r, arena, gates, arena_bf, wp, wtp, dz_bf, z_bf, zdst, cell_pos, wxp, wxtp, e_bf, dg_bf, ybuf, dhp, dlog, wave_marks, list_seg, all_cells, cell_ops, leaf_ops, all_leaves, loss_partial, dw_partial, de_fix, head_fix, rank_tmp, node_info, canon_hist, total;
+    uint32_t qcap, frame_cap, work_cap, wave_cap, cells_cap, canon_cap;
     int use_tc, Hp, tc_smem_fwd, tc_smem_bwd, want_grad, repro, clustered;
     uint64_t table_cap;
     size_t arrived_bytes, table_bytes, pair_bytes;

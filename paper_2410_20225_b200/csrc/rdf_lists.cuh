@@ -204,6 +204,7 @@ __global__ void __launch_bounds__(256) rdf_canon_keys_kernel(const DevCtx c, int
 
 __global__ void __launch_bounds__(256) rdf_canon_rank_kernel(const DevCtx c, int leaves) {
     if (c.ctl->status != 0) return;
+    if (c.canon_hist && c.canon_hist[c.canon_cap] == 0u) return;          // (the linear-time pass did it)
     const long long* key = reinterpret_cast<const long long*>(c.rank_tmp);
     const uint32_t* list = leaves ? c.all_leaves : c.all_cells;
     const uint32_t n = leaves ? min(c.ctl->all_leaves, c.frame_cap) : min(c.ctl->all_cells, c.cells_cap);
@@ -228,6 +229,78 @@ __global__ void __launch_bounds__(256) rdf_canon_rank_kernel(const DevCtx c, int
             below += (k < mine) || (k == mine && q < p);
         }
         c.cell_pos[list[p]] = c0 + below;
+    }
+}
+
+// ---- the same ranks in linear time, when the arguments are distinct node indices (the tree networks)
+// A stable counting sort of the nodes, taken in index order, by the depth of the cell (leaf) they carry: node_info[a] =
+// {list position + 1, depth + 1} is scattered from the list; the nodes are cut into segments of CANON_SEG, a warp per
+// segment counts its nodes per depth, the counts are scanned down the segments per depth, and the warp walks its
+// segment again, 32 nodes at a time in index order, handing out the places.  canon_hist[canon_cap] is a flag: set when
+// an argument is no node index or occurs twice, or the table does not fit -- the quadratic kernel then does the work.
+static const uint32_t CANON_SEG = 1024;
+
+__global__ void __launch_bounds__(256) rdf_canon_node_kernel(const DevCtx c, int leaves) {
+    if (c.ctl->status != 0) return;
+    const uint32_t* list = leaves ? c.all_leaves : c.all_cells;
+    const uint32_t n = leaves ? min(c.ctl->all_leaves, c.frame_cap) : min(c.ctl->all_cells, c.cells_cap);
+    const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap), B = (uint32_t)c.B;
+    uint32_t* flag = c.canon_hist + c.canon_cap;
+    const unsigned long long n_seg = ((unsigned long long)c.N + CANON_SEG - 1) / CANON_SEG;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && n_seg * nw > c.canon_cap) *flag = 1u;
+    auto start_of = [&](uint32_t k) { const uint4 m = c.wave_marks[k]; return leaves ? m.x - B - m.z : m.z; };
+    for (uint32_t p = blockIdx.x * blockDim.x + threadIdx.x; p < n; p += gridDim.x * blockDim.x) {
+        uint32_t lo = 0, hi = nw;
+        while (hi - lo > 1) {                                  // the depth that holds position p
+            const uint32_t mid = (lo + hi) / 2;
+            if (start_of(mid) <= p) lo = mid; else hi = mid;
+        }
+        const long long a = c.frames[list[p]].arg;
+        if (a < 0 || a >= c.N) { *flag = 1u; continue; }
+        const unsigned long long rec = (unsigned long long)(p + 1u) | ((unsigned long long)(lo + 1u) << 32);
+        if (atomicExch(reinterpret_cast<unsigned long long*>(&c.node_info[a]), rec) != 0ull) *flag = 1u;
+    }
+}
+
+// pass 0: count; pass 1: place (between them rdf_canon_colscan_kernel)
+__global__ void __launch_bounds__(256) rdf_canon_sweep_kernel(const DevCtx c, int leaves, int place) {
+    if (c.ctl->status != 0 || c.canon_hist[c.canon_cap] != 0u) return;
+    const uint32_t* list = leaves ? c.all_leaves : c.all_cells;
+    const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap), B = (uint32_t)c.B, lane = threadIdx.x % 32;
+    const uint32_t n_seg = (uint32_t)(((unsigned long long)c.N + CANON_SEG - 1) / CANON_SEG);
+    for (uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) / 32; seg < n_seg; seg += gridDim.x * blockDim.x / 32) {
+        uint32_t* hist = c.canon_hist + (size_t)seg * nw;
+        for (uint32_t j = 0; j < CANON_SEG; j += 32) {
+            const long long a = (long long)seg * CANON_SEG + j + lane;
+            const uint2 info = a < c.N ? c.node_info[a] : make_uint2(0u, 0u);
+            const uint32_t k1 = info.y;                                    // depth + 1, 0: no entry of this list
+            const unsigned peers = __match_any_sync(0xffffffffu, k1);
+            if (k1 == 0u) continue;
+            const uint32_t leader = __ffs(peers) - 1, cnt = __popc(peers);
+            uint32_t base = 0;
+            if (lane == leader) base = atomicAdd(&hist[k1 - 1], cnt);     // (pass 1: the places before this chunk)
+            if (place) {
+                base = __shfl_sync(peers, base, leader);
+                const uint4 m = c.wave_marks[k1 - 1];
+                const uint32_t c0 = leaves ? m.x - B - m.z : m.z;
+                c.cell_pos[list[info.x - 1]] = c0 + base + __popc(peers & ((1u << lane) - 1u));
+            }
+        }
+    }
+}
+
+// per depth, the counts of the segments become the number of entries in the segments before
+__global__ void __launch_bounds__(256) rdf_canon_colscan_kernel(const DevCtx c) {
+    if (c.ctl->status != 0 || c.canon_hist[c.canon_cap] != 0u) return;
+    const uint32_t nw = min(c.ctl->n_depth_waves, c.wave_cap);
+    const uint32_t n_seg = (uint32_t)(((unsigned long long)c.N + CANON_SEG - 1) / CANON_SEG);
+    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < nw; k += gridDim.x * blockDim.x) {
+        uint32_t run = 0;
+        for (uint32_t seg = 0; seg < n_seg; ++seg) {
+            const uint32_t t = c.canon_hist[(size_t)seg * nw + k];
+            c.canon_hist[(size_t)seg * nw + k] = run;
+            run += t;
+        }
     }
 }
 
